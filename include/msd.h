@@ -1,0 +1,151 @@
+/*
+ * msd.h - C ABI of the B200 (sm_100a) hot path of Multi-Scale Dequant (MSD).
+ *
+ * MSD keeps quantized weights / KV in their low-precision format and instead splits each BF16
+ * activation row (or query / softmax-probability tile) at run time into two low-precision components
+ * with their own scales; both components are multiplied against the quantized operand on the tensor
+ * cores and the partial products are combined with the scales in the epilogue.
+ *
+ * General rules for every call
+ *  - All pointers are DEVICE pointers unless the argument name ends in `_host`.  The caller owns every
+ *    buffer; the library allocates nothing on these paths and never synchronises the stream.
+ *  - `stream` is a cudaStream_t (NULL = default stream).  Work is enqueued asynchronously.
+ *  - BF16 tensors are raw 16-bit patterns; row-major, innermost dimension contiguous.
+ *  - Host-detectable problems (null pointer, bad shape, misalignment, short workspace) return an error
+ *    code BEFORE any launch.  A failed launch returns MSD_ERR_CUDA.  Device-side waits are bounded: a
+ *    kernel that gives up records MSD_ERR_TIMEOUT in a device status word and exits without trapping;
+ *    msd_last_device_status() reads and clears that word.
+ *  - Non-finite activations give unspecified values but never a hang or a fault.
+ *  - Workspaces: sizes come from the *_workspace_bytes functions; a workspace must be zero-filled once
+ *    before its first use (msd_workspace_init) and is left in a reusable state by every successful call.
+ *    Two calls that share a workspace must not overlap on the GPU.
+ */
+#ifndef MSD_H_
+#define MSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MSD_OK = 0,
+  MSD_ERR_NULL_POINTER = 1,
+  MSD_ERR_BAD_SHAPE = 2,
+  MSD_ERR_BAD_ALIGNMENT = 3,
+  MSD_ERR_UNSUPPORTED = 4,
+  MSD_ERR_WORKSPACE_TOO_SMALL = 5,
+  MSD_ERR_CUDA = 6,
+  MSD_ERR_TIMEOUT = 7
+} msd_status_t;
+
+typedef enum { MSD_OUT_BF16 = 0, MSD_OUT_FP32 = 1 } msd_out_t;
+
+const char* msd_status_string(msd_status_t s);
+
+/* Reads and clears the device status word after synchronising `stream`.  Returns MSD_OK, MSD_ERR_TIMEOUT
+ * (some kernel gave up on a bounded wait; its outputs are invalid and its workspace must be re-initialised)
+ * or MSD_ERR_CUDA. */
+msd_status_t msd_last_device_status(void* stream);
+
+/* Zero-fills a workspace (asynchronous memset on `stream`). */
+msd_status_t msd_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Two-pass INT8 decomposition of BF16 rows (Sec. 3.2, Eqs. alpha, x1, residual, beta, x2; Alg. 1 lines 1-5):
+ *   alpha_i = max_k |x_ik| / 127,  q1 = clamp(rne(x/alpha), -128, 127),  r = x - alpha*q1 (one FMA, exact),
+ *   beta_i = alpha_i / 254,        q2 = clamp(rne(r/beta), -128, 127);   a zero row gives zero scales and codes.
+ * All scale arithmetic is IEEE FP32 with true division and round-half-to-even.
+ *   x_bf16 [M, ldx] (ldx >= K elements, ldx % 8 == 0), q1/q2 [M, K] INT8, alpha/beta [M] FP32.
+ * K % 16 == 0; x_bf16, q1, q2 16-byte aligned.  M = 0 is a no-op.
+ */
+msd_status_t msd_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
+                                float* alpha, float* beta, void* stream);
+
+/*
+ * Two-pass MXFP4 decomposition per 32-element K block (Sec. 3.2.1, Alg. 2) on the E2M1 grid
+ * {0, .5, 1, 1.5, 2, 3, 4, 6} that block-scaled FP4 tensor cores multiply:
+ *   alpha = smallest power of two with blockmax <= 4.5*alpha (exponent kept >= -123), q1 = rne_e2m1(x/alpha),
+ *   r = x - alpha*q1 (exact), beta = alpha/16, q2 = rne_e2m1(r/beta), both saturating at +-6.
+ *   q1/q2 [M, K/2] bytes, element 2i in bits 3:0 and 2i+1 in bits 7:4 (sign in bit 3 of the nibble);
+ *   e8m0_1/e8m0_2 [M, K/32] bytes, value 2^(byte-127), row-major.
+ * K % 32 == 0; pointers 16-byte aligned; ldx % 8 == 0.
+ */
+msd_status_t msd_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
+                                 uint8_t* e8m0_1, uint8_t* e8m0_2, void* stream);
+
+/*
+ * W8A16 MSD linear layer (Alg. 1; pass fusion by stacking [X1; X2] along the rows, Sec. 3.9):
+ *   y[i,n] = w_scale[n] * (alpha_i * sum_k q1[i,k] w[n,k] + beta_i * sum_k q2[i,k] w[n,k]),
+ * the two sums exact in INT32, the combine in FP32.
+ *   x_bf16 [M,K]; w [N,K] INT8, K contiguous; w_scale [N] FP32; y [M,N] BF16 or FP32 (ytype);
+ *   acc_dbg nullable [2,M,N] INT32 (the two accumulators, for bit-exact checks).
+ * 1 <= M <= 128 (decode regime); K % 16 == 0; N % 8 == 0 when y is BF16; x, w, y 16-byte aligned.
+ * workspace: >= msd_gemm_w8a16_workspace_bytes(M,N,K) bytes, 1024-byte aligned.
+ */
+size_t msd_gemm_w8a16_workspace_bytes(int64_t M, int64_t N, int64_t K);
+msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
+                            int64_t K, void* y, msd_out_t ytype, int32_t* acc_dbg, void* workspace,
+                            size_t workspace_bytes, void* stream);
+
+/* Same computation with the activations and the result in HOST memory (pinned for asynchronous copies):
+ * copies x to the device workspace, runs msd_gemm_w8a16, copies y back; weights stay resident on the device.
+ * workspace: >= msd_gemm_w8a16_host_workspace_bytes(M,N,K). */
+size_t msd_gemm_w8a16_host_workspace_bytes(int64_t M, int64_t N, int64_t K);
+msd_status_t msd_gemm_w8a16_host(const void* x_bf16_host, const int8_t* w, const float* w_scale, int64_t M,
+                                 int64_t N, int64_t K, void* y_host, msd_out_t ytype, void* workspace,
+                                 size_t workspace_bytes, void* stream);
+
+/*
+ * Comparison path the method replaces (Sec. 3.1 first equation): weights dequantized to BF16,
+ * bf16(w_scale[n]*w[n,k]), then a BF16 x BF16 GEMM with FP32 accumulation.  Same shapes as msd_gemm_w8a16.
+ * workspace: >= msd_gemm_dequant_bf16_workspace_bytes(M,N,K) (holds the dequantized weights).
+ */
+size_t msd_gemm_dequant_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K);
+msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M,
+                                   int64_t N, int64_t K, void* y, msd_out_t ytype, void* workspace,
+                                   size_t workspace_bytes, void* stream);
+
+/*
+ * W4A16 MSD linear layer (Alg. 2 + Tab. mxfp4-compute): both MXFP4 components are multiplied against the
+ * MXFP4 weight by block-scaled FP4 MMAs accumulating in FP32,
+ *   y[i,n] = sum_blocks 2^(e1+ew) <q1,w> + 2^(e2+ew) <q2,w>.
+ *   x_bf16 [M,K]; w_fp4 [N,K/2] packed E2M1 (element 2i in bits 3:0); w_e8m0 [N,K/32]; y [M,N].
+ * K % 128 == 0, N % 8 == 0; pointers 16-byte aligned.
+ */
+size_t msd_gemm_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K);
+msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0, int64_t M, int64_t N,
+                            int64_t K, void* y, msd_out_t ytype, void* workspace, size_t workspace_bytes,
+                            void* stream);
+
+/*
+ * Decode attention over an INT8 KV cache (Sec. 4, Alg. 3; tiled form Sec. 4.3) with one scale per token per
+ * KV head, split over the context (flash-decoding) and merged with the log-sum-exp rule:
+ *   Q row decomposed two-pass INT8; S_j = (alpha_Q S1_j + beta_Q S2_j) * k_scale[j] * softmax_scale;
+ *   P = exp(S - running max); P~_j = P_j * v_scale[j] decomposed two-pass INT8 with the fixed scale
+ *   alpha_P = max(tile's v_scale)/127; O += alpha_P P1 V + beta_P P2 V; O / sum(P) at the end.
+ *   q_bf16 [B,Hq,D]; k_cache [T,Hkv,D] INT8; v_cache [T,Hkv,Dv] INT8 or NULL (V = first Dv entries of the K row);
+ *   k_scale [T,Hkv] FP32; v_scale [T,Hkv] or NULL (= k_scale); cu_seqlens [B+1] INT32 token offsets (device);
+ *   out_bf16 [B,Hq,Dv]; lse nullable [B,Hq] FP32 (natural-log sum of exp of the scaled scores).
+ * Hq % Hkv == 0; D % 16 == 0; Dv % 16 == 0; Dv <= D when v_cache is NULL.  Empty sequences give zeros.
+ */
+size_t msd_attn_decode_int8kv_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
+                                              int32_t max_seqlen);
+msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, const int8_t* v_cache,
+                                    const float* k_scale, const float* v_scale, const int32_t* cu_seqlens,
+                                    int32_t max_seqlen, int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
+                                    float softmax_scale, void* out_bf16, float* lse, void* workspace,
+                                    size_t workspace_bytes, void* stream);
+
+/* The split schedule msd_attn_decode_int8kv uses for a sequence of length L (so a checker can mirror it):
+ * writes the tile size and the number of context splits; split s covers tokens
+ * [s*L_split, min(L,(s+1)*L_split)) with L_split = ceil(ceil(L/n_splits)/tile)*tile. */
+msd_status_t msd_attn_decode_schedule(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen,
+                                      int32_t* tile, int32_t* n_splits);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MSD_H_ */

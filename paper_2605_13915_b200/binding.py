@@ -1,0 +1,224 @@
+"""Thin ctypes binding of the C ABI in ``include/msd.h``: argument marshalling only.
+
+Tensors are torch CUDA tensors (torch is used for device memory and streams); every step of the path runs in
+the library's kernels.  There is no fallback: a missing library or a non-zero status raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+MSD_OK = 0
+OUT_BF16, OUT_FP32 = 0, 1
+STATUS = {0: "MSD_OK", 1: "MSD_ERR_NULL_POINTER", 2: "MSD_ERR_BAD_SHAPE", 3: "MSD_ERR_BAD_ALIGNMENT",
+          4: "MSD_ERR_UNSUPPORTED", 5: "MSD_ERR_WORKSPACE_TOO_SMALL", 6: "MSD_ERR_CUDA", 7: "MSD_ERR_TIMEOUT"}
+
+
+class MsdError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {STATUS.get(code, code)} ({lib().msd_status_string(code).decode()})")
+
+
+_lib = None
+_vp, _i64, _i32, _sz, _f32 = C.c_void_p, C.c_int64, C.c_int32, C.c_size_t, C.c_float
+
+_SIGS = {
+    "msd_status_string": (C.c_char_p, [C.c_int]),
+    "msd_last_device_status": (C.c_int, [_vp]),
+    "msd_workspace_init": (C.c_int, [_vp, _sz, _vp]),
+    "msd_decompose_int8": (C.c_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp]),
+    "msd_decompose_mxfp4": (C.c_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp]),
+    "msd_gemm_w8a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "msd_gemm_w8a16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _vp, _sz, _vp]),
+    "msd_gemm_w8a16_host_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "msd_gemm_w8a16_host": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
+    "msd_gemm_dequant_bf16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "msd_gemm_dequant_bf16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
+    "msd_gemm_w4a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "msd_gemm_w4a16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
+    "msd_attn_decode_int8kv_workspace_bytes": (_sz, [_i32] * 6),
+    "msd_attn_decode_int8kv": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp,
+                                         _vp, _sz, _vp]),
+    "msd_attn_decode_schedule": (C.c_int, [_i32] * 6 + [C.POINTER(_i32), C.POINTER(_i32)]),
+}
+
+
+def lib():
+    """Loads ``libmsd.so`` (building it when the sources are newer); raises when that is impossible."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB_PATH
+        if _build.needs_build():
+            path = _build.build()
+        if not os.path.exists(path):
+            raise RuntimeError("libmsd.so is missing and could not be built; there is no fallback path")
+        h = C.CDLL(path)
+        for name, (res, args) in _SIGS.items():
+            fn = getattr(h, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = h
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(code, where):
+    if code != MSD_OK:
+        raise MsdError(code, where)
+
+
+def _need_cuda(*ts):
+    for t in ts:
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("expected contiguous CUDA tensors")
+
+
+def last_device_status():
+    _check(lib().msd_last_device_status(_stream()), "msd_last_device_status")
+
+
+def workspace(nbytes, device="cuda"):
+    """A zero-filled, 1024-byte aligned workspace of at least ``nbytes`` bytes."""
+    return torch.zeros(max(int(nbytes), 1024) + 1024, dtype=torch.uint8, device=device)
+
+
+def _ws_ptr(ws):
+    base = ws.data_ptr()
+    al = (base + 1023) // 1024 * 1024
+    return C.c_void_p(al), ws.numel() - (al - base)
+
+
+def decompose_int8(x):
+    """x [M,K] bfloat16 -> (q1, q2 int8 [M,K], alpha, beta float32 [M])."""
+    _need_cuda(x)
+    M, K = x.shape
+    q1 = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    q2 = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    a = torch.empty(M, dtype=torch.float32, device=x.device)
+    b = torch.empty(M, dtype=torch.float32, device=x.device)
+    _check(lib().msd_decompose_int8(_ptr(x), M, K, x.stride(0) if M else K, _ptr(q1), _ptr(q2), _ptr(a), _ptr(b), _stream()),
+           "msd_decompose_int8")
+    return q1, q2, a, b
+
+
+def decompose_mxfp4(x):
+    """x [M,K] bfloat16 -> (q1, q2 uint8 [M,K/2], e8m0_1, e8m0_2 uint8 [M,K/32])."""
+    _need_cuda(x)
+    M, K = x.shape
+    q1 = torch.empty((M, K // 2), dtype=torch.uint8, device=x.device)
+    q2 = torch.empty((M, K // 2), dtype=torch.uint8, device=x.device)
+    e1 = torch.empty((M, K // 32), dtype=torch.uint8, device=x.device)
+    e2 = torch.empty((M, K // 32), dtype=torch.uint8, device=x.device)
+    _check(lib().msd_decompose_mxfp4(_ptr(x), M, K, x.stride(0) if M else K, _ptr(q1), _ptr(q2), _ptr(e1), _ptr(e2), _stream()),
+           "msd_decompose_mxfp4")
+    return q1, q2, e1, e2
+
+
+def gemm_w8a16_workspace_bytes(M, N, K):
+    return int(lib().msd_gemm_w8a16_workspace_bytes(M, N, K))
+
+
+def gemm_w8a16(x, w, w_scale, out_dtype=torch.bfloat16, ws=None, want_acc=False, out=None):
+    """x [M,K] bf16, w [N,K] int8, w_scale [N] f32 -> y [M,N] (bf16 or f32); optional INT32 accumulators [2,M,N]."""
+    _need_cuda(x, w, w_scale)
+    M, K = x.shape
+    N = w.shape[0]
+    if ws is None:
+        ws = workspace(gemm_w8a16_workspace_bytes(M, N, K), x.device)
+    y = out if out is not None else torch.empty((M, N), dtype=out_dtype, device=x.device)
+    acc = torch.empty((2, M, N), dtype=torch.int32, device=x.device) if want_acc else None
+    wp, wb = _ws_ptr(ws)
+    code = lib().msd_gemm_w8a16(_ptr(x), _ptr(w), _ptr(w_scale), M, N, K, _ptr(y), OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32,
+                                _ptr(acc), wp, wb, _stream())
+    _check(code, "msd_gemm_w8a16")
+    return (y, acc) if want_acc else y
+
+
+def gemm_w8a16_host_workspace_bytes(M, N, K):
+    return int(lib().msd_gemm_w8a16_host_workspace_bytes(M, N, K))
+
+
+def gemm_w8a16_host(x_host, w, w_scale, y_host, ws):
+    """Activations and result in pinned host memory; weights resident on the device."""
+    M, K = x_host.shape
+    N = w.shape[0]
+    wp, wb = _ws_ptr(ws)
+    code = lib().msd_gemm_w8a16_host(_ptr(x_host), _ptr(w), _ptr(w_scale), M, N, K, _ptr(y_host),
+                                     OUT_BF16 if y_host.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream())
+    _check(code, "msd_gemm_w8a16_host")
+    return y_host
+
+
+def gemm_dequant_bf16_workspace_bytes(M, N, K):
+    return int(lib().msd_gemm_dequant_bf16_workspace_bytes(M, N, K))
+
+
+def gemm_dequant_bf16(x, w, w_scale, out_dtype=torch.bfloat16, ws=None):
+    _need_cuda(x, w, w_scale)
+    M, K = x.shape
+    N = w.shape[0]
+    if ws is None:
+        ws = workspace(gemm_dequant_bf16_workspace_bytes(M, N, K), x.device)
+    y = torch.empty((M, N), dtype=out_dtype, device=x.device)
+    wp, wb = _ws_ptr(ws)
+    _check(lib().msd_gemm_dequant_bf16(_ptr(x), _ptr(w), _ptr(w_scale), M, N, K, _ptr(y),
+                                       OUT_BF16 if out_dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream()),
+           "msd_gemm_dequant_bf16")
+    return y
+
+
+def gemm_w4a16_workspace_bytes(M, N, K):
+    return int(lib().msd_gemm_w4a16_workspace_bytes(M, N, K))
+
+
+def gemm_w4a16(x, w_fp4, w_e8m0, out_dtype=torch.bfloat16, ws=None, out=None):
+    _need_cuda(x, w_fp4, w_e8m0)
+    M, K = x.shape
+    N = w_fp4.shape[0]
+    if ws is None:
+        ws = workspace(gemm_w4a16_workspace_bytes(M, N, K), x.device)
+    y = out if out is not None else torch.empty((M, N), dtype=out_dtype, device=x.device)
+    wp, wb = _ws_ptr(ws)
+    _check(lib().msd_gemm_w4a16(_ptr(x), _ptr(w_fp4), _ptr(w_e8m0), M, N, K, _ptr(y),
+                                OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream()), "msd_gemm_w4a16")
+    return y
+
+
+def attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen):
+    tile, ns = _i32(0), _i32(0)
+    _check(lib().msd_attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen, C.byref(tile), C.byref(ns)), "msd_attn_decode_schedule")
+    return tile.value, ns.value
+
+
+def attn_decode_int8kv_workspace_bytes(B, Hq, Hkv, D, Dv, max_seqlen):
+    return int(lib().msd_attn_decode_int8kv_workspace_bytes(B, Hq, Hkv, D, Dv, max_seqlen))
+
+
+def attn_decode_int8kv(q, k, v, k_scale, v_scale, cu_seqlens, max_seqlen, softmax_scale, dv=None, ws=None, want_lse=False,
+                       out=None):
+    """q [B,Hq,D] bf16; k [T,Hkv,D] int8; v [T,Hkv,Dv] int8 or None; scales [T,Hkv] f32; cu_seqlens [B+1] int32."""
+    _need_cuda(q, k, v, k_scale, v_scale, cu_seqlens)
+    B, Hq, D = q.shape
+    Hkv = k.shape[1]
+    Dv = v.shape[2] if v is not None else int(dv)
+    if ws is None:
+        ws = workspace(attn_decode_int8kv_workspace_bytes(B, Hq, Hkv, D, Dv, max_seqlen), q.device)
+    o = out if out is not None else torch.empty((B, Hq, Dv), dtype=torch.bfloat16, device=q.device)
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    wp, wb = _ws_ptr(ws)
+    code = lib().msd_attn_decode_int8kv(_ptr(q), _ptr(k), _ptr(v), _ptr(k_scale), _ptr(v_scale), _ptr(cu_seqlens), max_seqlen,
+                                        B, Hq, Hkv, D, Dv, softmax_scale, _ptr(o), _ptr(lse), wp, wb, _stream())
+    _check(code, "msd_attn_decode_int8kv")
+    return (o, lse) if want_lse else o

@@ -1,0 +1,221 @@
+// Online activation decomposition kernels.
+//   INT8  (Sec. 3.2, Eqs. alpha..x2; Alg. 1 lines 1-5): one CTA per row, 128-bit BF16 loads, warp-shuffle
+//          row maximum, IEEE FP32 division + round-half-to-even, packed 128-bit INT8 stores.
+//   MXFP4 (Sec. 3.2.1, Alg. 2, on the E2M1 grid): one thread per 32-element block - the block maximum needs
+//          no cross-thread reduction and beta follows from alpha by a shift.
+#include <cuda_bf16.h>
+#include <cuda_fp4.h>
+
+#include "host_common.h"
+#include "sm100.cuh"
+
+namespace msd {
+
+constexpr int kDecThreads = 512;
+constexpr int kDecCache = 4;   // 16-element chunks a thread keeps in registers between the two passes
+
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+__device__ __forceinline__ float chunk_absmax(const uint4& a, const uint4& b) {
+  // |x| of a BF16 pair: clear both sign bits, then compare as floats
+  float m = 0.0f;
+  const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    m = fmaxf(m, fabsf(bf16lo(w[i])));
+    m = fmaxf(m, fabsf(bf16hi(w[i])));
+  }
+  return m;
+}
+
+__device__ __forceinline__ int quant_i8(float v, float scale) {
+  int q = __float2int_rn(__fdiv_rn(v, scale));     // true division, round-half-to-even
+  return max(-128, min(127, q));
+}
+
+// Two-pass quantisation of 16 values; returns the packed codes of both passes.
+__device__ __forceinline__ void chunk_quantize(const uint4& a, const uint4& b, float alpha, float beta, uint4& o1, uint4& o2) {
+  const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+  uint32_t p1[4] = {0, 0, 0, 0}, p2[4] = {0, 0, 0, 0};
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const float v = h ? bf16hi(w[i]) : bf16lo(w[i]);
+      int c1 = 0, c2 = 0;
+      if (alpha > 0.0f) {
+        c1 = quant_i8(v, alpha);                                          // Eq. x1
+        const float r = __fmaf_rn(-alpha, static_cast<float>(c1), v);     // Eq. residual, exact
+        if (beta > 0.0f) c2 = quant_i8(r, beta);                          // Eq. x2
+      }
+      const int e = 2 * i + h;
+      p1[e >> 2] |= static_cast<uint32_t>(c1 & 0xFF) << (8 * (e & 3));
+      p2[e >> 2] |= static_cast<uint32_t>(c2 & 0xFF) << (8 * (e & 3));
+    }
+  }
+  o1 = make_uint4(p1[0], p1[1], p1[2], p1[3]);
+  o2 = make_uint4(p2[0], p2[1], p2[2], p2[3]);
+}
+
+__global__ void __launch_bounds__(kDecThreads)
+decompose_int8_kernel(const uint16_t* __restrict__ x, int64_t ldx, int K, int8_t* __restrict__ q1,
+                      int8_t* __restrict__ q2, float* __restrict__ alpha_out, float* __restrict__ beta_out) {
+  pdl_launch_dependents();      // a dependent GEMM may start prefetching its weights right away
+  const int row = blockIdx.x;
+  const uint4* xr = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(row) * ldx);
+  const int nchunks = K >> 4;
+  uint4 ca[kDecCache], cb[kDecCache];
+  float m = 0.0f;
+#pragma unroll
+  for (int j = 0; j < kDecCache; ++j) {
+    const int c = threadIdx.x + j * kDecThreads;
+    if (c < nchunks) {
+      ca[j] = __ldg(xr + 2 * c);
+      cb[j] = __ldg(xr + 2 * c + 1);
+      m = fmaxf(m, chunk_absmax(ca[j], cb[j]));
+    }
+  }
+  for (int c = threadIdx.x + kDecCache * kDecThreads; c < nchunks; c += kDecThreads)
+    m = fmaxf(m, chunk_absmax(__ldg(xr + 2 * c), __ldg(xr + 2 * c + 1)));
+
+  __shared__ float warp_max[kDecThreads / 32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+  __syncthreads();
+  m = warp_max[0];
+#pragma unroll
+  for (int w = 1; w < kDecThreads / 32; ++w) m = fmaxf(m, warp_max[w]);
+
+  const float alpha = __fdiv_rn(m, 127.0f);        // Eq. alpha
+  const float beta = __fdiv_rn(alpha, 254.0f);     // Eq. beta
+  if (threadIdx.x == 0) {
+    alpha_out[row] = alpha;
+    beta_out[row] = beta;
+  }
+  uint4* o1 = reinterpret_cast<uint4*>(q1 + static_cast<int64_t>(row) * K);
+  uint4* o2 = reinterpret_cast<uint4*>(q2 + static_cast<int64_t>(row) * K);
+#pragma unroll
+  for (int j = 0; j < kDecCache; ++j) {
+    const int c = threadIdx.x + j * kDecThreads;
+    if (c < nchunks) {
+      uint4 r1, r2;
+      chunk_quantize(ca[j], cb[j], alpha, beta, r1, r2);
+      o1[c] = r1;
+      o2[c] = r2;
+    }
+  }
+  for (int c = threadIdx.x + kDecCache * kDecThreads; c < nchunks; c += kDecThreads) {
+    uint4 r1, r2;
+    chunk_quantize(__ldg(xr + 2 * c), __ldg(xr + 2 * c + 1), alpha, beta, r1, r2);
+    o1[c] = r1;
+    o2[c] = r2;
+  }
+}
+
+// ---- MXFP4 ------------------------------------------------------------------------------------------------------
+constexpr int kMxThreads = 256;
+
+// 2^e as an FP32 number for e in [-126, 127]
+__device__ __forceinline__ float pow2f(int e) { return __uint_as_float(static_cast<uint32_t>(e + 127) << 23); }
+
+__global__ void __launch_bounds__(kMxThreads)
+decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, int K, uint8_t* __restrict__ q1,
+                       uint8_t* __restrict__ q2, uint8_t* __restrict__ e1, uint8_t* __restrict__ e2) {
+  pdl_launch_dependents();
+  const int kblocks = K >> 5;
+  const int64_t nblocks = M * kblocks;
+  for (int64_t b = static_cast<int64_t>(blockIdx.x) * kMxThreads + threadIdx.x; b < nblocks;
+       b += static_cast<int64_t>(gridDim.x) * kMxThreads) {
+    const int64_t row = b / kblocks;
+    const int kb = static_cast<int>(b - row * kblocks);
+    const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx + kb * 32);
+    uint32_t w[16];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint4 t = __ldg(src + i);
+      w[4 * i] = t.x; w[4 * i + 1] = t.y; w[4 * i + 2] = t.z; w[4 * i + 3] = t.w;
+    }
+    uint32_t mbits = 0;    // maximum of |x| as BF16 bits (monotone in the value for finite inputs)
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      mbits = max(mbits, w[i] & 0x7FFFu);
+      mbits = max(mbits, (w[i] >> 16) & 0x7FFFu);
+    }
+    // alpha = smallest power of two with M_b <= 4.5 alpha: M_b = m 2^e, m in [1,2) -> exponent e - 2 + (m > 1.125)
+    const int expf = static_cast<int>(mbits >> 7);
+    int a = -123;
+    if (expf > 0) a = max(-123, (expf - 127) - 2 + (((mbits & 0x7Fu) > 0x10u) ? 1 : 0));
+    a = min(a, 127);
+    const int bexp = a - 4;                                   // beta = alpha / 16
+    // x / alpha and r / beta as two exact power-of-two multiplications (each factor stays a normal number)
+    const int na = -a, nb = -bexp;
+    const float sa1 = pow2f(na / 2), sa2 = pow2f(na - na / 2);
+    const float sb1 = pow2f(nb / 2), sb2 = pow2f(nb - nb / 2);
+    const float alpha = (a >= -126) ? pow2f(a) : 0.0f;        // a >= -123 always; kept for clarity
+    uint32_t o1[4] = {0, 0, 0, 0}, o2[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float v0 = bf16lo(w[i]), v1 = bf16hi(w[i]);
+      const __nv_fp4x2_storage_t c1 =
+          __nv_cvt_float2_to_fp4x2(make_float2((v0 * sa1) * sa2, (v1 * sa1) * sa2), __NV_E2M1, cudaRoundNearest);
+      const float2 d1 = __half22float2(__half2(__nv_cvt_fp4x2_to_halfraw2(c1, __NV_E2M1)));
+      const float r0 = __fmaf_rn(-alpha, d1.x, v0), r1 = __fmaf_rn(-alpha, d1.y, v1);   // exact residuals
+      const __nv_fp4x2_storage_t c2 =
+          __nv_cvt_float2_to_fp4x2(make_float2((r0 * sb1) * sb2, (r1 * sb1) * sb2), __NV_E2M1, cudaRoundNearest);
+      o1[i >> 2] |= static_cast<uint32_t>(c1) << (8 * (i & 3));
+      o2[i >> 2] |= static_cast<uint32_t>(c2) << (8 * (i & 3));
+    }
+    *reinterpret_cast<uint4*>(q1 + row * (K >> 1) + kb * 16) = make_uint4(o1[0], o1[1], o1[2], o1[3]);
+    *reinterpret_cast<uint4*>(q2 + row * (K >> 1) + kb * 16) = make_uint4(o2[0], o2[1], o2[2], o2[3]);
+    e1[row * kblocks + kb] = static_cast<uint8_t>(a + 127);
+    e2[row * kblocks + kb] = static_cast<uint8_t>(bexp + 127);
+  }
+}
+
+msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
+                                   float* alpha, float* beta, cudaStream_t stream) {
+  if (M == 0) return MSD_OK;
+  decompose_int8_kernel<<<static_cast<unsigned>(M), kDecThreads, 0, stream>>>(
+      static_cast<const uint16_t*>(x_bf16), ldx, static_cast<int>(K), q1, q2, alpha, beta);
+  return launch_status();
+}
+
+msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
+                                    uint8_t* e1, uint8_t* e2, cudaStream_t stream) {
+  if (M == 0) return MSD_OK;
+  const int64_t nblocks = M * (K >> 5);
+  const int64_t want = (nblocks + kMxThreads - 1) / kMxThreads;
+  const int64_t cap = static_cast<int64_t>(sm_count()) * 32;
+  const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
+  decompose_mxfp4_kernel<<<grid, kMxThreads, 0, stream>>>(static_cast<const uint16_t*>(x_bf16), ldx, M,
+                                                          static_cast<int>(K), q1, q2, e1, e2);
+  return launch_status();
+}
+
+}  // namespace msd
+
+extern "C" {
+
+msd_status_t msd_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
+                                float* alpha, float* beta, void* stream) {
+  if (M < 0 || K <= 0 || K % 16 != 0 || ldx < K || ldx % 8 != 0 || M > 0x7FFFFFFF || K > 0x7FFFFFF0) return MSD_ERR_BAD_SHAPE;
+  if (M == 0) return MSD_OK;
+  if (!x_bf16 || !q1 || !q2 || !alpha || !beta) return MSD_ERR_NULL_POINTER;
+  if (!msd::aligned(x_bf16, 16) || !msd::aligned(q1, 16) || !msd::aligned(q2, 16) || !msd::aligned(alpha, 4) ||
+      !msd::aligned(beta, 4))
+    return MSD_ERR_BAD_ALIGNMENT;
+  return msd::launch_decompose_int8(x_bf16, M, K, ldx, q1, q2, alpha, beta, static_cast<cudaStream_t>(stream));
+}
+
+msd_status_t msd_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
+                                 uint8_t* e8m0_1, uint8_t* e8m0_2, void* stream) {
+  if (M < 0 || K <= 0 || K % 32 != 0 || ldx < K || ldx % 8 != 0 || K > 0x7FFFFFE0) return MSD_ERR_BAD_SHAPE;
+  if (M == 0) return MSD_OK;
+  if (!x_bf16 || !q1 || !q2 || !e8m0_1 || !e8m0_2) return MSD_ERR_NULL_POINTER;
+  if (!msd::aligned(x_bf16, 16) || !msd::aligned(q1, 16) || !msd::aligned(q2, 16)) return MSD_ERR_BAD_ALIGNMENT;
+  return msd::launch_decompose_mxfp4(x_bf16, M, K, ldx, q1, q2, e8m0_1, e8m0_2, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

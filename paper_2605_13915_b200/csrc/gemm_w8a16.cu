@@ -1,0 +1,425 @@
+// W8A16 MSD linear layer for the decode regime (Alg. 1; Sec. 3.9 pass fusion by stacking the two components).
+//
+// Roles are swapped relative to the usual GEMM: a 128-row tile of the INT8 weight is the MMA "A" operand
+// (the M axis of tcgen05.mma), the stacked components [Q1; Q2] (NB = 2*ceil8(M) rows) are the "B" operand, so one
+// weight tile read from HBM serves both passes and the accumulator D[128 weight rows x NB] lives in TMEM.
+//
+// Work split ("stream-K"): the (weight tile, 128-byte K block) pairs are numbered tile-major and divided evenly over
+// the CTAs (one per SM), so every SM streams the same number of weight bytes.  A CTA whose range covers a whole tile
+// finishes it alone; a tile shared by several CTAs is reduced through per-CTA INT32 slots in the workspace and finished
+// by whichever CTA arrives last (integer sums: the result does not depend on the arrival order).
+//
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (+ TMEM owner), warps 2-5 = epilogue (one per TMEM lane group).
+#include <cuda_bf16.h>
+
+#include <cstdlib>
+
+#include "host_common.h"
+#include "sm100.cuh"
+
+namespace msd {
+
+constexpr int kTileN = 128;        // weight rows per tile (MMA M)
+constexpr int kBlockK = 128;       // K bytes per pipeline stage (one 128-byte swizzle row)
+constexpr int kMaxStages = 12;
+constexpr int kGemmThreads = 192;
+constexpr int kWStageBytes = kTileN * kBlockK;
+constexpr int kSmemBudget = 227 * 1024 - 4096;   // leaves room for the static barriers and the alignment pad
+
+struct GemmW8Params {
+  int M, Mp, NB, N, K;
+  int kblocks;             // K blocks per weight tile
+  int num_tiles;
+  long long total_blocks;  // num_tiles * kblocks
+  int num_stages;
+  int tmem_cols;
+  int ytype;
+  const float* w_scale;
+  const float* alpha;
+  const float* beta;
+  void* y;
+  int32_t* acc_dbg;
+  int32_t* slots;          // [gridDim.x * 2][NB][128]
+  unsigned* counters;      // [num_tiles]
+  unsigned* status;
+};
+
+__device__ __forceinline__ long long range_begin(long long cta, long long total, long long grid) { return cta * total / grid; }
+__device__ __forceinline__ long long block_owner(long long blk, long long total, long long grid) {
+  return ((blk + 1) * grid - 1) / total;
+}
+
+__device__ __forceinline__ void store_out(const GemmW8Params& p, int i, int n, float v, int32_t a, int32_t b) {
+  const long long idx = static_cast<long long>(i) * p.N + n;
+  if (p.ytype == MSD_OUT_BF16) static_cast<__nv_bfloat16*>(p.y)[idx] = __float2bfloat16_rn(v);
+  else static_cast<float*>(p.y)[idx] = v;
+  if (p.acc_dbg) {
+    p.acc_dbg[idx] = a;
+    p.acc_dbg[static_cast<long long>(p.M) * p.N + idx] = b;
+  }
+}
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
+                  const GemmW8Params p) {
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ __align__(8) uint64_t full_bar[kMaxStages];
+  __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
+  __shared__ __align__(8) uint64_t tfull_bar[2];
+  __shared__ __align__(8) uint64_t tempty_bar[2];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+  __shared__ int is_last_flag;
+  __shared__ float s_alpha[128], s_beta[128];
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+  const int x_stage_bytes = p.NB * kBlockK;
+  const int stage_bytes = kWStageBytes + x_stage_bytes;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.num_stages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&tfull_bar[a], 1);
+      mbar_init(&tempty_bar[a], 4);      // one arrival per epilogue warp
+    }
+    abort_flag = 0;
+    mbar_init_fence();
+    tma_prefetch_desc(&tmap_w);
+    tma_prefetch_desc(&tmap_x);
+  }
+  if (warp == 1) tmem_alloc(&tmem_base_slot, p.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  volatile int* abort = &abort_flag;
+
+  const long long grid = gridDim.x;
+  const long long blk_begin = range_begin(blockIdx.x, p.total_blocks, grid);
+  const long long blk_end = range_begin(blockIdx.x + 1, p.total_blocks, grid);
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      const uint64_t pol_w = policy_evict_first();    // weights are streamed once
+      const uint64_t pol_x = policy_evict_last();     // the stacked components are re-read by every CTA
+      int stage = 0;
+      uint32_t phase = 0;
+      // Weight tiles of the first stages do not depend on the decomposition kernel: issue them before waiting for it.
+      const long long nblk = blk_end - blk_begin;
+      const int pre = static_cast<int>(nblk < p.num_stages ? nblk : p.num_stages);
+      for (int i = 0; i < pre; ++i) {
+        const long long blk = blk_begin + i;
+        const int tile = static_cast<int>(blk / p.kblocks), kb = static_cast<int>(blk % p.kblocks);
+        mbar_arrive_expect_tx(&full_bar[i], stage_bytes);
+        tma_load_2d_hint(smem + i * stage_bytes, &tmap_w, kb * kBlockK, tile * kTileN, &full_bar[i], pol_w);
+      }
+      pdl_wait_primary();
+      for (int i = 0; i < pre; ++i) {
+        const int kb = static_cast<int>((blk_begin + i) % p.kblocks);
+        tma_load_2d_hint(smem + i * stage_bytes + kWStageBytes, &tmap_x, kb * kBlockK, 0, &full_bar[i], pol_x);
+      }
+      stage = pre % p.num_stages;
+      phase = (pre == p.num_stages) ? 1 : 0;
+      bool ok = true;
+      for (long long blk = blk_begin + pre; blk < blk_end && ok; ++blk) {
+        const int tile = static_cast<int>(blk / p.kblocks), kb = static_cast<int>(blk % p.kblocks);
+        ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&full_bar[stage], stage_bytes);
+        uint8_t* dst = smem + stage * stage_bytes;
+        tma_load_2d_hint(dst, &tmap_w, kb * kBlockK, tile * kTileN, &full_bar[stage], pol_w);
+        tma_load_2d_hint(dst + kWStageBytes, &tmap_x, kb * kBlockK, 0, &full_bar[stage], pol_x);
+        if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
+      }
+      if (!ok) {
+        // give copies already in flight a bounded time to land before the CTA goes away
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      const uint32_t idesc = idesc_dense(/*D=S32*/ 2, /*A=S8*/ 1, /*B=S8*/ 1, 0, 0, kTileN, p.NB);
+      int stage = 0;
+      uint32_t phase = 0;
+      int seg = 0;
+      bool ok = true;
+      long long blk = blk_begin;
+      while (blk < blk_end && ok) {
+        const int tile = static_cast<int>(blk / p.kblocks);
+        const long long tile_end = static_cast<long long>(tile + 1) * p.kblocks;
+        const long long seg_end = tile_end < blk_end ? tile_end : blk_end;
+        const int acc = seg & 1;
+        ok = wait_bounded(&tempty_bar[acc], ((seg >> 1) & 1) ^ 1, abort, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * p.NB;
+        for (long long b = blk; b < seg_end; ++b) {
+          ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t wa = smem_u32(smem + stage * stage_bytes);
+          const uint32_t xa = wa + kWStageBytes;
+#pragma unroll
+          for (int k = 0; k < kBlockK / 32; ++k) {
+            const uint64_t adesc = smem_desc(wa + k * 32, 16, 1024, kSwizzle128B);
+            const uint64_t bdesc = smem_desc(xa + k * 32, 16, 1024, kSwizzle128B);
+            mma_i8(d_tmem, adesc, bdesc, idesc, (b > blk || k > 0) ? 1u : 0u);
+          }
+          tc_commit(&empty_bar[stage]);          // frees the stage once these MMAs have read it
+          if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        tc_commit(&tfull_bar[acc]);              // accumulator of this segment complete
+        ++seg;
+        blk = seg_end;
+      }
+    }
+  } else {
+    // ------------------------------ epilogue (warps 2..5) ------------------------------
+    const int quad = warp & 3;                    // TMEM lane group this warp may read
+    const int r = quad * 32 + lane;               // weight row within the tile == TMEM lane
+    const int et = threadIdx.x - 64;              // 0..127
+    pdl_wait_primary();
+    if (et < p.M) {
+      s_alpha[et] = p.alpha[et];
+      s_beta[et] = p.beta[et];
+    }
+    named_bar_sync(1, 128);
+    int seg = 0;
+    bool ok = true;
+    long long blk = blk_begin;
+    while (blk < blk_end && ok) {
+      const int tile = static_cast<int>(blk / p.kblocks);
+      const long long tile_begin = static_cast<long long>(tile) * p.kblocks;
+      const long long tile_end = tile_begin + p.kblocks;
+      const long long seg_end = tile_end < blk_end ? tile_end : blk_end;
+      const bool complete = (blk == tile_begin) && (seg_end == tile_end);
+      const int acc = seg & 1;
+      ok = wait_bounded(&tfull_bar[acc], (seg >> 1) & 1, abort, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * p.NB;
+      const int n = tile * kTileN + r;
+      bool finish = complete;
+      int c_lo = 0, c_hi = -1;
+      if (!complete) {
+        // park this CTA's partial sums in its slot, then find out whether it is the last contributor of the tile
+        const int slot_id = 2 * blockIdx.x + ((blk_begin >= tile_begin) ? 0 : 1);
+        int32_t* slot = p.slots + static_cast<long long>(slot_id) * p.NB * kTileN;
+        for (int c0 = 0; c0 < p.NB; c0 += 8) {
+          uint32_t v[8];
+          tmem_ld8(t_row + c0, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) slot[(c0 + j) * kTileN + r] = static_cast<int32_t>(v[j]);
+        }
+        __threadfence();
+        named_bar_sync(1, 128);
+        c_lo = static_cast<int>(block_owner(tile_begin, p.total_blocks, grid));
+        c_hi = static_cast<int>(block_owner(tile_end - 1, p.total_blocks, grid));
+        if (et == 0) {
+          const unsigned prev = atomicAdd(&p.counters[tile], 1u);
+          const int last = (prev == static_cast<unsigned>(c_hi - c_lo)) ? 1 : 0;
+          if (last) p.counters[tile] = 0;          // leave the counter ready for the next call
+          is_last_flag = last;
+        }
+        named_bar_sync(1, 128);
+        finish = is_last_flag != 0;
+        if (finish) __threadfence();
+      }
+      if (finish) {
+        const float sw = (n < p.N) ? __ldg(p.w_scale + n) : 0.0f;
+        for (int c0 = 0; c0 < p.Mp; c0 += 8) {
+          uint32_t a[8], b[8];
+          tmem_ld8(t_row + c0, a);
+          tmem_ld8(t_row + p.Mp + c0, b);
+          tmem_ld_wait();
+          for (int c = c_lo; c <= c_hi; ++c) {
+            if (c == static_cast<int>(blockIdx.x)) continue;
+            const int sid = 2 * c + ((range_begin(c, p.total_blocks, grid) >= tile_begin) ? 0 : 1);
+            const int32_t* slot = p.slots + static_cast<long long>(sid) * p.NB * kTileN;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              a[j] += static_cast<uint32_t>(__ldcg(slot + (c0 + j) * kTileN + r));
+              b[j] += static_cast<uint32_t>(__ldcg(slot + (p.Mp + c0 + j) * kTileN + r));
+            }
+          }
+          if (n < p.N) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int i = c0 + j;
+              if (i < p.M) {
+                const int32_t ya = static_cast<int32_t>(a[j]), yb = static_cast<int32_t>(b[j]);
+                // y = s_W * (alpha * Y1 + beta * Y2)   (Alg. 1 line 8)
+                const float v = sw * __fmaf_rn(s_alpha[i], static_cast<float>(ya), s_beta[i] * static_cast<float>(yb));
+                store_out(p, i, n, v, ya, yb);
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+      ++seg;
+      blk = seg_end;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, p.tmem_cols);
+  }
+}
+
+static int pow2_at_least(int v) {
+  int p = 32;
+  while (p < v) p <<= 1;
+  return p;
+}
+
+struct GemmW8Plan {
+  int Mp, NB, kblocks, num_tiles, grid, stages, tmem_cols;
+  long long total_blocks;
+  size_t off_q, off_alpha, off_beta, off_counters, off_slots, bytes;
+  size_t smem_bytes;
+};
+
+static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K) {
+  GemmW8Plan pl;
+  pl.Mp = static_cast<int>((M + 7) / 8 * 8);
+  pl.NB = 2 * pl.Mp;
+  pl.kblocks = static_cast<int>((K + kBlockK - 1) / kBlockK);
+  pl.num_tiles = static_cast<int>((N + kTileN - 1) / kTileN);
+  pl.total_blocks = static_cast<long long>(pl.kblocks) * pl.num_tiles;
+  int grid = sm_count();
+  if (const char* e = getenv("MSD_GEMM_CTAS")) {
+    const int g = atoi(e);
+    if (g > 0) grid = g;
+  }
+  if (grid > pl.total_blocks) grid = static_cast<int>(pl.total_blocks);
+  if (grid < 1) grid = 1;
+  pl.grid = grid;
+  const int stage_bytes = kWStageBytes + pl.NB * kBlockK;
+  int stages = kSmemBudget / stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  pl.stages = stages;
+  pl.smem_bytes = static_cast<size_t>(stages) * stage_bytes + 1024;
+  pl.tmem_cols = pow2_at_least(2 * pl.NB);
+  size_t off = 0;
+  pl.off_q = off;         off = round_up(off + static_cast<size_t>(pl.NB) * K, 1024);
+  pl.off_alpha = off;     off = round_up(off + 128 * sizeof(float), 256);
+  pl.off_beta = off;      off = round_up(off + 128 * sizeof(float), 256);
+  pl.off_counters = off;  off = round_up(off + static_cast<size_t>(pl.num_tiles) * sizeof(unsigned), 1024);
+  // slot space sized for the largest grid the launcher may pick, so the same workspace serves any override
+  const int max_grid = sm_count() > 256 ? sm_count() : 256;
+  pl.off_slots = off;     off = round_up(off + static_cast<size_t>(max_grid) * 2 * pl.NB * kTileN * sizeof(int32_t), 1024);
+  pl.bytes = off;
+  return pl;
+}
+
+static msd_status_t check_w8_args(const void* x, const void* w, const void* ws, int64_t M, int64_t N, int64_t K,
+                                  const void* y, int ytype, const void* workspace) {
+  if (M < 1 || M > 128 || N < 1 || K < 16 || K % 16 != 0 || N > (1 << 24) || K > (1 << 24)) return MSD_ERR_BAD_SHAPE;
+  if (ytype != MSD_OUT_BF16 && ytype != MSD_OUT_FP32) return MSD_ERR_UNSUPPORTED;
+  if (ytype == MSD_OUT_BF16 && N % 8 != 0) return MSD_ERR_BAD_SHAPE;
+  if (!x || !w || !ws || !y || !workspace) return MSD_ERR_NULL_POINTER;
+  if (!aligned(x, 16) || !aligned(w, 16) || !aligned(y, 16) || !aligned(ws, 4) || !aligned(workspace, 1024))
+    return MSD_ERR_BAD_ALIGNMENT;
+  return MSD_OK;
+}
+
+}  // namespace msd
+
+extern "C" {
+
+size_t msd_gemm_w8a16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  if (M < 1 || M > 128 || N < 1 || K < 16) return 0;
+  return msd::plan_w8(M, N, K).bytes;
+}
+
+msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
+                            int64_t K, void* y, msd_out_t ytype, int32_t* acc_dbg, void* workspace,
+                            size_t workspace_bytes, void* stream) {
+  using namespace msd;
+  msd_status_t st = check_w8_args(x_bf16, w, w_scale, M, N, K, y, ytype, workspace);
+  if (st != MSD_OK) return st;
+  const GemmW8Plan pl = plan_w8(M, N, K);
+  if (workspace_bytes < pl.bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
+  unsigned* status = device_status_ptr();
+  if (!status) return MSD_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  int8_t* q = reinterpret_cast<int8_t*>(ws + pl.off_q);
+  float* alpha = reinterpret_cast<float*>(ws + pl.off_alpha);
+  float* beta = reinterpret_cast<float*>(ws + pl.off_beta);
+
+  // rows [0, M) of the stacked operand hold Q1, rows [Mp, Mp+M) hold Q2; the padding rows are never read back
+  st = launch_decompose_int8(x_bf16, M, K, K, q, q + static_cast<size_t>(pl.Mp) * K, alpha, beta, s);
+  if (st != MSD_OK) return st;
+
+  CUtensorMap tmap_w, tmap_x;
+  if (!encode_tmap_2d(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kBlockK, kTileN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, q, K, pl.NB, K, kBlockK, pl.NB, CU_TENSOR_MAP_SWIZZLE_128B))
+    return MSD_ERR_CUDA;
+
+  GemmW8Params p;
+  p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+  p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
+  p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
+  p.w_scale = w_scale; p.alpha = alpha; p.beta = beta; p.y = y; p.acc_dbg = acc_dbg;
+  p.slots = reinterpret_cast<int32_t*>(ws + pl.off_slots);
+  p.counters = reinterpret_cast<unsigned*>(ws + pl.off_counters);
+  p.status = status;
+
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(gemm_w8a16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
+      return MSD_ERR_CUDA;
+    attr_done = true;
+  }
+  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+  if (launch_pdl(gemm_w8a16_kernel, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl, tmap_w, tmap_x, p) != cudaSuccess)
+    return MSD_ERR_CUDA;
+  return MSD_OK;
+}
+
+size_t msd_gemm_w8a16_host_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  if (M < 1 || M > 128 || N < 1 || K < 16) return 0;
+  return msd::plan_w8(M, N, K).bytes + msd::round_up(static_cast<size_t>(M) * K * 2, 1024) +
+         msd::round_up(static_cast<size_t>(M) * N * 4, 1024);
+}
+
+msd_status_t msd_gemm_w8a16_host(const void* x_bf16_host, const int8_t* w, const float* w_scale, int64_t M,
+                                 int64_t N, int64_t K, void* y_host, msd_out_t ytype, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+  using namespace msd;
+  if (M < 1 || M > 128 || N < 1 || K < 16 || K % 16 != 0) return MSD_ERR_BAD_SHAPE;
+  if (!x_bf16_host || !y_host || !workspace) return MSD_ERR_NULL_POINTER;
+  if (!aligned(workspace, 1024)) return MSD_ERR_BAD_ALIGNMENT;
+  if (workspace_bytes < msd_gemm_w8a16_host_workspace_bytes(M, N, K)) return MSD_ERR_WORKSPACE_TOO_SMALL;
+  const size_t inner = plan_w8(M, N, K).bytes;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  uint8_t* x_dev = ws + inner;
+  uint8_t* y_dev = x_dev + round_up(static_cast<size_t>(M) * K * 2, 1024);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t ybytes = static_cast<size_t>(M) * N * (ytype == MSD_OUT_BF16 ? 2 : 4);
+  if (cudaMemcpyAsync(x_dev, x_bf16_host, static_cast<size_t>(M) * K * 2, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return MSD_ERR_CUDA;
+  msd_status_t st = msd_gemm_w8a16(x_dev, w, w_scale, M, N, K, y_dev, ytype, nullptr, workspace, inner, stream);
+  if (st != MSD_OK) return st;
+  if (cudaMemcpyAsync(y_host, y_dev, ybytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return MSD_ERR_CUDA;
+  return MSD_OK;
+}
+
+}  // extern "C"

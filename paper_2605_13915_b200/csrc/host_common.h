@@ -1,0 +1,54 @@
+// Host-side helpers shared by the C-ABI entry points: argument checks, the device status word,
+// tensor-map encoding through the driver entry point, launch-error mapping.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "msd.h"
+
+namespace msd {
+
+// Device address of this device's status word (one per device; NULL on failure).
+unsigned* device_status_ptr();
+
+int sm_count();
+
+// Encodes a 2-D tiled tensor map: `inner` contiguous elements per row, `outer` rows, rows `row_stride_bytes`
+// apart; the box is box_inner x box_outer elements.  Returns false on failure.
+bool encode_tmap_2d(CUtensorMap* out, CUtensorMapDataType dtype, const void* base, uint64_t inner, uint64_t outer,
+                    uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle swizzle);
+bool encode_tmap_3d(CUtensorMap* out, CUtensorMapDataType dtype, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
+                    uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t b0, uint32_t b1, uint32_t b2,
+                    CUtensorMapSwizzle swizzle);
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline msd_status_t launch_status() { return cudaGetLastError() == cudaSuccess ? MSD_OK : MSD_ERR_CUDA; }
+
+// Kernel launch with the programmatic-dependent-launch attribute (the kernel may start while its predecessor in
+// the stream is still running and must call griddepcontrol.wait before touching the predecessor's outputs).
+template <typename... Args>
+cudaError_t launch_pdl(void (*kernel)(Args...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool pdl,
+                       Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+// Internal entry used by the GEMM: decomposition written straight into the stacked operand buffer.
+msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
+                                   float* alpha, float* beta, cudaStream_t stream);
+msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
+                                    uint8_t* e1, uint8_t* e2, cudaStream_t stream);
+
+}  // namespace msd

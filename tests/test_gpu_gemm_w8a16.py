@@ -1,0 +1,108 @@
+"""GPU parity: W8A16 MSD GEMM against the CPU oracle (INT32 accumulators bit-exact, outputs within 1e-3 of the
+row L2 norm), across tile / split / ragged shapes and at the benchmark's full sizes on sampled columns."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_13915_b200 import binding, inputs
+from helpers import bf16_dev, bf16_bits, dev, rel_row_err
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-3          # max |y - y_oracle| <= TOL * ||y_oracle[i,:]||_2
+
+
+def _run(c, out_dtype, want_acc=True, ws=None):
+    x, w, s = bf16_dev(c.x), dev(c.w), dev(c.w_scale)
+    res = binding.gemm_w8a16(x, w, s, out_dtype=out_dtype, want_acc=want_acc, ws=ws)
+    torch.cuda.synchronize()
+    binding.last_device_status()
+    return res
+
+
+def _check(c, out_dtype=torch.float32, ws=None):
+    y, acc = _run(c, out_dtype, True, ws)
+    ref, oacc = oracle.gemm_w8a16(c.x, c.w, c.w_scale, "f64", want_acc=True)
+    assert np.array_equal(acc.cpu().numpy(), oacc), "INT32 accumulators differ"
+    if out_dtype == torch.float32:
+        got = y.cpu().numpy()
+    else:
+        got = oracle.bf16_bits_to_f64(bf16_bits(y))
+    assert rel_row_err(got, ref).max() <= TOL
+    if out_dtype == torch.bfloat16:
+        # at most one BF16 ulp from the oracle's once-rounded BF16 output
+        want = oracle.round_bf16(ref).view(np.int16).astype(np.int32)
+        have = bf16_bits(y).view(np.int16).astype(np.int32)
+        assert np.abs(want - have).max() <= 1
+    return got, ref
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 128, 128), (8, 256, 512), (16, 4096, 4096), (5, 384, 272), (128, 512, 1024),
+                                   (33, 1152, 2048), (1, 14336, 4096), (128, 4096, 2048)])
+def test_gemm_w8a16_parity_fp32(M, N, K):
+    _check(inputs.gemm_w8_case(M, N, K, seed=0), torch.float32)
+
+
+@pytest.mark.parametrize("M,N,K", [(4, 1024, 1024), (64, 2048, 512)])
+def test_gemm_w8a16_parity_bf16(M, N, K):
+    _check(inputs.gemm_w8_case(M, N, K, seed=1), torch.bfloat16)
+
+
+def test_ragged_n_fp32_and_workspace_reuse():
+    c = inputs.gemm_w8_case(7, 200, 400 - 400 % 16, seed=3)
+    ws = binding.workspace(binding.gemm_w8a16_workspace_bytes(7, 200, c.x.shape[1]))
+    for _ in range(3):                   # the split-K counters must come back to zero after every call
+        _check(c, torch.float32, ws)
+
+
+@pytest.mark.parametrize("ctas", ["1", "3", "37", "148", "200"])
+def test_split_schedules(ctas, monkeypatch):
+    """Different CTA counts move the tile/segment boundaries; the integer result must not change."""
+    monkeypatch.setenv("MSD_GEMM_CTAS", ctas)
+    _check(inputs.gemm_w8_case(16, 640, 1536, seed=5), torch.float32)
+    _check(inputs.gemm_w8_case(128, 256, 768, seed=6), torch.bfloat16)
+
+
+def test_without_programmatic_dependent_launch(monkeypatch):
+    monkeypatch.setenv("MSD_NO_PDL", "1")
+    _check(inputs.gemm_w8_case(16, 1024, 1024, seed=7), torch.float32)
+
+
+def test_msd_error_not_worse_than_dequant_reference():
+    """MSD error against the FP64 dequantized reference stays below the dequantize-to-BF16 path's error."""
+    c = inputs.gemm_w8_case(16, 1024, 4096, seed=0)
+    y = _run(c, torch.float32, want_acc=False).cpu().numpy()
+    ref = oracle.gemm_ref_w8(c.x, c.w, c.w_scale)
+    deq = oracle.gemm_dequant_bf16_w8(c.x, c.w, c.w_scale)
+    n = np.linalg.norm(ref)
+    assert np.linalg.norm(y - ref) / n <= np.linalg.norm(deq - ref) / n
+
+
+@pytest.mark.parametrize("M", [1, 16, 128])
+@pytest.mark.parametrize("N,K", [(14336, 4096), (4096, 14336)])
+def test_full_size_sampled_columns(M, N, K):
+    """The benchmark's decode shapes in its launch configuration; the oracle recomputes 96 sampled output columns."""
+    c = inputs.gemm_w8_case(M, N, K, seed=0)
+    y, acc = _run(c, torch.bfloat16, True)
+    cols = np.unique(np.concatenate([[0, 127, 128, N - 1], np.random.default_rng(0).integers(0, N, 92)]))
+    ref, oacc = oracle.gemm_w8a16(c.x, c.w[cols], c.w_scale[cols], "f64", want_acc=True)
+    assert np.array_equal(acc.cpu().numpy()[:, :, cols], oacc)
+    got = oracle.bf16_bits_to_f64(bf16_bits(y))[:, cols]
+    want = oracle.bf16_bits_to_f64(oracle.round_bf16(ref))
+    # sampled columns: compare per element against the BF16 spacing instead of the (unknown) full row norm
+    assert np.all(np.abs(got - want) <= np.abs(want) * 2.0 ** -7 + 1e-30)
+
+
+def test_host_buffer_entry_point():
+    c = inputs.gemm_w8_case(16, 1024, 1024, seed=9)
+    M, K = c.x.shape
+    N = c.w.shape[0]
+    xh = torch.from_numpy(c.x.view(np.int16)).view(torch.bfloat16).pin_memory()
+    yh = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    ws = binding.workspace(binding.gemm_w8a16_host_workspace_bytes(M, N, K))
+    binding.gemm_w8a16_host(xh, dev(c.w), dev(c.w_scale), yh, ws)
+    torch.cuda.synchronize()
+    ref = oracle.gemm_w8a16(c.x, c.w, c.w_scale, "f64")
+    assert rel_row_err(oracle.bf16_bits_to_f64(bf16_bits(yh)), ref).max() <= TOL
