@@ -1,0 +1,372 @@
+#!/usr/bin/env python
+"""Benchmark of the MSD hot path on B200.
+
+Workload (benchmark configs[1]): the W8A16 MSD GEMM decode sweep - M in {1,2,4,8,16,32,64,128} tokens against
+INT8 per-channel weights of shape [14336,4096] (MLP up/gate) and [4096,14336] (MLP down), BF16 output.  One *step* is
+one pass over the whole sweep (16 msd_gemm_w8a16 calls = 16 decomposition + 16 GEMM kernels).  Eight distinct weight
+buffers per shape are rotated so that every call streams weights that are not in L2 (one step touches 940 MB).
+
+The printed JSON line follows the repository's bench contract: `value` is the whole-job weight-streaming rate
+(algorithmic bytes / device time) with inputs resident in HBM, `e2e` the same metric through the host-buffer entry
+point, `roofline` the achieved fraction of the measured HBM copy bandwidth, `cpu_baseline` the CPU oracle timed on a
+bounded sample.  `--impl reference` times the CPU oracle alone.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+M_SWEEP = [1, 2, 4, 8, 16, 32, 64, 128]
+SHAPES = [(14336, 4096), (4096, 14336)]          # (N, K)
+NBUF = 8
+METRIC = "msd_w8a16_decode_gemm_weight_hbm_gbps"
+UNIT = "GB/s"
+
+
+def algorithmic_bytes(M, N, K):
+    """Bytes MSD itself must move for one call: INT8 weight once, BF16 activations, weight scales, BF16 output."""
+    return N * K + 2 * M * K + 4 * N + 2 * M * N
+
+
+def executed_ops(M, N, K):
+    """INT8 multiply-accumulates executed by the stacked GEMM, counted as 2 ops each: 2 * (2M) * N * K."""
+    return 2 * (2 * M) * N * K
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed regions run."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.samples = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 6:
+                self.samples.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for p in self.samples:
+            try:
+                sm.append(float(p[0]))
+                mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, p[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def make_inputs(torch, device, seed):
+    """Synthetic sweep inputs on the device: activations N(0,1) with 1 % of the channels x50, weights N(0,0.02)
+    quantized to INT8 per output channel (scale = rowmax/127, round-half-to-even)."""
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    data = {}
+    for (N, K) in SHAPES:
+        ws = []
+        for b in range(NBUF):
+            w = torch.randn((N, K), generator=g, device=device, dtype=torch.float32) * 0.02
+            s = w.abs().amax(dim=1) / 127.0
+            q = torch.clamp(torch.round(w / s[:, None]), -127, 127).to(torch.int8)
+            ws.append((q.contiguous(), s.contiguous()))
+            del w
+        xs = {}
+        n_out = K // 100
+        perm = torch.randperm(K, generator=g, device=device)[:n_out]
+        for M in M_SWEEP:
+            x = torch.randn((M, K), generator=g, device=device, dtype=torch.float32)
+            x[:, perm] *= 50.0
+            xs[M] = x.to(torch.bfloat16).contiguous()
+        data[(N, K)] = (ws, xs)
+    return data
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2605_13915_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the MSD path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=device)
+    binding.lib()
+
+    data = make_inputs(torch, device, seed=1234 + rank)
+    calls = []          # (M, N, K, x, w, s, y, workspace)
+    i = 0
+    for (N, K) in SHAPES:
+        ws_list, xs = data[(N, K)]
+        for M in M_SWEEP:
+            w, s = ws_list[i % NBUF]
+            i += 1
+            y = torch.empty((M, N), dtype=torch.bfloat16, device=device)
+            wsp = binding.workspace(binding.gemm_w8a16_workspace_bytes(M, N, K), device)
+            calls.append((M, N, K, xs[M], w, s, y, wsp))
+    step_bytes = sum(algorithmic_bytes(M, N, K) for (M, N, K, *_r) in calls)
+    step_ops = sum(executed_ops(M, N, K) for (M, N, K, *_r) in calls)
+
+    def step():
+        for (M, N, K, x, w, s, y, wsp) in calls:
+            binding.gemm_w8a16(x, w, s, ws=wsp, out=y)
+
+    stream = torch.cuda.Stream(device=device)
+
+    def capture(fn):
+        with torch.cuda.stream(stream):
+            fn()
+            stream.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                fn()
+        return g
+
+    graph = capture(step)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(replay, steps, warmup):
+        with torch.cuda.stream(stream):
+            for _ in range(warmup):
+                replay()
+            stream.synchronize()
+            barrier()
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(steps):
+                replay()
+            e1.record(stream)
+            stream.synchronize()
+            barrier()
+            ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.start()
+    ms = timed(graph.replay, args.steps, args.warmup)
+    binding.last_device_status()
+
+    # ---- end to end: activations and results in pinned host memory, copies inside the timed region ----
+    e2e_calls = []
+    for (M, N, K, x, w, s, y, wsp) in calls:
+        xh = x.cpu().pin_memory()
+        yh = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+        wsh = binding.workspace(binding.gemm_w8a16_host_workspace_bytes(M, N, K), device)
+        e2e_calls.append((xh, w, s, yh, wsh))
+
+    def e2e_step():
+        for (xh, w, s, yh, wsh) in e2e_calls:
+            binding.gemm_w8a16_host(xh, w, s, yh, wsh)
+
+    e2e_graph = capture(e2e_step)
+    e2e_steps = max(1, args.steps // 2)
+    ms_e2e = timed(e2e_graph.replay, e2e_steps, args.warmup)
+    binding.last_device_status()
+    h2d = sum(M * K * 2 for (M, N, K, *_r) in calls)
+    d2h = sum(M * N * 2 for (M, N, K, *_r) in calls)
+    clocks = sampler.stop() if sampler else None
+
+    # ---- per-call breakdown (one graph per call, outside the headline region) ----
+    per_call = []
+    if rank == 0 and not args.no_breakdown:
+        for (M, N, K, x, w, s, y, wsp) in calls:
+            ws_list = data[(N, K)][0]
+
+            def one(M=M, N=N, K=K, x=x, y=y, wsp=wsp, ws_list=ws_list):
+                for (wq, sc) in ws_list:
+                    binding.gemm_w8a16(x, wq, sc, ws=wsp, out=y)
+            gcall = capture(one)
+            t = timed(gcall.replay, 20, 3) / (20 * NBUF) * 1e3
+            per_call.append({"M": M, "N": N, "K": K, "us": round(t, 2),
+                             "gbps": round(algorithmic_bytes(M, N, K) / t / 1e3, 1),
+                             "tops": round(executed_ops(M, N, K) / t / 1e6, 2)})
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = load_peaks()
+    ms_per_step = ms / args.steps
+    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    e2e_value = world * step_bytes / (ms_e2e / e2e_steps * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": "configs[1]: W8A16 MSD GEMM decode sweep, M in {1..128} x {[14336,4096],[4096,14336]}, BF16 out",
+                   "calls_per_step": len(calls), "l2": f"{NBUF} weight buffers per shape rotated; one step streams "
+                   f"{step_bytes / 1e6:.0f} MB (> 126 MB L2)", "launch": "CUDA graph of one step"},
+        "tops": round(world * step_ops / (ms_per_step * 1e-3) / 1e12, 2),
+        "clocks": clocks,
+        "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "api": "msd_gemm_w8a16_host (pinned host activations and outputs, weights resident)"},
+        "gpu_launches": 2 * len(calls) * args.steps,
+        "roofline": {"bound": "hbm", "achieved": round(value / world, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": round(value / world / peaks["hbm_gbs"], 4), "peak_kind": f"of {peak_kind}",
+                     "traffic": None, "kernel": "gemm_w8a16_kernel (+ decompose_int8_kernel overlapped by PDL)",
+                     "note": "achieved = algorithmic bytes of the sweep / device time of the timed region"},
+        "per_call": per_call,
+    }
+    traffic_file = os.path.join(ROOT, "profiles", "gemm_w8a16_traffic.json")
+    if os.path.exists(traffic_file):
+        with open(traffic_file) as f:
+            out["roofline"]["traffic"] = json.load(f)
+    if not args.no_cpu_baseline and world == 1:
+        out["cpu_baseline"] = cpu_baseline(calls=[(16, N, K) for (N, K) in SHAPES], check=(binding, data, torch))
+    print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(calls, check=None, ncols=2048):
+    """Times the CPU oracle, as it stands, on a bounded sample: M=16 of the sweep on both weight shapes, restricted to
+    `ncols` evenly spaced output channels; the rate is scaled by the sample's own algorithmic bytes."""
+    import oracle
+    from paper_2605_13915_b200 import inputs
+    cores = oracle.max_threads()
+    tot_bytes, tot_s, parity = 0.0, 0.0, True
+    for (M, N, K) in calls:
+        cols = np.linspace(0, N - 1, ncols).astype(np.int64)
+        if check is not None:
+            binding, data, torch = check
+            wq, sc = data[(N, K)][0][0]
+            x = data[(N, K)][1][M]
+            w_np = wq[torch.from_numpy(cols).to(wq.device)].cpu().numpy()
+            s_np = sc[torch.from_numpy(cols).to(sc.device)].cpu().numpy()
+            x_np = x.cpu().view(torch.int16).numpy().view(np.uint16)
+        else:
+            c = inputs.gemm_w8_case(M, ncols, K, seed=0)
+            w_np, s_np, x_np = c.w, c.w_scale, c.x
+        t0 = time.perf_counter()
+        ref = oracle.gemm_w8a16(x_np, w_np, s_np, "f64")
+        tot_s += time.perf_counter() - t0
+        tot_bytes += algorithmic_bytes(M, ncols, K)
+        if check is not None:
+            y = binding.gemm_w8a16(x, wq, sc)
+            torch.cuda.synchronize()
+            got = y[:, torch.from_numpy(cols).to(y.device)].float().cpu().numpy().astype(np.float64)
+            parity = parity and bool(np.all(np.abs(got - ref) <= np.abs(ref) * 2.0 ** -7 + 1e-6))
+    res = {"value": round(tot_bytes / tot_s / 1e9, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": f"M=16 of the sweep on both weight shapes, {ncols} of N output channels each (full K); "
+                     f"{tot_s:.1f} s of CPU time", "seconds": round(tot_s, 2)}
+    if check is not None:
+        res["gpu_matches_oracle_on_sample"] = parity
+    return res
+
+
+def run_reference(args):
+    """The CPU oracle as the comparison arm: every step is the bounded sample cpu_baseline() uses."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2605_13915_b200 import inputs
+    ncols = 512
+    cases = [(inputs.gemm_w8_case(16, ncols, K, seed=0), K) for (_N, K) in SHAPES]
+    step_bytes = sum(algorithmic_bytes(16, ncols, K) for (_c, K) in cases)
+
+    def step():
+        for (c, _K) in cases:
+            oracle.gemm_w8a16(c.x, c.w, c.w_scale, "f64")
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = step_bytes * args.steps / dt / 1e9
+    sample = f"per step: M=16 on both weight shapes, {ncols} output channels each (full K)"
+    out = {"impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": world,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt / args.steps * 1e3, 3),
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+           "config": {"workload": "configs[1] sample: " + sample},
+           "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "kind": "oracle", "cores": oracle.max_threads(),
+                            "sample": sample},
+           "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="msd", choices=["msd", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-breakdown", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "msd" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

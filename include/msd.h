@@ -90,6 +90,11 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
                             int64_t K, void* y, msd_out_t ytype, int32_t* acc_dbg, void* workspace,
                             size_t workspace_bytes, void* stream);
 
+/* Diagnostic hook: when `device_buffer` is non-NULL, every later msd_gemm_w8a16 launch writes 16 64-bit SM-clock
+ * samples per CTA into it (entry, set-up done, producer / MMA / epilogue milestones); NULL switches it off.
+ * The buffer must hold 16 * 8 bytes per SM-count CTA (256 CTAs at most). */
+void msd_debug_set_trace(void* device_buffer);
+
 /* Same computation with the activations and the result in HOST memory (pinned for asynchronous copies):
  * copies x to the device workspace, runs msd_gemm_w8a16, copies y back; weights stay resident on the device.
  * workspace: >= msd_gemm_w8a16_host_workspace_bytes(M,N,K). */

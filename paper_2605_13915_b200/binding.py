@@ -35,6 +35,7 @@ _SIGS = {
     "msd_decompose_mxfp4": (C.c_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp]),
     "msd_gemm_w8a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_w8a16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _vp, _sz, _vp]),
+    "msd_debug_set_trace": (None, [_vp]),
     "msd_gemm_w8a16_host_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_w8a16_host": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_gemm_dequant_bf16_workspace_bytes": (_sz, [_i64, _i64, _i64]),

@@ -4,10 +4,13 @@
 // (the M axis of tcgen05.mma), the stacked components [Q1; Q2] (NB = 2*ceil8(M) rows) are the "B" operand, so one
 // weight tile read from HBM serves both passes and the accumulator D[128 weight rows x NB] lives in TMEM.
 //
-// Work split ("stream-K"): the (weight tile, 128-byte K block) pairs are numbered tile-major and divided evenly over
-// the CTAs (one per SM), so every SM streams the same number of weight bytes.  A CTA whose range covers a whole tile
-// finishes it alone; a tile shared by several CTAs is reduced through per-CTA INT32 slots in the workspace and finished
-// by whichever CTA arrives last (integer sums: the result does not depend on the arrival order).
+// Two work splits, chosen on the host:
+//  * row partition (tall weights): the N weight rows are cut into one band per CTA (band heights h and h+8, multiples
+//    of 8, at most 128), each CTA runs the whole K loop for its band and writes its outputs straight from TMEM.
+//  * stream-K (few rows per SM): the (128-row tile, 128-byte K block) pairs are numbered tile-major and divided evenly
+//    over the CTAs, so every SM streams the same number of weight bytes.  A CTA whose range covers a whole tile
+//    finishes it alone; a tile shared by several CTAs is reduced through per-CTA INT32 slots in the workspace and
+//    finished by whichever CTA arrives last (integer sums: the result does not depend on the arrival order).
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (+ TMEM owner), warps 2-5 = epilogue (one per TMEM lane group).
 #include <cuda_bf16.h>
@@ -21,13 +24,18 @@ namespace msd {
 
 constexpr int kTileN = 128;        // weight rows per tile (MMA M)
 constexpr int kBlockK = 128;       // K bytes per pipeline stage (one 128-byte swizzle row)
-constexpr int kMaxStages = 12;
+constexpr int kMaxStages = 16;
 constexpr int kGemmThreads = 192;
 constexpr int kWStageBytes = kTileN * kBlockK;
 constexpr int kSmemBudget = 227 * 1024 - 4096;   // leaves room for the static barriers and the alignment pad
 
 struct GemmW8Params {
   int M, Mp, NB, N, K;
+  int mode;                // 0 = stream-K over 128-row tiles, 1 = one row band per CTA
+  int groups8;             // ceil(N / 8): row groups divided over the CTAs in mode 1
+  int hmax;                // tallest band (box rows of tmap_w; tmap_w2 has hmax - 8)
+  int w_stage_bytes;       // shared-memory bytes reserved for the weight tile of one stage
+  int kb_rot_step;         // mode 1: CTA c starts its K loop at block (c * kb_rot_step) % kblocks
   int kblocks;             // K blocks per weight tile
   int num_tiles;
   long long total_blocks;  // num_tiles * kblocks
@@ -42,7 +50,12 @@ struct GemmW8Params {
   int32_t* slots;          // [gridDim.x * 2][NB][128]
   unsigned* counters;      // [num_tiles]
   unsigned* status;
+  long long* trace;        // nullable diagnostic buffer: 16 clock samples per CTA
 };
+
+__device__ __forceinline__ void trace_mark(const GemmW8Params& p, int slot) {
+  if (p.trace) p.trace[blockIdx.x * 16 + slot] = clock64();
+}
 
 __device__ __forceinline__ long long range_begin(long long cta, long long total, long long grid) { return cta * total / grid; }
 __device__ __forceinline__ long long block_owner(long long blk, long long total, long long grid) {
@@ -60,8 +73,8 @@ __device__ __forceinline__ void store_out(const GemmW8Params& p, int i, int n, f
 }
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
-                  const GemmW8Params p) {
+gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_w2,
+                  const __grid_constant__ CUtensorMap tmap_x, const GemmW8Params p) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ __align__(8) uint64_t full_bar[kMaxStages];
   __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
@@ -74,9 +87,15 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  if (threadIdx.x == 0 && p.trace) {
+    trace_mark(p, 0);
+    unsigned long long g;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g));
+    p.trace[blockIdx.x * 16 + 1] = static_cast<long long>(g);
+  }
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
   const int x_stage_bytes = p.NB * kBlockK;
-  const int stage_bytes = kWStageBytes + x_stage_bytes;
+  const int stage_bytes = p.w_stage_bytes + x_stage_bytes;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.num_stages; ++s) {
@@ -90,6 +109,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     abort_flag = 0;
     mbar_init_fence();
     tma_prefetch_desc(&tmap_w);
+    tma_prefetch_desc(&tmap_w2);
     tma_prefetch_desc(&tmap_x);
   }
   if (warp == 1) tmem_alloc(&tmem_base_slot, p.tmem_cols);
@@ -98,10 +118,28 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
   volatile int* abort = &abort_flag;
+  if (threadIdx.x == 0) trace_mark(p, 2);
 
   const long long grid = gridDim.x;
-  const long long blk_begin = range_begin(blockIdx.x, p.total_blocks, grid);
-  const long long blk_end = range_begin(blockIdx.x + 1, p.total_blocks, grid);
+  // mode 0: this CTA's slice of the tile-major (tile, K block) sequence; mode 1: its row band and every K block
+  long long blk_begin, blk_end;
+  int band_row0 = 0, band_h = kTileN;
+  if (p.mode == 0) {
+    blk_begin = range_begin(blockIdx.x, p.total_blocks, grid);
+    blk_end = range_begin(blockIdx.x + 1, p.total_blocks, grid);
+  } else {
+    const int g0 = static_cast<int>(range_begin(blockIdx.x, p.groups8, grid));
+    const int g1 = static_cast<int>(range_begin(blockIdx.x + 1, p.groups8, grid));
+    band_row0 = 8 * g0;
+    band_h = 8 * (g1 - g0);
+    blk_begin = 0;
+    blk_end = p.kblocks;
+  }
+  // Mode 1: every CTA walks K from its own starting block so that concurrent requests of the CTAs spread over the
+  // whole row instead of hitting the same 128-byte column of every row (integer sums do not depend on the order).
+  const int kb_rot = (p.mode == 1) ? static_cast<int>((static_cast<long long>(blockIdx.x) * p.kb_rot_step) % p.kblocks) : 0;
+  const CUtensorMap* wmap = (p.mode == 1 && band_h != p.hmax) ? &tmap_w2 : &tmap_w;
+  const int tx_bytes = (p.mode == 0 ? kWStageBytes : band_h * kBlockK) + x_stage_bytes;
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -115,28 +153,31 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       const int pre = static_cast<int>(nblk < p.num_stages ? nblk : p.num_stages);
       for (int i = 0; i < pre; ++i) {
         const long long blk = blk_begin + i;
-        const int tile = static_cast<int>(blk / p.kblocks), kb = static_cast<int>(blk % p.kblocks);
-        mbar_arrive_expect_tx(&full_bar[i], stage_bytes);
-        tma_load_2d_hint(smem + i * stage_bytes, &tmap_w, kb * kBlockK, tile * kTileN, &full_bar[i], pol_w);
+        const int tile = static_cast<int>(blk / p.kblocks), kb = static_cast<int>((blk + kb_rot) % p.kblocks);
+        mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
+        tma_load_2d_hint(smem + i * stage_bytes, wmap, kb * kBlockK, band_row0 + tile * kTileN, &full_bar[i], pol_w);
       }
+      trace_mark(p, 3);
       pdl_wait_primary();
+      trace_mark(p, 4);
       for (int i = 0; i < pre; ++i) {
-        const int kb = static_cast<int>((blk_begin + i) % p.kblocks);
-        tma_load_2d_hint(smem + i * stage_bytes + kWStageBytes, &tmap_x, kb * kBlockK, 0, &full_bar[i], pol_x);
+        const int kb = static_cast<int>((blk_begin + i + kb_rot) % p.kblocks);
+        tma_load_2d_hint(smem + i * stage_bytes + p.w_stage_bytes, &tmap_x, kb * kBlockK, 0, &full_bar[i], pol_x);
       }
       stage = pre % p.num_stages;
       phase = (pre == p.num_stages) ? 1 : 0;
       bool ok = true;
       for (long long blk = blk_begin + pre; blk < blk_end && ok; ++blk) {
-        const int tile = static_cast<int>(blk / p.kblocks), kb = static_cast<int>(blk % p.kblocks);
+        const int tile = static_cast<int>(blk / p.kblocks), kb = static_cast<int>((blk + kb_rot) % p.kblocks);
         ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
         if (!ok) break;
-        mbar_arrive_expect_tx(&full_bar[stage], stage_bytes);
+        mbar_arrive_expect_tx(&full_bar[stage], tx_bytes);
         uint8_t* dst = smem + stage * stage_bytes;
-        tma_load_2d_hint(dst, &tmap_w, kb * kBlockK, tile * kTileN, &full_bar[stage], pol_w);
-        tma_load_2d_hint(dst + kWStageBytes, &tmap_x, kb * kBlockK, 0, &full_bar[stage], pol_x);
+        tma_load_2d_hint(dst, wmap, kb * kBlockK, band_row0 + tile * kTileN, &full_bar[stage], pol_w);
+        tma_load_2d_hint(dst + p.w_stage_bytes, &tmap_x, kb * kBlockK, 0, &full_bar[stage], pol_x);
         if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
       }
+      trace_mark(p, 5);
       if (!ok) {
         // give copies already in flight a bounded time to land before the CTA goes away
         const long long t0 = clock64();
@@ -164,9 +205,10 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         for (long long b = blk; b < seg_end; ++b) {
           ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
           if (!ok) break;
+          if (b == blk_begin) trace_mark(p, 6);
           tc_fence_after();
           const uint32_t wa = smem_u32(smem + stage * stage_bytes);
-          const uint32_t xa = wa + kWStageBytes;
+          const uint32_t xa = wa + p.w_stage_bytes;   // the MMA reads 128 A rows; rows past the band are never used
 #pragma unroll
           for (int k = 0; k < kBlockK / 32; ++k) {
             const uint64_t adesc = smem_desc(wa + k * 32, 16, 1024, kSwizzle128B);
@@ -181,6 +223,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         ++seg;
         blk = seg_end;
       }
+      trace_mark(p, 7);
     }
   } else {
     // ------------------------------ epilogue (warps 2..5) ------------------------------
@@ -205,27 +248,30 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       const int acc = seg & 1;
       ok = wait_bounded(&tfull_bar[acc], (seg >> 1) & 1, abort, p.status);
       if (!ok) break;
+      if (et == 0) { if (seg == 0) trace_mark(p, 8); trace_mark(p, 9); }
       tc_fence_after();
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * p.NB;
-      const int n = tile * kTileN + r;
+      const int n = band_row0 + tile * kTileN + r;
+      const bool row_ok = (r < band_h) && (n < p.N);
+      const float sw = row_ok ? __ldg(p.w_scale + n) : 0.0f;
       bool finish = complete;
       int c_lo = 0, c_hi = -1;
       if (!complete) {
         // park this CTA's partial sums in its slot, then find out whether it is the last contributor of the tile
         const int slot_id = 2 * blockIdx.x + ((blk_begin >= tile_begin) ? 0 : 1);
         int32_t* slot = p.slots + static_cast<long long>(slot_id) * p.NB * kTileN;
-        for (int c0 = 0; c0 < p.NB; c0 += 8) {
-          uint32_t v[8];
-          tmem_ld8(t_row + c0, v);
+        for (int c0 = 0; c0 < p.NB; c0 += 16) {
+          uint32_t v[16];
+          tmem_ld16(t_row + c0, v);
           tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 8; ++j) slot[(c0 + j) * kTileN + r] = static_cast<int32_t>(v[j]);
+          for (int j = 0; j < 16; ++j) slot[(c0 + j) * kTileN + r] = static_cast<int32_t>(v[j]);
         }
-        __threadfence();
         named_bar_sync(1, 128);
         c_lo = static_cast<int>(block_owner(tile_begin, p.total_blocks, grid));
         c_hi = static_cast<int>(block_owner(tile_end - 1, p.total_blocks, grid));
         if (et == 0) {
+          __threadfence();     // cumulative: publishes the slot writes of all 128 threads ordered by the barrier above
           const unsigned prev = atomicAdd(&p.counters[tile], 1u);
           const int last = (prev == static_cast<unsigned>(c_hi - c_lo)) ? 1 : 0;
           if (last) p.counters[tile] = 0;          // leave the counter ready for the next call
@@ -236,7 +282,6 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         if (finish) __threadfence();
       }
       if (finish) {
-        const float sw = (n < p.N) ? __ldg(p.w_scale + n) : 0.0f;
         for (int c0 = 0; c0 < p.Mp; c0 += 8) {
           uint32_t a[8], b[8];
           tmem_ld8(t_row + c0, a);
@@ -252,7 +297,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
               b[j] += static_cast<uint32_t>(__ldcg(slot + (p.Mp + c0 + j) * kTileN + r));
             }
           }
-          if (n < p.N) {
+          if (row_ok) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               const int i = c0 + j;
@@ -272,15 +317,19 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       ++seg;
       blk = seg_end;
     }
+    if (et == 0) { trace_mark(p, 10); if (p.trace) p.trace[blockIdx.x * 16 + 11] = seg; }
   }
 
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) trace_mark(p, 12);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, p.tmem_cols);
   }
 }
+
+static long long* g_trace = nullptr;
 
 static int pow2_at_least(int v) {
   int p = 32;
@@ -290,10 +339,17 @@ static int pow2_at_least(int v) {
 
 struct GemmW8Plan {
   int Mp, NB, kblocks, num_tiles, grid, stages, tmem_cols;
+  int mode, groups8, hmax, w_stage_bytes;
   long long total_blocks;
   size_t off_q, off_alpha, off_beta, off_counters, off_slots, bytes;
   size_t smem_bytes;
 };
+
+static int env_int(const char* name, int fallback) {
+  const char* e = getenv(name);
+  if (!e || !*e) return fallback;
+  return atoi(e);
+}
 
 static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K) {
   GemmW8Plan pl;
@@ -302,19 +358,35 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K) {
   pl.kblocks = static_cast<int>((K + kBlockK - 1) / kBlockK);
   pl.num_tiles = static_cast<int>((N + kTileN - 1) / kTileN);
   pl.total_blocks = static_cast<long long>(pl.kblocks) * pl.num_tiles;
-  int grid = sm_count();
-  if (const char* e = getenv("MSD_GEMM_CTAS")) {
-    const int g = atoi(e);
-    if (g > 0) grid = g;
+  pl.groups8 = static_cast<int>((N + 7) / 8);
+  const int sms = sm_count();
+  int grid = env_int("MSD_GEMM_CTAS", sms);
+  if (grid < 1) grid = sms;
+  if (grid > 256) grid = 256;
+  // Row partition pays when every SM gets a band of at least 64 rows (the MMA always spans 128 rows, so shorter
+  // bands waste tensor time and TMA rows on the shared activation tile) and the bands still fit one MMA.
+  const int band_max = 8 * ((pl.groups8 + grid - 1) / grid);
+  const int band_min = 8 * (pl.groups8 / grid);
+  int mode = (band_min >= 64 && band_max <= kTileN) ? 1 : 0;
+  mode = env_int("MSD_GEMM_MODE", mode);
+  if (mode == 1 && (band_max > kTileN || band_min < 8)) mode = 0;
+  pl.mode = mode;
+  if (mode == 1) {
+    pl.hmax = band_max;
+    pl.w_stage_bytes = static_cast<int>(round_up(static_cast<size_t>(band_max) * kBlockK, 1024));
+  } else {
+    if (grid > pl.total_blocks) grid = static_cast<int>(pl.total_blocks);
+    pl.hmax = kTileN;
+    pl.w_stage_bytes = kWStageBytes;
   }
-  if (grid > pl.total_blocks) grid = static_cast<int>(pl.total_blocks);
-  if (grid < 1) grid = 1;
   pl.grid = grid;
-  const int stage_bytes = kWStageBytes + pl.NB * kBlockK;
-  int stages = kSmemBudget / stage_bytes;
+  const int stage_bytes = pl.w_stage_bytes + pl.NB * kBlockK;
+  const int tail_pad = kWStageBytes - pl.w_stage_bytes;     // the MMA reads a full 128-row A tile from every stage
+  int stages = (kSmemBudget - tail_pad) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
+  if (stages > pl.kblocks && mode == 1) stages = pl.kblocks > 1 ? pl.kblocks : 1;
   pl.stages = stages;
-  pl.smem_bytes = static_cast<size_t>(stages) * stage_bytes + 1024;
+  pl.smem_bytes = static_cast<size_t>(stages) * stage_bytes + tail_pad + 1024;
   pl.tmem_cols = pow2_at_least(2 * pl.NB);
   size_t off = 0;
   pl.off_q = off;         off = round_up(off + static_cast<size_t>(pl.NB) * K, 1024);
@@ -322,8 +394,7 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K) {
   pl.off_beta = off;      off = round_up(off + 128 * sizeof(float), 256);
   pl.off_counters = off;  off = round_up(off + static_cast<size_t>(pl.num_tiles) * sizeof(unsigned), 1024);
   // slot space sized for the largest grid the launcher may pick, so the same workspace serves any override
-  const int max_grid = sm_count() > 256 ? sm_count() : 256;
-  pl.off_slots = off;     off = round_up(off + static_cast<size_t>(max_grid) * 2 * pl.NB * kTileN * sizeof(int32_t), 1024);
+  pl.off_slots = off;     off = round_up(off + static_cast<size_t>(256) * 2 * pl.NB * kTileN * sizeof(int32_t), 1024);
   pl.bytes = off;
   return pl;
 }
@@ -368,19 +439,24 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
   st = launch_decompose_int8(x_bf16, M, K, K, q, q + static_cast<size_t>(pl.Mp) * K, alpha, beta, s);
   if (st != MSD_OK) return st;
 
-  CUtensorMap tmap_w, tmap_x;
-  if (!encode_tmap_2d(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kBlockK, kTileN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+  CUtensorMap tmap_w, tmap_w2, tmap_x;
+  const uint32_t box2 = (pl.mode == 1 && pl.hmax > 8) ? pl.hmax - 8 : pl.hmax;
+  if (!encode_tmap_2d(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kBlockK, pl.hmax, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_w2, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kBlockK, box2, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, q, K, pl.NB, K, kBlockK, pl.NB, CU_TENSOR_MAP_SWIZZLE_128B))
     return MSD_ERR_CUDA;
 
   GemmW8Params p;
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+  p.kb_rot_step = env_int("MSD_GEMM_KROT", 5);
+  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_stage_bytes = pl.w_stage_bytes;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
   p.w_scale = w_scale; p.alpha = alpha; p.beta = beta; p.y = y; p.acc_dbg = acc_dbg;
   p.slots = reinterpret_cast<int32_t*>(ws + pl.off_slots);
   p.counters = reinterpret_cast<unsigned*>(ws + pl.off_counters);
   p.status = status;
+  p.trace = g_trace;
 
   static bool attr_done = false;
   if (!attr_done) {
@@ -389,10 +465,12 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
     attr_done = true;
   }
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  if (launch_pdl(gemm_w8a16_kernel, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl, tmap_w, tmap_x, p) != cudaSuccess)
+  if (launch_pdl(gemm_w8a16_kernel, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
     return MSD_ERR_CUDA;
   return MSD_OK;
 }
+
+void msd_debug_set_trace(void* device_buffer) { msd::g_trace = static_cast<long long*>(device_buffer); }
 
 size_t msd_gemm_w8a16_host_workspace_bytes(int64_t M, int64_t N, int64_t K) {
   if (M < 1 || M > 128 || N < 1 || K < 16) return 0;

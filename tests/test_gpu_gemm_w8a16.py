@@ -65,6 +65,15 @@ def test_split_schedules(ctas, monkeypatch):
     _check(inputs.gemm_w8_case(128, 256, 768, seed=6), torch.bfloat16)
 
 
+@pytest.mark.parametrize("mode,ctas", [("0", "148"), ("1", "148"), ("1", "100"), ("1", "111")])
+def test_row_partition_and_stream_k_agree(mode, ctas, monkeypatch):
+    """Tall weights can run either split; band heights (multiples of 8, two sizes) and a ragged last band."""
+    monkeypatch.setenv("MSD_GEMM_MODE", mode)
+    monkeypatch.setenv("MSD_GEMM_CTAS", ctas)
+    _check(inputs.gemm_w8_case(16, 12000, 512, seed=8), torch.float32)
+    _check(inputs.gemm_w8_case(128, 10004, 256, seed=9), torch.float32)
+
+
 def test_without_programmatic_dependent_launch(monkeypatch):
     monkeypatch.setenv("MSD_NO_PDL", "1")
     _check(inputs.gemm_w8_case(16, 1024, 1024, seed=7), torch.float32)
