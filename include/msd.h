@@ -133,14 +133,16 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
  *   alpha_P = max(tile's v_scale)/127; O += alpha_P P1 V + beta_P P2 V; O / sum(P) at the end.
  *   q_bf16 [B,Hq,D]; k_cache [T,Hkv,D] INT8; v_cache [T,Hkv,Dv] INT8 or NULL (V = first Dv entries of the K row);
  *   k_scale [T,Hkv] FP32; v_scale [T,Hkv] or NULL (= k_scale); cu_seqlens [B+1] INT32 token offsets (device);
+ *   total_tokens = T, the number of token rows the caches hold (>= cu_seqlens[B]); max_seqlen >= every length;
  *   out_bf16 [B,Hq,Dv]; lse nullable [B,Hq] FP32 (natural-log sum of exp of the scaled scores).
- * Hq % Hkv == 0; D % 16 == 0; Dv % 16 == 0; Dv <= D when v_cache is NULL.  Empty sequences give zeros.
+ * Hq % Hkv == 0; D % 16 == 0, D <= 640; Dv % 16 == 0, Dv <= 512; Dv <= D when v_cache is NULL.
+ * Empty sequences give zeros and lse = -inf.
  */
 size_t msd_attn_decode_int8kv_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
                                               int32_t max_seqlen);
 msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, const int8_t* v_cache,
                                     const float* k_scale, const float* v_scale, const int32_t* cu_seqlens,
-                                    int32_t max_seqlen, int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
+                                    int64_t total_tokens, int32_t max_seqlen, int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
                                     float softmax_scale, void* out_bf16, float* lse, void* workspace,
                                     size_t workspace_bytes, void* stream);
 

@@ -43,7 +43,7 @@ _SIGS = {
     "msd_gemm_w4a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_w4a16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_attn_decode_int8kv_workspace_bytes": (_sz, [_i32] * 6),
-    "msd_attn_decode_int8kv": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp,
+    "msd_attn_decode_int8kv": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp,
                                          _vp, _sz, _vp]),
     "msd_attn_decode_schedule": (C.c_int, [_i32] * 6 + [C.POINTER(_i32), C.POINTER(_i32)]),
 }
@@ -219,7 +219,7 @@ def attn_decode_int8kv(q, k, v, k_scale, v_scale, cu_seqlens, max_seqlen, softma
     o = out if out is not None else torch.empty((B, Hq, Dv), dtype=torch.bfloat16, device=q.device)
     lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if want_lse else None
     wp, wb = _ws_ptr(ws)
-    code = lib().msd_attn_decode_int8kv(_ptr(q), _ptr(k), _ptr(v), _ptr(k_scale), _ptr(v_scale), _ptr(cu_seqlens), max_seqlen,
-                                        B, Hq, Hkv, D, Dv, softmax_scale, _ptr(o), _ptr(lse), wp, wb, _stream())
+    code = lib().msd_attn_decode_int8kv(_ptr(q), _ptr(k), _ptr(v), _ptr(k_scale), _ptr(v_scale), _ptr(cu_seqlens), int(k.shape[0]),
+                                        max_seqlen, B, Hq, Hkv, D, Dv, softmax_scale, _ptr(o), _ptr(lse), wp, wb, _stream())
     _check(code, "msd_attn_decode_int8kv")
     return (o, lse) if want_lse else o

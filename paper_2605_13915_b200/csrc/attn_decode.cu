@@ -1,0 +1,497 @@
+// Decode attention over an INT8 KV cache with MSD on Q and on the softmax probabilities (Sec. 4, Alg. 3; tiled
+// form Sec. 4.3), split over the context (flash-decoding) and merged with the log-sum-exp rule.
+//
+// One CTA handles one (sequence, KV head, group of up to HG query heads, context split) and walks its tokens in
+// tiles of 128.  Both GEMMs run on tcgen05 with the TOKENS on the MMA M axis / TMEM lanes:
+//   S^T[128 tokens x Rp]  = K_tile[128 x D] (K-major, TMA, 128-byte swizzle)  x  Qstack[Rp x D]^T
+//   O^T[128 dv x Rp]      = V_tile^T[dv x 128 tokens] (the same TMA layout read as an MN-major operand)  x  Pstack[Rp x 128]^T
+// where Rp = 2*HG stacked rows: rows [0,HG) hold the first INT8 component of each head, rows [HG,2HG) the second,
+// so one KV tile read from HBM serves both passes.  When v_cache is NULL the V operand aliases the first Dv bytes of
+// the K rows already in shared memory (MLA latent cache) and nothing is loaded twice.
+//
+// Warps: 0 = TMA producer, 1 = MMA issuer + TMEM owner, 2..5 = softmax / merge (thread = token lane for the softmax,
+// = dv lane for the merge).  The next tile's QK^T is issued while the current tile's softmax runs (S^T is double
+// buffered in TMEM).  Every wait is bounded.
+#include <cuda_bf16.h>
+
+#include <cmath>
+#include <cstdlib>
+
+#include "host_common.h"
+#include "sm100.cuh"
+
+namespace msd {
+
+constexpr int kTok = 128;           // tokens per tile
+constexpr int kAttnThreads = 192;
+constexpr int kChunk = 128;         // bytes of D / Dv per TMA box and per shared-memory operand chunk
+constexpr int kChunkBytes = kTok * kChunk;
+
+struct AttnParams {
+  const uint16_t* q;      // [B,Hq,D] BF16
+  const float* k_scale;   // [T,Hkv]
+  const float* v_scale;   // [T,Hkv]
+  const int32_t* cu;      // [B+1]
+  float* partial;         // [B,Hq,n_splits,Dv+2]: m, l, O[Dv]
+  int B, Hq, Hkv, D, Dv, G;
+  int HG, Rp, groups;     // heads per CTA, stacked rows, head groups per KV head
+  int DC, DVT;            // 128-byte chunks of D / Dv
+  int n_splits, stages;
+  int v_alias;            // 1: V is the first Dv bytes of the K rows
+  int tmem_cols;
+  float scale;
+  unsigned* status;
+};
+
+__device__ __forceinline__ int swz_off(int row, int byte_in_row) {
+  // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
+  return row * 128 + ((((byte_in_row >> 4) ^ (row & 7)) & 7) << 4) + (byte_in_row & 15);
+}
+
+template <int kMaxHG, int kMaxDVT>
+__global__ void __launch_bounds__(kAttnThreads)
+attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], s_full[2], p_full, o_full, o_empty;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+  __shared__ float s_aq[kMaxHG], s_bq[kMaxHG];
+  __shared__ float red[4][kMaxHG + 1];
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x;
+  int unit = blockIdx.y;
+  const int grp = unit % p.groups; unit /= p.groups;
+  const int hk = unit % p.Hkv;
+  const int b = unit / p.Hkv;
+  const int seq0 = p.cu[b];
+  const int L = p.cu[b + 1] - seq0;
+  const int per = (L + p.n_splits - 1) / p.n_splits;
+  const int Lsplit = (per + kTok - 1) / kTok * kTok;
+  const int t_begin = split * Lsplit;
+  const int t_end = min(L, t_begin + Lsplit);
+  const int h0 = hk * p.G + grp * p.HG;                      // first query head of this CTA
+  const int nh = min(p.HG, p.G - grp * p.HG);                // heads actually present
+  const int ntiles = (t_end > t_begin) ? (t_end - t_begin + kTok - 1) / kTok : 0;
+
+  if (ntiles == 0) {      // nothing in this split: neutral partials, before any barrier or TMEM use
+    for (int i = threadIdx.x; i < nh * (p.Dv + 2); i += blockDim.x) {
+      const int h = i / (p.Dv + 2), e = i % (p.Dv + 2);
+      float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + h) * p.n_splits + split) * (p.Dv + 2);
+      dst[e] = (e == 0) ? -INFINITY : 0.0f;
+    }
+    return;
+  }
+
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+  const int kv_stage_bytes = (p.DC + (p.v_alias ? 0 : p.DVT)) * kChunkBytes;
+  uint8_t* sm_q = smem + p.stages * kv_stage_bytes;          // DC chunks of [Rp x 128]
+  uint8_t* sm_p = sm_q + p.DC * p.Rp * kChunk;               // [Rp x 128]
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
+    mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1);
+    mbar_init(&p_full, 4); mbar_init(&o_full, 1); mbar_init(&o_empty, 4);
+    abort_flag = 0;
+    mbar_init_fence();
+    tma_prefetch_desc(&tmap_k);
+    tma_prefetch_desc(&tmap_v);
+  }
+  if (warp == 1) tmem_alloc(&tmem_base_slot, p.tmem_cols);
+  // zero the stacked Q operand (unused head slots and the padding of the last D chunk must be zero)
+  for (int i = threadIdx.x; i < p.DC * p.Rp * kChunk / 16; i += blockDim.x) reinterpret_cast<uint4*>(sm_q)[i] = make_uint4(0, 0, 0, 0);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  const uint32_t tmem_o = tmem_base + 2 * p.Rp;             // O^T tiles after the two S^T buffers
+  volatile int* abort = &abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer: K (and V) tiles ------------------------------
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      for (int t = 0; t < ntiles; ++t) {
+        if (!wait_bounded(&kv_empty[stage], phase ^ 1, abort, p.status)) break;
+        mbar_arrive_expect_tx(&kv_full[stage], kv_stage_bytes);
+        uint8_t* dst = smem + stage * kv_stage_bytes;
+        const int tok = seq0 + t_begin + t * kTok;
+        for (int c = 0; c < p.DC; ++c) tma_load_3d(dst + c * kChunkBytes, &tmap_k, c * kChunk, hk, tok, &kv_full[stage]);
+        if (!p.v_alias)
+          for (int j = 0; j < p.DVT; ++j)
+            tma_load_3d(dst + (p.DC + j) * kChunkBytes, &tmap_v, j * kChunk, hk, tok, &kv_full[stage]);
+        if (++stage == p.stages) { stage = 0; phase ^= 1; }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      const uint32_t idesc_qk = idesc_dense(2, 1, 1, 0, 0, kTok, p.Rp);     // S8 x S8 -> S32, both K-major
+      const uint32_t idesc_pv = idesc_dense(2, 1, 1, 1, 0, kTok, p.Rp);     // A (V^T) MN-major
+      bool ok = true;
+      // the stacked Q operand is written by the softmax warps; they arrive on p_full once before the first tile
+      ok = wait_bounded(&p_full, 0, abort, p.status);
+      auto issue_qk = [&](int t) {
+        const int st = t % p.stages;
+        if (!wait_bounded(&kv_full[st], (t / p.stages) & 1, abort, p.status)) return false;
+        tc_fence_after();
+        const uint32_t ka = smem_u32(smem + st * kv_stage_bytes);
+        const uint32_t qa = smem_u32(sm_q);
+        const uint32_t d = tmem_base + (t & 1) * p.Rp;
+        for (int c = 0; c < p.DC; ++c)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            mma_i8(d, smem_desc(ka + c * kChunkBytes + k * 32, 16, 1024, kSwizzle128B),
+                   smem_desc(qa + c * p.Rp * kChunk + k * 32, 16, 1024, kSwizzle128B), idesc_qk, (c > 0 || k > 0) ? 1u : 0u);
+        tc_commit(&s_full[t & 1]);
+        return true;
+      };
+      if (ok) ok = issue_qk(0);
+      for (int t = 0; t < ntiles && ok; ++t) {
+        if (t + 1 < ntiles) { ok = issue_qk(t + 1); if (!ok) break; }
+        ok = wait_bounded(&p_full, (t + 1) & 1, abort, p.status);             // P of tile t is in shared memory
+        if (!ok) break;
+        ok = wait_bounded(&o_empty, (t & 1) ^ 1, abort, p.status);           // O^T of tile t-1 has been merged
+        if (!ok) break;
+        tc_fence_after();
+        const int st = t % p.stages;
+        const uint32_t va = smem_u32(smem + st * kv_stage_bytes) + (p.v_alias ? 0 : p.DC * kChunkBytes);
+        const uint32_t pa = smem_u32(sm_p);
+        for (int j = 0; j < p.DVT; ++j)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)        // 32 tokens per MMA: four 8-token groups of 1024 bytes
+            mma_i8(tmem_o + j * p.Rp, smem_desc(va + j * kChunkBytes + k * 4096, 16384, 1024, kSwizzle128B),
+                   smem_desc(pa + k * 32, 16, 1024, kSwizzle128B), idesc_pv, k > 0 ? 1u : 0u);
+        tc_commit(&o_full);
+        tc_commit(&kv_empty[st]);
+      }
+    }
+  } else {
+    // ------------------------------ softmax + merge warps ------------------------------
+    const int quad = warp & 3;
+    const int tl = quad * 32 + lane;                // token lane (softmax) / dv lane (merge)
+    const int wi = warp - 2;                        // 0..3
+    // c1: decompose the query rows of this CTA's heads (one warp per head, round robin) into the stacked operand
+    for (int h = wi; h < nh; h += 4) {
+      const uint16_t* qrow = p.q + (static_cast<long long>(b) * p.Hq + h0 + h) * p.D;
+      float m = 0.0f;
+      for (int d = lane; d < p.D; d += 32) m = fmaxf(m, fabsf(__uint_as_float(static_cast<uint32_t>(qrow[d]) << 16)));
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      const float alpha = __fdiv_rn(m, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
+      if (lane == 0) { s_aq[h] = alpha; s_bq[h] = beta; }
+      for (int d = lane; d < p.D; d += 32) {
+        const float v = __uint_as_float(static_cast<uint32_t>(qrow[d]) << 16);
+        int c1 = 0, c2 = 0;
+        if (alpha > 0.0f) {
+          c1 = max(-128, min(127, __float2int_rn(__fdiv_rn(v, alpha))));
+          const float r = __fmaf_rn(-alpha, static_cast<float>(c1), v);
+          if (beta > 0.0f) c2 = max(-128, min(127, __float2int_rn(__fdiv_rn(r, beta))));
+        }
+        uint8_t* chunk = sm_q + (d >> 7) * p.Rp * kChunk;
+        chunk[swz_off(h, d & 127)] = static_cast<uint8_t>(c1);
+        chunk[swz_off(p.HG + h, d & 127)] = static_cast<uint8_t>(c2);
+      }
+    }
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&p_full);            // phase 0 of p_full: "Q operand ready"
+    named_bar_sync(1, 128);                         // s_aq / s_bq visible to all four warps
+
+    float m_run[kMaxHG], l_part[kMaxHG], aq[kMaxHG], bq[kMaxHG];
+    float o_run[kMaxDVT][kMaxHG];
+#pragma unroll
+    for (int h = 0; h < kMaxHG; ++h) {
+      m_run[h] = -INFINITY; l_part[h] = 0.0f;
+      aq[h] = (h < nh) ? s_aq[h] : 0.0f; bq[h] = (h < nh) ? s_bq[h] : 0.0f;
+#pragma unroll
+      for (int j = 0; j < kMaxDVT; ++j) o_run[j][h] = 0.0f;
+    }
+    const float kLog2e = 1.4426950408889634f;
+    bool ok = true;
+    for (int t = 0; t < ntiles && ok; ++t) {
+      const int tok_rel = t_begin + t * kTok + tl;
+      const bool valid = tok_rel < t_end;
+      const long long sidx = static_cast<long long>(seq0 + tok_rel) * p.Hkv + hk;
+      const float ks = valid ? __ldg(p.k_scale + sidx) * p.scale : 0.0f;
+      const float vs = valid ? __ldg(p.v_scale + sidx) : 0.0f;
+      ok = wait_bounded(&s_full[t & 1], (t >> 1) & 1, abort, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      // c3: merge the two integer products and apply the key scale
+      float s[kMaxHG];
+      const uint32_t srow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + (t & 1) * p.Rp;
+      if constexpr (kMaxHG == 8) {
+        uint32_t v[16];
+        tmem_ld16(srow, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int h = 0; h < 8; ++h)
+          s[h] = valid ? __fmaf_rn(aq[h], static_cast<float>(static_cast<int32_t>(v[h])), bq[h] * static_cast<float>(static_cast<int32_t>(v[8 + h]))) * ks : -INFINITY;
+      } else {
+        uint32_t v1[16], v2[16];
+        tmem_ld16(srow, v1);
+        tmem_ld16(srow + 16, v2);
+        tmem_ld_wait();
+#pragma unroll
+        for (int h = 0; h < 16; ++h)
+          s[h] = valid ? __fmaf_rn(aq[h], static_cast<float>(static_cast<int32_t>(v1[h])), bq[h] * static_cast<float>(static_cast<int32_t>(v2[h]))) * ks : -INFINITY;
+      }
+      // c4: tile maxima per head (and of the value scales) over the 128 token lanes
+      float tm[kMaxHG + 1];
+#pragma unroll
+      for (int h = 0; h < kMaxHG; ++h) tm[h] = s[h];
+      tm[kMaxHG] = vs;
+#pragma unroll
+      for (int h = 0; h <= kMaxHG; ++h) {
+        if (h < p.HG || h == kMaxHG) {
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) tm[h] = fmaxf(tm[h], __shfl_xor_sync(0xffffffffu, tm[h], o));
+        }
+      }
+      if (lane == 0) {
+#pragma unroll
+        for (int h = 0; h <= kMaxHG; ++h) red[wi][h] = tm[h];
+      }
+      named_bar_sync(1, 128);
+      float resc[kMaxHG];
+#pragma unroll
+      for (int h = 0; h < kMaxHG; ++h) {
+        const float mt = fmaxf(fmaxf(red[0][h], red[1][h]), fmaxf(red[2][h], red[3][h]));
+        const float mn = fmaxf(m_run[h], mt);
+        resc[h] = (m_run[h] == -INFINITY) ? 0.0f : exp2f((m_run[h] - mn) * kLog2e);
+        m_run[h] = mn;
+      }
+      const float vs_max = fmaxf(fmaxf(red[0][kMaxHG], red[1][kMaxHG]), fmaxf(red[2][kMaxHG], red[3][kMaxHG]));
+      named_bar_sync(1, 128);                       // everyone has read `red` before the next tile overwrites it
+      // c5: P = exp(S - m), fold the value scale, two-pass INT8 with the fixed scale alpha_P = max(v_scale)/127
+      const float alpha_p = __fdiv_rn(vs_max, 127.0f), beta_p = __fdiv_rn(alpha_p, 254.0f);
+      const float inv_a = alpha_p > 0.0f ? 1.0f / alpha_p : 0.0f, inv_b = beta_p > 0.0f ? 1.0f / beta_p : 0.0f;
+      // the previous tile's PV must have finished reading the P operand before it is overwritten: it has, because
+      // these threads waited for o_full of that tile before merging it
+#pragma unroll
+      for (int h = 0; h < kMaxHG; ++h) {
+        if (h < p.HG) {
+          int c1 = 0, c2 = 0;
+          if (h < nh && valid) {
+            const float pr = exp2f((s[h] - m_run[h]) * kLog2e);
+            l_part[h] = l_part[h] * resc[h] + pr;
+            const float pt = pr * vs;
+            c1 = max(-128, min(127, __float2int_rn(pt * inv_a)));
+            const float r = __fmaf_rn(-alpha_p, static_cast<float>(c1), pt);
+            c2 = max(-128, min(127, __float2int_rn(r * inv_b)));
+          } else {
+            l_part[h] *= resc[h];
+          }
+          sm_p[swz_off(h, tl)] = static_cast<uint8_t>(c1);
+          sm_p[swz_off(p.HG + h, tl)] = static_cast<uint8_t>(c2);
+        }
+      }
+      fence_proxy_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&p_full);
+      // c6/c7: wait for O^T of this tile, merge it into the running output with the rescale factors
+      ok = wait_bounded(&o_full, t & 1, abort, p.status);
+      if (!ok) break;
+      tc_fence_after();
+#pragma unroll
+      for (int j = 0; j < kMaxDVT; ++j) {
+        if (j < p.DVT) {
+          const uint32_t orow = tmem_o + (static_cast<uint32_t>(quad * 32) << 16) + j * p.Rp;
+          if constexpr (kMaxHG == 8) {
+            uint32_t v[16];
+            tmem_ld16(orow, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int h = 0; h < 8; ++h)
+              o_run[j][h] = __fmaf_rn(o_run[j][h], resc[h], __fmaf_rn(alpha_p, static_cast<float>(static_cast<int32_t>(v[h])), beta_p * static_cast<float>(static_cast<int32_t>(v[8 + h]))));
+          } else {
+            uint32_t v1[16], v2[16];
+            tmem_ld16(orow, v1);
+            tmem_ld16(orow + 16, v2);
+            tmem_ld_wait();
+#pragma unroll
+            for (int h = 0; h < 16; ++h)
+              o_run[j][h] = __fmaf_rn(o_run[j][h], resc[h], __fmaf_rn(alpha_p, static_cast<float>(static_cast<int32_t>(v1[h])), beta_p * static_cast<float>(static_cast<int32_t>(v2[h]))));
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&o_empty);
+    }
+    // partial results of this split: running max, sum of P and unnormalised output per head
+    if (ok) {
+#pragma unroll
+      for (int h = 0; h < kMaxHG; ++h) {
+        if (h < nh) {
+          float l = l_part[h];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+          if (lane == 0) red[wi][h] = l;
+        }
+      }
+      named_bar_sync(1, 128);
+#pragma unroll
+      for (int h = 0; h < kMaxHG; ++h) {
+        if (h < nh) {
+          float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + h) * p.n_splits + split) * (p.Dv + 2);
+          if (tl == 0) { dst[0] = m_run[h]; dst[1] = red[0][h] + red[1][h] + red[2][h] + red[3][h]; }
+#pragma unroll
+          for (int j = 0; j < kMaxDVT; ++j)
+            if (j < p.DVT && j * kChunk + tl < p.Dv) dst[2 + j * kChunk + tl] = o_run[j][h];
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, p.tmem_cols);
+  }
+}
+
+// c8: merge the splits of one (sequence, query head) and normalise:  O = sum_s e^{m_s - m} O_s / sum_s e^{m_s - m} l_s
+__global__ void __launch_bounds__(128)
+attn_combine_kernel(const float* __restrict__ partial, int n_splits, int Dv, __nv_bfloat16* __restrict__ out,
+                    float* __restrict__ lse) {
+  const long long row = blockIdx.x;
+  const float* base = partial + row * n_splits * (Dv + 2);
+  float m = -INFINITY;
+  for (int s = 0; s < n_splits; ++s) m = fmaxf(m, base[s * (Dv + 2)]);
+  float l = 0.0f;
+  for (int s = 0; s < n_splits; ++s) {
+    const float ms = base[s * (Dv + 2)];
+    if (ms != -INFINITY) l += expf(ms - m) * base[s * (Dv + 2) + 1];
+  }
+  for (int d = threadIdx.x; d < Dv; d += blockDim.x) {
+    float acc = 0.0f;
+    for (int s = 0; s < n_splits; ++s) {
+      const float ms = base[s * (Dv + 2)];
+      if (ms != -INFINITY) acc += expf(ms - m) * base[s * (Dv + 2) + 2 + d];
+    }
+    out[row * Dv + d] = __float2bfloat16_rn(l > 0.0f ? acc / l : 0.0f);
+  }
+  if (lse && threadIdx.x == 0) lse[row] = (l > 0.0f) ? m + logf(l) : -INFINITY;
+}
+
+struct AttnPlan {
+  int HG, Rp, groups, DC, DVT, n_splits, stages, tmem_cols, v_alias;
+  size_t smem_bytes, ws_bytes;
+};
+
+static int attn_env_int(const char* name, int fallback) {
+  const char* e = getenv(name);
+  return (e && *e) ? atoi(e) : fallback;
+}
+
+static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, bool v_alias, AttnPlan* pl) {
+  if (B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || D < 16 || D % 16 != 0 || Dv < 16 || Dv % 16 != 0) return false;
+  const int G = Hq / Hkv;
+  pl->HG = (G <= 8) ? 8 : 16;
+  pl->Rp = 2 * pl->HG;
+  pl->groups = (G + pl->HG - 1) / pl->HG;
+  pl->DC = (D + kChunk - 1) / kChunk;
+  pl->DVT = (Dv + kChunk - 1) / kChunk;
+  if (pl->DC > 5 || pl->DVT > 4) return false;
+  if (pl->DVT == 3) pl->DVT = 4;
+  if (v_alias && Dv > D) return false;
+  pl->v_alias = v_alias ? 1 : 0;
+  const int kv_stage = (pl->DC + (v_alias ? 0 : pl->DVT)) * kChunkBytes;
+  pl->stages = (kv_stage <= 32 * 1024) ? 2 : 2;
+  const int tiles = (max_seqlen + kTok - 1) / kTok;
+  const long long units = static_cast<long long>(B) * Hkv * pl->groups;
+  int ns = static_cast<int>((static_cast<long long>(sm_count()) * 4 + units - 1) / units);
+  if (ns > tiles) ns = tiles;
+  if (ns < 1) ns = 1;
+  if (ns > 64) ns = 64;
+  ns = attn_env_int("MSD_ATTN_SPLITS", ns);
+  if (ns < 1) ns = 1;
+  pl->n_splits = ns;
+  pl->smem_bytes = static_cast<size_t>(pl->stages) * kv_stage + static_cast<size_t>(pl->DC) * pl->Rp * kChunk + pl->Rp * kChunk + 1024;
+  int cols = 32;
+  while (cols < 2 * pl->Rp + pl->DVT * pl->Rp) cols <<= 1;
+  pl->tmem_cols = cols;
+  pl->ws_bytes = round_up(static_cast<size_t>(B) * Hq * ns * (Dv + 2) * sizeof(float), 1024);
+  return pl->smem_bytes <= 227 * 1024 - 2048;
+}
+
+}  // namespace msd
+
+extern "C" {
+
+size_t msd_attn_decode_int8kv_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen) {
+  msd::AttnPlan pl;
+  if (!msd::plan_attn(B, Hq, Hkv, D, Dv, max_seqlen, false, &pl)) return 0;
+  return pl.ws_bytes;
+}
+
+msd_status_t msd_attn_decode_schedule(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen,
+                                      int32_t* tile, int32_t* n_splits) {
+  msd::AttnPlan pl;
+  if (!tile || !n_splits) return MSD_ERR_NULL_POINTER;
+  if (!msd::plan_attn(B, Hq, Hkv, D, Dv, max_seqlen, false, &pl)) return MSD_ERR_BAD_SHAPE;
+  *tile = msd::kTok;
+  *n_splits = pl.n_splits;
+  return MSD_OK;
+}
+
+msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, const int8_t* v_cache,
+                                    const float* k_scale, const float* v_scale, const int32_t* cu_seqlens,
+                                    int64_t total_tokens, int32_t max_seqlen, int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
+                                    float softmax_scale, void* out_bf16, float* lse, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
+  using namespace msd;
+  if (B < 0 || max_seqlen < 0 || total_tokens < 0 || total_tokens > 0x7FFFFFFF) return MSD_ERR_BAD_SHAPE;
+  if (B == 0) return MSD_OK;
+  AttnPlan pl;
+  if (!plan_attn(B, Hq, Hkv, D, Dv, max_seqlen > 0 ? max_seqlen : 1, v_cache == nullptr, &pl)) return MSD_ERR_BAD_SHAPE;
+  if (!q_bf16 || !k_cache || !k_scale || !cu_seqlens || !out_bf16 || !workspace) return MSD_ERR_NULL_POINTER;
+  if (!aligned(q_bf16, 16) || !aligned(k_cache, 16) || (v_cache && !aligned(v_cache, 16)) || !aligned(out_bf16, 16) ||
+      !aligned(workspace, 1024))
+    return MSD_ERR_BAD_ALIGNMENT;
+  if (workspace_bytes < pl.ws_bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
+  unsigned* status = device_status_ptr();
+  if (!status) return MSD_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+  // The tensor maps end at total_tokens: a tile that runs past the cache is zero-filled instead of read.
+  const uint64_t T_extent = static_cast<uint64_t>(total_tokens > 0 ? total_tokens : 1);
+  CUtensorMap tmap_k, tmap_v;
+  if (!encode_tmap_3d(&tmap_k, CU_TENSOR_MAP_DATA_TYPE_UINT8, k_cache, D, Hkv, T_extent, D, static_cast<uint64_t>(Hkv) * D,
+                      kChunk, 1, kTok, CU_TENSOR_MAP_SWIZZLE_128B))
+    return MSD_ERR_CUDA;
+  const void* vbase = v_cache ? static_cast<const void*>(v_cache) : static_cast<const void*>(k_cache);
+  const int vD = v_cache ? Dv : D;
+  if (!encode_tmap_3d(&tmap_v, CU_TENSOR_MAP_DATA_TYPE_UINT8, vbase, vD, Hkv, T_extent, vD, static_cast<uint64_t>(Hkv) * vD,
+                      kChunk, 1, kTok, CU_TENSOR_MAP_SWIZZLE_128B))
+    return MSD_ERR_CUDA;
+
+  AttnParams p;
+  p.q = static_cast<const uint16_t*>(q_bf16);
+  p.k_scale = k_scale;
+  p.v_scale = v_scale ? v_scale : k_scale;
+  p.cu = cu_seqlens;
+  p.partial = static_cast<float*>(workspace);
+  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.Dv = Dv; p.G = Hq / Hkv;
+  p.HG = pl.HG; p.Rp = pl.Rp; p.groups = pl.groups; p.DC = pl.DC; p.DVT = pl.DVT;
+  p.n_splits = pl.n_splits; p.stages = pl.stages; p.v_alias = pl.v_alias; p.tmem_cols = pl.tmem_cols;
+  p.scale = softmax_scale;
+  p.status = status;
+
+  void (*kernel)(CUtensorMap, CUtensorMap, AttnParams) = nullptr;
+  if (pl.HG == 8) kernel = (pl.DVT == 1) ? attn_decode_kernel<8, 1> : (pl.DVT == 2) ? attn_decode_kernel<8, 2> : attn_decode_kernel<8, 4>;
+  else kernel = (pl.DVT == 1) ? attn_decode_kernel<16, 1> : (pl.DVT == 2) ? attn_decode_kernel<16, 2> : attn_decode_kernel<16, 4>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
+    return MSD_ERR_CUDA;
+  dim3 grid(pl.n_splits, B * Hkv * pl.groups);
+  kernel<<<grid, kAttnThreads, pl.smem_bytes, s>>>(tmap_k, tmap_v, p);
+  if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
+  attn_combine_kernel<<<B * Hq, 128, 0, s>>>(p.partial, pl.n_splits, Dv, static_cast<__nv_bfloat16*>(out_bf16), lse);
+  return launch_status();
+}
+
+}  // extern "C"

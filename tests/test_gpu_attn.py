@@ -1,0 +1,129 @@
+"""GPU parity: INT8-KV decode attention against the CPU oracle's tiled mode (which mirrors the kernel's tile and
+split schedule), within 1e-3 of the row L2 norm; plus the accuracy ordering against the dequantize-to-BF16 path."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_13915_b200 import binding, inputs
+from helpers import bf16_dev, bf16_bits, dev, rel_row_err
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-3
+
+
+def _split_starts(seqlens, tile, ns):
+    L = np.asarray(seqlens, dtype=np.int64)
+    per = -(-L // ns)
+    lsplit = -(-per // tile) * tile
+    return np.minimum(L[:, None], np.arange(ns + 1)[None, :] * lsplit[:, None]).astype(np.int32)
+
+
+def _run_gpu(c, want_lse=True):
+    B, Hq, D = c.q.shape
+    Hkv = c.k.shape[1]
+    q = bf16_dev(c.q)
+    k = dev(c.k)
+    v = None if c.v is None else dev(c.v)
+    ks = dev(c.k_scale)
+    vs = None if c.v_scale is None else dev(c.v_scale)
+    cu = dev(c.cu_seqlens)
+    out = binding.attn_decode_int8kv(q, k, v, ks, vs, cu, max(c.max_seqlen, 1), c.softmax_scale, dv=c.dv, want_lse=want_lse)
+    torch.cuda.synchronize()
+    binding.last_device_status()
+    return out
+
+
+def _oracle_tiled(c, B_sched=None, max_seqlen=None):
+    B, Hq, D = c.q.shape
+    Hkv = c.k.shape[1]
+    tile, ns = binding.attn_decode_schedule(B_sched or B, Hq, Hkv, D, c.dv, max(max_seqlen or c.max_seqlen, 1))
+    ss = _split_starts(np.diff(c.cu_seqlens), tile, ns)
+    return oracle.attn_decode_int8kv(c.q, c.k, c.v, c.k_scale, c.v_scale, c.cu_seqlens, c.softmax_scale, dv=c.dv,
+                                     mode="tiled", tile=tile, split_starts=ss, want_lse=True)
+
+
+def _check(c):
+    o, lse = _run_gpu(c)
+    ref, lse_ref = _oracle_tiled(c)
+    got = oracle.bf16_bits_to_f64(bf16_bits(o))
+    err = rel_row_err(got, ref)
+    assert err.max() <= TOL, err.max()
+    live = np.isfinite(lse_ref)
+    assert np.allclose(lse.cpu().numpy()[live], lse_ref[live], rtol=0, atol=2e-3)
+    assert np.all(np.isneginf(lse.cpu().numpy()[~live]))
+    return got, ref
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,seqlens", [
+    (1, 4, 1, [128]), (3, 8, 2, [700, 64, 1500]), (2, 32, 8, [129, 4000]), (4, 8, 8, [1, 127, 0, 300]),
+    (2, 32, 2, [513, 2222]), (1, 24, 2, [999]),
+])
+def test_gqa_parity(B, Hq, Hkv, seqlens):
+    _check(inputs.gqa_case(B, Hq, Hkv, 128, seqlens, seed=B + Hq))
+
+
+@pytest.mark.parametrize("seqlens", [[300, 1000], [16384 // 8]])
+def test_mla_parity(seqlens):
+    _check(inputs.mla_case(len(seqlens), 64, 576, 512, seqlens, seed=11))
+
+
+def test_other_head_dims():
+    c = inputs.gqa_case(2, 8, 2, 64, [400, 77], seed=5)          # D = Dv = 64: half-filled chunk
+    _check(c)
+    c = inputs.gqa_case(2, 4, 2, 256, [300, 640], seed=6)        # two chunks of D and Dv
+    _check(c)
+
+
+@pytest.mark.parametrize("splits", ["1", "2", "7"])
+def test_split_counts(splits, monkeypatch):
+    monkeypatch.setenv("MSD_ATTN_SPLITS", splits)
+    _check(inputs.gqa_case(2, 8, 2, 128, [1000, 3000], seed=9))
+
+
+def test_accuracy_ordering_vs_dequant():
+    c = inputs.gqa_case(4, 32, 8, 128, [2048, 3000, 4096, 777], seed=1)
+    o = _run_gpu(c, want_lse=False)
+    got = oracle.bf16_bits_to_f64(bf16_bits(o))
+    args = (c.q, c.k, c.v, c.k_scale, c.v_scale, c.cu_seqlens, c.softmax_scale)
+    ref = oracle.attn_decode_int8kv(*args, mode="ref")
+    deq = oracle.bf16_bits_to_f64(oracle.round_bf16(oracle.attn_decode_int8kv(*args, mode="dequant")))
+    n = np.linalg.norm(ref)
+    assert np.linalg.norm(got - ref) / n <= np.linalg.norm(deq - ref) / n
+    # distance to the untiled definition (global softmax maximum) stays inside the same budget
+    glob = oracle.attn_decode_int8kv(*args, mode="global")
+    assert rel_row_err(got, glob).max() <= TOL
+
+
+def _subcase(c, seqs):
+    """The sub-problem made of the listed sequences only (all heads)."""
+    cu = c.cu_seqlens
+    tok = np.concatenate([np.arange(cu[b], cu[b + 1]) for b in seqs])
+    L = [int(cu[b + 1] - cu[b]) for b in seqs]
+    ncu = np.zeros(len(seqs) + 1, np.int32)
+    ncu[1:] = np.cumsum(L)
+    return inputs.AttnCase(c.q[seqs], c.k[tok], None if c.v is None else c.v[tok], c.k_scale[tok],
+                           None if c.v_scale is None else c.v_scale[tok], ncu, c.dv, c.softmax_scale)
+
+
+def test_gqa_full_size_sampled_sequences():
+    """BASELINE config 3 in the benchmark's launch configuration; the oracle recomputes three sequences."""
+    B, Hq, Hkv, D = 32, 32, 8, 128
+    c = inputs.gqa_case(B, Hq, Hkv, D, inputs.seqlens_uniform(B, 2048, 8192, seed=0), seed=0)
+    o = _run_gpu(c, want_lse=False)
+    got = oracle.bf16_bits_to_f64(bf16_bits(o))
+    seqs = [0, 17, 31]
+    sub = _subcase(c, seqs)
+    ref, _ = _oracle_tiled(sub, B_sched=B, max_seqlen=c.max_seqlen)
+    assert rel_row_err(got[seqs], ref).max() <= TOL
+
+
+def test_mla_full_size_sampled_sequence():
+    """BASELINE config 4 (B=64, 64 heads, d=576/512, 16384 tokens); the oracle recomputes one sequence."""
+    B, Hq, D, Dv, L = 64, 64, 576, 512, 16384
+    c = inputs.mla_case(B, Hq, D, Dv, [L] * B, seed=0)
+    o = _run_gpu(c, want_lse=False)
+    got = oracle.bf16_bits_to_f64(bf16_bits(o))
+    sub = _subcase(c, [37])
+    ref, _ = _oracle_tiled(sub, B_sched=B, max_seqlen=L)
+    assert rel_row_err(got[[37]], ref).max() <= TOL
