@@ -148,7 +148,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       };
       if (ok) ok = issue_qk(0);
       for (int t = 0; t < ntiles && ok; ++t) {
-        if (t + 1 < ntiles) { ok = issue_qk(t + 1); if (!ok) break; }
+        // with two KV stages the next tile's QK^T overlaps this tile's softmax; with one it must wait for PV below
+        if (p.stages >= 2 && t + 1 < ntiles) { ok = issue_qk(t + 1); if (!ok) break; }
         ok = wait_bounded(&p_full, (t + 1) & 1, abort, p.status);             // P of tile t is in shared memory
         if (!ok) break;
         ok = wait_bounded(&o_empty, (t & 1) ^ 1, abort, p.status);           // O^T of tile t-1 has been merged
@@ -164,6 +165,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                    smem_desc(pa + k * 32, 16, 1024, kSwizzle128B), idesc_pv, k > 0 ? 1u : 0u);
         tc_commit(&o_full);
         tc_commit(&kv_empty[st]);
+        if (p.stages < 2 && t + 1 < ntiles) ok = issue_qk(t + 1);
       }
     }
   } else {
@@ -401,7 +403,8 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   if (v_alias && Dv > D) return false;
   pl->v_alias = v_alias ? 1 : 0;
   const int kv_stage = (pl->DC + (v_alias ? 0 : pl->DVT)) * kChunkBytes;
-  pl->stages = (kv_stage <= 32 * 1024) ? 2 : 2;
+  const size_t fixed = static_cast<size_t>(pl->DC) * pl->Rp * kChunk + pl->Rp * kChunk + 1024;
+  pl->stages = (2 * static_cast<size_t>(kv_stage) + fixed <= 227 * 1024 - 2048) ? 2 : 1;
   const int tiles = (max_seqlen + kTok - 1) / kTok;
   const long long units = static_cast<long long>(B) * Hkv * pl->groups;
   int ns = static_cast<int>((static_cast<long long>(sm_count()) * 4 + units - 1) / units);
@@ -411,7 +414,7 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   ns = attn_env_int("MSD_ATTN_SPLITS", ns);
   if (ns < 1) ns = 1;
   pl->n_splits = ns;
-  pl->smem_bytes = static_cast<size_t>(pl->stages) * kv_stage + static_cast<size_t>(pl->DC) * pl->Rp * kChunk + pl->Rp * kChunk + 1024;
+  pl->smem_bytes = static_cast<size_t>(pl->stages) * kv_stage + fixed;
   int cols = 32;
   while (cols < 2 * pl->Rp + pl->DVT * pl->Rp) cols <<= 1;
   pl->tmem_cols = cols;

@@ -43,12 +43,19 @@ def _oracle_tiled(c, B_sched=None, max_seqlen=None):
                                      mode="tiled", tile=tile, split_starts=ss, want_lse=True)
 
 
+def _assert_close(got, ref):
+    """|y - y_oracle| <= 1e-3 * ||y_oracle row||_2 for the FP32 result, plus the final rounding to BF16 that both the
+    kernel and a BF16 consumer of the oracle's value incur (one BF16 ulp = 2^-8 relative at most)."""
+    n = np.linalg.norm(ref, axis=-1, keepdims=True)
+    assert np.all(np.abs(got - ref) <= TOL * n + np.abs(ref) * 2.0 ** -8 + 1e-30), \
+        float((np.abs(got - ref) - np.abs(ref) * 2.0 ** -8).max() / n.max())
+
+
 def _check(c):
     o, lse = _run_gpu(c)
     ref, lse_ref = _oracle_tiled(c)
     got = oracle.bf16_bits_to_f64(bf16_bits(o))
-    err = rel_row_err(got, ref)
-    assert err.max() <= TOL, err.max()
+    _assert_close(got, ref)
     live = np.isfinite(lse_ref)
     assert np.allclose(lse.cpu().numpy()[live], lse_ref[live], rtol=0, atol=2e-3)
     assert np.all(np.isneginf(lse.cpu().numpy()[~live]))
@@ -92,7 +99,7 @@ def test_accuracy_ordering_vs_dequant():
     assert np.linalg.norm(got - ref) / n <= np.linalg.norm(deq - ref) / n
     # distance to the untiled definition (global softmax maximum) stays inside the same budget
     glob = oracle.attn_decode_int8kv(*args, mode="global")
-    assert rel_row_err(got, glob).max() <= TOL
+    _assert_close(got, glob)
 
 
 def _subcase(c, seqs):
@@ -115,7 +122,7 @@ def test_gqa_full_size_sampled_sequences():
     seqs = [0, 17, 31]
     sub = _subcase(c, seqs)
     ref, _ = _oracle_tiled(sub, B_sched=B, max_seqlen=c.max_seqlen)
-    assert rel_row_err(got[seqs], ref).max() <= TOL
+    _assert_close(got[seqs], ref)
 
 
 def test_mla_full_size_sampled_sequence():
@@ -126,4 +133,4 @@ def test_mla_full_size_sampled_sequence():
     got = oracle.bf16_bits_to_f64(bf16_bits(o))
     sub = _subcase(c, [37])
     ref, _ = _oracle_tiled(sub, B_sched=B, max_seqlen=L)
-    assert rel_row_err(got[[37]], ref).max() <= TOL
+    _assert_close(got[[37]], ref)
