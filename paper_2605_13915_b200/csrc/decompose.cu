@@ -122,7 +122,7 @@ __device__ __forceinline__ float pow2f(int e) { return __uint_as_float(static_ca
 
 __global__ void __launch_bounds__(kMxThreads)
 decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, int K, uint8_t* __restrict__ q1,
-                       uint8_t* __restrict__ q2, uint8_t* __restrict__ e1, uint8_t* __restrict__ e2) {
+                       uint8_t* __restrict__ q2, uint8_t* __restrict__ e1, uint8_t* __restrict__ e2, int sf_kgroups) {
   pdl_launch_dependents();
   const int kblocks = K >> 5;
   const int64_t nblocks = M * kblocks;
@@ -169,8 +169,13 @@ decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, i
     }
     *reinterpret_cast<uint4*>(q1 + row * (K >> 1) + kb * 16) = make_uint4(o1[0], o1[1], o1[2], o1[3]);
     *reinterpret_cast<uint4*>(q2 + row * (K >> 1) + kb * 16) = make_uint4(o2[0], o2[1], o2[2], o2[3]);
-    e1[row * kblocks + kb] = static_cast<uint8_t>(a + 127);
-    e2[row * kblocks + kb] = static_cast<uint8_t>(bexp + 127);
+    // sf_kgroups == 0: row-major [M, K/32]; otherwise the 512-byte blocks (128 rows x 4 scales) the block-scaled
+    // MMA's shared-memory -> TMEM scale copy expects: block (row/128, kb/4), byte (row%32)*16 + ((row/32)%4)*4 + kb%4
+    const int64_t so = sf_kgroups == 0
+                           ? row * kblocks + kb
+                           : ((row >> 7) * sf_kgroups + (kb >> 2)) * 512 + (row & 31) * 16 + ((row >> 5) & 3) * 4 + (kb & 3);
+    e1[so] = static_cast<uint8_t>(a + 127);
+    e2[so] = static_cast<uint8_t>(bexp + 127);
   }
 }
 
@@ -183,14 +188,14 @@ msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int
 }
 
 msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
-                                    uint8_t* e1, uint8_t* e2, cudaStream_t stream) {
+                                    uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream) {
   if (M == 0) return MSD_OK;
   const int64_t nblocks = M * (K >> 5);
   const int64_t want = (nblocks + kMxThreads - 1) / kMxThreads;
   const int64_t cap = static_cast<int64_t>(sm_count()) * 32;
   const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
   decompose_mxfp4_kernel<<<grid, kMxThreads, 0, stream>>>(static_cast<const uint16_t*>(x_bf16), ldx, M,
-                                                          static_cast<int>(K), q1, q2, e1, e2);
+                                                          static_cast<int>(K), q1, q2, e1, e2, sf_kgroups);
   return launch_status();
 }
 
@@ -215,7 +220,7 @@ msd_status_t msd_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64
   if (M == 0) return MSD_OK;
   if (!x_bf16 || !q1 || !q2 || !e8m0_1 || !e8m0_2) return MSD_ERR_NULL_POINTER;
   if (!msd::aligned(x_bf16, 16) || !msd::aligned(q1, 16) || !msd::aligned(q2, 16)) return MSD_ERR_BAD_ALIGNMENT;
-  return msd::launch_decompose_mxfp4(x_bf16, M, K, ldx, q1, q2, e8m0_1, e8m0_2, static_cast<cudaStream_t>(stream));
+  return msd::launch_decompose_mxfp4(x_bf16, M, K, ldx, q1, q2, e8m0_1, e8m0_2, 0, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

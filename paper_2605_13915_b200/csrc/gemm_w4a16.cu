@@ -1,0 +1,299 @@
+// W4A16 MSD linear layer (Sec. 3.2.1, Alg. 2; Tab. mxfp4-compute): both MXFP4 components of the activation are
+// multiplied against the MXFP4 weight by block-scaled FP4 MMAs (tcgen05.mma kind::mxf4, E8M0 scale per 32 K) that
+// accumulate into the SAME FP32 tile in TMEM, so the "one add" of the two passes costs nothing and each weight tile
+// is read once for both passes.
+//
+// Tile: 128 activation rows x 256 weight rows, K walked in stages of 256 elements (128 packed bytes = one 128-byte
+// swizzle row).  Per stage TMA brings the A1, A2 (128 x 128 B) and B (256 x 128 B) tiles, bulk copies bring the scale
+// blocks (512-byte blocks of 128 rows x 4 scales, the layout the shared-memory -> TMEM scale copy expects), the MMA
+// warp copies the scales into TMEM and issues 4 K-steps x 2 passes.  Persistent CTAs walk the tiles with the
+// activation-row index fastest so that concurrent CTAs share weight tiles in L2.
+//
+// Warps: 0 = producer, 1 = MMA issuer + TMEM owner, 2..5 = epilogue (FP32 -> BF16/FP32, row-major stores).
+#include <cuda_bf16.h>
+
+#include <cstdlib>
+
+#include "host_common.h"
+#include "sm100.cuh"
+
+namespace msd {
+
+constexpr int kW4TileM = 128;
+constexpr int kW4TileN = 256;
+constexpr int kW4BlockK = 256;                                  // elements per stage (128 packed bytes)
+constexpr int kW4Threads = 192;
+constexpr int kW4ABytes = kW4TileM * 128;                       // 16 KB
+constexpr int kW4BBytes = kW4TileN * 128;                       // 32 KB
+constexpr int kW4SfBytes = 1024 + 1024 + 2048;                  // SFA1, SFA2 (2 k-groups each), SFB (2 row tiles x 2 k-groups)
+constexpr int kW4StageBytes = 2 * kW4ABytes + kW4BBytes + kW4SfBytes;   // 69632
+constexpr int kW4Stages = 3;
+constexpr int kW4TmemCols = 512;
+constexpr int kW4SfCol = 256;                                   // scale columns follow the 256 accumulator columns
+
+struct GemmW4Params {
+  int M, N, K;
+  int m_tiles, n_tiles, kstages;
+  int sf_kgroups;               // 128-element K groups per row of the blocked scale arrays (even)
+  const uint8_t* sfa1;
+  const uint8_t* sfa2;
+  const uint8_t* sfb;
+  void* y;
+  int ytype;
+  unsigned* status;
+};
+
+// Relayout of row-major E8M0 scales [rows, K/32] into 512-byte blocks (128 rows x 4 scales).
+__global__ void sf_block_layout_kernel(const uint8_t* __restrict__ src, int64_t rows, int kblocks, int sf_kgroups,
+                                       uint8_t* __restrict__ dst) {
+  const int64_t total = rows * kblocks;
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t row = i / kblocks;
+    const int kb = static_cast<int>(i - row * kblocks);
+    dst[((row >> 7) * sf_kgroups + (kb >> 2)) * 512 + (row & 31) * 16 + ((row >> 5) & 3) * 4 + (kb & 3)] = src[i];
+  }
+}
+
+__global__ void __launch_bounds__(kW4Threads, 1)
+gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
+                  const __grid_constant__ CUtensorMap tmap_b, const GemmW4Params p) {
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ __align__(8) uint64_t full_bar[kW4Stages], empty_bar[kW4Stages], tfull_bar, tempty_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kW4Stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    mbar_init(&tfull_bar, 1);
+    mbar_init(&tempty_bar, 4);
+    abort_flag = 0;
+    mbar_init_fence();
+    tma_prefetch_desc(&tmap_a1);
+    tma_prefetch_desc(&tmap_a2);
+    tma_prefetch_desc(&tmap_b);
+  }
+  if (warp == 1) tmem_alloc(&tmem_base_slot, kW4TmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  volatile int* abort = &abort_flag;
+  const int total_tiles = p.m_tiles * p.n_tiles;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      pdl_wait_primary();           // components and blocked scales come from the kernels launched just before
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+        for (int ks = 0; ks < p.kstages; ++ks) {
+          ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&full_bar[stage], kW4StageBytes);
+          uint8_t* dst = smem + stage * kW4StageBytes;
+          tma_load_2d(dst, &tmap_a1, ks * 128, mt * kW4TileM, &full_bar[stage]);
+          tma_load_2d(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, &full_bar[stage]);
+          tma_load_2d(dst + 2 * kW4ABytes, &tmap_b, ks * 128, nt * kW4TileN, &full_bar[stage]);
+          uint8_t* sf = dst + 2 * kW4ABytes + kW4BBytes;
+          const size_t a_off = (static_cast<size_t>(mt) * p.sf_kgroups + 2 * ks) * 512;
+          bulk_load(sf, p.sfa1 + a_off, 1024, &full_bar[stage]);
+          bulk_load(sf + 1024, p.sfa2 + a_off, 1024, &full_bar[stage]);
+          bulk_load(sf + 2048, p.sfb + (static_cast<size_t>(2 * nt) * p.sf_kgroups + 2 * ks) * 512, 1024, &full_bar[stage]);
+          bulk_load(sf + 3072, p.sfb + (static_cast<size_t>(2 * nt + 1) * p.sf_kgroups + 2 * ks) * 512, 1024, &full_bar[stage]);
+          if (++stage == kW4Stages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      const uint32_t sfa1_t = tmem_base + kW4SfCol;          // 2 k-groups x 4 columns
+      const uint32_t sfa2_t = tmem_base + kW4SfCol + 8;
+      const uint32_t sfb_t = tmem_base + kW4SfCol + 16;      // 2 k-groups x 8 columns (256 weight rows)
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+        ok = wait_bounded(&tempty_bar, (it & 1) ^ 1, abort, p.status);      // epilogue has drained the accumulator
+        if (!ok) break;
+        tc_fence_after();
+        for (int ks = 0; ks < p.kstages; ++ks) {
+          ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t base = smem_u32(smem + stage * kW4StageBytes);
+          const uint32_t a1 = base, a2 = base + kW4ABytes, bb = base + 2 * kW4ABytes, sf = bb + kW4BBytes;
+          // scale blocks: 32 rows x 16 bytes each, eight-row groups 128 bytes apart, no swizzle
+          for (int g = 0; g < 2; ++g) {
+            tc_cp_32x128b_warpx4(sfa1_t + 4 * g, smem_desc(sf + g * 512, 0, 128, 0));
+            tc_cp_32x128b_warpx4(sfa2_t + 4 * g, smem_desc(sf + 1024 + g * 512, 0, 128, 0));
+            tc_cp_32x128b_warpx4(sfb_t + 8 * g, smem_desc(sf + 2048 + g * 512, 0, 128, 0));
+            tc_cp_32x128b_warpx4(sfb_t + 8 * g + 4, smem_desc(sf + 3072 + g * 512, 0, 128, 0));
+          }
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {                    // 64 elements (32 bytes) per MMA
+            const int g = kk >> 1;
+            const uint32_t sid = (kk & 1) * 2;                // which pair of scale bytes of the 4-scale column
+            const uint32_t idesc = idesc_block_scaled(/*E2M1*/ 1, 1, kW4TileM, kW4TileN, sid, sid);
+            const uint64_t bdesc = smem_desc(bb + kk * 32, 16, 1024, kSwizzle128B);
+            mma_mxf4(tmem_base, smem_desc(a1 + kk * 32, 16, 1024, kSwizzle128B), bdesc, idesc, sfa1_t + 4 * g,
+                     sfb_t + 8 * g, (ks > 0 || kk > 0) ? 1u : 0u);
+            mma_mxf4(tmem_base, smem_desc(a2 + kk * 32, 16, 1024, kSwizzle128B), bdesc, idesc, sfa2_t + 4 * g,
+                     sfb_t + 8 * g, 1u);
+          }
+          tc_commit(&empty_bar[stage]);
+          if (++stage == kW4Stages) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        tc_commit(&tfull_bar);
+      }
+    }
+  } else {
+    const int quad = warp & 3;
+    const int r = quad * 32 + lane;
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+      const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+      ok = wait_bounded(&tfull_bar, it & 1, abort, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      const int row = mt * kW4TileM + r;
+      const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+      for (int c0 = 0; c0 < kW4TileN; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld16(trow + c0, v);
+        tmem_ld_wait();
+        const int col = nt * kW4TileN + c0;
+        if (row < p.M && col < p.N) {
+          if (p.ytype == MSD_OUT_BF16) {
+            uint32_t o[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+              o[j] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.y) + static_cast<long long>(row) * p.N + col;
+            if (col + 16 <= p.N) {
+              reinterpret_cast<uint4*>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
+              reinterpret_cast<uint4*>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+            } else {
+              for (int j = 0; j < 16 && col + j < p.N; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+            }
+          } else {
+            float* dst = static_cast<float*>(p.y) + static_cast<long long>(row) * p.N + col;
+            for (int j = 0; j < 16 && col + j < p.N; ++j) dst[j] = __uint_as_float(v[j]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty_bar);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kW4TmemCols);
+  }
+}
+
+struct GemmW4Plan {
+  int m_tiles, n_tiles, kstages, sf_kgroups, grid;
+  size_t off_q1, off_q2, off_sfa1, off_sfa2, off_sfb, bytes;
+};
+
+static GemmW4Plan plan_w4(int64_t M, int64_t N, int64_t K) {
+  GemmW4Plan pl;
+  pl.m_tiles = static_cast<int>((M + kW4TileM - 1) / kW4TileM);
+  pl.n_tiles = static_cast<int>((N + kW4TileN - 1) / kW4TileN);
+  pl.kstages = static_cast<int>((K + kW4BlockK - 1) / kW4BlockK);
+  pl.sf_kgroups = 2 * pl.kstages;
+  const int tiles = pl.m_tiles * pl.n_tiles;
+  int grid = sm_count();
+  if (grid > tiles) grid = tiles;
+  pl.grid = grid;
+  size_t off = 0;
+  pl.off_q1 = off;   off = round_up(off + static_cast<size_t>(M) * (K / 2), 1024);
+  pl.off_q2 = off;   off = round_up(off + static_cast<size_t>(M) * (K / 2), 1024);
+  pl.off_sfa1 = off; off = round_up(off + static_cast<size_t>(pl.m_tiles) * pl.sf_kgroups * 512, 1024);
+  pl.off_sfa2 = off; off = round_up(off + static_cast<size_t>(pl.m_tiles) * pl.sf_kgroups * 512, 1024);
+  pl.off_sfb = off;  off = round_up(off + static_cast<size_t>(2 * pl.n_tiles) * pl.sf_kgroups * 512, 1024);
+  pl.bytes = off;
+  return pl;
+}
+
+}  // namespace msd
+
+extern "C" {
+
+size_t msd_gemm_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  if (M < 1 || N < 1 || K < 128 || K % 128 != 0) return 0;
+  return msd::plan_w4(M, N, K).bytes;
+}
+
+msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0, int64_t M, int64_t N,
+                            int64_t K, void* y, msd_out_t ytype, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+  using namespace msd;
+  if (M < 1 || N < 1 || K < 128 || K % 128 != 0 || N % 8 != 0 || M > (1 << 24) || N > (1 << 24) || K > (1 << 24))
+    return MSD_ERR_BAD_SHAPE;
+  if (ytype != MSD_OUT_BF16 && ytype != MSD_OUT_FP32) return MSD_ERR_UNSUPPORTED;
+  if (!x_bf16 || !w_fp4 || !w_e8m0 || !y || !workspace) return MSD_ERR_NULL_POINTER;
+  if (!aligned(x_bf16, 16) || !aligned(w_fp4, 16) || !aligned(y, 16) || !aligned(workspace, 1024)) return MSD_ERR_BAD_ALIGNMENT;
+  const GemmW4Plan pl = plan_w4(M, N, K);
+  if (workspace_bytes < pl.bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
+  unsigned* status = device_status_ptr();
+  if (!status) return MSD_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  uint8_t* q1 = ws + pl.off_q1;
+  uint8_t* q2 = ws + pl.off_q2;
+
+  // weight scales into the blocked layout (padding entries keep the workspace's zero fill: scale 2^-127 on zero data)
+  {
+    const int64_t total = N * (K / 32);
+    const int threads = 256;
+    int64_t blocks = (total + threads - 1) / threads;
+    const int64_t cap = static_cast<int64_t>(sm_count()) * 16;
+    if (blocks > cap) blocks = cap;
+    sf_block_layout_kernel<<<static_cast<unsigned>(blocks), threads, 0, s>>>(w_e8m0, N, static_cast<int>(K / 32), pl.sf_kgroups,
+                                                                            ws + pl.off_sfb);
+    if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
+  }
+  msd_status_t st = launch_decompose_mxfp4(x_bf16, M, K, K, q1, q2, ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s);
+  if (st != MSD_OK) return st;
+
+  CUtensorMap tmap_a1, tmap_a2, tmap_b;
+  const uint64_t kb = static_cast<uint64_t>(K / 2);
+  if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, kb, M, kb, 128, kW4TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, q2, kb, M, kb, 128, kW4TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, w_fp4, kb, N, kb, 128, kW4TileN, CU_TENSOR_MAP_SWIZZLE_128B))
+    return MSD_ERR_CUDA;
+
+  GemmW4Params p;
+  p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+  p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.kstages = pl.kstages; p.sf_kgroups = pl.sf_kgroups;
+  p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
+  p.y = y; p.ytype = ytype; p.status = status;
+
+  const size_t smem_bytes = static_cast<size_t>(kW4Stages) * kW4StageBytes + 1024;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(gemm_w4a16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes)) != cudaSuccess)
+      return MSD_ERR_CUDA;
+    attr_done = true;
+  }
+  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+  if (launch_pdl(gemm_w4a16_kernel, dim3(pl.grid), dim3(kW4Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, p) != cudaSuccess)
+    return MSD_ERR_CUDA;
+  return MSD_OK;
+}
+
+}  // extern "C"

@@ -49,6 +49,6 @@ cudaError_t launch_pdl(void (*kernel)(Args...), dim3 grid, dim3 block, size_t sm
 msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
                                    float* alpha, float* beta, cudaStream_t stream);
 msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
-                                    uint8_t* e1, uint8_t* e2, cudaStream_t stream);
+                                    uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream);
 
 }  // namespace msd

@@ -6,7 +6,4 @@ extern "C" {
 size_t msd_gemm_dequant_bf16_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
 msd_status_t msd_gemm_dequant_bf16(const void*, const int8_t*, const float*, int64_t, int64_t, int64_t, void*, msd_out_t,
                                    void*, size_t, void*) { return MSD_ERR_UNSUPPORTED; }
-size_t msd_gemm_w4a16_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
-msd_status_t msd_gemm_w4a16(const void*, const uint8_t*, const uint8_t*, int64_t, int64_t, int64_t, void*, msd_out_t,
-                            void*, size_t, void*) { return MSD_ERR_UNSUPPORTED; }
 }  // extern "C"
