@@ -72,6 +72,10 @@ __device__ __forceinline__ void store_out(const GemmW8Params& p, int i, int n, f
   }
 }
 
+// kBase = false: the MSD path (INT8 x INT8 -> INT32, stacked components, scale-combine epilogue).
+// kBase = true : the comparison path the method replaces - the same pipeline on BF16 weights that a preceding kernel
+//                dequantized into the workspace, BF16 x BF16 -> FP32, no decomposition and no scales in the epilogue.
+template <bool kBase>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_w2,
                   const __grid_constant__ CUtensorMap tmap_x, const GemmW8Params p) {
@@ -151,6 +155,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       // Weight tiles of the first stages do not depend on the decomposition kernel: issue them before waiting for it.
       const long long nblk = blk_end - blk_begin;
       const int pre = static_cast<int>(nblk < p.num_stages ? nblk : p.num_stages);
+      if constexpr (kBase) pdl_wait_primary();     // here the weights themselves come from the preceding kernel
       for (int i = 0; i < pre; ++i) {
         const long long blk = blk_begin + i;
         const int tile = static_cast<int>(blk / p.kblocks), kb = static_cast<int>((blk + kb_rot) % p.kblocks);
@@ -187,7 +192,8 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
-      const uint32_t idesc = idesc_dense(/*D=S32*/ 2, /*A=S8*/ 1, /*B=S8*/ 1, 0, 0, kTileN, p.NB);
+      const uint32_t idesc = kBase ? idesc_dense(/*D=F32*/ 1, /*A=BF16*/ 1, /*B=BF16*/ 1, 0, 0, kTileN, p.NB)
+                                   : idesc_dense(/*D=S32*/ 2, /*A=S8*/ 1, /*B=S8*/ 1, 0, 0, kTileN, p.NB);
       int stage = 0;
       uint32_t phase = 0;
       int seg = 0;
@@ -213,7 +219,8 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
           for (int k = 0; k < kBlockK / 32; ++k) {
             const uint64_t adesc = smem_desc(wa + k * 32, 16, 1024, kSwizzle128B);
             const uint64_t bdesc = smem_desc(xa + k * 32, 16, 1024, kSwizzle128B);
-            mma_i8(d_tmem, adesc, bdesc, idesc, (b > blk || k > 0) ? 1u : 0u);
+            if constexpr (kBase) mma_f16(d_tmem, adesc, bdesc, idesc, (b > blk || k > 0) ? 1u : 0u);
+            else mma_i8(d_tmem, adesc, bdesc, idesc, (b > blk || k > 0) ? 1u : 0u);
           }
           tc_commit(&empty_bar[stage]);          // frees the stage once these MMAs have read it
           if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
@@ -230,10 +237,12 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     const int quad = warp & 3;                    // TMEM lane group this warp may read
     const int r = quad * 32 + lane;               // weight row within the tile == TMEM lane
     const int et = threadIdx.x - 64;              // 0..127
-    pdl_wait_primary();
-    if (et < p.M) {
-      s_alpha[et] = p.alpha[et];
-      s_beta[et] = p.beta[et];
+    if constexpr (!kBase) {
+      pdl_wait_primary();
+      if (et < p.M) {
+        s_alpha[et] = p.alpha[et];
+        s_beta[et] = p.beta[et];
+      }
     }
     named_bar_sync(1, 128);
     int seg = 0;
@@ -253,7 +262,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * p.NB;
       const int n = band_row0 + tile * kTileN + r;
       const bool row_ok = (r < band_h) && (n < p.N);
-      const float sw = row_ok ? __ldg(p.w_scale + n) : 0.0f;
+      const float sw = (!kBase && row_ok) ? __ldg(p.w_scale + n) : 0.0f;
       bool finish = complete;
       int c_lo = 0, c_hi = -1;
       if (!complete) {
@@ -285,7 +294,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         for (int c0 = 0; c0 < p.Mp; c0 += 8) {
           uint32_t a[8], b[8];
           tmem_ld8(t_row + c0, a);
-          tmem_ld8(t_row + p.Mp + c0, b);
+          if constexpr (!kBase) tmem_ld8(t_row + p.Mp + c0, b);
           tmem_ld_wait();
           for (int c = c_lo; c <= c_hi; ++c) {
             if (c == static_cast<int>(blockIdx.x)) continue;
@@ -293,8 +302,12 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             const int32_t* slot = p.slots + static_cast<long long>(sid) * p.NB * kTileN;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-              a[j] += static_cast<uint32_t>(__ldcg(slot + (c0 + j) * kTileN + r));
-              b[j] += static_cast<uint32_t>(__ldcg(slot + (p.Mp + c0 + j) * kTileN + r));
+              if constexpr (kBase) {
+                a[j] = __float_as_uint(__uint_as_float(a[j]) + __int_as_float(__ldcg(slot + (c0 + j) * kTileN + r)));
+              } else {
+                a[j] += static_cast<uint32_t>(__ldcg(slot + (c0 + j) * kTileN + r));
+                b[j] += static_cast<uint32_t>(__ldcg(slot + (p.Mp + c0 + j) * kTileN + r));
+              }
             }
           }
           if (row_ok) {
@@ -302,10 +315,14 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             for (int j = 0; j < 8; ++j) {
               const int i = c0 + j;
               if (i < p.M) {
-                const int32_t ya = static_cast<int32_t>(a[j]), yb = static_cast<int32_t>(b[j]);
-                // y = s_W * (alpha * Y1 + beta * Y2)   (Alg. 1 line 8)
-                const float v = sw * __fmaf_rn(s_alpha[i], static_cast<float>(ya), s_beta[i] * static_cast<float>(yb));
-                store_out(p, i, n, v, ya, yb);
+                if constexpr (kBase) {
+                  store_out(p, i, n, __uint_as_float(a[j]), 0, 0);
+                } else {
+                  const int32_t ya = static_cast<int32_t>(a[j]), yb = static_cast<int32_t>(b[j]);
+                  // y = s_W * (alpha * Y1 + beta * Y2)   (Alg. 1 line 8)
+                  const float v = sw * __fmaf_rn(s_alpha[i], static_cast<float>(ya), s_beta[i] * static_cast<float>(yb));
+                  store_out(p, i, n, v, ya, yb);
+                }
               }
             }
           }
@@ -351,11 +368,13 @@ static int env_int(const char* name, int fallback) {
   return atoi(e);
 }
 
-static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K) {
+// `base`: plan for the dequantize-to-BF16 comparison path (K counted in bytes of BF16, one operand row per token).
+static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   GemmW8Plan pl;
-  pl.Mp = static_cast<int>((M + 7) / 8 * 8);
-  pl.NB = 2 * pl.Mp;
-  pl.kblocks = static_cast<int>((K + kBlockK - 1) / kBlockK);
+  pl.Mp = base ? static_cast<int>((M + 15) / 16 * 16) : static_cast<int>((M + 7) / 8 * 8);
+  pl.NB = base ? pl.Mp : 2 * pl.Mp;
+  const int64_t kbytes = base ? 2 * K : K;
+  pl.kblocks = static_cast<int>((kbytes + kBlockK - 1) / kBlockK);
   pl.num_tiles = static_cast<int>((N + kTileN - 1) / kTileN);
   pl.total_blocks = static_cast<long long>(pl.kblocks) * pl.num_tiles;
   pl.groups8 = static_cast<int>((N + 7) / 8);
@@ -389,7 +408,7 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K) {
   pl.smem_bytes = static_cast<size_t>(stages) * stage_bytes + tail_pad + 1024;
   pl.tmem_cols = pow2_at_least(2 * pl.NB);
   size_t off = 0;
-  pl.off_q = off;         off = round_up(off + static_cast<size_t>(pl.NB) * K, 1024);
+  pl.off_q = off;         off = round_up(off + (base ? static_cast<size_t>(N) * K * 2 : static_cast<size_t>(pl.NB) * K), 1024);
   pl.off_alpha = off;     off = round_up(off + 128 * sizeof(float), 256);
   pl.off_beta = off;      off = round_up(off + 128 * sizeof(float), 256);
   pl.off_counters = off;  off = round_up(off + static_cast<size_t>(pl.num_tiles) * sizeof(unsigned), 1024);
@@ -397,6 +416,32 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K) {
   pl.off_slots = off;     off = round_up(off + static_cast<size_t>(256) * 2 * pl.NB * kTileN * sizeof(int32_t), 1024);
   pl.bytes = off;
   return pl;
+}
+
+// The step MSD removes (Sec. 3.1, first equation): INT8 weights -> bf16(s_W * w), written back to memory.
+__global__ void dequant_w8_to_bf16_kernel(const int8_t* __restrict__ w, const float* __restrict__ w_scale, int64_t N, int64_t K,
+                                          __nv_bfloat16* __restrict__ out) {
+  pdl_launch_dependents();
+  const int64_t chunks_per_row = K >> 4;
+  const int64_t total = N * chunks_per_row;
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t n = i / chunks_per_row;
+    const float s = __ldg(w_scale + n);
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(w) + i);
+    const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+    uint32_t o[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int b0 = static_cast<int8_t>((wv[j >> 1] >> (16 * (j & 1))) & 0xFF);
+      const int b1 = static_cast<int8_t>((wv[j >> 1] >> (16 * (j & 1) + 8)) & 0xFF);
+      const __nv_bfloat162 h = __floats2bfloat162_rn(s * static_cast<float>(b0), s * static_cast<float>(b1));
+      o[j] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    uint4* dst = reinterpret_cast<uint4*>(out) + 2 * i;
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+  }
 }
 
 static msd_status_t check_w8_args(const void* x, const void* w, const void* ws, int64_t M, int64_t N, int64_t K,
@@ -460,12 +505,68 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
 
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(gemm_w8a16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_w8a16_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
       return MSD_ERR_CUDA;
     attr_done = true;
   }
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  if (launch_pdl(gemm_w8a16_kernel, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
+  if (launch_pdl(gemm_w8a16_kernel<false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
+    return MSD_ERR_CUDA;
+  return MSD_OK;
+}
+
+size_t msd_gemm_dequant_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  if (M < 1 || M > 128 || N < 1 || K < 16) return 0;
+  return msd::plan_w8(M, N, K, true).bytes;
+}
+
+msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
+                                   int64_t K, void* y, msd_out_t ytype, void* workspace, size_t workspace_bytes,
+                                   void* stream) {
+  using namespace msd;
+  msd_status_t st = check_w8_args(x_bf16, w, w_scale, M, N, K, y, ytype, workspace);
+  if (st != MSD_OK) return st;
+  const GemmW8Plan pl = plan_w8(M, N, K, true);
+  if (workspace_bytes < pl.bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
+  unsigned* status = device_status_ptr();
+  if (!status) return MSD_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  __nv_bfloat16* wbf = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_q);
+  {
+    const int64_t total = N * (K >> 4);
+    int64_t blocks = (total + 255) / 256;
+    const int64_t cap = static_cast<int64_t>(sm_count()) * 16;
+    if (blocks > cap) blocks = cap;
+    dequant_w8_to_bf16_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(w, w_scale, N, K, wbf);
+    if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
+  }
+  CUtensorMap tmap_w, tmap_w2, tmap_x;
+  const uint64_t kb = static_cast<uint64_t>(2 * K);
+  const uint32_t box2 = (pl.mode == 1 && pl.hmax > 8) ? pl.hmax - 8 : pl.hmax;
+  if (!encode_tmap_2d(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, wbf, kb, N, kb, kBlockK, pl.hmax, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_w2, CU_TENSOR_MAP_DATA_TYPE_UINT8, wbf, kb, N, kb, kBlockK, box2, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, x_bf16, kb, M, kb, kBlockK, pl.NB, CU_TENSOR_MAP_SWIZZLE_128B))
+    return MSD_ERR_CUDA;
+  GemmW8Params p;
+  p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+  p.kb_rot_step = 0;
+  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_stage_bytes = pl.w_stage_bytes;
+  p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
+  p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
+  p.w_scale = w_scale; p.alpha = nullptr; p.beta = nullptr; p.y = y; p.acc_dbg = nullptr;
+  p.slots = reinterpret_cast<int32_t*>(ws + pl.off_slots);
+  p.counters = reinterpret_cast<unsigned*>(ws + pl.off_counters);
+  p.status = status;
+  p.trace = nullptr;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(gemm_w8a16_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
+      return MSD_ERR_CUDA;
+    attr_done = true;
+  }
+  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+  if (launch_pdl(gemm_w8a16_kernel<true>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
     return MSD_ERR_CUDA;
   return MSD_OK;
 }

@@ -115,3 +115,21 @@ def test_host_buffer_entry_point():
     torch.cuda.synchronize()
     ref = oracle.gemm_w8a16(c.x, c.w, c.w_scale, "f64")
     assert rel_row_err(oracle.bf16_bits_to_f64(bf16_bits(yh)), ref).max() <= TOL
+
+
+@pytest.mark.parametrize("M,N,K,ctas", [(16, 1024, 1024, None), (128, 640, 1536, "37"), (5, 12000, 512, None), (1, 4096, 4096, None)])
+def test_dequant_bf16_comparison_kernel(M, N, K, ctas, monkeypatch):
+    """The path MSD replaces: bf16(s_W * w) written back, then a BF16 x BF16 GEMM with FP32 accumulation."""
+    if ctas:
+        monkeypatch.setenv("MSD_GEMM_CTAS", ctas)
+    c = inputs.gemm_w8_case(M, N, K, seed=4)
+    y = binding.gemm_dequant_bf16(bf16_dev(c.x), dev(c.w), dev(c.w_scale), out_dtype=torch.float32)
+    torch.cuda.synchronize()
+    binding.last_device_status()
+    ref = oracle.gemm_dequant_bf16_w8(c.x, c.w, c.w_scale)
+    assert rel_row_err(y.cpu().numpy(), ref).max() <= TOL
+    # and it is the less accurate of the two paths against the FP64 product with the dequantized weight
+    truth = oracle.gemm_ref_w8(c.x, c.w, c.w_scale)
+    msd = binding.gemm_w8a16(bf16_dev(c.x), dev(c.w), dev(c.w_scale), out_dtype=torch.float32).cpu().numpy()
+    n = np.linalg.norm(truth)
+    assert np.linalg.norm(msd - truth) / n <= np.linalg.norm(y.cpu().numpy() - truth) / n
