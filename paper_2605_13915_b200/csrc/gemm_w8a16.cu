@@ -23,7 +23,7 @@
 namespace msd {
 
 constexpr int kTileN = 128;        // weight rows per tile (MMA M)
-constexpr int kBlockK = 128;       // K bytes per pipeline stage (one 128-byte swizzle row)
+constexpr int kBlockK = 128;       // K bytes per TMA box (one 128-byte swizzle row); a stage holds `kw` adjacent boxes
 constexpr int kMaxStages = 16;
 constexpr int kGemmThreads = 192;
 constexpr int kWStageBytes = kTileN * kBlockK;
@@ -34,7 +34,8 @@ struct GemmW8Params {
   int mode;                // 0 = stream-K over 128-row tiles, 1 = one row band per CTA
   int groups8;             // ceil(N / 8): row groups divided over the CTAs in mode 1
   int hmax;                // tallest band (box rows of tmap_w; tmap_w2 has hmax - 8)
-  int w_stage_bytes;       // shared-memory bytes reserved for the weight tile of one stage
+  int w_chunk_bytes;       // shared-memory bytes reserved for one weight box (band rows x 128 B, 1 KB granules)
+  int kw;                  // adjacent 128-byte K boxes per stage: each weight row is then read kw*128 B at a time
   int kb_rot_step;         // mode 1: CTA c starts its K loop at block (c * kb_rot_step) % kblocks
   int kblocks;             // K blocks per weight tile
   int num_tiles;
@@ -47,7 +48,7 @@ struct GemmW8Params {
   const float* beta;
   void* y;
   int32_t* acc_dbg;
-  int32_t* slots;          // [gridDim.x * 2][NB][128]
+  int32_t* accum;          // [num_tiles][NB][128] split-K meeting place, zero between calls (INT32 or FP32 bits)
   unsigned* counters;      // [num_tiles]
   unsigned* status;
   long long* trace;        // nullable diagnostic buffer: 16 clock samples per CTA
@@ -72,6 +73,59 @@ __device__ __forceinline__ void store_out(const GemmW8Params& p, int i, int n, f
   }
 }
 
+// One chunk of W accumulator columns of the final epilogue.  The sums come from TMEM (tile finished by this CTA alone)
+// or from the split-K meeting place in global memory (which is read and left zeroed for the next call).
+template <bool kBase, int W>
+__device__ __forceinline__ void epilogue_chunk(const GemmW8Params& p, uint32_t t_row, int32_t* acc_tile, int c0, int r, int n,
+                                               bool row_ok, float sw, const float* s_alpha, const float* s_beta) {
+  uint32_t a[W], b[W];
+  if (acc_tile == nullptr) {
+    tmem_ldw<W>(t_row + c0, a);
+    if constexpr (!kBase) tmem_ldw<W>(t_row + p.Mp + c0, b);
+    tmem_ld_wait();
+  } else {
+#pragma unroll
+    for (int j = 0; j < W; ++j) {
+      a[j] = static_cast<uint32_t>(__ldcg(acc_tile + (c0 + j) * kTileN + r));
+      if constexpr (!kBase) b[j] = static_cast<uint32_t>(__ldcg(acc_tile + (p.Mp + c0 + j) * kTileN + r));
+    }
+#pragma unroll
+    for (int j = 0; j < W; ++j) {
+      __stcg(acc_tile + (c0 + j) * kTileN + r, 0);
+      if constexpr (!kBase) __stcg(acc_tile + (p.Mp + c0 + j) * kTileN + r, 0);
+    }
+  }
+  if (row_ok) {
+#pragma unroll
+    for (int j = 0; j < W; ++j) {
+      const int i = c0 + j;
+      if (i < p.M) {
+        if constexpr (kBase) {
+          store_out(p, i, n, __uint_as_float(a[j]), 0, 0);
+        } else {
+          const int32_t ya = static_cast<int32_t>(a[j]), yb = static_cast<int32_t>(b[j]);
+          // y = s_W * (alpha * Y1 + beta * Y2)   (Alg. 1 line 8)
+          const float v = sw * __fmaf_rn(s_alpha[i], static_cast<float>(ya), s_beta[i] * static_cast<float>(yb));
+          store_out(p, i, n, v, ya, yb);
+        }
+      }
+    }
+  }
+}
+
+// Adds W accumulator columns of a partial tile into the split-K meeting place (reductions without return value).
+template <bool kBase, int W>
+__device__ __forceinline__ void partial_chunk(uint32_t t_row, int32_t* acc_tile, int c0, int r) {
+  uint32_t v[W];
+  tmem_ldw<W>(t_row + c0, v);
+  tmem_ld_wait();
+#pragma unroll
+  for (int j = 0; j < W; ++j) {
+    if constexpr (kBase) atomicAdd(reinterpret_cast<float*>(acc_tile) + (c0 + j) * kTileN + r, __uint_as_float(v[j]));
+    else atomicAdd(acc_tile + (c0 + j) * kTileN + r, static_cast<int32_t>(v[j]));
+  }
+}
+
 // kBase = false: the MSD path (INT8 x INT8 -> INT32, stacked components, scale-combine epilogue).
 // kBase = true : the comparison path the method replaces - the same pipeline on BF16 weights that a preceding kernel
 //                dequantized into the workspace, BF16 x BF16 -> FP32, no decomposition and no scales in the epilogue.
@@ -91,6 +145,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  if (p.num_stages < 1 || p.kw < 1 || p.kblocks < 1) return;     // malformed plan: touch nothing
   if (threadIdx.x == 0 && p.trace) {
     trace_mark(p, 0);
     unsigned long long g;
@@ -98,8 +153,9 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     p.trace[blockIdx.x * 16 + 1] = static_cast<long long>(g);
   }
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
-  const int x_stage_bytes = p.NB * kBlockK;
-  const int stage_bytes = p.w_stage_bytes + x_stage_bytes;
+  const int x_chunk_bytes = p.NB * kBlockK;
+  const int w_stage_bytes = p.kw * p.w_chunk_bytes;
+  const int stage_bytes = w_stage_bytes + p.kw * x_chunk_bytes;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.num_stages; ++s) {
@@ -143,7 +199,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   // whole row instead of hitting the same 128-byte column of every row (integer sums do not depend on the order).
   const int kb_rot = (p.mode == 1) ? static_cast<int>((static_cast<long long>(blockIdx.x) * p.kb_rot_step) % p.kblocks) : 0;
   const CUtensorMap* wmap = (p.mode == 1 && band_h != p.hmax) ? &tmap_w2 : &tmap_w;
-  const int tx_bytes = (p.mode == 0 ? kWStageBytes : band_h * kBlockK) + x_stage_bytes;
+  const int tx_bytes = p.kw * ((p.mode == 0 ? kWStageBytes : band_h * kBlockK) + x_chunk_bytes);
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -160,14 +216,18 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         const long long blk = blk_begin + i;
         const int tile = static_cast<int>(blk / p.kblocks), kb = static_cast<int>((blk + kb_rot) % p.kblocks);
         mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
-        tma_load_2d_hint(smem + i * stage_bytes, wmap, kb * kBlockK, band_row0 + tile * kTileN, &full_bar[i], pol_w);
+        for (int c = 0; c < p.kw; ++c)
+          tma_load_2d_hint(smem + i * stage_bytes + c * p.w_chunk_bytes, wmap, (kb * p.kw + c) * kBlockK,
+                           band_row0 + tile * kTileN, &full_bar[i], pol_w);
       }
       trace_mark(p, 3);
       pdl_wait_primary();
       trace_mark(p, 4);
       for (int i = 0; i < pre; ++i) {
         const int kb = static_cast<int>((blk_begin + i + kb_rot) % p.kblocks);
-        tma_load_2d_hint(smem + i * stage_bytes + p.w_stage_bytes, &tmap_x, kb * kBlockK, 0, &full_bar[i], pol_x);
+        for (int c = 0; c < p.kw; ++c)
+          tma_load_2d_hint(smem + i * stage_bytes + w_stage_bytes + c * x_chunk_bytes, &tmap_x, (kb * p.kw + c) * kBlockK, 0,
+                           &full_bar[i], pol_x);
       }
       stage = pre % p.num_stages;
       phase = (pre == p.num_stages) ? 1 : 0;
@@ -178,8 +238,11 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         if (!ok) break;
         mbar_arrive_expect_tx(&full_bar[stage], tx_bytes);
         uint8_t* dst = smem + stage * stage_bytes;
-        tma_load_2d_hint(dst, wmap, kb * kBlockK, band_row0 + tile * kTileN, &full_bar[stage], pol_w);
-        tma_load_2d_hint(dst + p.w_stage_bytes, &tmap_x, kb * kBlockK, 0, &full_bar[stage], pol_x);
+        for (int c = 0; c < p.kw; ++c)
+          tma_load_2d_hint(dst + c * p.w_chunk_bytes, wmap, (kb * p.kw + c) * kBlockK, band_row0 + tile * kTileN,
+                           &full_bar[stage], pol_w);
+        for (int c = 0; c < p.kw; ++c)
+          tma_load_2d_hint(dst + w_stage_bytes + c * x_chunk_bytes, &tmap_x, (kb * p.kw + c) * kBlockK, 0, &full_bar[stage], pol_x);
         if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
       }
       trace_mark(p, 5);
@@ -214,13 +277,16 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
           if (b == blk_begin) trace_mark(p, 6);
           tc_fence_after();
           const uint32_t wa = smem_u32(smem + stage * stage_bytes);
-          const uint32_t xa = wa + p.w_stage_bytes;   // the MMA reads 128 A rows; rows past the band are never used
+          const uint32_t xa = wa + w_stage_bytes;     // the MMA reads 128 A rows; rows past the band are never used
+          for (int c = 0; c < p.kw; ++c) {
 #pragma unroll
-          for (int k = 0; k < kBlockK / 32; ++k) {
-            const uint64_t adesc = smem_desc(wa + k * 32, 16, 1024, kSwizzle128B);
-            const uint64_t bdesc = smem_desc(xa + k * 32, 16, 1024, kSwizzle128B);
-            if constexpr (kBase) mma_f16(d_tmem, adesc, bdesc, idesc, (b > blk || k > 0) ? 1u : 0u);
-            else mma_i8(d_tmem, adesc, bdesc, idesc, (b > blk || k > 0) ? 1u : 0u);
+            for (int k = 0; k < kBlockK / 32; ++k) {
+              const uint64_t adesc = smem_desc(wa + c * p.w_chunk_bytes + k * 32, 16, 1024, kSwizzle128B);
+              const uint64_t bdesc = smem_desc(xa + c * x_chunk_bytes + k * 32, 16, 1024, kSwizzle128B);
+              const uint32_t accum = (b > blk || c > 0 || k > 0) ? 1u : 0u;
+              if constexpr (kBase) mma_f16(d_tmem, adesc, bdesc, idesc, accum);
+              else mma_i8(d_tmem, adesc, bdesc, idesc, accum);
+            }
           }
           tc_commit(&empty_bar[stage]);          // frees the stage once these MMAs have read it
           if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
@@ -264,23 +330,18 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       const bool row_ok = (r < band_h) && (n < p.N);
       const float sw = (!kBase && row_ok) ? __ldg(p.w_scale + n) : 0.0f;
       bool finish = complete;
-      int c_lo = 0, c_hi = -1;
+      int32_t* acc_tile = nullptr;
       if (!complete) {
-        // park this CTA's partial sums in its slot, then find out whether it is the last contributor of the tile
-        const int slot_id = 2 * blockIdx.x + ((blk_begin >= tile_begin) ? 0 : 1);
-        int32_t* slot = p.slots + static_cast<long long>(slot_id) * p.NB * kTileN;
-        for (int c0 = 0; c0 < p.NB; c0 += 16) {
-          uint32_t v[16];
-          tmem_ld16(t_row + c0, v);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 16; ++j) slot[(c0 + j) * kTileN + r] = static_cast<int32_t>(v[j]);
-        }
+        // add this CTA's partial sums into the tile's meeting place, then find out whether it was the last contributor
+        acc_tile = p.accum + static_cast<long long>(tile) * p.NB * kTileN;
+        int c0 = 0;
+        for (; c0 + 32 <= p.NB; c0 += 32) partial_chunk<kBase, 32>(t_row, acc_tile, c0, r);
+        if (c0 + 16 <= p.NB) partial_chunk<kBase, 16>(t_row, acc_tile, c0, r);
         named_bar_sync(1, 128);
-        c_lo = static_cast<int>(block_owner(tile_begin, p.total_blocks, grid));
-        c_hi = static_cast<int>(block_owner(tile_end - 1, p.total_blocks, grid));
         if (et == 0) {
-          __threadfence();     // cumulative: publishes the slot writes of all 128 threads ordered by the barrier above
+          const int c_lo = static_cast<int>(block_owner(tile_begin, p.total_blocks, grid));
+          const int c_hi = static_cast<int>(block_owner(tile_end - 1, p.total_blocks, grid));
+          __threadfence();     // cumulative: publishes the additions of all 128 threads ordered by the barrier above
           const unsigned prev = atomicAdd(&p.counters[tile], 1u);
           const int last = (prev == static_cast<unsigned>(c_hi - c_lo)) ? 1 : 0;
           if (last) p.counters[tile] = 0;          // leave the counter ready for the next call
@@ -291,42 +352,10 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         if (finish) __threadfence();
       }
       if (finish) {
-        for (int c0 = 0; c0 < p.Mp; c0 += 8) {
-          uint32_t a[8], b[8];
-          tmem_ld8(t_row + c0, a);
-          if constexpr (!kBase) tmem_ld8(t_row + p.Mp + c0, b);
-          tmem_ld_wait();
-          for (int c = c_lo; c <= c_hi; ++c) {
-            if (c == static_cast<int>(blockIdx.x)) continue;
-            const int sid = 2 * c + ((range_begin(c, p.total_blocks, grid) >= tile_begin) ? 0 : 1);
-            const int32_t* slot = p.slots + static_cast<long long>(sid) * p.NB * kTileN;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              if constexpr (kBase) {
-                a[j] = __float_as_uint(__uint_as_float(a[j]) + __int_as_float(__ldcg(slot + (c0 + j) * kTileN + r)));
-              } else {
-                a[j] += static_cast<uint32_t>(__ldcg(slot + (c0 + j) * kTileN + r));
-                b[j] += static_cast<uint32_t>(__ldcg(slot + (p.Mp + c0 + j) * kTileN + r));
-              }
-            }
-          }
-          if (row_ok) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const int i = c0 + j;
-              if (i < p.M) {
-                if constexpr (kBase) {
-                  store_out(p, i, n, __uint_as_float(a[j]), 0, 0);
-                } else {
-                  const int32_t ya = static_cast<int32_t>(a[j]), yb = static_cast<int32_t>(b[j]);
-                  // y = s_W * (alpha * Y1 + beta * Y2)   (Alg. 1 line 8)
-                  const float v = sw * __fmaf_rn(s_alpha[i], static_cast<float>(ya), s_beta[i] * static_cast<float>(yb));
-                  store_out(p, i, n, v, ya, yb);
-                }
-              }
-            }
-          }
-        }
+        int c0 = 0;
+        for (; c0 + 32 <= p.Mp; c0 += 32) epilogue_chunk<kBase, 32>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta);
+        if (c0 + 16 <= p.Mp) { epilogue_chunk<kBase, 16>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta); c0 += 16; }
+        if (c0 + 8 <= p.Mp) epilogue_chunk<kBase, 8>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta);
       }
       tc_fence_before();
       __syncwarp();
@@ -356,7 +385,7 @@ static int pow2_at_least(int v) {
 
 struct GemmW8Plan {
   int Mp, NB, kblocks, num_tiles, grid, stages, tmem_cols;
-  int mode, groups8, hmax, w_stage_bytes;
+  int mode, groups8, hmax, w_chunk_bytes, kw;
   long long total_blocks;
   size_t off_q, off_alpha, off_beta, off_counters, off_slots, bytes;
   size_t smem_bytes;
@@ -374,7 +403,15 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   pl.Mp = base ? static_cast<int>((M + 15) / 16 * 16) : static_cast<int>((M + 7) / 8 * 8);
   pl.NB = base ? pl.Mp : 2 * pl.Mp;
   const int64_t kbytes = base ? 2 * K : K;
-  pl.kblocks = static_cast<int>((kbytes + kBlockK - 1) / kBlockK);
+  // K boxes per stage: wide stages read each weight row in runs of kw*128 bytes (good for DRAM page locality);
+  // the operand tile of the stacked components grows with kw too, so wide activations get narrower stages.
+  int kw = (pl.NB <= 64) ? 4 : 2;
+  kw = env_int("MSD_GEMM_KW", kw);
+  if (kw < 1) kw = 1;
+  if (kw > 8) kw = 8;
+  while (kw > 1 && static_cast<int64_t>(kw) * kBlockK > kbytes) kw >>= 1;
+  pl.kw = kw;
+  pl.kblocks = static_cast<int>((kbytes + static_cast<int64_t>(kw) * kBlockK - 1) / (static_cast<int64_t>(kw) * kBlockK));
   pl.num_tiles = static_cast<int>((N + kTileN - 1) / kTileN);
   pl.total_blocks = static_cast<long long>(pl.kblocks) * pl.num_tiles;
   pl.groups8 = static_cast<int>((N + 7) / 8);
@@ -392,18 +429,26 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   pl.mode = mode;
   if (mode == 1) {
     pl.hmax = band_max;
-    pl.w_stage_bytes = static_cast<int>(round_up(static_cast<size_t>(band_max) * kBlockK, 1024));
+    pl.w_chunk_bytes = static_cast<int>(round_up(static_cast<size_t>(band_max) * kBlockK, 1024));
   } else {
     if (grid > pl.total_blocks) grid = static_cast<int>(pl.total_blocks);
     pl.hmax = kTileN;
-    pl.w_stage_bytes = kWStageBytes;
+    pl.w_chunk_bytes = kWStageBytes;
   }
   pl.grid = grid;
-  const int stage_bytes = pl.w_stage_bytes + pl.NB * kBlockK;
-  const int tail_pad = kWStageBytes - pl.w_stage_bytes;     // the MMA reads a full 128-row A tile from every stage
+  const int tail_pad = kWStageBytes - pl.w_chunk_bytes;     // the MMA reads a full 128-row A tile from every box
+  // at least two stages must fit: narrow the stage (and recount the K blocks) until they do
+  int stage_bytes = pl.kw * (pl.w_chunk_bytes + pl.NB * kBlockK);
+  while (pl.kw > 1 && (kSmemBudget - tail_pad) / stage_bytes < 2) {
+    pl.kw >>= 1;
+    stage_bytes = pl.kw * (pl.w_chunk_bytes + pl.NB * kBlockK);
+  }
+  pl.kblocks = static_cast<int>((kbytes + static_cast<int64_t>(pl.kw) * kBlockK - 1) / (static_cast<int64_t>(pl.kw) * kBlockK));
+  pl.total_blocks = static_cast<long long>(pl.kblocks) * pl.num_tiles;
+  if (mode == 0 && pl.grid > pl.total_blocks) pl.grid = static_cast<int>(pl.total_blocks);
   int stages = (kSmemBudget - tail_pad) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
-  if (stages > pl.kblocks && mode == 1) stages = pl.kblocks > 1 ? pl.kblocks : 1;
+  if (stages < 1) stages = 1;      // cannot happen: one 128-byte box of the widest operands is 48 KB
   pl.stages = stages;
   pl.smem_bytes = static_cast<size_t>(stages) * stage_bytes + tail_pad + 1024;
   pl.tmem_cols = pow2_at_least(2 * pl.NB);
@@ -412,8 +457,8 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   pl.off_alpha = off;     off = round_up(off + 128 * sizeof(float), 256);
   pl.off_beta = off;      off = round_up(off + 128 * sizeof(float), 256);
   pl.off_counters = off;  off = round_up(off + static_cast<size_t>(pl.num_tiles) * sizeof(unsigned), 1024);
-  // slot space sized for the largest grid the launcher may pick, so the same workspace serves any override
-  pl.off_slots = off;     off = round_up(off + static_cast<size_t>(256) * 2 * pl.NB * kTileN * sizeof(int32_t), 1024);
+  // split-K meeting place: one [NB x 128] tile of sums per weight tile (used by the stream-K split only)
+  pl.off_slots = off;     off = round_up(off + static_cast<size_t>(pl.num_tiles) * pl.NB * kTileN * sizeof(int32_t), 1024);
   pl.bytes = off;
   return pl;
 }
@@ -494,11 +539,11 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
   GemmW8Params p;
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = env_int("MSD_GEMM_KROT", 5);
-  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_stage_bytes = pl.w_stage_bytes;
+  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
   p.w_scale = w_scale; p.alpha = alpha; p.beta = beta; p.y = y; p.acc_dbg = acc_dbg;
-  p.slots = reinterpret_cast<int32_t*>(ws + pl.off_slots);
+  p.accum = reinterpret_cast<int32_t*>(ws + pl.off_slots);
   p.counters = reinterpret_cast<unsigned*>(ws + pl.off_counters);
   p.status = status;
   p.trace = g_trace;
@@ -551,11 +596,11 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   GemmW8Params p;
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = 0;
-  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_stage_bytes = pl.w_stage_bytes;
+  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
   p.w_scale = w_scale; p.alpha = nullptr; p.beta = nullptr; p.y = y; p.acc_dbg = nullptr;
-  p.slots = reinterpret_cast<int32_t*>(ws + pl.off_slots);
+  p.accum = reinterpret_cast<int32_t*>(ws + pl.off_slots);
   p.counters = reinterpret_cast<unsigned*>(ws + pl.off_counters);
   p.status = status;
   p.trace = nullptr;
