@@ -6,13 +6,16 @@
 #include <cuda_bf16.h>
 #include <cuda_fp4.h>
 
+#include <cstdlib>
+
 #include "host_common.h"
 #include "sm100.cuh"
 
 namespace msd {
 
-constexpr int kDecThreads = 512;
-constexpr int kDecCache = 4;   // 16-element chunks a thread keeps in registers between the two passes
+// 256 threads x 64 registers leave room for a CTA of the dependent GEMM (192 threads x ~224 registers) on the same SM,
+// so that GEMM can start prefetching weights everywhere while this kernel still runs.
+constexpr int kDecCache = 4;   // 16-element chunks a thread keeps in registers between the two passes (K <= 16384)
 
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
@@ -29,13 +32,24 @@ __device__ __forceinline__ float chunk_absmax(const uint4& a, const uint4& b) {
   return m;
 }
 
-__device__ __forceinline__ int quant_i8(float v, float scale) {
-  int q = __float2int_rn(__fdiv_rn(v, scale));     // true division, round-half-to-even
+// clamp(rne(fl(v / scale)), -128, 127), bit for bit, without paying for an IEEE division per element:
+// c = rne(v * (1/scale)) can differ from the rounded true quotient only when the quotient sits within a few ulps of a
+// half-integer: |v*inv - v/scale| <= 127 * 2^-23 < 2^-16, so whenever the exact remainder v - scale*c is further than
+// 2^-14 * scale from +-scale/2, c is the nearest integer of the true quotient with a margin that the quotient's own
+// FP32 rounding (< 2^-17) cannot cross.  The rare elements inside that band take the true division.
+__device__ __forceinline__ int quant_i8(float v, float scale, float inv_scale) {
+  const float c = rintf(v * inv_scale);
+  const float rem = __fmaf_rn(-scale, c, v);                  // exact for |c| <= 2^7 and BF16-derived inputs
+  const float dist = fabsf(fabsf(rem) - 0.5f * scale);
+  int q;
+  if (dist > scale * 6.103515625e-05f && fabsf(c) <= 127.0f) q = __float2int_rn(c);
+  else q = __float2int_rn(__fdiv_rn(v, scale));               // true division, round-half-to-even
   return max(-128, min(127, q));
 }
 
 // Two-pass quantisation of 16 values; returns the packed codes of both passes.
-__device__ __forceinline__ void chunk_quantize(const uint4& a, const uint4& b, float alpha, float beta, uint4& o1, uint4& o2) {
+__device__ __forceinline__ void chunk_quantize(const uint4& a, const uint4& b, float alpha, float beta, float inv_alpha,
+                                               float inv_beta, uint4& o1, uint4& o2) {
   const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
   uint32_t p1[4] = {0, 0, 0, 0}, p2[4] = {0, 0, 0, 0};
 #pragma unroll
@@ -45,9 +59,9 @@ __device__ __forceinline__ void chunk_quantize(const uint4& a, const uint4& b, f
       const float v = h ? bf16hi(w[i]) : bf16lo(w[i]);
       int c1 = 0, c2 = 0;
       if (alpha > 0.0f) {
-        c1 = quant_i8(v, alpha);                                          // Eq. x1
+        c1 = quant_i8(v, alpha, inv_alpha);                               // Eq. x1
         const float r = __fmaf_rn(-alpha, static_cast<float>(c1), v);     // Eq. residual, exact
-        if (beta > 0.0f) c2 = quant_i8(r, beta);                          // Eq. x2
+        if (beta > 0.0f) c2 = quant_i8(r, beta, inv_beta);                // Eq. x2
       }
       const int e = 2 * i + h;
       p1[e >> 2] |= static_cast<uint32_t>(c1 & 0xFF) << (8 * (e & 3));
@@ -58,10 +72,15 @@ __device__ __forceinline__ void chunk_quantize(const uint4& a, const uint4& b, f
   o2 = make_uint4(p2[0], p2[1], p2[2], p2[3]);
 }
 
+template <int kDecThreads>
 __global__ void __launch_bounds__(kDecThreads)
 decompose_int8_kernel(const uint16_t* __restrict__ x, int64_t ldx, int K, int8_t* __restrict__ q1,
                       int8_t* __restrict__ q2, float* __restrict__ alpha_out, float* __restrict__ beta_out) {
-  pdl_launch_dependents();      // a dependent GEMM may start prefetching its weights right away
+  // When launched as a programmatic dependent of whatever precedes it in the stream it may become resident early, but
+  // it reads nothing before that work has completed (the wait is a no-op for a plain launch); only then may its own
+  // dependent (the GEMM) start prefetching weights.
+  pdl_wait_primary();
+  pdl_launch_dependents();
   const int row = blockIdx.x;
   const uint4* xr = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(row) * ldx);
   const int nchunks = K >> 4;
@@ -90,6 +109,9 @@ decompose_int8_kernel(const uint16_t* __restrict__ x, int64_t ldx, int K, int8_t
 
   const float alpha = __fdiv_rn(m, 127.0f);        // Eq. alpha
   const float beta = __fdiv_rn(alpha, 254.0f);     // Eq. beta
+  // reciprocals only steer the fast path of quant_i8; infinities (tiny scales) simply send every element to the division
+  const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f;
+  const float inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
   if (threadIdx.x == 0) {
     alpha_out[row] = alpha;
     beta_out[row] = beta;
@@ -101,14 +123,14 @@ decompose_int8_kernel(const uint16_t* __restrict__ x, int64_t ldx, int K, int8_t
     const int c = threadIdx.x + j * kDecThreads;
     if (c < nchunks) {
       uint4 r1, r2;
-      chunk_quantize(ca[j], cb[j], alpha, beta, r1, r2);
+      chunk_quantize(ca[j], cb[j], alpha, beta, inv_alpha, inv_beta, r1, r2);
       o1[c] = r1;
       o2[c] = r2;
     }
   }
   for (int c = threadIdx.x + kDecCache * kDecThreads; c < nchunks; c += kDecThreads) {
     uint4 r1, r2;
-    chunk_quantize(__ldg(xr + 2 * c), __ldg(xr + 2 * c + 1), alpha, beta, r1, r2);
+    chunk_quantize(__ldg(xr + 2 * c), __ldg(xr + 2 * c + 1), alpha, beta, inv_alpha, inv_beta, r1, r2);
     o1[c] = r1;
     o2[c] = r2;
   }
@@ -182,9 +204,22 @@ decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, i
 msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
                                    float* alpha, float* beta, cudaStream_t stream) {
   if (M == 0) return MSD_OK;
-  decompose_int8_kernel<<<static_cast<unsigned>(M), kDecThreads, 0, stream>>>(
-      static_cast<const uint16_t*>(x_bf16), ldx, static_cast<int>(K), q1, q2, alpha, beta);
-  return launch_status();
+  // Chained programmatic launch (this kernel resident while its predecessor still runs) is opt-in: measured slower.
+  const bool pdl = getenv("MSD_DEC_CHAIN") != nullptr && getenv("MSD_NO_PDL") == nullptr;
+  const char* te = getenv("MSD_DEC_THREADS");
+  // this kernel sits on the critical path of the GEMM behind it: more threads per row = shorter latency
+  const int threads = te ? atoi(te) : (K >= 8192 ? 1024 : (K >= 2048 ? 512 : 256));
+  cudaError_t err;
+  if (threads >= 1024)
+    err = launch_pdl(decompose_int8_kernel<1024>, dim3(static_cast<unsigned>(M)), dim3(1024), 0, stream, pdl,
+                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta);
+  else if (threads >= 512)
+    err = launch_pdl(decompose_int8_kernel<512>, dim3(static_cast<unsigned>(M)), dim3(512), 0, stream, pdl,
+                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta);
+  else
+    err = launch_pdl(decompose_int8_kernel<256>, dim3(static_cast<unsigned>(M)), dim3(256), 0, stream, pdl,
+                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta);
+  return err == cudaSuccess ? MSD_OK : MSD_ERR_CUDA;
 }
 
 msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
@@ -194,6 +229,11 @@ msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, in
   const int64_t want = (nblocks + kMxThreads - 1) / kMxThreads;
   const int64_t cap = static_cast<int64_t>(sm_count()) * 32;
   const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
+  static bool carve_done = false;
+  if (!carve_done) {
+    cudaFuncSetAttribute(decompose_mxfp4_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    carve_done = true;
+  }
   decompose_mxfp4_kernel<<<grid, kMxThreads, 0, stream>>>(static_cast<const uint16_t*>(x_bf16), ldx, M,
                                                           static_cast<int>(K), q1, q2, e1, e2, sf_kgroups);
   return launch_status();

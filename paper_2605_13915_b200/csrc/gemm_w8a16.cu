@@ -9,8 +9,8 @@
 //    of 8, at most 128), each CTA runs the whole K loop for its band and writes its outputs straight from TMEM.
 //  * stream-K (few rows per SM): the (128-row tile, 128-byte K block) pairs are numbered tile-major and divided evenly
 //    over the CTAs, so every SM streams the same number of weight bytes.  A CTA whose range covers a whole tile
-//    finishes it alone; a tile shared by several CTAs is reduced through per-CTA INT32 slots in the workspace and
-//    finished by whichever CTA arrives last (integer sums: the result does not depend on the arrival order).
+//    finishes it alone; the CTAs that share a tile add their INT32 partial sums into the tile's meeting place in the
+//    workspace and whichever arrives last reads it back, re-zeroes it and finishes (integer sums: order-free).
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (+ TMEM owner), warps 2-5 = epilogue (one per TMEM lane group).
 #include <cuda_bf16.h>
@@ -146,6 +146,8 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   if (p.num_stages < 1 || p.kw < 1 || p.kblocks < 1) return;     // malformed plan: touch nothing
+  // lets a decomposition kernel queued behind this GEMM become resident early (it still waits for this grid to finish)
+  pdl_launch_dependents();
   if (threadIdx.x == 0 && p.trace) {
     trace_mark(p, 0);
     unsigned long long g;
@@ -368,7 +370,12 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
 
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0) trace_mark(p, 12);
+  if (threadIdx.x == 0 && p.trace) {
+    trace_mark(p, 12);
+    unsigned long long g;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g));
+    p.trace[blockIdx.x * 16 + 13] = static_cast<long long>(g);
+  }
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, p.tmem_cols);
