@@ -90,6 +90,28 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
                             int64_t K, void* y, msd_out_t ytype, int32_t* acc_dbg, void* workspace,
                             size_t workspace_bytes, void* stream);
 
+/*
+ * The same W8A16 layer for callers that cannot allocate device memory.  (The paper has no counterpart; this is a
+ * packaging variant of msd_gemm_w8a16, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a plug-in called from inside somebody else's serving
+ * loop that forbids allocation on the hot path, a host whose memory pool is owned by another runtime and handed out
+ * only as ready-made input/output tensors, or a latency-critical thread that must not take the allocator's lock.
+ * Such a caller can still pass inputs and outputs, but has no way to obtain a workspace.  This entry point therefore
+ * takes none: its scratch is a fixed array inside the library's device image (3 MB + 1 KB per GPU that loads the
+ * library, held until the process exits).  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ * Limits: 1 <= M <= 16, N <= 16384, K <= 16384 (and the shape rules of msd_gemm_w8a16); anything larger returns
+ * MSD_ERR_UNSUPPORTED before any launch - use msd_gemm_w8a16 with your own workspace instead.
+ * First use on a device resolves the array's device address (cudaGetSymbolAddress, with that device current); make
+ * that first call outside any stream capture.  All calls on a device share the one array: it still holds the
+ * previous call's contents (the parts that must start at zero are cleared on `stream` at the start of every call), and
+ * two calls that overlap on the GPU - different streams, or a graph replayed concurrently - race on it.  Results are
+ * identical to msd_gemm_w8a16.
+ */
+msd_status_t msd_gemm_w8a16_noalloc(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
+                                    int64_t K, void* y, msd_out_t ytype, void* stream);
+
 /* Diagnostic hook: when `device_buffer` is non-NULL, every later msd_gemm_w8a16 launch writes 16 64-bit SM-clock
  * samples per CTA into it (entry, set-up done, producer / MMA / epilogue milestones); NULL switches it off.
  * The buffer must hold 16 * 8 bytes per SM-count CTA (256 CTAs at most). */

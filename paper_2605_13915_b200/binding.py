@@ -35,6 +35,7 @@ _SIGS = {
     "msd_decompose_mxfp4": (C.c_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp]),
     "msd_gemm_w8a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_w8a16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _vp, _sz, _vp]),
+    "msd_gemm_w8a16_noalloc": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp]),
     "msd_debug_set_trace": (None, [_vp]),
     "msd_gemm_w8a16_host_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_w8a16_host": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
@@ -145,6 +146,18 @@ def gemm_w8a16(x, w, w_scale, out_dtype=torch.bfloat16, ws=None, want_acc=False,
                                 _ptr(acc), wp, wb, _stream())
     _check(code, "msd_gemm_w8a16")
     return (y, acc) if want_acc else y
+
+
+def gemm_w8a16_noalloc(x, w, w_scale, out):
+    """W8A16 layer through the entry point that owns its scratch (for callers that may not allocate device memory):
+    the caller passes inputs and a preallocated output only.  M <= 16, N <= 16384, K <= 16384."""
+    _need_cuda(x, w, w_scale, out)
+    M, K = x.shape
+    N = w.shape[0]
+    code = lib().msd_gemm_w8a16_noalloc(_ptr(x), _ptr(w), _ptr(w_scale), M, N, K, _ptr(out),
+                                        OUT_BF16 if out.dtype == torch.bfloat16 else OUT_FP32, _stream())
+    _check(code, "msd_gemm_w8a16_noalloc")
+    return out
 
 
 def gemm_w8a16_host_workspace_bytes(M, N, K):

@@ -623,6 +623,54 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   return MSD_OK;
 }
 
+// ---------------------------------------------------------------------------------------------------------------------
+// Entry point for callers that cannot allocate device memory (see msd.h).  The scratch the GEMM needs lives in this
+// file-scope device array, which every GPU that loads the library holds until the process exits.
+// ---------------------------------------------------------------------------------------------------------------------
+}  // extern "C"
+
+namespace msd {
+constexpr int64_t kStaticMaxM = 16;
+constexpr int64_t kStaticMaxN = 16384;
+constexpr int64_t kStaticMaxK = 16384;
+constexpr size_t kStaticScratchBytes = 3u << 20;      // covers the workspace of M<=16, N<=16384, K<=16384 (about 2.6 MB)
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes + 1024];
+
+// Device address of the scratch array on the current device (resolved once per device); NULL on failure.
+// In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel could use.
+static unsigned char* static_scratch_ptr() {
+  static unsigned char* cache[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cache[dev]) {
+    unsigned char* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess || !ptr) return nullptr;
+    cache[dev] = ptr;
+  }
+  return cache[dev];
+}
+}  // namespace msd
+
+extern "C" {
+
+msd_status_t msd_gemm_w8a16_noalloc(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
+                                    int64_t K, void* y, msd_out_t ytype, void* stream) {
+  using namespace msd;
+  if (M < 1 || N < 1 || K < 16) return MSD_ERR_BAD_SHAPE;
+  if (M > kStaticMaxM || N > kStaticMaxN || K > kStaticMaxK) return MSD_ERR_UNSUPPORTED;   // beyond the built-in scratch
+  unsigned char* raw = static_scratch_ptr();
+  if (!raw) return MSD_ERR_CUDA;
+  unsigned char* ws = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  const size_t avail = kStaticScratchBytes + 1024 - static_cast<size_t>(ws - raw);
+  const GemmW8Plan pl = plan_w8(M, N, K);
+  if (pl.bytes > avail) return MSD_ERR_UNSUPPORTED;
+  // The array keeps whatever the previous call left.  The split-K counters and meeting place must start at zero; a
+  // completed call leaves them so, but a call that gave up on a wait may not have, so they are cleared every time.
+  if (cudaMemsetAsync(ws + pl.off_counters, 0, pl.bytes - pl.off_counters, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return MSD_ERR_CUDA;
+  return msd_gemm_w8a16(x_bf16, w, w_scale, M, N, K, y, ytype, nullptr, ws, avail, stream);
+}
+
 void msd_debug_set_trace(void* device_buffer) { msd::g_trace = static_cast<long long*>(device_buffer); }
 
 size_t msd_gemm_w8a16_host_workspace_bytes(int64_t M, int64_t N, int64_t K) {
