@@ -265,6 +265,7 @@ def run_gpu(args):
                 "api": "msd_gemm_w8a16_host (pinned host activations and outputs, weights resident)"},
         "gpu_launches": 2 * len(calls) * args.steps,
         "roofline": {"bound": "hbm", "achieved": round(value / world, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "bytes_per_launch": step_bytes // len(calls), "us_per_launch": round(ms_per_step * 1e3 / len(calls), 3),
                      "frac": round(value / world / peaks["hbm_gbs"], 4), "peak_kind": f"of {peak_kind}",
                      "traffic": None, "kernel": "gemm_w8a16_kernel (+ decompose_int8_kernel overlapped by PDL)",
                      "note": "achieved = algorithmic bytes of the sweep / device time of the timed region"},
@@ -273,7 +274,9 @@ def run_gpu(args):
     traffic_file = os.path.join(ROOT, "profiles", "gemm_w8a16_traffic.json")
     if os.path.exists(traffic_file):
         with open(traffic_file) as f:
-            out["roofline"]["traffic"] = json.load(f)
+            tr = json.load(f)
+        out["roofline"]["traffic"] = tr["dram_bytes"]
+        out["roofline"]["traffic_of"] = tr["launch"] + f"; algorithmic bytes of that launch {tr['algorithmic_bytes']}"
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(check=(binding, data, torch))
     print(json.dumps(out), flush=True)
