@@ -48,15 +48,22 @@ __device__ __forceinline__ int swz_off(int row, int byte_in_row) {
   return row * 128 + ((((byte_in_row >> 4) ^ (row & 7)) & 7) << 4) + (byte_in_row & 15);
 }
 
-template <int kMaxHG, int kMaxDVT>
-__global__ void __launch_bounds__(kAttnThreads)
+// order-preserving float <-> int map (an involution), so that a warp maximum can use the integer redux instruction
+__device__ __forceinline__ int f2ord(float f) { const int i = __float_as_int(f); return i ^ ((i >> 31) & 0x7fffffff); }
+__device__ __forceinline__ float ord2f(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
+__device__ __forceinline__ float warp_max(float v) { return ord2f(__reduce_max_sync(0xffffffffu, f2ord(v))); }
+
+// kMaxHG: head slots of the stacked operand (8 or 16); kNH: heads the code is unrolled for (<= kMaxHG);
+// kMaxDVT: 128-wide tiles of Dv.
+template <int kMaxHG, int kNH, int kMaxDVT>
+__global__ void __launch_bounds__(kAttnThreads, (kNH <= 8 && kMaxDVT == 1) ? 3 : 1)
 attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], s_full[2], p_full, o_full, o_empty;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ float s_aq[kMaxHG], s_bq[kMaxHG];
-  __shared__ float red[4][kMaxHG + 1];
+  __shared__ float red[2][4][kNH + 1];             // per-warp tile maxima, double buffered by tile parity
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x;
@@ -200,94 +207,80 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     if (lane == 0) mbar_arrive(&p_full);            // phase 0 of p_full: "Q operand ready"
     named_bar_sync(1, 128);                         // s_aq / s_bq visible to all four warps
 
-    float m_run[kMaxHG], l_part[kMaxHG], aq[kMaxHG], bq[kMaxHG];
-    float o_run[kMaxDVT][kMaxHG];
+    // running state per head; scores are kept in the log2 domain (log2(e) is folded into the key scale)
+    float m_run[kNH], l_part[kNH], aq[kNH], bq[kNH];
+    float o_run[kMaxDVT][kNH];
 #pragma unroll
-    for (int h = 0; h < kMaxHG; ++h) {
+    for (int h = 0; h < kNH; ++h) {
       m_run[h] = -INFINITY; l_part[h] = 0.0f;
       aq[h] = (h < nh) ? s_aq[h] : 0.0f; bq[h] = (h < nh) ? s_bq[h] : 0.0f;
 #pragma unroll
       for (int j = 0; j < kMaxDVT; ++j) o_run[j][h] = 0.0f;
     }
     const float kLog2e = 1.4426950408889634f;
+    const float scale2 = p.scale * kLog2e;
     bool ok = true;
     for (int t = 0; t < ntiles && ok; ++t) {
       const int tok_rel = t_begin + t * kTok + tl;
       const bool valid = tok_rel < t_end;
       const long long sidx = static_cast<long long>(seq0 + tok_rel) * p.Hkv + hk;
-      const float ks = valid ? __ldg(p.k_scale + sidx) * p.scale : 0.0f;
+      const float ks = valid ? __ldg(p.k_scale + sidx) * scale2 : 0.0f;
       const float vs = valid ? __ldg(p.v_scale + sidx) : 0.0f;
       ok = wait_bounded(&s_full[t & 1], (t >> 1) & 1, abort, p.status);
       if (!ok) break;
       tc_fence_after();
       // c3: merge the two integer products and apply the key scale
-      float s[kMaxHG];
+      float s[kNH];
       const uint32_t srow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + (t & 1) * p.Rp;
-      if constexpr (kMaxHG == 8) {
-        uint32_t v[16];
-        tmem_ld16(srow, v);
+      {
+        uint32_t v1[kMaxHG], v2[kMaxHG];          // first / second component columns
+        tmem_ldw<kMaxHG>(srow, v1);
+        tmem_ldw<kMaxHG>(srow + kMaxHG, v2);
         tmem_ld_wait();
 #pragma unroll
-        for (int h = 0; h < 8; ++h)
-          s[h] = valid ? __fmaf_rn(aq[h], static_cast<float>(static_cast<int32_t>(v[h])), bq[h] * static_cast<float>(static_cast<int32_t>(v[8 + h]))) * ks : -INFINITY;
-      } else {
-        uint32_t v1[16], v2[16];
-        tmem_ld16(srow, v1);
-        tmem_ld16(srow + 16, v2);
-        tmem_ld_wait();
-#pragma unroll
-        for (int h = 0; h < 16; ++h)
+        for (int h = 0; h < kNH; ++h)
           s[h] = valid ? __fmaf_rn(aq[h], static_cast<float>(static_cast<int32_t>(v1[h])), bq[h] * static_cast<float>(static_cast<int32_t>(v2[h]))) * ks : -INFINITY;
       }
       // c4: tile maxima per head (and of the value scales) over the 128 token lanes
-      float tm[kMaxHG + 1];
+      float (*rb)[kNH + 1] = red[t & 1];
 #pragma unroll
-      for (int h = 0; h < kMaxHG; ++h) tm[h] = s[h];
-      tm[kMaxHG] = vs;
-#pragma unroll
-      for (int h = 0; h <= kMaxHG; ++h) {
-        if (h < p.HG || h == kMaxHG) {
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) tm[h] = fmaxf(tm[h], __shfl_xor_sync(0xffffffffu, tm[h], o));
-        }
+      for (int h = 0; h < kNH; ++h) {
+        const float wm = warp_max(s[h]);
+        if (lane == 0) rb[wi][h] = wm;
       }
-      if (lane == 0) {
-#pragma unroll
-        for (int h = 0; h <= kMaxHG; ++h) red[wi][h] = tm[h];
+      {
+        const float wv = warp_max(vs);
+        if (lane == 0) rb[wi][kNH] = wv;
       }
-      named_bar_sync(1, 128);
-      float resc[kMaxHG];
+      named_bar_sync(1, 128);      // one barrier per tile: the other parity buffer is rewritten only after the next one
+      float resc[kNH];
 #pragma unroll
-      for (int h = 0; h < kMaxHG; ++h) {
-        const float mt = fmaxf(fmaxf(red[0][h], red[1][h]), fmaxf(red[2][h], red[3][h]));
+      for (int h = 0; h < kNH; ++h) {
+        const float mt = fmaxf(fmaxf(rb[0][h], rb[1][h]), fmaxf(rb[2][h], rb[3][h]));
         const float mn = fmaxf(m_run[h], mt);
-        resc[h] = (m_run[h] == -INFINITY) ? 0.0f : exp2f((m_run[h] - mn) * kLog2e);
+        resc[h] = (m_run[h] == -INFINITY) ? 0.0f : exp2f(m_run[h] - mn);
         m_run[h] = mn;
       }
-      const float vs_max = fmaxf(fmaxf(red[0][kMaxHG], red[1][kMaxHG]), fmaxf(red[2][kMaxHG], red[3][kMaxHG]));
-      named_bar_sync(1, 128);                       // everyone has read `red` before the next tile overwrites it
+      const float vs_max = fmaxf(fmaxf(rb[0][kNH], rb[1][kNH]), fmaxf(rb[2][kNH], rb[3][kNH]));
       // c5: P = exp(S - m), fold the value scale, two-pass INT8 with the fixed scale alpha_P = max(v_scale)/127
       const float alpha_p = __fdiv_rn(vs_max, 127.0f), beta_p = __fdiv_rn(alpha_p, 254.0f);
       const float inv_a = alpha_p > 0.0f ? 1.0f / alpha_p : 0.0f, inv_b = beta_p > 0.0f ? 1.0f / beta_p : 0.0f;
-      // the previous tile's PV must have finished reading the P operand before it is overwritten: it has, because
-      // these threads waited for o_full of that tile before merging it
+      // the previous tile's PV has finished reading the P operand: these threads waited for its o_full before merging
 #pragma unroll
-      for (int h = 0; h < kMaxHG; ++h) {
-        if (h < p.HG) {
-          int c1 = 0, c2 = 0;
-          if (h < nh && valid) {
-            const float pr = exp2f((s[h] - m_run[h]) * kLog2e);
-            l_part[h] = l_part[h] * resc[h] + pr;
-            const float pt = pr * vs;
-            c1 = max(-128, min(127, __float2int_rn(pt * inv_a)));
-            const float r = __fmaf_rn(-alpha_p, static_cast<float>(c1), pt);
-            c2 = max(-128, min(127, __float2int_rn(r * inv_b)));
-          } else {
-            l_part[h] *= resc[h];
-          }
-          sm_p[swz_off(h, tl)] = static_cast<uint8_t>(c1);
-          sm_p[swz_off(p.HG + h, tl)] = static_cast<uint8_t>(c2);
+      for (int h = 0; h < kNH; ++h) {
+        int c1 = 0, c2 = 0;
+        if (h < nh && valid) {
+          const float pr = exp2f(s[h] - m_run[h]);
+          l_part[h] = __fmaf_rn(l_part[h], resc[h], pr);
+          const float pt = pr * vs;
+          c1 = max(-128, min(127, __float2int_rn(pt * inv_a)));
+          const float r = __fmaf_rn(-alpha_p, static_cast<float>(c1), pt);
+          c2 = max(-128, min(127, __float2int_rn(r * inv_b)));
+        } else {
+          l_part[h] *= resc[h];
         }
+        sm_p[swz_off(h, tl)] = static_cast<uint8_t>(c1);
+        sm_p[swz_off(kMaxHG + h, tl)] = static_cast<uint8_t>(c2);
       }
       fence_proxy_async_smem();
       tc_fence_before();
@@ -301,22 +294,13 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       for (int j = 0; j < kMaxDVT; ++j) {
         if (j < p.DVT) {
           const uint32_t orow = tmem_o + (static_cast<uint32_t>(quad * 32) << 16) + j * p.Rp;
-          if constexpr (kMaxHG == 8) {
-            uint32_t v[16];
-            tmem_ld16(orow, v);
-            tmem_ld_wait();
+          uint32_t v1[kMaxHG], v2[kMaxHG];
+          tmem_ldw<kMaxHG>(orow, v1);
+          tmem_ldw<kMaxHG>(orow + kMaxHG, v2);
+          tmem_ld_wait();
 #pragma unroll
-            for (int h = 0; h < 8; ++h)
-              o_run[j][h] = __fmaf_rn(o_run[j][h], resc[h], __fmaf_rn(alpha_p, static_cast<float>(static_cast<int32_t>(v[h])), beta_p * static_cast<float>(static_cast<int32_t>(v[8 + h]))));
-          } else {
-            uint32_t v1[16], v2[16];
-            tmem_ld16(orow, v1);
-            tmem_ld16(orow + 16, v2);
-            tmem_ld_wait();
-#pragma unroll
-            for (int h = 0; h < 16; ++h)
-              o_run[j][h] = __fmaf_rn(o_run[j][h], resc[h], __fmaf_rn(alpha_p, static_cast<float>(static_cast<int32_t>(v1[h])), beta_p * static_cast<float>(static_cast<int32_t>(v2[h]))));
-          }
+          for (int h = 0; h < kNH; ++h)
+            o_run[j][h] = __fmaf_rn(o_run[j][h], resc[h], __fmaf_rn(alpha_p, static_cast<float>(static_cast<int32_t>(v1[h])), beta_p * static_cast<float>(static_cast<int32_t>(v2[h]))));
         }
       }
       tc_fence_before();
@@ -325,21 +309,22 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     }
     // partial results of this split: running max, sum of P and unnormalised output per head
     if (ok) {
+      float (*rb)[kNH + 1] = red[ntiles & 1];
+      named_bar_sync(1, 128);
 #pragma unroll
-      for (int h = 0; h < kMaxHG; ++h) {
-        if (h < nh) {
-          float l = l_part[h];
+      for (int h = 0; h < kNH; ++h) {
+        float l = l_part[h];
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-          if (lane == 0) red[wi][h] = l;
-        }
+        for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+        if (lane == 0) rb[wi][h] = l;
       }
       named_bar_sync(1, 128);
 #pragma unroll
-      for (int h = 0; h < kMaxHG; ++h) {
+      for (int h = 0; h < kNH; ++h) {
         if (h < nh) {
           float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + h) * p.n_splits + split) * (p.Dv + 2);
-          if (tl == 0) { dst[0] = m_run[h]; dst[1] = red[0][h] + red[1][h] + red[2][h] + red[3][h]; }
+          // the running maximum goes out in natural-log units (it was kept in the log2 domain)
+          if (tl == 0) { dst[0] = m_run[h] * 0.6931471805599453f; dst[1] = rb[0][h] + rb[1][h] + rb[2][h] + rb[3][h]; }
 #pragma unroll
           for (int j = 0; j < kMaxDVT; ++j)
             if (j < p.DVT && j * kChunk + tl < p.Dv) dst[2 + j * kChunk + tl] = o_run[j][h];
@@ -407,7 +392,7 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   pl->stages = (2 * static_cast<size_t>(kv_stage) + fixed <= 227 * 1024 - 2048) ? 2 : 1;
   const int tiles = (max_seqlen + kTok - 1) / kTok;
   const long long units = static_cast<long long>(B) * Hkv * pl->groups;
-  int ns = static_cast<int>((static_cast<long long>(sm_count()) * 4 + units - 1) / units);
+  int ns = static_cast<int>((static_cast<long long>(sm_count()) * 6 + units - 1) / units);
   if (ns > tiles) ns = tiles;
   if (ns < 1) ns = 1;
   if (ns > 64) ns = 64;
@@ -486,8 +471,15 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
   p.status = status;
 
   void (*kernel)(CUtensorMap, CUtensorMap, AttnParams) = nullptr;
-  if (pl.HG == 8) kernel = (pl.DVT == 1) ? attn_decode_kernel<8, 1> : (pl.DVT == 2) ? attn_decode_kernel<8, 2> : attn_decode_kernel<8, 4>;
-  else kernel = (pl.DVT == 1) ? attn_decode_kernel<16, 1> : (pl.DVT == 2) ? attn_decode_kernel<16, 2> : attn_decode_kernel<16, 4>;
+  const int G = Hq / Hkv;
+#define MSD_ATTN_PICK(HG_, NH_) \
+  kernel = (pl.DVT == 1) ? attn_decode_kernel<HG_, NH_, 1> : (pl.DVT == 2) ? attn_decode_kernel<HG_, NH_, 2> : attn_decode_kernel<HG_, NH_, 4>
+  if (pl.HG == 8) {
+    if (G <= 4) { MSD_ATTN_PICK(8, 4); } else { MSD_ATTN_PICK(8, 8); }
+  } else {
+    MSD_ATTN_PICK(16, 16);
+  }
+#undef MSD_ATTN_PICK
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
     return MSD_ERR_CUDA;
   dim3 grid(pl.n_splits, B * Hkv * pl.groups);
