@@ -116,6 +116,9 @@ msd_status_t msd_gemm_w8a16_noalloc(const void* x_bf16, const int8_t* w, const f
  * samples per CTA into it (entry, set-up done, producer / MMA / epilogue milestones); NULL switches it off.
  * The buffer must hold 16 * 8 bytes per SM-count CTA (256 CTAs at most). */
 void msd_debug_set_trace(void* device_buffer);
+/* Same for msd_attn_decode_int8kv: 32 samples per CTA for the first 1024 CTAs (entry, set-up done, then for the first
+ * six tiles: scores ready, P written, O ready, O merged; loop end; exit). */
+void msd_debug_set_attn_trace(void* device_buffer);
 
 /* Same computation with the activations and the result in HOST memory (pinned for asynchronous copies):
  * copies x to the device workspace, runs msd_gemm_w8a16, copies y back; weights stay resident on the device.
@@ -168,11 +171,11 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
                                     float softmax_scale, void* out_bf16, float* lse, void* workspace,
                                     size_t workspace_bytes, void* stream);
 
-/* The split schedule msd_attn_decode_int8kv uses for a sequence of length L (so a checker can mirror it):
- * writes the tile size and the number of context splits; split s covers tokens
- * [s*L_split, min(L,(s+1)*L_split)) with L_split = ceil(ceil(L/n_splits)/tile)*tile. */
+/* The split schedule msd_attn_decode_int8kv uses (so a checker can mirror it): writes the tile size, the number of
+ * context splits and the tokens per split; split s of a sequence of length L covers tokens
+ * [s*split_tokens, min(L, (s+1)*split_tokens)) and is walked in tiles of `tile` tokens (splits past L are empty). */
 msd_status_t msd_attn_decode_schedule(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen,
-                                      int32_t* tile, int32_t* n_splits);
+                                      int32_t* tile, int32_t* n_splits, int32_t* split_tokens);
 
 #ifdef __cplusplus
 }

@@ -37,6 +37,7 @@ _SIGS = {
     "msd_gemm_w8a16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _vp, _sz, _vp]),
     "msd_gemm_w8a16_noalloc": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp]),
     "msd_debug_set_trace": (None, [_vp]),
+    "msd_debug_set_attn_trace": (None, [_vp]),
     "msd_gemm_w8a16_host_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_w8a16_host": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_gemm_dequant_bf16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
@@ -46,7 +47,7 @@ _SIGS = {
     "msd_attn_decode_int8kv_workspace_bytes": (_sz, [_i32] * 6),
     "msd_attn_decode_int8kv": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp,
                                          _vp, _sz, _vp]),
-    "msd_attn_decode_schedule": (C.c_int, [_i32] * 6 + [C.POINTER(_i32), C.POINTER(_i32)]),
+    "msd_attn_decode_schedule": (C.c_int, [_i32] * 6 + [C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
 }
 
 
@@ -211,9 +212,10 @@ def gemm_w4a16(x, w_fp4, w_e8m0, out_dtype=torch.bfloat16, ws=None, out=None):
 
 
 def attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen):
-    tile, ns = _i32(0), _i32(0)
-    _check(lib().msd_attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen, C.byref(tile), C.byref(ns)), "msd_attn_decode_schedule")
-    return tile.value, ns.value
+    tile, ns, st = _i32(0), _i32(0), _i32(0)
+    _check(lib().msd_attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen, C.byref(tile), C.byref(ns), C.byref(st)),
+           "msd_attn_decode_schedule")
+    return tile.value, ns.value, st.value
 
 
 def attn_decode_int8kv_workspace_bytes(B, Hq, Hkv, D, Dv, max_seqlen):

@@ -18,6 +18,7 @@
 #include <cstdlib>
 
 #include "host_common.h"
+#include "quant.cuh"
 #include "sm100.cuh"
 
 namespace msd {
@@ -36,12 +37,18 @@ struct AttnParams {
   int B, Hq, Hkv, D, Dv, G;
   int HG, Rp, groups;     // heads per CTA, stacked rows, head groups per KV head
   int DC, DVT;            // 128-byte chunks of D / Dv
-  int n_splits, stages;
+  int n_splits, stages, chunk;   // chunk: tokens per split (a multiple of the tile)
   int v_alias;            // 1: V is the first Dv bytes of the K rows
   int tmem_cols;
   float scale;
   unsigned* status;
+  long long* trace;       // nullable diagnostic buffer: 32 clock samples per CTA (first 1024 CTAs)
 };
+
+__device__ __forceinline__ void attn_mark(const AttnParams& p, int slot) {
+  const int cta = blockIdx.y * gridDim.x + blockIdx.x;
+  if (p.trace && cta < 1024) p.trace[cta * 32 + slot] = clock64();
+}
 
 __device__ __forceinline__ int swz_off(int row, int byte_in_row) {
   // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
@@ -73,13 +80,18 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   const int b = unit / p.Hkv;
   const int seq0 = p.cu[b];
   const int L = p.cu[b + 1] - seq0;
-  const int per = (L + p.n_splits - 1) / p.n_splits;
-  const int Lsplit = (per + kTok - 1) / kTok * kTok;
-  const int t_begin = split * Lsplit;
-  const int t_end = min(L, t_begin + Lsplit);
+  const int t_begin = split * p.chunk;                       // every split covers the same number of tokens
+  const int t_end = min(L, t_begin + p.chunk);
   const int h0 = hk * p.G + grp * p.HG;                      // first query head of this CTA
   const int nh = min(p.HG, p.G - grp * p.HG);                // heads actually present
   const int ntiles = (t_end > t_begin) ? (t_end - t_begin + kTok - 1) / kTok : 0;
+  if (threadIdx.x == 0 && p.trace) {
+    attn_mark(p, 0);
+    unsigned long long g;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g));
+    const int cta = blockIdx.y * gridDim.x + blockIdx.x;
+    if (cta < 1024) { p.trace[cta * 32 + 1] = static_cast<long long>(g); p.trace[cta * 32 + 2] = ntiles; }
+  }
 
   if (ntiles == 0) {      // nothing in this split: neutral partials, before any barrier or TMEM use
     for (int i = threadIdx.x; i < nh * (p.Dv + 2); i += blockDim.x) {
@@ -188,14 +200,15 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
       const float alpha = __fdiv_rn(m, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
+      const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f, inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
       if (lane == 0) { s_aq[h] = alpha; s_bq[h] = beta; }
       for (int d = lane; d < p.D; d += 32) {
         const float v = __uint_as_float(static_cast<uint32_t>(qrow[d]) << 16);
         int c1 = 0, c2 = 0;
         if (alpha > 0.0f) {
-          c1 = max(-128, min(127, __float2int_rn(__fdiv_rn(v, alpha))));
+          c1 = quant_i8(v, alpha, inv_alpha);                         // same bit-exact rule as msd_decompose_int8
           const float r = __fmaf_rn(-alpha, static_cast<float>(c1), v);
-          if (beta > 0.0f) c2 = max(-128, min(127, __float2int_rn(__fdiv_rn(r, beta))));
+          if (beta > 0.0f) c2 = quant_i8(r, beta, inv_beta);
         }
         uint8_t* chunk = sm_q + (d >> 7) * p.Rp * kChunk;
         chunk[swz_off(h, d & 127)] = static_cast<uint8_t>(c1);
@@ -206,6 +219,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     __syncwarp();
     if (lane == 0) mbar_arrive(&p_full);            // phase 0 of p_full: "Q operand ready"
     named_bar_sync(1, 128);                         // s_aq / s_bq visible to all four warps
+    if (threadIdx.x == 64) attn_mark(p, 3);
 
     // running state per head; scores are kept in the log2 domain (log2(e) is folded into the key scale)
     float m_run[kNH], l_part[kNH], aq[kNH], bq[kNH];
@@ -228,6 +242,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       const float vs = valid ? __ldg(p.v_scale + sidx) : 0.0f;
       ok = wait_bounded(&s_full[t & 1], (t >> 1) & 1, abort, p.status);
       if (!ok) break;
+      if (threadIdx.x == 64 && t < 6) attn_mark(p, 4 + 4 * t);
       tc_fence_after();
       // c3: merge the two integer products and apply the key scale
       float s[kNH];
@@ -286,9 +301,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&p_full);
+      if (threadIdx.x == 64 && t < 6) attn_mark(p, 5 + 4 * t);
       // c6/c7: wait for O^T of this tile, merge it into the running output with the rescale factors
       ok = wait_bounded(&o_full, t & 1, abort, p.status);
       if (!ok) break;
+      if (threadIdx.x == 64 && t < 6) attn_mark(p, 6 + 4 * t);
       tc_fence_after();
 #pragma unroll
       for (int j = 0; j < kMaxDVT; ++j) {
@@ -306,7 +323,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&o_empty);
+      if (threadIdx.x == 64 && t < 6) attn_mark(p, 7 + 4 * t);
     }
+    if (threadIdx.x == 64) attn_mark(p, 28);
     // partial results of this split: running max, sum of P and unnormalised output per head
     if (ok) {
       float (*rb)[kNH + 1] = red[ntiles & 1];
@@ -335,13 +354,17 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) attn_mark(p, 29);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, p.tmem_cols);
   }
 }
 
+static long long* g_attn_trace = nullptr;
+
 // c8: merge the splits of one (sequence, query head) and normalise:  O = sum_s e^{m_s - m} O_s / sum_s e^{m_s - m} l_s
+// (a separate small kernel: letting the last-arriving split do it inside the attention kernel measured slower)
 __global__ void __launch_bounds__(128)
 attn_combine_kernel(const float* __restrict__ partial, int n_splits, int Dv, __nv_bfloat16* __restrict__ out,
                     float* __restrict__ lse) {
@@ -366,8 +389,8 @@ attn_combine_kernel(const float* __restrict__ partial, int n_splits, int Dv, __n
 }
 
 struct AttnPlan {
-  int HG, Rp, groups, DC, DVT, n_splits, stages, tmem_cols, v_alias;
-  size_t smem_bytes, ws_bytes;
+  int HG, Rp, groups, DC, DVT, n_splits, stages, tmem_cols, v_alias, chunk;
+  size_t smem_bytes, ws_bytes, ws_partial_bytes;
 };
 
 static int attn_env_int(const char* name, int fallback) {
@@ -390,26 +413,36 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   const int kv_stage = (pl->DC + (v_alias ? 0 : pl->DVT)) * kChunkBytes;
   const size_t fixed = static_cast<size_t>(pl->DC) * pl->Rp * kChunk + pl->Rp * kChunk + 1024;
   pl->stages = (2 * static_cast<size_t>(kv_stage) + fixed <= 227 * 1024 - 2048) ? 2 : 1;
+  // Splits of equal size (a fixed number of tiles) keep the CTAs' work uniform whatever the mix of sequence lengths;
+  // the size is shrunk until there are enough splits to fill the machine a few times over.
   const int tiles = (max_seqlen + kTok - 1) / kTok;
   const long long units = static_cast<long long>(B) * Hkv * pl->groups;
-  int ns = static_cast<int>((static_cast<long long>(sm_count()) * 6 + units - 1) / units);
-  if (ns > tiles) ns = tiles;
+  int chunk_tiles = attn_env_int("MSD_ATTN_CHUNK_TILES", pl->Rp <= 16 ? 16 : 32);
+  if (chunk_tiles < 1) chunk_tiles = 1;
+  while (chunk_tiles > 2 && units * ((tiles + chunk_tiles - 1) / chunk_tiles) < static_cast<long long>(sm_count()) * 4) chunk_tiles >>= 1;
+  int ns = (tiles + chunk_tiles - 1) / chunk_tiles;
   if (ns < 1) ns = 1;
-  if (ns > 64) ns = 64;
-  ns = attn_env_int("MSD_ATTN_SPLITS", ns);
-  if (ns < 1) ns = 1;
+  if (const int forced = attn_env_int("MSD_ATTN_SPLITS", 0)) {      // testing aid: a given number of splits
+    ns = forced < 1 ? 1 : forced;
+    chunk_tiles = (tiles + ns - 1) / ns;
+    if (chunk_tiles < 1) chunk_tiles = 1;
+  }
   pl->n_splits = ns;
+  pl->chunk = chunk_tiles * kTok;
   pl->smem_bytes = static_cast<size_t>(pl->stages) * kv_stage + fixed;
   int cols = 32;
   while (cols < 2 * pl->Rp + pl->DVT * pl->Rp) cols <<= 1;
   pl->tmem_cols = cols;
-  pl->ws_bytes = round_up(static_cast<size_t>(B) * Hq * ns * (Dv + 2) * sizeof(float), 1024);
+  pl->ws_partial_bytes = round_up(static_cast<size_t>(B) * Hq * ns * (Dv + 2) * sizeof(float), 1024);
+  pl->ws_bytes = pl->ws_partial_bytes + round_up(static_cast<size_t>(units) * sizeof(unsigned), 1024);
   return pl->smem_bytes <= 227 * 1024 - 2048;
 }
 
 }  // namespace msd
 
 extern "C" {
+
+void msd_debug_set_attn_trace(void* device_buffer) { msd::g_attn_trace = static_cast<long long*>(device_buffer); }
 
 size_t msd_attn_decode_int8kv_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen) {
   msd::AttnPlan pl;
@@ -418,12 +451,13 @@ size_t msd_attn_decode_int8kv_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv
 }
 
 msd_status_t msd_attn_decode_schedule(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen,
-                                      int32_t* tile, int32_t* n_splits) {
+                                      int32_t* tile, int32_t* n_splits, int32_t* split_tokens) {
   msd::AttnPlan pl;
   if (!tile || !n_splits) return MSD_ERR_NULL_POINTER;
   if (!msd::plan_attn(B, Hq, Hkv, D, Dv, max_seqlen, false, &pl)) return MSD_ERR_BAD_SHAPE;
   *tile = msd::kTok;
   *n_splits = pl.n_splits;
+  if (split_tokens) *split_tokens = pl.chunk;
   return MSD_OK;
 }
 
@@ -466,9 +500,11 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
   p.partial = static_cast<float*>(workspace);
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.Dv = Dv; p.G = Hq / Hkv;
   p.HG = pl.HG; p.Rp = pl.Rp; p.groups = pl.groups; p.DC = pl.DC; p.DVT = pl.DVT;
+  p.chunk = pl.chunk;
   p.n_splits = pl.n_splits; p.stages = pl.stages; p.v_alias = pl.v_alias; p.tmem_cols = pl.tmem_cols;
   p.scale = softmax_scale;
   p.status = status;
+  p.trace = g_attn_trace;
 
   void (*kernel)(CUtensorMap, CUtensorMap, AttnParams) = nullptr;
   const int G = Hq / Hkv;
@@ -480,8 +516,21 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
     MSD_ATTN_PICK(16, 16);
   }
 #undef MSD_ATTN_PICK
-  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
-    return MSD_ERR_CUDA;
+  {
+    // raise the dynamic shared-memory limit once per kernel instantiation
+    static void* done[16] = {};
+    bool seen = false;
+    int free_slot = -1;
+    for (int i = 0; i < 16; ++i) {
+      if (done[i] == reinterpret_cast<void*>(kernel)) seen = true;
+      if (!done[i] && free_slot < 0) free_slot = i;
+    }
+    if (!seen) {
+      if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
+        return MSD_ERR_CUDA;
+      if (free_slot >= 0) done[free_slot] = reinterpret_cast<void*>(kernel);
+    }
+  }
   dim3 grid(pl.n_splits, B * Hkv * pl.groups);
   kernel<<<grid, kAttnThreads, pl.smem_bytes, s>>>(tmap_k, tmap_v, p);
   if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;

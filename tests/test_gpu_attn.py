@@ -12,11 +12,9 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-3
 
 
-def _split_starts(seqlens, tile, ns):
+def _split_starts(seqlens, ns, split_tokens):
     L = np.asarray(seqlens, dtype=np.int64)
-    per = -(-L // ns)
-    lsplit = -(-per // tile) * tile
-    return np.minimum(L[:, None], np.arange(ns + 1)[None, :] * lsplit[:, None]).astype(np.int32)
+    return np.minimum(L[:, None], np.arange(ns + 1)[None, :] * split_tokens).astype(np.int32)
 
 
 def _run_gpu(c, want_lse=True):
@@ -37,8 +35,8 @@ def _run_gpu(c, want_lse=True):
 def _oracle_tiled(c, B_sched=None, max_seqlen=None):
     B, Hq, D = c.q.shape
     Hkv = c.k.shape[1]
-    tile, ns = binding.attn_decode_schedule(B_sched or B, Hq, Hkv, D, c.dv, max(max_seqlen or c.max_seqlen, 1))
-    ss = _split_starts(np.diff(c.cu_seqlens), tile, ns)
+    tile, ns, st = binding.attn_decode_schedule(B_sched or B, Hq, Hkv, D, c.dv, max(max_seqlen or c.max_seqlen, 1))
+    ss = _split_starts(np.diff(c.cu_seqlens), ns, st)
     return oracle.attn_decode_int8kv(c.q, c.k, c.v, c.k_scale, c.v_scale, c.cu_seqlens, c.softmax_scale, dv=c.dv,
                                      mode="tiled", tile=tile, split_starts=ss, want_lse=True)
 
