@@ -55,22 +55,32 @@ __device__ __forceinline__ int swz_off(int row, int byte_in_row) {
   return row * 128 + ((((byte_in_row >> 4) ^ (row & 7)) & 7) << 4) + (byte_in_row & 15);
 }
 
+// 2^x for x <= 0 (flushes tiny results to zero): one MUFU instruction
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // order-preserving float <-> int map (an involution), so that a warp maximum can use the integer redux instruction
 __device__ __forceinline__ int f2ord(float f) { const int i = __float_as_int(f); return i ^ ((i >> 31) & 0x7fffffff); }
 __device__ __forceinline__ float ord2f(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
 __device__ __forceinline__ float warp_max(float v) { return ord2f(__reduce_max_sync(0xffffffffu, f2ord(v))); }
 
-// kMaxHG: head slots of the stacked operand (8 or 16); kNH: heads the code is unrolled for (<= kMaxHG);
-// kMaxDVT: 128-wide tiles of Dv.
-template <int kMaxHG, int kNH, int kMaxDVT>
-__global__ void __launch_bounds__(kAttnThreads, (kNH <= 8 && kMaxDVT == 1) ? 3 : 1)
+// kMaxHG: head slots one softmax thread looks after (8 or 16); kNH: heads its code is unrolled for (<= kMaxHG);
+// kMaxDVT: 128-wide tiles of Dv; kWG: groups of four softmax warps, each owning kMaxHG of the CTA's kMaxHG*kWG
+// head slots (two groups let one CTA serve 32 heads of a KV head with one pass over its KV tiles).
+template <int kMaxHG, int kNH, int kMaxDVT, int kWG>
+__global__ void __launch_bounds__(64 + 128 * kWG, (kNH <= 8 && kMaxDVT == 1 && kWG == 1) ? 3 : 1)
 attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
   extern __shared__ uint8_t smem_dyn[];
-  __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], s_full[2], p_full, o_full, o_empty;
+  __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], s_full[2], p_full[2], q_ready, o_full, o_empty;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
-  __shared__ float s_aq[kMaxHG], s_bq[kMaxHG];
-  __shared__ float red[2][4][kNH + 1];             // per-warp tile maxima, double buffered by tile parity
+  constexpr int kSlots = kMaxHG * kWG;             // head slots of the stacked operands: rows [0,kSlots) first
+  constexpr int kNSW = 4 * kWG;                    // component, rows [kSlots, 2*kSlots) second component
+  __shared__ float s_aq[kSlots], s_bq[kSlots];
+  __shared__ float red[2][kWG][4][kNH + 1];        // per-warp tile maxima, double buffered by tile parity
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x;
@@ -110,7 +120,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
     mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1);
-    mbar_init(&p_full, 4); mbar_init(&o_full, 1); mbar_init(&o_empty, 4);
+    // one P barrier per P buffer: the softmax may run one tile ahead of the PV issue, and a single barrier could then
+    // be two phases past the one the MMA warp is testing, which a parity test cannot tell from "not yet"
+    mbar_init(&p_full[0], kNSW); mbar_init(&p_full[1], kNSW); mbar_init(&q_ready, kNSW);
+    mbar_init(&o_full, 1); mbar_init(&o_empty, kNSW);
     abort_flag = 0;
     mbar_init_fence();
     tma_prefetch_desc(&tmap_k);
@@ -149,10 +162,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       const uint32_t idesc_pv = idesc_dense(2, 1, 1, 1, 0, kTok, p.Rp);     // A (V^T) MN-major
       bool ok = true;
       // the stacked Q operand is written by the softmax warps; they arrive on p_full once before the first tile
-      ok = wait_bounded(&p_full, 0, abort, p.status);
+      ok = wait_bounded(&q_ready, 0, abort, p.status);
       auto issue_qk = [&](int t) {
         const int st = t % p.stages;
-        if (!wait_bounded(&kv_full[st], (t / p.stages) & 1, abort, p.status)) return false;
         tc_fence_after();
         const uint32_t ka = smem_u32(smem + st * kv_stage_bytes);
         const uint32_t qa = smem_u32(sm_q);
@@ -163,20 +175,12 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             mma_i8(d, smem_desc(ka + c * kChunkBytes + k * 32, 16, 1024, kSwizzle128B),
                    smem_desc(qa + c * p.Rp * kChunk + k * 32, 16, 1024, kSwizzle128B), idesc_qk, (c > 0 || k > 0) ? 1u : 0u);
         tc_commit(&s_full[t & 1]);
-        return true;
       };
-      if (ok) ok = issue_qk(0);
-      for (int t = 0; t < ntiles && ok; ++t) {
-        // with two KV stages the next tile's QK^T overlaps this tile's softmax; with one it must wait for PV below
-        if (p.stages >= 2 && t + 1 < ntiles) { ok = issue_qk(t + 1); if (!ok) break; }
-        ok = wait_bounded(&p_full, (t + 1) & 1, abort, p.status);             // P of tile t is in shared memory
-        if (!ok) break;
-        ok = wait_bounded(&o_empty, (t & 1) ^ 1, abort, p.status);           // O^T of tile t-1 has been merged
-        if (!ok) break;
+      auto issue_pv = [&](int t) {
         tc_fence_after();
         const int st = t % p.stages;
         const uint32_t va = smem_u32(smem + st * kv_stage_bytes) + (p.v_alias ? 0 : p.DC * kChunkBytes);
-        const uint32_t pa = smem_u32(sm_p);
+        const uint32_t pa = smem_u32(sm_p) + (t & 1) * p.Rp * kChunk;
         for (int j = 0; j < p.DVT; ++j)
 #pragma unroll
           for (int k = 0; k < 4; ++k)        // 32 tokens per MMA: four 8-token groups of 1024 bytes
@@ -184,42 +188,100 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                    smem_desc(pa + k * 32, 16, 1024, kSwizzle128B), idesc_pv, k > 0 ? 1u : 0u);
         tc_commit(&o_full);
         tc_commit(&kv_empty[st]);
-        if (p.stages < 2 && t + 1 < ntiles) ok = issue_qk(t + 1);
+      };
+      // Two streams of work, each in tile order, issued as soon as their inputs are there (whichever comes first):
+      //   QK^T(q) needs the KV tile q in shared memory and the score buffer q&1 drained (P of tile q-2 written);
+      //   PV(v)   needs P of tile v written, O^T of tile v-1 merged, and QK^T(v) already issued.
+      // A QK^T that waits for its KV tile must not hold back a PV whose operands are ready, and vice versa.
+      int q = 0, v = 0;
+      long long t_idle = clock64();
+      while (ok && v < ntiles) {
+        bool progressed = false;
+        if (q < ntiles && q < v + 2 &&
+            mbar_try_wait(&kv_full[q % p.stages], (q / p.stages) & 1)) {    // (q < v + 2 implies P of tile q-2 is written)
+          issue_qk(q);
+          ++q;
+          progressed = true;
+        }
+        if (v < q && mbar_try_wait(&p_full[v & 1], (v >> 1) & 1) && (v == 0 || mbar_try_wait(&o_empty, (v - 1) & 1))) {
+          issue_pv(v);
+          ++v;
+          progressed = true;
+        }
+        if (progressed) {
+          t_idle = clock64();
+        } else {
+          if (*abort) { ok = false; break; }
+          if (clock64() - t_idle > kWaitBudgetCycles) {
+            *abort = 1;
+            atomicMax(p.status, kStatusTimeout);
+            ok = false;
+          }
+        }
       }
     }
   } else {
     // ------------------------------ softmax + merge warps ------------------------------
     const int quad = warp & 3;
     const int tl = quad * 32 + lane;                // token lane (softmax) / dv lane (merge)
-    const int wi = warp - 2;                        // 0..3
+    const int wi = warp - 2;                        // 0 .. kNSW-1
+    const int hh = wi >> 2;                         // which group of head slots this warp looks after
+    const int wq = wi & 3;
+    const int hs0 = hh * kMaxHG;                    // its first head slot
     // c1: decompose the query rows of this CTA's heads (one warp per head, round robin) into the stacked operand
-    for (int h = wi; h < nh; h += 4) {
-      const uint16_t* qrow = p.q + (static_cast<long long>(b) * p.Hq + h0 + h) * p.D;
+    for (int h = wi; h < nh; h += kNSW) {
+      const uint4* qrow = reinterpret_cast<const uint4*>(p.q + (static_cast<long long>(b) * p.Hq + h0 + h) * p.D);
+      const int nvec = p.D >> 3;                    // 8 BF16 values per 16-byte load (D % 16 == 0, D <= 640)
+      uint4 qv[3];                                  // the whole row stays in registers between the two passes
       float m = 0.0f;
-      for (int d = lane; d < p.D; d += 32) m = fmaxf(m, fabsf(__uint_as_float(static_cast<uint32_t>(qrow[d]) << 16)));
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      for (int j = 0; j < 3; ++j) {
+        const int i = lane + 32 * j;
+        qv[j] = (i < nvec) ? __ldg(qrow + i) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int j = 0; j < 3; ++j) {
+        const uint32_t w[4] = {qv[j].x, qv[j].y, qv[j].z, qv[j].w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          m = fmaxf(m, fabsf(__uint_as_float(w[k] << 16)));
+          m = fmaxf(m, fabsf(__uint_as_float(w[k] & 0xFFFF0000u)));
+        }
+      }
+      m = warp_max(m);
       const float alpha = __fdiv_rn(m, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
       const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f, inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
       if (lane == 0) { s_aq[h] = alpha; s_bq[h] = beta; }
-      for (int d = lane; d < p.D; d += 32) {
-        const float v = __uint_as_float(static_cast<uint32_t>(qrow[d]) << 16);
-        int c1 = 0, c2 = 0;
-        if (alpha > 0.0f) {
-          c1 = quant_i8(v, alpha, inv_alpha);                         // same bit-exact rule as msd_decompose_int8
-          const float r = __fmaf_rn(-alpha, static_cast<float>(c1), v);
-          if (beta > 0.0f) c2 = quant_i8(r, beta, inv_beta);
+#pragma unroll
+      for (int j = 0; j < 3; ++j) {
+        const int i = lane + 32 * j;
+        if (i >= nvec) continue;
+        const uint32_t w[4] = {qv[j].x, qv[j].y, qv[j].z, qv[j].w};
+        uint32_t o1[2] = {0, 0}, o2[2] = {0, 0};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float x = (e & 1) ? __uint_as_float(w[e >> 1] & 0xFFFF0000u) : __uint_as_float(w[e >> 1] << 16);
+          int c1 = 0, c2 = 0;
+          if (alpha > 0.0f) {
+            c1 = quant_i8(x, alpha, inv_alpha);                       // same bit-exact rule as msd_decompose_int8
+            const float r = __fmaf_rn(-alpha, static_cast<float>(c1), x);
+            if (beta > 0.0f) c2 = quant_i8(r, beta, inv_beta);
+          }
+          o1[e >> 2] |= static_cast<uint32_t>(c1 & 0xFF) << (8 * (e & 3));
+          o2[e >> 2] |= static_cast<uint32_t>(c2 & 0xFF) << (8 * (e & 3));
         }
+        const int d = i << 3;                       // eight consecutive bytes stay inside one 16-byte swizzle chunk
         uint8_t* chunk = sm_q + (d >> 7) * p.Rp * kChunk;
-        chunk[swz_off(h, d & 127)] = static_cast<uint8_t>(c1);
-        chunk[swz_off(p.HG + h, d & 127)] = static_cast<uint8_t>(c2);
+        *reinterpret_cast<uint2*>(chunk + swz_off(h, d & 127)) = make_uint2(o1[0], o1[1]);
+        *reinterpret_cast<uint2*>(chunk + swz_off(kSlots + h, d & 127)) = make_uint2(o2[0], o2[1]);
       }
     }
     fence_proxy_async_smem();
     __syncwarp();
-    if (lane == 0) mbar_arrive(&p_full);            // phase 0 of p_full: "Q operand ready"
-    named_bar_sync(1, 128);                         // s_aq / s_bq visible to all four warps
+    if (lane == 0) mbar_arrive(&q_ready);           // the stacked Q operand is in shared memory
+    named_bar_sync(3, 128 * kWG);                   // s_aq / s_bq visible to all softmax warps
     if (threadIdx.x == 64) attn_mark(p, 3);
+    const int bar_id = 1 + hh;                      // each group of four warps synchronises on its own
 
     // running state per head; scores are kept in the log2 domain (log2(e) is folded into the key scale)
     float m_run[kNH], l_part[kNH], aq[kNH], bq[kNH];
@@ -227,82 +289,91 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
     for (int h = 0; h < kNH; ++h) {
       m_run[h] = -INFINITY; l_part[h] = 0.0f;
-      aq[h] = (h < nh) ? s_aq[h] : 0.0f; bq[h] = (h < nh) ? s_bq[h] : 0.0f;
+      aq[h] = (hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f; bq[h] = (hs0 + h < nh) ? s_bq[hs0 + h] : 0.0f;
 #pragma unroll
       for (int j = 0; j < kMaxDVT; ++j) o_run[j][h] = 0.0f;
     }
     const float kLog2e = 1.4426950408889634f;
     const float scale2 = p.scale * kLog2e;
     bool ok = true;
-    for (int t = 0; t < ntiles && ok; ++t) {
+    // State a tile's softmax hands to its merge: rescale factors and the P scales.  The softmax of tile t+1 runs
+    // BEFORE the merge of tile t (it overlaps the PV product of tile t), so two sets are alive at a time.
+    float resc_cur[kNH], resc_nxt[kNH];
+    float ap_cur = 0.0f, bp_cur = 0.0f, ap_nxt = 0.0f, bp_nxt = 0.0f;
+
+    // c3-c5 for tile t: scores -> running max -> P -> two INT8 components into P buffer (t & 1)
+    auto softmax_tile = [&](int t, float (&resc)[kNH], float& alpha_p, float& beta_p) -> bool {
       const int tok_rel = t_begin + t * kTok + tl;
       const bool valid = tok_rel < t_end;
       const long long sidx = static_cast<long long>(seq0 + tok_rel) * p.Hkv + hk;
       const float ks = valid ? __ldg(p.k_scale + sidx) * scale2 : 0.0f;
       const float vs = valid ? __ldg(p.v_scale + sidx) : 0.0f;
-      ok = wait_bounded(&s_full[t & 1], (t >> 1) & 1, abort, p.status);
-      if (!ok) break;
+      if (!wait_bounded(&s_full[t & 1], (t >> 1) & 1, abort, p.status)) return false;
       if (threadIdx.x == 64 && t < 6) attn_mark(p, 4 + 4 * t);
       tc_fence_after();
-      // c3: merge the two integer products and apply the key scale
       float s[kNH];
       const uint32_t srow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + (t & 1) * p.Rp;
       {
         uint32_t v1[kMaxHG], v2[kMaxHG];          // first / second component columns
-        tmem_ldw<kMaxHG>(srow, v1);
-        tmem_ldw<kMaxHG>(srow + kMaxHG, v2);
+        tmem_ldw<kMaxHG>(srow + hs0, v1);
+        tmem_ldw<kMaxHG>(srow + kSlots + hs0, v2);
         tmem_ld_wait();
 #pragma unroll
         for (int h = 0; h < kNH; ++h)
           s[h] = valid ? __fmaf_rn(aq[h], static_cast<float>(static_cast<int32_t>(v1[h])), bq[h] * static_cast<float>(static_cast<int32_t>(v2[h]))) * ks : -INFINITY;
       }
       // c4: tile maxima per head (and of the value scales) over the 128 token lanes
-      float (*rb)[kNH + 1] = red[t & 1];
+      float (*rb)[kNH + 1] = red[t & 1][hh];
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
         const float wm = warp_max(s[h]);
-        if (lane == 0) rb[wi][h] = wm;
+        if (lane == 0) rb[wq][h] = wm;
       }
       {
         const float wv = warp_max(vs);
-        if (lane == 0) rb[wi][kNH] = wv;
+        if (lane == 0) rb[wq][kNH] = wv;
       }
-      named_bar_sync(1, 128);      // one barrier per tile: the other parity buffer is rewritten only after the next one
-      float resc[kNH];
+      named_bar_sync(bar_id, 128);  // one barrier per tile: the other parity buffer is rewritten only after the next one
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
         const float mt = fmaxf(fmaxf(rb[0][h], rb[1][h]), fmaxf(rb[2][h], rb[3][h]));
         const float mn = fmaxf(m_run[h], mt);
-        resc[h] = (m_run[h] == -INFINITY) ? 0.0f : exp2f(m_run[h] - mn);
+        resc[h] = (m_run[h] == -INFINITY) ? 0.0f : ex2_approx(m_run[h] - mn);
         m_run[h] = mn;
       }
       const float vs_max = fmaxf(fmaxf(rb[0][kNH], rb[1][kNH]), fmaxf(rb[2][kNH], rb[3][kNH]));
       // c5: P = exp(S - m), fold the value scale, two-pass INT8 with the fixed scale alpha_P = max(v_scale)/127
-      const float alpha_p = __fdiv_rn(vs_max, 127.0f), beta_p = __fdiv_rn(alpha_p, 254.0f);
-      const float inv_a = alpha_p > 0.0f ? 1.0f / alpha_p : 0.0f, inv_b = beta_p > 0.0f ? 1.0f / beta_p : 0.0f;
-      // the previous tile's PV has finished reading the P operand: these threads waited for its o_full before merging
+      alpha_p = vs_max * (1.0f / 127.0f);
+      beta_p = alpha_p * (1.0f / 254.0f);
+      const float inv_a = alpha_p > 0.0f ? __frcp_rn(alpha_p) : 0.0f, inv_b = beta_p > 0.0f ? __frcp_rn(beta_p) : 0.0f;
+      uint8_t* pbuf = sm_p + (t & 1) * p.Rp * kChunk;      // PV of tile t-2 (same buffer) finished before merge(t-2)
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
-        int c1 = 0, c2 = 0;
-        if (h < nh && valid) {
-          const float pr = exp2f(s[h] - m_run[h]);
-          l_part[h] = __fmaf_rn(l_part[h], resc[h], pr);
-          const float pt = pr * vs;
-          c1 = max(-128, min(127, __float2int_rn(pt * inv_a)));
-          const float r = __fmaf_rn(-alpha_p, static_cast<float>(c1), pt);
-          c2 = max(-128, min(127, __float2int_rn(r * inv_b)));
-        } else {
-          l_part[h] *= resc[h];
-        }
-        sm_p[swz_off(h, tl)] = static_cast<uint8_t>(c1);
-        sm_p[swz_off(kMaxHG + h, tl)] = static_cast<uint8_t>(c2);
+        // branch-free: an absent head or a token past the end contributes P = 0 (s is -inf there)
+        const float pr = (hs0 + h < nh) ? ex2_approx(s[h] - m_run[h]) : 0.0f;
+        l_part[h] = __fmaf_rn(l_part[h], resc[h], pr);
+        const float pt = pr * vs;
+        const int c1 = min(127, __float2int_rn(pt * inv_a));
+        const float r = __fmaf_rn(-alpha_p, static_cast<float>(c1), pt);
+        const int c2 = max(-128, min(127, __float2int_rn(r * inv_b)));
+        pbuf[swz_off(hs0 + h, tl)] = static_cast<uint8_t>(c1);
+        pbuf[swz_off(kSlots + hs0 + h, tl)] = static_cast<uint8_t>(c2);
       }
       fence_proxy_async_smem();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&p_full);
+      if (lane == 0) mbar_arrive(&p_full[t & 1]);
       if (threadIdx.x == 64 && t < 6) attn_mark(p, 5 + 4 * t);
-      // c6/c7: wait for O^T of this tile, merge it into the running output with the rescale factors
+      return true;
+    };
+
+    ok = softmax_tile(0, resc_cur, ap_cur, bp_cur);
+    for (int t = 0; t < ntiles && ok; ++t) {
+      if (t + 1 < ntiles) {
+        ok = softmax_tile(t + 1, resc_nxt, ap_nxt, bp_nxt);     // overlaps the PV product of tile t
+        if (!ok) break;
+      }
+      // c6/c7: wait for O^T of tile t, merge it into the running output with that tile's rescale factors
       ok = wait_bounded(&o_full, t & 1, abort, p.status);
       if (!ok) break;
       if (threadIdx.x == 64 && t < 6) attn_mark(p, 6 + 4 * t);
@@ -312,36 +383,40 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         if (j < p.DVT) {
           const uint32_t orow = tmem_o + (static_cast<uint32_t>(quad * 32) << 16) + j * p.Rp;
           uint32_t v1[kMaxHG], v2[kMaxHG];
-          tmem_ldw<kMaxHG>(orow, v1);
-          tmem_ldw<kMaxHG>(orow + kMaxHG, v2);
+          tmem_ldw<kMaxHG>(orow + hs0, v1);
+          tmem_ldw<kMaxHG>(orow + kSlots + hs0, v2);
           tmem_ld_wait();
 #pragma unroll
           for (int h = 0; h < kNH; ++h)
-            o_run[j][h] = __fmaf_rn(o_run[j][h], resc[h], __fmaf_rn(alpha_p, static_cast<float>(static_cast<int32_t>(v1[h])), beta_p * static_cast<float>(static_cast<int32_t>(v2[h]))));
+            o_run[j][h] = __fmaf_rn(o_run[j][h], resc_cur[h], __fmaf_rn(ap_cur, static_cast<float>(static_cast<int32_t>(v1[h])), bp_cur * static_cast<float>(static_cast<int32_t>(v2[h]))));
         }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&o_empty);
       if (threadIdx.x == 64 && t < 6) attn_mark(p, 7 + 4 * t);
+#pragma unroll
+      for (int h = 0; h < kNH; ++h) resc_cur[h] = resc_nxt[h];
+      ap_cur = ap_nxt;
+      bp_cur = bp_nxt;
     }
     if (threadIdx.x == 64) attn_mark(p, 28);
     // partial results of this split: running max, sum of P and unnormalised output per head
     if (ok) {
-      float (*rb)[kNH + 1] = red[ntiles & 1];
-      named_bar_sync(1, 128);
+      float (*rb)[kNH + 1] = red[ntiles & 1][hh];
+      named_bar_sync(bar_id, 128);
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
         float l = l_part[h];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-        if (lane == 0) rb[wi][h] = l;
+        if (lane == 0) rb[wq][h] = l;
       }
-      named_bar_sync(1, 128);
+      named_bar_sync(bar_id, 128);
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
-        if (h < nh) {
-          float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + h) * p.n_splits + split) * (p.Dv + 2);
+        if (hs0 + h < nh) {
+          float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + hs0 + h) * p.n_splits + split) * (p.Dv + 2);
           // the running maximum goes out in natural-log units (it was kept in the log2 domain)
           if (tl == 0) { dst[0] = m_run[h] * 0.6931471805599453f; dst[1] = rb[0][h] + rb[1][h] + rb[2][h] + rb[3][h]; }
 #pragma unroll
@@ -401,7 +476,7 @@ static int attn_env_int(const char* name, int fallback) {
 static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, bool v_alias, AttnPlan* pl) {
   if (B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || D < 16 || D % 16 != 0 || Dv < 16 || Dv % 16 != 0) return false;
   const int G = Hq / Hkv;
-  pl->HG = (G <= 8) ? 8 : 16;
+  pl->HG = (G <= 8) ? 8 : (G <= 16 ? 16 : 32);
   pl->Rp = 2 * pl->HG;
   pl->groups = (G + pl->HG - 1) / pl->HG;
   pl->DC = (D + kChunk - 1) / kChunk;
@@ -411,7 +486,7 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   if (v_alias && Dv > D) return false;
   pl->v_alias = v_alias ? 1 : 0;
   const int kv_stage = (pl->DC + (v_alias ? 0 : pl->DVT)) * kChunkBytes;
-  const size_t fixed = static_cast<size_t>(pl->DC) * pl->Rp * kChunk + pl->Rp * kChunk + 1024;
+  const size_t fixed = static_cast<size_t>(pl->DC) * pl->Rp * kChunk + 2 * pl->Rp * kChunk + 1024;   // Q stack, two P buffers
   pl->stages = (2 * static_cast<size_t>(kv_stage) + fixed <= 227 * 1024 - 2048) ? 2 : 1;
   // Splits of equal size (a fixed number of tiles) keep the CTAs' work uniform whatever the mix of sequence lengths;
   // the size is shrunk until there are enough splits to fill the machine a few times over.
@@ -508,12 +583,17 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
 
   void (*kernel)(CUtensorMap, CUtensorMap, AttnParams) = nullptr;
   const int G = Hq / Hkv;
-#define MSD_ATTN_PICK(HG_, NH_) \
-  kernel = (pl.DVT == 1) ? attn_decode_kernel<HG_, NH_, 1> : (pl.DVT == 2) ? attn_decode_kernel<HG_, NH_, 2> : attn_decode_kernel<HG_, NH_, 4>
+#define MSD_ATTN_PICK(HG_, NH_, WG_) \
+  kernel = (pl.DVT == 1) ? attn_decode_kernel<HG_, NH_, 1, WG_> : (pl.DVT == 2) ? attn_decode_kernel<HG_, NH_, 2, WG_> \
+                                                                                  : attn_decode_kernel<HG_, NH_, 4, WG_>
+  int block_threads = kAttnThreads;
   if (pl.HG == 8) {
-    if (G <= 4) { MSD_ATTN_PICK(8, 4); } else { MSD_ATTN_PICK(8, 8); }
+    if (G <= 4) { MSD_ATTN_PICK(8, 4, 1); } else { MSD_ATTN_PICK(8, 8, 1); }
+  } else if (pl.HG == 16) {
+    MSD_ATTN_PICK(16, 16, 1);
   } else {
-    MSD_ATTN_PICK(16, 16);
+    MSD_ATTN_PICK(16, 16, 2);
+    block_threads = 64 + 128 * 2;
   }
 #undef MSD_ATTN_PICK
   {
@@ -532,7 +612,7 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
     }
   }
   dim3 grid(pl.n_splits, B * Hkv * pl.groups);
-  kernel<<<grid, kAttnThreads, pl.smem_bytes, s>>>(tmap_k, tmap_v, p);
+  kernel<<<grid, block_threads, pl.smem_bytes, s>>>(tmap_k, tmap_v, p);
   if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
   attn_combine_kernel<<<B * Hq, 128, 0, s>>>(p.partial, pl.n_splits, Dv, static_cast<__nv_bfloat16*>(out_bf16), lse);
   return launch_status();
