@@ -74,7 +74,7 @@ template <int kMaxHG, int kNH, int kMaxDVT, int kWG>
 __global__ void __launch_bounds__(64 + 128 * kWG, (kNH <= 8 && kMaxDVT == 1 && kWG == 1) ? 3 : 1)
 attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
   extern __shared__ uint8_t smem_dyn[];
-  __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], s_full[2], p_full[2], q_ready, o_full, o_empty;
+  __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], v_full[4], v_empty[4], s_full[2], p_full[2], q_ready, o_full, o_empty;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   constexpr int kSlots = kMaxHG * kWG;             // head slots of the stacked operands: rows [0,kSlots) first
@@ -118,7 +118,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   uint8_t* sm_p = sm_q + p.DC * p.Rp * kChunk;               // [Rp x 128]
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1);
+      mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
+    }
     mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1);
     // one P barrier per P buffer: the softmax may run one tile ahead of the PV issue, and a single barrier could then
     // be two phases past the one the MMA warp is testing, which a parity test cannot tell from "not yet"
@@ -142,17 +145,42 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   if (warp == 0) {
     // ------------------------------ TMA producer: K (and V) tiles ------------------------------
     if (lane == 0) {
-      int stage = 0; uint32_t phase = 0;
-      for (int t = 0; t < ntiles; ++t) {
-        if (!wait_bounded(&kv_empty[stage], phase ^ 1, abort, p.status)) break;
-        mbar_arrive_expect_tx(&kv_full[stage], kv_stage_bytes);
-        uint8_t* dst = smem + stage * kv_stage_bytes;
-        const int tok = seq0 + t_begin + t * kTok;
-        for (int c = 0; c < p.DC; ++c) tma_load_3d(dst + c * kChunkBytes, &tmap_k, c * kChunk, hk, tok, &kv_full[stage]);
-        if (!p.v_alias)
-          for (int j = 0; j < p.DVT; ++j)
-            tma_load_3d(dst + (p.DC + j) * kChunkBytes, &tmap_v, j * kChunk, hk, tok, &kv_full[stage]);
-        if (++stage == p.stages) { stage = 0; phase ^= 1; }
+      // K tiles and (when V is a separate cache) V tiles travel in rings of their own: a K buffer is free again as
+      // soon as QK^T has read it, long before the PV product of the same tile releases the V buffer, so the next K
+      // tile can be fetched that much earlier.  With V aliased to the K rows there is only the K ring.
+      const int k_bytes = p.DC * kChunkBytes, v_bytes = p.DVT * kChunkBytes;
+      int kq = 0, vq = p.v_alias ? ntiles : 0;
+      long long t_idle = clock64();
+      while (kq < ntiles || vq < ntiles) {
+        bool progressed = false;
+        if (kq < ntiles && mbar_try_wait(&kv_empty[kq % p.stages], ((kq / p.stages) & 1) ^ 1)) {
+          const int st = kq % p.stages;
+          mbar_arrive_expect_tx(&kv_full[st], k_bytes);
+          uint8_t* dst = smem + st * kv_stage_bytes;
+          const int tok = seq0 + t_begin + kq * kTok;
+          for (int c = 0; c < p.DC; ++c) tma_load_3d(dst + c * kChunkBytes, &tmap_k, c * kChunk, hk, tok, &kv_full[st]);
+          ++kq;
+          progressed = true;
+        }
+        if (vq < ntiles && mbar_try_wait(&v_empty[vq % p.stages], ((vq / p.stages) & 1) ^ 1)) {
+          const int st = vq % p.stages;
+          mbar_arrive_expect_tx(&v_full[st], v_bytes);
+          uint8_t* dst = smem + st * kv_stage_bytes + k_bytes;
+          const int tok = seq0 + t_begin + vq * kTok;
+          for (int j = 0; j < p.DVT; ++j) tma_load_3d(dst + j * kChunkBytes, &tmap_v, j * kChunk, hk, tok, &v_full[st]);
+          ++vq;
+          progressed = true;
+        }
+        if (progressed) {
+          t_idle = clock64();
+        } else {
+          if (*abort) break;
+          if (clock64() - t_idle > kWaitBudgetCycles) {
+            *abort = 1;
+            atomicMax(p.status, kStatusTimeout);
+            break;
+          }
+        }
       }
     }
   } else if (warp == 1) {
@@ -175,6 +203,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             mma_i8(d, smem_desc(ka + c * kChunkBytes + k * 32, 16, 1024, kSwizzle128B),
                    smem_desc(qa + c * p.Rp * kChunk + k * 32, 16, 1024, kSwizzle128B), idesc_qk, (c > 0 || k > 0) ? 1u : 0u);
         tc_commit(&s_full[t & 1]);
+        if (!p.v_alias) tc_commit(&kv_empty[st]);       // separate V: the K buffer is free once QK^T has read it
       };
       auto issue_pv = [&](int t) {
         tc_fence_after();
@@ -187,7 +216,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             mma_i8(tmem_o + j * p.Rp, smem_desc(va + j * kChunkBytes + k * 4096, 16384, 1024, kSwizzle128B),
                    smem_desc(pa + k * 32, 16, 1024, kSwizzle128B), idesc_pv, k > 0 ? 1u : 0u);
         tc_commit(&o_full);
-        tc_commit(&kv_empty[st]);
+        tc_commit(p.v_alias ? &kv_empty[st] : &v_empty[st]);
       };
       // Two streams of work, each in tile order, issued as soon as their inputs are there (whichever comes first):
       //   QK^T(q) needs the KV tile q in shared memory and the score buffer q&1 drained (P of tile q-2 written);
@@ -203,7 +232,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           ++q;
           progressed = true;
         }
-        if (v < q && mbar_try_wait(&p_full[v & 1], (v >> 1) & 1) && (v == 0 || mbar_try_wait(&o_empty, (v - 1) & 1))) {
+        if (v < q && mbar_try_wait(&p_full[v & 1], (v >> 1) & 1) && (v == 0 || mbar_try_wait(&o_empty, (v - 1) & 1)) &&
+            (p.v_alias || mbar_try_wait(&v_full[v % p.stages], (v / p.stages) & 1))) {
           issue_pv(v);
           ++v;
           progressed = true;
@@ -279,7 +309,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     fence_proxy_async_smem();
     __syncwarp();
     if (lane == 0) mbar_arrive(&q_ready);           // the stacked Q operand is in shared memory
-    named_bar_sync(3, 128 * kWG);                   // s_aq / s_bq visible to all softmax warps
+    named_bar_sync(8, 128 * kWG);                   // s_aq / s_bq visible to all softmax warps
     if (threadIdx.x == 64) attn_mark(p, 3);
     const int bar_id = 1 + hh;                      // each group of four warps synchronises on its own
 
@@ -591,9 +621,12 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
     if (G <= 4) { MSD_ATTN_PICK(8, 4, 1); } else { MSD_ATTN_PICK(8, 8, 1); }
   } else if (pl.HG == 16) {
     MSD_ATTN_PICK(16, 16, 1);
-  } else {
-    MSD_ATTN_PICK(16, 16, 2);
+  } else if (attn_env_int("MSD_ATTN_WIDE", 4) == 2) {
+    MSD_ATTN_PICK(16, 16, 2);          // 32 heads per CTA as two groups of four warps, 16 heads per thread
     block_threads = 64 + 128 * 2;
+  } else {
+    MSD_ATTN_PICK(8, 8, 4);            // 32 heads per CTA as four groups of four warps, 8 heads per thread
+    block_threads = 64 + 128 * 4;
   }
 #undef MSD_ATTN_PICK
   {
