@@ -50,10 +50,6 @@ __device__ __forceinline__ void attn_mark(const AttnParams& p, int slot) {
   if (p.trace && cta < 1024) p.trace[cta * 32 + slot] = clock64();
 }
 
-__device__ __forceinline__ int swz_off(int row, int byte_in_row) {
-  // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
-  return row * 128 + ((((byte_in_row >> 4) ^ (row & 7)) & 7) << 4) + (byte_in_row & 15);
-}
 
 // 2^x for x <= 0 (flushes tiny results to zero): one MUFU instruction
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -61,11 +57,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-
-// order-preserving float <-> int map (an involution), so that a warp maximum can use the integer redux instruction
-__device__ __forceinline__ int f2ord(float f) { const int i = __float_as_int(f); return i ^ ((i >> 31) & 0x7fffffff); }
-__device__ __forceinline__ float ord2f(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
-__device__ __forceinline__ float warp_max(float v) { return ord2f(__reduce_max_sync(0xffffffffu, f2ord(v))); }
 
 // kMaxHG: head slots one softmax thread looks after (8 or 16); kNH: heads its code is unrolled for (<= kMaxHG);
 // kMaxDVT: 128-wide tiles of Dv; kWG: groups of four softmax warps, each owning kMaxHG of the CTA's kMaxHG*kWG

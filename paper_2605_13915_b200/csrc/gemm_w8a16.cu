@@ -18,6 +18,7 @@
 #include <cstdlib>
 
 #include "host_common.h"
+#include "quant.cuh"
 #include "sm100.cuh"
 
 namespace msd {
@@ -46,6 +47,8 @@ struct GemmW8Params {
   const float* w_scale;
   const float* alpha;
   const float* beta;
+  const uint16_t* x;       // fused path only: the BF16 activations [M, ldx], decomposed inside the kernel
+  long long ldx;
   void* y;
   int32_t* acc_dbg;
   int32_t* accum;          // [num_tiles][NB][128] split-K meeting place, zero between calls (INT32 or FP32 bits)
@@ -129,8 +132,12 @@ __device__ __forceinline__ void partial_chunk(uint32_t t_row, int32_t* acc_tile,
 // kBase = false: the MSD path (INT8 x INT8 -> INT32, stacked components, scale-combine epilogue).
 // kBase = true : the comparison path the method replaces - the same pipeline on BF16 weights that a preceding kernel
 //                dequantized into the workspace, BF16 x BF16 -> FP32, no decomposition and no scales in the epilogue.
-template <bool kBase>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+// kFused (small M): no separate decomposition kernel - four extra warps compute the row scales and quantise the
+//                stacked operand tile of every stage straight into shared memory ("online activation decomposition",
+//                Sec. 3.9), so the activations never round-trip through HBM and nothing waits for a previous launch.
+constexpr int kFusedThreads = kGemmThreads + 128;
+template <bool kBase, bool kFused>
+__global__ void __launch_bounds__(kFused ? kFusedThreads : kGemmThreads, 1)
 gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_w2,
                   const __grid_constant__ CUtensorMap tmap_x, const GemmW8Params p) {
   extern __shared__ uint8_t smem_dyn[];
@@ -142,6 +149,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   __shared__ int abort_flag;
   __shared__ int is_last_flag;
   __shared__ float s_alpha[128], s_beta[128];
+  __shared__ float s_inva[8], s_invb[8], s_qmax[2][4];       // fused path: reciprocals of the scales, row-max scratch
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -161,7 +169,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.num_stages; ++s) {
-      mbar_init(&full_bar[s], 1);
+      mbar_init(&full_bar[s], kFused ? 2 : 1);     // fused: the producer's arrive plus the quantiser warp of the stage
       mbar_init(&empty_bar[s], 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -201,7 +209,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   // whole row instead of hitting the same 128-byte column of every row (integer sums do not depend on the order).
   const int kb_rot = (p.mode == 1) ? static_cast<int>((static_cast<long long>(blockIdx.x) * p.kb_rot_step) % p.kblocks) : 0;
   const CUtensorMap* wmap = (p.mode == 1 && band_h != p.hmax) ? &tmap_w2 : &tmap_w;
-  const int tx_bytes = p.kw * ((p.mode == 0 ? kWStageBytes : band_h * kBlockK) + x_chunk_bytes);
+  const int tx_bytes = p.kw * ((p.mode == 0 ? kWStageBytes : band_h * kBlockK) + (kFused ? 0 : x_chunk_bytes));
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -225,7 +233,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       trace_mark(p, 3);
       pdl_wait_primary();
       trace_mark(p, 4);
-      for (int i = 0; i < pre; ++i) {
+      for (int i = 0; i < pre && !kFused; ++i) {
         const int kb = static_cast<int>((blk_begin + i + kb_rot) % p.kblocks);
         for (int c = 0; c < p.kw; ++c)
           tma_load_2d_hint(smem + i * stage_bytes + w_stage_bytes + c * x_chunk_bytes, &tmap_x, (kb * p.kw + c) * kBlockK, 0,
@@ -243,7 +251,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         for (int c = 0; c < p.kw; ++c)
           tma_load_2d_hint(dst + c * p.w_chunk_bytes, wmap, (kb * p.kw + c) * kBlockK, band_row0 + tile * kTileN,
                            &full_bar[stage], pol_w);
-        for (int c = 0; c < p.kw; ++c)
+        for (int c = 0; c < p.kw && !kFused; ++c)
           tma_load_2d_hint(dst + w_stage_bytes + c * x_chunk_bytes, &tmap_x, (kb * p.kw + c) * kBlockK, 0, &full_bar[stage], pol_x);
         if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
       }
@@ -300,12 +308,91 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       }
       trace_mark(p, 7);
     }
+  } else if (kFused && warp >= 6) {
+    // ------------------------------ quantiser warps (fused path) ------------------------------
+    const int qt = threadIdx.x - kGemmThreads;    // 0..127
+    const int qw = warp - 6;
+    const int nvec_row = p.K >> 3;                // 16-byte vectors of 8 BF16 values per row
+    // a1: row maxima over the whole K, then alpha = max/127, beta = alpha/254 (Eq. alpha, Eq. beta)
+    for (int i = 0; i < p.M; ++i) {
+      const uint4* xr = reinterpret_cast<const uint4*>(p.x + static_cast<long long>(i) * p.ldx);
+      float m = 0.0f;
+      for (int c = qt; c < nvec_row; c += 128) {
+        const uint4 v = __ldg(xr + c);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          m = fmaxf(m, fabsf(__uint_as_float(w[k] << 16)));
+          m = fmaxf(m, fabsf(__uint_as_float(w[k] & 0xFFFF0000u)));
+        }
+      }
+      m = warp_max(m);
+      if (lane == 0) s_qmax[i & 1][qw] = m;
+      named_bar_sync(3, 128);
+      if (qt == 0) {
+        const float mm = fmaxf(fmaxf(s_qmax[i & 1][0], s_qmax[i & 1][1]), fmaxf(s_qmax[i & 1][2], s_qmax[i & 1][3]));
+        const float alpha = __fdiv_rn(mm, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
+        s_alpha[i] = alpha;
+        s_beta[i] = beta;
+        s_inva[i] = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f;
+        s_invb[i] = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
+      }
+    }
+    named_bar_sync(2, 256);                       // scales visible to the quantiser and the epilogue warps
+    // a2-a3: per stage, quantise the M x (kw*128) slice of X into the stacked operand tile (rows i and Mp+i).
+    // Each warp owns a fixed subset of the ring's stages (stage s belongs to warp s % 4) and fills them in order, so
+    // several stages are being filled at a time (one warp's load latency does not pace the pipeline) while every
+    // barrier is still waited on phase by phase by a single warp - a warp that could run two ring cycles ahead of
+    // another would make the parity test of the wait ambiguous.
+    const int vec_per_row = p.kw * 16;            // vectors of 8 elements per row and stage
+    const int nvec = p.M * vec_per_row;
+    bool ok = true;
+    for (long long blk = blk_begin; blk < blk_end && ok; ++blk) {
+      const long long it = blk - blk_begin;
+      const int stage = static_cast<int>(it % p.num_stages);
+      if ((stage & 3) != qw) continue;
+      const uint32_t phase = static_cast<uint32_t>((it / p.num_stages) & 1);
+      const int kb = static_cast<int>((blk + kb_rot) % p.kblocks);
+      ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
+      if (!ok) break;
+      uint8_t* xt = smem + stage * stage_bytes + w_stage_bytes;
+      for (int v = lane; v < nvec; v += 32) {
+        const int i = v / vec_per_row, r = v - i * vec_per_row;
+        const int c = r >> 4, e8 = r & 15;
+        const long long k = (static_cast<long long>(kb) * p.kw + c) * kBlockK + e8 * 8;
+        uint4 xv = make_uint4(0, 0, 0, 0);
+        if (k < p.K) xv = __ldg(reinterpret_cast<const uint4*>(p.x + static_cast<long long>(i) * p.ldx + k));
+        const float alpha = s_alpha[i], beta = s_beta[i], inva = s_inva[i], invb = s_invb[i];
+        const uint32_t w[4] = {xv.x, xv.y, xv.z, xv.w};
+        uint32_t o1[2] = {0, 0}, o2[2] = {0, 0};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float xf = (e & 1) ? __uint_as_float(w[e >> 1] & 0xFFFF0000u) : __uint_as_float(w[e >> 1] << 16);
+          int c1 = 0, c2 = 0;
+          if (alpha > 0.0f) {
+            c1 = quant_i8(xf, alpha, inva);                                  // Eq. x1
+            const float res = __fmaf_rn(-alpha, static_cast<float>(c1), xf); // Eq. residual (exact)
+            if (beta > 0.0f) c2 = quant_i8(res, beta, invb);                 // Eq. x2
+          }
+          o1[e >> 2] |= static_cast<uint32_t>(c1 & 0xFF) << (8 * (e & 3));
+          o2[e >> 2] |= static_cast<uint32_t>(c2 & 0xFF) << (8 * (e & 3));
+        }
+        uint8_t* dst = xt + c * x_chunk_bytes;
+        *reinterpret_cast<uint2*>(dst + swz_off(i, e8 * 8)) = make_uint2(o1[0], o1[1]);
+        *reinterpret_cast<uint2*>(dst + swz_off(p.Mp + i, e8 * 8)) = make_uint2(o2[0], o2[1]);
+      }
+      fence_proxy_async_smem();                   // the MMA reads this tile through the async proxy
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&full_bar[stage]);
+    }
   } else {
     // ------------------------------ epilogue (warps 2..5) ------------------------------
     const int quad = warp & 3;                    // TMEM lane group this warp may read
     const int r = quad * 32 + lane;               // weight row within the tile == TMEM lane
     const int et = threadIdx.x - 64;              // 0..127
-    if constexpr (!kBase) {
+    if constexpr (kFused) {
+      named_bar_sync(2, 256);                     // the quantiser warps have written s_alpha / s_beta
+    } else if constexpr (!kBase) {
       pdl_wait_primary();
       if (et < p.M) {
         s_alpha[et] = p.alpha[et];
@@ -337,7 +424,8 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         // add this CTA's partial sums into the tile's meeting place, then find out whether it was the last contributor
         acc_tile = p.accum + static_cast<long long>(tile) * p.NB * kTileN;
         int c0 = 0;
-        for (; c0 + 32 <= p.NB; c0 += 32) partial_chunk<kBase, 32>(t_row, acc_tile, c0, r);
+        if constexpr (!kFused)
+          for (; c0 + 32 <= p.NB; c0 += 32) partial_chunk<kBase, 32>(t_row, acc_tile, c0, r);
         if (c0 + 16 <= p.NB) partial_chunk<kBase, 16>(t_row, acc_tile, c0, r);
         named_bar_sync(1, 128);
         if (et == 0) {
@@ -355,8 +443,10 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       }
       if (finish) {
         int c0 = 0;
-        for (; c0 + 32 <= p.Mp; c0 += 32) epilogue_chunk<kBase, 32>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta);
-        if (c0 + 16 <= p.Mp) { epilogue_chunk<kBase, 16>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta); c0 += 16; }
+        if constexpr (!kFused) {
+          for (; c0 + 32 <= p.Mp; c0 += 32) epilogue_chunk<kBase, 32>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta);
+          if (c0 + 16 <= p.Mp) { epilogue_chunk<kBase, 16>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta); c0 += 16; }
+        }
         if (c0 + 8 <= p.Mp) epilogue_chunk<kBase, 8>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta);
       }
       tc_fence_before();
@@ -532,9 +622,15 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
   float* alpha = reinterpret_cast<float*>(ws + pl.off_alpha);
   float* beta = reinterpret_cast<float*>(ws + pl.off_beta);
 
-  // rows [0, M) of the stacked operand hold Q1, rows [Mp, Mp+M) hold Q2; the padding rows are never read back
-  st = launch_decompose_int8(x_bf16, M, K, K, q, q + static_cast<size_t>(pl.Mp) * K, alpha, beta, s);
-  if (st != MSD_OK) return st;
+  // Small M: the decomposition runs inside the GEMM kernel.  Otherwise a separate kernel writes the stacked operand:
+  // rows [0, M) hold Q1, rows [Mp, Mp+M) hold Q2; the padding rows are never read back.
+  // Opt-in (MSD_GEMM_FUSED_MAXM=<largest M>): with one quantiser warp per stage the in-kernel path measured no faster
+  // than the two-kernel path at M = 1 and slower from M = 2 on, so the default keeps the separate kernel.
+  const bool fused = (M <= env_int("MSD_GEMM_FUSED_MAXM", 0)) && M <= 8;
+  if (!fused) {
+    st = launch_decompose_int8(x_bf16, M, K, K, q, q + static_cast<size_t>(pl.Mp) * K, alpha, beta, s);
+    if (st != MSD_OK) return st;
+  }
 
   CUtensorMap tmap_w, tmap_w2, tmap_x;
   const uint32_t box2 = (pl.mode == 1 && pl.hmax > 8) ? pl.hmax - 8 : pl.hmax;
@@ -555,14 +651,23 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
   p.status = status;
   p.trace = g_trace;
 
+  p.x = static_cast<const uint16_t*>(x_bf16);
+  p.ldx = K;
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(gemm_w8a16_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_w8a16_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w8a16_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
       return MSD_ERR_CUDA;
     attr_done = true;
   }
+  if (fused) {
+    // a plain launch: this kernel reads x directly, so it must not start before earlier work in the stream is done
+    if (launch_pdl(gemm_w8a16_kernel<false, true>, dim3(pl.grid), dim3(kFusedThreads), pl.smem_bytes, s, false, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
+      return MSD_ERR_CUDA;
+    return MSD_OK;
+  }
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  if (launch_pdl(gemm_w8a16_kernel<false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
+  if (launch_pdl(gemm_w8a16_kernel<false, false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
     return MSD_ERR_CUDA;
   return MSD_OK;
 }
@@ -607,18 +712,19 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
   p.w_scale = w_scale; p.alpha = nullptr; p.beta = nullptr; p.y = y; p.acc_dbg = nullptr;
+  p.x = nullptr; p.ldx = 0;
   p.accum = reinterpret_cast<int32_t*>(ws + pl.off_slots);
   p.counters = reinterpret_cast<unsigned*>(ws + pl.off_counters);
   p.status = status;
   p.trace = nullptr;
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(gemm_w8a16_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_w8a16_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
       return MSD_ERR_CUDA;
     attr_done = true;
   }
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  if (launch_pdl(gemm_w8a16_kernel<true>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
+  if (launch_pdl(gemm_w8a16_kernel<true, false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
     return MSD_ERR_CUDA;
   return MSD_OK;
 }

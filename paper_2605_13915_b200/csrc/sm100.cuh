@@ -232,6 +232,18 @@ __device__ __forceinline__ void tmem_ldw(uint32_t taddr, uint32_t (&v)[W]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// Byte offset of (row, byte) in a tile of 128-byte rows under the 128-byte swizzle: the 16-byte chunk index is XORed
+// with the row index modulo 8 (what TMA writes and what the K-major / MN-major operand descriptors expect).
+__device__ __forceinline__ int swz_off(int row, int byte_in_row) {
+  // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
+  return row * 128 + ((((byte_in_row >> 4) ^ (row & 7)) & 7) << 4) + (byte_in_row & 15);
+}
+
+// order-preserving float <-> int map (an involution), so that a warp maximum can use the integer redux instruction
+__device__ __forceinline__ int f2ord(float f) { const int i = __float_as_int(f); return i ^ ((i >> 31) & 0x7fffffff); }
+__device__ __forceinline__ float ord2f(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
+__device__ __forceinline__ float warp_max(float v) { return ord2f(__reduce_max_sync(0xffffffffu, f2ord(v))); }
+
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }

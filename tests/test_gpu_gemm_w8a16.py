@@ -74,6 +74,16 @@ def test_row_partition_and_stream_k_agree(mode, ctas, monkeypatch):
     _check(inputs.gemm_w8_case(128, 10004, 256, seed=9), torch.float32)
 
 
+@pytest.mark.parametrize("fused", ["0", "8"])
+def test_small_m_with_and_without_in_kernel_decomposition(fused, monkeypatch):
+    """M <= 8 can decompose the activations inside the GEMM kernel (opt-in); it must agree with the two-kernel path
+    and the oracle bit for bit."""
+    monkeypatch.setenv("MSD_GEMM_FUSED_MAXM", fused)
+    _check(inputs.gemm_w8_case(1, 1152, 2048, seed=11), torch.float32)
+    _check(inputs.gemm_w8_case(8, 12000, 528, seed=12), torch.float32)
+    _check(inputs.gemm_w8_case(3, 640, 1536 + 16, seed=13), torch.bfloat16)
+
+
 def test_without_programmatic_dependent_launch(monkeypatch):
     monkeypatch.setenv("MSD_NO_PDL", "1")
     _check(inputs.gemm_w8_case(16, 1024, 1024, seed=7), torch.float32)
