@@ -243,6 +243,10 @@ def run_gpu(args):
                              "gbps": round(algorithmic_bytes(M, N, K) / t / 1e3, 1),
                              "tops": round(executed_ops(M, N, K) / t / 1e6, 2)})
 
+    other = {}
+    if rank == 0 and not args.no_breakdown:
+        other = other_configs(torch, binding, device, capture, timed)
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -270,6 +274,7 @@ def run_gpu(args):
                      "traffic": None, "kernel": "gemm_w8a16_kernel (+ decompose_int8_kernel overlapped by PDL)",
                      "note": "achieved = algorithmic bytes of the sweep / device time of the timed region"},
         "per_call": per_call,
+        "other_configs": other,
     }
     traffic_file = os.path.join(ROOT, "profiles", "gemm_w8a16_traffic.json")
     if os.path.exists(traffic_file):
@@ -282,6 +287,84 @@ def run_gpu(args):
     print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def other_configs(torch, binding, device, capture, timed):
+    """The other parts of the headline metric, each timed on its own (graph of 4 calls, device time): the comparison
+    GEMM the method replaces, the W4A16 prefill GEMM (configs[2]) and the INT8-KV decode attention (configs[3], [4])."""
+    peaks, _ = load_peaks()
+    res = {}
+    g = torch.Generator(device=device)
+    g.manual_seed(7)
+
+    def per_call_us(fn, reps=4, steps=5):
+        def many():
+            for _ in range(reps):
+                fn()
+        gr = capture(many)
+        return timed(gr.replay, steps, 3) / (steps * reps) * 1e3
+
+    # dequantize-then-BF16 comparison GEMM at M = 16 of both sweep shapes
+    base = {}
+    for (N, K) in SHAPES:
+        x = torch.randn((16, K), generator=g, device=device).to(torch.bfloat16)
+        ws = [torch.randint(-127, 128, (N, K), generator=g, dtype=torch.int8, device=device) for _ in range(4)]
+        sc = torch.rand(N, generator=g, device=device) * 0.01
+        wsp_b = binding.workspace(binding.gemm_dequant_bf16_workspace_bytes(16, N, K), device)
+        wsp_m = binding.workspace(binding.gemm_w8a16_workspace_bytes(16, N, K), device)
+        y = torch.empty((16, N), dtype=torch.bfloat16, device=device)
+        it = [0]
+
+        def f_base():
+            it[0] += 1
+            wp, wb = binding._ws_ptr(wsp_b)
+            binding._check(binding.lib().msd_gemm_dequant_bf16(x.data_ptr(), ws[it[0] % 4].data_ptr(), sc.data_ptr(), 16, N, K,
+                                                             y.data_ptr(), 0, wp, wb, torch.cuda.current_stream().cuda_stream), "dequant")
+
+        def f_msd():
+            it[0] += 1
+            binding.gemm_w8a16(x, ws[it[0] % 4], sc, ws=wsp_m, out=y)
+        tb, tm = per_call_us(f_base), per_call_us(f_msd)
+        base[f"M16_N{N}_K{K}"] = {"dequant_bf16_us": round(tb, 2), "msd_us": round(tm, 2), "speedup": round(tb / tm, 2)}
+        del ws
+    res["w8a16_vs_dequant_bf16"] = base
+
+    # configs[2]: W4A16 prefill, M=4096, N=8192, K=8192
+    M, N, K = 4096, 8192, 8192
+    x = torch.randn((M, K), generator=g, device=device).to(torch.bfloat16)
+    w4 = torch.randint(0, 256, (N, K // 2), generator=g, dtype=torch.uint8, device=device)
+    e4 = torch.randint(118, 124, (N, K // 32), generator=g, dtype=torch.uint8, device=device)
+    wsp = binding.workspace(binding.gemm_w4a16_workspace_bytes(M, N, K), device)
+    y = torch.empty((M, N), dtype=torch.bfloat16, device=device)
+    t = per_call_us(lambda: binding.gemm_w4a16(x, w4, e4, ws=wsp, out=y))
+    pf = 4.0 * M * N * K / t / 1e9
+    res["w4a16_prefill_M4096_N8192_K8192"] = {
+        "us": round(t, 1), "executed_fp4_pflops": round(pf, 3), "effective_pflops": round(pf / 2, 3),
+        "frac_of_4x_measured_bf16": round(pf * 1e3 / (4 * peaks["bf16_tflops"]), 3), "frac_of_nominal_9pf": round(pf / 9.0, 3)}
+    del x, w4, e4, y, wsp
+
+    # configs[3] GQA and configs[4] MLA decode attention
+    from paper_2605_13915_b200 import inputs as gen
+    for name, (B, Hq, Hkv, D, Dv, L, alias) in {
+            "gqa_B32_Hq32_Hkv8_d128_L2048-8192": (32, 32, 8, 128, 128, gen.seqlens_uniform(32, 2048, 8192, seed=0), False),
+            "mla_B64_Hq64_d576_L16384": (64, 64, 1, 576, 512, np.full(64, 16384, np.int32), True)}.items():
+        T = int(np.sum(L))
+        cu = torch.zeros(B + 1, dtype=torch.int32)
+        cu[1:] = torch.from_numpy(np.cumsum(L).astype(np.int32))
+        cu = cu.to(device)
+        q = torch.randn((B, Hq, D), generator=g, device=device).to(torch.bfloat16)
+        k = torch.randint(-127, 128, (T, Hkv, D), generator=g, dtype=torch.int8, device=device)
+        v = None if alias else torch.randint(-127, 128, (T, Hkv, Dv), generator=g, dtype=torch.int8, device=device)
+        ks = torch.rand((T, Hkv), generator=g, device=device) * 0.02 + 0.01
+        vs = None if alias else torch.rand((T, Hkv), generator=g, device=device) * 0.02 + 0.01
+        wsp = binding.workspace(binding.attn_decode_int8kv_workspace_bytes(B, Hq, Hkv, D, Dv, int(L.max())), device)
+        o = torch.empty((B, Hq, Dv), dtype=torch.bfloat16, device=device)
+        t = per_call_us(lambda: binding.attn_decode_int8kv(q, k, v, ks, vs, cu, int(L.max()), D ** -0.5, dv=Dv, ws=wsp, out=o), reps=2)
+        byts = T * Hkv * ((D + 4) + (0 if alias else Dv + 4))
+        res["attn_" + name] = {"us": round(t, 1), "tokens_per_s": round(B / t * 1e6), "kv_gbps": round(byts / t / 1e3, 1),
+                               "frac_of_measured_hbm": round(byts / t / 1e3 / peaks["hbm_gbs"], 3)}
+        del k, v, ks, vs, q
+    return res
 
 
 def cpu_baseline(check=None):
