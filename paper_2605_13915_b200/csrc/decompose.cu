@@ -61,12 +61,13 @@ __device__ __forceinline__ void chunk_quantize(const uint4& a, const uint4& b, f
 template <int kDecThreads>
 __global__ void __launch_bounds__(kDecThreads)
 decompose_int8_kernel(const uint16_t* __restrict__ x, int64_t ldx, int K, int8_t* __restrict__ q1,
-                      int8_t* __restrict__ q2, float* __restrict__ alpha_out, float* __restrict__ beta_out) {
+                      int8_t* __restrict__ q2, float* __restrict__ alpha_out, float* __restrict__ beta_out, int early_trigger) {
   // When launched as a programmatic dependent of whatever precedes it in the stream it may become resident early, but
   // it reads nothing before that work has completed (the wait is a no-op for a plain launch); only then may its own
   // dependent (the GEMM) start prefetching weights.
+  if (early_trigger) pdl_launch_dependents();
   pdl_wait_primary();
-  pdl_launch_dependents();
+  if (!early_trigger) pdl_launch_dependents();
   const int row = blockIdx.x;
   const uint4* xr = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(row) * ldx);
   const int nchunks = K >> 4;
@@ -192,19 +193,20 @@ msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int
   if (M == 0) return MSD_OK;
   // Chained programmatic launch (this kernel resident while its predecessor still runs) is opt-in: measured slower.
   const bool pdl = getenv("MSD_DEC_CHAIN") != nullptr && getenv("MSD_NO_PDL") == nullptr;
+  const int early = (pdl && atoi(getenv("MSD_DEC_CHAIN")) >= 2) ? 1 : 0;
   const char* te = getenv("MSD_DEC_THREADS");
   // this kernel sits on the critical path of the GEMM behind it: more threads per row = shorter latency
   const int threads = te ? atoi(te) : (K >= 8192 ? 1024 : (K >= 2048 ? 512 : 256));
   cudaError_t err;
   if (threads >= 1024)
     err = launch_pdl(decompose_int8_kernel<1024>, dim3(static_cast<unsigned>(M)), dim3(1024), 0, stream, pdl,
-                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta);
+                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, early);
   else if (threads >= 512)
     err = launch_pdl(decompose_int8_kernel<512>, dim3(static_cast<unsigned>(M)), dim3(512), 0, stream, pdl,
-                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta);
+                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, early);
   else
     err = launch_pdl(decompose_int8_kernel<256>, dim3(static_cast<unsigned>(M)), dim3(256), 0, stream, pdl,
-                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta);
+                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, early);
   return err == cudaSuccess ? MSD_OK : MSD_ERR_CUDA;
 }
 

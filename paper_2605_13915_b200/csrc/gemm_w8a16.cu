@@ -16,6 +16,7 @@
 #include <cuda_bf16.h>
 
 #include <cstdlib>
+#include <type_traits>
 
 #include "host_common.h"
 #include "quant.cuh"
@@ -28,7 +29,8 @@ constexpr int kBlockK = 128;       // K bytes per TMA box (one 128-byte swizzle 
 constexpr int kMaxStages = 16;
 constexpr int kGemmThreads = 192;
 constexpr int kWStageBytes = kTileN * kBlockK;
-constexpr int kSmemBudget = 227 * 1024 - 4096;   // leaves room for the static barriers and the alignment pad
+constexpr int kEpiBytes = 16 * 1024;               // epilogue transpose buffer [32 tokens][128 rows] FP32
+constexpr int kSmemBudget = 227 * 1024 - 4096 - kEpiBytes;   // leaves room for the static barriers and the alignment pad
 
 struct GemmW8Params {
   int M, Mp, NB, N, K;
@@ -37,6 +39,7 @@ struct GemmW8Params {
   int hmax;                // tallest band (box rows of tmap_w; tmap_w2 has hmax - 8)
   int w_chunk_bytes;       // shared-memory bytes reserved for one weight box (band rows x 128 B, 1 KB granules)
   int kw;                  // adjacent 128-byte K boxes per stage: each weight row is then read kw*128 B at a time
+  int epi_off;             // byte offset of the epilogue's transpose buffer in dynamic shared memory
   int kb_rot_step;         // mode 1: CTA c starts its K loop at block (c * kb_rot_step) % kblocks
   int kblocks;             // K blocks per weight tile
   int num_tiles;
@@ -66,25 +69,35 @@ __device__ __forceinline__ long long block_owner(long long blk, long long total,
   return ((blk + 1) * grid - 1) / total;
 }
 
-__device__ __forceinline__ void store_out(const GemmW8Params& p, int i, int n, float v, int32_t a, int32_t b) {
-  const long long idx = static_cast<long long>(i) * p.N + n;
-  if (p.ytype == MSD_OUT_BF16) static_cast<__nv_bfloat16*>(p.y)[idx] = __float2bfloat16_rn(v);
-  else static_cast<float*>(p.y)[idx] = v;
-  if (p.acc_dbg) {
-    p.acc_dbg[idx] = a;
-    p.acc_dbg[static_cast<long long>(p.M) * p.N + idx] = b;
-  }
-}
-
-// One chunk of W accumulator columns of the final epilogue.  The sums come from TMEM (tile finished by this CTA alone)
-// or from the split-K meeting place in global memory (which is read and left zeroed for the next call).
-template <bool kBase, int W>
+// One chunk of W accumulator columns (= W tokens) of the final epilogue.  The sums come from TMEM (tile finished by this
+// CTA alone) or from the split-K meeting place in global memory (which is read and left zeroed for the next call).
+// A thread owns one weight row n, so its W results belong to W different rows of y; they are transposed through a
+// 16 KB shared-memory buffer [W][128] and leave as full 16-byte vectors along n (2-byte scattered stores were the
+// slowest part of the kernel at large M).  Called by the 128 epilogue threads together.
+template <bool kBase, bool kBf16, int W>
 __device__ __forceinline__ void epilogue_chunk(const GemmW8Params& p, uint32_t t_row, int32_t* acc_tile, int c0, int r, int n,
-                                               bool row_ok, float sw, const float* s_alpha, const float* s_beta) {
+                                               bool row_ok, float sw, const float* s_alpha, const float* s_beta,
+                                               uint8_t* stage_buf, int et, int n0, int rows_valid) {
+  using OutT = typename std::conditional<kBf16, __nv_bfloat16, float>::type;
+  constexpr int kEsz = static_cast<int>(sizeof(OutT));
   uint32_t a[W], b[W];
+  float al[kBase ? 1 : W], be[kBase ? 1 : W];
   if (acc_tile == nullptr) {
     tmem_ldw<W>(t_row + c0, a);
     if constexpr (!kBase) tmem_ldw<W>(t_row + p.Mp + c0, b);
+  }
+  if constexpr (!kBase) {
+    // the per-token scales of the chunk, fetched as vectors up front: read one by one inside the loop below they
+    // would each wait for the preceding shared-memory store (possible aliasing) with nothing to hide the latency
+#pragma unroll
+    for (int j = 0; j < W; j += 4) {
+      const float4 va = *reinterpret_cast<const float4*>(s_alpha + c0 + j);
+      const float4 vb = *reinterpret_cast<const float4*>(s_beta + c0 + j);
+      al[j] = va.x; al[j + 1] = va.y; al[j + 2] = va.z; al[j + 3] = va.w;
+      be[j] = vb.x; be[j + 1] = vb.y; be[j + 2] = vb.z; be[j + 3] = vb.w;
+    }
+  }
+  if (acc_tile == nullptr) {
     tmem_ld_wait();
   } else {
 #pragma unroll
@@ -98,22 +111,74 @@ __device__ __forceinline__ void epilogue_chunk(const GemmW8Params& p, uint32_t t
       if constexpr (!kBase) __stcg(acc_tile + (p.Mp + c0 + j) * kTileN + r, 0);
     }
   }
-  if (row_ok) {
+  OutT* stage = reinterpret_cast<OutT*>(stage_buf);
 #pragma unroll
-    for (int j = 0; j < W; ++j) {
-      const int i = c0 + j;
-      if (i < p.M) {
-        if constexpr (kBase) {
-          store_out(p, i, n, __uint_as_float(a[j]), 0, 0);
-        } else {
-          const int32_t ya = static_cast<int32_t>(a[j]), yb = static_cast<int32_t>(b[j]);
-          // y = s_W * (alpha * Y1 + beta * Y2)   (Alg. 1 line 8)
-          const float v = sw * __fmaf_rn(s_alpha[i], static_cast<float>(ya), s_beta[i] * static_cast<float>(yb));
-          store_out(p, i, n, v, ya, yb);
+  for (int j = 0; j < W; ++j) {
+    float v;
+    if constexpr (kBase) {
+      v = __uint_as_float(a[j]);
+    } else {
+      const int32_t ya = static_cast<int32_t>(a[j]), yb = static_cast<int32_t>(b[j]);
+      // y = s_W * (alpha * Y1 + beta * Y2)   (Alg. 1 line 8)
+      v = sw * __fmaf_rn(al[j], static_cast<float>(ya), be[j] * static_cast<float>(yb));
+    }
+    if constexpr (kBf16) stage[j * kTileN + r] = __float2bfloat16_rn(v);
+    else stage[j * kTileN + r] = v;
+  }
+  if constexpr (!kBase) {
+    if (p.acc_dbg && row_ok) {
+#pragma unroll
+      for (int j = 0; j < W; ++j) {
+        const int i = c0 + j;
+        if (i < p.M) {
+          const long long idx = static_cast<long long>(i) * p.N + n;
+          p.acc_dbg[idx] = static_cast<int32_t>(a[j]);
+          p.acc_dbg[static_cast<long long>(p.M) * p.N + idx] = static_cast<int32_t>(b[j]);
         }
       }
     }
   }
+  named_bar_sync(1, 128);
+  const int wm = min(W, p.M - c0);                               // tokens of this chunk that exist
+  int nv = min(rows_valid, p.N - n0);                            // weight rows of this tile / band that exist
+  if (nv < 0) nv = 0;
+  OutT* y = static_cast<OutT*>(p.y);
+  const bool vec_ok = ((static_cast<long long>(p.N) * kEsz) & 15) == 0 && ((static_cast<long long>(n0) * kEsz) & 15) == 0;
+  if (vec_ok) {
+    constexpr int kEpv = 16 / kEsz, kSegs = kTileN / kEpv;
+    const int sg = et % kSegs, nf = sg * kEpv;
+    if (nf + kEpv <= nv) {
+#pragma unroll 4
+      for (int j = et / kSegs; j < wm; j += 128 / kSegs) {
+        const uint4 val = *reinterpret_cast<const uint4*>(stage + j * kTileN + nf);
+        *reinterpret_cast<uint4*>(y + static_cast<long long>(c0 + j) * p.N + n0 + nf) = val;
+      }
+    } else if (nf < nv) {
+      for (int j = et / kSegs; j < wm; j += 128 / kSegs)
+        for (int e = nf; e < nv; ++e) y[static_cast<long long>(c0 + j) * p.N + n0 + e] = stage[j * kTileN + e];
+    }
+  } else {
+    if (et < nv)
+      for (int j = 0; j < wm; ++j) y[static_cast<long long>(c0 + j) * p.N + n0 + et] = stage[j * kTileN + et];
+  }
+  named_bar_sync(1, 128);            // the buffer is free for the next chunk
+}
+
+// All token chunks of one finished tile.
+template <bool kBase, bool kFused, bool kBf16>
+__device__ __forceinline__ void epilogue_tile(const GemmW8Params& p, uint32_t t_row, int32_t* acc_tile, int r, int n, bool row_ok,
+                                              float sw, const float* s_alpha, const float* s_beta, uint8_t* stage_buf, int et,
+                                              int n0, int rows_valid) {
+  int c0 = 0;
+  if constexpr (!kFused) {
+    if constexpr (kBase)
+      for (; c0 + 32 <= p.Mp; c0 += 32)
+        epilogue_chunk<kBase, kBf16, 32>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid);
+    for (; c0 + 16 <= p.Mp; c0 += 16)      // 16 tokens at a time: two sums and two scales per token stay in registers
+      epilogue_chunk<kBase, kBf16, 16>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid);
+  }
+  if (c0 + 8 <= p.Mp)
+    epilogue_chunk<kBase, kBf16, 8>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid);
 }
 
 // Adds W accumulator columns of a partial tile into the split-K meeting place (reductions without return value).
@@ -148,7 +213,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ int is_last_flag;
-  __shared__ float s_alpha[128], s_beta[128];
+  __shared__ __align__(16) float s_alpha[128], s_beta[128];
   __shared__ float s_inva[8], s_invb[8], s_qmax[2][4];       // fused path: reciprocals of the scales, row-max scratch
 
   const int warp = threadIdx.x >> 5;
@@ -163,6 +228,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     p.trace[blockIdx.x * 16 + 1] = static_cast<long long>(g);
   }
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+  uint8_t* epi_buf = smem + p.epi_off;             // 16 KB transpose buffer of the epilogue, after the pipeline stages
   const int x_chunk_bytes = p.NB * kBlockK;
   const int w_stage_bytes = p.kw * p.w_chunk_bytes;
   const int stage_bytes = w_stage_bytes + p.kw * x_chunk_bytes;
@@ -442,12 +508,10 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         if (finish) __threadfence();
       }
       if (finish) {
-        int c0 = 0;
-        if constexpr (!kFused) {
-          for (; c0 + 32 <= p.Mp; c0 += 32) epilogue_chunk<kBase, 32>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta);
-          if (c0 + 16 <= p.Mp) { epilogue_chunk<kBase, 16>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta); c0 += 16; }
-        }
-        if (c0 + 8 <= p.Mp) epilogue_chunk<kBase, 8>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta);
+        if (p.ytype == MSD_OUT_BF16)
+          epilogue_tile<kBase, kFused, true>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h);
+        else
+          epilogue_tile<kBase, kFused, false>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h);
       }
       tc_fence_before();
       __syncwarp();
@@ -482,7 +546,7 @@ static int pow2_at_least(int v) {
 
 struct GemmW8Plan {
   int Mp, NB, kblocks, num_tiles, grid, stages, tmem_cols;
-  int mode, groups8, hmax, w_chunk_bytes, kw;
+  int mode, groups8, hmax, w_chunk_bytes, kw, epi_off;
   long long total_blocks;
   size_t off_q, off_alpha, off_beta, off_counters, off_slots, bytes;
   size_t smem_bytes;
@@ -547,7 +611,8 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 1) stages = 1;      // cannot happen: one 128-byte box of the widest operands is 48 KB
   pl.stages = stages;
-  pl.smem_bytes = static_cast<size_t>(stages) * stage_bytes + tail_pad + 1024;
+  pl.epi_off = static_cast<int>(round_up(static_cast<size_t>(stages) * stage_bytes + tail_pad, 1024));
+  pl.smem_bytes = static_cast<size_t>(pl.epi_off) + kEpiBytes + 1024;
   pl.tmem_cols = pow2_at_least(2 * pl.NB);
   size_t off = 0;
   pl.off_q = off;         off = round_up(off + (base ? static_cast<size_t>(N) * K * 2 : static_cast<size_t>(pl.NB) * K), 1024);
@@ -642,7 +707,7 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
   GemmW8Params p;
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = env_int("MSD_GEMM_KROT", 5);
-  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw;
+  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
   p.w_scale = w_scale; p.alpha = alpha; p.beta = beta; p.y = y; p.acc_dbg = acc_dbg;
@@ -708,7 +773,7 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   GemmW8Params p;
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = 0;
-  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw;
+  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
   p.w_scale = w_scale; p.alpha = nullptr; p.beta = nullptr; p.y = y; p.acc_dbg = nullptr;
