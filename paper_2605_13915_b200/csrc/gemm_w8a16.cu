@@ -39,6 +39,8 @@ struct GemmW8Params {
   int hmax;                // tallest band (box rows of tmap_w; tmap_w2 has hmax - 8)
   int w_chunk_bytes;       // shared-memory bytes reserved for one weight box (band rows x 128 B, 1 KB granules)
   int kw;                  // adjacent 128-byte K boxes per stage: each weight row is then read kw*128 B at a time
+  int csplit;              // mode 2: CTAs per cluster = K slices per weight tile
+  int pre_stages;          // stages whose weight boxes are requested before waiting for the preceding kernel
   int epi_off;             // byte offset of the epilogue's transpose buffer in dynamic shared memory
   int kb_rot_step;         // mode 1: CTA c starts its K loop at block (c * kb_rot_step) % kblocks
   int kblocks;             // K blocks per weight tile
@@ -64,7 +66,11 @@ __device__ __forceinline__ void trace_mark(const GemmW8Params& p, int slot) {
   if (p.trace) p.trace[blockIdx.x * 16 + slot] = clock64();
 }
 
-__device__ __forceinline__ long long range_begin(long long cta, long long total, long long grid) { return cta * total / grid; }
+__device__ __forceinline__ long long range_begin(long long cta, long long total, long long grid) {
+  // 32-bit division when the product fits (every realistic size): the 64-bit one costs hundreds of cycles at kernel start
+  if ((cta + 1) * total < (1LL << 32)) return static_cast<unsigned>(cta * total) / static_cast<unsigned>(grid);
+  return cta * total / grid;
+}
 __device__ __forceinline__ long long block_owner(long long blk, long long total, long long grid) {
   return ((blk + 1) * grid - 1) / total;
 }
@@ -74,10 +80,19 @@ __device__ __forceinline__ long long block_owner(long long blk, long long total,
 // A thread owns one weight row n, so its W results belong to W different rows of y; they are transposed through a
 // 16 KB shared-memory buffer [W][128] and leave as full 16-byte vectors along n (2-byte scattered stores were the
 // slowest part of the kernel at large M).  Called by the 128 epilogue threads together.
+// Mode 2: where the partial sums of the other CTAs of the cluster were delivered in this CTA's shared memory.
+// Slot s (from cluster rank s) holds [pass][token group of 4][128 weight rows][4 tokens] sums for this CTA's token
+// range [t0, t0 + T): a warp's 16-byte accesses (one weight row per lane) cover 512 contiguous bytes, which is what
+// both the remote stores and the local loads want.
+struct RecvInfo {
+  const int32_t* base;     // nullptr: nothing to add
+  int S, self, slot_words, T, t0;
+};
+
 template <bool kBase, bool kBf16, int W>
 __device__ __forceinline__ void epilogue_chunk(const GemmW8Params& p, uint32_t t_row, int32_t* acc_tile, int c0, int r, int n,
                                                bool row_ok, float sw, const float* s_alpha, const float* s_beta,
-                                               uint8_t* stage_buf, int et, int n0, int rows_valid) {
+                                               uint8_t* stage_buf, int et, int n0, int rows_valid, const RecvInfo& rv) {
   using OutT = typename std::conditional<kBf16, __nv_bfloat16, float>::type;
   constexpr int kEsz = static_cast<int>(sizeof(OutT));
   uint32_t a[W], b[W];
@@ -99,6 +114,30 @@ __device__ __forceinline__ void epilogue_chunk(const GemmW8Params& p, uint32_t t
   }
   if (acc_tile == nullptr) {
     tmem_ld_wait();
+    if (rv.base != nullptr) {
+      // the other K slices of this tile, in cluster-rank order (a fixed order: the FP32 sums of the comparison
+      // path come out the same on every run)
+      for (int s = 0; s < rv.S; ++s) {
+        if (s == rv.self) continue;
+        const int32_t* q = rv.base + (s < rv.self ? s : s - 1) * rv.slot_words + ((c0 - rv.t0) >> 2) * (kTileN * 4) + r * 4;
+#pragma unroll
+        for (int j = 0; j < W; j += 4) {
+          const int4 va = *reinterpret_cast<const int4*>(q + (j >> 2) * (kTileN * 4));
+          if constexpr (kBase) {
+            a[j] = __float_as_uint(__uint_as_float(a[j]) + __int_as_float(va.x));
+            a[j + 1] = __float_as_uint(__uint_as_float(a[j + 1]) + __int_as_float(va.y));
+            a[j + 2] = __float_as_uint(__uint_as_float(a[j + 2]) + __int_as_float(va.z));
+            a[j + 3] = __float_as_uint(__uint_as_float(a[j + 3]) + __int_as_float(va.w));
+          } else {
+            const int4 vb = *reinterpret_cast<const int4*>(q + rv.T * kTileN + (j >> 2) * (kTileN * 4));
+            a[j] += static_cast<uint32_t>(va.x); a[j + 1] += static_cast<uint32_t>(va.y);
+            a[j + 2] += static_cast<uint32_t>(va.z); a[j + 3] += static_cast<uint32_t>(va.w);
+            b[j] += static_cast<uint32_t>(vb.x); b[j + 1] += static_cast<uint32_t>(vb.y);
+            b[j + 2] += static_cast<uint32_t>(vb.z); b[j + 3] += static_cast<uint32_t>(vb.w);
+          }
+        }
+      }
+    }
   } else {
 #pragma unroll
     for (int j = 0; j < W; ++j) {
@@ -164,21 +203,21 @@ __device__ __forceinline__ void epilogue_chunk(const GemmW8Params& p, uint32_t t
   named_bar_sync(1, 128);            // the buffer is free for the next chunk
 }
 
-// All token chunks of one finished tile.
+// The token chunks [tok0, tok1) of one finished tile (both multiples of 8).
 template <bool kBase, bool kFused, bool kBf16>
 __device__ __forceinline__ void epilogue_tile(const GemmW8Params& p, uint32_t t_row, int32_t* acc_tile, int r, int n, bool row_ok,
                                               float sw, const float* s_alpha, const float* s_beta, uint8_t* stage_buf, int et,
-                                              int n0, int rows_valid) {
-  int c0 = 0;
+                                              int n0, int rows_valid, int tok0, int tok1, const RecvInfo& rv) {
+  int c0 = tok0;
   if constexpr (!kFused) {
     if constexpr (kBase)
-      for (; c0 + 32 <= p.Mp; c0 += 32)
-        epilogue_chunk<kBase, kBf16, 32>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid);
-    for (; c0 + 16 <= p.Mp; c0 += 16)      // 16 tokens at a time: two sums and two scales per token stay in registers
-      epilogue_chunk<kBase, kBf16, 16>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid);
+      for (; c0 + 32 <= tok1; c0 += 32)
+        epilogue_chunk<kBase, kBf16, 32>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv);
+    for (; c0 + 16 <= tok1; c0 += 16)      // 16 tokens at a time: two sums and two scales per token stay in registers
+      epilogue_chunk<kBase, kBf16, 16>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv);
   }
-  if (c0 + 8 <= p.Mp)
-    epilogue_chunk<kBase, kBf16, 8>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid);
+  for (; c0 + 8 <= tok1; c0 += 8)
+    epilogue_chunk<kBase, kBf16, 8>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv);
 }
 
 // Adds W accumulator columns of a partial tile into the split-K meeting place (reductions without return value).
@@ -192,6 +231,56 @@ __device__ __forceinline__ void partial_chunk(uint32_t t_row, int32_t* acc_tile,
     if constexpr (kBase) atomicAdd(reinterpret_cast<float*>(acc_tile) + (c0 + j) * kTileN + r, __uint_as_float(v[j]));
     else atomicAdd(acc_tile + (c0 + j) * kTileN + r, static_cast<int32_t>(v[j]));
   }
+}
+
+// Fused path, step a1: the scales of all M <= kFusedMaxM rows (alpha = max|x|/127, beta = alpha/254; Eq. alpha, Eq. beta)
+// computed by the 256 threads of the epilogue and quantiser warps together.  Every thread keeps one running maximum
+// per row and requests the vectors of all rows before using any, so the whole phase costs a few L2 round trips
+// instead of one per row.  x may come from the preceding kernel of the stream: nothing is read before it has finished.
+constexpr int kFusedMaxM = 8;
+__device__ __forceinline__ void fused_row_scales(const GemmW8Params& p, int t256, float (*s_qmax)[8], float* s_alpha,
+                                                 float* s_beta, float* s_inva, float* s_invb) {
+  pdl_wait_primary();
+  const int nvec_row = p.K >> 3;                // 16-byte vectors of 8 BF16 values per row
+  float m[kFusedMaxM];
+#pragma unroll
+  for (int i = 0; i < kFusedMaxM; ++i) m[i] = 0.0f;
+  for (int c = t256; c < nvec_row; c += 256) {
+    uint4 v[kFusedMaxM];
+#pragma unroll
+    for (int i = 0; i < kFusedMaxM; ++i)
+      if (i < p.M) v[i] = __ldg(reinterpret_cast<const uint4*>(p.x + static_cast<long long>(i) * p.ldx) + c);
+#pragma unroll
+    for (int i = 0; i < kFusedMaxM; ++i) {
+      if (i < p.M) {
+        const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          m[i] = fmaxf(m[i], fabsf(__uint_as_float(w[k] << 16)));
+          m[i] = fmaxf(m[i], fabsf(__uint_as_float(w[k] & 0xFFFF0000u)));
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kFusedMaxM; ++i) {
+    if (i < p.M) {
+      const float mm = warp_max(m[i]);
+      if ((t256 & 31) == 0) s_qmax[i][t256 >> 5] = mm;
+    }
+  }
+  named_bar_sync(2, 256);
+  if (t256 < p.M) {
+    float mm = 0.0f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) mm = fmaxf(mm, s_qmax[t256][w]);
+    const float alpha = __fdiv_rn(mm, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
+    s_alpha[t256] = alpha;
+    s_beta[t256] = beta;
+    s_inva[t256] = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f;
+    s_invb[t256] = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
+  }
+  named_bar_sync(2, 256);                       // scales visible to the quantiser and the epilogue warps
 }
 
 // kBase = false: the MSD path (INT8 x INT8 -> INT32, stacked components, scale-combine epilogue).
@@ -210,17 +299,23 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
   __shared__ __align__(8) uint64_t tfull_bar[2];
   __shared__ __align__(8) uint64_t tempty_bar[2];
+  __shared__ __align__(8) uint64_t cfree_bar, crecv_bar, cdone_bar;      // mode 2: "pipelines of the cluster drained", "partials delivered"
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ int is_last_flag;
   __shared__ __align__(16) float s_alpha[128], s_beta[128];
-  __shared__ float s_inva[8], s_invb[8], s_qmax[2][4];       // fused path: reciprocals of the scales, row-max scratch
+  __shared__ float s_inva[kFusedMaxM], s_invb[kFusedMaxM], s_qmax[kFusedMaxM][8];   // fused path: reciprocals of the scales, row-max scratch
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   if (p.num_stages < 1 || p.kw < 1 || p.kblocks < 1) return;     // malformed plan: touch nothing
   // lets a decomposition kernel queued behind this GEMM become resident early (it still waits for this grid to finish)
   pdl_launch_dependents();
+  if (threadIdx.x == 64) {       // first thing: the descriptor fetches are on the way to the first copy
+    tma_prefetch_desc(&tmap_w);
+    tma_prefetch_desc(&tmap_w2);
+    tma_prefetch_desc(&tmap_x);
+  }
   if (threadIdx.x == 0 && p.trace) {
     trace_mark(p, 0);
     unsigned long long g;
@@ -233,29 +328,6 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   const int w_stage_bytes = p.kw * p.w_chunk_bytes;
   const int stage_bytes = w_stage_bytes + p.kw * x_chunk_bytes;
 
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < p.num_stages; ++s) {
-      mbar_init(&full_bar[s], kFused ? 2 : 1);     // fused: the producer's arrive plus the quantiser warp of the stage
-      mbar_init(&empty_bar[s], 1);
-    }
-    for (int a = 0; a < 2; ++a) {
-      mbar_init(&tfull_bar[a], 1);
-      mbar_init(&tempty_bar[a], 4);      // one arrival per epilogue warp
-    }
-    abort_flag = 0;
-    mbar_init_fence();
-    tma_prefetch_desc(&tmap_w);
-    tma_prefetch_desc(&tmap_w2);
-    tma_prefetch_desc(&tmap_x);
-  }
-  if (warp == 1) tmem_alloc(&tmem_base_slot, p.tmem_cols);
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = tmem_base_slot;
-  volatile int* abort = &abort_flag;
-  if (threadIdx.x == 0) trace_mark(p, 2);
-
   const long long grid = gridDim.x;
   // mode 0: this CTA's slice of the tile-major (tile, K block) sequence; mode 1: its row band and every K block
   long long blk_begin, blk_end;
@@ -263,6 +335,11 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   if (p.mode == 0) {
     blk_begin = range_begin(blockIdx.x, p.total_blocks, grid);
     blk_end = range_begin(blockIdx.x + 1, p.total_blocks, grid);
+  } else if (p.mode == 2) {
+    // a cluster of csplit CTAs per weight tile, CTA `rank` of it takes the rank-th slice of the tile's K blocks
+    const int tile2 = blockIdx.x / p.csplit, rank = blockIdx.x - tile2 * p.csplit;
+    blk_begin = static_cast<long long>(tile2) * p.kblocks + rank * p.kblocks / p.csplit;
+    blk_end = static_cast<long long>(tile2) * p.kblocks + (rank + 1) * p.kblocks / p.csplit;
   } else {
     const int g0 = static_cast<int>(range_begin(blockIdx.x, p.groups8, grid));
     const int g1 = static_cast<int>(range_begin(blockIdx.x + 1, p.groups8, grid));
@@ -277,56 +354,125 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   const CUtensorMap* wmap = (p.mode == 1 && band_h != p.hmax) ? &tmap_w2 : &tmap_w;
   const int tx_bytes = p.kw * ((p.mode == 0 ? kWStageBytes : band_h * kBlockK) + (kFused ? 0 : x_chunk_bytes));
 
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.num_stages; ++s) {
+      mbar_init(&full_bar[s], kFused ? 2 : 1);     // fused: the producer's arrive plus the quantiser warp of the stage
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&tfull_bar[a], 1);
+      mbar_init(&tempty_bar[a], 4);      // one arrival per epilogue warp
+    }
+    if (p.mode == 2) {
+      mbar_init(&cfree_bar, p.csplit);               // one arrival per CTA of the cluster
+      mbar_init(&crecv_bar, 1);                      // this CTA's own arrival; the peers' copies count in bytes
+      {
+        // finishing CTAs this one sends to: each lets it know when its copy has landed
+        const int G8i = p.Mp >> 3, Fi = p.csplit < G8i ? p.csplit : G8i;
+        const int ranki = static_cast<int>(blockIdx.x) % p.csplit;
+        const int n_to = Fi - (ranki < Fi ? 1 : 0);
+        mbar_init(&cdone_bar, n_to > 0 ? n_to : 1);
+      }
+    }
+    abort_flag = 0;
+    mbar_init_fence();
+  }
+  // ------------------------------ TMA producer, first part ------------------------------
+  // Runs before the CTA-wide barrier below: the thread that initialised the mbarriers is in this warp, and the sooner
+  // the first weight boxes are requested the sooner the stream from HBM starts.
+  uint64_t pol_w = 0, pol_x = 0;
+  bool w_lane = false, x_lane = false;
+  int c = 0, tile = 0, kbi = 0, kbr = 0, kbr0 = 0, pre = 0, pre0 = 0;
+  auto advance = [&]() {
+    if (++kbi == p.kblocks) { kbi = 0; ++tile; }
+    if (++kbr == p.kblocks) kbr = 0;
+  };
   if (warp == 0) {
-    // ------------------------------ TMA producer ------------------------------
-    if (lane == 0) {
-      const uint64_t pol_w = policy_evict_first();    // weights are streamed once
-      const uint64_t pol_x = policy_evict_last();     // the stacked components are re-read by every CTA
-      int stage = 0;
-      uint32_t phase = 0;
-      // Weight tiles of the first stages do not depend on the decomposition kernel: issue them before waiting for it.
-      const long long nblk = blk_end - blk_begin;
-      const int pre = static_cast<int>(nblk < p.num_stages ? nblk : p.num_stages);
-      if constexpr (kBase) pdl_wait_primary();     // here the weights themselves come from the preceding kernel
+    __syncwarp();
+    // The whole warp takes part: lane 0 owns the barriers, lanes [0, kw) each issue one weight box of a stage and
+    // lanes [kw, 2 kw) one box of the stacked components, so the copies of a stage are issued side by side instead
+    // of one after another by a single thread.
+    pol_w = policy_evict_first();    // weights are streamed once
+    pol_x = policy_evict_last();      // the stacked components are re-read by every CTA
+    w_lane = lane < p.kw;
+    x_lane = !kFused && lane >= p.kw && lane < 2 * p.kw;
+    c = w_lane ? lane : lane - p.kw;
+    // (tile, K block) of the next block to load, advanced by one per stage; kbr = rotated K block
+    const int tile0 = blk_begin < (1LL << 32) ? static_cast<int>(static_cast<unsigned>(blk_begin) / static_cast<unsigned>(p.kblocks))
+                                              : static_cast<int>(blk_begin / p.kblocks);
+    const int kbi0 = static_cast<int>(blk_begin - static_cast<long long>(tile0) * p.kblocks);
+    tile = tile0; kbi = kbi0;
+    kbr = kbi + kb_rot;
+    if (kbr >= p.kblocks) kbr -= p.kblocks;
+    kbr0 = kbr;
+    // Weight tiles of the first stages do not depend on the decomposition kernel: issue them before waiting for it.
+    const long long nblk = blk_end - blk_begin;
+    pre = static_cast<int>(nblk < p.num_stages ? nblk : p.num_stages);
+    pre0 = pre < p.pre_stages ? pre : p.pre_stages;
+    if constexpr (kBase) pdl_wait_primary();     // here the weights themselves come from the preceding kernel
+    for (int i = 0; i < pre0; ++i) {
+      if (lane == 0) mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
+      __syncwarp();
+      if (w_lane)
+        tma_load_2d_hint(smem + i * stage_bytes + c * p.w_chunk_bytes, wmap, (kbr * p.kw + c) * kBlockK,
+                         band_row0 + tile * kTileN, &full_bar[i], pol_w);
+      advance();
+    }
+    if (lane == 0) trace_mark(p, 3);
+  }
+  if (warp == 1) tmem_alloc(&tmem_base_slot, p.tmem_cols);
+  tc_fence_before();
+  if (p.mode == 2) cluster_arrive_all();    // "my barriers are initialised": the epilogue warps wait for the peers' before their first remote arrive
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  volatile int* abort = &abort_flag;
+  if (threadIdx.x == 0) trace_mark(p, 2);
+
+  if (warp == 0) {
+    pdl_wait_primary();
+    if (lane == 0) trace_mark(p, 4);
+    {
+      int kx = kbr0;
       for (int i = 0; i < pre; ++i) {
-        const long long blk = blk_begin + i;
-        const int tile = static_cast<int>(blk / p.kblocks), kb = static_cast<int>((blk + kb_rot) % p.kblocks);
-        mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
-        for (int c = 0; c < p.kw; ++c)
-          tma_load_2d_hint(smem + i * stage_bytes + c * p.w_chunk_bytes, wmap, (kb * p.kw + c) * kBlockK,
-                           band_row0 + tile * kTileN, &full_bar[i], pol_w);
-      }
-      trace_mark(p, 3);
-      pdl_wait_primary();
-      trace_mark(p, 4);
-      for (int i = 0; i < pre && !kFused; ++i) {
-        const int kb = static_cast<int>((blk_begin + i + kb_rot) % p.kblocks);
-        for (int c = 0; c < p.kw; ++c)
-          tma_load_2d_hint(smem + i * stage_bytes + w_stage_bytes + c * x_chunk_bytes, &tmap_x, (kb * p.kw + c) * kBlockK, 0,
+        if (i >= pre0) {     // weight boxes held back so that the wait above was not queued behind them
+          if (lane == 0) mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
+          __syncwarp();
+          if (w_lane)
+            tma_load_2d_hint(smem + i * stage_bytes + c * p.w_chunk_bytes, wmap, (kbr * p.kw + c) * kBlockK,
+                             band_row0 + tile * kTileN, &full_bar[i], pol_w);
+          advance();
+        }
+        if (x_lane)
+          tma_load_2d_hint(smem + i * stage_bytes + w_stage_bytes + c * x_chunk_bytes, &tmap_x, (kx * p.kw + c) * kBlockK, 0,
                            &full_bar[i], pol_x);
+        if (++kx == p.kblocks) kx = 0;
       }
-      stage = pre % p.num_stages;
-      phase = (pre == p.num_stages) ? 1 : 0;
-      bool ok = true;
-      for (long long blk = blk_begin + pre; blk < blk_end && ok; ++blk) {
-        const int tile = static_cast<int>(blk / p.kblocks), kb = static_cast<int>((blk + kb_rot) % p.kblocks);
+    }
+    int stage = pre % p.num_stages;
+    uint32_t phase = (pre == p.num_stages) ? 1 : 0;
+    bool ok = true;
+    for (long long blk = blk_begin + pre; blk < blk_end; ++blk) {
+      if (lane == 0) {
         ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
-        if (!ok) break;
-        mbar_arrive_expect_tx(&full_bar[stage], tx_bytes);
-        uint8_t* dst = smem + stage * stage_bytes;
-        for (int c = 0; c < p.kw; ++c)
-          tma_load_2d_hint(dst + c * p.w_chunk_bytes, wmap, (kb * p.kw + c) * kBlockK, band_row0 + tile * kTileN,
-                           &full_bar[stage], pol_w);
-        for (int c = 0; c < p.kw && !kFused; ++c)
-          tma_load_2d_hint(dst + w_stage_bytes + c * x_chunk_bytes, &tmap_x, (kb * p.kw + c) * kBlockK, 0, &full_bar[stage], pol_x);
-        if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
+        if (ok) mbar_arrive_expect_tx(&full_bar[stage], tx_bytes);
       }
-      trace_mark(p, 5);
-      if (!ok) {
-        // give copies already in flight a bounded time to land before the CTA goes away
-        const long long t0 = clock64();
-        while (clock64() - t0 < 2000000LL) {}
-      }
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      uint8_t* dst = smem + stage * stage_bytes;
+      if (w_lane)
+        tma_load_2d_hint(dst + c * p.w_chunk_bytes, wmap, (kbr * p.kw + c) * kBlockK, band_row0 + tile * kTileN,
+                         &full_bar[stage], pol_w);
+      else if (x_lane)
+        tma_load_2d_hint(dst + w_stage_bytes + c * x_chunk_bytes, &tmap_x, (kbr * p.kw + c) * kBlockK, 0, &full_bar[stage], pol_x);
+      advance();
+      if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
+    }
+    if (lane == 0) trace_mark(p, 5);
+    if (!ok) {
+      // give copies already in flight a bounded time to land before the CTA goes away
+      const long long t0 = clock64();
+      while (clock64() - t0 < 2000000LL) {}
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
@@ -378,33 +524,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     // ------------------------------ quantiser warps (fused path) ------------------------------
     const int qt = threadIdx.x - kGemmThreads;    // 0..127
     const int qw = warp - 6;
-    const int nvec_row = p.K >> 3;                // 16-byte vectors of 8 BF16 values per row
-    // a1: row maxima over the whole K, then alpha = max/127, beta = alpha/254 (Eq. alpha, Eq. beta)
-    for (int i = 0; i < p.M; ++i) {
-      const uint4* xr = reinterpret_cast<const uint4*>(p.x + static_cast<long long>(i) * p.ldx);
-      float m = 0.0f;
-      for (int c = qt; c < nvec_row; c += 128) {
-        const uint4 v = __ldg(xr + c);
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          m = fmaxf(m, fabsf(__uint_as_float(w[k] << 16)));
-          m = fmaxf(m, fabsf(__uint_as_float(w[k] & 0xFFFF0000u)));
-        }
-      }
-      m = warp_max(m);
-      if (lane == 0) s_qmax[i & 1][qw] = m;
-      named_bar_sync(3, 128);
-      if (qt == 0) {
-        const float mm = fmaxf(fmaxf(s_qmax[i & 1][0], s_qmax[i & 1][1]), fmaxf(s_qmax[i & 1][2], s_qmax[i & 1][3]));
-        const float alpha = __fdiv_rn(mm, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
-        s_alpha[i] = alpha;
-        s_beta[i] = beta;
-        s_inva[i] = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f;
-        s_invb[i] = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
-      }
-    }
-    named_bar_sync(2, 256);                       // scales visible to the quantiser and the epilogue warps
+    fused_row_scales(p, qt + 128, s_qmax, s_alpha, s_beta, s_inva, s_invb);
     // a2-a3: per stage, quantise the M x (kw*128) slice of X into the stacked operand tile (rows i and Mp+i).
     // Each warp owns a fixed subset of the ring's stages (stage s belongs to warp s % 4) and fills them in order, so
     // several stages are being filled at a time (one warp's load latency does not pace the pipeline) while every
@@ -457,7 +577,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     const int r = quad * 32 + lane;               // weight row within the tile == TMEM lane
     const int et = threadIdx.x - 64;              // 0..127
     if constexpr (kFused) {
-      named_bar_sync(2, 256);                     // the quantiser warps have written s_alpha / s_beta
+      fused_row_scales(p, et, s_qmax, s_alpha, s_beta, s_inva, s_invb);   // together with the quantiser warps
     } else if constexpr (!kBase) {
       pdl_wait_primary();
       if (et < p.M) {
@@ -467,6 +587,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     }
     named_bar_sync(1, 128);
     int seg = 0;
+    int sent_to = 0;           // mode 2: finishing CTAs whose acknowledgement is outstanding
     bool ok = true;
     long long blk = blk_begin;
     while (blk < blk_end && ok) {
@@ -486,7 +607,82 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       const float sw = (!kBase && row_ok) ? __ldg(p.w_scale + n) : 0.0f;
       bool finish = complete;
       int32_t* acc_tile = nullptr;
-      if (!complete) {
+      int tok0 = 0, tok1 = p.Mp;
+      RecvInfo rv = {nullptr, 0, 0, 0, 0, 0};
+      if (!kFused && p.mode == 2 && p.csplit > 1) {
+        // ---- split-K inside a cluster: partial sums travel through the peers' shared memory ----
+        // Finishing is shared out as well: owner f < F completes the tokens of its groups of 8 for the whole tile.
+        const int S = p.csplit, rank = static_cast<int>(blockIdx.x) - tile * S;
+        const int G8 = p.Mp >> 3, F = S < G8 ? S : G8;
+        const int tmax = 8 * ((G8 + F - 1) / F);
+        const int passes = kBase ? 1 : 2;
+        const int slot_words = passes * tmax * kTileN;
+        // shared memory of the drained pipeline: S-1 incoming slots (one per peer), then the outgoing staging slots
+        uint8_t* stage_out = smem + static_cast<size_t>(S - 1) * slot_words * 4;
+        // 1. this CTA's own MMAs are complete, so it may overwrite its own buffers: stage what the others will finish
+        int oi = 0;
+        for (int f = 0; f < F; ++f) {
+          if (f == rank) continue;
+          const int ft0 = 8 * (f * G8 / F), ft1 = 8 * ((f + 1) * G8 / F), fT = ft1 - ft0;
+          uint8_t* so = stage_out + static_cast<size_t>(oi) * slot_words * 4;
+          for (int ps = 0; ps < passes; ++ps) {
+            uint8_t* srow = so + static_cast<size_t>(ps * fT * kTileN + r * 4) * 4;
+            for (int c = ft0; c < ft1; c += 32) {
+              const int nc = ft1 - c < 32 ? ft1 - c : 32;     // up to 32 columns per round, their TMEM loads in flight together
+              uint32_t v[4][8];
+#pragma unroll
+              for (int g = 0; g < 4; ++g)
+                if (g * 8 < nc) tmem_ld8(t_row + ps * p.Mp + c + g * 8, v[g]);
+              tmem_ld_wait();
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                if (g * 8 < nc) {
+                  uint8_t* d = srow + static_cast<size_t>(((c - ft0 + g * 8) >> 2) * (kTileN * 4)) * 4;
+                  *reinterpret_cast<uint4*>(d) = make_uint4(v[g][0], v[g][1], v[g][2], v[g][3]);
+                  *reinterpret_cast<uint4*>(d + kTileN * 16) = make_uint4(v[g][4], v[g][5], v[g][6], v[g][7]);
+                }
+              }
+            }
+          }
+          ++oi;
+        }
+        fence_proxy_async_smem();               // the copy engine reads what these threads wrote
+        finish = rank < F;
+        if (finish) {
+          tok0 = 8 * (rank * G8 / F);
+          tok1 = 8 * ((rank + 1) * G8 / F);
+          // bytes this CTA is going to receive (posted before any peer can start sending)
+          if (et == 0) mbar_arrive_expect_tx(&crecv_bar, static_cast<uint32_t>((S - 1) * passes * (tok1 - tok0) * kTileN * 4));
+        }
+        named_bar_sync(1, 128);
+        // 2. the pipelines of all CTAs of the cluster are drained: tell every CTA (itself included), wait for all
+        cluster_wait_all();                     // every CTA of the cluster has initialised its barriers
+        if (et < S) mbar_arrive_cluster(mapa_shared(smem_u32(&cfree_bar), et));
+        ok = wait_bounded_cluster(&cfree_bar, 0, abort, p.status);
+        if (!ok) break;
+        // 3. one bulk copy per finishing peer, straight into its slot for this rank
+        if (et == 0) {
+          oi = 0;
+          for (int f = 0; f < F; ++f) {
+            if (f == rank) continue;
+            const int fT = 8 * ((f + 1) * G8 / F) - 8 * (f * G8 / F);
+            const int slot = rank < f ? rank : rank - 1;
+            bulk_copy_to_peer(mapa_shared(smem_u32(smem) + static_cast<uint32_t>(slot * slot_words) * 4u, f),
+                              stage_out + static_cast<size_t>(oi) * slot_words * 4,
+                              static_cast<uint32_t>(passes * fT * kTileN * 4), mapa_shared(smem_u32(&crecv_bar), f));
+            ++oi;
+          }
+        }
+        if (finish) {
+          ok = wait_bounded_cluster(&crecv_bar, 0, abort, p.status);
+          if (!ok) break;
+          // the senders may let go of their staging buffers (and exit)
+          if (et < S && et != rank) mbar_arrive_cluster(mapa_shared(smem_u32(&cdone_bar), et));
+          rv.base = reinterpret_cast<const int32_t*>(smem);
+          rv.S = S; rv.self = rank; rv.slot_words = slot_words; rv.T = tok1 - tok0; rv.t0 = tok0;
+        }
+        sent_to = F - (rank < F ? 1 : 0);
+      } else if (!complete) {
         // add this CTA's partial sums into the tile's meeting place, then find out whether it was the last contributor
         acc_tile = p.accum + static_cast<long long>(tile) * p.NB * kTileN;
         int c0 = 0;
@@ -509,9 +705,9 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       }
       if (finish) {
         if (p.ytype == MSD_OUT_BF16)
-          epilogue_tile<kBase, kFused, true>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h);
+          epilogue_tile<kBase, kFused, true>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h, tok0, tok1, rv);
         else
-          epilogue_tile<kBase, kFused, false>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h);
+          epilogue_tile<kBase, kFused, false>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h, tok0, tok1, rv);
       }
       tc_fence_before();
       __syncwarp();
@@ -519,6 +715,8 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       ++seg;
       blk = seg_end;
     }
+    // mode 2: the staging buffers must outlive the copies that read them
+    if (sent_to > 0 && ok) wait_bounded_cluster(&cdone_bar, 0, abort, p.status);
     if (et == 0) { trace_mark(p, 10); if (p.trace) p.trace[blockIdx.x * 16 + 11] = seg; }
   }
 
@@ -546,7 +744,7 @@ static int pow2_at_least(int v) {
 
 struct GemmW8Plan {
   int Mp, NB, kblocks, num_tiles, grid, stages, tmem_cols;
-  int mode, groups8, hmax, w_chunk_bytes, kw, epi_off;
+  int mode, groups8, hmax, w_chunk_bytes, kw, epi_off, csplit;
   long long total_blocks;
   size_t off_q, off_alpha, off_beta, off_counters, off_slots, bytes;
   size_t smem_bytes;
@@ -559,6 +757,9 @@ static int env_int(const char* name, int fallback) {
 }
 
 // `base`: plan for the dequantize-to-BF16 comparison path (K counted in bytes of BF16, one operand row per token).
+// How many clusters of S CTAs of the GEMM kernel the device can hold at once (cached per configuration); 0 on error.
+static int max_resident_clusters(bool base, int S, size_t smem_bytes);
+
 static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   GemmW8Plan pl;
   pl.Mp = base ? static_cast<int>((M + 15) / 16 * 16) : static_cast<int>((M + 7) / 8 * 8);
@@ -585,7 +786,9 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   const int band_max = 8 * ((pl.groups8 + grid - 1) / grid);
   const int band_min = 8 * (pl.groups8 / grid);
   int mode = (band_min >= 64 && band_max <= kTileN) ? 1 : 0;
-  mode = env_int("MSD_GEMM_MODE", mode);
+  const int mode_env = env_int("MSD_GEMM_MODE", -1);     // 0 / 1 / 2 force a schedule where it is feasible
+  if (mode_env == 0 || mode_env == 1) mode = mode_env;
+  if (mode_env == 2) mode = 0;
   if (mode == 1 && (band_max > kTileN || band_min < 8)) mode = 0;
   pl.mode = mode;
   if (mode == 1) {
@@ -613,6 +816,30 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   pl.stages = stages;
   pl.epi_off = static_cast<int>(round_up(static_cast<size_t>(stages) * stage_bytes + tail_pad, 1024));
   pl.smem_bytes = static_cast<size_t>(pl.epi_off) + kEpiBytes + 1024;
+  // Few weight tiles (small N): instead of the stream-K split with its global atomics, a cluster of S CTAs per tile
+  // splits K evenly and sums the partial tiles through distributed shared memory (mode 2).  Taken when the clusters
+  // cover at least three quarters of the SMs, all of them are resident at once, and the partials fit the
+  // pipeline buffers they are delivered into.
+  pl.csplit = 1;
+  if (mode == 0 && mode_env != 0 && pl.num_tiles > 0) {
+    int S = grid / pl.num_tiles;
+    if (S > 8) S = 8;
+    if (S > pl.kblocks) S = pl.kblocks;
+    for (; S >= 2; --S) {
+      // S-1 incoming and S-1 outgoing slots of [passes][longest token range][128] sums live in the drained pipeline
+      const int G8 = pl.Mp / 8, F = S < G8 ? S : G8;
+      const size_t xfer = 2 * static_cast<size_t>(S - 1) * (base ? 1 : 2) * 8 * ((G8 + F - 1) / F) * kTileN * sizeof(int32_t);
+      if (xfer <= static_cast<size_t>(pl.epi_off)) break;
+    }
+    if (S >= 2) {
+      const bool covers = static_cast<long long>(pl.num_tiles) * S * 4 >= 3LL * grid;
+      if ((covers || mode_env == 2) && max_resident_clusters(base, S, pl.smem_bytes) >= pl.num_tiles) {
+        pl.mode = 2;
+        pl.csplit = S;
+        pl.grid = pl.num_tiles * S;
+      }
+    }
+  }
   pl.tmem_cols = pow2_at_least(2 * pl.NB);
   size_t off = 0;
   pl.off_q = off;         off = round_up(off + (base ? static_cast<size_t>(N) * K * 2 : static_cast<size_t>(pl.NB) * K), 1024);
@@ -623,6 +850,47 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   pl.off_slots = off;     off = round_up(off + static_cast<size_t>(pl.num_tiles) * pl.NB * kTileN * sizeof(int32_t), 1024);
   pl.bytes = off;
   return pl;
+}
+
+static bool ensure_smem_attr() {
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(gemm_w8a16_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w8a16_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w8a16_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
+    {
+      cudaGetLastError();
+      return false;
+    }
+    attr_done = true;
+  }
+  return true;
+}
+
+static int max_resident_clusters(bool base, int S, size_t smem_bytes) {
+  struct Entry { bool base; int S; size_t smem; int n; };
+  static Entry cache[32];
+  static int used = 0;
+  for (int i = 0; i < used; ++i)
+    if (cache[i].base == base && cache[i].S == S && cache[i].smem == smem_bytes) return cache[i].n;
+  if (!ensure_smem_attr()) return 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(S) * 64);
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(S);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  const cudaError_t e = base ? cudaOccupancyMaxActiveClusters(&n, gemm_w8a16_kernel<true, false>, &cfg)
+                             : cudaOccupancyMaxActiveClusters(&n, gemm_w8a16_kernel<false, false>, &cfg);
+  if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
+  if (used < 32) cache[used++] = Entry{base, S, smem_bytes, n};
+  return n;
 }
 
 // The step MSD removes (Sec. 3.1, first equation): INT8 weights -> bf16(s_W * w), written back to memory.
@@ -691,7 +959,7 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
   // rows [0, M) hold Q1, rows [Mp, Mp+M) hold Q2; the padding rows are never read back.
   // Opt-in (MSD_GEMM_FUSED_MAXM=<largest M>): with one quantiser warp per stage the in-kernel path measured no faster
   // than the two-kernel path at M = 1 and slower from M = 2 on, so the default keeps the separate kernel.
-  const bool fused = (M <= env_int("MSD_GEMM_FUSED_MAXM", 0)) && M <= 8;
+  const bool fused = (M <= env_int("MSD_GEMM_FUSED_MAXM", 0)) && M <= kFusedMaxM && pl.mode != 2;
   if (!fused) {
     st = launch_decompose_int8(x_bf16, M, K, K, q, q + static_cast<size_t>(pl.Mp) * K, alpha, beta, s);
     if (st != MSD_OK) return st;
@@ -707,7 +975,8 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
   GemmW8Params p;
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = env_int("MSD_GEMM_KROT", 5);
-  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off;
+  p.pre_stages = env_int("MSD_GEMM_PRE", 64);
+  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off; p.csplit = pl.csplit;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
   p.w_scale = w_scale; p.alpha = alpha; p.beta = beta; p.y = y; p.acc_dbg = acc_dbg;
@@ -718,21 +987,17 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
 
   p.x = static_cast<const uint16_t*>(x_bf16);
   p.ldx = K;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(gemm_w8a16_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_w8a16_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
-      return MSD_ERR_CUDA;
-    attr_done = true;
-  }
+  if (!ensure_smem_attr()) return MSD_ERR_CUDA;
   if (fused) {
-    // a plain launch: this kernel reads x directly, so it must not start before earlier work in the stream is done
-    if (launch_pdl(gemm_w8a16_kernel<false, true>, dim3(pl.grid), dim3(kFusedThreads), pl.smem_bytes, s, false, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
+    // may become resident while earlier work in the stream still runs: it prefetches weights, then waits for that
+    // work to finish before it reads x or touches the split-K workspace
+    if (launch_pdl(gemm_w8a16_kernel<false, true>, dim3(pl.grid), dim3(kFusedThreads), pl.smem_bytes, s, getenv("MSD_NO_PDL") == nullptr, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
       return MSD_ERR_CUDA;
     return MSD_OK;
   }
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  if (launch_pdl(gemm_w8a16_kernel<false, false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
+  if (launch_pdl_cluster(gemm_w8a16_kernel<false, false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl,
+                         static_cast<unsigned>(pl.csplit), tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
     return MSD_ERR_CUDA;
   return MSD_OK;
 }
@@ -773,7 +1038,8 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   GemmW8Params p;
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = 0;
-  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off;
+  p.pre_stages = 64;
+  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off; p.csplit = pl.csplit;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
   p.w_scale = w_scale; p.alpha = nullptr; p.beta = nullptr; p.y = y; p.acc_dbg = nullptr;
@@ -782,14 +1048,10 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   p.counters = reinterpret_cast<unsigned*>(ws + pl.off_counters);
   p.status = status;
   p.trace = nullptr;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(gemm_w8a16_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
-      return MSD_ERR_CUDA;
-    attr_done = true;
-  }
+  if (!ensure_smem_attr()) return MSD_ERR_CUDA;
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  if (launch_pdl(gemm_w8a16_kernel<true, false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
+  if (launch_pdl_cluster(gemm_w8a16_kernel<true, false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl,
+                         static_cast<unsigned>(pl.csplit), tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
     return MSD_ERR_CUDA;
   return MSD_OK;
 }

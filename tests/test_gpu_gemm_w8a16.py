@@ -74,6 +74,29 @@ def test_row_partition_and_stream_k_agree(mode, ctas, monkeypatch):
     _check(inputs.gemm_w8_case(128, 10004, 256, seed=9), torch.float32)
 
 
+@pytest.mark.parametrize("ctas", ["148", "40", "24", "9"])
+def test_cluster_split_k(ctas, monkeypatch):
+    """Few weight tiles: a cluster of CTAs per tile splits K and sums the partial tiles through distributed shared
+    memory.  The CTA count sets the cluster size (8, 5 / 4, 3 / 2, ...); token counts cover one finishing CTA (M <= 8),
+    fewer owners than CTAs, uneven token groups and the full 128; a ragged last tile; both output types."""
+    monkeypatch.setenv("MSD_GEMM_MODE", "2")
+    monkeypatch.setenv("MSD_GEMM_CTAS", ctas)
+    _check(inputs.gemm_w8_case(3, 640, 4096, seed=21), torch.float32)
+    _check(inputs.gemm_w8_case(24, 1000, 4096 + 16, seed=22), torch.bfloat16)
+    _check(inputs.gemm_w8_case(128, 512, 6144, seed=23), torch.float32)
+    _check(inputs.gemm_w8_case(72, 384, 8192, seed=24), torch.bfloat16)
+
+
+def test_cluster_split_k_comparison_kernel(monkeypatch):
+    monkeypatch.setenv("MSD_GEMM_MODE", "2")
+    c = inputs.gemm_w8_case(40, 512, 4096, seed=25)
+    y = binding.gemm_dequant_bf16(bf16_dev(c.x), dev(c.w), dev(c.w_scale), out_dtype=torch.float32)
+    torch.cuda.synchronize()
+    binding.last_device_status()
+    ref = oracle.gemm_dequant_bf16_w8(c.x, c.w, c.w_scale)
+    assert rel_row_err(y.cpu().numpy(), ref).max() <= TOL
+
+
 @pytest.mark.parametrize("fused", ["0", "8"])
 def test_small_m_with_and_without_in_kernel_decomposition(fused, monkeypatch):
     """M <= 8 can decompose the activations inside the GEMM kernel (opt-in); it must agree with the two-kernel path
