@@ -35,8 +35,9 @@ constexpr int kSmemBudget = 227 * 1024 - 4096 - kEpiBytes;   // leaves room for 
 struct GemmW8Params {
   int M, Mp, NB, N, K;
   int mode;                // 0 = stream-K over 128-row tiles, 1 = one row band per CTA
-  int groups8;             // ceil(N / 8): row groups divided over the CTAs in mode 1
-  int hmax;                // tallest band (box rows of tmap_w; tmap_w2 has hmax - 8)
+  int groups8;             // ceil(N / gran): row groups divided over the CTAs in mode 1
+  int gran;                // rows per group: 8 keeps every band 16-byte aligned in y, 1 balances the bands to one row
+  int hmax;                // tallest band (box rows of tmap_w; tmap_w2 has hmax - gran)
   int w_chunk_bytes;       // shared-memory bytes reserved for one weight box (band rows x 128 B, 1 KB granules)
   int kw;                  // adjacent 128-byte K boxes per stage: each weight row is then read kw*128 B at a time
   int csplit;              // mode 2: CTAs per cluster = K slices per weight tile
@@ -343,8 +344,8 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   } else {
     const int g0 = static_cast<int>(range_begin(blockIdx.x, p.groups8, grid));
     const int g1 = static_cast<int>(range_begin(blockIdx.x + 1, p.groups8, grid));
-    band_row0 = 8 * g0;
-    band_h = 8 * (g1 - g0);
+    band_row0 = p.gran * g0;
+    band_h = p.gran * (g1 - g0);
     blk_begin = 0;
     blk_end = p.kblocks;
   }
@@ -744,7 +745,7 @@ static int pow2_at_least(int v) {
 
 struct GemmW8Plan {
   int Mp, NB, kblocks, num_tiles, grid, stages, tmem_cols;
-  int mode, groups8, hmax, w_chunk_bytes, kw, epi_off, csplit;
+  int mode, groups8, gran, hmax, w_chunk_bytes, kw, epi_off, csplit;
   long long total_blocks;
   size_t off_q, off_alpha, off_beta, off_counters, off_slots, bytes;
   size_t smem_bytes;
@@ -776,15 +777,19 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   pl.kblocks = static_cast<int>((kbytes + static_cast<int64_t>(kw) * kBlockK - 1) / (static_cast<int64_t>(kw) * kBlockK));
   pl.num_tiles = static_cast<int>((N + kTileN - 1) / kTileN);
   pl.total_blocks = static_cast<long long>(pl.kblocks) * pl.num_tiles;
-  pl.groups8 = static_cast<int>((N + 7) / 8);
+  // Row bands of mode 1 come in two heights that differ by one group.  Groups of 8 rows keep every band on a 16-byte
+  // boundary of y (vector stores); balancing the bands to a single row (MSD_GEMM_GRAN=1) measured no faster.
+  pl.gran = env_int("MSD_GEMM_GRAN", 8);
+  if (pl.gran != 1 && pl.gran != 2 && pl.gran != 4) pl.gran = 8;
+  pl.groups8 = static_cast<int>((N + pl.gran - 1) / pl.gran);
   const int sms = sm_count();
   int grid = env_int("MSD_GEMM_CTAS", sms);
   if (grid < 1) grid = sms;
   if (grid > 256) grid = 256;
   // Row partition pays when every SM gets a band of at least 64 rows (the MMA always spans 128 rows, so shorter
   // bands waste tensor time and TMA rows on the shared activation tile) and the bands still fit one MMA.
-  const int band_max = 8 * ((pl.groups8 + grid - 1) / grid);
-  const int band_min = 8 * (pl.groups8 / grid);
+  const int band_max = pl.gran * ((pl.groups8 + grid - 1) / grid);
+  const int band_min = pl.gran * (pl.groups8 / grid);
   int mode = (band_min >= 64 && band_max <= kTileN) ? 1 : 0;
   const int mode_env = env_int("MSD_GEMM_MODE", -1);     // 0 / 1 / 2 force a schedule where it is feasible
   if (mode_env == 0 || mode_env == 1) mode = mode_env;
@@ -966,7 +971,7 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
   }
 
   CUtensorMap tmap_w, tmap_w2, tmap_x;
-  const uint32_t box2 = (pl.mode == 1 && pl.hmax > 8) ? pl.hmax - 8 : pl.hmax;
+  const uint32_t box2 = (pl.mode == 1 && pl.hmax > pl.gran) ? pl.hmax - pl.gran : pl.hmax;
   if (!encode_tmap_2d(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kBlockK, pl.hmax, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_w2, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kBlockK, box2, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, q, K, pl.NB, K, kBlockK, pl.NB, CU_TENSOR_MAP_SWIZZLE_128B))
@@ -976,7 +981,7 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = env_int("MSD_GEMM_KROT", 5);
   p.pre_stages = env_int("MSD_GEMM_PRE", 64);
-  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off; p.csplit = pl.csplit;
+  p.mode = pl.mode; p.groups8 = pl.groups8; p.gran = pl.gran; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off; p.csplit = pl.csplit;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
   p.w_scale = w_scale; p.alpha = alpha; p.beta = beta; p.y = y; p.acc_dbg = acc_dbg;
@@ -1030,7 +1035,7 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   }
   CUtensorMap tmap_w, tmap_w2, tmap_x;
   const uint64_t kb = static_cast<uint64_t>(2 * K);
-  const uint32_t box2 = (pl.mode == 1 && pl.hmax > 8) ? pl.hmax - 8 : pl.hmax;
+  const uint32_t box2 = (pl.mode == 1 && pl.hmax > pl.gran) ? pl.hmax - pl.gran : pl.hmax;
   if (!encode_tmap_2d(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, wbf, kb, N, kb, kBlockK, pl.hmax, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_w2, CU_TENSOR_MAP_DATA_TYPE_UINT8, wbf, kb, N, kb, kBlockK, box2, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, x_bf16, kb, M, kb, kBlockK, pl.NB, CU_TENSOR_MAP_SWIZZLE_128B))
@@ -1039,7 +1044,7 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = 0;
   p.pre_stages = 64;
-  p.mode = pl.mode; p.groups8 = pl.groups8; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off; p.csplit = pl.csplit;
+  p.mode = pl.mode; p.groups8 = pl.groups8; p.gran = pl.gran; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off; p.csplit = pl.csplit;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
   p.w_scale = w_scale; p.alpha = nullptr; p.beta = nullptr; p.y = y; p.acc_dbg = nullptr;
