@@ -363,6 +363,31 @@ def other_configs(torch, binding, device, capture, timed):
         byts = T * Hkv * ((D + 4) + (0 if alias else Dv + 4))
         res["attn_" + name] = {"us": round(t, 1), "tokens_per_s": round(B / t * 1e6), "kv_gbps": round(byts / t / 1e3, 1),
                                "frac_of_measured_hbm": round(byts / t / 1e3 / peaks["hbm_gbs"], 3)}
+        if not alias:
+            # comparison arm: our cache-expansion kernel (INT8 -> BF16 in memory), then a library BF16 attention
+            # (torch SDPA, one call per sequence) on the expanded cache
+            kb = torch.empty((T, Hkv, D), dtype=torch.bfloat16, device=device)
+            vb = torch.empty((T, Hkv, Dv), dtype=torch.bfloat16, device=device)
+            t_deq = per_call_us(lambda: (binding.kv_dequant_bf16(k, ks, out=kb), binding.kv_dequant_bf16(v, vs, out=vb)), reps=2)
+            cu_h = cu.cpu().tolist()
+            sdpa = torch.nn.functional.scaled_dot_product_attention
+
+            def f_lib():
+                for b in range(B):
+                    t0, t1 = cu_h[b], cu_h[b + 1]
+                    sdpa(q[b][None, :, None, :], kb[t0:t1].permute(1, 0, 2)[None], vb[t0:t1].permute(1, 0, 2)[None],
+                         scale=D ** -0.5, enable_gqa=True)
+            try:
+                t_lib = per_call_us(f_lib, reps=1)
+                res["attn_" + name]["comparison_dequant_bf16"] = {
+                    "dequant_us": round(t_deq, 1), "library_bf16_attention_us": round(t_lib, 1),
+                    "total_us": round(t_deq + t_lib, 1), "msd_speedup": round((t_deq + t_lib) / t, 2),
+                    "traffic_floor_us": round((3 * T * Hkv * (D + Dv) + 2 * T * Hkv * (D + Dv)) / peaks["hbm_gbs"] / 1e3, 1),
+                    "note": "dequant = msd_kv_dequant_bf16 (ours); attention = torch SDPA per sequence (library); "
+                            "traffic_floor = 5 bytes per cache element at the measured HBM peak"}
+            except Exception as e:  # the library arm is context, never the product
+                res["attn_" + name]["comparison_dequant_bf16"] = {"dequant_us": round(t_deq, 1), "library_error": str(e)[:120]}
+            del kb, vb
         del k, v, ks, vs, q
     return res
 

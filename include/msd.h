@@ -177,6 +177,13 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
 msd_status_t msd_attn_decode_schedule(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen,
                                       int32_t* tile, int32_t* n_splits, int32_t* split_tokens);
 
+/* Comparison kernel, not part of the MSD path: the cache expansion that MSD attention removes (Sec. 2.3; the
+ * "Dequant" arm of Sec. 6.4).  out[t,h,:] = bf16(scale[t,h] * cache[t,h,:]), FP32 product rounded to nearest even.
+ * cache [T,H,D] INT8, scale [T,H] FP32, out [T,H,D] BF16, all device pointers; cache and out 16-byte aligned;
+ * D % 16 == 0.  T = 0 is a no-op.  A BF16 attention kernel reading `out` completes the comparison arm. */
+msd_status_t msd_kv_dequant_bf16(const int8_t* cache, const float* scale, int64_t T, int32_t H, int32_t D,
+                                 void* out_bf16, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

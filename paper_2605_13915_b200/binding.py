@@ -48,6 +48,7 @@ _SIGS = {
     "msd_attn_decode_int8kv": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp,
                                          _vp, _sz, _vp]),
     "msd_attn_decode_schedule": (C.c_int, [_i32] * 6 + [C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
+    "msd_kv_dequant_bf16": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, _i32, _i32, C.c_void_p, C.c_void_p]),
 }
 
 
@@ -216,6 +217,17 @@ def attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen):
     _check(lib().msd_attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen, C.byref(tile), C.byref(ns), C.byref(st)),
            "msd_attn_decode_schedule")
     return tile.value, ns.value, st.value
+
+
+def kv_dequant_bf16(cache, scale, out=None):
+    """cache [T,H,D] int8, scale [T,H] f32 -> bf16(scale * cache) [T,H,D] (the comparison arm's cache expansion)."""
+    _need_cuda(cache, scale)
+    T, H, D = cache.shape
+    if out is None:
+        out = torch.empty((T, H, D), dtype=torch.bfloat16, device=cache.device)
+    _check(lib().msd_kv_dequant_bf16(cache.data_ptr(), scale.data_ptr(), T, H, D, out.data_ptr(), _stream()),
+           "msd_kv_dequant_bf16")
+    return out
 
 
 def attn_decode_int8kv_workspace_bytes(B, Hq, Hkv, D, Dv, max_seqlen):
