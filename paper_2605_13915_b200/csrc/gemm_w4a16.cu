@@ -3,7 +3,7 @@
 // accumulate into the SAME FP32 tile in TMEM, so the "one add" of the two passes costs nothing and each weight tile
 // is read once for both passes.
 //
-// Tile: 128 activation rows x 256 weight rows, K walked in stages of 256 elements (128 packed bytes = one 128-byte
+// Tile: 128 activation rows x 224 (default) or 256 weight rows, K walked in stages of 256 elements (128 packed bytes = one 128-byte
 // swizzle row).  Per stage TMA brings the A1, A2 (128 x 128 B) and B (256 x 128 B) tiles, bulk copies bring the scale
 // blocks (512-byte blocks of 128 rows x 4 scales, the layout the shared-memory -> TMEM scale copy expects), the MMA
 // warp copies the scales into TMEM and issues 4 K-steps x 2 passes.  Persistent CTAs walk the tiles with the
@@ -43,23 +43,33 @@ struct GemmW4Params {
   unsigned* status;
 };
 
-// Relayout of row-major E8M0 scales [rows, K/32] into 512-byte blocks (128 rows x 4 scales).
+// Relayout of row-major E8M0 scales [rows, K/32] into 512-byte blocks (128 rows x 4 scales).  Rows are first cut into
+// tiles of `tile_rows` (a multiple of 32), every tile into two blocks (the second one partly used when tile_rows < 256).
 __global__ void sf_block_layout_kernel(const uint8_t* __restrict__ src, int64_t rows, int kblocks, int sf_kgroups,
-                                       uint8_t* __restrict__ dst) {
+                                       int tile_rows, uint8_t* __restrict__ dst) {
   const int64_t total = rows * kblocks;
   for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
        i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
     const int64_t row = i / kblocks;
     const int kb = static_cast<int>(i - row * kblocks);
-    dst[((row >> 7) * sf_kgroups + (kb >> 2)) * 512 + (row & 31) * 16 + ((row >> 5) & 3) * 4 + (kb & 3)] = src[i];
+    const int64_t t = row / tile_rows;
+    const int lr = static_cast<int>(row - t * tile_rows);
+    dst[((2 * t + (lr >> 7)) * sf_kgroups + (kb >> 2)) * 512 + (lr & 31) * 16 + ((lr >> 5) & 3) * 4 + (kb & 3)] = src[i];
   }
 }
 
+// kTN = weight rows per tile: 256 (one accumulator) or 224 (two accumulators of 224 columns + the two sets of scale
+// columns fill the 512 TMEM columns exactly, so the epilogue of a tile overlaps the MMAs of the next).
+template <int kTN>
 __global__ void __launch_bounds__(kW4Threads, 1)
 gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
                   const __grid_constant__ CUtensorMap tmap_b, const GemmW4Params p) {
+  constexpr int kBBytes = kTN * 128;
+  constexpr int kStageBytes = 2 * kW4ABytes + kBBytes + kW4SfBytes;
+  constexpr int kAcc = (2 * kTN + 64 <= kW4TmemCols) ? 2 : 1;       // accumulators that fit beside 2 x 32 scale columns
+  constexpr int kSfCol = kAcc * kTN;
   extern __shared__ uint8_t smem_dyn[];
-  __shared__ __align__(8) uint64_t full_bar[kW4Stages], empty_bar[kW4Stages], tfull_bar, tempty_bar;
+  __shared__ __align__(8) uint64_t full_bar[kW4Stages], empty_bar[kW4Stages], tfull_bar[2], tempty_bar[2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
@@ -68,8 +78,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kW4Stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    mbar_init(&tfull_bar, 1);
-    mbar_init(&tempty_bar, 4);
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], 4); }
     abort_flag = 0;
     mbar_init_fence();
     tma_prefetch_desc(&tmap_a1);
@@ -94,12 +103,12 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
         for (int ks = 0; ks < p.kstages; ++ks) {
           ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
           if (!ok) break;
-          mbar_arrive_expect_tx(&full_bar[stage], kW4StageBytes);
-          uint8_t* dst = smem + stage * kW4StageBytes;
+          mbar_arrive_expect_tx(&full_bar[stage], kStageBytes);
+          uint8_t* dst = smem + stage * kStageBytes;
           tma_load_2d(dst, &tmap_a1, ks * 128, mt * kW4TileM, &full_bar[stage]);
           tma_load_2d(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, &full_bar[stage]);
-          tma_load_2d(dst + 2 * kW4ABytes, &tmap_b, ks * 128, nt * kW4TileN, &full_bar[stage]);
-          uint8_t* sf = dst + 2 * kW4ABytes + kW4BBytes;
+          tma_load_2d(dst + 2 * kW4ABytes, &tmap_b, ks * 128, nt * kTN, &full_bar[stage]);
+          uint8_t* sf = dst + 2 * kW4ABytes + kBBytes;
           const size_t a_off = (static_cast<size_t>(mt) * p.sf_kgroups + 2 * ks) * 512;
           bulk_load(sf, p.sfa1 + a_off, 1024, &full_bar[stage]);
           bulk_load(sf + 1024, p.sfa2 + a_off, 1024, &full_bar[stage]);
@@ -114,19 +123,25 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
       int stage = 0; uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      const uint32_t sfa1_t = tmem_base + kW4SfCol;          // 2 k-groups x 4 columns
-      const uint32_t sfa2_t = tmem_base + kW4SfCol + 8;
-      const uint32_t sfb_t = tmem_base + kW4SfCol + 16;      // 2 k-groups x 8 columns (256 weight rows)
+      uint32_t sfpar = 0;                                    // the scale columns alternate between two sets per stage
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-        ok = wait_bounded(&tempty_bar, (it & 1) ^ 1, abort, p.status);      // epilogue has drained the accumulator
+        const int acc = (kAcc == 2) ? (it & 1) : 0;
+        const uint32_t tphase = (kAcc == 2) ? ((it >> 1) & 1) : (it & 1);
+        const uint32_t d_tmem = tmem_base + acc * kTN;
+        ok = wait_bounded(&tempty_bar[acc], tphase ^ 1, abort, p.status);      // epilogue has drained this accumulator
         if (!ok) break;
         tc_fence_after();
         for (int ks = 0; ks < p.kstages; ++ks) {
           ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t base = smem_u32(smem + stage * kW4StageBytes);
-          const uint32_t a1 = base, a2 = base + kW4ABytes, bb = base + 2 * kW4ABytes, sf = bb + kW4BBytes;
+          const uint32_t base = smem_u32(smem + stage * kStageBytes);
+          const uint32_t a1 = base, a2 = base + kW4ABytes, bb = base + 2 * kW4ABytes, sf = bb + kBBytes;
+          // a copy into the set the previous stage's MMAs are not reading need not wait for them
+          const uint32_t sfa1_t = tmem_base + kSfCol + 32 * sfpar;     // 2 k-groups x 4 columns
+          const uint32_t sfa2_t = sfa1_t + 8;
+          const uint32_t sfb_t = sfa1_t + 16;                            // 2 k-groups x 8 columns (256 weight rows)
+          sfpar ^= 1;
           // scale blocks: 32 rows x 16 bytes each, eight-row groups 128 bytes apart, no swizzle
           for (int g = 0; g < 2; ++g) {
             tc_cp_32x128b_warpx4(sfa1_t + 4 * g, smem_desc(sf + g * 512, 0, 128, 0));
@@ -138,18 +153,18 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           for (int kk = 0; kk < 4; ++kk) {                    // 64 elements (32 bytes) per MMA
             const int g = kk >> 1;
             const uint32_t sid = (kk & 1) * 2;                // which pair of scale bytes of the 4-scale column
-            const uint32_t idesc = idesc_block_scaled(/*E2M1*/ 1, 1, kW4TileM, kW4TileN, sid, sid);
+            const uint32_t idesc = idesc_block_scaled(/*E2M1*/ 1, 1, kW4TileM, kTN, sid, sid);
             const uint64_t bdesc = smem_desc(bb + kk * 32, 16, 1024, kSwizzle128B);
-            mma_mxf4(tmem_base, smem_desc(a1 + kk * 32, 16, 1024, kSwizzle128B), bdesc, idesc, sfa1_t + 4 * g,
+            mma_mxf4(d_tmem, smem_desc(a1 + kk * 32, 16, 1024, kSwizzle128B), bdesc, idesc, sfa1_t + 4 * g,
                      sfb_t + 8 * g, (ks > 0 || kk > 0) ? 1u : 0u);
-            mma_mxf4(tmem_base, smem_desc(a2 + kk * 32, 16, 1024, kSwizzle128B), bdesc, idesc, sfa2_t + 4 * g,
+            mma_mxf4(d_tmem, smem_desc(a2 + kk * 32, 16, 1024, kSwizzle128B), bdesc, idesc, sfa2_t + 4 * g,
                      sfb_t + 8 * g, 1u);
           }
           tc_commit(&empty_bar[stage]);
           if (++stage == kW4Stages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
-        tc_commit(&tfull_bar);
+        tc_commit(&tfull_bar[acc]);
       }
     }
   } else {
@@ -159,6 +174,181 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
       const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+      const int acc = (kAcc == 2) ? (it & 1) : 0;
+      const uint32_t tphase = (kAcc == 2) ? ((it >> 1) & 1) : (it & 1);
+      ok = wait_bounded(&tfull_bar[acc], tphase, abort, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      const int row = mt * kW4TileM + r;
+      const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * kTN;
+      for (int c0 = 0; c0 < kTN; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld16(trow + c0, v);
+        tmem_ld_wait();
+        const int col = nt * kTN + c0;
+        if (row < p.M && col < p.N) {
+          if (p.ytype == MSD_OUT_BF16) {
+            uint32_t o[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+              o[j] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.y) + static_cast<long long>(row) * p.N + col;
+            if (col + 16 <= p.N) {
+              reinterpret_cast<uint4*>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
+              reinterpret_cast<uint4*>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+            } else {
+              for (int j = 0; j < 16 && col + j < p.N; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+            }
+          } else {
+            float* dst = static_cast<float*>(p.y) + static_cast<long long>(row) * p.N + col;
+            for (int j = 0; j < 16 && col + j < p.N; ++j) dst[j] = __uint_as_float(v[j]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kW4TmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------------------
+// CTA-pair variant (opt-in, MSD_W4_PAIR=1): two CTAs of a cluster share one 256 x 256 tile.  Each CTA loads its own 128 activation
+// rows (both components) and HALF of the weight tile; one tcgen05.mma.cta_group::2 per K step, issued by the even CTA,
+// multiplies all 256 rows against all 256 weight rows, each CTA's accumulator (its 128 rows x 256 columns) staying in
+// its own TMEM.  Per CTA and stage 52 KB enter shared memory instead of 68 KB and four stages fit instead of three;
+// measured no faster than the single-CTA kernel (the scale copies into TMEM and the unoverlapped epilogue, not the
+// fill rate, are what idles the tensor pipe), so it is not the default.  Scale blocks come through 2-D tensor
+// maps over the blocked scale arrays (rows of 512 bytes) so that, like the operand tiles, they complete on the
+// leader's barrier.
+constexpr int kW4PairStageBytes = 2 * kW4ABytes + kW4ABytes + kW4SfBytes;      // A1, A2, half of B, scales: 53248
+constexpr int kW4PairStages = 4;
+
+__global__ void __launch_bounds__(kW4Threads, 1)
+gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
+                       const __grid_constant__ CUtensorMap tmap_bh, const __grid_constant__ CUtensorMap tmap_sfa1,
+                       const __grid_constant__ CUtensorMap tmap_sfa2, const __grid_constant__ CUtensorMap tmap_sfb,
+                       const GemmW4Params p) {
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ __align__(8) uint64_t full_bar[kW4PairStages], empty_bar[kW4PairStages], tfull_bar, tempty_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kW4PairStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    mbar_init(&tfull_bar, 1);
+    mbar_init(&tempty_bar, 8);          // four epilogue warps in each CTA of the pair (used in the leader only)
+    abort_flag = 0;
+    mbar_init_fence();
+    tma_prefetch_desc(&tmap_a1);
+    tma_prefetch_desc(&tmap_a2);
+    tma_prefetch_desc(&tmap_bh);
+    tma_prefetch_desc(&tmap_sfa1);
+    tma_prefetch_desc(&tmap_sfa2);
+    tma_prefetch_desc(&tmap_sfb);
+  }
+  if (warp == 1) tmem_alloc_pair(&tmem_base_slot, kW4TmemCols);
+  tc_fence_before();
+  cluster_arrive_all();        // both CTAs' barriers exist before either signals the other's
+  cluster_wait_all();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  volatile int* abort = &abort_flag;
+  const int m_pairs = (p.m_tiles + 1) >> 1;
+  const int total_tiles = m_pairs * p.n_tiles;
+  const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      pdl_wait_primary();           // components and blocked scales come from the kernels launched just before
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
+        const int mt = 2 * (tile % m_pairs) + static_cast<int>(rank), nt = tile / m_pairs;
+        for (int ks = 0; ks < p.kstages; ++ks) {
+          ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
+          if (!ok) break;
+          // the leader's barrier counts the bytes of both CTAs
+          if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * kW4PairStageBytes);
+          const uint32_t bar = mapa_shared(smem_u32(&full_bar[stage]), 0);
+          uint8_t* dst = smem + stage * kW4PairStageBytes;
+          tma_load_2d_pair(dst, &tmap_a1, ks * 128, mt * kW4TileM, bar);
+          tma_load_2d_pair(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, bar);
+          tma_load_2d_pair(dst + 2 * kW4ABytes, &tmap_bh, ks * 128, nt * kW4TileN + static_cast<int>(rank) * 128, bar);
+          uint8_t* sf = dst + 3 * kW4ABytes;
+          tma_load_2d_pair(sf, &tmap_sfa1, 0, mt * p.sf_kgroups + 2 * ks, bar);
+          tma_load_2d_pair(sf + 1024, &tmap_sfa2, 0, mt * p.sf_kgroups + 2 * ks, bar);
+          tma_load_2d_pair(sf + 2048, &tmap_sfb, 0, (2 * nt) * p.sf_kgroups + 2 * ks, bar);
+          tma_load_2d_pair(sf + 3072, &tmap_sfb, 0, (2 * nt + 1) * p.sf_kgroups + 2 * ks, bar);
+          if (++stage == kW4PairStages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      int stage = 0; uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      uint32_t sfpar = 0;                                    // the scale columns alternate between two sets per stage
+      for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++it) {
+        ok = wait_bounded_cluster(&tempty_bar, (it & 1) ^ 1, abort, p.status);   // both epilogues have drained their accumulators
+        if (!ok) break;
+        tc_fence_after();
+        for (int ks = 0; ks < p.kstages; ++ks) {
+          ok = wait_bounded_cluster(&full_bar[stage], phase, abort, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t base = smem_u32(smem + stage * kW4PairStageBytes);
+          const uint32_t a1 = base, a2 = base + kW4ABytes, bb = base + 2 * kW4ABytes, sf = base + 3 * kW4ABytes;
+          const uint32_t sfa1_t = tmem_base + kW4SfCol + 32 * sfpar;     // 2 k-groups x 4 columns
+          const uint32_t sfa2_t = sfa1_t + 8;
+          const uint32_t sfb_t = sfa1_t + 16;                            // 2 k-groups x 8 columns (256 weight rows)
+          sfpar ^= 1;
+          for (int g = 0; g < 2; ++g) {
+            tc_cp_32x128b_warpx4_pair(sfa1_t + 4 * g, smem_desc(sf + g * 512, 0, 128, 0));
+            tc_cp_32x128b_warpx4_pair(sfa2_t + 4 * g, smem_desc(sf + 1024 + g * 512, 0, 128, 0));
+            tc_cp_32x128b_warpx4_pair(sfb_t + 8 * g, smem_desc(sf + 2048 + g * 512, 0, 128, 0));
+            tc_cp_32x128b_warpx4_pair(sfb_t + 8 * g + 4, smem_desc(sf + 3072 + g * 512, 0, 128, 0));
+          }
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {                    // 64 elements (32 bytes) per MMA
+            const int g = kk >> 1;
+            const uint32_t sid = (kk & 1) * 2;
+            const uint32_t idesc = idesc_block_scaled(/*E2M1*/ 1, 1, 2 * kW4TileM, kW4TileN, sid, sid);
+            const uint64_t bdesc = smem_desc(bb + kk * 32, 16, 1024, kSwizzle128B);
+            mma_mxf4_pair(tmem_base, smem_desc(a1 + kk * 32, 16, 1024, kSwizzle128B), bdesc, idesc, sfa1_t + 4 * g,
+                          sfb_t + 8 * g, (ks > 0 || kk > 0) ? 1u : 0u);
+            mma_mxf4_pair(tmem_base, smem_desc(a2 + kk * 32, 16, 1024, kSwizzle128B), bdesc, idesc, sfa2_t + 4 * g,
+                          sfb_t + 8 * g, 1u);
+          }
+          tc_commit_pair(&empty_bar[stage], 3);     // frees the stage in both CTAs
+          if (++stage == kW4PairStages) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        tc_commit_pair(&tfull_bar, 3);
+      }
+    }
+  } else {
+    const int quad = warp & 3;
+    const int r = quad * 32 + lane;
+    int it = 0;
+    bool ok = true;
+    const uint32_t leader_tempty = mapa_shared(smem_u32(&tempty_bar), 0);
+    for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++it) {
+      const int mt = 2 * (tile % m_pairs) + static_cast<int>(rank), nt = tile / m_pairs;
       ok = wait_bounded(&tfull_bar, it & 1, abort, p.status);
       if (!ok) break;
       tc_fence_after();
@@ -192,27 +382,40 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&tempty_bar);
+      if (lane == 0) mbar_arrive_cluster(leader_tempty);
     }
   }
 
+  // Neither CTA leaves while the other may still signal its barriers or (through the pair MMAs) read its shared memory.
   tc_fence_before();
   __syncthreads();
+  cluster_arrive_all();
+  cluster_wait_all();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, kW4TmemCols);
+    tmem_dealloc_pair(tmem_base, kW4TmemCols);
   }
 }
 
 struct GemmW4Plan {
-  int m_tiles, n_tiles, kstages, sf_kgroups, grid;
+  int m_tiles, n_tiles, kstages, sf_kgroups, grid, tile_n;
   size_t off_q1, off_q2, off_sfa1, off_sfa2, off_sfb, bytes;
 };
 
+// Weight rows per tile of the single-CTA kernel (the CTA-pair kernel always uses 256).
+static int w4_tile_n() {
+  const char* e = getenv("MSD_W4_TILEN");
+  const char* pe = getenv("MSD_W4_PAIR");
+  if (pe && atoi(pe) != 0) return 256;
+  return (e && atoi(e) == 256) ? 256 : 224;
+}
+
 static GemmW4Plan plan_w4(int64_t M, int64_t N, int64_t K) {
   GemmW4Plan pl;
+  const int tile_n = w4_tile_n();
+  pl.tile_n = tile_n;
   pl.m_tiles = static_cast<int>((M + kW4TileM - 1) / kW4TileM);
-  pl.n_tiles = static_cast<int>((N + kW4TileN - 1) / kW4TileN);
+  pl.n_tiles = static_cast<int>((N + tile_n - 1) / tile_n);
   pl.kstages = static_cast<int>((K + kW4BlockK - 1) / kW4BlockK);
   pl.sf_kgroups = 2 * pl.kstages;
   const int tiles = pl.m_tiles * pl.n_tiles;
@@ -264,7 +467,7 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
     const int64_t cap = static_cast<int64_t>(sm_count()) * 16;
     if (blocks > cap) blocks = cap;
     sf_block_layout_kernel<<<static_cast<unsigned>(blocks), threads, 0, s>>>(w_e8m0, N, static_cast<int>(K / 32), pl.sf_kgroups,
-                                                                            ws + pl.off_sfb);
+                                                                            pl.tile_n, ws + pl.off_sfb);
     if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
   }
   msd_status_t st = launch_decompose_mxfp4(x_bf16, M, K, K, q1, q2, ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s);
@@ -274,7 +477,7 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   const uint64_t kb = static_cast<uint64_t>(K / 2);
   if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, kb, M, kb, 128, kW4TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, q2, kb, M, kb, 128, kW4TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !encode_tmap_2d(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, w_fp4, kb, N, kb, 128, kW4TileN, CU_TENSOR_MAP_SWIZZLE_128B))
+      !encode_tmap_2d(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, w_fp4, kb, N, kb, 128, static_cast<uint32_t>(pl.tile_n), CU_TENSOR_MAP_SWIZZLE_128B))
     return MSD_ERR_CUDA;
 
   GemmW4Params p;
@@ -283,16 +486,47 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
   p.y = y; p.ytype = ytype; p.status = status;
 
-  const size_t smem_bytes = static_cast<size_t>(kW4Stages) * kW4StageBytes + 1024;
+  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+  const char* pair_env = getenv("MSD_W4_PAIR");
+  // opt-in: measured equal to the single-CTA kernel at M = 4096 (272 vs 266 us per call), so the bound is not the
+  // shared-memory fill it halves for the weights
+  const bool pair = pair_env ? atoi(pair_env) != 0 : false;
+  if (pair) {
+    // CTA pairs: weight half-tiles of 128 rows, scale blocks as rows of 128 32-bit words (512 bytes), two per box
+    CUtensorMap tmap_bh, tmap_sfa1, tmap_sfa2, tmap_sfb;
+    const uint64_t a_blocks = static_cast<uint64_t>(pl.m_tiles) * pl.sf_kgroups, b_blocks = static_cast<uint64_t>(2 * pl.n_tiles) * pl.sf_kgroups;
+    if (!encode_tmap_2d(&tmap_bh, CU_TENSOR_MAP_DATA_TYPE_UINT8, w_fp4, kb, N, kb, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !encode_tmap_2d(&tmap_sfa1, CU_TENSOR_MAP_DATA_TYPE_UINT32, p.sfa1, 128, a_blocks, 512, 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !encode_tmap_2d(&tmap_sfa2, CU_TENSOR_MAP_DATA_TYPE_UINT32, p.sfa2, 128, a_blocks, 512, 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !encode_tmap_2d(&tmap_sfb, CU_TENSOR_MAP_DATA_TYPE_UINT32, p.sfb, 128, b_blocks, 512, 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE))
+      return MSD_ERR_CUDA;
+    const size_t smem_pair = static_cast<size_t>(kW4PairStages) * kW4PairStageBytes + 1024;
+    static bool attr_pair_done = false;
+    if (!attr_pair_done) {
+      if (cudaFuncSetAttribute(gemm_w4a16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_pair)) != cudaSuccess)
+        return MSD_ERR_CUDA;
+      attr_pair_done = true;
+    }
+    const int pair_tiles = ((pl.m_tiles + 1) / 2) * pl.n_tiles;
+    int clusters = sm_count() / 2;
+    if (clusters > pair_tiles) clusters = pair_tiles;
+    if (launch_pdl_cluster(gemm_w4a16_pair_kernel, dim3(2 * clusters), dim3(kW4Threads), smem_pair, s, pdl, 2u, tmap_a1, tmap_a2,
+                           tmap_bh, tmap_sfa1, tmap_sfa2, tmap_sfb, p) != cudaSuccess)
+      return MSD_ERR_CUDA;
+    return MSD_OK;
+  }
+  const size_t smem_bytes = static_cast<size_t>(kW4Stages) * (2 * kW4ABytes + pl.tile_n * 128 + kW4SfBytes) + 1024;
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(gemm_w4a16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes)) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_w4a16_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w4a16_kernel<224>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
       return MSD_ERR_CUDA;
     attr_done = true;
   }
-  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  if (launch_pdl(gemm_w4a16_kernel, dim3(pl.grid), dim3(kW4Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, p) != cudaSuccess)
-    return MSD_ERR_CUDA;
+  const cudaError_t le = pl.tile_n == 256
+      ? launch_pdl(gemm_w4a16_kernel<256>, dim3(pl.grid), dim3(kW4Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, p)
+      : launch_pdl(gemm_w4a16_kernel<224>, dim3(pl.grid), dim3(kW4Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, p);
+  if (le != cudaSuccess) return MSD_ERR_CUDA;
   return MSD_OK;
 }
 

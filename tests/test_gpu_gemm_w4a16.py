@@ -75,3 +75,14 @@ def test_full_size_sampled():
     got = oracle.bf16_bits_to_f64(bf16_bits(y))[np.ix_(rows, cols)]
     # sampled columns: the row norm over the sample stands in for the full row norm (it is smaller, so stricter)
     _close(got, ref, True)
+
+
+@pytest.mark.parametrize("pair", ["0", "1"])
+def test_single_cta_and_cta_pair_kernels_agree(pair, monkeypatch):
+    """The opt-in CTA-pair kernel (one 256 x 256 tile per pair of CTAs) against the default one, at both sizes,
+    including a pair whose second CTA has no rows at all and an odd number of 128-row tiles."""
+    monkeypatch.setenv("MSD_W4_PAIR", pair)
+    for (M, N, K) in [(64, 512, 512), (384, 264, 1024), (520, 1032, 768)]:
+        c = inputs.gemm_w4_case(M, N, K, seed=7 + M)
+        y = _run(c, torch.float32).cpu().numpy().astype(np.float64)
+        _close(y, oracle.gemm_w4a16(c.x, c.w_fp4, c.w_e8m0, "f64"), False)
