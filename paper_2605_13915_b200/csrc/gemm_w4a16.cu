@@ -123,7 +123,11 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
       int stage = 0; uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      uint32_t sfpar = 0;                                    // the scale columns alternate between two sets per stage
+      uint32_t sfpar = 0;
+      const uint64_t op_desc = smem_desc(0, 16, 1024, kSwizzle128B);    // 128-byte-swizzled K-major operand tile
+      const uint64_t sf_desc = smem_desc(0, 0, 128, 0);                 // scale block: eight-row groups 128 bytes apart, no swizzle
+      const uint32_t idesc_lo = idesc_block_scaled(/*E2M1*/ 1, 1, kW4TileM, kTN, 0, 0);
+      const uint32_t idesc_hi = idesc_block_scaled(/*E2M1*/ 1, 1, kW4TileM, kTN, 2, 2);
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
         const int acc = (kAcc == 2) ? (it & 1) : 0;
         const uint32_t tphase = (kAcc == 2) ? ((it >> 1) & 1) : (it & 1);
@@ -135,30 +139,29 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t base = smem_u32(smem + stage * kStageBytes);
-          const uint32_t a1 = base, a2 = base + kW4ABytes, bb = base + 2 * kW4ABytes, sf = bb + kBBytes;
-          // a copy into the set the previous stage's MMAs are not reading need not wait for them
-          const uint32_t sfa1_t = tmem_base + kSfCol + 32 * sfpar;     // 2 k-groups x 4 columns
+          // Descriptors differ from the templates only in the 16-byte-granular address field (bits 0-13; shared
+          // memory is far below its range), so every operand costs one 64-bit add: this single thread's instruction
+          // count per stage, not the tensor pipe, was what paced the kernel.
+          const uint64_t enc = static_cast<uint64_t>(smem_u32(smem + stage * kStageBytes) >> 4);
+          const uint64_t a1d = op_desc + enc, a2d = a1d + (kW4ABytes >> 4), bd = a1d + (2 * kW4ABytes >> 4);
+          const uint64_t sfd = sf_desc + enc + ((2 * kW4ABytes + kBBytes) >> 4);
+          const uint32_t sfa1_t = tmem_base + kSfCol + 32 * sfpar;     // 2 k-groups x 4 columns; the two sets alternate
           const uint32_t sfa2_t = sfa1_t + 8;
           const uint32_t sfb_t = sfa1_t + 16;                            // 2 k-groups x 8 columns (256 weight rows)
           sfpar ^= 1;
-          // scale blocks: 32 rows x 16 bytes each, eight-row groups 128 bytes apart, no swizzle
+#pragma unroll
           for (int g = 0; g < 2; ++g) {
-            tc_cp_32x128b_warpx4(sfa1_t + 4 * g, smem_desc(sf + g * 512, 0, 128, 0));
-            tc_cp_32x128b_warpx4(sfa2_t + 4 * g, smem_desc(sf + 1024 + g * 512, 0, 128, 0));
-            tc_cp_32x128b_warpx4(sfb_t + 8 * g, smem_desc(sf + 2048 + g * 512, 0, 128, 0));
-            tc_cp_32x128b_warpx4(sfb_t + 8 * g + 4, smem_desc(sf + 3072 + g * 512, 0, 128, 0));
+            tc_cp_32x128b_warpx4(sfa1_t + 4 * g, sfd + (g * 512 >> 4));
+            tc_cp_32x128b_warpx4(sfa2_t + 4 * g, sfd + ((1024 + g * 512) >> 4));
+            tc_cp_32x128b_warpx4(sfb_t + 8 * g, sfd + ((2048 + g * 512) >> 4));
+            tc_cp_32x128b_warpx4(sfb_t + 8 * g + 4, sfd + ((3072 + g * 512) >> 4));
           }
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {                    // 64 elements (32 bytes) per MMA
             const int g = kk >> 1;
-            const uint32_t sid = (kk & 1) * 2;                // which pair of scale bytes of the 4-scale column
-            const uint32_t idesc = idesc_block_scaled(/*E2M1*/ 1, 1, kW4TileM, kTN, sid, sid);
-            const uint64_t bdesc = smem_desc(bb + kk * 32, 16, 1024, kSwizzle128B);
-            mma_mxf4(d_tmem, smem_desc(a1 + kk * 32, 16, 1024, kSwizzle128B), bdesc, idesc, sfa1_t + 4 * g,
-                     sfb_t + 8 * g, (ks > 0 || kk > 0) ? 1u : 0u);
-            mma_mxf4(d_tmem, smem_desc(a2 + kk * 32, 16, 1024, kSwizzle128B), bdesc, idesc, sfa2_t + 4 * g,
-                     sfb_t + 8 * g, 1u);
+            const uint32_t idesc = (kk & 1) ? idesc_hi : idesc_lo;   // which pair of scale bytes of the 4-scale column
+            mma_mxf4(d_tmem, a1d + 2 * kk, bd + 2 * kk, idesc, sfa1_t + 4 * g, sfb_t + 8 * g, (ks > 0 || kk > 0) ? 1u : 0u);
+            mma_mxf4(d_tmem, a2d + 2 * kk, bd + 2 * kk, idesc, sfa2_t + 4 * g, sfb_t + 8 * g, 1u);
           }
           tc_commit(&empty_bar[stage]);
           if (++stage == kW4Stages) { stage = 0; phase ^= 1; }
