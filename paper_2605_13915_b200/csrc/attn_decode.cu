@@ -144,7 +144,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       long long t_idle = clock64();
       while (kq < ntiles || vq < ntiles) {
         bool progressed = false;
-        if (kq < ntiles && mbar_try_wait(&kv_empty[kq % p.stages], ((kq / p.stages) & 1) ^ 1)) {
+        if (kq < ntiles && mbar_test_wait(&kv_empty[kq % p.stages], ((kq / p.stages) & 1) ^ 1)) {
           const int st = kq % p.stages;
           mbar_arrive_expect_tx(&kv_full[st], k_bytes);
           uint8_t* dst = smem + st * kv_stage_bytes;
@@ -153,7 +153,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           ++kq;
           progressed = true;
         }
-        if (vq < ntiles && mbar_try_wait(&v_empty[vq % p.stages], ((vq / p.stages) & 1) ^ 1)) {
+        if (vq < ntiles && mbar_test_wait(&v_empty[vq % p.stages], ((vq / p.stages) & 1) ^ 1)) {
           const int st = vq % p.stages;
           mbar_arrive_expect_tx(&v_full[st], v_bytes);
           uint8_t* dst = smem + st * kv_stage_bytes + k_bytes;
@@ -182,30 +182,43 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       bool ok = true;
       // the stacked Q operand is written by the softmax warps; they arrive on p_full once before the first tile
       ok = wait_bounded(&q_ready, 0, abort, p.status);
+      // Operand descriptors differ from three templates only in the 16-byte-granular address field (bits 0-13), so each
+      // costs one 64-bit add: with 36 MMAs per MLA tile this thread's instruction count is on the critical path.
+      const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);         // K-major tiles: K, stacked Q, P
+      const uint64_t dvt = smem_desc(0, 16384, 1024, kSwizzle128B);     // V^T read MN-major from the token-major tile
+      const uint64_t q_enc = dk + (smem_u32(sm_q) >> 4);
+      const uint64_t p_enc = dk + (smem_u32(sm_p) >> 4);
+      const uint32_t smem_enc = smem_u32(smem) >> 4;
+      const uint32_t q_step = static_cast<uint32_t>(p.Rp * kChunk) >> 4, p_step = q_step;
       auto issue_qk = [&](int t) {
         const int st = t % p.stages;
         tc_fence_after();
-        const uint32_t ka = smem_u32(smem + st * kv_stage_bytes);
-        const uint32_t qa = smem_u32(sm_q);
+        uint64_t ka = dk + smem_enc + static_cast<uint32_t>(st * (kv_stage_bytes >> 4));
+        uint64_t qa = q_enc;
         const uint32_t d = tmem_base + (t & 1) * p.Rp;
-        for (int c = 0; c < p.DC; ++c)
+        for (int c = 0; c < p.DC; ++c) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            mma_i8(d, smem_desc(ka + c * kChunkBytes + k * 32, 16, 1024, kSwizzle128B),
-                   smem_desc(qa + c * p.Rp * kChunk + k * 32, 16, 1024, kSwizzle128B), idesc_qk, (c > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < 4; ++k) mma_i8(d, ka + 2 * k, qa + 2 * k, idesc_qk, (c > 0 || k > 0) ? 1u : 0u);
+          ka += kChunkBytes >> 4;
+          qa += q_step;
+        }
         tc_commit(&s_full[t & 1]);
         if (!p.v_alias) tc_commit(&kv_empty[st]);       // separate V: the K buffer is free once QK^T has read it
       };
       auto issue_pv = [&](int t) {
         tc_fence_after();
         const int st = t % p.stages;
-        const uint32_t va = smem_u32(smem + st * kv_stage_bytes) + (p.v_alias ? 0 : p.DC * kChunkBytes);
-        const uint32_t pa = smem_u32(sm_p) + (t & 1) * p.Rp * kChunk;
-        for (int j = 0; j < p.DVT; ++j)
+        uint64_t va = dvt + smem_enc + static_cast<uint32_t>(st * (kv_stage_bytes >> 4)) +
+                      (p.v_alias ? 0u : static_cast<uint32_t>(p.DC * (kChunkBytes >> 4)));
+        const uint64_t pa = p_enc + (t & 1) * p_step;
+        uint32_t d = tmem_o;
+        for (int j = 0; j < p.DVT; ++j) {
 #pragma unroll
           for (int k = 0; k < 4; ++k)        // 32 tokens per MMA: four 8-token groups of 1024 bytes
-            mma_i8(tmem_o + j * p.Rp, smem_desc(va + j * kChunkBytes + k * 4096, 16384, 1024, kSwizzle128B),
-                   smem_desc(pa + k * 32, 16, 1024, kSwizzle128B), idesc_pv, k > 0 ? 1u : 0u);
+            mma_i8(d, va + k * (4096 >> 4), pa + 2 * k, idesc_pv, k > 0 ? 1u : 0u);
+          va += kChunkBytes >> 4;
+          d += p.Rp;
+        }
         tc_commit(&o_full);
         tc_commit(p.v_alias ? &kv_empty[st] : &v_empty[st]);
       };
@@ -218,13 +231,13 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       while (ok && v < ntiles) {
         bool progressed = false;
         if (q < ntiles && q < v + 2 &&
-            mbar_try_wait(&kv_full[q % p.stages], (q / p.stages) & 1)) {    // (q < v + 2 implies P of tile q-2 is written)
+            mbar_test_wait(&kv_full[q % p.stages], (q / p.stages) & 1)) {    // (q < v + 2 implies P of tile q-2 is written)
           issue_qk(q);
           ++q;
           progressed = true;
         }
-        if (v < q && mbar_try_wait(&p_full[v & 1], (v >> 1) & 1) && (v == 0 || mbar_try_wait(&o_empty, (v - 1) & 1)) &&
-            (p.v_alias || mbar_try_wait(&v_full[v % p.stages], (v / p.stages) & 1))) {
+        if (v < q && mbar_test_wait(&p_full[v & 1], (v >> 1) & 1) && (v == 0 || mbar_test_wait(&o_empty, (v - 1) & 1)) &&
+            (p.v_alias || mbar_test_wait(&v_full[v % p.stages], (v / p.stages) & 1))) {
           issue_pv(v);
           ++v;
           progressed = true;
