@@ -130,19 +130,16 @@ def make_inputs(torch, device, seed):
 
 def run_gpu(args):
     import torch
-    import torch.distributed as dist
     from paper_2605_13915_b200 import binding
+    from paper_2605_13915_b200.ranks import Ranks
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the MSD path has no CPU fallback")
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=device)
+    ranks = Ranks("nccl", device)        # replicas only: barrier, MAX of the times, no data-path collective
+    world, rank = ranks.world, ranks.rank
     binding.lib()
 
     data = make_inputs(torch, device, seed=1234 + rank)
@@ -177,16 +174,18 @@ def run_gpu(args):
     graph = capture(step)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        ranks.barrier()
         torch.cuda.synchronize()
 
-    def timed(replay, steps, warmup):
+    def timed(replay, steps, warmup, all_ranks=False):
+        """Device time of `steps` replays in ms.  all_ranks: barrier on both sides and the MAX over ranks (the
+        headline and end-to-end regions, which every rank runs); otherwise this rank alone (rank 0's breakdown)."""
+        sync = barrier if all_ranks else torch.cuda.synchronize
         with torch.cuda.stream(stream):
             for _ in range(warmup):
                 replay()
             stream.synchronize()
-            barrier()
+            sync()
             e0 = torch.cuda.Event(enable_timing=True)
             e1 = torch.cuda.Event(enable_timing=True)
             e0.record(stream)
@@ -194,18 +193,14 @@ def run_gpu(args):
                 replay()
             e1.record(stream)
             stream.synchronize()
-            barrier()
+            sync()
             ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=device, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return ranks.max_over_ranks(ms) if all_ranks else ms
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     if sampler:
         sampler.start()
-    ms = timed(graph.replay, args.steps, args.warmup)
+    ms = timed(graph.replay, args.steps, args.warmup, all_ranks=True)
     binding.last_device_status()
 
     # ---- end to end: activations and results in pinned host memory, copies inside the timed region ----
@@ -222,7 +217,7 @@ def run_gpu(args):
 
     e2e_graph = capture(e2e_step)
     e2e_steps = max(1, args.steps // 2)
-    ms_e2e = timed(e2e_graph.replay, e2e_steps, args.warmup)
+    ms_e2e = timed(e2e_graph.replay, e2e_steps, args.warmup, all_ranks=True)
     binding.last_device_status()
     h2d = sum(M * K * 2 for (M, N, K, *_r) in calls)
     d2h = sum(M * N * 2 for (M, N, K, *_r) in calls)
@@ -248,8 +243,7 @@ def run_gpu(args):
         other = other_configs(torch, binding, device, capture, timed)
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        ranks.close()
         return
 
     peaks, peak_kind = load_peaks()
@@ -285,8 +279,7 @@ def run_gpu(args):
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(check=(binding, data, torch))
     print(json.dumps(out), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    ranks.close()
 
 
 def other_configs(torch, binding, device, capture, timed):
