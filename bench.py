@@ -225,7 +225,7 @@ def run_gpu(args):
 
     # ---- per-call breakdown (one graph per call, outside the headline region) ----
     per_call = []
-    if rank == 0 and not args.no_breakdown:
+    if rank == 0 and world == 1 and not args.no_breakdown:      # single-GPU runs only: the scaling runs stay short
         for (M, N, K, x, w, s, y, wsp) in calls:
             ws_list = data[(N, K)][0]
 
@@ -239,7 +239,7 @@ def run_gpu(args):
                              "tops": round(executed_ops(M, N, K) / t / 1e6, 2)})
 
     other = {}
-    if rank == 0 and not args.no_breakdown:
+    if rank == 0 and world == 1 and not args.no_breakdown:
         other = other_configs(torch, binding, device, capture, timed)
 
     if rank != 0:
