@@ -51,10 +51,14 @@ struct GemmW8Params {
   int tmem_cols;
   int ytype;
   const float* w_scale;
-  const float* alpha;
-  const float* beta;
-  const uint16_t* x;       // fused path only: the BF16 activations [M, ldx], decomposed inside the kernel
+  float* alpha;
+  float* beta;
+  const uint16_t* x;       // in-kernel decomposition: the BF16 activations [M, ldx]
   long long ldx;
+  int inline_dec;          // 1: the first dec_ctas CTAs decompose the rows before the main loop, the others wait for a flag
+  int dec_ctas;
+  int8_t* q;               // stacked components [NB, K] (rows [0,M) = Q1, [Mp, Mp+M) = Q2) in the workspace
+  unsigned* flags;         // [2]: rows decomposed, CTAs that have seen all of them (both zero between calls)
   void* y;
   int32_t* acc_dbg;
   int32_t* accum;          // [num_tiles][NB][128] split-K meeting place, zero between calls (INT32 or FP32 bits)
@@ -300,7 +304,9 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
   __shared__ __align__(8) uint64_t tfull_bar[2];
   __shared__ __align__(8) uint64_t tempty_bar[2];
-  __shared__ __align__(8) uint64_t cfree_bar, crecv_bar, cdone_bar;      // mode 2: "pipelines of the cluster drained", "partials delivered"
+  __shared__ __align__(8) uint64_t cfree_bar, crecv_bar, cdone_bar;
+  __shared__ __align__(8) uint64_t xready_bar;               // in-kernel decomposition: every row is in memory
+  __shared__ float s_red[4];      // mode 2: "pipelines of the cluster drained", "partials delivered"
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ int is_last_flag;
@@ -364,6 +370,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       mbar_init(&tfull_bar[a], 1);
       mbar_init(&tempty_bar[a], 4);      // one arrival per epilogue warp
     }
+    mbar_init(&xready_bar, 1);
     if (p.mode == 2) {
       mbar_init(&cfree_bar, p.csplit);               // one arrival per CTA of the cluster
       mbar_init(&crecv_bar, 1);                      // this CTA's own arrival; the peers' copies count in bytes
@@ -431,7 +438,16 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   if (threadIdx.x == 0) trace_mark(p, 2);
 
   if (warp == 0) {
-    pdl_wait_primary();
+    if (!kBase && !kFused && p.inline_dec) {
+      // the stacked components are written by CTAs of this very kernel: the epilogue warps tell when all rows are there
+      int okw = 1;
+      if (lane == 0) okw = wait_bounded(&xready_bar, 0, abort, p.status) ? 1 : 0;
+      okw = __shfl_sync(0xffffffffu, okw, 0);
+      fence_proxy_async_all();      // generic-proxy stores of other CTAs, acquired above, before this warp's TMA reads
+      if (!okw) pre = 0, blk_end = blk_begin;
+    } else {
+      pdl_wait_primary();
+    }
     if (lane == 0) trace_mark(p, 4);
     {
       int kx = kbr0;
@@ -577,19 +593,78 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     const int quad = warp & 3;                    // TMEM lane group this warp may read
     const int r = quad * 32 + lane;               // weight row within the tile == TMEM lane
     const int et = threadIdx.x - 64;              // 0..127
+    bool return_early = false;
     if constexpr (kFused) {
       fused_row_scales(p, et, s_qmax, s_alpha, s_beta, s_inva, s_invb);   // together with the quantiser warps
     } else if constexpr (!kBase) {
       pdl_wait_primary();
-      if (et < p.M) {
-        s_alpha[et] = p.alpha[et];
-        s_beta[et] = p.beta[et];
+      if (p.inline_dec) {
+        // ---- a1-a3 inside the GEMM kernel: CTA c < dec_ctas decomposes rows c, c + dec_ctas, ... with its epilogue
+        // warps (idle until the first accumulator is complete) while its producer already streams weights; a counter
+        // in the workspace tells every CTA when all rows are in memory.  No kernel boundary between a3 and a4.
+        const int ndec = static_cast<int>(gridDim.x) < p.dec_ctas ? static_cast<int>(gridDim.x) : p.dec_ctas;
+        int rows_done = 0;
+        if (static_cast<int>(blockIdx.x) < ndec) {
+          const int nchunks = p.K >> 4;
+          for (int row = blockIdx.x; row < p.M; row += ndec, ++rows_done) {
+            const uint4* xr = reinterpret_cast<const uint4*>(p.x + static_cast<long long>(row) * p.ldx);
+            float m = 0.0f;
+            for (int c = et; c < nchunks; c += 128) m = fmaxf(m, chunk_absmax(__ldg(xr + 2 * c), __ldg(xr + 2 * c + 1)));
+            m = warp_max(m);
+            if (lane == 0) s_red[warp & 3] = m;
+            named_bar_sync(1, 128);
+            m = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+            named_bar_sync(1, 128);                              // s_red is rewritten for the next row
+            const float alpha = __fdiv_rn(m, 127.0f);            // Eq. alpha
+            const float beta = __fdiv_rn(alpha, 254.0f);         // Eq. beta
+            const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f;
+            const float inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
+            if (et == 0) { p.alpha[row] = alpha; p.beta[row] = beta; }
+            uint4* o1 = reinterpret_cast<uint4*>(p.q + static_cast<long long>(row) * p.K);
+            uint4* o2 = reinterpret_cast<uint4*>(p.q + static_cast<long long>(p.Mp + row) * p.K);
+            for (int c = et; c < nchunks; c += 128) {
+              uint4 r1, r2;
+              chunk_quantize(__ldg(xr + 2 * c), __ldg(xr + 2 * c + 1), alpha, beta, inv_alpha, inv_beta, r1, r2);
+              o1[c] = r1;
+              o2[c] = r2;
+            }
+          }
+        }
+        if (rows_done > 0) {
+          __threadfence();
+          fence_proxy_async_all();          // these rows are read through TMA (async proxy) by every CTA
+          named_bar_sync(1, 128);
+          if (et == 0) atomicAdd(&p.flags[0], static_cast<unsigned>(rows_done));
+        }
+        if (et == 0) {
+          // bounded poll for "all M rows decomposed"
+          const long long t0 = clock64();
+          bool seen = false;
+          while (true) {
+            unsigned v;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.flags) : "memory");
+            if (v >= static_cast<unsigned>(p.M)) { seen = true; break; }
+            if (*abort) break;
+            if (clock64() - t0 > kWaitBudgetCycles) { *abort = 1; atomicMax(p.status, kStatusTimeout); break; }
+          }
+          if (seen) {
+            mbar_arrive(&xready_bar);       // lets this CTA's producer request the component tiles
+            // the CTA that is last to see the full count leaves both counters zero for the next call
+            if (atomicAdd(&p.flags[1], 1u) == gridDim.x - 1) { p.flags[0] = 0; p.flags[1] = 0; }
+          }
+        }
+        named_bar_sync(1, 128);
+        if (*abort) return_early = true;
+      }
+      if (et < p.M && !return_early) {
+        s_alpha[et] = __ldcg(p.alpha + et);
+        s_beta[et] = __ldcg(p.beta + et);
       }
     }
     named_bar_sync(1, 128);
     int seg = 0;
     int sent_to = 0;           // mode 2: finishing CTAs whose acknowledgement is outstanding
-    bool ok = true;
+    bool ok = !return_early;
     long long blk = blk_begin;
     while (blk < blk_end && ok) {
       const int tile = static_cast<int>(blk / p.kblocks);
@@ -850,7 +925,8 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   pl.off_q = off;         off = round_up(off + (base ? static_cast<size_t>(N) * K * 2 : static_cast<size_t>(pl.NB) * K), 1024);
   pl.off_alpha = off;     off = round_up(off + 128 * sizeof(float), 256);
   pl.off_beta = off;      off = round_up(off + 128 * sizeof(float), 256);
-  pl.off_counters = off;  off = round_up(off + static_cast<size_t>(pl.num_tiles) * sizeof(unsigned), 1024);
+  // one arrival counter per weight tile, then the two counters of the in-kernel decomposition
+  pl.off_counters = off;  off = round_up(off + static_cast<size_t>(pl.num_tiles + 2) * sizeof(unsigned), 1024);
   // split-K meeting place: one [NB x 128] tile of sums per weight tile (used by the stream-K split only)
   pl.off_slots = off;     off = round_up(off + static_cast<size_t>(pl.num_tiles) * pl.NB * kTileN * sizeof(int32_t), 1024);
   pl.bytes = off;
@@ -965,7 +1041,12 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
   // Opt-in (MSD_GEMM_FUSED_MAXM=<largest M>): with one quantiser warp per stage the in-kernel path measured no faster
   // than the two-kernel path at M = 1 and slower from M = 2 on, so the default keeps the separate kernel.
   const bool fused = (M <= env_int("MSD_GEMM_FUSED_MAXM", 0)) && M <= kFusedMaxM && pl.mode != 2;
-  if (!fused) {
+  // Opt-in (MSD_GEMM_INLINE_DEC=1): rows are decomposed inside the GEMM kernel by its first CTAs, the others wait for a
+  // counter - no kernel boundary between a3 and a4.  Measured slower (M = 1: 20.0 vs 17.0 us at K = 4096, 33 vs 20 us
+  // at K = 14336): 128 threads per row and five dependent memory round trips (load, store + fence, counter, poll,
+  // TMA) cost more than the boundary they remove, whatever the weight prefetch depth.
+  const bool inline_dec = !fused && env_int("MSD_GEMM_INLINE_DEC", 0) != 0;
+  if (!fused && !inline_dec) {
     st = launch_decompose_int8(x_bf16, M, K, K, q, q + static_cast<size_t>(pl.Mp) * K, alpha, beta, s);
     if (st != MSD_OK) return st;
   }
@@ -992,6 +1073,10 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
 
   p.x = static_cast<const uint16_t*>(x_bf16);
   p.ldx = K;
+  p.inline_dec = inline_dec ? 1 : 0;
+  p.dec_ctas = sm_count();
+  p.q = q;
+  p.flags = p.counters + pl.num_tiles;
   if (!ensure_smem_attr()) return MSD_ERR_CUDA;
   if (fused) {
     // may become resident while earlier work in the stream still runs: it prefetches weights, then waits for that
@@ -1044,6 +1129,7 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = 0;
   p.pre_stages = 64;
+  p.inline_dec = 0; p.dec_ctas = 0; p.q = nullptr; p.flags = nullptr; p.x = nullptr; p.ldx = 0;
   p.mode = pl.mode; p.groups8 = pl.groups8; p.gran = pl.gran; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off; p.csplit = pl.csplit;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;

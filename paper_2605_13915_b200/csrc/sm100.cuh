@@ -105,6 +105,8 @@ __device__ __forceinline__ void bulk_copy_to_peer(uint32_t dst_caddr, const void
                ::"r"(dst_caddr), "r"(smem_u32(src_local)), "r"(bytes), "r"(mbar_caddr)
                : "memory");
 }
+// generic <-> async proxy ordering for every state space (global memory written with plain stores, read by TMA)
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 // arrive (release, cluster scope) on a barrier that may live in another CTA of the cluster
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t caddr) {

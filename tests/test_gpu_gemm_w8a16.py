@@ -97,6 +97,23 @@ def test_cluster_split_k_comparison_kernel(monkeypatch):
     assert rel_row_err(y.cpu().numpy(), ref).max() <= TOL
 
 
+def test_rows_decomposed_by_the_gemm_kernels_first_ctas(monkeypatch):
+    """Opt-in: no separate decomposition kernel; the first CTAs of the GEMM decompose the rows and a counter in the
+    workspace releases the others.  Same bits; repeated calls on one workspace check that the counters return to zero;
+    more rows than CTAs, and more CTAs than SMs."""
+    monkeypatch.setenv("MSD_GEMM_INLINE_DEC", "1")
+    c = inputs.gemm_w8_case(16, 640, 1536, seed=41)
+    ws = binding.workspace(binding.gemm_w8a16_workspace_bytes(16, 640, 1536))
+    for _ in range(3):
+        _check(c, torch.float32, ws)
+    _check(inputs.gemm_w8_case(128, 512, 6144, seed=42), torch.bfloat16)
+    _check(inputs.gemm_w8_case(1, 14336, 4096, seed=43), torch.float32)
+    monkeypatch.setenv("MSD_GEMM_CTAS", "3")
+    _check(inputs.gemm_w8_case(40, 256, 768, seed=44), torch.float32)
+    monkeypatch.setenv("MSD_GEMM_CTAS", "200")
+    _check(inputs.gemm_w8_case(33, 1152, 2048, seed=45), torch.float32)
+
+
 @pytest.mark.parametrize("fused", ["0", "8"])
 def test_small_m_with_and_without_in_kernel_decomposition(fused, monkeypatch):
     """M <= 8 can decompose the activations inside the GEMM kernel (opt-in); it must agree with the two-kernel path
