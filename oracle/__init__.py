@@ -43,6 +43,7 @@ def lib():
         _lib.msdo_max_threads.restype = C.c_int
         _lib.msdo_int8_gemm_acc.restype = C.c_int64
         _lib.msdo_gemm_w8a16.restype = C.c_int64
+        _lib.msdo_gemm_w8a16_c.restype = C.c_int64
     return _lib
 
 
@@ -105,14 +106,21 @@ def quantize_rows_int8(x_bits):
 
 
 # --- decompositions ----------------------------------------------------------
-def decompose_int8(x_bits):
+# Scaling constants of the two passes: Eq. alpha / Eq. beta, and the "fractional scaling" pair of Sec. 3.3 (as FP32).
+SCALING_DEFAULT = (127.0, 254.0)
+SCALING_FRACTIONAL = (127.49, 254.98)
+
+
+def decompose_int8(x_bits, fractional=False):
     x_bits = _c(x_bits, np.uint16)
     M, K = x_bits.shape
     q1 = np.empty((M, K), np.int8)
     q2 = np.empty((M, K), np.int8)
     a = np.empty(M, np.float32)
     b = np.empty(M, np.float32)
-    lib().msdo_decompose_int8(_p(x_bits), C.c_int64(M), C.c_int64(K), C.c_int64(K), _p(q1), _p(q2), _p(a), _p(b))
+    c1, c2 = SCALING_FRACTIONAL if fractional else SCALING_DEFAULT
+    lib().msdo_decompose_int8_c(_p(x_bits), C.c_int64(M), C.c_int64(K), C.c_int64(K), C.c_float(c1), C.c_float(c2),
+                                _p(q1), _p(q2), _p(a), _p(b))
     return q1, q2, a, b
 
 
@@ -175,7 +183,7 @@ def int8_gemm_acc(a, w):
 _YT = {"bf16": (0, np.uint16), "f32": (1, np.float32), "f64": (2, np.float64)}
 
 
-def gemm_w8a16(x_bits, w, w_scale, ytype="f64", want_acc=False):
+def gemm_w8a16(x_bits, w, w_scale, ytype="f64", want_acc=False, fractional=False):
     x_bits = _c(x_bits, np.uint16)
     w = _c(w, np.int8)
     w_scale = _c(w_scale, np.float32)
@@ -184,7 +192,9 @@ def gemm_w8a16(x_bits, w, w_scale, ytype="f64", want_acc=False):
     code, dt = _YT[ytype]
     y = np.empty((M, N), dt)
     acc = np.empty((2, M, N), np.int32) if want_acc else None
-    ov = lib().msdo_gemm_w8a16(_p(x_bits), _p(w), _p(w_scale), C.c_int64(M), C.c_int64(N), C.c_int64(K), _p(y), C.c_int(code), _p(acc))
+    c1, c2 = SCALING_FRACTIONAL if fractional else SCALING_DEFAULT
+    ov = lib().msdo_gemm_w8a16_c(_p(x_bits), _p(w), _p(w_scale), C.c_int64(M), C.c_int64(N), C.c_int64(K), C.c_float(c1),
+                                 C.c_float(c2), _p(y), C.c_int(code), _p(acc))
     assert ov == 0, "INT32 accumulator overflow"
     return (y, acc) if want_acc else y
 

@@ -77,17 +77,21 @@ inline int8_t clamp_i8(float v) {
 // residual, beta, x2; Algorithm 1 lines 1-5).  `alpha_fixed` < 0 means "derive
 // alpha from the row maximum"; otherwise the given alpha is used (the constant
 // scale of the softmax probabilities, Sec. 4.2 step 3).
+// (c1, c2) are the scaling constants: (127, 254) in Eq. alpha / Eq. beta, or the
+// "fractional scaling" pair (127.49, 254.98) of Sec. 3.3, which keeps the extreme
+// element's residual below alpha/2 and tightens the bound to M/65015.
 void two_pass_int8(const float* x, int64_t n, int64_t stride, float alpha_fixed,
-                   int8_t* q1, int8_t* q2, float* alpha_out, float* beta_out) {
+                   int8_t* q1, int8_t* q2, float* alpha_out, float* beta_out,
+                   float c1 = 127.0f, float c2 = 254.0f) {
   float alpha;
   if (alpha_fixed >= 0.0f) {
     alpha = alpha_fixed;
   } else {
     float m = 0.0f;
     for (int64_t k = 0; k < n; ++k) m = std::max(m, std::fabs(x[k * stride]));
-    alpha = m / 127.0f;                                  // Eq. alpha
+    alpha = m / c1;                                      // Eq. alpha
   }
-  float beta = alpha / 254.0f;                           // Eq. beta
+  float beta = alpha / c2;                               // Eq. beta
   for (int64_t k = 0; k < n; ++k) {
     float v = x[k * stride];
     int8_t a = 0, b = 0;
@@ -274,15 +278,22 @@ void msdo_quantize_rows_int8(const uint16_t* x_bf16, int64_t rows, int64_t D, in
 // Decompositions
 // ---------------------------------------------------------------------------
 
-// Two-pass INT8 decomposition per row (Sec. 3.2, Eqs. alpha..x2; Alg. 1 lines 1-5).
-void msdo_decompose_int8(const uint16_t* x_bf16, int64_t M, int64_t K, int64_t ldx,
-                         int8_t* q1, int8_t* q2, float* alpha, float* beta) {
+// Two-pass INT8 decomposition per row (Sec. 3.2, Eqs. alpha..x2; Alg. 1 lines 1-5) with the
+// scaling constants given (Sec. 3.3, "fractional scaling": 127.49 and 254.98 instead of 127 and 254).
+void msdo_decompose_int8_c(const uint16_t* x_bf16, int64_t M, int64_t K, int64_t ldx, float c1, float c2,
+                           int8_t* q1, int8_t* q2, float* alpha, float* beta) {
 #pragma omp parallel for schedule(static)
   for (int64_t i = 0; i < M; ++i) {
     std::vector<float> row(K);
     for (int64_t k = 0; k < K; ++k) row[k] = bf16_to_f32(x_bf16[i * ldx + k]);
-    two_pass_int8(row.data(), K, 1, -1.0f, q1 + i * K, q2 + i * K, alpha + i, beta + i);
+    two_pass_int8(row.data(), K, 1, -1.0f, q1 + i * K, q2 + i * K, alpha + i, beta + i, c1, c2);
   }
+}
+
+// Two-pass INT8 decomposition per row (Sec. 3.2, Eqs. alpha..x2; Alg. 1 lines 1-5).
+void msdo_decompose_int8(const uint16_t* x_bf16, int64_t M, int64_t K, int64_t ldx,
+                         int8_t* q1, int8_t* q2, float* alpha, float* beta) {
+  msdo_decompose_int8_c(x_bf16, M, K, ldx, 127.0f, 254.0f, q1, q2, alpha, beta);
 }
 
 // Same rule on FP32 data with a caller-fixed alpha (< 0: derive from the row max).  Used by the
@@ -366,11 +377,11 @@ int64_t msdo_int8_gemm_acc(const int8_t* a, const int8_t* w, int64_t M, int64_t 
 // W8A16 MSD linear layer (Alg. 1): decompose, two exact integer GEMMs, y = s_W * (alpha*Y1 + beta*Y2)
 // combined in FP64 and rounded once.  ytype 0: BF16 (uint16_t), 1: FP32, 2: FP64 (unrounded).
 // acc_dbg (nullable): [2, M, N] INT32 accumulators.
-int64_t msdo_gemm_w8a16(const uint16_t* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
-                        int64_t K, void* y, int ytype, int32_t* acc_dbg) {
+int64_t msdo_gemm_w8a16_c(const uint16_t* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
+                          int64_t K, float c1, float c2, void* y, int ytype, int32_t* acc_dbg) {
   std::vector<int8_t> q1(M * K), q2(M * K);
   std::vector<float> alpha(M), beta(M);
-  msdo_decompose_int8(x_bf16, M, K, K, q1.data(), q2.data(), alpha.data(), beta.data());
+  msdo_decompose_int8_c(x_bf16, M, K, K, c1, c2, q1.data(), q2.data(), alpha.data(), beta.data());
   std::vector<int32_t> acc(2 * M * N);
   int64_t ov = msdo_int8_gemm_acc(q1.data(), w, M, N, K, acc.data());
   ov += msdo_int8_gemm_acc(q2.data(), w, M, N, K, acc.data() + M * N);
@@ -384,6 +395,11 @@ int64_t msdo_gemm_w8a16(const uint16_t* x_bf16, const int8_t* w, const float* w_
       else static_cast<double*>(y)[i * N + n] = v;
     }
   return ov;
+}
+
+int64_t msdo_gemm_w8a16(const uint16_t* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
+                        int64_t K, void* y, int ytype, int32_t* acc_dbg) {
+  return msdo_gemm_w8a16_c(x_bf16, w, w_scale, M, N, K, 127.0f, 254.0f, y, ytype, acc_dbg);
 }
 
 // FP64 reference on the dequantized weights: y = sum_k x[i,k] * (s_W[n] * w[n,k])  (Eq. in Sec. 3.1).

@@ -43,6 +43,38 @@ def test_theorem1_bound_and_ranges(outliers):
     assert np.allclose(a, M / 127, rtol=1e-6) and np.allclose(b, M / 127 / 254, rtol=1e-6)
 
 
+def test_fractional_scaling_bound_and_extreme_element():
+    """Sec. 3.3 "fractional scaling": alpha = M/127.49, beta = alpha/254.98 tightens the bound to M/65015
+    (= 127.49 * 254.98 * 2), still without clipping; the extreme element maps to 127 with residual 0.49 alpha,
+    i.e. second code round(0.49 * 254.98) = 125; and the default constants stay what they were."""
+    xb = _x_rows(64, 4096, 5, True)
+    x = oracle.bf16_bits_to_f64(xb)
+    M = np.abs(x).max(axis=1)
+    q1, q2, a, b = oracle.decompose_int8(xb, fractional=True)
+    assert np.allclose(a, M / 127.49, rtol=2e-7) and np.allclose(b, a / 254.98, rtol=2e-7)
+    rec = a.astype(np.float64)[:, None] * q1 + b.astype(np.float64)[:, None] * q2
+    ratio = np.abs(x - rec).max(axis=1) / (M / (127.49 * 254.98 * 2.0))
+    assert ratio.max() <= 1.0 + 2.0 ** -15 and ratio.max() > 0.9
+    assert np.abs(q1).max() == 127 and np.abs(q2).max() <= 127
+    for i in range(len(M)):
+        k = int(np.argmax(np.abs(x[i])))
+        assert abs(int(q1[i, k])) == 127 and abs(int(q2[i, k])) == 125
+        assert np.sign(q2[i, k]) == np.sign(x[i, k])
+    # the tighter bound shows in the data as well, and the default call is untouched by the new parameter
+    d1, d2, da, db = oracle.decompose_int8(xb)
+    assert np.array_equal(da, (M / 127.0).astype(np.float32)) or np.allclose(da, M / 127.0, rtol=2e-7)
+    err_def = np.abs(x - (da.astype(np.float64)[:, None] * d1 + db.astype(np.float64)[:, None] * d2)).max(axis=1)
+    assert np.mean(np.abs(x - rec).max(axis=1) / err_def) < 1.0
+    # the GEMM with the flag is the stacked integer product of exactly these components
+    c = inputs.gemm_w8_case(4, 64, 256, seed=9)
+    y, acc = oracle.gemm_w8a16(c.x, c.w, c.w_scale, "f64", want_acc=True, fractional=True)
+    g1, g2, ga, gb = oracle.decompose_int8(c.x, fractional=True)
+    w = c.w.astype(np.int64)
+    assert np.array_equal(acc[0], g1.astype(np.int64) @ w.T) and np.array_equal(acc[1], g2.astype(np.int64) @ w.T)
+    want = c.w_scale.astype(np.float64)[None, :] * (ga.astype(np.float64)[:, None] * acc[0] + gb.astype(np.float64)[:, None] * acc[1])
+    assert np.allclose(y, want, rtol=1e-14, atol=0)
+
+
 def test_special_rows():
     K = 256
     x = np.zeros((5, K), np.float32)
