@@ -41,6 +41,12 @@ typedef enum {
   MSD_ERR_TIMEOUT = 7
 } msd_status_t;
 
+/* Scaling constants of the two INT8 passes: alpha = max|x| / c1, beta = alpha / c2.
+ * DEFAULT: c1 = 127, c2 = 254 (Eq. alpha, Eq. beta).  FRACTIONAL: c1 = 127.49, c2 = 254.98 (Sec. 3.3, "fractional
+ * scaling"): the extreme element keeps a residual of 0.49 alpha, the reconstruction bound tightens from max/64516 to
+ * max/65015, still no clipping. */
+typedef enum { MSD_SCALING_DEFAULT = 0, MSD_SCALING_FRACTIONAL = 1 } msd_scaling_t;
+
 typedef enum { MSD_OUT_BF16 = 0, MSD_OUT_FP32 = 1 } msd_out_t;
 
 const char* msd_status_string(msd_status_t s);
@@ -63,6 +69,9 @@ msd_status_t msd_workspace_init(void* workspace, size_t workspace_bytes, void* s
  */
 msd_status_t msd_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
                                 float* alpha, float* beta, void* stream);
+/* The same with the scaling constants chosen (msd_scaling_t above); anything else: MSD_ERR_UNSUPPORTED. */
+msd_status_t msd_decompose_int8_ex(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
+                                   float* alpha, float* beta, msd_scaling_t scaling, void* stream);
 
 /*
  * Two-pass MXFP4 decomposition per 32-element K block (Sec. 3.2.1, Alg. 2) on the E2M1 grid
@@ -89,6 +98,11 @@ size_t msd_gemm_w8a16_workspace_bytes(int64_t M, int64_t N, int64_t K);
 msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
                             int64_t K, void* y, msd_out_t ytype, int32_t* acc_dbg, void* workspace,
                             size_t workspace_bytes, void* stream);
+/* The same layer with the scaling constants of the activation decomposition chosen (Sec. 3.3); the weights, the
+ * integer GEMM and the combine are unchanged. */
+msd_status_t msd_gemm_w8a16_ex(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
+                               int64_t K, void* y, msd_out_t ytype, int32_t* acc_dbg, msd_scaling_t scaling,
+                               void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * The same W8A16 layer for callers that cannot allocate device memory.  (The paper has no counterpart; this is a

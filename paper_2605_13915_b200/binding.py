@@ -32,9 +32,11 @@ _SIGS = {
     "msd_last_device_status": (C.c_int, [_vp]),
     "msd_workspace_init": (C.c_int, [_vp, _sz, _vp]),
     "msd_decompose_int8": (C.c_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp]),
+    "msd_decompose_int8_ex": (C.c_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, C.c_int, _vp]),
     "msd_decompose_mxfp4": (C.c_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp]),
     "msd_gemm_w8a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_w8a16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _vp, _sz, _vp]),
+    "msd_gemm_w8a16_ex": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_gemm_w8a16_noalloc": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp]),
     "msd_debug_set_trace": (None, [_vp]),
     "msd_debug_set_attn_trace": (None, [_vp]),
@@ -104,14 +106,21 @@ def _ws_ptr(ws):
     return C.c_void_p(al), ws.numel() - (al - base)
 
 
-def decompose_int8(x):
-    """x [M,K] bfloat16 -> (q1, q2 int8 [M,K], alpha, beta float32 [M])."""
+SCALING_DEFAULT, SCALING_FRACTIONAL = 0, 1
+
+
+def decompose_int8(x, fractional=False):
+    """x [M,K] bfloat16 -> (q1, q2 int8 [M,K], alpha, beta float32 [M]); fractional: scaling constants 127.49 / 254.98."""
     _need_cuda(x)
     M, K = x.shape
     q1 = torch.empty((M, K), dtype=torch.int8, device=x.device)
     q2 = torch.empty((M, K), dtype=torch.int8, device=x.device)
     a = torch.empty(M, dtype=torch.float32, device=x.device)
     b = torch.empty(M, dtype=torch.float32, device=x.device)
+    if fractional:
+        _check(lib().msd_decompose_int8_ex(_ptr(x), M, K, x.stride(0) if M else K, _ptr(q1), _ptr(q2), _ptr(a), _ptr(b),
+                                           SCALING_FRACTIONAL, _stream()), "msd_decompose_int8_ex")
+        return q1, q2, a, b
     _check(lib().msd_decompose_int8(_ptr(x), M, K, x.stride(0) if M else K, _ptr(q1), _ptr(q2), _ptr(a), _ptr(b), _stream()),
            "msd_decompose_int8")
     return q1, q2, a, b
@@ -134,7 +143,7 @@ def gemm_w8a16_workspace_bytes(M, N, K):
     return int(lib().msd_gemm_w8a16_workspace_bytes(M, N, K))
 
 
-def gemm_w8a16(x, w, w_scale, out_dtype=torch.bfloat16, ws=None, want_acc=False, out=None):
+def gemm_w8a16(x, w, w_scale, out_dtype=torch.bfloat16, ws=None, want_acc=False, out=None, fractional=False):
     """x [M,K] bf16, w [N,K] int8, w_scale [N] f32 -> y [M,N] (bf16 or f32); optional INT32 accumulators [2,M,N]."""
     _need_cuda(x, w, w_scale)
     M, K = x.shape
@@ -144,8 +153,12 @@ def gemm_w8a16(x, w, w_scale, out_dtype=torch.bfloat16, ws=None, want_acc=False,
     y = out if out is not None else torch.empty((M, N), dtype=out_dtype, device=x.device)
     acc = torch.empty((2, M, N), dtype=torch.int32, device=x.device) if want_acc else None
     wp, wb = _ws_ptr(ws)
-    code = lib().msd_gemm_w8a16(_ptr(x), _ptr(w), _ptr(w_scale), M, N, K, _ptr(y), OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32,
-                                _ptr(acc), wp, wb, _stream())
+    yt = OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32
+    if fractional:
+        code = lib().msd_gemm_w8a16_ex(_ptr(x), _ptr(w), _ptr(w_scale), M, N, K, _ptr(y), yt, _ptr(acc), SCALING_FRACTIONAL, wp, wb,
+                                       _stream())
+    else:
+        code = lib().msd_gemm_w8a16(_ptr(x), _ptr(w), _ptr(w_scale), M, N, K, _ptr(y), yt, _ptr(acc), wp, wb, _stream())
     _check(code, "msd_gemm_w8a16")
     return (y, acc) if want_acc else y
 

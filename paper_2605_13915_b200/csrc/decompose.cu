@@ -22,7 +22,8 @@ constexpr int kDecCache = 4;   // 16-element chunks a thread keeps in registers 
 template <int kDecThreads>
 __global__ void __launch_bounds__(kDecThreads)
 decompose_int8_kernel(const uint16_t* __restrict__ x, int64_t ldx, int K, int8_t* __restrict__ q1,
-                      int8_t* __restrict__ q2, float* __restrict__ alpha_out, float* __restrict__ beta_out, int early_trigger) {
+                      int8_t* __restrict__ q2, float* __restrict__ alpha_out, float* __restrict__ beta_out, int early_trigger,
+                      float c1, float c2) {
   // When launched as a programmatic dependent of whatever precedes it in the stream it may become resident early, but
   // it reads nothing before that work has completed (the wait is a no-op for a plain launch); only then may its own
   // dependent (the GEMM) start prefetching weights.
@@ -55,8 +56,8 @@ decompose_int8_kernel(const uint16_t* __restrict__ x, int64_t ldx, int K, int8_t
 #pragma unroll
   for (int w = 1; w < kDecThreads / 32; ++w) m = fmaxf(m, warp_max[w]);
 
-  const float alpha = __fdiv_rn(m, 127.0f);        // Eq. alpha
-  const float beta = __fdiv_rn(alpha, 254.0f);     // Eq. beta
+  const float alpha = __fdiv_rn(m, c1);            // Eq. alpha (c1 = 127, or 127.49 with fractional scaling, Sec. 3.3)
+  const float beta = __fdiv_rn(alpha, c2);         // Eq. beta  (c2 = 254, or 254.98)
   // reciprocals only steer the fast path of quant_i8; infinities (tiny scales) simply send every element to the division
   const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f;
   const float inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
@@ -150,7 +151,7 @@ decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, i
 }
 
 msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
-                                   float* alpha, float* beta, cudaStream_t stream) {
+                                   float* alpha, float* beta, float c1, float c2, cudaStream_t stream) {
   if (M == 0) return MSD_OK;
   // Chained programmatic launch (this kernel resident while its predecessor still runs) is opt-in: measured slower.
   const bool pdl = getenv("MSD_DEC_CHAIN") != nullptr && getenv("MSD_NO_PDL") == nullptr;
@@ -161,13 +162,13 @@ msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int
   cudaError_t err;
   if (threads >= 1024)
     err = launch_pdl(decompose_int8_kernel<1024>, dim3(static_cast<unsigned>(M)), dim3(1024), 0, stream, pdl,
-                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, early);
+                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, early, c1, c2);
   else if (threads >= 512)
     err = launch_pdl(decompose_int8_kernel<512>, dim3(static_cast<unsigned>(M)), dim3(512), 0, stream, pdl,
-                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, early);
+                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, early, c1, c2);
   else
     err = launch_pdl(decompose_int8_kernel<256>, dim3(static_cast<unsigned>(M)), dim3(256), 0, stream, pdl,
-                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, early);
+                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, early, c1, c2);
   return err == cudaSuccess ? MSD_OK : MSD_ERR_CUDA;
 }
 
@@ -192,15 +193,22 @@ msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, in
 
 extern "C" {
 
-msd_status_t msd_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
-                                float* alpha, float* beta, void* stream) {
+msd_status_t msd_decompose_int8_ex(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
+                                   float* alpha, float* beta, msd_scaling_t scaling, void* stream) {
+  if (scaling != MSD_SCALING_DEFAULT && scaling != MSD_SCALING_FRACTIONAL) return MSD_ERR_UNSUPPORTED;
   if (M < 0 || K <= 0 || K % 16 != 0 || ldx < K || ldx % 8 != 0 || M > 0x7FFFFFFF || K > 0x7FFFFFF0) return MSD_ERR_BAD_SHAPE;
   if (M == 0) return MSD_OK;
   if (!x_bf16 || !q1 || !q2 || !alpha || !beta) return MSD_ERR_NULL_POINTER;
   if (!msd::aligned(x_bf16, 16) || !msd::aligned(q1, 16) || !msd::aligned(q2, 16) || !msd::aligned(alpha, 4) ||
       !msd::aligned(beta, 4))
     return MSD_ERR_BAD_ALIGNMENT;
-  return msd::launch_decompose_int8(x_bf16, M, K, ldx, q1, q2, alpha, beta, static_cast<cudaStream_t>(stream));
+  return msd::launch_decompose_int8(x_bf16, M, K, ldx, q1, q2, alpha, beta, msd::scaling_c1(scaling), msd::scaling_c2(scaling),
+                                    static_cast<cudaStream_t>(stream));
+}
+
+msd_status_t msd_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
+                                float* alpha, float* beta, void* stream) {
+  return msd_decompose_int8_ex(x_bf16, M, K, ldx, q1, q2, alpha, beta, MSD_SCALING_DEFAULT, stream);
 }
 
 msd_status_t msd_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,

@@ -57,6 +57,7 @@ struct GemmW8Params {
   long long ldx;
   int inline_dec;          // 1: the first dec_ctas CTAs decompose the rows before the main loop, the others wait for a flag
   int dec_ctas;
+  float c1, c2;            // scaling constants of the in-kernel decompositions (alpha = max/c1, beta = alpha/c2)
   int8_t* q;               // stacked components [NB, K] (rows [0,M) = Q1, [Mp, Mp+M) = Q2) in the workspace
   unsigned* flags;         // [2]: rows decomposed, CTAs that have seen all of them (both zero between calls)
   void* y;
@@ -279,7 +280,7 @@ __device__ __forceinline__ void fused_row_scales(const GemmW8Params& p, int t256
     float mm = 0.0f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) mm = fmaxf(mm, s_qmax[t256][w]);
-    const float alpha = __fdiv_rn(mm, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
+    const float alpha = __fdiv_rn(mm, p.c1), beta = __fdiv_rn(alpha, p.c2);
     s_alpha[t256] = alpha;
     s_beta[t256] = beta;
     s_inva[t256] = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f;
@@ -615,8 +616,8 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             named_bar_sync(1, 128);
             m = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
             named_bar_sync(1, 128);                              // s_red is rewritten for the next row
-            const float alpha = __fdiv_rn(m, 127.0f);            // Eq. alpha
-            const float beta = __fdiv_rn(alpha, 254.0f);         // Eq. beta
+            const float alpha = __fdiv_rn(m, p.c1);              // Eq. alpha
+            const float beta = __fdiv_rn(alpha, p.c2);           // Eq. beta
             const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f;
             const float inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
             if (et == 0) { p.alpha[row] = alpha; p.beta[row] = beta; }
@@ -1023,7 +1024,14 @@ size_t msd_gemm_w8a16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
                             int64_t K, void* y, msd_out_t ytype, int32_t* acc_dbg, void* workspace,
                             size_t workspace_bytes, void* stream) {
+  return msd_gemm_w8a16_ex(x_bf16, w, w_scale, M, N, K, y, ytype, acc_dbg, MSD_SCALING_DEFAULT, workspace, workspace_bytes, stream);
+}
+
+msd_status_t msd_gemm_w8a16_ex(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
+                               int64_t K, void* y, msd_out_t ytype, int32_t* acc_dbg, msd_scaling_t scaling,
+                               void* workspace, size_t workspace_bytes, void* stream) {
   using namespace msd;
+  if (scaling != MSD_SCALING_DEFAULT && scaling != MSD_SCALING_FRACTIONAL) return MSD_ERR_UNSUPPORTED;
   msd_status_t st = check_w8_args(x_bf16, w, w_scale, M, N, K, y, ytype, workspace);
   if (st != MSD_OK) return st;
   const GemmW8Plan pl = plan_w8(M, N, K);
@@ -1047,7 +1055,8 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
   // TMA) cost more than the boundary they remove, whatever the weight prefetch depth.
   const bool inline_dec = !fused && env_int("MSD_GEMM_INLINE_DEC", 0) != 0;
   if (!fused && !inline_dec) {
-    st = launch_decompose_int8(x_bf16, M, K, K, q, q + static_cast<size_t>(pl.Mp) * K, alpha, beta, s);
+    st = launch_decompose_int8(x_bf16, M, K, K, q, q + static_cast<size_t>(pl.Mp) * K, alpha, beta, scaling_c1(scaling),
+                               scaling_c2(scaling), s);
     if (st != MSD_OK) return st;
   }
 
@@ -1074,6 +1083,8 @@ msd_status_t msd_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_
   p.x = static_cast<const uint16_t*>(x_bf16);
   p.ldx = K;
   p.inline_dec = inline_dec ? 1 : 0;
+  p.c1 = scaling_c1(scaling);
+  p.c2 = scaling_c2(scaling);
   p.dec_ctas = sm_count();
   p.q = q;
   p.flags = p.counters + pl.num_tiles;
@@ -1129,7 +1140,7 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = 0;
   p.pre_stages = 64;
-  p.inline_dec = 0; p.dec_ctas = 0; p.q = nullptr; p.flags = nullptr; p.x = nullptr; p.ldx = 0;
+  p.c1 = 127.0f; p.c2 = 254.0f; p.inline_dec = 0; p.dec_ctas = 0; p.q = nullptr; p.flags = nullptr; p.x = nullptr; p.ldx = 0;
   p.mode = pl.mode; p.groups8 = pl.groups8; p.gran = pl.gran; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off; p.csplit = pl.csplit;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;

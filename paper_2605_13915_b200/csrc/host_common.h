@@ -62,8 +62,11 @@ cudaError_t launch_pdl(void (*kernel)(Args...), dim3 grid, dim3 block, size_t sm
 }
 
 // Internal entry used by the GEMM: decomposition written straight into the stacked operand buffer.
+// (c1, c2): the scaling constants of the two passes, alpha = max/c1 and beta = alpha/c2.
 msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
-                                   float* alpha, float* beta, cudaStream_t stream);
+                                   float* alpha, float* beta, float c1, float c2, cudaStream_t stream);
+inline float scaling_c1(msd_scaling_t s) { return s == MSD_SCALING_FRACTIONAL ? 127.49f : 127.0f; }
+inline float scaling_c2(msd_scaling_t s) { return s == MSD_SCALING_FRACTIONAL ? 254.98f : 254.0f; }
 msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
                                     uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream);
 

@@ -83,3 +83,20 @@ def test_decompose_mxfp4_extreme_exponents():
     assert np.array_equal(e1.cpu().numpy(), oe1) and np.array_equal(e2.cpu().numpy(), oe2)
     assert np.array_equal(canon_fp4(q1.cpu().numpy()), canon_fp4(o1))
     assert np.array_equal(canon_fp4(q2.cpu().numpy()), canon_fp4(o2))
+
+
+@pytest.mark.parametrize("M,K", [(3, 48), (16, 4096), (5, 14336)])
+def test_decompose_int8_fractional_scaling_bit_exact(M, K):
+    """Sec. 3.3: alpha = max/127.49, beta = alpha/254.98 through msd_decompose_int8_ex; an unknown scaling is refused."""
+    xb = inputs.activations(M, K, seed=2 * M + K)
+    q1, q2, a, b = binding.decompose_int8(bf16_dev(xb), fractional=True)
+    o1, o2, oa, ob = oracle.decompose_int8(xb, fractional=True)
+    assert np.array_equal(a.cpu().numpy(), oa) and np.array_equal(b.cpu().numpy(), ob)
+    assert np.array_equal(q1.cpu().numpy(), o1) and np.array_equal(q2.cpu().numpy(), o2)
+    d1, _d2, da, _db = oracle.decompose_int8(xb)
+    assert not np.array_equal(oa, da)                      # the flag does change the scales
+    x = bf16_dev(xb)
+    code = binding.lib().msd_decompose_int8_ex(x.data_ptr(), M, K, K, q1.data_ptr(), q2.data_ptr(), a.data_ptr(), b.data_ptr(), 7,
+                                               None)
+    assert code == 4                                       # MSD_ERR_UNSUPPORTED
+    binding.last_device_status()

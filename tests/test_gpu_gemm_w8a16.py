@@ -97,6 +97,23 @@ def test_cluster_split_k_comparison_kernel(monkeypatch):
     assert rel_row_err(y.cpu().numpy(), ref).max() <= TOL
 
 
+@pytest.mark.parametrize("inline", ["0", "1"])
+def test_fractional_scaling_layer(inline, monkeypatch):
+    """msd_gemm_w8a16_ex with the scaling constants of Sec. 3.3 (127.49 / 254.98): accumulators bit-exact against the
+    oracle run with the same constants, through the separate decomposition kernel and the in-kernel one."""
+    monkeypatch.setenv("MSD_GEMM_INLINE_DEC", inline)
+    for (M, N, K, seed) in [(5, 384, 272, 51), (16, 4096, 4096, 52), (128, 512, 1024, 53)]:
+        c = inputs.gemm_w8_case(M, N, K, seed=seed)
+        y, acc = binding.gemm_w8a16(bf16_dev(c.x), dev(c.w), dev(c.w_scale), out_dtype=torch.float32, want_acc=True, fractional=True)
+        torch.cuda.synchronize()
+        binding.last_device_status()
+        ref, oacc = oracle.gemm_w8a16(c.x, c.w, c.w_scale, "f64", want_acc=True, fractional=True)
+        assert np.array_equal(acc.cpu().numpy(), oacc)
+        assert rel_row_err(y.cpu().numpy(), ref).max() <= TOL
+        _, dacc = oracle.gemm_w8a16(c.x, c.w, c.w_scale, "f64", want_acc=True)
+        assert not np.array_equal(oacc, dacc)
+
+
 def test_rows_decomposed_by_the_gemm_kernels_first_ctas(monkeypatch):
     """Opt-in: no separate decomposition kernel; the first CTAs of the GEMM decompose the rows and a counter in the
     workspace releases the others.  Same bits; repeated calls on one workspace check that the counters return to zero;
