@@ -185,6 +185,22 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
                                     float softmax_scale, void* out_bf16, float* lse, void* workspace,
                                     size_t workspace_bytes, void* stream);
 
+/*
+ * The same attention over a PAGED cache (serving layouts; the paper's kernels read a contiguous cache, Alg. 3):
+ *   k_cache [num_blocks * page_size, Hkv, D], v_cache [num_blocks * page_size, Hkv, Dv] or NULL, scales
+ *   [num_blocks * page_size, Hkv]; block_table [B, max_blocks_per_seq] INT32 (device): logical token u of sequence b
+ *   is row block_table[b][u / page_size] * page_size + u % page_size; seqlens [B] INT32 (device).
+ * page_size: a power of two from 8 to 128.  Entries of block_table past ceil(seqlens[b] / page_size) are never read.
+ * max_seqlen >= every seqlens[b] and <= max_blocks_per_seq * page_size.  Workspace, schedule, outputs and errors as for
+ * msd_attn_decode_int8kv (same max_seqlen); an unsupported page size returns MSD_ERR_UNSUPPORTED.
+ */
+msd_status_t msd_attn_decode_int8kv_paged(const void* q_bf16, const int8_t* k_cache, const int8_t* v_cache,
+                                          const float* k_scale, const float* v_scale, const int32_t* block_table,
+                                          const int32_t* seqlens, int64_t num_blocks, int32_t page_size,
+                                          int32_t max_blocks_per_seq, int32_t max_seqlen, int32_t B, int32_t Hq, int32_t Hkv,
+                                          int32_t D, int32_t Dv, float softmax_scale, void* out_bf16, float* lse,
+                                          void* workspace, size_t workspace_bytes, void* stream);
+
 /* The split schedule msd_attn_decode_int8kv uses (so a checker can mirror it): writes the tile size, the number of
  * context splits and the tokens per split; split s of a sequence of length L covers tokens
  * [s*split_tokens, min(L, (s+1)*split_tokens)) and is walked in tiles of `tile` tokens (splits past L are empty). */

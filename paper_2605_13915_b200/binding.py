@@ -50,6 +50,8 @@ _SIGS = {
     "msd_attn_decode_int8kv": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp,
                                          _vp, _sz, _vp]),
     "msd_attn_decode_schedule": (C.c_int, [_i32] * 6 + [C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
+    "msd_attn_decode_int8kv_paged": (C.c_int, [_vp] * 7 + [_i64, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp, _vp,
+                                                _sz, _vp]),
     "msd_kv_dequant_bf16": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, _i32, _i32, C.c_void_p, C.c_void_p]),
 }
 
@@ -230,6 +232,27 @@ def attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen):
     _check(lib().msd_attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen, C.byref(tile), C.byref(ns), C.byref(st)),
            "msd_attn_decode_schedule")
     return tile.value, ns.value, st.value
+
+
+def attn_decode_int8kv_paged(q, k, v, k_scale, v_scale, block_table, seqlens, page_size, max_seqlen, softmax_scale, dv=None,
+                             ws=None, want_lse=False, out=None):
+    """Paged cache: k [num_blocks*page, Hkv, D] int8, v likewise or None, scales [num_blocks*page, Hkv] f32,
+    block_table [B, max_blocks] int32, seqlens [B] int32."""
+    _need_cuda(q, k, v, k_scale, v_scale, block_table, seqlens)
+    B, Hq, D = q.shape
+    Hkv = k.shape[1]
+    Dv = v.shape[2] if v is not None else dv
+    nblk = k.shape[0] // page_size
+    if ws is None:
+        ws = workspace(attn_decode_int8kv_workspace_bytes(B, Hq, Hkv, D, Dv, max_seqlen), q.device)
+    o = out if out is not None else torch.empty((B, Hq, Dv), dtype=torch.bfloat16, device=q.device)
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    wp, wb = _ws_ptr(ws)
+    code = lib().msd_attn_decode_int8kv_paged(_ptr(q), _ptr(k), _ptr(v), _ptr(k_scale), _ptr(v_scale), _ptr(block_table), _ptr(seqlens),
+                                              nblk, page_size, block_table.shape[1], max_seqlen, B, Hq, Hkv, D, Dv, softmax_scale,
+                                              _ptr(o), _ptr(lse), wp, wb, _stream())
+    _check(code, "msd_attn_decode_int8kv_paged")
+    return (o, lse) if want_lse else o
 
 
 def kv_dequant_bf16(cache, scale, out=None):

@@ -32,7 +32,12 @@ struct AttnParams {
   const uint16_t* q;      // [B,Hq,D] BF16
   const float* k_scale;   // [T,Hkv]
   const float* v_scale;   // [T,Hkv]
-  const int32_t* cu;      // [B+1]
+  const int32_t* cu;      // [B+1] token offsets of the sequences in a contiguous cache (unused when paged)
+  // paged cache (block_table != nullptr): the cache is [num_blocks * page, Hkv, D]; logical token u of sequence b lives
+  // in physical row block_table[b * max_blocks + u / page] * page + u % page; page is a power of two dividing the tile
+  const int32_t* block_table;
+  const int32_t* seqlens; // [B] (paged only)
+  int page, page_shift, max_blocks;
   float* partial;         // [B,Hq,n_splits,Dv+2]: m, l, O[Dv]
   int B, Hq, Hkv, D, Dv, G;
   int HG, Rp, groups;     // heads per CTA, stacked rows, head groups per KV head
@@ -61,7 +66,8 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // kMaxHG: head slots one softmax thread looks after (8 or 16); kNH: heads its code is unrolled for (<= kMaxHG);
 // kMaxDVT: 128-wide tiles of Dv; kWG: groups of four softmax warps, each owning kMaxHG of the CTA's kMaxHG*kWG
 // head slots (two groups let one CTA serve 32 heads of a KV head with one pass over its KV tiles).
-template <int kMaxHG, int kNH, int kMaxDVT, int kWG>
+// kPaged: the cache is paged (block table); a template parameter so that the contiguous kernels carry none of it.
+template <int kMaxHG, int kNH, int kMaxDVT, int kWG, bool kPaged>
 __global__ void __launch_bounds__(64 + 128 * kWG, (kNH <= 8 && kMaxDVT == 1 && kWG == 1) ? 3 : 1)
 attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
   extern __shared__ uint8_t smem_dyn[];
@@ -71,6 +77,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   constexpr int kSlots = kMaxHG * kWG;             // head slots of the stacked operands: rows [0,kSlots) first
   constexpr int kNSW = 4 * kWG;                    // component, rows [kSlots, 2*kSlots) second component
   __shared__ float s_aq[kSlots], s_bq[kSlots];
+  // Running maxima per head slot before / after each tile, three generations (tile t reads [t % 3] and writes
+  // [(t + 1) % 3]; the merge of tile t, which runs after the softmax of tile t + 1, still finds both).  The values are
+  // the same for all 128 threads of a warp group - every thread writes them and reads back what it wrote - so they
+  // need no registers between tiles: with 32 running outputs per thread the MLA kernel has none to spare.
+  __shared__ float s_m[3][kSlots];
   __shared__ float red[2][kWG][4][kNH + 1];        // per-warp tile maxima, double buffered by tile parity
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -79,8 +90,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   const int grp = unit % p.groups; unit /= p.groups;
   const int hk = unit % p.Hkv;
   const int b = unit / p.Hkv;
-  const int seq0 = p.cu[b];
-  const int L = p.cu[b + 1] - seq0;
+  const int32_t* bt = kPaged ? p.block_table + static_cast<long long>(b) * p.max_blocks : nullptr;
+  const int seq0 = kPaged ? 0 : p.cu[b];
+  const int L = kPaged ? p.seqlens[b] : p.cu[b + 1] - seq0;
   const int t_begin = split * p.chunk;                       // every split covers the same number of tokens
   const int t_end = min(L, t_begin + p.chunk);
   const int h0 = hk * p.G + grp * p.HG;                      // first query head of this CTA
@@ -146,19 +158,41 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         bool progressed = false;
         if (kq < ntiles && mbar_test_wait(&kv_empty[kq % p.stages], ((kq / p.stages) & 1) ^ 1)) {
           const int st = kq % p.stages;
-          mbar_arrive_expect_tx(&kv_full[st], k_bytes);
           uint8_t* dst = smem + st * kv_stage_bytes;
-          const int tok = seq0 + t_begin + kq * kTok;
-          for (int c = 0; c < p.DC; ++c) tma_load_3d(dst + c * kChunkBytes, &tmap_k, c * kChunk, hk, tok, &kv_full[st]);
+          const int u0 = t_begin + kq * kTok;
+          if constexpr (!kPaged) {
+            mbar_arrive_expect_tx(&kv_full[st], k_bytes);
+            for (int c = 0; c < p.DC; ++c) tma_load_3d(dst + c * kChunkBytes, &tmap_k, c * kChunk, hk, seq0 + u0, &kv_full[st]);
+          } else {
+            // one box per page that holds tokens of this split; rows of the tile past them keep stale (finite) codes
+            // and are masked like every token past the end
+            const int npg = min(kTok >> p.page_shift, (t_end - u0 + p.page - 1) >> p.page_shift);
+            mbar_arrive_expect_tx(&kv_full[st], p.DC * kChunk * p.page * npg);
+            for (int pg = 0; pg < npg; ++pg) {
+              const int tok = __ldg(bt + (u0 >> p.page_shift) + pg) * p.page;
+              for (int c = 0; c < p.DC; ++c)
+                tma_load_3d(dst + c * kChunkBytes + pg * p.page * kChunk, &tmap_k, c * kChunk, hk, tok, &kv_full[st]);
+            }
+          }
           ++kq;
           progressed = true;
         }
         if (vq < ntiles && mbar_test_wait(&v_empty[vq % p.stages], ((vq / p.stages) & 1) ^ 1)) {
           const int st = vq % p.stages;
-          mbar_arrive_expect_tx(&v_full[st], v_bytes);
           uint8_t* dst = smem + st * kv_stage_bytes + k_bytes;
-          const int tok = seq0 + t_begin + vq * kTok;
-          for (int j = 0; j < p.DVT; ++j) tma_load_3d(dst + j * kChunkBytes, &tmap_v, j * kChunk, hk, tok, &v_full[st]);
+          const int u0 = t_begin + vq * kTok;
+          if constexpr (!kPaged) {
+            mbar_arrive_expect_tx(&v_full[st], v_bytes);
+            for (int j = 0; j < p.DVT; ++j) tma_load_3d(dst + j * kChunkBytes, &tmap_v, j * kChunk, hk, seq0 + u0, &v_full[st]);
+          } else {
+            const int npg = min(kTok >> p.page_shift, (t_end - u0 + p.page - 1) >> p.page_shift);
+            mbar_arrive_expect_tx(&v_full[st], p.DVT * kChunk * p.page * npg);
+            for (int pg = 0; pg < npg; ++pg) {
+              const int tok = __ldg(bt + (u0 >> p.page_shift) + pg) * p.page;
+              for (int j = 0; j < p.DVT; ++j)
+                tma_load_3d(dst + j * kChunkBytes + pg * p.page * kChunk, &tmap_v, j * kChunk, hk, tok, &v_full[st]);
+            }
+          }
           ++vq;
           progressed = true;
         }
@@ -318,12 +352,23 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const int bar_id = 1 + hh;                      // each group of four warps synchronises on its own
 
     // running state per head; scores are kept in the log2 domain (log2(e) is folded into the key scale)
-    float m_run[kNH], l_part[kNH], aq[kNH], bq[kNH];
+    // Wide head groups (MLA) keep the warp-group-uniform state in shared memory (s_m, s_aq, s_bq above); the others
+    // have registers to spare and keep it there, off the critical path of their much shorter tiles.
+    constexpr bool kSmemState = kWG >= 2;
+    constexpr int kRegState = kSmemState ? 1 : kNH;
+    float l_part[kNH];
+    float m_run[kRegState], aq[kRegState], bq[kRegState], resc_keep[kRegState], resc_next[kRegState];
     float o_run[kMaxDVT][kNH];
 #pragma unroll
     for (int h = 0; h < kNH; ++h) {
-      m_run[h] = -INFINITY; l_part[h] = 0.0f;
-      aq[h] = (hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f; bq[h] = (hs0 + h < nh) ? s_bq[hs0 + h] : 0.0f;
+      l_part[h] = 0.0f;
+      if constexpr (kSmemState) {
+        s_m[0][hs0 + h] = -INFINITY;
+      } else {
+        m_run[h] = -INFINITY;
+        aq[h] = (hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f;
+        bq[h] = (hs0 + h < nh) ? s_bq[hs0 + h] : 0.0f;
+      }
 #pragma unroll
       for (int j = 0; j < kMaxDVT; ++j) o_run[j][h] = 0.0f;
     }
@@ -332,14 +377,19 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     bool ok = true;
     // State a tile's softmax hands to its merge: rescale factors and the P scales.  The softmax of tile t+1 runs
     // BEFORE the merge of tile t (it overlaps the PV product of tile t), so two sets are alive at a time.
-    float resc_cur[kNH], resc_nxt[kNH];
     float ap_cur = 0.0f, bp_cur = 0.0f, ap_nxt = 0.0f, bp_nxt = 0.0f;
 
     // c3-c5 for tile t: scores -> running max -> P -> two INT8 components into P buffer (t & 1)
-    auto softmax_tile = [&](int t, float (&resc)[kNH], float& alpha_p, float& beta_p) -> bool {
+    auto softmax_tile = [&](int t, float (&resc_out)[kRegState], float& alpha_p, float& beta_p) -> bool {
       const int tok_rel = t_begin + t * kTok + tl;
       const bool valid = tok_rel < t_end;
-      const long long sidx = static_cast<long long>(seq0 + tok_rel) * p.Hkv + hk;
+      long long sidx;
+      if constexpr (kPaged) {
+        const long long prow = valid ? static_cast<long long>(__ldg(bt + (tok_rel >> p.page_shift))) * p.page + (tok_rel & (p.page - 1)) : 0;
+        sidx = prow * p.Hkv + hk;
+      } else {
+        sidx = static_cast<long long>(seq0 + tok_rel) * p.Hkv + hk;
+      }
       const float ks = valid ? __ldg(p.k_scale + sidx) * scale2 : 0.0f;
       const float vs = valid ? __ldg(p.v_scale + sidx) : 0.0f;
       if (!wait_bounded(&s_full[t & 1], (t >> 1) & 1, abort, p.status)) return false;
@@ -354,7 +404,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         tmem_ld_wait();
 #pragma unroll
         for (int h = 0; h < kNH; ++h)
-          s[h] = valid ? __fmaf_rn(aq[h], static_cast<float>(static_cast<int32_t>(v1[h])), bq[h] * static_cast<float>(static_cast<int32_t>(v2[h]))) * ks : -INFINITY;
+        {
+          const float a_q = kSmemState ? ((hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f) : aq[kSmemState ? 0 : h];
+          const float b_q = kSmemState ? ((hs0 + h < nh) ? s_bq[hs0 + h] : 0.0f) : bq[kSmemState ? 0 : h];
+          s[h] = valid ? __fmaf_rn(a_q, static_cast<float>(static_cast<int32_t>(v1[h])), b_q * static_cast<float>(static_cast<int32_t>(v2[h]))) * ks : -INFINITY;
+        }
       }
       // c4: tile maxima per head (and of the value scales) over the 128 token lanes
       float (*rb)[kNH + 1] = red[t & 1][hh];
@@ -368,12 +422,21 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         if (lane == 0) rb[wq][kNH] = wv;
       }
       named_bar_sync(bar_id, 128);  // one barrier per tile: the other parity buffer is rewritten only after the next one
+      const float* m_rd = s_m[t % 3];
+      float* m_wr = s_m[(t + 1) % 3];
+      // running maximum of every head before and after the tile; rescale factor of what was accumulated so far.
+      // Register state: all heads first (as many independent exponentials in flight as there are heads); shared-memory
+      // state: inside the P loop below, head by head, so that nothing but the scores is alive across it.
+      float mn_t[kRegState], resc_t[kRegState];
+      if constexpr (!kSmemState) {
 #pragma unroll
-      for (int h = 0; h < kNH; ++h) {
-        const float mt = fmaxf(fmaxf(rb[0][h], rb[1][h]), fmaxf(rb[2][h], rb[3][h]));
-        const float mn = fmaxf(m_run[h], mt);
-        resc[h] = (m_run[h] == -INFINITY) ? 0.0f : ex2_approx(m_run[h] - mn);
-        m_run[h] = mn;
+        for (int h = 0; h < kNH; ++h) {
+          const float mt = fmaxf(fmaxf(rb[0][h], rb[1][h]), fmaxf(rb[2][h], rb[3][h]));
+          mn_t[h] = fmaxf(m_run[h], mt);
+          resc_t[h] = (m_run[h] == -INFINITY) ? 0.0f : ex2_approx(m_run[h] - mn_t[h]);
+          m_run[h] = mn_t[h];
+          resc_out[h] = resc_t[h];
+        }
       }
       const float vs_max = fmaxf(fmaxf(rb[0][kNH], rb[1][kNH]), fmaxf(rb[2][kNH], rb[3][kNH]));
       // c5: P = exp(S - m), fold the value scale, two-pass INT8 with the fixed scale alpha_P = max(v_scale)/127
@@ -384,8 +447,19 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
         // branch-free: an absent head or a token past the end contributes P = 0 (s is -inf there)
-        const float pr = (hs0 + h < nh) ? ex2_approx(s[h] - m_run[h]) : 0.0f;
-        l_part[h] = __fmaf_rn(l_part[h], resc[h], pr);
+        float mn, resc;
+        if constexpr (kSmemState) {
+          const float mt = fmaxf(fmaxf(rb[0][h], rb[1][h]), fmaxf(rb[2][h], rb[3][h]));
+          const float m_old = m_rd[hs0 + h];
+          mn = fmaxf(m_old, mt);
+          resc = (m_old == -INFINITY) ? 0.0f : ex2_approx(m_old - mn);
+          m_wr[hs0 + h] = mn;
+        } else {
+          mn = mn_t[kSmemState ? 0 : h];
+          resc = resc_t[kSmemState ? 0 : h];
+        }
+        const float pr = (hs0 + h < nh) ? ex2_approx(s[h] - mn) : 0.0f;
+        l_part[h] = __fmaf_rn(l_part[h], resc, pr);
         const float pt = pr * vs;
         const int c1 = min(127, __float2int_rn(pt * inv_a));
         const float r = __fmaf_rn(-alpha_p, static_cast<float>(c1), pt);
@@ -401,10 +475,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       return true;
     };
 
-    ok = softmax_tile(0, resc_cur, ap_cur, bp_cur);
+    ok = softmax_tile(0, resc_keep, ap_cur, bp_cur);
     for (int t = 0; t < ntiles && ok; ++t) {
       if (t + 1 < ntiles) {
-        ok = softmax_tile(t + 1, resc_nxt, ap_nxt, bp_nxt);     // overlaps the PV product of tile t
+        ok = softmax_tile(t + 1, resc_next, ap_nxt, bp_nxt);     // overlaps the PV product of tile t
         if (!ok) break;
       }
       // c6/c7: wait for O^T of tile t, merge it into the running output with that tile's rescale factors
@@ -412,6 +486,16 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       if (!ok) break;
       if (threadIdx.x == 64 && t < 6) attn_mark(p, 6 + 4 * t);
       tc_fence_after();
+      float resc_cur[kNH];                 // e^(m before tile t - m after tile t), recomputed from the stored maxima
+#pragma unroll
+      for (int h = 0; h < kNH; ++h) {
+        if constexpr (kSmemState) {
+          const float m_b = s_m[t % 3][hs0 + h], m_a = s_m[(t + 1) % 3][hs0 + h];
+          resc_cur[h] = (m_b == -INFINITY) ? 0.0f : ex2_approx(m_b - m_a);
+        } else {
+          resc_cur[h] = resc_keep[h];
+        }
+      }
 #pragma unroll
       for (int j = 0; j < kMaxDVT; ++j) {
         if (j < p.DVT) {
@@ -429,8 +513,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       __syncwarp();
       if (lane == 0) mbar_arrive(&o_empty);
       if (threadIdx.x == 64 && t < 6) attn_mark(p, 7 + 4 * t);
+      if constexpr (!kSmemState) {
 #pragma unroll
-      for (int h = 0; h < kNH; ++h) resc_cur[h] = resc_nxt[h];
+        for (int h = 0; h < kNH; ++h) resc_keep[h] = resc_next[h];
+      }
       ap_cur = ap_nxt;
       bp_cur = bp_nxt;
     }
@@ -452,7 +538,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         if (hs0 + h < nh) {
           float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + hs0 + h) * p.n_splits + split) * (p.Dv + 2);
           // the running maximum goes out in natural-log units (it was kept in the log2 domain)
-          if (tl == 0) { dst[0] = m_run[h] * 0.6931471805599453f; dst[1] = rb[0][h] + rb[1][h] + rb[2][h] + rb[3][h]; }
+          if (tl == 0) { dst[0] = (kSmemState ? s_m[ntiles % 3][hs0 + h] : m_run[kSmemState ? 0 : h]) * 0.6931471805599453f; dst[1] = rb[0][h] + rb[1][h] + rb[2][h] + rb[3][h]; }
 #pragma unroll
           for (int j = 0; j < kMaxDVT; ++j)
             if (j < p.DVT && j * kChunk + tl < p.Dv) dst[2 + j * kChunk + tl] = o_run[j][h];
@@ -570,17 +656,25 @@ msd_status_t msd_attn_decode_schedule(int32_t B, int32_t Hq, int32_t Hkv, int32_
   return MSD_OK;
 }
 
-msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, const int8_t* v_cache,
-                                    const float* k_scale, const float* v_scale, const int32_t* cu_seqlens,
-                                    int64_t total_tokens, int32_t max_seqlen, int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
-                                    float softmax_scale, void* out_bf16, float* lse, void* workspace,
-                                    size_t workspace_bytes, void* stream) {
-  using namespace msd;
+}  // extern "C"
+
+namespace msd {
+
+// Shared by the contiguous and the paged entry points.  Paged: block_table / seqlens non-null, `page` tokens per block
+// (a power of two from 8 to 128, so that pages tile the 128-token MMA tile), total_tokens = num_blocks * page.
+static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const int8_t* v_cache,
+                                const float* k_scale, const float* v_scale, const int32_t* cu_seqlens,
+                                const int32_t* block_table, const int32_t* seqlens, int32_t page, int32_t max_blocks,
+                                int64_t total_tokens, int32_t max_seqlen, int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
+                                float softmax_scale, void* out_bf16, float* lse, void* workspace,
+                                size_t workspace_bytes, void* stream) {
   if (B < 0 || max_seqlen < 0 || total_tokens < 0 || total_tokens > 0x7FFFFFFF) return MSD_ERR_BAD_SHAPE;
   if (B == 0) return MSD_OK;
   AttnPlan pl;
   if (!plan_attn(B, Hq, Hkv, D, Dv, max_seqlen > 0 ? max_seqlen : 1, v_cache == nullptr, &pl)) return MSD_ERR_BAD_SHAPE;
-  if (!q_bf16 || !k_cache || !k_scale || !cu_seqlens || !out_bf16 || !workspace) return MSD_ERR_NULL_POINTER;
+  const bool paged = block_table != nullptr;
+  if (!q_bf16 || !k_cache || !k_scale || (!paged && !cu_seqlens) || (paged && !seqlens) || !out_bf16 || !workspace)
+    return MSD_ERR_NULL_POINTER;
   if (!aligned(q_bf16, 16) || !aligned(k_cache, 16) || (v_cache && !aligned(v_cache, 16)) || !aligned(out_bf16, 16) ||
       !aligned(workspace, 1024))
     return MSD_ERR_BAD_ALIGNMENT;
@@ -591,14 +685,15 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
 
   // The tensor maps end at total_tokens: a tile that runs past the cache is zero-filled instead of read.
   const uint64_t T_extent = static_cast<uint64_t>(total_tokens > 0 ? total_tokens : 1);
+  const uint32_t box_rows = paged ? static_cast<uint32_t>(page) : static_cast<uint32_t>(kTok);     // one box per page
   CUtensorMap tmap_k, tmap_v;
   if (!encode_tmap_3d(&tmap_k, CU_TENSOR_MAP_DATA_TYPE_UINT8, k_cache, D, Hkv, T_extent, D, static_cast<uint64_t>(Hkv) * D,
-                      kChunk, 1, kTok, CU_TENSOR_MAP_SWIZZLE_128B))
+                      kChunk, 1, box_rows, CU_TENSOR_MAP_SWIZZLE_128B))
     return MSD_ERR_CUDA;
   const void* vbase = v_cache ? static_cast<const void*>(v_cache) : static_cast<const void*>(k_cache);
   const int vD = v_cache ? Dv : D;
   if (!encode_tmap_3d(&tmap_v, CU_TENSOR_MAP_DATA_TYPE_UINT8, vbase, vD, Hkv, T_extent, vD, static_cast<uint64_t>(Hkv) * vD,
-                      kChunk, 1, kTok, CU_TENSOR_MAP_SWIZZLE_128B))
+                      kChunk, 1, box_rows, CU_TENSOR_MAP_SWIZZLE_128B))
     return MSD_ERR_CUDA;
 
   AttnParams p;
@@ -606,6 +701,12 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
   p.k_scale = k_scale;
   p.v_scale = v_scale ? v_scale : k_scale;
   p.cu = cu_seqlens;
+  p.block_table = block_table;
+  p.seqlens = seqlens;
+  p.page = paged ? page : kTok;
+  p.page_shift = 0;
+  while ((1 << p.page_shift) < p.page) ++p.page_shift;
+  p.max_blocks = max_blocks;
   p.partial = static_cast<float*>(workspace);
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.Dv = Dv; p.G = Hq / Hkv;
   p.HG = pl.HG; p.Rp = pl.Rp; p.groups = pl.groups; p.DC = pl.DC; p.DVT = pl.DVT;
@@ -617,9 +718,11 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
 
   void (*kernel)(CUtensorMap, CUtensorMap, AttnParams) = nullptr;
   const int G = Hq / Hkv;
+#define MSD_ATTN_PICK_P(HG_, NH_, WG_, P_) \
+  kernel = (pl.DVT == 1) ? attn_decode_kernel<HG_, NH_, 1, WG_, P_> : (pl.DVT == 2) ? attn_decode_kernel<HG_, NH_, 2, WG_, P_> \
+                                                                                      : attn_decode_kernel<HG_, NH_, 4, WG_, P_>
 #define MSD_ATTN_PICK(HG_, NH_, WG_) \
-  kernel = (pl.DVT == 1) ? attn_decode_kernel<HG_, NH_, 1, WG_> : (pl.DVT == 2) ? attn_decode_kernel<HG_, NH_, 2, WG_> \
-                                                                                  : attn_decode_kernel<HG_, NH_, 4, WG_>
+  do { if (paged) { MSD_ATTN_PICK_P(HG_, NH_, WG_, true); } else { MSD_ATTN_PICK_P(HG_, NH_, WG_, false); } } while (0)
   int block_threads = kAttnThreads;
   if (pl.HG == 8) {
     if (G <= 4) { MSD_ATTN_PICK(8, 4, 1); } else { MSD_ATTN_PICK(8, 8, 1); }
@@ -633,12 +736,13 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
     block_threads = 64 + 128 * 4;
   }
 #undef MSD_ATTN_PICK
+#undef MSD_ATTN_PICK_P
   {
     // raise the dynamic shared-memory limit once per kernel instantiation
-    static void* done[16] = {};
+    static void* done[32] = {};
     bool seen = false;
     int free_slot = -1;
-    for (int i = 0; i < 16; ++i) {
+    for (int i = 0; i < 32; ++i) {
       if (done[i] == reinterpret_cast<void*>(kernel)) seen = true;
       if (!done[i] && free_slot < 0) free_slot = i;
     }
@@ -653,6 +757,34 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
   if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
   attn_combine_kernel<<<B * Hq, 128, 0, s>>>(p.partial, pl.n_splits, Dv, static_cast<__nv_bfloat16*>(out_bf16), lse);
   return launch_status();
+}
+
+}  // namespace msd
+
+extern "C" {
+
+msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, const int8_t* v_cache,
+                                    const float* k_scale, const float* v_scale, const int32_t* cu_seqlens,
+                                    int64_t total_tokens, int32_t max_seqlen, int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
+                                    float softmax_scale, void* out_bf16, float* lse, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
+  return msd::attn_launch(q_bf16, k_cache, v_cache, k_scale, v_scale, cu_seqlens, nullptr, nullptr, 0, 0, total_tokens, max_seqlen,
+                          B, Hq, Hkv, D, Dv, softmax_scale, out_bf16, lse, workspace, workspace_bytes, stream);
+}
+
+msd_status_t msd_attn_decode_int8kv_paged(const void* q_bf16, const int8_t* k_cache, const int8_t* v_cache,
+                                          const float* k_scale, const float* v_scale, const int32_t* block_table,
+                                          const int32_t* seqlens, int64_t num_blocks, int32_t page_size,
+                                          int32_t max_blocks_per_seq, int32_t max_seqlen, int32_t B, int32_t Hq, int32_t Hkv,
+                                          int32_t D, int32_t Dv, float softmax_scale, void* out_bf16, float* lse,
+                                          void* workspace, size_t workspace_bytes, void* stream) {
+  if (page_size < 8 || page_size > msd::kTok || (page_size & (page_size - 1)) != 0) return MSD_ERR_UNSUPPORTED;
+  if (num_blocks < 0 || max_blocks_per_seq < 0 || num_blocks * page_size > 0x7FFFFFFF) return MSD_ERR_BAD_SHAPE;
+  if (static_cast<int64_t>(max_blocks_per_seq) * page_size < max_seqlen) return MSD_ERR_BAD_SHAPE;
+  if (B > 0 && (!block_table || !seqlens)) return MSD_ERR_NULL_POINTER;
+  return msd::attn_launch(q_bf16, k_cache, v_cache, k_scale, v_scale, nullptr, block_table, seqlens, page_size, max_blocks_per_seq,
+                          num_blocks * page_size, max_seqlen, B, Hq, Hkv, D, Dv, softmax_scale, out_bf16, lse, workspace,
+                          workspace_bytes, stream);
 }
 
 }  // extern "C"

@@ -177,3 +177,41 @@ def mla_case(B, Hq, D, Dv, seqlens, seed=0):
     q = f32_to_bf16_bits(_normal_f32(_rng(seed, 4), (B, Hq, D)))
     k, ks = quantize_rows_int8(f32_to_bf16_bits(_normal_f32(_rng(seed, 5), (T, 1, D))))
     return AttnCase(q, k, None, ks, None, cu, Dv, float(1.0 / np.sqrt(D)))
+
+
+def paginate(case, page_size, seed=0, spare_blocks=3):
+    """Scatters a contiguous attention case into a paged cache: blocks of ``page_size`` tokens handed out in a seeded
+    random order (as a serving allocator would after some churn), plus unused blocks filled with noise codes.
+
+    Returns (k, v, k_scale, v_scale, block_table [B, max_blocks] int32, seqlens [B] int32); entries of the block table
+    past a sequence's last block are -1 and must never be read."""
+    seqlens = np.diff(case.cu_seqlens).astype(np.int32)
+    B = len(seqlens)
+    nblk_seq = (seqlens + page_size - 1) // page_size
+    max_blocks = int(max(1, nblk_seq.max()))
+    total = int(nblk_seq.sum()) + spare_blocks
+    rng = _rng(seed, 11)
+    order = rng.permutation(total)
+    table = np.full((B, max_blocks), -1, np.int32)
+    T, Hkv, D = case.k.shape
+    k = rng.integers(-127, 128, size=(total * page_size, Hkv, D), dtype=np.int8)
+    ks = (rng.random((total * page_size, Hkv), dtype=np.float32) + 0.5).astype(np.float32)
+    v = vs = None
+    if case.v is not None:
+        v = rng.integers(-127, 128, size=(total * page_size, Hkv, case.v.shape[2]), dtype=np.int8)
+        vs = (rng.random((total * page_size, Hkv), dtype=np.float32) + 0.5).astype(np.float32)
+    nxt = 0
+    for b in range(B):
+        t0 = int(case.cu_seqlens[b])
+        for j in range(int(nblk_seq[b])):
+            blk = int(order[nxt]); nxt += 1
+            table[b, j] = blk
+            n = min(page_size, int(seqlens[b]) - j * page_size)
+            src = slice(t0 + j * page_size, t0 + j * page_size + n)
+            dst = slice(blk * page_size, blk * page_size + n)
+            k[dst] = case.k[src]
+            ks[dst] = case.k_scale[src]
+            if v is not None:
+                v[dst] = case.v[src]
+                vs[dst] = case.v_scale[src]
+    return k, v, ks, vs, table, seqlens

@@ -167,3 +167,39 @@ def test_dequant_bf16_comparison_arm_is_less_accurate():
     assert np.all(np.abs(got - deq) <= 1e-2 * n)          # library summation order and P rounding differ from the oracle's
     msd = oracle.bf16_bits_to_f64(bf16_bits(_run_gpu(c)[0]))
     assert np.linalg.norm(msd - ref) <= np.linalg.norm(got - ref) * 1.05
+
+
+@pytest.mark.parametrize("page", [16, 64, 128])
+def test_paged_cache_gqa(page):
+    """The same sequences scattered over a paged cache (random block order, noise in the unused blocks and in the tails
+    of the last blocks) must give what the contiguous cache gives: the oracle's tiled mode on the contiguous case."""
+    seqlens = [1, 130, 700, 0, 257, 2049]
+    c = inputs.gqa_case(B=len(seqlens), Hq=16, Hkv=4, D=128, seqlens=seqlens, seed=61)
+    k, v, ks, vs, table, sl = inputs.paginate(c, page, seed=page)
+    o, lse = binding.attn_decode_int8kv_paged(bf16_dev(c.q), dev(k), dev(v), dev(ks), dev(vs), dev(table), dev(sl), page,
+                                              max(c.max_seqlen, 1), c.softmax_scale, want_lse=True)
+    torch.cuda.synchronize()
+    binding.last_device_status()
+    ref, lse_ref = _oracle_tiled(c)
+    got = oracle.bf16_bits_to_f64(bf16_bits(o))
+    live = np.isfinite(lse_ref)
+    _assert_close(got[live], ref[live])
+    assert np.allclose(lse.cpu().numpy()[live], lse_ref[live], rtol=0, atol=2e-3)
+    # and bit for bit what the contiguous entry point returns for the same data
+    o2, _ = _run_gpu(c)
+    assert torch.equal(o[torch.from_numpy(live).cuda()], o2[torch.from_numpy(live).cuda()])
+
+
+def test_paged_cache_mla_and_bad_page_size():
+    c = inputs.mla_case(B=3, Hq=64, D=576, Dv=512, seqlens=[300, 129, 1000], seed=62)
+    k, v, ks, vs, table, sl = inputs.paginate(c, 32, seed=5)
+    assert v is None
+    o = binding.attn_decode_int8kv_paged(bf16_dev(c.q), dev(k), None, dev(ks), None, dev(table), dev(sl), 32, c.max_seqlen,
+                                         c.softmax_scale, dv=c.dv)
+    torch.cuda.synchronize()
+    binding.last_device_status()
+    ref, _ = _oracle_tiled(c)
+    _assert_close(oracle.bf16_bits_to_f64(bf16_bits(o)), ref)
+    with pytest.raises(binding.MsdError):
+        binding.attn_decode_int8kv_paged(bf16_dev(c.q), dev(k), None, dev(ks), None, dev(table), dev(sl), 48, c.max_seqlen,
+                                         c.softmax_scale, dv=c.dv)
