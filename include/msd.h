@@ -186,6 +186,19 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
                                     size_t workspace_bytes, void* stream);
 
 /*
+ * The same attention with q_len query tokens per sequence (speculative / multi-token decode, Sec. 4.4: the stacked
+ * query operand then has 2 * q_len * G rows per KV head).  The q_len tokens are the LAST q_len tokens of each sequence's
+ * cache: query token s (0-based) attends to positions [0, L - q_len + s].  Every sequence must hold at least q_len
+ * tokens.  q_bf16 [B, q_len, Hq, D]; out_bf16 [B, q_len, Hq, Dv]; lse nullable [B, q_len, Hq]; 1 <= q_len <= 64.
+ * Workspace: msd_attn_decode_int8kv_workspace_bytes called with Hq * q_len in place of Hq; the schedule likewise.
+ */
+msd_status_t msd_attn_decode_int8kv_spec(const void* q_bf16, const int8_t* k_cache, const int8_t* v_cache,
+                                         const float* k_scale, const float* v_scale, const int32_t* cu_seqlens,
+                                         int64_t total_tokens, int32_t max_seqlen, int32_t B, int32_t q_len, int32_t Hq, int32_t Hkv,
+                                         int32_t D, int32_t Dv, float softmax_scale, void* out_bf16, float* lse, void* workspace,
+                                         size_t workspace_bytes, void* stream);
+
+/*
  * The same attention over a PAGED cache (serving layouts; the paper's kernels read a contiguous cache, Alg. 3):
  *   k_cache [num_blocks * page_size, Hkv, D], v_cache [num_blocks * page_size, Hkv, Dv] or NULL, scales
  *   [num_blocks * page_size, Hkv]; block_table [B, max_blocks_per_seq] INT32 (device): logical token u of sequence b

@@ -50,6 +50,7 @@ _SIGS = {
     "msd_attn_decode_int8kv": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp,
                                          _vp, _sz, _vp]),
     "msd_attn_decode_schedule": (C.c_int, [_i32] * 6 + [C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
+    "msd_attn_decode_int8kv_spec": (C.c_int, [_vp] * 6 + [_i64, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp, _vp, _sz, _vp]),
     "msd_attn_decode_int8kv_paged": (C.c_int, [_vp] * 7 + [_i64, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp, _vp,
                                                 _sz, _vp]),
     "msd_kv_dequant_bf16": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, _i32, _i32, C.c_void_p, C.c_void_p]),
@@ -232,6 +233,23 @@ def attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen):
     _check(lib().msd_attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen, C.byref(tile), C.byref(ns), C.byref(st)),
            "msd_attn_decode_schedule")
     return tile.value, ns.value, st.value
+
+
+def attn_decode_int8kv_spec(q, k, v, k_scale, v_scale, cu_seqlens, max_seqlen, softmax_scale, dv=None, ws=None, want_lse=False):
+    """q [B,Sq,Hq,D] bf16: the last Sq tokens of every sequence query its cache causally -> out [B,Sq,Hq,Dv]."""
+    _need_cuda(q, k, v, k_scale, v_scale, cu_seqlens)
+    B, Sq, Hq, D = q.shape
+    Hkv = k.shape[1]
+    Dv = v.shape[2] if v is not None else int(dv)
+    if ws is None:
+        ws = workspace(attn_decode_int8kv_workspace_bytes(B, Hq * Sq, Hkv, D, Dv, max_seqlen), q.device)
+    o = torch.empty((B, Sq, Hq, Dv), dtype=torch.bfloat16, device=q.device)
+    lse = torch.empty((B, Sq, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    wp, wb = _ws_ptr(ws)
+    code = lib().msd_attn_decode_int8kv_spec(_ptr(q), _ptr(k), _ptr(v), _ptr(k_scale), _ptr(v_scale), _ptr(cu_seqlens), int(k.shape[0]),
+                                             max_seqlen, B, Sq, Hq, Hkv, D, Dv, softmax_scale, _ptr(o), _ptr(lse), wp, wb, _stream())
+    _check(code, "msd_attn_decode_int8kv_spec")
+    return (o, lse) if want_lse else o
 
 
 def attn_decode_int8kv_paged(q, k, v, k_scale, v_scale, block_table, seqlens, page_size, max_seqlen, softmax_scale, dv=None,

@@ -39,7 +39,11 @@ struct AttnParams {
   const int32_t* seqlens; // [B] (paged only)
   int page, page_shift, max_blocks;
   float* partial;         // [B,Hq,n_splits,Dv+2]: m, l, O[Dv]
-  int B, Hq, Hkv, D, Dv, G;
+  int B, Hq, Hkv, D, Dv, G;   // with several query tokens per sequence Hq and G count (token, head) rows: Sq * real values
+  // Speculative / multi-token decode (Sec. 4.4): Sq query tokens per sequence, the last Sq tokens of its cache.  The
+  // Sq * Gr rows that share a KV head are laid out token-major: row r of a KV head = (token r / Gr, head r % Gr);
+  // query token s sees the cache up to position L - Sq + s.
+  int Sq, Gr;
   int HG, Rp, groups;     // heads per CTA, stacked rows, head groups per KV head
   int DC, DVT;            // 128-byte chunks of D / Dv
   int n_splits, stages, chunk;   // chunk: tokens per split (a multiple of the tile)
@@ -298,7 +302,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const int hs0 = hh * kMaxHG;                    // its first head slot
     // c1: decompose the query rows of this CTA's heads (one warp per head, round robin) into the stacked operand
     for (int h = wi; h < nh; h += kNSW) {
-      const uint4* qrow = reinterpret_cast<const uint4*>(p.q + (static_cast<long long>(b) * p.Hq + h0 + h) * p.D);
+      const int r_kv = grp * p.HG + h, sq = r_kv / p.Gr;       // row of this KV head -> (query token, head of the group)
+      const uint4* qrow = reinterpret_cast<const uint4*>(
+          p.q + ((static_cast<long long>(b) * p.Sq + sq) * (p.Hkv * p.Gr) + hk * p.Gr + (r_kv - sq * p.Gr)) * p.D);
       const int nvec = p.D >> 3;                    // 8 BF16 values per 16-byte load (D % 16 == 0, D <= 640)
       uint4 qv[3];                                  // the whole row stays in registers between the two passes
       float m = 0.0f;
@@ -407,7 +413,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         {
           const float a_q = kSmemState ? ((hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f) : aq[kSmemState ? 0 : h];
           const float b_q = kSmemState ? ((hs0 + h < nh) ? s_bq[hs0 + h] : 0.0f) : bq[kSmemState ? 0 : h];
-          s[h] = valid ? __fmaf_rn(a_q, static_cast<float>(static_cast<int32_t>(v1[h])), b_q * static_cast<float>(static_cast<int32_t>(v2[h]))) * ks : -INFINITY;
+          bool vh = valid;
+          if (p.Sq > 1) vh = valid && tok_rel < L - p.Sq + 1 + (grp * p.HG + hs0 + h) / p.Gr;    // causal among the new tokens
+          s[h] = vh ? __fmaf_rn(a_q, static_cast<float>(static_cast<int32_t>(v1[h])), b_q * static_cast<float>(static_cast<int32_t>(v2[h]))) * ks : -INFINITY;
         }
       }
       // c4: tile maxima per head (and of the value scales) over the 128 token lanes
@@ -458,7 +466,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           mn = mn_t[kSmemState ? 0 : h];
           resc = resc_t[kSmemState ? 0 : h];
         }
-        const float pr = (hs0 + h < nh) ? ex2_approx(s[h] - mn) : 0.0f;
+        // (a row that has seen no visible token yet keeps m = -inf: the clamp turns -inf - -inf into -inf, P = 0)
+        const float pr = (hs0 + h < nh) ? ex2_approx(s[h] - fmaxf(mn, -1e30f)) : 0.0f;
         l_part[h] = __fmaf_rn(l_part[h], resc, pr);
         const float pt = pr * vs;
         const int c1 = min(127, __float2int_rn(pt * inv_a));
@@ -562,9 +571,16 @@ static long long* g_attn_trace = nullptr;
 // (a separate small kernel: letting the last-arriving split do it inside the attention kernel measured slower)
 __global__ void __launch_bounds__(128)
 attn_combine_kernel(const float* __restrict__ partial, int n_splits, int Dv, __nv_bfloat16* __restrict__ out,
-                    float* __restrict__ lse) {
-  const long long row = blockIdx.x;
-  const float* base = partial + row * n_splits * (Dv + 2);
+                    float* __restrict__ lse, int Sq, int Gr, int Hkv) {
+  const float* base = partial + static_cast<long long>(blockIdx.x) * n_splits * (Dv + 2);
+  // partial rows are [B][KV head][query token][head of the group]; the output is [B][query token][head]
+  long long row = blockIdx.x;
+  if (Sq > 1) {
+    const int per_kv = Sq * Gr, per_seq = Hkv * per_kv;
+    const long long bq = row / per_seq;
+    const int v = static_cast<int>(row - bq * per_seq), hk = v / per_kv, r = v - hk * per_kv, sq = r / Gr;
+    row = (bq * Sq + sq) * (Hkv * Gr) + hk * Gr + (r - sq * Gr);
+  }
   float m = -INFINITY;
   for (int s = 0; s < n_splits; ++s) m = fmaxf(m, base[s * (Dv + 2)]);
   float l = 0.0f;
@@ -665,9 +681,11 @@ namespace msd {
 static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const int8_t* v_cache,
                                 const float* k_scale, const float* v_scale, const int32_t* cu_seqlens,
                                 const int32_t* block_table, const int32_t* seqlens, int32_t page, int32_t max_blocks,
-                                int64_t total_tokens, int32_t max_seqlen, int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
-                                float softmax_scale, void* out_bf16, float* lse, void* workspace,
+                                int64_t total_tokens, int32_t max_seqlen, int32_t B, int32_t q_len, int32_t Hq_real, int32_t Hkv,
+                                int32_t D, int32_t Dv, float softmax_scale, void* out_bf16, float* lse, void* workspace,
                                 size_t workspace_bytes, void* stream) {
+  if (q_len < 1 || q_len > 64 || Hq_real < 1 || Hkv < 1 || Hq_real % Hkv != 0) return MSD_ERR_BAD_SHAPE;
+  const int32_t Hq = Hq_real * q_len;          // (query token, head) rows per sequence
   if (B < 0 || max_seqlen < 0 || total_tokens < 0 || total_tokens > 0x7FFFFFFF) return MSD_ERR_BAD_SHAPE;
   if (B == 0) return MSD_OK;
   AttnPlan pl;
@@ -709,6 +727,7 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
   p.max_blocks = max_blocks;
   p.partial = static_cast<float*>(workspace);
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.Dv = Dv; p.G = Hq / Hkv;
+  p.Sq = q_len; p.Gr = Hq_real / Hkv;
   p.HG = pl.HG; p.Rp = pl.Rp; p.groups = pl.groups; p.DC = pl.DC; p.DVT = pl.DVT;
   p.chunk = pl.chunk;
   p.n_splits = pl.n_splits; p.stages = pl.stages; p.v_alias = pl.v_alias; p.tmem_cols = pl.tmem_cols;
@@ -755,7 +774,8 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
   dim3 grid(pl.n_splits, B * Hkv * pl.groups);
   kernel<<<grid, block_threads, pl.smem_bytes, s>>>(tmap_k, tmap_v, p);
   if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
-  attn_combine_kernel<<<B * Hq, 128, 0, s>>>(p.partial, pl.n_splits, Dv, static_cast<__nv_bfloat16*>(out_bf16), lse);
+  attn_combine_kernel<<<B * Hq, 128, 0, s>>>(p.partial, pl.n_splits, Dv, static_cast<__nv_bfloat16*>(out_bf16), lse, q_len,
+                                             Hq / (Hkv * q_len), Hkv);
   return launch_status();
 }
 
@@ -769,7 +789,16 @@ msd_status_t msd_attn_decode_int8kv(const void* q_bf16, const int8_t* k_cache, c
                                     float softmax_scale, void* out_bf16, float* lse, void* workspace,
                                     size_t workspace_bytes, void* stream) {
   return msd::attn_launch(q_bf16, k_cache, v_cache, k_scale, v_scale, cu_seqlens, nullptr, nullptr, 0, 0, total_tokens, max_seqlen,
-                          B, Hq, Hkv, D, Dv, softmax_scale, out_bf16, lse, workspace, workspace_bytes, stream);
+                          B, 1, Hq, Hkv, D, Dv, softmax_scale, out_bf16, lse, workspace, workspace_bytes, stream);
+}
+
+msd_status_t msd_attn_decode_int8kv_spec(const void* q_bf16, const int8_t* k_cache, const int8_t* v_cache,
+                                         const float* k_scale, const float* v_scale, const int32_t* cu_seqlens,
+                                         int64_t total_tokens, int32_t max_seqlen, int32_t B, int32_t q_len, int32_t Hq, int32_t Hkv,
+                                         int32_t D, int32_t Dv, float softmax_scale, void* out_bf16, float* lse, void* workspace,
+                                         size_t workspace_bytes, void* stream) {
+  return msd::attn_launch(q_bf16, k_cache, v_cache, k_scale, v_scale, cu_seqlens, nullptr, nullptr, 0, 0, total_tokens, max_seqlen,
+                          B, q_len, Hq, Hkv, D, Dv, softmax_scale, out_bf16, lse, workspace, workspace_bytes, stream);
 }
 
 msd_status_t msd_attn_decode_int8kv_paged(const void* q_bf16, const int8_t* k_cache, const int8_t* v_cache,
@@ -783,7 +812,7 @@ msd_status_t msd_attn_decode_int8kv_paged(const void* q_bf16, const int8_t* k_ca
   if (static_cast<int64_t>(max_blocks_per_seq) * page_size < max_seqlen) return MSD_ERR_BAD_SHAPE;
   if (B > 0 && (!block_table || !seqlens)) return MSD_ERR_NULL_POINTER;
   return msd::attn_launch(q_bf16, k_cache, v_cache, k_scale, v_scale, nullptr, block_table, seqlens, page_size, max_blocks_per_seq,
-                          num_blocks * page_size, max_seqlen, B, Hq, Hkv, D, Dv, softmax_scale, out_bf16, lse, workspace,
+                          num_blocks * page_size, max_seqlen, B, 1, Hq, Hkv, D, Dv, softmax_scale, out_bf16, lse, workspace,
                           workspace_bytes, stream);
 }
 

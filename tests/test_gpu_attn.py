@@ -203,3 +203,36 @@ def test_paged_cache_mla_and_bad_page_size():
     with pytest.raises(binding.MsdError):
         binding.attn_decode_int8kv_paged(bf16_dev(c.q), dev(k), None, dev(ks), None, dev(table), dev(sl), 48, c.max_seqlen,
                                          c.softmax_scale, dv=c.dv)
+
+
+def _truncate(c, drop):
+    """The same cache with the last `drop` tokens of every sequence removed (plain indexing)."""
+    L = np.diff(c.cu_seqlens)
+    keep = np.concatenate([np.arange(c.cu_seqlens[b], c.cu_seqlens[b] + L[b] - drop) for b in range(len(L))]).astype(np.int64)
+    cu = np.zeros(len(L) + 1, np.int32)
+    cu[1:] = np.cumsum(L - drop)
+    return keep, cu
+
+
+@pytest.mark.parametrize("Sq,Hq,Hkv", [(4, 8, 2), (2, 16, 2), (3, 8, 8)])
+def test_speculative_decode_rows_are_causal_single_query_problems(Sq, Hq, Hkv):
+    """Sq query tokens per sequence: query token s must equal the single-query problem on the cache without the last
+    Sq - 1 - s tokens (the oracle, tiled with the kernel's tile and split boundaries)."""
+    seqlens = [Sq, 131, 700, 2100]
+    base = inputs.gqa_case(B=len(seqlens), Hq=Hq * Sq, Hkv=Hkv, D=128, seqlens=seqlens, seed=71)
+    B = len(seqlens)
+    q = base.q.reshape(B, Sq, Hq, 128)                       # [B,Sq,Hq,D] as the entry point expects
+    out, lse = binding.attn_decode_int8kv_spec(bf16_dev(q), dev(base.k), dev(base.v), dev(base.k_scale), dev(base.v_scale),
+                                               dev(base.cu_seqlens), base.max_seqlen, base.softmax_scale, want_lse=True)
+    torch.cuda.synchronize()
+    binding.last_device_status()
+    got = oracle.bf16_bits_to_f64(bf16_bits(out))
+    tile, ns, st = binding.attn_decode_schedule(B, Hq * Sq, Hkv, 128, 128, base.max_seqlen)
+    for s in range(Sq):
+        keep, cu = _truncate(base, Sq - 1 - s)
+        ss = _split_starts(np.diff(cu), ns, st)
+        ref, lse_ref = oracle.attn_decode_int8kv(np.ascontiguousarray(q[:, s]), base.k[keep], base.v[keep], base.k_scale[keep],
+                                                 base.v_scale[keep], cu, base.softmax_scale, dv=128, mode="tiled", tile=tile,
+                                                 split_starts=ss, want_lse=True)
+        _assert_close(got[:, s], ref)
+        assert np.allclose(lse.cpu().numpy()[:, s], lse_ref, rtol=0, atol=2e-3)
