@@ -351,6 +351,33 @@ def other_configs(torch, binding, device, capture, timed):
         "frac_of_4x_measured_bf16": round(pf * 1e3 / (4 * peaks["bf16_tflops"]), 3), "frac_of_nominal_9pf": round(pf / 9.0, 3)}
     del x, w4, e4, y, wsp
 
+    # grouped W8A16 GEMM (MoE experts): 32 experts of [2048, 7168], 16 routed tokens each, against one call per expert
+    E, Ng, Kg, per = 32, 2048, 7168, 16
+    xg = torch.randn((E * per, Kg), generator=g, device=device).to(torch.bfloat16)
+    wg = [torch.randint(-127, 128, (E, Ng, Kg), generator=g, dtype=torch.int8, device=device) for _ in range(2)]
+    sg = torch.rand((E, Ng), generator=g, device=device) * 0.01
+    yg = torch.empty((E * per, Ng), dtype=torch.bfloat16, device=device)
+    wsg = binding.workspace(int(binding.lib().msd_grouped_gemm_w8a16_workspace_bytes(E * per, per, E, Ng, Kg)), device)
+    ws1 = binding.workspace(binding.gemm_w8a16_workspace_bytes(per, Ng, Kg), device)
+    itg = [0]
+
+    def f_grouped():
+        itg[0] += 1
+        binding.grouped_gemm_w8a16(xg, wg[itg[0] % 2], sg, [per] * E, ws=wsg, out=yg)
+
+    def f_loop():
+        itg[0] += 1
+        wcur = wg[itg[0] % 2]
+        for e in range(E):
+            binding.gemm_w8a16(xg[e * per:(e + 1) * per], wcur[e], sg[e], ws=ws1, out=yg[e * per:(e + 1) * per])
+    tg = per_call_us(f_grouped, reps=2)
+    tl = per_call_us(f_loop, reps=1)
+    res["moe_grouped_w8a16_E32_N2048_K7168_16_tokens_per_expert"] = {
+        "us": round(tg, 1), "weight_gbps": round(E * Ng * Kg / tg / 1e3, 1),
+        "frac_of_measured_hbm": round(E * Ng * Kg / tg / 1e3 / peaks["hbm_gbs"], 3),
+        "one_call_per_expert_us": round(tl, 1), "speedup": round(tl / tg, 2)}
+    del xg, wg, sg, yg, wsg
+
     # configs[3] GQA and configs[4] MLA decode attention
     from paper_2605_13915_b200 import inputs as gen
     for name, (B, Hq, Hkv, D, Dv, L, alias) in {

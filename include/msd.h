@@ -105,6 +105,23 @@ msd_status_t msd_gemm_w8a16_ex(const void* x_bf16, const int8_t* w, const float*
                                void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Grouped W8A16 MSD layer for mixture-of-experts blocks (Sec. 7.2: the decomposition works per activation row, so it
+ * carries over to grouped matrix multiplication unchanged).  The rows of x are sorted by expert; expert e owns the next
+ * group_sizes[e] rows and multiplies them against its own weight:
+ *   y[i,:] = msd_gemm_w8a16 row result of x[i,:] with w[e], w_scale[e]   for the rows i of group e.
+ *   x_bf16 [M_total, K] (device), w [E, N, K] INT8, w_scale [E, N] FP32, y [M_total, N] (device);
+ *   group_sizes_host [E] INT32 in HOST memory, each 0..128 (decode regime per expert), M_total = their sum.
+ * Empty groups are skipped (their weights are not read).  One decomposition launch over all rows, then one stream-K
+ * GEMM launch per 64 non-empty groups.  K % 16 == 0; N % 8 == 0 when y is BF16; E * N < 2^31.
+ * workspace: >= msd_grouped_gemm_w8a16_workspace_bytes(M_total, largest group, E, N, K), 1024-byte aligned, zeroed once
+ * (msd_workspace_init); the library leaves its counters zero after every call.
+ */
+size_t msd_grouped_gemm_w8a16_workspace_bytes(int64_t M_total, int32_t max_group_size, int32_t E, int64_t N, int64_t K);
+msd_status_t msd_grouped_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_scale, const int32_t* group_sizes_host,
+                                    int32_t E, int64_t N, int64_t K, void* y, msd_out_t ytype, void* workspace,
+                                    size_t workspace_bytes, void* stream);
+
+/*
  * The same W8A16 layer for callers that cannot allocate device memory.  (The paper has no counterpart; this is a
  * packaging variant of msd_gemm_w8a16, not a step of the method.)
  *

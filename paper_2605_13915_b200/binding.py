@@ -37,6 +37,8 @@ _SIGS = {
     "msd_gemm_w8a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_w8a16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _vp, _sz, _vp]),
     "msd_gemm_w8a16_ex": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, C.c_int, _vp, _sz, _vp]),
+    "msd_grouped_gemm_w8a16_workspace_bytes": (_sz, [_i64, _i32, _i32, _i64, _i64]),
+    "msd_grouped_gemm_w8a16": (C.c_int, [_vp, _vp, _vp, _vp, _i32, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_gemm_w8a16_noalloc": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp]),
     "msd_debug_set_trace": (None, [_vp]),
     "msd_debug_set_attn_trace": (None, [_vp]),
@@ -164,6 +166,24 @@ def gemm_w8a16(x, w, w_scale, out_dtype=torch.bfloat16, ws=None, want_acc=False,
         code = lib().msd_gemm_w8a16(_ptr(x), _ptr(w), _ptr(w_scale), M, N, K, _ptr(y), yt, _ptr(acc), wp, wb, _stream())
     _check(code, "msd_gemm_w8a16")
     return (y, acc) if want_acc else y
+
+
+def grouped_gemm_w8a16(x, w, w_scale, group_sizes, out_dtype=torch.bfloat16, ws=None, out=None):
+    """MoE experts: x [M_total,K] bf16 with rows sorted by expert, w [E,N,K] int8, w_scale [E,N] f32, group_sizes: E host ints
+    (rows per expert, each <= 128) -> y [M_total,N]."""
+    _need_cuda(x, w, w_scale)
+    E, N, K = w.shape
+    sizes = (C.c_int32 * E)(*[int(v) for v in group_sizes])
+    M_total = int(sum(int(v) for v in group_sizes))
+    assert x.shape[0] == M_total and x.shape[1] == K
+    if ws is None:
+        ws = workspace(int(lib().msd_grouped_gemm_w8a16_workspace_bytes(M_total, max(int(v) for v in group_sizes), E, N, K)), x.device)
+    y = out if out is not None else torch.empty((M_total, N), dtype=out_dtype, device=x.device)
+    wp, wb = _ws_ptr(ws)
+    code = lib().msd_grouped_gemm_w8a16(_ptr(x), _ptr(w), _ptr(w_scale), C.cast(sizes, C.c_void_p), E, N, K, _ptr(y),
+                                        OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream())
+    _check(code, "msd_grouped_gemm_w8a16")
+    return y
 
 
 def gemm_w8a16_noalloc(x, w, w_scale, out):

@@ -68,6 +68,20 @@ struct GemmW8Params {
   long long* trace;        // nullable diagnostic buffer: 16 clock samples per CTA
 };
 
+// Grouped GEMM (MoE experts, Sec. 7.2 "Extension to MoE"): the problems of one launch.  Group g multiplies the token rows
+// [off[g], off[g] + m[g]) of x against expert expert[g]'s weight [N, K]; all groups share N, K and the kernel's tile shapes.
+constexpr int kMaxGroups = 64;
+struct GemmW8Groups {
+  int n;                      // groups in this launch (0: not a grouped launch)
+  int tiles_per_group;        // ceil(N / 128)
+  int xq2_row0;               // row of the stacked-components buffer where the second components start
+  int expert[kMaxGroups], off[kMaxGroups], m[kMaxGroups];
+};
+
+struct GemmW8NoGroups {};      // what the ungrouped instantiations take in its place: no parameter bytes to copy per launch
+template <bool kGrouped> struct GroupArg { using type = GemmW8NoGroups; };
+template <> struct GroupArg<true> { using type = GemmW8Groups; };
+
 __device__ __forceinline__ void trace_mark(const GemmW8Params& p, int slot) {
   if (p.trace) p.trace[blockIdx.x * 16 + slot] = clock64();
 }
@@ -98,7 +112,8 @@ struct RecvInfo {
 template <bool kBase, bool kBf16, int W>
 __device__ __forceinline__ void epilogue_chunk(const GemmW8Params& p, uint32_t t_row, int32_t* acc_tile, int c0, int r, int n,
                                                bool row_ok, float sw, const float* s_alpha, const float* s_beta,
-                                               uint8_t* stage_buf, int et, int n0, int rows_valid, const RecvInfo& rv) {
+                                               uint8_t* stage_buf, int et, int n0, int rows_valid, const RecvInfo& rv,
+                                               int m_valid, long long y_row0) {
   using OutT = typename std::conditional<kBf16, __nv_bfloat16, float>::type;
   constexpr int kEsz = static_cast<int>(sizeof(OutT));
   uint32_t a[W], b[W];
@@ -184,7 +199,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmW8Params& p, uint32_t t
     }
   }
   named_bar_sync(1, 128);
-  const int wm = min(W, p.M - c0);                               // tokens of this chunk that exist
+  const int wm = min(W, m_valid - c0);                           // tokens of this chunk that exist
   int nv = min(rows_valid, p.N - n0);                            // weight rows of this tile / band that exist
   if (nv < 0) nv = 0;
   OutT* y = static_cast<OutT*>(p.y);
@@ -196,15 +211,15 @@ __device__ __forceinline__ void epilogue_chunk(const GemmW8Params& p, uint32_t t
 #pragma unroll 4
       for (int j = et / kSegs; j < wm; j += 128 / kSegs) {
         const uint4 val = *reinterpret_cast<const uint4*>(stage + j * kTileN + nf);
-        *reinterpret_cast<uint4*>(y + static_cast<long long>(c0 + j) * p.N + n0 + nf) = val;
+        *reinterpret_cast<uint4*>(y + (y_row0 + c0 + j) * p.N + n0 + nf) = val;
       }
     } else if (nf < nv) {
       for (int j = et / kSegs; j < wm; j += 128 / kSegs)
-        for (int e = nf; e < nv; ++e) y[static_cast<long long>(c0 + j) * p.N + n0 + e] = stage[j * kTileN + e];
+        for (int e = nf; e < nv; ++e) y[(y_row0 + c0 + j) * p.N + n0 + e] = stage[j * kTileN + e];
     }
   } else {
     if (et < nv)
-      for (int j = 0; j < wm; ++j) y[static_cast<long long>(c0 + j) * p.N + n0 + et] = stage[j * kTileN + et];
+      for (int j = 0; j < wm; ++j) y[(y_row0 + c0 + j) * p.N + n0 + et] = stage[j * kTileN + et];
   }
   named_bar_sync(1, 128);            // the buffer is free for the next chunk
 }
@@ -213,17 +228,18 @@ __device__ __forceinline__ void epilogue_chunk(const GemmW8Params& p, uint32_t t
 template <bool kBase, bool kFused, bool kBf16>
 __device__ __forceinline__ void epilogue_tile(const GemmW8Params& p, uint32_t t_row, int32_t* acc_tile, int r, int n, bool row_ok,
                                               float sw, const float* s_alpha, const float* s_beta, uint8_t* stage_buf, int et,
-                                              int n0, int rows_valid, int tok0, int tok1, const RecvInfo& rv) {
+                                              int n0, int rows_valid, int tok0, int tok1, const RecvInfo& rv, int m_valid,
+                                              long long y_row0) {
   int c0 = tok0;
   if constexpr (!kFused) {
     if constexpr (kBase)
       for (; c0 + 32 <= tok1; c0 += 32)
-        epilogue_chunk<kBase, kBf16, 32>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv);
+        epilogue_chunk<kBase, kBf16, 32>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv, m_valid, y_row0);
     for (; c0 + 16 <= tok1; c0 += 16)      // 16 tokens at a time: two sums and two scales per token stay in registers
-      epilogue_chunk<kBase, kBf16, 16>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv);
+      epilogue_chunk<kBase, kBf16, 16>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv, m_valid, y_row0);
   }
   for (; c0 + 8 <= tok1; c0 += 8)
-    epilogue_chunk<kBase, kBf16, 8>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv);
+    epilogue_chunk<kBase, kBf16, 8>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv, m_valid, y_row0);
 }
 
 // Adds W accumulator columns of a partial tile into the split-K meeting place (reductions without return value).
@@ -296,10 +312,14 @@ __device__ __forceinline__ void fused_row_scales(const GemmW8Params& p, int t256
 //                stacked operand tile of every stage straight into shared memory ("online activation decomposition",
 //                Sec. 3.9), so the activations never round-trip through HBM and nothing waits for a previous launch.
 constexpr int kFusedThreads = kGemmThreads + 128;
-template <bool kBase, bool kFused>
+// kGrouped: several (token rows, expert weight) problems in one stream-K launch; the group table travels as a kernel
+//                parameter, weight tiles are addressed in the stacked [E*N, K] weight, the two components of a
+//                group's rows come as two boxes of the component buffer.
+template <bool kBase, bool kFused, bool kGrouped = false>
 __global__ void __launch_bounds__(kFused ? kFusedThreads : kGemmThreads, 1)
 gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_w2,
-                  const __grid_constant__ CUtensorMap tmap_x, const GemmW8Params p) {
+                  const __grid_constant__ CUtensorMap tmap_x, const GemmW8Params p,
+                  const __grid_constant__ typename GroupArg<kGrouped>::type grp) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ __align__(8) uint64_t full_bar[kMaxStages];
   __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
@@ -391,7 +411,21 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   // the first weight boxes are requested the sooner the stream from HBM starts.
   uint64_t pol_w = 0, pol_x = 0;
   bool w_lane = false, x_lane = false;
-  int c = 0, tile = 0, kbi = 0, kbr = 0, kbr0 = 0, pre = 0, pre0 = 0;
+  int c = 0, x_half = 0, tile = 0, kbi = 0, kbr = 0, kbr0 = 0, pre = 0, pre0 = 0, tile_first = 0, kbi_first = 0;
+  // first weight row of a tile in the weight tensor, and first row of its stacked components in the component buffer
+  auto w_row = [&](int t) -> int {
+    if constexpr (kGrouped) {
+      const int g = t / grp.tiles_per_group;
+      return grp.expert[g] * p.N + (t - g * grp.tiles_per_group) * kTileN;
+    } else {
+      return band_row0 + t * kTileN;
+    }
+  };
+  auto x_row = [&](int t) -> int {
+    if constexpr (kGrouped) return grp.off[t / grp.tiles_per_group] + x_half * grp.xq2_row0;
+    else return 0;
+  };
+  const int x_half_bytes = kGrouped ? p.Mp * kBlockK : 0;
   auto advance = [&]() {
     if (++kbi == p.kblocks) { kbi = 0; ++tile; }
     if (++kbr == p.kblocks) kbr = 0;
@@ -404,13 +438,15 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     pol_w = policy_evict_first();    // weights are streamed once
     pol_x = policy_evict_last();      // the stacked components are re-read by every CTA
     w_lane = lane < p.kw;
-    x_lane = !kFused && lane >= p.kw && lane < 2 * p.kw;
-    c = w_lane ? lane : lane - p.kw;
+    x_lane = !kFused && lane >= p.kw && lane < (kGrouped ? 3 : 2) * p.kw;     // grouped: one box per component
+    c = w_lane ? lane : (lane - p.kw) % p.kw;
+    x_half = w_lane ? 0 : (lane - p.kw) / p.kw;
     // (tile, K block) of the next block to load, advanced by one per stage; kbr = rotated K block
     const int tile0 = blk_begin < (1LL << 32) ? static_cast<int>(static_cast<unsigned>(blk_begin) / static_cast<unsigned>(p.kblocks))
                                               : static_cast<int>(blk_begin / p.kblocks);
     const int kbi0 = static_cast<int>(blk_begin - static_cast<long long>(tile0) * p.kblocks);
     tile = tile0; kbi = kbi0;
+    tile_first = tile0; kbi_first = kbi0;
     kbr = kbi + kb_rot;
     if (kbr >= p.kblocks) kbr -= p.kblocks;
     kbr0 = kbr;
@@ -424,7 +460,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       __syncwarp();
       if (w_lane)
         tma_load_2d_hint(smem + i * stage_bytes + c * p.w_chunk_bytes, wmap, (kbr * p.kw + c) * kBlockK,
-                         band_row0 + tile * kTileN, &full_bar[i], pol_w);
+                         w_row(tile), &full_bar[i], pol_w);
       advance();
     }
     if (lane == 0) trace_mark(p, 3);
@@ -458,12 +494,12 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
           __syncwarp();
           if (w_lane)
             tma_load_2d_hint(smem + i * stage_bytes + c * p.w_chunk_bytes, wmap, (kbr * p.kw + c) * kBlockK,
-                             band_row0 + tile * kTileN, &full_bar[i], pol_w);
+                             w_row(tile), &full_bar[i], pol_w);
           advance();
         }
         if (x_lane)
-          tma_load_2d_hint(smem + i * stage_bytes + w_stage_bytes + c * x_chunk_bytes, &tmap_x, (kx * p.kw + c) * kBlockK, 0,
-                           &full_bar[i], pol_x);
+          tma_load_2d_hint(smem + i * stage_bytes + w_stage_bytes + c * x_chunk_bytes + x_half * x_half_bytes, &tmap_x,
+                           (kx * p.kw + c) * kBlockK, x_row(tile_first + (kbi_first + i) / p.kblocks), &full_bar[i], pol_x);
         if (++kx == p.kblocks) kx = 0;
       }
     }
@@ -479,10 +515,10 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       if (!ok) break;
       uint8_t* dst = smem + stage * stage_bytes;
       if (w_lane)
-        tma_load_2d_hint(dst + c * p.w_chunk_bytes, wmap, (kbr * p.kw + c) * kBlockK, band_row0 + tile * kTileN,
-                         &full_bar[stage], pol_w);
+        tma_load_2d_hint(dst + c * p.w_chunk_bytes, wmap, (kbr * p.kw + c) * kBlockK, w_row(tile), &full_bar[stage], pol_w);
       else if (x_lane)
-        tma_load_2d_hint(dst + w_stage_bytes + c * x_chunk_bytes, &tmap_x, (kbr * p.kw + c) * kBlockK, 0, &full_bar[stage], pol_x);
+        tma_load_2d_hint(dst + w_stage_bytes + c * x_chunk_bytes + x_half * x_half_bytes, &tmap_x, (kbr * p.kw + c) * kBlockK,
+                         x_row(tile), &full_bar[stage], pol_x);
       advance();
       if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
     }
@@ -657,7 +693,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         named_bar_sync(1, 128);
         if (*abort) return_early = true;
       }
-      if (et < p.M && !return_early) {
+      if (!kGrouped && et < p.M && !return_early) {
         s_alpha[et] = __ldcg(p.alpha + et);
         s_beta[et] = __ldcg(p.beta + et);
       }
@@ -679,9 +715,19 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       if (et == 0) { if (seg == 0) trace_mark(p, 8); trace_mark(p, 9); }
       tc_fence_after();
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * p.NB;
-      const int n = band_row0 + tile * kTileN + r;
+      // weight row within its matrix; grouped: also which rows of x / y and which expert's scales this tile is about
+      int n = band_row0 + tile * kTileN + r;
+      int m_valid = p.M;
+      long long y_row0 = 0, sw_row0 = 0;
+      if constexpr (kGrouped) {
+        const int g = tile / grp.tiles_per_group;
+        n = (tile - g * grp.tiles_per_group) * kTileN + r;
+        m_valid = grp.m[g];
+        y_row0 = grp.off[g];
+        sw_row0 = static_cast<long long>(grp.expert[g]) * p.N;
+      }
       const bool row_ok = (r < band_h) && (n < p.N);
-      const float sw = (!kBase && row_ok) ? __ldg(p.w_scale + n) : 0.0f;
+      const float sw = (!kBase && row_ok) ? __ldg(p.w_scale + sw_row0 + n) : 0.0f;
       bool finish = complete;
       int32_t* acc_tile = nullptr;
       int tok0 = 0, tok1 = p.Mp;
@@ -781,10 +827,21 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         if (finish) __threadfence();
       }
       if (finish) {
+        if constexpr (kGrouped) {
+          // the scales of this group's token rows (the previous tile's epilogue has finished reading the old ones)
+          named_bar_sync(1, 128);
+          if (et < m_valid) {
+            s_alpha[et] = __ldcg(p.alpha + y_row0 + et);
+            s_beta[et] = __ldcg(p.beta + y_row0 + et);
+          }
+          named_bar_sync(1, 128);
+        }
         if (p.ytype == MSD_OUT_BF16)
-          epilogue_tile<kBase, kFused, true>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h, tok0, tok1, rv);
+          epilogue_tile<kBase, kFused, true>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h, tok0, tok1, rv,
+                                             m_valid, y_row0);
         else
-          epilogue_tile<kBase, kFused, false>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h, tok0, tok1, rv);
+          epilogue_tile<kBase, kFused, false>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h, tok0, tok1, rv,
+                                              m_valid, y_row0);
       }
       tc_fence_before();
       __syncwarp();
@@ -939,7 +996,8 @@ static bool ensure_smem_attr() {
   if (!attr_done) {
     if (cudaFuncSetAttribute(gemm_w8a16_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
         cudaFuncSetAttribute(gemm_w8a16_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_w8a16_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
+        cudaFuncSetAttribute(gemm_w8a16_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w8a16_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
     {
       cudaGetLastError();
       return false;
@@ -1089,16 +1147,17 @@ msd_status_t msd_gemm_w8a16_ex(const void* x_bf16, const int8_t* w, const float*
   p.q = q;
   p.flags = p.counters + pl.num_tiles;
   if (!ensure_smem_attr()) return MSD_ERR_CUDA;
+  GemmW8NoGroups no_groups;
   if (fused) {
     // may become resident while earlier work in the stream still runs: it prefetches weights, then waits for that
     // work to finish before it reads x or touches the split-K workspace
-    if (launch_pdl(gemm_w8a16_kernel<false, true>, dim3(pl.grid), dim3(kFusedThreads), pl.smem_bytes, s, getenv("MSD_NO_PDL") == nullptr, tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
+    if (launch_pdl(gemm_w8a16_kernel<false, true>, dim3(pl.grid), dim3(kFusedThreads), pl.smem_bytes, s, getenv("MSD_NO_PDL") == nullptr, tmap_w, tmap_w2, tmap_x, p, no_groups) != cudaSuccess)
       return MSD_ERR_CUDA;
     return MSD_OK;
   }
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
   if (launch_pdl_cluster(gemm_w8a16_kernel<false, false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl,
-                         static_cast<unsigned>(pl.csplit), tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
+                         static_cast<unsigned>(pl.csplit), tmap_w, tmap_w2, tmap_x, p, no_groups) != cudaSuccess)
     return MSD_ERR_CUDA;
   return MSD_OK;
 }
@@ -1151,9 +1210,10 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   p.status = status;
   p.trace = nullptr;
   if (!ensure_smem_attr()) return MSD_ERR_CUDA;
+  GemmW8NoGroups no_groups;
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
   if (launch_pdl_cluster(gemm_w8a16_kernel<true, false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl,
-                         static_cast<unsigned>(pl.csplit), tmap_w, tmap_w2, tmap_x, p) != cudaSuccess)
+                         static_cast<unsigned>(pl.csplit), tmap_w, tmap_w2, tmap_x, p, no_groups) != cudaSuccess)
     return MSD_ERR_CUDA;
   return MSD_OK;
 }
@@ -1161,6 +1221,129 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
 // ---------------------------------------------------------------------------------------------------------------------
 // Entry point for callers that cannot allocate device memory (see msd.h).  The scratch the GEMM needs lives in this
 // file-scope device array, which every GPU that loads the library holds until the process exits.
+// ---------------------------------------------------------------------------------------------------------------------
+// Grouped W8A16 layer (MoE experts, Sec. 7.2): x rows sorted by expert, group g = rows [off_g, off_g + m_g) against
+// expert e_g's weight.  One decomposition launch over all rows, then stream-K launches of up to kMaxGroups non-empty
+// groups each; empty groups cost nothing (their weights are never read).
+struct GroupedPlan {
+  msd::GemmW8Plan base;       // tile shapes for the largest group
+  int64_t mt_pad;             // rows reserved per component in the stacked buffer
+  size_t off_q, off_alpha, off_beta, off_counters, off_slots, bytes;
+};
+
+static GroupedPlan plan_grouped(int64_t M_total, int max_group, int E, int64_t N, int64_t K) {
+  using namespace msd;
+  GroupedPlan g;
+  g.base = plan_w8(max_group < 1 ? 1 : max_group, N, K);
+  g.mt_pad = static_cast<int64_t>(round_up(static_cast<size_t>(M_total), 8)) + 128;     // a box may start at the last row
+  const int groups_per_launch = E < kMaxGroups ? E : kMaxGroups;
+  const size_t tiles = static_cast<size_t>(groups_per_launch) * g.base.num_tiles;
+  size_t off = 0;
+  g.off_q = off;        off = round_up(off + 2 * static_cast<size_t>(g.mt_pad) * K, 1024);
+  g.off_alpha = off;    off = round_up(off + static_cast<size_t>(M_total + 1) * sizeof(float), 256);
+  g.off_beta = off;     off = round_up(off + static_cast<size_t>(M_total + 1) * sizeof(float), 256);
+  g.off_counters = off; off = round_up(off + (tiles + 2) * sizeof(unsigned), 1024);
+  g.off_slots = off;    off = round_up(off + tiles * g.base.NB * kTileN * sizeof(int32_t), 1024);
+  g.bytes = off;
+  return g;
+}
+
+size_t msd_grouped_gemm_w8a16_workspace_bytes(int64_t M_total, int32_t max_group_size, int32_t E, int64_t N, int64_t K) {
+  if (M_total < 0 || max_group_size < 0 || max_group_size > 128 || E < 1 || N < 1 || K < 16) return 0;
+  return plan_grouped(M_total, max_group_size, E, N, K).bytes;
+}
+
+msd_status_t msd_grouped_gemm_w8a16(const void* x_bf16, const int8_t* w, const float* w_scale, const int32_t* group_sizes_host,
+                                    int32_t E, int64_t N, int64_t K, void* y, msd_out_t ytype, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
+  using namespace msd;
+  if (E < 1 || N < 1 || K < 16 || K % 16 != 0 || N > (1 << 24) || K > (1 << 24)) return MSD_ERR_BAD_SHAPE;
+  if (!group_sizes_host) return MSD_ERR_NULL_POINTER;
+  if (ytype != MSD_OUT_BF16 && ytype != MSD_OUT_FP32) return MSD_ERR_UNSUPPORTED;
+  if (ytype == MSD_OUT_BF16 && N % 8 != 0) return MSD_ERR_BAD_SHAPE;
+  if (static_cast<int64_t>(E) * N > 0x7FFFFFFF) return MSD_ERR_BAD_SHAPE;
+  int64_t M_total = 0;
+  int max_group = 0;
+  for (int e = 0; e < E; ++e) {
+    if (group_sizes_host[e] < 0 || group_sizes_host[e] > 128) return MSD_ERR_BAD_SHAPE;      // decode regime per expert
+    M_total += group_sizes_host[e];
+    if (group_sizes_host[e] > max_group) max_group = group_sizes_host[e];
+  }
+  if (M_total == 0) return MSD_OK;
+  if (!x_bf16 || !w || !w_scale || !y || !workspace) return MSD_ERR_NULL_POINTER;
+  if (!aligned(x_bf16, 16) || !aligned(w, 16) || !aligned(y, 16) || !aligned(workspace, 1024)) return MSD_ERR_BAD_ALIGNMENT;
+  const GroupedPlan gp = plan_grouped(M_total, max_group, E, N, K);
+  if (workspace_bytes < gp.bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
+  unsigned* status = device_status_ptr();
+  if (!status) return MSD_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  int8_t* q = reinterpret_cast<int8_t*>(ws + gp.off_q);
+  float* alpha = reinterpret_cast<float*>(ws + gp.off_alpha);
+  float* beta = reinterpret_cast<float*>(ws + gp.off_beta);
+  msd_status_t st = launch_decompose_int8(x_bf16, M_total, K, K, q, q + static_cast<size_t>(gp.mt_pad) * K, alpha, beta, 127.0f,
+                                          254.0f, s);
+  if (st != MSD_OK) return st;
+
+  const GemmW8Plan& pl = gp.base;
+  const int kw = pl.kw;
+  const int kblocks = pl.kblocks;
+  CUtensorMap tmap_w, tmap_x;
+  if (!encode_tmap_2d(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, static_cast<uint64_t>(E) * N, K, kBlockK, kTileN,
+                      CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, q, K, 2 * static_cast<uint64_t>(gp.mt_pad), K, kBlockK, pl.Mp,
+                      CU_TENSOR_MAP_SWIZZLE_128B))
+    return MSD_ERR_CUDA;
+  if (!ensure_smem_attr()) return MSD_ERR_CUDA;
+
+  GemmW8Params p;
+  p.M = pl.Mp; p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+  p.kb_rot_step = 0; p.pre_stages = 64;
+  p.mode = 0; p.groups8 = 1; p.gran = 8; p.hmax = kTileN; p.w_chunk_bytes = kWStageBytes; p.kw = kw; p.csplit = 1;
+  p.kblocks = kblocks; p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
+  // the planner laid the stages out for row bands when N is large; stream-K always stages full 128-row weight boxes
+  {
+    const int stage_bytes = kw * (kWStageBytes + pl.NB * kBlockK);
+    int stages = kSmemBudget / stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < 1) return MSD_ERR_UNSUPPORTED;
+    p.num_stages = stages;
+    p.epi_off = static_cast<int>(round_up(static_cast<size_t>(stages) * stage_bytes, 1024));
+  }
+  const size_t smem_bytes = static_cast<size_t>(p.epi_off) + kEpiBytes + 1024;
+  p.w_scale = w_scale; p.alpha = alpha; p.beta = beta; p.y = y; p.acc_dbg = nullptr;
+  p.accum = reinterpret_cast<int32_t*>(ws + gp.off_slots);
+  p.counters = reinterpret_cast<unsigned*>(ws + gp.off_counters);
+  p.status = status; p.trace = nullptr;
+  p.x = nullptr; p.ldx = 0; p.inline_dec = 0; p.dec_ctas = 0; p.c1 = 127.0f; p.c2 = 254.0f; p.q = q; p.flags = nullptr;
+
+  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+  int e = 0;
+  int64_t off = 0;
+  while (e < E) {
+    GemmW8Groups g;
+    g.n = 0; g.tiles_per_group = pl.num_tiles; g.xq2_row0 = static_cast<int>(gp.mt_pad);
+    while (e < E && g.n < kMaxGroups) {
+      const int m = group_sizes_host[e];
+      if (m > 0) {
+        g.expert[g.n] = e; g.off[g.n] = static_cast<int>(off); g.m[g.n] = m;
+        ++g.n;
+      }
+      off += m;
+      ++e;
+    }
+    if (g.n == 0) break;
+    p.num_tiles = g.n * pl.num_tiles;
+    p.total_blocks = static_cast<long long>(p.num_tiles) * kblocks;
+    int grid = sm_count();
+    if (grid > p.total_blocks) grid = static_cast<int>(p.total_blocks);
+    if (launch_pdl(gemm_w8a16_kernel<false, false, true>, dim3(grid), dim3(kGemmThreads), smem_bytes, s, pdl, tmap_w, tmap_w, tmap_x, p, g) !=
+        cudaSuccess)
+      return MSD_ERR_CUDA;
+  }
+  return MSD_OK;
+}
+
 // ---------------------------------------------------------------------------------------------------------------------
 }  // extern "C"
 
