@@ -182,6 +182,20 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
                             void* stream);
 
 /*
+ * The paper-literal MXFP4 components (Sec. 3.2.1, Alg. 2; Tab. mxfp4-evolution): both passes round onto the E1M2 grid
+ * {0, .25, ..., 1.75}, alpha = 2^ceil(log2(blockmax / 1.859375)) (exponent kept >= -123), beta = alpha / 16, error bound
+ * alpha / 64.  Tensor cores have no E1M2 operand type; every E1M2 value is an E4M3 number, so the components are
+ * emitted as E4M3 bytes and multiplied with tcgen05.mma kind::mxf8f6f4 (E4M3 x E2M1, block scales) at the FP8 rate.
+ *   msd_decompose_mxfp4_e1m2: q1/q2 [M, K] E4M3 bytes, e8m0_1/e8m0_2 [M, K/32] row-major; K % 32 == 0.
+ *   msd_gemm_w4a16_e1m2: same arguments and result layout as msd_gemm_w4a16; K % 128 == 0; w_fp4 32-byte aligned.
+ */
+msd_status_t msd_decompose_mxfp4_e1m2(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1_e4m3, uint8_t* q2_e4m3,
+                                      uint8_t* e8m0_1, uint8_t* e8m0_2, void* stream);
+size_t msd_gemm_w4a16_e1m2_workspace_bytes(int64_t M, int64_t N, int64_t K);
+msd_status_t msd_gemm_w4a16_e1m2(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0, int64_t M, int64_t N,
+                                 int64_t K, void* y, msd_out_t ytype, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Decode attention over an INT8 KV cache (Sec. 4, Alg. 3; tiled form Sec. 4.3) with one scale per token per
  * KV head, split over the context (flash-decoding) and merged with the log-sum-exp rule:
  *   Q row decomposed two-pass INT8; S_j = (alpha_Q S1_j + beta_Q S2_j) * k_scale[j] * softmax_scale;

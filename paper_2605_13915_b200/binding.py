@@ -52,6 +52,9 @@ _SIGS = {
     "msd_attn_decode_int8kv": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp,
                                          _vp, _sz, _vp]),
     "msd_attn_decode_schedule": (C.c_int, [_i32] * 6 + [C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
+    "msd_decompose_mxfp4_e1m2": (C.c_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp]),
+    "msd_gemm_w4a16_e1m2_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "msd_gemm_w4a16_e1m2": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_attn_decode_int8kv_spec": (C.c_int, [_vp] * 6 + [_i64, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp, _vp, _sz, _vp]),
     "msd_attn_decode_int8kv_paged": (C.c_int, [_vp] * 7 + [_i64, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp, _vp,
                                                 _sz, _vp]),
@@ -253,6 +256,34 @@ def attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen):
     _check(lib().msd_attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen, C.byref(tile), C.byref(ns), C.byref(st)),
            "msd_attn_decode_schedule")
     return tile.value, ns.value, st.value
+
+
+def decompose_mxfp4_e1m2(x):
+    """x [M,K] bfloat16 -> (q1, q2 uint8 [M,K] E4M3 bytes of the E1M2 components, e8m0_1, e8m0_2 uint8 [M,K/32])."""
+    _need_cuda(x)
+    M, K = x.shape
+    q1 = torch.empty((M, K), dtype=torch.uint8, device=x.device)
+    q2 = torch.empty((M, K), dtype=torch.uint8, device=x.device)
+    e1 = torch.empty((M, K // 32), dtype=torch.uint8, device=x.device)
+    e2 = torch.empty((M, K // 32), dtype=torch.uint8, device=x.device)
+    _check(lib().msd_decompose_mxfp4_e1m2(_ptr(x), M, K, x.stride(0) if M else K, _ptr(q1), _ptr(q2), _ptr(e1), _ptr(e2), _stream()),
+           "msd_decompose_mxfp4_e1m2")
+    return q1, q2, e1, e2
+
+
+def gemm_w4a16_e1m2(x, w_fp4, w_e8m0, out_dtype=torch.bfloat16, ws=None, out=None):
+    """W4A16 with the paper-literal E1M2 components (FP8-rate tensor-core path)."""
+    _need_cuda(x, w_fp4, w_e8m0)
+    M, K = x.shape
+    N = w_fp4.shape[0]
+    if ws is None:
+        ws = workspace(int(lib().msd_gemm_w4a16_e1m2_workspace_bytes(M, N, K)), x.device)
+    y = out if out is not None else torch.empty((M, N), dtype=out_dtype, device=x.device)
+    wp, wb = _ws_ptr(ws)
+    code = lib().msd_gemm_w4a16_e1m2(_ptr(x), _ptr(w_fp4), _ptr(w_e8m0), M, N, K, _ptr(y),
+                                     OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream())
+    _check(code, "msd_gemm_w4a16_e1m2")
+    return y
 
 
 def attn_decode_int8kv_spec(q, k, v, k_scale, v_scale, cu_seqlens, max_seqlen, softmax_scale, dv=None, ws=None, want_lse=False):
