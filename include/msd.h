@@ -56,6 +56,11 @@ const char* msd_status_string(msd_status_t s);
  * or MSD_ERR_CUDA. */
 msd_status_t msd_last_device_status(void* stream);
 
+/* Self-test of the give-up path every device-side wait of this library has: launches a tiny kernel that waits, with
+ * the given budget in SM cycles (clamped to [1e3, 2e8]), on a barrier nobody arrives on.  The kernel ends by itself,
+ * and the next msd_last_device_status returns MSD_ERR_TIMEOUT; the context stays usable. */
+msd_status_t msd_debug_timeout_selftest(int64_t budget_cycles, void* stream);
+
 /* Zero-fills a workspace (asynchronous memset on `stream`). */
 msd_status_t msd_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 

@@ -58,6 +58,7 @@ _SIGS = {
     "msd_attn_decode_int8kv_spec": (C.c_int, [_vp] * 6 + [_i64, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp, _vp, _sz, _vp]),
     "msd_attn_decode_int8kv_paged": (C.c_int, [_vp] * 7 + [_i64, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp, _vp,
                                                 _sz, _vp]),
+    "msd_debug_timeout_selftest": (C.c_int, [_i64, _vp]),
     "msd_kv_dequant_bf16": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, _i32, _i32, C.c_void_p, C.c_void_p]),
 }
 

@@ -2,6 +2,7 @@
 #include <mutex>
 
 #include "host_common.h"
+#include "sm100.cuh"
 
 namespace msd {
 
@@ -77,6 +78,25 @@ bool encode_tmap_3d(CUtensorMap* out, CUtensorMapDataType dtype, const void* bas
 
 }  // namespace msd
 
+namespace msd {
+// Exercises the give-up path of the bounded waits without harming anything: one warp waits on a barrier that nobody
+// ever arrives on, with a short cycle budget; when it runs out the wait records MSD_ERR_TIMEOUT in the status word,
+// raises the CTA's abort flag (which the second warp, waiting with the full budget, sees at once) and the kernel ends.
+__global__ void timeout_selftest_kernel(unsigned* status, long long budget) {
+  __shared__ __align__(8) uint64_t never;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&never, 1);
+    abort_flag = 0;
+    mbar_init_fence();
+  }
+  __syncthreads();
+  volatile int* abort = &abort_flag;
+  if (threadIdx.x < 32) wait_bounded_cycles(&never, 0, abort, status, budget);
+  else wait_bounded(&never, 0, abort, status);
+}
+}  // namespace msd
+
 extern "C" {
 
 const char* msd_status_string(msd_status_t s) {
@@ -106,6 +126,15 @@ msd_status_t msd_last_device_status(void* stream) {
     if (cudaStreamSynchronize(s) != cudaSuccess) return MSD_ERR_CUDA;
   }
   return v == 0 ? MSD_OK : (v == MSD_ERR_TIMEOUT ? MSD_ERR_TIMEOUT : MSD_ERR_CUDA);
+}
+
+msd_status_t msd_debug_timeout_selftest(int64_t budget_cycles, void* stream) {
+  unsigned* p = msd::device_status_ptr();
+  if (!p) return MSD_ERR_CUDA;
+  if (budget_cycles < 1000) budget_cycles = 1000;
+  if (budget_cycles > 200000000LL) budget_cycles = 200000000LL;      // a tenth of a second at most
+  msd::timeout_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(p, static_cast<long long>(budget_cycles));
+  return msd::launch_status();
 }
 
 msd_status_t msd_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {

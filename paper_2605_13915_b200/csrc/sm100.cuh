@@ -66,18 +66,22 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
 
 // Waits for the barrier phase; gives up after the cycle budget or as soon as another role of the CTA has
 // raised *abort.  Returns false on give-up (status word and *abort are then set).
-__device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort, unsigned* status) {
+__device__ __forceinline__ bool wait_bounded_cycles(uint64_t* bar, uint32_t parity, volatile int* abort, unsigned* status,
+                                                    long long budget) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort) return false;
-    if (clock64() - t0 > kWaitBudgetCycles) {
+    if (clock64() - t0 > budget) {
       *abort = 1;
       atomicMax(status, kStatusTimeout);
       return false;
     }
   }
+}
+__device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort, unsigned* status) {
+  return wait_bounded_cycles(bar, parity, abort, status, kWaitBudgetCycles);
 }
 
 // ---- thread-block cluster: peers' shared memory and barriers ------------------------------------------------
