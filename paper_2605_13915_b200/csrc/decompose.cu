@@ -91,14 +91,44 @@ constexpr int kMxThreads = 256;
 // 2^e as an FP32 number for e in [-126, 127]
 __device__ __forceinline__ float pow2f(int e) { return __uint_as_float(static_cast<uint32_t>(e + 127) << 23); }
 
+// Relayout of row-major E8M0 scales [rows, kblocks] into the 512-byte blocks (128 rows x 4 scales) of the block-scaled
+// MMA.  Rows are first cut into tiles of `tile_rows` (a multiple of 32), every tile into two blocks (the second one
+// partly used when tile_rows < 256); entries outside the matrix are written as zero.  One thread per 16 bytes of
+// the result: the four scales of rows l, l+32, l+64, l+96 of one block.
+__device__ void sf_relayout(const SfRelayout& j, int64_t first, int64_t step) {
+  const int64_t total = static_cast<int64_t>(j.row_blocks) * j.sf_kgroups * 32;
+  for (int64_t d = first; d < total; d += step) {
+    const int l = static_cast<int>(d & 31);
+    const int64_t blk = d >> 5;
+    const int64_t tb = blk / j.sf_kgroups;
+    const int kg = static_cast<int>(blk - tb * j.sf_kgroups);
+    const int64_t t = tb >> 1;
+    uint32_t v[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int lr = static_cast<int>(tb & 1) * 128 + l + 32 * q;
+      const int64_t row = t * j.tile_rows + lr;
+      v[q] = (lr < j.tile_rows && row < j.rows && 4 * kg < j.kblocks)
+                 ? __ldg(reinterpret_cast<const uint32_t*>(j.src + row * j.kblocks + 4 * kg)) : 0u;
+    }
+    reinterpret_cast<uint4*>(j.dst)[d] = make_uint4(v[0], v[1], v[2], v[3]);
+  }
+}
+
+// The first `rl.blocks` CTAs do the (independent) scale relayout `rl`, the others the decomposition.
 __global__ void __launch_bounds__(kMxThreads)
 decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, int K, uint8_t* __restrict__ q1,
-                       uint8_t* __restrict__ q2, uint8_t* __restrict__ e1, uint8_t* __restrict__ e2, int sf_kgroups) {
+                       uint8_t* __restrict__ q2, uint8_t* __restrict__ e1, uint8_t* __restrict__ e2, int sf_kgroups,
+                       const SfRelayout rl) {
   pdl_launch_dependents();
+  if (static_cast<int>(blockIdx.x) < rl.blocks) {
+    sf_relayout(rl, static_cast<int64_t>(blockIdx.x) * kMxThreads + threadIdx.x, static_cast<int64_t>(rl.blocks) * kMxThreads);
+    return;
+  }
   const int kblocks = K >> 5;
   const int64_t nblocks = M * kblocks;
-  for (int64_t b = static_cast<int64_t>(blockIdx.x) * kMxThreads + threadIdx.x; b < nblocks;
-       b += static_cast<int64_t>(gridDim.x) * kMxThreads) {
+  for (int64_t b = static_cast<int64_t>(blockIdx.x - rl.blocks) * kMxThreads + threadIdx.x; b < nblocks;
+       b += static_cast<int64_t>(gridDim.x - rl.blocks) * kMxThreads) {
     const int64_t row = b / kblocks;
     const int kb = static_cast<int>(b - row * kblocks);
     const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx + kb * 32);
@@ -173,19 +203,26 @@ msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int
 }
 
 msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
-                                    uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream) {
+                                    uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream, const SfRelayout* relayout) {
   if (M == 0) return MSD_OK;
+  SfRelayout rl = {};
+  if (relayout) {
+    rl = *relayout;
+    const int64_t chunks = static_cast<int64_t>(rl.row_blocks) * rl.sf_kgroups * 32;
+    const int64_t rb = (chunks + kMxThreads - 1) / kMxThreads;
+    rl.blocks = static_cast<int>(rb < 4 * sm_count() ? rb : 4 * sm_count());
+  }
   const int64_t nblocks = M * (K >> 5);
   const int64_t want = (nblocks + kMxThreads - 1) / kMxThreads;
   const int64_t cap = static_cast<int64_t>(sm_count()) * 32;
-  const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
+  const unsigned grid = static_cast<unsigned>(want < cap ? want : cap) + static_cast<unsigned>(rl.blocks);
   static bool carve_done = false;
   if (!carve_done) {
     cudaFuncSetAttribute(decompose_mxfp4_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     carve_done = true;
   }
   decompose_mxfp4_kernel<<<grid, kMxThreads, 0, stream>>>(static_cast<const uint16_t*>(x_bf16), ldx, M,
-                                                          static_cast<int>(K), q1, q2, e1, e2, sf_kgroups);
+                                                          static_cast<int>(K), q1, q2, e1, e2, sf_kgroups, rl);
   return launch_status();
 }
 

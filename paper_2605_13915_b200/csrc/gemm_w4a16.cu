@@ -22,12 +22,14 @@ namespace msd {
 constexpr int kW4TileM = 128;
 constexpr int kW4TileN = 256;
 constexpr int kW4BlockK = 256;                                  // elements per stage (128 packed bytes)
-constexpr int kW4Threads = 192;
+constexpr int kW4ThreadsSf = 352;      // producer, MMA, four epilogue warps, four warps that write the scales into TMEM, scale producer
+constexpr int kW4PairThreads = 320;    // the same without the separate scale producer
 constexpr int kW4ABytes = kW4TileM * 128;                       // 16 KB
 constexpr int kW4BBytes = kW4TileN * 128;                       // 32 KB
 constexpr int kW4SfBytes = 1024 + 1024 + 2048;                  // SFA1, SFA2 (2 k-groups each), SFB (2 row tiles x 2 k-groups)
 constexpr int kW4StageBytes = 2 * kW4ABytes + kW4BBytes + kW4SfBytes;   // 69632
 constexpr int kW4Stages = 3;
+constexpr int kW4StoreBytes = 2048;                              // one epilogue chunk: 32 rows x 64 bytes
 constexpr int kW4TmemCols = 512;
 constexpr int kW4SfCol = 256;                                   // scale columns follow the 256 accumulator columns
 
@@ -40,36 +42,26 @@ struct GemmW4Params {
   const uint8_t* sfb;
   void* y;
   int ytype;
+  int n_fastest;                // tile index -> (token tile, weight tile): weight tile fastest (1) or token tile fastest (0)
+  int sf_warps;                 // 1: warps 6..9 write the scales into TMEM (tcgen05.st); 0: the MMA thread copies them (tcgen05.cp)
   unsigned* status;
 };
-
-// Relayout of row-major E8M0 scales [rows, K/32] into 512-byte blocks (128 rows x 4 scales).  Rows are first cut into
-// tiles of `tile_rows` (a multiple of 32), every tile into two blocks (the second one partly used when tile_rows < 256).
-__global__ void sf_block_layout_kernel(const uint8_t* __restrict__ src, int64_t rows, int kblocks, int sf_kgroups,
-                                       int tile_rows, uint8_t* __restrict__ dst) {
-  const int64_t total = rows * kblocks;
-  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
-       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
-    const int64_t row = i / kblocks;
-    const int kb = static_cast<int>(i - row * kblocks);
-    const int64_t t = row / tile_rows;
-    const int lr = static_cast<int>(row - t * tile_rows);
-    dst[((2 * t + (lr >> 7)) * sf_kgroups + (kb >> 2)) * 512 + (lr & 31) * 16 + ((lr >> 5) & 3) * 4 + (kb & 3)] = src[i];
-  }
-}
 
 // kTN = weight rows per tile: 256 (one accumulator) or 224 (two accumulators of 224 columns + the two sets of scale
 // columns fill the 512 TMEM columns exactly, so the epilogue of a tile overlaps the MMAs of the next).
 template <int kTN>
-__global__ void __launch_bounds__(kW4Threads, 1)
+__global__ void __launch_bounds__(kW4ThreadsSf, 1)
 gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
-                  const __grid_constant__ CUtensorMap tmap_b, const GemmW4Params p) {
+                  const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_y,
+                  const GemmW4Params p) {
   constexpr int kBBytes = kTN * 128;
   constexpr int kStageBytes = 2 * kW4ABytes + kBBytes + kW4SfBytes;
   constexpr int kAcc = (2 * kTN + 64 <= kW4TmemCols) ? 2 : 1;       // accumulators that fit beside 2 x 32 scale columns
   constexpr int kSfCol = kAcc * kTN;
   extern __shared__ uint8_t smem_dyn[];
   __shared__ __align__(8) uint64_t full_bar[kW4Stages], empty_bar[kW4Stages], tfull_bar[2], tempty_bar[2];
+  // the two sets of scale columns in TMEM: written by warps 6..9 (sf_ready), read by the MMAs of a stage (sf_free)
+  __shared__ __align__(8) uint64_t sf_ready[2], sf_free[2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
@@ -79,6 +71,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
   if (threadIdx.x == 0) {
     for (int s = 0; s < kW4Stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&sf_ready[a], 4); mbar_init(&sf_free[a], 1); }
     abort_flag = 0;
     mbar_init_fence();
     tma_prefetch_desc(&tmap_a1);
@@ -93,27 +86,34 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
   volatile int* abort = &abort_flag;
   const int total_tiles = p.m_tiles * p.n_tiles;
 
-  if (warp == 0) {
+  if (warp == 0 || warp == 10) {
+    // Two producer threads: issuing a bulk copy costs its thread 50-100 ns, and the time a freed stage waits for its
+    // refill to be requested is part of the pipeline's round trip.  Warp 0 requests the operand tiles, warp 10 the
+    // scale blocks (their bytes may be counted before warp 0's arrival announces them: the phase cannot end without it).
     if (lane == 0) {
       pdl_wait_primary();           // components and blocked scales come from the kernels launched just before
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
+      const bool sf_smem = p.sf_warps != 2;             // otherwise warps 6..9 read the scales from global memory
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+        const int mt = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles, nt = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
         for (int ks = 0; ks < p.kstages; ++ks) {
           ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
           if (!ok) break;
-          mbar_arrive_expect_tx(&full_bar[stage], kStageBytes);
           uint8_t* dst = smem + stage * kStageBytes;
-          tma_load_2d(dst, &tmap_a1, ks * 128, mt * kW4TileM, &full_bar[stage]);
-          tma_load_2d(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, &full_bar[stage]);
-          tma_load_2d(dst + 2 * kW4ABytes, &tmap_b, ks * 128, nt * kTN, &full_bar[stage]);
-          uint8_t* sf = dst + 2 * kW4ABytes + kBBytes;
-          const size_t a_off = (static_cast<size_t>(mt) * p.sf_kgroups + 2 * ks) * 512;
-          bulk_load(sf, p.sfa1 + a_off, 1024, &full_bar[stage]);
-          bulk_load(sf + 1024, p.sfa2 + a_off, 1024, &full_bar[stage]);
-          bulk_load(sf + 2048, p.sfb + (static_cast<size_t>(2 * nt) * p.sf_kgroups + 2 * ks) * 512, 1024, &full_bar[stage]);
-          bulk_load(sf + 3072, p.sfb + (static_cast<size_t>(2 * nt + 1) * p.sf_kgroups + 2 * ks) * 512, 1024, &full_bar[stage]);
+          if (warp == 0) {
+            mbar_arrive_expect_tx(&full_bar[stage], sf_smem ? kStageBytes : kStageBytes - kW4SfBytes);
+            tma_load_2d(dst, &tmap_a1, ks * 128, mt * kW4TileM, &full_bar[stage]);
+            tma_load_2d(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, &full_bar[stage]);
+            tma_load_2d(dst + 2 * kW4ABytes, &tmap_b, ks * 128, nt * kTN, &full_bar[stage]);
+          } else if (sf_smem) {
+            uint8_t* sf = dst + 2 * kW4ABytes + kBBytes;
+            const size_t a_off = (static_cast<size_t>(mt) * p.sf_kgroups + 2 * ks) * 512;
+            bulk_load(sf, p.sfa1 + a_off, 1024, &full_bar[stage]);
+            bulk_load(sf + 1024, p.sfa2 + a_off, 1024, &full_bar[stage]);
+            bulk_load(sf + 2048, p.sfb + (static_cast<size_t>(2 * nt) * p.sf_kgroups + 2 * ks) * 512, 1024, &full_bar[stage]);
+            bulk_load(sf + 3072, p.sfb + (static_cast<size_t>(2 * nt + 1) * p.sf_kgroups + 2 * ks) * 512, 1024, &full_bar[stage]);
+          }
           if (++stage == kW4Stages) { stage = 0; phase ^= 1; }
         }
       }
@@ -124,6 +124,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
       int it = 0;
       bool ok = true;
       uint32_t sfpar = 0;
+      int nstage = 0;                                                   // stages issued so far (all tiles)
       const uint64_t op_desc = smem_desc(0, 16, 1024, kSwizzle128B);    // 128-byte-swizzled K-major operand tile
       const uint64_t sf_desc = smem_desc(0, 0, 128, 0);                 // scale block: eight-row groups 128 bytes apart, no swizzle
       const uint32_t idesc_lo = idesc_block_scaled(/*E2M1*/ 1, 1, kW4TileM, kTN, 0, 0);
@@ -148,13 +149,20 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           const uint32_t sfa1_t = tmem_base + kSfCol + 32 * sfpar;     // 2 k-groups x 4 columns; the two sets alternate
           const uint32_t sfa2_t = sfa1_t + 8;
           const uint32_t sfb_t = sfa1_t + 16;                            // 2 k-groups x 8 columns (256 weight rows)
-          sfpar ^= 1;
+          if (p.sf_warps) {
+            // the scale columns of this stage were written by warps 6..9 (the shared-memory -> TMEM copies of the tensor
+            // pipe run in order with the MMAs and cost a sixth of its time)
+            ok = wait_bounded(&sf_ready[sfpar], (nstage >> 1) & 1, abort, p.status);
+            if (!ok) break;
+            tc_fence_after();
+          } else {
 #pragma unroll
-          for (int g = 0; g < 2; ++g) {
-            tc_cp_32x128b_warpx4(sfa1_t + 4 * g, sfd + (g * 512 >> 4));
-            tc_cp_32x128b_warpx4(sfa2_t + 4 * g, sfd + ((1024 + g * 512) >> 4));
-            tc_cp_32x128b_warpx4(sfb_t + 8 * g, sfd + ((2048 + g * 512) >> 4));
-            tc_cp_32x128b_warpx4(sfb_t + 8 * g + 4, sfd + ((3072 + g * 512) >> 4));
+            for (int g = 0; g < 2; ++g) {
+              tc_cp_32x128b_warpx4(sfa1_t + 4 * g, sfd + (g * 512 >> 4));
+              tc_cp_32x128b_warpx4(sfa2_t + 4 * g, sfd + ((1024 + g * 512) >> 4));
+              tc_cp_32x128b_warpx4(sfb_t + 8 * g, sfd + ((2048 + g * 512) >> 4));
+              tc_cp_32x128b_warpx4(sfb_t + 8 * g + 4, sfd + ((3072 + g * 512) >> 4));
+            }
           }
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {                    // 64 elements (32 bytes) per MMA
@@ -163,6 +171,9 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
             mma_mxf4(d_tmem, a1d + 2 * kk, bd + 2 * kk, idesc, sfa1_t + 4 * g, sfb_t + 8 * g, (ks > 0 || kk > 0) ? 1u : 0u);
             mma_mxf4(d_tmem, a2d + 2 * kk, bd + 2 * kk, idesc, sfa2_t + 4 * g, sfb_t + 8 * g, 1u);
           }
+          tc_commit(&sf_free[sfpar]);                // this set of scale columns may be rewritten once these MMAs are done
+          sfpar ^= 1;
+          ++nstage;
           tc_commit(&empty_bar[stage]);
           if (++stage == kW4Stages) { stage = 0; phase ^= 1; }
         }
@@ -170,13 +181,325 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
         tc_commit(&tfull_bar[acc]);
       }
     }
+  } else if (warp >= 6) {      // (warp 10 went the producers' way above)
+    // Scale warps.  A 512-byte scale block holds, for 128 rows and one 128-element K group, 32 rows of 16 bytes: row l
+    // carries the four scales of rows l, l+32, l+64, l+96, and every 32-lane quadrant of TMEM wants the same four
+    // 32-bit columns.  Each warp reads the stage's eight blocks (one 16-byte row per lane and block) and stores them as
+    // 32 columns of its own quadrant.
+    if (p.sf_warps == 2) {
+      // Scales straight from global memory (L2), one stage ahead in registers: they stay out of the shared-memory
+      // pipeline, and a set of scale columns is ready before the stage's operands land.
+      const int quad = warp & 3;
+      pdl_wait_primary();           // the blocked scales come from the kernels launched just before
+      int n = 0;
+      bool ok = true;
+      uint4 q[8];
+      auto fetch = [&](int tile, int ks) {
+        const int mt = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles, nt = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
+        const size_t a_off = (static_cast<size_t>(mt) * p.sf_kgroups + 2 * ks) * 512 + lane * 16;
+        const size_t b0_off = (static_cast<size_t>(2 * nt) * p.sf_kgroups + 2 * ks) * 512 + lane * 16;
+        const size_t b1_off = b0_off + static_cast<size_t>(p.sf_kgroups) * 512;
+        q[0] = __ldg(reinterpret_cast<const uint4*>(p.sfa1 + a_off));
+        q[1] = __ldg(reinterpret_cast<const uint4*>(p.sfa1 + a_off + 512));
+        q[2] = __ldg(reinterpret_cast<const uint4*>(p.sfa2 + a_off));
+        q[3] = __ldg(reinterpret_cast<const uint4*>(p.sfa2 + a_off + 512));
+        q[4] = __ldg(reinterpret_cast<const uint4*>(p.sfb + b0_off));
+        q[5] = __ldg(reinterpret_cast<const uint4*>(p.sfb + b1_off));
+        q[6] = __ldg(reinterpret_cast<const uint4*>(p.sfb + b0_off + 512));
+        q[7] = __ldg(reinterpret_cast<const uint4*>(p.sfb + b1_off + 512));
+      };
+      if (static_cast<int>(blockIdx.x) < total_tiles) fetch(blockIdx.x, 0);
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int ks = 0; ks < p.kstages; ++ks, ++n) {
+          const int set = n & 1;
+          uint32_t v[32];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) { v[4 * j] = q[j].x; v[4 * j + 1] = q[j].y; v[4 * j + 2] = q[j].z; v[4 * j + 3] = q[j].w; }
+          if (ks + 1 < p.kstages) fetch(tile, ks + 1);
+          else if (tile + static_cast<int>(gridDim.x) < total_tiles) fetch(tile + gridDim.x, 0);
+          if (n >= 2) {                        // the MMAs that read this set two stages ago are done
+            ok = wait_bounded(&sf_free[set], ((n >> 1) - 1) & 1, abort, p.status);
+            if (!ok) break;
+            tc_fence_after();
+          }
+          tmem_st32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + kSfCol + 32 * set, v);
+          tmem_st_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sf_ready[set]);
+        }
+      }
+    } else if (p.sf_warps) {
+      const int quad = warp & 3;
+      int stage = 0; uint32_t phase = 0;
+      int n = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int ks = 0; ks < p.kstages; ++ks, ++n) {
+          const int set = n & 1;
+          ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
+          if (!ok) break;
+          if (n >= 2) {                        // the MMAs that read this set two stages ago are done
+            ok = wait_bounded(&sf_free[set], ((n >> 1) - 1) & 1, abort, p.status);
+            if (!ok) break;
+            tc_fence_after();
+          }
+          const uint4* sf = reinterpret_cast<const uint4*>(smem + stage * kStageBytes + 2 * kW4ABytes + kBBytes) + lane;
+          uint32_t v[32];
+          // column order of a set: sfa1 (g0, g1), sfa2 (g0, g1), then per K group the two halves of the weight tile
+          constexpr int kBlk[8] = {0, 1, 2, 3, 4, 6, 5, 7};
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint4 q = sf[kBlk[j] * 32];
+            v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
+          }
+          tmem_st32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + kSfCol + 32 * set, v);
+          tmem_st_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sf_ready[set]);
+          if (++stage == kW4Stages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else {
+    // Epilogue: TMEM -> registers -> (BF16) -> this warp's staging buffer in shared memory -> TMA store.  A chunk is
+    // 64 bytes of every row of the warp's 32 rows (32 BF16 or 16 FP32 columns), laid out with the 64-byte swizzle of
+    // the output tensor map so that the 16-byte stores of the 32 lanes spread over all banks; two buffers per warp,
+    // the store of one chunk in flight while the next is converted.  Rows past M and columns past N are clipped by
+    // the store itself.
+    const int quad = warp & 3;
+    uint8_t* stage_buf = smem + kW4Stages * kStageBytes + quad * (2 * kW4StoreBytes);
+    const int ccols = (p.ytype == MSD_OUT_BF16) ? 32 : 16;
+    const uint32_t swz = static_cast<uint32_t>((lane >> 1) & 3);
+    int it = 0, buf = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+      const int mt = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles, nt = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
+      const int acc = (kAcc == 2) ? (it & 1) : 0;
+      const uint32_t tphase = (kAcc == 2) ? ((it >> 1) & 1) : (it & 1);
+      ok = wait_bounded(&tfull_bar[acc], tphase, abort, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      const int row0 = mt * kW4TileM + quad * 32;
+      const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * kTN;
+      for (int c0 = 0; c0 < kTN; c0 += ccols, buf ^= 1) {
+        uint32_t o[16];
+        if (p.ytype == MSD_OUT_BF16) {
+          uint32_t v[32];
+          tmem_ld32(trow + c0, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+            o[j] = *reinterpret_cast<const uint32_t*>(&h);
+          }
+        } else {
+          tmem_ld16(trow + c0, o);
+          tmem_ld_wait();
+        }
+        if (c0 + ccols >= kTN) {                    // all of this accumulator is in registers: the MMAs may have it back
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+        }
+        uint8_t* sb = stage_buf + buf * kW4StoreBytes;
+        if (lane == 0) bulk_wait_group_read<1>();    // the store that read this buffer two chunks ago is done with it
+        __syncwarp();
+        uint8_t* srow = sb + lane * 64;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          *reinterpret_cast<uint4*>(srow + ((static_cast<uint32_t>(j) ^ swz) << 4)) = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        const int col = nt * kTN + c0;
+        if (lane == 0 && row0 < p.M && col < p.N) {
+          tma_store_2d(&tmap_y, col, row0, sb);
+          bulk_commit_group();
+        }
+      }
+    }
+    if (lane == 0) bulk_wait_group<0>();            // every store has been written before the CTA goes away
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kW4TmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------------------
+// CTA-pair kernel: two CTAs of a cluster share one 256 x kTN tile.  Each CTA loads its own 128 activation rows (both
+// components) and HALF of the weight tile; one tcgen05.mma.cta_group::2 per K step, issued by the even CTA, multiplies
+// all 256 rows against all kTN weight rows, each CTA's accumulator (its 128 rows x kTN columns) staying in its own
+// TMEM.  Why: the single-CTA kernel is bound by the round trip of its shared-memory pipeline (a freed stage is refilled
+// from L2 about 1.9 us later; three 64 KB stages in flight feed 80 GB/s per SM where the tensor pipe wants 116).  A
+// pair needs 46 KB of operands for the same tensor time and holds four stages.
+//
+// Barriers.  Operand tiles of both CTAs complete on the LEADER's full_bar; the scale blocks complete on each CTA's own
+// sf_full (its scale warps read them); the scale warps of both CTAs arrive on the leader's sf_ready (8 arrivals); the
+// leader's commits (empty_bar, sf_free, tfull_bar) are multicast to both CTAs; both epilogues arrive on the leader's
+// tempty_bar.
+constexpr int kW4PairStages = 4;
+
+template <int kTN>
+__global__ void __launch_bounds__(kW4PairThreads, 1)
+gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
+                       const __grid_constant__ CUtensorMap tmap_bh, const GemmW4Params p) {
+  constexpr int kBHalfBytes = (kTN / 2) * 128;
+  constexpr int kOpBytes = 2 * kW4ABytes + kBHalfBytes;             // operand bytes per CTA and stage
+  constexpr int kStageBytes = kOpBytes + kW4SfBytes;
+  constexpr int kAcc = (2 * kTN + 64 <= kW4TmemCols) ? 2 : 1;
+  constexpr int kSfCol = kAcc * kTN;
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ __align__(8) uint64_t full_bar[kW4PairStages], empty_bar[kW4PairStages], sf_full[kW4PairStages];
+  __shared__ __align__(8) uint64_t tfull_bar[2], tempty_bar[2], sf_ready[2], sf_free[2];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kW4PairStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); mbar_init(&sf_full[s], 1); }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&tfull_bar[a], 1);
+      mbar_init(&tempty_bar[a], 8);     // four epilogue warps in each CTA of the pair (used in the leader only)
+      mbar_init(&sf_ready[a], 8);       // four scale warps in each CTA (used in the leader only)
+      mbar_init(&sf_free[a], 1);
+    }
+    abort_flag = 0;
+    mbar_init_fence();
+    tma_prefetch_desc(&tmap_a1);
+    tma_prefetch_desc(&tmap_a2);
+    tma_prefetch_desc(&tmap_bh);
+  }
+  if (warp == 1) tmem_alloc_pair(&tmem_base_slot, kW4TmemCols);
+  tc_fence_before();
+  cluster_arrive_all();        // both CTAs' barriers exist before either signals the other's
+  cluster_wait_all();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  volatile int* abort = &abort_flag;
+  const int m_pairs = (p.m_tiles + 1) >> 1;
+  const int total_tiles = m_pairs * p.n_tiles;
+  const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      pdl_wait_primary();           // components and blocked scales come from the kernels launched just before
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
+        const int mt = 2 * (tile % m_pairs) + static_cast<int>(rank), nt = tile / m_pairs;
+        const int mt_sf = mt < p.m_tiles ? mt : p.m_tiles - 1;       // the odd last pair: rows past M are zero-filled anyway
+        for (int ks = 0; ks < p.kstages; ++ks) {
+          ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
+          if (!ok) break;
+          // the leader's barrier counts the operand bytes of both CTAs
+          if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * kOpBytes);
+          const uint32_t bar = mapa_shared(smem_u32(&full_bar[stage]), 0);
+          uint8_t* dst = smem + stage * kStageBytes;
+          tma_load_2d_pair(dst, &tmap_a1, ks * 128, mt * kW4TileM, bar);
+          tma_load_2d_pair(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, bar);
+          tma_load_2d_pair(dst + 2 * kW4ABytes, &tmap_bh, ks * 128, nt * kTN + static_cast<int>(rank) * (kTN / 2), bar);
+          uint8_t* sf = dst + kOpBytes;
+          mbar_arrive_expect_tx(&sf_full[stage], kW4SfBytes);
+          const size_t a_off = (static_cast<size_t>(mt_sf) * p.sf_kgroups + 2 * ks) * 512;
+          bulk_load(sf, p.sfa1 + a_off, 1024, &sf_full[stage]);
+          bulk_load(sf + 1024, p.sfa2 + a_off, 1024, &sf_full[stage]);
+          bulk_load(sf + 2048, p.sfb + (static_cast<size_t>(2 * nt) * p.sf_kgroups + 2 * ks) * 512, 1024, &sf_full[stage]);
+          bulk_load(sf + 3072, p.sfb + (static_cast<size_t>(2 * nt + 1) * p.sf_kgroups + 2 * ks) * 512, 1024, &sf_full[stage]);
+          if (++stage == kW4PairStages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      int stage = 0; uint32_t phase = 0;
+      int it = 0, nstage = 0;
+      bool ok = true;
+      const uint64_t op_desc = smem_desc(0, 16, 1024, kSwizzle128B);    // 128-byte-swizzled K-major operand tile
+      const uint32_t idesc_lo = idesc_block_scaled(/*E2M1*/ 1, 1, 2 * kW4TileM, kTN, 0, 0);
+      const uint32_t idesc_hi = idesc_block_scaled(/*E2M1*/ 1, 1, 2 * kW4TileM, kTN, 2, 2);
+      for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++it) {
+        const int acc = (kAcc == 2) ? (it & 1) : 0;
+        const uint32_t tphase = (kAcc == 2) ? ((it >> 1) & 1) : (it & 1);
+        const uint32_t d_tmem = tmem_base + acc * kTN;
+        ok = wait_bounded_cluster(&tempty_bar[acc], tphase ^ 1, abort, p.status);   // both epilogues have drained this accumulator
+        if (!ok) break;
+        tc_fence_after();
+        for (int ks = 0; ks < p.kstages; ++ks, ++nstage) {
+          const int set = nstage & 1;
+          ok = wait_bounded_cluster(&full_bar[stage], phase, abort, p.status);
+          if (!ok) break;
+          ok = wait_bounded_cluster(&sf_ready[set], (nstage >> 1) & 1, abort, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t enc = static_cast<uint64_t>(smem_u32(smem + stage * kStageBytes) >> 4);
+          const uint64_t a1d = op_desc + enc, a2d = a1d + (kW4ABytes >> 4), bd = a1d + (2 * kW4ABytes >> 4);
+          const uint32_t sfa1_t = tmem_base + kSfCol + 32 * set;        // 2 k-groups x 4 columns; the two sets alternate
+          const uint32_t sfa2_t = sfa1_t + 8;
+          const uint32_t sfb_t = sfa1_t + 16;                            // 2 k-groups x 8 columns (256 weight rows)
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {                    // 64 elements (32 bytes) per MMA
+            const int g = kk >> 1;
+            const uint32_t idesc = (kk & 1) ? idesc_hi : idesc_lo;   // which pair of scale bytes of the 4-scale column
+            mma_mxf4_pair(d_tmem, a1d + 2 * kk, bd + 2 * kk, idesc, sfa1_t + 4 * g, sfb_t + 8 * g, (ks > 0 || kk > 0) ? 1u : 0u);
+            mma_mxf4_pair(d_tmem, a2d + 2 * kk, bd + 2 * kk, idesc, sfa2_t + 4 * g, sfb_t + 8 * g, 1u);
+          }
+          tc_commit_pair(&sf_free[set], 3);         // this set of scale columns may be rewritten in both CTAs
+          tc_commit_pair(&empty_bar[stage], 3);     // frees the stage in both CTAs
+          if (++stage == kW4PairStages) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        tc_commit_pair(&tfull_bar[acc], 3);
+      }
+    }
+  } else if (warp >= 6) {
+    // Scale warps: each CTA writes its own TMEM (its activation rows' scales and all of the weight tile's).
+    const int quad = warp & 3;
+    const uint32_t leader_ready[2] = {mapa_shared(smem_u32(&sf_ready[0]), 0), mapa_shared(smem_u32(&sf_ready[1]), 0)};
+    int stage = 0; uint32_t phase = 0;
+    int n = 0;
+    bool ok = true;
+    for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
+      for (int ks = 0; ks < p.kstages; ++ks, ++n) {
+        const int set = n & 1;
+        ok = wait_bounded(&sf_full[stage], phase, abort, p.status);
+        if (!ok) break;
+        if (n >= 2) {                        // the MMAs that read this set two stages ago are done
+          ok = wait_bounded(&sf_free[set], ((n >> 1) - 1) & 1, abort, p.status);
+          if (!ok) break;
+          tc_fence_after();
+        }
+        const uint4* sf = reinterpret_cast<const uint4*>(smem + stage * kStageBytes + kOpBytes) + lane;
+        uint32_t v[32];
+        constexpr int kBlk[8] = {0, 1, 2, 3, 4, 6, 5, 7};     // column order: sfa1 (g0, g1), sfa2 (g0, g1), then per K group the two weight-row blocks
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint4 q = sf[kBlk[j] * 32];
+          v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
+        }
+        tmem_st32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + kSfCol + 32 * set, v);
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(leader_ready[set]);
+        if (++stage == kW4PairStages) { stage = 0; phase ^= 1; }
+      }
+    }
   } else {
     const int quad = warp & 3;
     const int r = quad * 32 + lane;
     int it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-      const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+    const uint32_t leader_tempty[2] = {mapa_shared(smem_u32(&tempty_bar[0]), 0), mapa_shared(smem_u32(&tempty_bar[1]), 0)};
+    for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++it) {
+      const int mt = 2 * (tile % m_pairs) + static_cast<int>(rank), nt = tile / m_pairs;
       const int acc = (kAcc == 2) ? (it & 1) : 0;
       const uint32_t tphase = (kAcc == 2) ? ((it >> 1) & 1) : (it & 1);
       ok = wait_bounded(&tfull_bar[acc], tphase, abort, p.status);
@@ -212,180 +535,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&tempty_bar[acc]);
-    }
-  }
-
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 1) {
-    tc_fence_after();
-    tmem_dealloc(tmem_base, kW4TmemCols);
-  }
-}
-
-// ---------------------------------------------------------------------------------------------------------------------
-// CTA-pair variant (opt-in, MSD_W4_PAIR=1): two CTAs of a cluster share one 256 x 256 tile.  Each CTA loads its own 128 activation
-// rows (both components) and HALF of the weight tile; one tcgen05.mma.cta_group::2 per K step, issued by the even CTA,
-// multiplies all 256 rows against all 256 weight rows, each CTA's accumulator (its 128 rows x 256 columns) staying in
-// its own TMEM.  Per CTA and stage 52 KB enter shared memory instead of 68 KB and four stages fit instead of three;
-// measured no faster than the single-CTA kernel (the scale copies into TMEM and the unoverlapped epilogue, not the
-// fill rate, are what idles the tensor pipe), so it is not the default.  Scale blocks come through 2-D tensor
-// maps over the blocked scale arrays (rows of 512 bytes) so that, like the operand tiles, they complete on the
-// leader's barrier.
-constexpr int kW4PairStageBytes = 2 * kW4ABytes + kW4ABytes + kW4SfBytes;      // A1, A2, half of B, scales: 53248
-constexpr int kW4PairStages = 4;
-
-__global__ void __launch_bounds__(kW4Threads, 1)
-gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
-                       const __grid_constant__ CUtensorMap tmap_bh, const __grid_constant__ CUtensorMap tmap_sfa1,
-                       const __grid_constant__ CUtensorMap tmap_sfa2, const __grid_constant__ CUtensorMap tmap_sfb,
-                       const GemmW4Params p) {
-  extern __shared__ uint8_t smem_dyn[];
-  __shared__ __align__(8) uint64_t full_bar[kW4PairStages], empty_bar[kW4PairStages], tfull_bar, tempty_bar;
-  __shared__ uint32_t tmem_base_slot;
-  __shared__ int abort_flag;
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kW4PairStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    mbar_init(&tfull_bar, 1);
-    mbar_init(&tempty_bar, 8);          // four epilogue warps in each CTA of the pair (used in the leader only)
-    abort_flag = 0;
-    mbar_init_fence();
-    tma_prefetch_desc(&tmap_a1);
-    tma_prefetch_desc(&tmap_a2);
-    tma_prefetch_desc(&tmap_bh);
-    tma_prefetch_desc(&tmap_sfa1);
-    tma_prefetch_desc(&tmap_sfa2);
-    tma_prefetch_desc(&tmap_sfb);
-  }
-  if (warp == 1) tmem_alloc_pair(&tmem_base_slot, kW4TmemCols);
-  tc_fence_before();
-  cluster_arrive_all();        // both CTAs' barriers exist before either signals the other's
-  cluster_wait_all();
-  tc_fence_after();
-  const uint32_t tmem_base = tmem_base_slot;
-  volatile int* abort = &abort_flag;
-  const int m_pairs = (p.m_tiles + 1) >> 1;
-  const int total_tiles = m_pairs * p.n_tiles;
-  const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
-
-  if (warp == 0) {
-    if (lane == 0) {
-      pdl_wait_primary();           // components and blocked scales come from the kernels launched just before
-      int stage = 0; uint32_t phase = 0;
-      bool ok = true;
-      for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
-        const int mt = 2 * (tile % m_pairs) + static_cast<int>(rank), nt = tile / m_pairs;
-        for (int ks = 0; ks < p.kstages; ++ks) {
-          ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
-          if (!ok) break;
-          // the leader's barrier counts the bytes of both CTAs
-          if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * kW4PairStageBytes);
-          const uint32_t bar = mapa_shared(smem_u32(&full_bar[stage]), 0);
-          uint8_t* dst = smem + stage * kW4PairStageBytes;
-          tma_load_2d_pair(dst, &tmap_a1, ks * 128, mt * kW4TileM, bar);
-          tma_load_2d_pair(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, bar);
-          tma_load_2d_pair(dst + 2 * kW4ABytes, &tmap_bh, ks * 128, nt * kW4TileN + static_cast<int>(rank) * 128, bar);
-          uint8_t* sf = dst + 3 * kW4ABytes;
-          tma_load_2d_pair(sf, &tmap_sfa1, 0, mt * p.sf_kgroups + 2 * ks, bar);
-          tma_load_2d_pair(sf + 1024, &tmap_sfa2, 0, mt * p.sf_kgroups + 2 * ks, bar);
-          tma_load_2d_pair(sf + 2048, &tmap_sfb, 0, (2 * nt) * p.sf_kgroups + 2 * ks, bar);
-          tma_load_2d_pair(sf + 3072, &tmap_sfb, 0, (2 * nt + 1) * p.sf_kgroups + 2 * ks, bar);
-          if (++stage == kW4PairStages) { stage = 0; phase ^= 1; }
-        }
-      }
-    }
-  } else if (warp == 1) {
-    if (lane == 0 && rank == 0) {
-      int stage = 0; uint32_t phase = 0;
-      int it = 0;
-      bool ok = true;
-      uint32_t sfpar = 0;                                    // the scale columns alternate between two sets per stage
-      for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++it) {
-        ok = wait_bounded_cluster(&tempty_bar, (it & 1) ^ 1, abort, p.status);   // both epilogues have drained their accumulators
-        if (!ok) break;
-        tc_fence_after();
-        for (int ks = 0; ks < p.kstages; ++ks) {
-          ok = wait_bounded_cluster(&full_bar[stage], phase, abort, p.status);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t base = smem_u32(smem + stage * kW4PairStageBytes);
-          const uint32_t a1 = base, a2 = base + kW4ABytes, bb = base + 2 * kW4ABytes, sf = base + 3 * kW4ABytes;
-          const uint32_t sfa1_t = tmem_base + kW4SfCol + 32 * sfpar;     // 2 k-groups x 4 columns
-          const uint32_t sfa2_t = sfa1_t + 8;
-          const uint32_t sfb_t = sfa1_t + 16;                            // 2 k-groups x 8 columns (256 weight rows)
-          sfpar ^= 1;
-          for (int g = 0; g < 2; ++g) {
-            tc_cp_32x128b_warpx4_pair(sfa1_t + 4 * g, smem_desc(sf + g * 512, 0, 128, 0));
-            tc_cp_32x128b_warpx4_pair(sfa2_t + 4 * g, smem_desc(sf + 1024 + g * 512, 0, 128, 0));
-            tc_cp_32x128b_warpx4_pair(sfb_t + 8 * g, smem_desc(sf + 2048 + g * 512, 0, 128, 0));
-            tc_cp_32x128b_warpx4_pair(sfb_t + 8 * g + 4, smem_desc(sf + 3072 + g * 512, 0, 128, 0));
-          }
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {                    // 64 elements (32 bytes) per MMA
-            const int g = kk >> 1;
-            const uint32_t sid = (kk & 1) * 2;
-            const uint32_t idesc = idesc_block_scaled(/*E2M1*/ 1, 1, 2 * kW4TileM, kW4TileN, sid, sid);
-            const uint64_t bdesc = smem_desc(bb + kk * 32, 16, 1024, kSwizzle128B);
-            mma_mxf4_pair(tmem_base, smem_desc(a1 + kk * 32, 16, 1024, kSwizzle128B), bdesc, idesc, sfa1_t + 4 * g,
-                          sfb_t + 8 * g, (ks > 0 || kk > 0) ? 1u : 0u);
-            mma_mxf4_pair(tmem_base, smem_desc(a2 + kk * 32, 16, 1024, kSwizzle128B), bdesc, idesc, sfa2_t + 4 * g,
-                          sfb_t + 8 * g, 1u);
-          }
-          tc_commit_pair(&empty_bar[stage], 3);     // frees the stage in both CTAs
-          if (++stage == kW4PairStages) { stage = 0; phase ^= 1; }
-        }
-        if (!ok) break;
-        tc_commit_pair(&tfull_bar, 3);
-      }
-    }
-  } else {
-    const int quad = warp & 3;
-    const int r = quad * 32 + lane;
-    int it = 0;
-    bool ok = true;
-    const uint32_t leader_tempty = mapa_shared(smem_u32(&tempty_bar), 0);
-    for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++it) {
-      const int mt = 2 * (tile % m_pairs) + static_cast<int>(rank), nt = tile / m_pairs;
-      ok = wait_bounded(&tfull_bar, it & 1, abort, p.status);
-      if (!ok) break;
-      tc_fence_after();
-      const int row = mt * kW4TileM + r;
-      const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
-      for (int c0 = 0; c0 < kW4TileN; c0 += 16) {
-        uint32_t v[16];
-        tmem_ld16(trow + c0, v);
-        tmem_ld_wait();
-        const int col = nt * kW4TileN + c0;
-        if (row < p.M && col < p.N) {
-          if (p.ytype == MSD_OUT_BF16) {
-            uint32_t o[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-              o[j] = *reinterpret_cast<const uint32_t*>(&h);
-            }
-            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.y) + static_cast<long long>(row) * p.N + col;
-            if (col + 16 <= p.N) {
-              reinterpret_cast<uint4*>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
-              reinterpret_cast<uint4*>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
-            } else {
-              for (int j = 0; j < 16 && col + j < p.N; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
-            }
-          } else {
-            float* dst = static_cast<float*>(p.y) + static_cast<long long>(row) * p.N + col;
-            for (int j = 0; j < 16 && col + j < p.N; ++j) dst[j] = __uint_as_float(v[j]);
-          }
-        }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(leader_tempty);
+      if (lane == 0) mbar_arrive_cluster(leader_tempty[acc]);
     }
   }
 
@@ -405,12 +555,16 @@ struct GemmW4Plan {
   size_t off_q1, off_q2, off_sfa1, off_sfa2, off_sfb, bytes;
 };
 
-// Weight rows per tile of the single-CTA kernel (the CTA-pair kernel always uses 256).
+// Weight rows per tile: 224 (two accumulators) unless MSD_W4_TILEN=256.
 static int w4_tile_n() {
   const char* e = getenv("MSD_W4_TILEN");
-  const char* pe = getenv("MSD_W4_PAIR");
-  if (pe && atoi(pe) != 0) return 256;
   return (e && atoi(e) == 256) ? 256 : 224;
+}
+
+// The CTA-pair kernel is opt-in (MSD_W4_PAIR=1): measured slower than the single-CTA kernel.
+static bool w4_use_pair(int) {
+  const char* pe = getenv("MSD_W4_PAIR");
+  return pe && atoi(pe) != 0;
 }
 
 static GemmW4Plan plan_w4(int64_t M, int64_t N, int64_t K) {
@@ -462,18 +616,11 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   uint8_t* q1 = ws + pl.off_q1;
   uint8_t* q2 = ws + pl.off_q2;
 
-  // weight scales into the blocked layout (padding entries keep the workspace's zero fill: scale 2^-127 on zero data)
-  {
-    const int64_t total = N * (K / 32);
-    const int threads = 256;
-    int64_t blocks = (total + threads - 1) / threads;
-    const int64_t cap = static_cast<int64_t>(sm_count()) * 16;
-    if (blocks > cap) blocks = cap;
-    sf_block_layout_kernel<<<static_cast<unsigned>(blocks), threads, 0, s>>>(w_e8m0, N, static_cast<int>(K / 32), pl.sf_kgroups,
-                                                                            pl.tile_n, ws + pl.off_sfb);
-    if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
-  }
-  msd_status_t st = launch_decompose_mxfp4(x_bf16, M, K, K, q1, q2, ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s);
+  // the weight scales go into the blocked layout in the same launch as the decomposition of x
+  SfRelayout rl = {};
+  rl.src = w_e8m0; rl.dst = ws + pl.off_sfb; rl.rows = N; rl.kblocks = static_cast<int>(K / 32);
+  rl.sf_kgroups = pl.sf_kgroups; rl.tile_rows = pl.tile_n; rl.row_blocks = 2 * pl.n_tiles;
+  msd_status_t st = launch_decompose_mxfp4(x_bf16, M, K, K, q1, q2, ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s, &rl);
   if (st != MSD_OK) return st;
 
   CUtensorMap tmap_a1, tmap_a2, tmap_b;
@@ -488,37 +635,45 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.kstages = pl.kstages; p.sf_kgroups = pl.sf_kgroups;
   p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
   p.y = y; p.ytype = ytype; p.status = status;
+  {
+    const char* sfe = getenv("MSD_W4_SFWARPS");
+    p.sf_warps = sfe ? atoi(sfe) : 1;
+    // Tile order.  The operand that is swept once per tile of the other one should be the one that stays in L2: the
+    // CTAs walk the weight tiles fastest when the two components of x (M x K bytes) outweigh the weights (N x K / 2).
+    const char* oe = getenv("MSD_W4_ORDER");
+    p.n_fastest = oe ? (atoi(oe) != 0) : (2 * M > N);
+  }
 
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  const char* pair_env = getenv("MSD_W4_PAIR");
-  // opt-in: measured equal to the single-CTA kernel at M = 4096 (272 vs 266 us per call), so the bound is not the
-  // shared-memory fill it halves for the weights
-  const bool pair = pair_env ? atoi(pair_env) != 0 : false;
-  if (pair) {
-    // CTA pairs: weight half-tiles of 128 rows, scale blocks as rows of 128 32-bit words (512 bytes), two per box
-    CUtensorMap tmap_bh, tmap_sfa1, tmap_sfa2, tmap_sfb;
-    const uint64_t a_blocks = static_cast<uint64_t>(pl.m_tiles) * pl.sf_kgroups, b_blocks = static_cast<uint64_t>(2 * pl.n_tiles) * pl.sf_kgroups;
-    if (!encode_tmap_2d(&tmap_bh, CU_TENSOR_MAP_DATA_TYPE_UINT8, w_fp4, kb, N, kb, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !encode_tmap_2d(&tmap_sfa1, CU_TENSOR_MAP_DATA_TYPE_UINT32, p.sfa1, 128, a_blocks, 512, 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !encode_tmap_2d(&tmap_sfa2, CU_TENSOR_MAP_DATA_TYPE_UINT32, p.sfa2, 128, a_blocks, 512, 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !encode_tmap_2d(&tmap_sfb, CU_TENSOR_MAP_DATA_TYPE_UINT32, p.sfb, 128, b_blocks, 512, 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE))
+  if (w4_use_pair(pl.m_tiles)) {
+    // CTA pairs: each CTA loads half of the weight tile's rows
+    CUtensorMap tmap_bh;
+    if (!encode_tmap_2d(&tmap_bh, CU_TENSOR_MAP_DATA_TYPE_UINT8, w_fp4, kb, N, kb, 128, static_cast<uint32_t>(pl.tile_n / 2),
+                        CU_TENSOR_MAP_SWIZZLE_128B))
       return MSD_ERR_CUDA;
-    const size_t smem_pair = static_cast<size_t>(kW4PairStages) * kW4PairStageBytes + 1024;
+    const size_t smem_pair = static_cast<size_t>(kW4PairStages) * (2 * kW4ABytes + (pl.tile_n / 2) * 128 + kW4SfBytes) + 1024;
     static bool attr_pair_done = false;
     if (!attr_pair_done) {
-      if (cudaFuncSetAttribute(gemm_w4a16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_pair)) != cudaSuccess)
+      if (cudaFuncSetAttribute(gemm_w4a16_pair_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
+          cudaFuncSetAttribute(gemm_w4a16_pair_kernel<224>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
         return MSD_ERR_CUDA;
       attr_pair_done = true;
     }
     const int pair_tiles = ((pl.m_tiles + 1) / 2) * pl.n_tiles;
     int clusters = sm_count() / 2;
     if (clusters > pair_tiles) clusters = pair_tiles;
-    if (launch_pdl_cluster(gemm_w4a16_pair_kernel, dim3(2 * clusters), dim3(kW4Threads), smem_pair, s, pdl, 2u, tmap_a1, tmap_a2,
-                           tmap_bh, tmap_sfa1, tmap_sfa2, tmap_sfb, p) != cudaSuccess)
-      return MSD_ERR_CUDA;
+    const cudaError_t pe = pl.tile_n == 256
+        ? launch_pdl_cluster(gemm_w4a16_pair_kernel<256>, dim3(2 * clusters), dim3(kW4PairThreads), smem_pair, s, pdl, 2u, tmap_a1, tmap_a2, tmap_bh, p)
+        : launch_pdl_cluster(gemm_w4a16_pair_kernel<224>, dim3(2 * clusters), dim3(kW4PairThreads), smem_pair, s, pdl, 2u, tmap_a1, tmap_a2, tmap_bh, p);
+    if (pe != cudaSuccess) return MSD_ERR_CUDA;
     return MSD_OK;
   }
-  const size_t smem_bytes = static_cast<size_t>(kW4Stages) * (2 * kW4ABytes + pl.tile_n * 128 + kW4SfBytes) + 1024;
+  CUtensorMap tmap_y;
+  const bool ybf = ytype == MSD_OUT_BF16;
+  if (!encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, static_cast<uint64_t>(N),
+                      static_cast<uint64_t>(M), static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+    return MSD_ERR_CUDA;
+  const size_t smem_bytes = static_cast<size_t>(kW4Stages) * (2 * kW4ABytes + pl.tile_n * 128 + kW4SfBytes) + 8 * kW4StoreBytes + 1024;
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(gemm_w4a16_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
@@ -527,8 +682,8 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
     attr_done = true;
   }
   const cudaError_t le = pl.tile_n == 256
-      ? launch_pdl(gemm_w4a16_kernel<256>, dim3(pl.grid), dim3(kW4Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, p)
-      : launch_pdl(gemm_w4a16_kernel<224>, dim3(pl.grid), dim3(kW4Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, p);
+      ? launch_pdl(gemm_w4a16_kernel<256>, dim3(pl.grid), dim3(kW4ThreadsSf), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p)
+      : launch_pdl(gemm_w4a16_kernel<224>, dim3(pl.grid), dim3(kW4ThreadsSf), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p);
   if (le != cudaSuccess) return MSD_ERR_CUDA;
   return MSD_OK;
 }

@@ -67,7 +67,17 @@ msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int
                                    float* alpha, float* beta, float c1, float c2, cudaStream_t stream);
 inline float scaling_c1(msd_scaling_t s) { return s == MSD_SCALING_FRACTIONAL ? 127.49f : 127.0f; }
 inline float scaling_c2(msd_scaling_t s) { return s == MSD_SCALING_FRACTIONAL ? 254.98f : 254.0f; }
+// A scale relayout that rides along with the MXFP4 decomposition kernel (extra CTAs of the same launch): row-major
+// E8M0 scales src[rows, kblocks] -> 512-byte blocks at dst, `row_blocks` = 2 x number of row tiles of `tile_rows` rows.
+struct SfRelayout {
+  const uint8_t* src;
+  uint8_t* dst;
+  int64_t rows;
+  int kblocks, sf_kgroups, tile_rows, row_blocks;
+  int blocks;          // filled in by the launcher
+};
 msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
-                                    uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream);
+                                    uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream,
+                                    const SfRelayout* relayout = nullptr);
 
 }  // namespace msd

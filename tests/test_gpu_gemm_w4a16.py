@@ -79,10 +79,15 @@ def test_full_size_sampled():
 
 @pytest.mark.parametrize("pair", ["0", "1"])
 def test_single_cta_and_cta_pair_kernels_agree(pair, monkeypatch):
-    """The opt-in CTA-pair kernel (one 256 x 256 tile per pair of CTAs) against the default one, at both sizes,
-    including a pair whose second CTA has no rows at all and an odd number of 128-row tiles."""
+    """The single-CTA kernel and the CTA-pair kernel (one 256-token tile per pair of CTAs), each forced on every shape,
+    including a pair whose second CTA has no rows at all and an odd number of 128-row tiles; both tile widths."""
     monkeypatch.setenv("MSD_W4_PAIR", pair)
     for (M, N, K) in [(64, 512, 512), (384, 264, 1024), (520, 1032, 768)]:
         c = inputs.gemm_w4_case(M, N, K, seed=7 + M)
         y = _run(c, torch.float32).cpu().numpy().astype(np.float64)
-        _close(y, oracle.gemm_w4a16(c.x, c.w_fp4, c.w_e8m0, "f64"), False)
+        ref = oracle.gemm_w4a16(c.x, c.w_fp4, c.w_e8m0, "f64")
+        _close(y, ref, False)
+        monkeypatch.setenv("MSD_W4_TILEN", "256")
+        y = _run(c, torch.float32).cpu().numpy().astype(np.float64)
+        monkeypatch.delenv("MSD_W4_TILEN")
+        _close(y, ref, False)
