@@ -115,20 +115,29 @@ __device__ void sf_relayout(const SfRelayout& j, int64_t first, int64_t step) {
   }
 }
 
-// The first `rl.blocks` CTAs do the (independent) scale relayout `rl`, the others the decomposition.
+// The first `rl.blocks` CTAs do the (independent) scale relayout `rl`, the others the decomposition, 256 consecutive
+// 32-element blocks (row-major) per CTA and round.  With `ready` != nullptr the kernel publishes its progress so that a
+// GEMM launched as its programmatic dependent can start on the first token tiles while the rest is still being
+// decomposed: ready[t] counts the finished blocks of token tile t (128 rows), ready[tiles] the finished relayout CTAs.
 __global__ void __launch_bounds__(kMxThreads)
 decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, int K, uint8_t* __restrict__ q1,
                        uint8_t* __restrict__ q2, uint8_t* __restrict__ e1, uint8_t* __restrict__ e2, int sf_kgroups,
-                       const SfRelayout rl) {
+                       const SfRelayout rl, unsigned* __restrict__ ready) {
   pdl_launch_dependents();
-  if (static_cast<int>(blockIdx.x) < rl.blocks) {
-    sf_relayout(rl, static_cast<int64_t>(blockIdx.x) * kMxThreads + threadIdx.x, static_cast<int64_t>(rl.blocks) * kMxThreads);
-    return;
-  }
   const int kblocks = K >> 5;
   const int64_t nblocks = M * kblocks;
-  for (int64_t b = static_cast<int64_t>(blockIdx.x - rl.blocks) * kMxThreads + threadIdx.x; b < nblocks;
-       b += static_cast<int64_t>(gridDim.x - rl.blocks) * kMxThreads) {
+  if (static_cast<int>(blockIdx.x) < rl.blocks) {
+    sf_relayout(rl, static_cast<int64_t>(blockIdx.x) * kMxThreads + threadIdx.x, static_cast<int64_t>(rl.blocks) * kMxThreads);
+    if (ready) {
+      __syncthreads();
+      if (threadIdx.x == 0) { __threadfence(); atomicAdd(&ready[(M + 127) >> 7], 1u); }
+    }
+    return;
+  }
+  const int64_t units = (nblocks + kMxThreads - 1) / kMxThreads;
+  for (int64_t u = blockIdx.x - rl.blocks; u < units; u += gridDim.x - rl.blocks) {
+    const int64_t b = u * kMxThreads + threadIdx.x;
+    if (b < nblocks) {
     const int64_t row = b / kblocks;
     const int kb = static_cast<int>(b - row * kblocks);
     const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx + kb * 32);
@@ -177,6 +186,17 @@ decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, i
                            : ((row >> 7) * sf_kgroups + (kb >> 2)) * 512 + (row & 31) * 16 + ((row >> 5) & 3) * 4 + (kb & 3);
     e1[so] = static_cast<uint8_t>(a + 127);
     e2[so] = static_cast<uint8_t>(bexp + 127);
+    }
+    if (ready) {
+      // 128 x kblocks is a multiple of 256 (K is a multiple of 128 here), so a round never straddles two token tiles
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        const int64_t first = u * kMxThreads;
+        const int64_t left = nblocks - first;
+        __threadfence();
+        atomicAdd(&ready[(first / kblocks) >> 7], static_cast<unsigned>(left < kMxThreads ? left : kMxThreads));
+      }
+    }
   }
 }
 
@@ -203,18 +223,23 @@ msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int
 }
 
 msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
-                                    uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream, const SfRelayout* relayout) {
+                                    uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream, SfRelayout* relayout,
+                                    unsigned* ready) {
   if (M == 0) return MSD_OK;
+  // With progress flags the grid is small enough (two CTAs per SM, one more for the relayout) to be resident at
+  // once and to leave room for the dependent GEMM's CTA beside it.
+  const int per_sm = ready ? 2 : 32, rl_per_sm = ready ? 1 : 4;
   SfRelayout rl = {};
   if (relayout) {
     rl = *relayout;
     const int64_t chunks = static_cast<int64_t>(rl.row_blocks) * rl.sf_kgroups * 32;
     const int64_t rb = (chunks + kMxThreads - 1) / kMxThreads;
-    rl.blocks = static_cast<int>(rb < 4 * sm_count() ? rb : 4 * sm_count());
+    rl.blocks = static_cast<int>(rb < rl_per_sm * sm_count() ? rb : rl_per_sm * sm_count());
+    relayout->blocks = rl.blocks;
   }
   const int64_t nblocks = M * (K >> 5);
   const int64_t want = (nblocks + kMxThreads - 1) / kMxThreads;
-  const int64_t cap = static_cast<int64_t>(sm_count()) * 32;
+  const int64_t cap = static_cast<int64_t>(sm_count()) * per_sm;
   const unsigned grid = static_cast<unsigned>(want < cap ? want : cap) + static_cast<unsigned>(rl.blocks);
   static bool carve_done = false;
   if (!carve_done) {
@@ -222,7 +247,7 @@ msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, in
     carve_done = true;
   }
   decompose_mxfp4_kernel<<<grid, kMxThreads, 0, stream>>>(static_cast<const uint16_t*>(x_bf16), ldx, M,
-                                                          static_cast<int>(K), q1, q2, e1, e2, sf_kgroups, rl);
+                                                          static_cast<int>(K), q1, q2, e1, e2, sf_kgroups, rl, ready);
   return launch_status();
 }
 

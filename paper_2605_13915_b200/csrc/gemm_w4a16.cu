@@ -42,10 +42,32 @@ struct GemmW4Params {
   const uint8_t* sfb;
   void* y;
   int ytype;
+  const unsigned* ready;        // progress of the decomposition kernel running beside this one (nullptr: it has finished):
+                                // [t] finished 32-element blocks of token tile t, [m_tiles] finished relayout CTAs
+  unsigned ready_sfb;           // value of ready[m_tiles] when the weight scales are all in place
   int n_fastest;                // tile index -> (token tile, weight tile): weight tile fastest (1) or token tile fastest (0)
   int sf_warps;                 // 1: warps 6..9 write the scales into TMEM (tcgen05.st); 0: the MMA thread copies them (tcgen05.cp)
   unsigned* status;
 };
+
+// Bounded wait for a progress counter of the kernel this one depends on (see GemmW4Params::ready); afterwards the
+// async proxy (TMA) may read what that kernel's threads wrote.
+__device__ __forceinline__ bool wait_progress(const unsigned* counter, unsigned target, volatile int* abort, unsigned* status) {
+  const long long t0 = clock64();
+  while (true) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if (v >= target) break;
+    if (*abort) return false;
+    if (clock64() - t0 > kWaitBudgetCycles) {
+      *abort = 1;
+      atomicMax(status, kStatusTimeout);
+      return false;
+    }
+  }
+  fence_proxy_async_all();
+  return true;
+}
 
 // kTN = weight rows per tile: 256 (one accumulator) or 224 (two accumulators of 224 columns + the two sets of scale
 // columns fill the 512 TMEM columns exactly, so the epilogue of a tile overlaps the MMAs of the next).
@@ -91,22 +113,31 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
     // refill to be requested is part of the pipeline's round trip.  Warp 0 requests the operand tiles, warp 10 the
     // scale blocks (their bytes may be counted before warp 0's arrival announces them: the phase cannot end without it).
     if (lane == 0) {
-      pdl_wait_primary();           // components and blocked scales come from the kernels launched just before
-      int stage = 0; uint32_t phase = 0;
+      // Components and blocked scales come from the kernel launched just before: either it has finished
+      // (griddepcontrol.wait), or it runs beside this one and says per token tile how far it is.
       bool ok = true;
-      const bool sf_smem = p.sf_warps != 2;             // otherwise warps 6..9 read the scales from global memory
+      if (!p.ready) pdl_wait_primary();
+      else ok = wait_progress(p.ready + p.m_tiles, p.ready_sfb, abort, p.status);
+      int stage = 0; uint32_t phase = 0;
+      int mt_ready = -1;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const int mt = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles, nt = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
+        if (p.ready && mt != mt_ready) {
+          const int rows = p.M - mt * kW4TileM < kW4TileM ? p.M - mt * kW4TileM : kW4TileM;
+          ok = wait_progress(p.ready + mt, static_cast<unsigned>(rows) * static_cast<unsigned>(p.K >> 5), abort, p.status);
+          if (!ok) break;
+          mt_ready = mt;
+        }
         for (int ks = 0; ks < p.kstages; ++ks) {
           ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
           if (!ok) break;
           uint8_t* dst = smem + stage * kStageBytes;
           if (warp == 0) {
-            mbar_arrive_expect_tx(&full_bar[stage], sf_smem ? kStageBytes : kStageBytes - kW4SfBytes);
+            mbar_arrive_expect_tx(&full_bar[stage], kStageBytes);
             tma_load_2d(dst, &tmap_a1, ks * 128, mt * kW4TileM, &full_bar[stage]);
             tma_load_2d(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, &full_bar[stage]);
             tma_load_2d(dst + 2 * kW4ABytes, &tmap_b, ks * 128, nt * kTN, &full_bar[stage]);
-          } else if (sf_smem) {
+          } else {
             uint8_t* sf = dst + 2 * kW4ABytes + kBBytes;
             const size_t a_off = (static_cast<size_t>(mt) * p.sf_kgroups + 2 * ks) * 512;
             bulk_load(sf, p.sfa1 + a_off, 1024, &full_bar[stage]);
@@ -186,50 +217,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
     // carries the four scales of rows l, l+32, l+64, l+96, and every 32-lane quadrant of TMEM wants the same four
     // 32-bit columns.  Each warp reads the stage's eight blocks (one 16-byte row per lane and block) and stores them as
     // 32 columns of its own quadrant.
-    if (p.sf_warps == 2) {
-      // Scales straight from global memory (L2), one stage ahead in registers: they stay out of the shared-memory
-      // pipeline, and a set of scale columns is ready before the stage's operands land.
-      const int quad = warp & 3;
-      pdl_wait_primary();           // the blocked scales come from the kernels launched just before
-      int n = 0;
-      bool ok = true;
-      uint4 q[8];
-      auto fetch = [&](int tile, int ks) {
-        const int mt = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles, nt = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
-        const size_t a_off = (static_cast<size_t>(mt) * p.sf_kgroups + 2 * ks) * 512 + lane * 16;
-        const size_t b0_off = (static_cast<size_t>(2 * nt) * p.sf_kgroups + 2 * ks) * 512 + lane * 16;
-        const size_t b1_off = b0_off + static_cast<size_t>(p.sf_kgroups) * 512;
-        q[0] = __ldg(reinterpret_cast<const uint4*>(p.sfa1 + a_off));
-        q[1] = __ldg(reinterpret_cast<const uint4*>(p.sfa1 + a_off + 512));
-        q[2] = __ldg(reinterpret_cast<const uint4*>(p.sfa2 + a_off));
-        q[3] = __ldg(reinterpret_cast<const uint4*>(p.sfa2 + a_off + 512));
-        q[4] = __ldg(reinterpret_cast<const uint4*>(p.sfb + b0_off));
-        q[5] = __ldg(reinterpret_cast<const uint4*>(p.sfb + b1_off));
-        q[6] = __ldg(reinterpret_cast<const uint4*>(p.sfb + b0_off + 512));
-        q[7] = __ldg(reinterpret_cast<const uint4*>(p.sfb + b1_off + 512));
-      };
-      if (static_cast<int>(blockIdx.x) < total_tiles) fetch(blockIdx.x, 0);
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        for (int ks = 0; ks < p.kstages; ++ks, ++n) {
-          const int set = n & 1;
-          uint32_t v[32];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) { v[4 * j] = q[j].x; v[4 * j + 1] = q[j].y; v[4 * j + 2] = q[j].z; v[4 * j + 3] = q[j].w; }
-          if (ks + 1 < p.kstages) fetch(tile, ks + 1);
-          else if (tile + static_cast<int>(gridDim.x) < total_tiles) fetch(tile + gridDim.x, 0);
-          if (n >= 2) {                        // the MMAs that read this set two stages ago are done
-            ok = wait_bounded(&sf_free[set], ((n >> 1) - 1) & 1, abort, p.status);
-            if (!ok) break;
-            tc_fence_after();
-          }
-          tmem_st32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + kSfCol + 32 * set, v);
-          tmem_st_wait();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&sf_ready[set]);
-        }
-      }
-    } else if (p.sf_warps) {
+    if (p.sf_warps) {
       const int quad = warp & 3;
       int stage = 0; uint32_t phase = 0;
       int n = 0;
@@ -283,7 +271,16 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
       tc_fence_after();
       const int row0 = mt * kW4TileM + quad * 32;
       const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * kTN;
-      for (int c0 = 0; c0 < kTN; c0 += ccols, buf ^= 1) {
+      // columns of this tile inside the matrix (a warp whose rows are all past M has nothing to store); chunks
+      // beyond them are skipped altogether, so every pass through the loop commits exactly one store group
+      const int cols_here = p.N - nt * kTN < kTN ? p.N - nt * kTN : kTN;
+      const int cend = row0 < p.M ? cols_here : 0;
+      if (cend == 0) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+      }
+      for (int c0 = 0; c0 < cend; c0 += ccols, buf ^= 1) {
         uint32_t o[16];
         if (p.ytype == MSD_OUT_BF16) {
           uint32_t v[32];
@@ -298,7 +295,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           tmem_ld16(trow + c0, o);
           tmem_ld_wait();
         }
-        if (c0 + ccols >= kTN) {                    // all of this accumulator is in registers: the MMAs may have it back
+        if (c0 + ccols >= cend) {                   // all that is needed of this accumulator is in registers: the MMAs may have it back
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&tempty_bar[acc]);
@@ -312,9 +309,8 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           *reinterpret_cast<uint4*>(srow + ((static_cast<uint32_t>(j) ^ swz) << 4)) = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
         fence_proxy_async_smem();
         __syncwarp();
-        const int col = nt * kTN + c0;
-        if (lane == 0 && row0 < p.M && col < p.N) {
-          tma_store_2d(&tmap_y, col, row0, sb);
+        if (lane == 0) {
+          tma_store_2d(&tmap_y, nt * kTN + c0, row0, sb);
           bulk_commit_group();
         }
       }
@@ -552,7 +548,7 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
 
 struct GemmW4Plan {
   int m_tiles, n_tiles, kstages, sf_kgroups, grid, tile_n;
-  size_t off_q1, off_q2, off_sfa1, off_sfa2, off_sfb, bytes;
+  size_t off_q1, off_q2, off_sfa1, off_sfa2, off_sfb, off_ready, bytes;
 };
 
 // Weight rows per tile: 224 (two accumulators) unless MSD_W4_TILEN=256.
@@ -585,6 +581,7 @@ static GemmW4Plan plan_w4(int64_t M, int64_t N, int64_t K) {
   pl.off_sfa1 = off; off = round_up(off + static_cast<size_t>(pl.m_tiles) * pl.sf_kgroups * 512, 1024);
   pl.off_sfa2 = off; off = round_up(off + static_cast<size_t>(pl.m_tiles) * pl.sf_kgroups * 512, 1024);
   pl.off_sfb = off;  off = round_up(off + static_cast<size_t>(2 * pl.n_tiles) * pl.sf_kgroups * 512, 1024);
+  pl.off_ready = off; off = round_up(off + static_cast<size_t>(pl.m_tiles + 1) * sizeof(unsigned), 1024);
   pl.bytes = off;
   return pl;
 }
@@ -616,11 +613,22 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   uint8_t* q1 = ws + pl.off_q1;
   uint8_t* q2 = ws + pl.off_q2;
 
-  // the weight scales go into the blocked layout in the same launch as the decomposition of x
+  // The weight scales go into the blocked layout in the same launch as the decomposition of x.  Opt-in
+  // (MSD_W4_OVERLAP=1, single-CTA kernel): that launch also publishes its progress per token tile (counters zeroed
+  // here) and the GEMM, its programmatic dependent, starts on the first token tiles while the others are still being
+  // decomposed.  Measured: the GEMM's CTAs do enter 5-9 us after the decomposition starts, but the decomposition,
+  // held to two CTAs per SM so that both fit, then takes 47 instead of 25 us and the GEMM beside it is slower by as
+  // much as the earlier start gains.
+  const bool use_pair = w4_use_pair(pl.m_tiles);
+  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+  const char* ove = getenv("MSD_W4_OVERLAP");
+  const bool overlap = !use_pair && pdl && ove && atoi(ove) != 0;
+  unsigned* ready = overlap ? reinterpret_cast<unsigned*>(ws + pl.off_ready) : nullptr;
+  if (ready && cudaMemsetAsync(ready, 0, static_cast<size_t>(pl.m_tiles + 1) * sizeof(unsigned), s) != cudaSuccess) return MSD_ERR_CUDA;
   SfRelayout rl = {};
   rl.src = w_e8m0; rl.dst = ws + pl.off_sfb; rl.rows = N; rl.kblocks = static_cast<int>(K / 32);
   rl.sf_kgroups = pl.sf_kgroups; rl.tile_rows = pl.tile_n; rl.row_blocks = 2 * pl.n_tiles;
-  msd_status_t st = launch_decompose_mxfp4(x_bf16, M, K, K, q1, q2, ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s, &rl);
+  msd_status_t st = launch_decompose_mxfp4(x_bf16, M, K, K, q1, q2, ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s, &rl, ready);
   if (st != MSD_OK) return st;
 
   CUtensorMap tmap_a1, tmap_a2, tmap_b;
@@ -635,17 +643,21 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.kstages = pl.kstages; p.sf_kgroups = pl.sf_kgroups;
   p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
   p.y = y; p.ytype = ytype; p.status = status;
+  p.ready = ready; p.ready_sfb = static_cast<unsigned>(rl.blocks);
   {
     const char* sfe = getenv("MSD_W4_SFWARPS");
     p.sf_warps = sfe ? atoi(sfe) : 1;
-    // Tile order.  The operand that is swept once per tile of the other one should be the one that stays in L2: the
-    // CTAs walk the weight tiles fastest when the two components of x (M x K bytes) outweigh the weights (N x K / 2).
+    // Tile order.  A wave of CTAs either shares a few weight tiles and sweeps the token tiles (token tile fastest)
+    // or the other way round; the operand that is swept should be the one that stays in L2 (40 MB assumed usable for
+    // it).  Both components of x weigh M x K bytes, the weights N x K / 2.  With the decomposition running beside
+    // the GEMM the first wave should need only the first token tiles: weight tile fastest.
     const char* oe = getenv("MSD_W4_ORDER");
-    p.n_fastest = oe ? (atoi(oe) != 0) : (2 * M > N);
+    const double l2 = 40.0 * 1024 * 1024, a_bytes = static_cast<double>(M) * K, w_bytes = static_cast<double>(N) * K / 2;
+    const bool n_fast = overlap ? true : (a_bytes <= l2 ? false : (w_bytes <= l2 ? true : a_bytes > w_bytes));
+    p.n_fastest = oe ? (atoi(oe) != 0) : n_fast;
   }
 
-  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  if (w4_use_pair(pl.m_tiles)) {
+  if (use_pair) {
     // CTA pairs: each CTA loads half of the weight tile's rows
     CUtensorMap tmap_bh;
     if (!encode_tmap_2d(&tmap_bh, CU_TENSOR_MAP_DATA_TYPE_UINT8, w_fp4, kb, N, kb, 128, static_cast<uint32_t>(pl.tile_n / 2),

@@ -74,10 +74,10 @@ struct SfRelayout {
   uint8_t* dst;
   int64_t rows;
   int kblocks, sf_kgroups, tile_rows, row_blocks;
-  int blocks;          // filled in by the launcher
+  int blocks;          // filled in by the launcher (returned through the pointer when `ready` is used)
 };
 msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
                                     uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream,
-                                    const SfRelayout* relayout = nullptr);
+                                    SfRelayout* relayout = nullptr, unsigned* ready = nullptr);
 
 }  // namespace msd

@@ -91,3 +91,13 @@ def test_single_cta_and_cta_pair_kernels_agree(pair, monkeypatch):
         y = _run(c, torch.float32).cpu().numpy().astype(np.float64)
         monkeypatch.delenv("MSD_W4_TILEN")
         _close(y, ref, False)
+
+
+def test_gemm_beside_the_decomposition(monkeypatch):
+    """Opt-in mode in which the GEMM starts while the decomposition kernel is still running and follows its per-tile
+    progress counters: same results, including a ragged last token tile and several tiles per CTA."""
+    monkeypatch.setenv("MSD_W4_OVERLAP", "1")
+    for (M, N, K) in [(1000, 4104, 1024), (130, 256, 512)]:
+        c = inputs.gemm_w4_case(M, N, K, seed=11 + M)
+        y = _run(c, torch.float32).cpu().numpy().astype(np.float64)
+        _close(y, oracle.gemm_w4a16(c.x, c.w_fp4, c.w_e8m0, "f64"), False)
