@@ -135,8 +135,11 @@ decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, i
     return;
   }
   const int64_t units = (nblocks + kMxThreads - 1) / kMxThreads;
+  // whole warps of valid blocks and word-aligned scale positions (the scale arrays are then 4-byte aligned as well)
+  const bool pack4 = (kblocks & 3) == 0 && ((reinterpret_cast<uintptr_t>(e1) | reinterpret_cast<uintptr_t>(e2)) & 3) == 0;
   for (int64_t u = blockIdx.x - rl.blocks; u < units; u += gridDim.x - rl.blocks) {
     const int64_t b = u * kMxThreads + threadIdx.x;
+    const unsigned lanes = __ballot_sync(0xffffffffu, b < nblocks);      // the lanes of this warp that have a block
     if (b < nblocks) {
     const int64_t row = b / kblocks;
     const int kb = static_cast<int>(b - row * kblocks);
@@ -147,33 +150,29 @@ decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, i
       const uint4 t = __ldg(src + i);
       w[4 * i] = t.x; w[4 * i + 1] = t.y; w[4 * i + 2] = t.z; w[4 * i + 3] = t.w;
     }
-    uint32_t mbits = 0;    // maximum of |x| as BF16 bits (monotone in the value for finite inputs)
+    uint32_t m2 = 0;       // maximum of |x| as BF16 bits (monotone in the value for finite inputs), both halves at once
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      mbits = max(mbits, w[i] & 0x7FFFu);
-      mbits = max(mbits, (w[i] >> 16) & 0x7FFFu);
-    }
-    // alpha = smallest power of two with M_b <= 4.5 alpha: M_b = m 2^e, m in [1,2) -> exponent e - 2 + (m > 1.125)
+    for (int i = 0; i < 16; ++i) m2 = __vmaxu2(m2, w[i] & 0x7FFF7FFFu);
+    const uint32_t mbits = max(m2 & 0xFFFFu, m2 >> 16);
     const int expf = static_cast<int>(mbits >> 7);
     int a = -123;
     if (expf > 0) a = max(-123, (expf - 127) - 2 + (((mbits & 0x7Fu) > 0x10u) ? 1 : 0));
     a = min(a, 127);
     const int bexp = a - 4;                                   // beta = alpha / 16
-    // x / alpha and r / beta as two exact power-of-two multiplications (each factor stays a normal number)
-    const int na = -a, nb = -bexp;
-    const float sa1 = pow2f(na / 2), sa2 = pow2f(na - na / 2);
-    const float sb1 = pow2f(nb / 2), sb2 = pow2f(nb - nb / 2);
-    const float alpha = (a >= -126) ? pow2f(a) : 0.0f;        // a >= -123 always; kept for clarity
+    // x / alpha and r / beta are exact multiplications by a power of two: a is in [-123, 126] for finite BF16 inputs
+    // (largest exponent 127, minus 2, plus at most 1), so 2^-a and 2^(4-a) are normal FP32 numbers
+    const float sa = pow2f(max(-a, -126)), sb = pow2f(-bexp);
+    const float alpha = pow2f(a);
     uint32_t o1[4] = {0, 0, 0, 0}, o2[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
       const float v0 = bf16lo(w[i]), v1 = bf16hi(w[i]);
       const __nv_fp4x2_storage_t c1 =
-          __nv_cvt_float2_to_fp4x2(make_float2((v0 * sa1) * sa2, (v1 * sa1) * sa2), __NV_E2M1, cudaRoundNearest);
+          __nv_cvt_float2_to_fp4x2(make_float2(v0 * sa, v1 * sa), __NV_E2M1, cudaRoundNearest);
       const float2 d1 = __half22float2(__half2(__nv_cvt_fp4x2_to_halfraw2(c1, __NV_E2M1)));
       const float r0 = __fmaf_rn(-alpha, d1.x, v0), r1 = __fmaf_rn(-alpha, d1.y, v1);   // exact residuals
       const __nv_fp4x2_storage_t c2 =
-          __nv_cvt_float2_to_fp4x2(make_float2((r0 * sb1) * sb2, (r1 * sb1) * sb2), __NV_E2M1, cudaRoundNearest);
+          __nv_cvt_float2_to_fp4x2(make_float2(r0 * sb, r1 * sb), __NV_E2M1, cudaRoundNearest);
       o1[i >> 2] |= static_cast<uint32_t>(c1) << (8 * (i & 3));
       o2[i >> 2] |= static_cast<uint32_t>(c2) << (8 * (i & 3));
     }
@@ -184,8 +183,19 @@ decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, i
     const int64_t so = sf_kgroups == 0
                            ? row * kblocks + kb
                            : ((row >> 7) * sf_kgroups + (kb >> 2)) * 512 + (row & 31) * 16 + ((row >> 5) & 3) * 4 + (kb & 3);
-    e1[so] = static_cast<uint8_t>(a + 127);
-    e2[so] = static_cast<uint8_t>(bexp + 127);
+    if (pack4) {
+      // four neighbouring lanes hold the four scales of one aligned 32-bit word (kblocks is a multiple of 4)
+      uint32_t w1 = static_cast<uint32_t>(a + 127) << (8 * (threadIdx.x & 3)), w2 = static_cast<uint32_t>(bexp + 127) << (8 * (threadIdx.x & 3));
+      w1 |= __shfl_xor_sync(lanes, w1, 1); w2 |= __shfl_xor_sync(lanes, w2, 1);
+      w1 |= __shfl_xor_sync(lanes, w1, 2); w2 |= __shfl_xor_sync(lanes, w2, 2);
+      if ((threadIdx.x & 3) == 0) {
+        *reinterpret_cast<uint32_t*>(e1 + so) = w1;
+        *reinterpret_cast<uint32_t*>(e2 + so) = w2;
+      }
+    } else {
+      e1[so] = static_cast<uint8_t>(a + 127);
+      e2[so] = static_cast<uint8_t>(bexp + 127);
+    }
     }
     if (ready) {
       // 128 x kblocks is a multiple of 256 (K is a multiple of 128 here), so a round never straddles two token tiles
