@@ -7,7 +7,9 @@
 // slot of shared memory, which is the layout this MMA kind reads for 4-bit operands).
 //
 // Tile 128 activation rows x 256 weight rows, K stages of 128 elements (one 128-byte swizzle row per operand row), both
-// passes into the same FP32 accumulator.  Warps: 0 producer, 1 MMA issuer + TMEM owner, 2..5 epilogue.
+// passes into the same FP32 accumulator.  Warps as in the E2M1 kernel: 0 operand producer, 1 MMA issuer + TMEM owner,
+// 2..5 epilogue (TMA stores through swizzled staging buffers), 6..9 scale warps (shared memory -> TMEM by tcgen05.st),
+// 10 scale producer.
 #include <cuda_bf16.h>
 
 #include <cstdlib>
@@ -20,7 +22,7 @@ namespace msd {
 constexpr int kE1TileM = 128;
 constexpr int kE1TileN = 256;
 constexpr int kE1BlockK = 128;                                  // elements per stage
-constexpr int kE1Threads = 192;
+constexpr int kE1Threads = 352;
 constexpr int kE1ABytes = kE1TileM * 128;                       // 16 KB (one byte per element)
 constexpr int kE1BBytes = kE1TileN * 128;                       // 32 KB (one byte slot per 4-bit element)
 constexpr int kE1SfBytes = 512 + 512 + 1024;                    // SFA1, SFA2, SFB (two row tiles): 4 scales per row each
@@ -31,6 +33,7 @@ constexpr int kE1StageTxBytes = 2 * kE1ABytes + kE1BBytes / 2 + kE1SfBytes;
 constexpr int kE1Stages = 3;
 constexpr int kE1TmemCols = 512;
 constexpr int kE1SfCol = 256;
+constexpr int kE1StoreBytes = 2048;                             // one epilogue chunk: 32 rows x 64 bytes
 
 struct GemmE1Params {
   int M, N, K;
@@ -58,11 +61,17 @@ __device__ __forceinline__ uint32_t e1m2_as_e4m3(int k, uint32_t sign) {
 // row-major [M, K/32] (sf_kgroups == 0) or in 512-byte blocks of 128 rows x 4 scales.
 __global__ void __launch_bounds__(256)
 decompose_e1m2_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, int K, uint8_t* __restrict__ q1,
-                      uint8_t* __restrict__ q2, uint8_t* __restrict__ e1, uint8_t* __restrict__ e2, int sf_kgroups) {
+                      uint8_t* __restrict__ q2, uint8_t* __restrict__ e1, uint8_t* __restrict__ e2, int sf_kgroups,
+                      const SfRelayout rl) {
   pdl_launch_dependents();
+  if (static_cast<int>(blockIdx.x) < rl.blocks) {          // the first CTAs bring the weight scales into the blocked layout
+    sf_relayout(rl, static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x, static_cast<int64_t>(rl.blocks) * 256);
+    return;
+  }
   const int kblocks = K >> 5;
   const int64_t nblocks = M * kblocks;
-  for (int64_t b = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x; b < nblocks; b += static_cast<int64_t>(gridDim.x) * 256) {
+  for (int64_t b = static_cast<int64_t>(blockIdx.x - rl.blocks) * 256 + threadIdx.x; b < nblocks;
+       b += static_cast<int64_t>(gridDim.x - rl.blocks) * 256) {
     const int64_t row = b / kblocks;
     const int kb = static_cast<int>(b - row * kblocks);
     const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx + kb * 32);
@@ -115,18 +124,6 @@ decompose_e1m2_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, in
   }
 }
 
-// Row-major E8M0 scales [rows, K/32] -> 512-byte blocks (128 rows x 4 scales).
-__global__ void e1_sf_block_layout_kernel(const uint8_t* __restrict__ src, int64_t rows, int kblocks, int sf_kgroups,
-                                          uint8_t* __restrict__ dst) {
-  const int64_t total = rows * kblocks;
-  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
-       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
-    const int64_t row = i / kblocks;
-    const int kb = static_cast<int>(i - row * kblocks);
-    dst[((row >> 7) * sf_kgroups + (kb >> 2)) * 512 + (row & 31) * 16 + ((row >> 5) & 3) * 4 + (kb & 3)] = src[i];
-  }
-}
-
 __device__ __forceinline__ void mma_mxf8f6f4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                              uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
   asm volatile(
@@ -139,9 +136,12 @@ __device__ __forceinline__ void mma_mxf8f6f4(uint32_t d_tmem, uint64_t a_desc, u
 
 __global__ void __launch_bounds__(kE1Threads, 1)
 gemm_w4a16_e1m2_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
-                       const __grid_constant__ CUtensorMap tmap_b, const GemmE1Params p) {
+                       const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_y,
+                       const GemmE1Params p) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ __align__(8) uint64_t full_bar[kE1Stages], empty_bar[kE1Stages], tfull_bar, tempty_bar;
+  // the two sets of scale columns in TMEM: written by warps 6..9 (sf_ready), read by the MMAs of a stage (sf_free)
+  __shared__ __align__(8) uint64_t sf_ready[2], sf_free[2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
@@ -152,6 +152,7 @@ gemm_w4a16_e1m2_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
     for (int s = 0; s < kE1Stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     mbar_init(&tfull_bar, 1);
     mbar_init(&tempty_bar, 4);
+    for (int a = 0; a < 2; ++a) { mbar_init(&sf_ready[a], 4); mbar_init(&sf_free[a], 1); }
     abort_flag = 0;
     mbar_init_fence();
     tma_prefetch_desc(&tmap_a1);
@@ -166,7 +167,8 @@ gemm_w4a16_e1m2_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
   volatile int* abort = &abort_flag;
   const int total_tiles = p.m_tiles * p.n_tiles;
 
-  if (warp == 0) {
+  if (warp == 0 || warp == 10) {
+    // two producer threads (a bulk-copy instruction costs its thread 50-100 ns): warp 0 the operand tiles, warp 10 the scales
     if (lane == 0) {
       pdl_wait_primary();
       int stage = 0; uint32_t phase = 0;
@@ -176,17 +178,20 @@ gemm_w4a16_e1m2_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
         for (int ks = 0; ks < p.kstages; ++ks) {
           ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
           if (!ok) break;
-          mbar_arrive_expect_tx(&full_bar[stage], kE1StageTxBytes);
           uint8_t* dst = smem + stage * kE1StageBytes;
-          tma_load_2d(dst, &tmap_a1, ks * kE1BlockK, mt * kE1TileM, &full_bar[stage]);
-          tma_load_2d(dst + kE1ABytes, &tmap_a2, ks * kE1BlockK, mt * kE1TileM, &full_bar[stage]);
-          tma_load_2d(dst + 2 * kE1ABytes, &tmap_b, ks * kE1BlockK, nt * kE1TileN, &full_bar[stage]);   // coordinates in elements
-          uint8_t* sf = dst + 2 * kE1ABytes + kE1BBytes;
-          const size_t a_off = (static_cast<size_t>(mt) * p.sf_kgroups + ks) * 512;
-          bulk_load(sf, p.sfa1 + a_off, 512, &full_bar[stage]);
-          bulk_load(sf + 512, p.sfa2 + a_off, 512, &full_bar[stage]);
-          bulk_load(sf + 1024, p.sfb + (static_cast<size_t>(2 * nt) * p.sf_kgroups + ks) * 512, 512, &full_bar[stage]);
-          bulk_load(sf + 1536, p.sfb + (static_cast<size_t>(2 * nt + 1) * p.sf_kgroups + ks) * 512, 512, &full_bar[stage]);
+          if (warp == 0) {
+            mbar_arrive_expect_tx(&full_bar[stage], kE1StageTxBytes);
+            tma_load_2d(dst, &tmap_a1, ks * kE1BlockK, mt * kE1TileM, &full_bar[stage]);
+            tma_load_2d(dst + kE1ABytes, &tmap_a2, ks * kE1BlockK, mt * kE1TileM, &full_bar[stage]);
+            tma_load_2d(dst + 2 * kE1ABytes, &tmap_b, ks * kE1BlockK, nt * kE1TileN, &full_bar[stage]);   // coordinates in elements
+          } else {
+            uint8_t* sf = dst + 2 * kE1ABytes + kE1BBytes;
+            const size_t a_off = (static_cast<size_t>(mt) * p.sf_kgroups + ks) * 512;
+            bulk_load(sf, p.sfa1 + a_off, 512, &full_bar[stage]);
+            bulk_load(sf + 512, p.sfa2 + a_off, 512, &full_bar[stage]);
+            bulk_load(sf + 1024, p.sfb + (static_cast<size_t>(2 * nt) * p.sf_kgroups + ks) * 512, 512, &full_bar[stage]);
+            bulk_load(sf + 1536, p.sfb + (static_cast<size_t>(2 * nt + 1) * p.sf_kgroups + ks) * 512, 512, &full_bar[stage]);
+          }
           if (++stage == kE1Stages) { stage = 0; phase ^= 1; }
         }
       }
@@ -196,9 +201,8 @@ gemm_w4a16_e1m2_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
       int stage = 0; uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      uint32_t sfpar = 0;
+      int nstage = 0;                                                   // stages issued so far (all tiles)
       const uint64_t op_desc = smem_desc(0, 16, 1024, kSwizzle128B);
-      const uint64_t sf_desc = smem_desc(0, 0, 128, 0);
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
         ok = wait_bounded(&tempty_bar, (it & 1) ^ 1, abort, p.status);
         if (!ok) break;
@@ -209,21 +213,21 @@ gemm_w4a16_e1m2_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
           tc_fence_after();
           const uint64_t enc = static_cast<uint64_t>(smem_u32(smem + stage * kE1StageBytes) >> 4);
           const uint64_t a1d = op_desc + enc, a2d = a1d + (kE1ABytes >> 4), bd = a1d + (2 * kE1ABytes >> 4);
-          const uint64_t sfd = sf_desc + enc + ((2 * kE1ABytes + kE1BBytes) >> 4);
-          const uint32_t sfa1_t = tmem_base + kE1SfCol + 16 * sfpar;      // 4 columns: 4 scales (K = 128) per row
+          const int set = nstage & 1;
+          ok = wait_bounded(&sf_ready[set], (nstage >> 1) & 1, abort, p.status);      // warps 6..9 have written this stage's scales
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sfa1_t = tmem_base + kE1SfCol + 16 * set;        // 4 columns: 4 scales (K = 128) per row
           const uint32_t sfa2_t = sfa1_t + 4;
           const uint32_t sfb_t = sfa1_t + 8;                              // 8 columns: 256 weight rows
-          sfpar ^= 1;
-          tc_cp_32x128b_warpx4(sfa1_t, sfd);
-          tc_cp_32x128b_warpx4(sfa2_t, sfd + (512 >> 4));
-          tc_cp_32x128b_warpx4(sfb_t, sfd + (1024 >> 4));
-          tc_cp_32x128b_warpx4(sfb_t + 4, sfd + (1536 >> 4));
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {                    // 32 elements (32 byte slots) per MMA, scale byte kk of the column
             const uint32_t idesc = idesc_block_scaled(/*A: E4M3*/ 0, /*B: E2M1*/ 5, kE1TileM, kE1TileN, kk, kk);
             mma_mxf8f6f4(tmem_base, a1d + 2 * kk, bd + 2 * kk, idesc, sfa1_t, sfb_t, (ks > 0 || kk > 0) ? 1u : 0u);
             mma_mxf8f6f4(tmem_base, a2d + 2 * kk, bd + 2 * kk, idesc, sfa2_t, sfb_t, 1u);
           }
+          tc_commit(&sf_free[set]);                  // this set of scale columns may be rewritten once these MMAs are done
+          ++nstage;
           tc_commit(&empty_bar[stage]);
           if (++stage == kE1Stages) { stage = 0; phase ^= 1; }
         }
@@ -231,48 +235,98 @@ gemm_w4a16_e1m2_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
         tc_commit(&tfull_bar);
       }
     }
-  } else {
+  } else if (warp >= 6) {
+    // Scale warps: lane l of every 32-lane TMEM quadrant wants bytes 16 l .. 16 l + 15 of each 512-byte scale block as
+    // four 32-bit columns; the stage's four blocks (SFA1, SFA2, SFB rows 0-127, SFB rows 128-255) make one set of 16.
     const int quad = warp & 3;
-    const int r = quad * 32 + lane;
-    int it = 0;
+    int stage = 0; uint32_t phase = 0;
+    int n = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (int ks = 0; ks < p.kstages; ++ks, ++n) {
+        const int set = n & 1;
+        ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
+        if (!ok) break;
+        if (n >= 2) {                        // the MMAs that read this set two stages ago are done
+          ok = wait_bounded(&sf_free[set], ((n >> 1) - 1) & 1, abort, p.status);
+          if (!ok) break;
+          tc_fence_after();
+        }
+        const uint4* sf = reinterpret_cast<const uint4*>(smem + stage * kE1StageBytes + 2 * kE1ABytes + kE1BBytes) + lane;
+        uint32_t v[16];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint4 q = sf[j * 32];
+          v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
+        }
+        tmem_st16(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + kE1SfCol + 16 * set, v);
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sf_ready[set]);
+        if (++stage == kE1Stages) { stage = 0; phase ^= 1; }
+      }
+    }
+  } else {
+    // Epilogue: TMEM -> registers -> (BF16) -> this warp's staging buffer (64-byte-swizzled rows of 64 bytes) -> TMA
+    // store; two buffers per warp; rows past M and columns past N are clipped by the store.
+    const int quad = warp & 3;
+    uint8_t* stage_buf = smem + kE1Stages * kE1StageBytes + quad * (2 * kE1StoreBytes);
+    const int ccols = (p.ytype == MSD_OUT_BF16) ? 32 : 16;
+    const uint32_t swz = static_cast<uint32_t>((lane >> 1) & 3);
+    int it = 0, buf = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
       const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
       ok = wait_bounded(&tfull_bar, it & 1, abort, p.status);
       if (!ok) break;
       tc_fence_after();
-      const int row = mt * kE1TileM + r;
+      const int row0 = mt * kE1TileM + quad * 32;
       const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
-      for (int c0 = 0; c0 < kE1TileN; c0 += 16) {
-        uint32_t v[16];
-        tmem_ld16(trow + c0, v);
-        tmem_ld_wait();
-        const int col = nt * kE1TileN + c0;
-        if (row < p.M && col < p.N) {
-          if (p.ytype == MSD_OUT_BF16) {
-            uint32_t o[8];
+      // chunks beyond the matrix are skipped altogether, so every pass through the loop commits exactly one store group
+      const int cols_here = p.N - nt * kE1TileN < kE1TileN ? p.N - nt * kE1TileN : kE1TileN;
+      const int cend = row0 < p.M ? cols_here : 0;
+      if (cend == 0) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty_bar);
+      }
+      for (int c0 = 0; c0 < cend; c0 += ccols, buf ^= 1) {
+        uint32_t o[16];
+        if (p.ytype == MSD_OUT_BF16) {
+          uint32_t v[32];
+          tmem_ld32(trow + c0, v);
+          tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-              o[j] = *reinterpret_cast<const uint32_t*>(&h);
-            }
-            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.y) + static_cast<long long>(row) * p.N + col;
-            if (col + 16 <= p.N) {
-              reinterpret_cast<uint4*>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
-              reinterpret_cast<uint4*>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
-            } else {
-              for (int j = 0; j < 16 && col + j < p.N; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
-            }
-          } else {
-            float* dst = static_cast<float*>(p.y) + static_cast<long long>(row) * p.N + col;
-            for (int j = 0; j < 16 && col + j < p.N; ++j) dst[j] = __uint_as_float(v[j]);
+          for (int j = 0; j < 16; ++j) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+            o[j] = *reinterpret_cast<const uint32_t*>(&h);
           }
+        } else {
+          tmem_ld16(trow + c0, o);
+          tmem_ld_wait();
+        }
+        if (c0 + ccols >= cend) {                   // all that is needed of the accumulator is in registers
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tempty_bar);
+        }
+        uint8_t* sb = stage_buf + buf * kE1StoreBytes;
+        if (lane == 0) bulk_wait_group_read<1>();    // the store that read this buffer two chunks ago is done with it
+        __syncwarp();
+        uint8_t* srow = sb + lane * 64;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          *reinterpret_cast<uint4*>(srow + ((static_cast<uint32_t>(j) ^ swz) << 4)) = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_2d(&tmap_y, nt * kE1TileN + c0, row0, sb);
+          bulk_commit_group();
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&tempty_bar);
     }
+    if (lane == 0) bulk_wait_group<0>();            // every store has been written before the CTA goes away
   }
 
   tc_fence_before();
@@ -309,14 +363,22 @@ static GemmE1Plan plan_e1(int64_t M, int64_t N, int64_t K) {
 }
 
 static msd_status_t launch_decompose_e1m2(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
-                                          uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream) {
+                                          uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream,
+                                          const SfRelayout* relayout = nullptr) {
   if (M == 0) return MSD_OK;
+  SfRelayout rl = {};
+  if (relayout) {
+    rl = *relayout;
+    const int64_t chunks = static_cast<int64_t>(rl.row_blocks) * rl.sf_kgroups * 32;
+    const int64_t rb = (chunks + 255) / 256;
+    rl.blocks = static_cast<int>(rb < 4 * sm_count() ? rb : 4 * sm_count());
+  }
   const int64_t nblocks = M * (K >> 5);
   const int64_t want = (nblocks + 255) / 256;
   const int64_t cap = static_cast<int64_t>(sm_count()) * 32;
-  const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
+  const unsigned grid = static_cast<unsigned>(want < cap ? want : cap) + static_cast<unsigned>(rl.blocks);
   decompose_e1m2_kernel<<<grid, 256, 0, stream>>>(static_cast<const uint16_t*>(x_bf16), ldx, M, static_cast<int>(K), q1, q2, e1, e2,
-                                                  sf_kgroups);
+                                                  sf_kgroups, rl);
   return launch_status();
 }
 
@@ -354,16 +416,11 @@ msd_status_t msd_gemm_w4a16_e1m2(const void* x_bf16, const uint8_t* w_fp4, const
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   uint8_t* q1 = ws + pl.off_q1;
   uint8_t* q2 = ws + pl.off_q2;
-  {
-    const int64_t total = N * (K / 32);
-    int64_t blocks = (total + 255) / 256;
-    const int64_t cap = static_cast<int64_t>(sm_count()) * 16;
-    if (blocks > cap) blocks = cap;
-    e1_sf_block_layout_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(w_e8m0, N, static_cast<int>(K / 32), pl.sf_kgroups,
-                                                                           ws + pl.off_sfb);
-    if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
-  }
-  msd_status_t st = launch_decompose_e1m2(x_bf16, M, K, K, q1, q2, ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s);
+  // the weight scales go into the blocked layout (two 128-row blocks per 256-row tile) in the decomposition launch
+  SfRelayout rl = {};
+  rl.src = w_e8m0; rl.dst = ws + pl.off_sfb; rl.rows = N; rl.kblocks = static_cast<int>(K / 32);
+  rl.sf_kgroups = pl.sf_kgroups; rl.tile_rows = kE1TileN; rl.row_blocks = 2 * pl.n_tiles;
+  msd_status_t st = launch_decompose_e1m2(x_bf16, M, K, K, q1, q2, ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s, &rl);
   if (st != MSD_OK) return st;
 
   CUtensorMap tmap_a1, tmap_a2, tmap_b;
@@ -378,7 +435,12 @@ msd_status_t msd_gemm_w4a16_e1m2(const void* x_bf16, const uint8_t* w_fp4, const
   p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.kstages = pl.kstages; p.sf_kgroups = pl.sf_kgroups;
   p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
   p.y = y; p.ytype = ytype; p.status = status;
-  const size_t smem_bytes = static_cast<size_t>(kE1Stages) * kE1StageBytes + 1024;
+  CUtensorMap tmap_y;
+  const bool ybf = ytype == MSD_OUT_BF16;
+  if (!encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, static_cast<uint64_t>(N),
+                      static_cast<uint64_t>(M), static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+    return MSD_ERR_CUDA;
+  const size_t smem_bytes = static_cast<size_t>(kE1Stages) * kE1StageBytes + 8 * kE1StoreBytes + 1024;
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(gemm_w4a16_e1m2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes)) != cudaSuccess)
@@ -386,7 +448,7 @@ msd_status_t msd_gemm_w4a16_e1m2(const void* x_bf16, const uint8_t* w_fp4, const
     attr_done = true;
   }
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  if (launch_pdl(gemm_w4a16_e1m2_kernel, dim3(pl.grid), dim3(kE1Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, p) != cudaSuccess)
+  if (launch_pdl(gemm_w4a16_e1m2_kernel, dim3(pl.grid), dim3(kE1Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p) != cudaSuccess)
     return MSD_ERR_CUDA;
   return MSD_OK;
 }

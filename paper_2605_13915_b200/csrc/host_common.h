@@ -80,4 +80,31 @@ msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, in
                                     uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream,
                                     SfRelayout* relayout = nullptr, unsigned* ready = nullptr);
 
+#ifdef __CUDACC__
+// Relayout of row-major E8M0 scales [rows, kblocks] into the 512-byte blocks (128 rows x 4 scales) of the block-scaled
+// MMA.  Rows are first cut into tiles of `tile_rows` (a multiple of 32), every tile into two blocks (the second one
+// partly used when tile_rows < 256); entries outside the matrix are written as zero.  One thread per 16 bytes of
+// the result: the four scales of rows l, l+32, l+64, l+96 of one block.
+__device__ inline void sf_relayout(const SfRelayout& j, int64_t first, int64_t step) {
+  const int64_t total = static_cast<int64_t>(j.row_blocks) * j.sf_kgroups * 32;
+  for (int64_t d = first; d < total; d += step) {
+    const int l = static_cast<int>(d & 31);
+    const int64_t blk = d >> 5;
+    const int64_t tb = blk / j.sf_kgroups;
+    const int kg = static_cast<int>(blk - tb * j.sf_kgroups);
+    const int64_t t = tb >> 1;
+    uint32_t v[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int lr = static_cast<int>(tb & 1) * 128 + l + 32 * q;
+      const int64_t row = t * j.tile_rows + lr;
+      v[q] = (lr < j.tile_rows && row < j.rows && 4 * kg < j.kblocks)
+                 ? __ldg(reinterpret_cast<const uint32_t*>(j.src + row * j.kblocks + 4 * kg)) : 0u;
+    }
+    reinterpret_cast<uint4*>(j.dst)[d] = make_uint4(v[0], v[1], v[2], v[3]);
+  }
+}
+#endif
+
+
 }  // namespace msd
