@@ -29,7 +29,11 @@ constexpr int kChunk = 128;         // bytes of D / Dv per TMA box and per share
 constexpr int kChunkBytes = kTok * kChunk;
 
 struct AttnParams {
-  const uint16_t* q;      // [B,Hq,D] BF16
+  const uint16_t* q;      // [B,Hq,D] BF16 (read by attn_qstack_kernel only)
+  // written by attn_qstack_kernel, one entry per (sequence, KV head, head group): the stacked INT8 operand exactly as
+  // it lies in shared memory (DC chunks of [Rp x 128] bytes, 128-byte swizzle, unused slots zero) and alpha_Q[HG], beta_Q[HG]
+  const uint8_t* q_img;
+  const float* q_scales;
   const float* k_scale;   // [T,Hkv]
   const float* v_scale;   // [T,Hkv]
   const int32_t* cu;      // [B+1] token offsets of the sequences in a contiguous cache (unused when paged)
@@ -65,6 +69,77 @@ __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// c1 (Alg. 3 lines 1-2) once per (sequence, KV head, head group) instead of once per context split: the query rows of
+// the group's heads are decomposed into two INT8 components (same bit-exact rule as msd_decompose_int8) and written
+// as the stacked operand image the attention CTAs copy into shared memory with one bulk copy per chunk.  One CTA per
+// unit, one warp per head round robin.
+__global__ void __launch_bounds__(256)
+attn_qstack_kernel(const AttnParams p, uint8_t* __restrict__ q_img, float* __restrict__ q_scales) {
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int unit = blockIdx.x;
+  const int grp = unit % p.groups; unit /= p.groups;
+  const int hk = unit % p.Hkv;
+  const int b = unit / p.Hkv;
+  const int nh = min(p.HG, p.G - grp * p.HG);
+  const int img_bytes = p.DC * p.Rp * kChunk;
+  uint8_t* img = q_img + static_cast<size_t>(blockIdx.x) * img_bytes;
+  float* sc = q_scales + static_cast<size_t>(blockIdx.x) * 2 * p.HG;
+  // unused head slots and the padding of the last D chunk must be zero
+  for (int i = threadIdx.x; i < img_bytes / 16; i += blockDim.x) reinterpret_cast<uint4*>(img)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = threadIdx.x; i < 2 * p.HG; i += blockDim.x) sc[i] = 0.0f;
+  __syncthreads();
+  for (int h = warp; h < nh; h += 8) {
+    const int r_kv = grp * p.HG + h, sq = r_kv / p.Gr;       // row of this KV head -> (query token, head of the group)
+    const uint4* qrow = reinterpret_cast<const uint4*>(
+        p.q + ((static_cast<long long>(b) * p.Sq + sq) * (p.Hkv * p.Gr) + hk * p.Gr + (r_kv - sq * p.Gr)) * p.D);
+    const int nvec = p.D >> 3;                    // 8 BF16 values per 16-byte load (D % 16 == 0, D <= 640)
+    uint4 qv[3];                                  // the whole row stays in registers between the two passes
+    float m = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+      const int i = lane + 32 * j;
+      qv[j] = (i < nvec) ? __ldg(qrow + i) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+      const uint32_t w[4] = {qv[j].x, qv[j].y, qv[j].z, qv[j].w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        m = fmaxf(m, fabsf(__uint_as_float(w[k] << 16)));
+        m = fmaxf(m, fabsf(__uint_as_float(w[k] & 0xFFFF0000u)));
+      }
+    }
+    m = warp_max(m);
+    const float alpha = __fdiv_rn(m, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
+    const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f, inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
+    if (lane == 0) { sc[h] = alpha; sc[p.HG + h] = beta; }
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+      const int i = lane + 32 * j;
+      if (i >= nvec) continue;
+      const uint32_t w[4] = {qv[j].x, qv[j].y, qv[j].z, qv[j].w};
+      uint32_t o1[2] = {0, 0}, o2[2] = {0, 0};
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float x = (e & 1) ? __uint_as_float(w[e >> 1] & 0xFFFF0000u) : __uint_as_float(w[e >> 1] << 16);
+        int c1 = 0, c2 = 0;
+        if (alpha > 0.0f) {
+          c1 = quant_i8(x, alpha, inv_alpha);
+          const float r = __fmaf_rn(-alpha, static_cast<float>(c1), x);
+          if (beta > 0.0f) c2 = quant_i8(r, beta, inv_beta);
+        }
+        o1[e >> 2] |= static_cast<uint32_t>(c1 & 0xFF) << (8 * (e & 3));
+        o2[e >> 2] |= static_cast<uint32_t>(c2 & 0xFF) << (8 * (e & 3));
+      }
+      const int d = i << 3;                       // eight consecutive bytes stay inside one 16-byte swizzle chunk
+      uint8_t* chunk = img + (d >> 7) * p.Rp * kChunk;
+      *reinterpret_cast<uint2*>(chunk + swz_off(h, d & 127)) = make_uint2(o1[0], o1[1]);
+      *reinterpret_cast<uint2*>(chunk + swz_off(p.HG + h, d & 127)) = make_uint2(o2[0], o2[1]);
+    }
+  }
 }
 
 // kMaxHG: head slots one softmax thread looks after (8 or 16); kNH: heads its code is unrolled for (<= kMaxHG);
@@ -132,7 +207,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1);
     // one P barrier per P buffer: the softmax may run one tile ahead of the PV issue, and a single barrier could then
     // be two phases past the one the MMA warp is testing, which a parity test cannot tell from "not yet"
-    mbar_init(&p_full[0], kNSW); mbar_init(&p_full[1], kNSW); mbar_init(&q_ready, kNSW);
+    mbar_init(&p_full[0], kNSW); mbar_init(&p_full[1], kNSW); mbar_init(&q_ready, 1);
     mbar_init(&o_full, 1); mbar_init(&o_empty, kNSW);
     abort_flag = 0;
     mbar_init_fence();
@@ -140,8 +215,6 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     tma_prefetch_desc(&tmap_v);
   }
   if (warp == 1) tmem_alloc(&tmem_base_slot, p.tmem_cols);
-  // zero the stacked Q operand (unused head slots and the padding of the last D chunk must be zero)
-  for (int i = threadIdx.x; i < p.DC * p.Rp * kChunk / 16; i += blockDim.x) reinterpret_cast<uint4*>(sm_q)[i] = make_uint4(0, 0, 0, 0);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -218,7 +291,15 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       const uint32_t idesc_qk = idesc_dense(2, 1, 1, 0, 0, kTok, p.Rp);     // S8 x S8 -> S32, both K-major
       const uint32_t idesc_pv = idesc_dense(2, 1, 1, 1, 0, kTok, p.Rp);     // A (V^T) MN-major
       bool ok = true;
-      // the stacked Q operand is written by the softmax warps; they arrive on p_full once before the first tile
+      // the stacked Q operand of this (sequence, KV head, head group) comes ready-made from attn_qstack_kernel, the
+      // kernel launched just before this one (the producer's KV loads, which do not depend on it, are already under way)
+      pdl_wait_primary();
+      {
+        const int unit_q = blockIdx.y, chunk_bytes = p.Rp * kChunk;
+        mbar_arrive_expect_tx(&q_ready, p.DC * chunk_bytes);
+        for (int c = 0; c < p.DC; ++c)
+          bulk_load(sm_q + c * chunk_bytes, p.q_img + (static_cast<size_t>(unit_q) * p.DC + c) * chunk_bytes, chunk_bytes, &q_ready);
+      }
       ok = wait_bounded(&q_ready, 0, abort, p.status);
       // Operand descriptors differ from three templates only in the 16-byte-granular address field (bits 0-13), so each
       // costs one 64-bit add: with 36 MMAs per MLA tile this thread's instruction count is on the critical path.
@@ -300,59 +381,13 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const int hh = wi >> 2;                         // which group of head slots this warp looks after
     const int wq = wi & 3;
     const int hs0 = hh * kMaxHG;                    // its first head slot
-    // c1: decompose the query rows of this CTA's heads (one warp per head, round robin) into the stacked operand
-    for (int h = wi; h < nh; h += kNSW) {
-      const int r_kv = grp * p.HG + h, sq = r_kv / p.Gr;       // row of this KV head -> (query token, head of the group)
-      const uint4* qrow = reinterpret_cast<const uint4*>(
-          p.q + ((static_cast<long long>(b) * p.Sq + sq) * (p.Hkv * p.Gr) + hk * p.Gr + (r_kv - sq * p.Gr)) * p.D);
-      const int nvec = p.D >> 3;                    // 8 BF16 values per 16-byte load (D % 16 == 0, D <= 640)
-      uint4 qv[3];                                  // the whole row stays in registers between the two passes
-      float m = 0.0f;
-#pragma unroll
-      for (int j = 0; j < 3; ++j) {
-        const int i = lane + 32 * j;
-        qv[j] = (i < nvec) ? __ldg(qrow + i) : make_uint4(0, 0, 0, 0);
-      }
-#pragma unroll
-      for (int j = 0; j < 3; ++j) {
-        const uint32_t w[4] = {qv[j].x, qv[j].y, qv[j].z, qv[j].w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          m = fmaxf(m, fabsf(__uint_as_float(w[k] << 16)));
-          m = fmaxf(m, fabsf(__uint_as_float(w[k] & 0xFFFF0000u)));
-        }
-      }
-      m = warp_max(m);
-      const float alpha = __fdiv_rn(m, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
-      const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f, inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
-      if (lane == 0) { s_aq[h] = alpha; s_bq[h] = beta; }
-#pragma unroll
-      for (int j = 0; j < 3; ++j) {
-        const int i = lane + 32 * j;
-        if (i >= nvec) continue;
-        const uint32_t w[4] = {qv[j].x, qv[j].y, qv[j].z, qv[j].w};
-        uint32_t o1[2] = {0, 0}, o2[2] = {0, 0};
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float x = (e & 1) ? __uint_as_float(w[e >> 1] & 0xFFFF0000u) : __uint_as_float(w[e >> 1] << 16);
-          int c1 = 0, c2 = 0;
-          if (alpha > 0.0f) {
-            c1 = quant_i8(x, alpha, inv_alpha);                       // same bit-exact rule as msd_decompose_int8
-            const float r = __fmaf_rn(-alpha, static_cast<float>(c1), x);
-            if (beta > 0.0f) c2 = quant_i8(r, beta, inv_beta);
-          }
-          o1[e >> 2] |= static_cast<uint32_t>(c1 & 0xFF) << (8 * (e & 3));
-          o2[e >> 2] |= static_cast<uint32_t>(c2 & 0xFF) << (8 * (e & 3));
-        }
-        const int d = i << 3;                       // eight consecutive bytes stay inside one 16-byte swizzle chunk
-        uint8_t* chunk = sm_q + (d >> 7) * p.Rp * kChunk;
-        *reinterpret_cast<uint2*>(chunk + swz_off(h, d & 127)) = make_uint2(o1[0], o1[1]);
-        *reinterpret_cast<uint2*>(chunk + swz_off(kSlots + h, d & 127)) = make_uint2(o2[0], o2[1]);
-      }
+    // alpha_Q / beta_Q of this CTA's heads, computed by attn_qstack_kernel (launched just before this kernel)
+    pdl_wait_primary();
+    {
+      const int i = threadIdx.x - 64;
+      const float* sc = p.q_scales + static_cast<size_t>(blockIdx.y) * 2 * p.HG;
+      if (i < kSlots) { s_aq[i] = __ldg(sc + i); s_bq[i] = __ldg(sc + p.HG + i); }
     }
-    fence_proxy_async_smem();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&q_ready);           // the stacked Q operand is in shared memory
     named_bar_sync(8, 128 * kWG);                   // s_aq / s_bq visible to all softmax warps
     if (threadIdx.x == 64) attn_mark(p, 3);
     const int bar_id = 1 + hh;                      // each group of four warps synchronises on its own
@@ -601,7 +636,7 @@ attn_combine_kernel(const float* __restrict__ partial, int n_splits, int Dv, __n
 
 struct AttnPlan {
   int HG, Rp, groups, DC, DVT, n_splits, stages, tmem_cols, v_alias, chunk;
-  size_t smem_bytes, ws_bytes, ws_partial_bytes;
+  size_t smem_bytes, ws_bytes, ws_partial_bytes, ws_qimg_bytes, ws_qscale_bytes;
 };
 
 static int attn_env_int(const char* name, int fallback) {
@@ -645,7 +680,9 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   while (cols < 2 * pl->Rp + pl->DVT * pl->Rp) cols <<= 1;
   pl->tmem_cols = cols;
   pl->ws_partial_bytes = round_up(static_cast<size_t>(B) * Hq * ns * (Dv + 2) * sizeof(float), 1024);
-  pl->ws_bytes = pl->ws_partial_bytes + round_up(static_cast<size_t>(units) * sizeof(unsigned), 1024);
+  pl->ws_qimg_bytes = round_up(static_cast<size_t>(units) * pl->DC * pl->Rp * kChunk, 1024);     // stacked Q operands
+  pl->ws_qscale_bytes = round_up(static_cast<size_t>(units) * 2 * pl->HG * sizeof(float), 1024);
+  pl->ws_bytes = pl->ws_partial_bytes + round_up(static_cast<size_t>(units) * sizeof(unsigned), 1024) + pl->ws_qimg_bytes + pl->ws_qscale_bytes;
   return pl->smem_bytes <= 227 * 1024 - 2048;
 }
 
@@ -726,6 +763,9 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
   while ((1 << p.page_shift) < p.page) ++p.page_shift;
   p.max_blocks = max_blocks;
   p.partial = static_cast<float*>(workspace);
+  uint8_t* q_img = static_cast<uint8_t*>(workspace) + (pl.ws_bytes - pl.ws_qimg_bytes - pl.ws_qscale_bytes);
+  float* q_scales = reinterpret_cast<float*>(q_img + pl.ws_qimg_bytes);
+  p.q_img = q_img; p.q_scales = q_scales;
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.Dv = Dv; p.G = Hq / Hkv;
   p.Sq = q_len; p.Gr = Hq_real / Hkv;
   p.HG = pl.HG; p.Rp = pl.Rp; p.groups = pl.groups; p.DC = pl.DC; p.DVT = pl.DVT;
@@ -772,8 +812,11 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
     }
   }
   dim3 grid(pl.n_splits, B * Hkv * pl.groups);
-  kernel<<<grid, block_threads, pl.smem_bytes, s>>>(tmap_k, tmap_v, p);
+  attn_qstack_kernel<<<B * Hkv * pl.groups, 256, 0, s>>>(p, q_img, q_scales);
   if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
+  // programmatic dependent of the Q kernel: the CTAs start their KV loads while it runs
+  if (launch_pdl(kernel, grid, dim3(block_threads), pl.smem_bytes, s, getenv("MSD_NO_PDL") == nullptr, tmap_k, tmap_v, p) != cudaSuccess)
+    return MSD_ERR_CUDA;
   attn_combine_kernel<<<B * Hq, 128, 0, s>>>(p.partial, pl.n_splits, Dv, static_cast<__nv_bfloat16*>(out_bf16), lse, q_len,
                                              Hq / (Hkv * q_len), Hkv);
   return launch_status();
