@@ -1060,8 +1060,8 @@ __global__ void dequant_w8_to_bf16_kernel(const int8_t* __restrict__ w, const fl
 }
 
 static msd_status_t check_w8_args(const void* x, const void* w, const void* ws, int64_t M, int64_t N, int64_t K,
-                                  const void* y, int ytype, const void* workspace) {
-  if (M < 1 || M > 128 || N < 1 || K < 16 || K % 16 != 0 || N > (1 << 24) || K > (1 << 24)) return MSD_ERR_BAD_SHAPE;
+                                  const void* y, int ytype, const void* workspace, int64_t max_m = 128) {
+  if (M < 1 || M > max_m || N < 1 || K < 16 || K % 16 != 0 || N > (1 << 24) || K > (1 << 24)) return MSD_ERR_BAD_SHAPE;
   if (ytype != MSD_OUT_BF16 && ytype != MSD_OUT_FP32) return MSD_ERR_UNSUPPORTED;
   if (ytype == MSD_OUT_BF16 && N % 8 != 0) return MSD_ERR_BAD_SHAPE;
   if (!x || !w || !ws || !y || !workspace) return MSD_ERR_NULL_POINTER;
@@ -1075,7 +1075,8 @@ static msd_status_t check_w8_args(const void* x, const void* w, const void* ws, 
 extern "C" {
 
 size_t msd_gemm_w8a16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
-  if (M < 1 || M > 128 || N < 1 || K < 16) return 0;
+  if (M < 1 || M > (1 << 24) || N < 1 || K < 16) return 0;
+  if (M > 128) return msd::w8_prefill_workspace_bytes(M, N, K);
   return msd::plan_w8(M, N, K).bytes;
 }
 
@@ -1090,8 +1091,14 @@ msd_status_t msd_gemm_w8a16_ex(const void* x_bf16, const int8_t* w, const float*
                                void* workspace, size_t workspace_bytes, void* stream) {
   using namespace msd;
   if (scaling != MSD_SCALING_DEFAULT && scaling != MSD_SCALING_FRACTIONAL) return MSD_ERR_UNSUPPORTED;
-  msd_status_t st = check_w8_args(x_bf16, w, w_scale, M, N, K, y, ytype, workspace);
+  msd_status_t st = check_w8_args(x_bf16, w, w_scale, M, N, K, y, ytype, workspace, 1 << 24);
   if (st != MSD_OK) return st;
+  if (M > 128) {
+    // many rows: tokens on the MMA M axis, both components against the same weight tile (gemm_w8a16_prefill.cu)
+    if (ytype == MSD_OUT_FP32 && N % 4 != 0) return MSD_ERR_BAD_SHAPE;     // the output rows are written by TMA stores
+    return w8_prefill_launch(x_bf16, w, w_scale, M, N, K, y, ytype, acc_dbg, scaling_c1(scaling), scaling_c2(scaling), workspace,
+                             workspace_bytes, static_cast<cudaStream_t>(stream));
+  }
   const GemmW8Plan pl = plan_w8(M, N, K);
   if (workspace_bytes < pl.bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
   unsigned* status = device_status_ptr();

@@ -1,0 +1,300 @@
+// W8A16 MSD linear layer for many activation rows (prefill; Alg. 1 with the two passes kept as two INT32 accumulators):
+//   y[i,n] = w_scale[n] * (alpha_i * sum_k q1[i,k] w[n,k] + beta_i * sum_k q2[i,k] w[n,k]).
+// The decode kernel puts the weight rows on the MMA M axis and streams the weights once; here the tokens are many, so
+// they sit on the M axis in tiles of 128, a tile of 256 weight rows is the N operand, and both components of the token
+// tile are multiplied against the same weight tile in shared memory (tcgen05.mma kind::i8, S8 x S8 -> S32):
+// accumulator D1 in TMEM columns [0,256), D2 in [256,512).  K stages of 128 elements (one 128-byte swizzle row per
+// operand row): 16 + 16 + 32 KB, three stages.
+//
+// Persistent CTAs, 10 warps: 0 producer (TMA), 1 MMA issuer + TMEM owner, 2..9 epilogue (warp w reads TMEM lanes
+// 32 (w % 4) .., columns 128 ((w - 2) / 4) ..: both accumulators of 32 columns at a time, combined with alpha_i,
+// beta_i and w_scale[n], through a swizzled staging buffer into a TMA store).  The 512 TMEM columns hold one
+// tile, so the epilogue of a tile does not overlap the MMAs of the next; eight warps keep it short.
+#include <cuda_bf16.h>
+
+#include <cstdlib>
+
+#include "host_common.h"
+#include "sm100.cuh"
+
+namespace msd {
+
+constexpr int kP8TileM = 128;
+constexpr int kP8TileN = 256;
+constexpr int kP8BlockK = 128;                                  // elements (= bytes) per stage and operand row
+constexpr int kP8Threads = 320;                                 // producer, MMA, eight epilogue warps
+constexpr int kP8ABytes = kP8TileM * kP8BlockK;                 // 16 KB
+constexpr int kP8BBytes = kP8TileN * kP8BlockK;                 // 32 KB
+constexpr int kP8StageBytes = 2 * kP8ABytes + kP8BBytes;        // 64 KB
+constexpr int kP8Stages = 3;
+constexpr int kP8StoreBytes = 2048;                             // one epilogue chunk: 32 rows x 64 bytes
+constexpr int kP8TmemCols = 512;
+
+struct GemmP8Params {
+  int M, N, K;
+  int m_tiles, n_tiles, kstages;
+  int n_fastest;                // tile index -> (token tile, weight tile): weight tile fastest (1) or token tile fastest (0)
+  const float* alpha;           // [M]
+  const float* beta;            // [M]
+  const float* w_scale;         // [N]
+  int32_t* acc_dbg;             // nullable [2, M, N]
+  int ytype;
+  unsigned* status;
+};
+
+__global__ void __launch_bounds__(kP8Threads, 1)
+gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
+                          const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_y,
+                          const GemmP8Params p) {
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ __align__(8) uint64_t full_bar[kP8Stages], empty_bar[kP8Stages], tfull_bar, tempty_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kP8Stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    mbar_init(&tfull_bar, 1);
+    mbar_init(&tempty_bar, 8);
+    abort_flag = 0;
+    mbar_init_fence();
+    tma_prefetch_desc(&tmap_a1);
+    tma_prefetch_desc(&tmap_a2);
+    tma_prefetch_desc(&tmap_b);
+    tma_prefetch_desc(&tmap_y);
+  }
+  if (warp == 1) tmem_alloc(&tmem_base_slot, kP8TmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  volatile int* abort = &abort_flag;
+  const int total_tiles = p.m_tiles * p.n_tiles;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      pdl_wait_primary();           // the components and their scales come from the kernel launched just before
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int mt = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles, nt = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
+        for (int ks = 0; ks < p.kstages; ++ks) {
+          ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
+          if (!ok) break;
+          uint8_t* dst = smem + stage * kP8StageBytes;
+          mbar_arrive_expect_tx(&full_bar[stage], kP8StageBytes);
+          tma_load_2d(dst, &tmap_a1, ks * kP8BlockK, mt * kP8TileM, &full_bar[stage]);
+          tma_load_2d(dst + kP8ABytes, &tmap_a2, ks * kP8BlockK, mt * kP8TileM, &full_bar[stage]);
+          tma_load_2d(dst + 2 * kP8ABytes, &tmap_b, ks * kP8BlockK, nt * kP8TileN, &full_bar[stage]);
+          if (++stage == kP8Stages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      const uint64_t op_desc = smem_desc(0, 16, 1024, kSwizzle128B);    // 128-byte-swizzled K-major operand tile
+      const uint32_t idesc = idesc_dense(/*D=S32*/ 2, /*A=S8*/ 1, /*B=S8*/ 1, 0, 0, kP8TileM, kP8TileN);
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+        ok = wait_bounded(&tempty_bar, (it & 1) ^ 1, abort, p.status);        // the epilogue has drained both accumulators
+        if (!ok) break;
+        tc_fence_after();
+        for (int ks = 0; ks < p.kstages; ++ks) {
+          ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t enc = static_cast<uint64_t>(smem_u32(smem + stage * kP8StageBytes) >> 4);
+          const uint64_t a1d = op_desc + enc, a2d = a1d + (kP8ABytes >> 4), bd = a1d + (2 * kP8ABytes >> 4);
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {                    // 32 elements (32 bytes) per MMA
+            const uint32_t acc = (ks > 0 || kk > 0) ? 1u : 0u;
+            mma_i8(tmem_base, a1d + 2 * kk, bd + 2 * kk, idesc, acc);
+            mma_i8(tmem_base + kP8TileN, a2d + 2 * kk, bd + 2 * kk, idesc, acc);
+          }
+          tc_commit(&empty_bar[stage]);
+          if (++stage == kP8Stages) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        tc_commit(&tfull_bar);
+      }
+    }
+  } else if (warp < 10) {
+    // Epilogue (a5): a chunk is 64 bytes of every row of the warp's 32 rows (32 BF16 or 16 FP32 columns), staged in the
+    // 64-byte-swizzled layout of the output tensor map and written by a TMA store (two buffers per warp); rows past M
+    // and columns past N are clipped by the store.
+    const int quad = warp & 3, half = (warp - 2) >> 2;
+    uint8_t* stage_buf = smem + kP8Stages * kP8StageBytes + (warp - 2) * (2 * kP8StoreBytes);
+    const int ccols = (p.ytype == MSD_OUT_BF16) ? 32 : 16;
+    const uint32_t swz = static_cast<uint32_t>((lane >> 1) & 3);
+    int it = 0, buf = 0;
+    bool ok = true;
+    pdl_wait_primary();             // alpha and beta come from the decomposition kernel launched just before
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+      const int mt = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles, nt = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
+      const int row0 = mt * kP8TileM + quad * 32, row = row0 + lane;
+      const float a_i = row < p.M ? __ldg(p.alpha + row) : 0.0f, b_i = row < p.M ? __ldg(p.beta + row) : 0.0f;
+      ok = wait_bounded(&tfull_bar, it & 1, abort, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + half * 128;
+      // this warp's columns of the tile that lie inside the matrix; chunks beyond them are skipped altogether, so every
+      // pass through the loop commits exactly one store group
+      const int col_base = nt * kP8TileN + half * 128;
+      const int cols_here = p.N - col_base < 128 ? p.N - col_base : 128;
+      const int cend = row0 < p.M ? (cols_here > 0 ? cols_here : 0) : 0;
+      if (cend == 0) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty_bar);
+      }
+      for (int c0 = 0; c0 < cend; c0 += ccols, buf ^= 1) {
+        uint32_t o[16];
+        const int col = col_base + c0;
+        if (p.ytype == MSD_OUT_BF16) {
+          uint32_t v1[32], v2[32];
+          tmem_ld32(trow + c0, v1);
+          tmem_ld32(trow + kP8TileN + c0, v2);
+          tmem_ld_wait();
+          if (p.acc_dbg && row < p.M) {
+            for (int j = 0; j < 32 && col + j < p.N; ++j) {
+              p.acc_dbg[static_cast<long long>(row) * p.N + col + j] = static_cast<int32_t>(v1[j]);
+              p.acc_dbg[(static_cast<long long>(p.M) + row) * p.N + col + j] = static_cast<int32_t>(v2[j]);
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            // columns past N (a multiple of 8) are clipped by the store; their scale reads stay inside the array
+            const int c = col + 2 * j < p.N ? col + 2 * j : 0;
+            const float sw0 = __ldg(p.w_scale + c), sw1 = __ldg(p.w_scale + c + 1);
+            const float y0 = sw0 * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[2 * j])), b_i * static_cast<float>(static_cast<int32_t>(v2[2 * j])));
+            const float y1 = sw1 * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[2 * j + 1])), b_i * static_cast<float>(static_cast<int32_t>(v2[2 * j + 1])));
+            const __nv_bfloat162 h = __floats2bfloat162_rn(y0, y1);
+            o[j] = *reinterpret_cast<const uint32_t*>(&h);
+          }
+        } else {
+          uint32_t v1[16], v2[16];
+          tmem_ld16(trow + c0, v1);
+          tmem_ld16(trow + kP8TileN + c0, v2);
+          tmem_ld_wait();
+          if (p.acc_dbg && row < p.M) {
+            for (int j = 0; j < 16 && col + j < p.N; ++j) {
+              p.acc_dbg[static_cast<long long>(row) * p.N + col + j] = static_cast<int32_t>(v1[j]);
+              p.acc_dbg[(static_cast<long long>(p.M) + row) * p.N + col + j] = static_cast<int32_t>(v2[j]);
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float sw = __ldg(p.w_scale + (col + j < p.N ? col + j : 0));
+            o[j] = __float_as_uint(sw * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[j])), b_i * static_cast<float>(static_cast<int32_t>(v2[j]))));
+          }
+        }
+        if (c0 + ccols >= cend) {                   // all that is needed of the accumulators is in registers
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tempty_bar);
+        }
+        uint8_t* sb = stage_buf + buf * kP8StoreBytes;
+        if (lane == 0) bulk_wait_group_read<1>();    // the store that read this buffer two chunks ago is done with it
+        __syncwarp();
+        uint8_t* srow = sb + lane * 64;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          *reinterpret_cast<uint4*>(srow + ((static_cast<uint32_t>(j) ^ swz) << 4)) = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_2d(&tmap_y, col, row0, sb);
+          bulk_commit_group();
+        }
+      }
+    }
+    if (lane == 0) bulk_wait_group<0>();            // every store has been written before the CTA goes away
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kP8TmemCols);
+  }
+}
+
+struct GemmP8Plan {
+  int m_tiles, n_tiles, kstages, grid;
+  size_t off_q1, off_q2, off_alpha, off_beta, bytes;
+};
+
+static GemmP8Plan plan_p8(int64_t M, int64_t N, int64_t K) {
+  GemmP8Plan pl;
+  pl.m_tiles = static_cast<int>((M + kP8TileM - 1) / kP8TileM);
+  pl.n_tiles = static_cast<int>((N + kP8TileN - 1) / kP8TileN);
+  pl.kstages = static_cast<int>((K + kP8BlockK - 1) / kP8BlockK);
+  const long long tiles = static_cast<long long>(pl.m_tiles) * pl.n_tiles;
+  pl.grid = static_cast<int>(tiles < sm_count() ? tiles : sm_count());
+  size_t off = 0;
+  pl.off_q1 = off;    off = round_up(off + static_cast<size_t>(M) * K, 1024);
+  pl.off_q2 = off;    off = round_up(off + static_cast<size_t>(M) * K, 1024);
+  pl.off_alpha = off; off = round_up(off + static_cast<size_t>(M) * sizeof(float), 1024);
+  pl.off_beta = off;  off = round_up(off + static_cast<size_t>(M) * sizeof(float), 1024);
+  pl.bytes = off;
+  return pl;
+}
+
+size_t w8_prefill_workspace_bytes(int64_t M, int64_t N, int64_t K) { return plan_p8(M, N, K).bytes; }
+
+// Arguments already checked by the caller (msd_gemm_w8a16_ex); M > 128.
+msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N, int64_t K,
+                               void* y, int ytype, int32_t* acc_dbg, float c1, float c2, void* workspace,
+                               size_t workspace_bytes, cudaStream_t s) {
+  if (static_cast<long long>((M + kP8TileM - 1) / kP8TileM) * ((N + kP8TileN - 1) / kP8TileN) > 0x7FFFFFFFLL) return MSD_ERR_BAD_SHAPE;
+  const GemmP8Plan pl = plan_p8(M, N, K);
+  if (workspace_bytes < pl.bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
+  unsigned* status = device_status_ptr();
+  if (!status) return MSD_ERR_CUDA;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  int8_t* q1 = reinterpret_cast<int8_t*>(ws + pl.off_q1);
+  int8_t* q2 = reinterpret_cast<int8_t*>(ws + pl.off_q2);
+  float* alpha = reinterpret_cast<float*>(ws + pl.off_alpha);
+  float* beta = reinterpret_cast<float*>(ws + pl.off_beta);
+  msd_status_t st = launch_decompose_int8(x_bf16, M, K, K, q1, q2, alpha, beta, c1, c2, s);
+  if (st != MSD_OK) return st;
+
+  CUtensorMap tmap_a1, tmap_a2, tmap_b, tmap_y;
+  const bool ybf = ytype == MSD_OUT_BF16;
+  if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, K, M, K, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, q2, K, M, K, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kP8BlockK, kP8TileN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, static_cast<uint64_t>(N),
+                      static_cast<uint64_t>(M), static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+    return MSD_ERR_CUDA;
+
+  GemmP8Params p;
+  p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+  p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.kstages = pl.kstages;
+  p.alpha = alpha; p.beta = beta; p.w_scale = w_scale; p.acc_dbg = acc_dbg; p.ytype = ytype; p.status = status;
+  {
+    // A wave of CTAs either shares a few weight tiles and sweeps the token tiles (token tile fastest) or the other way
+    // round; the operand that is swept should be the one that stays in L2 (40 MB assumed usable for it).
+    const char* oe = getenv("MSD_P8_ORDER");
+    const double l2 = 40.0 * 1024 * 1024, a_bytes = 2.0 * static_cast<double>(M) * K, w_bytes = static_cast<double>(N) * K;
+    const bool n_fast = a_bytes <= l2 ? false : (w_bytes <= l2 ? true : a_bytes > w_bytes);
+    p.n_fastest = oe ? (atoi(oe) != 0) : n_fast;
+  }
+  const size_t smem_bytes = static_cast<size_t>(kP8Stages) * kP8StageBytes + 16 * kP8StoreBytes + 1024;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(gemm_w8a16_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes)) != cudaSuccess)
+      return MSD_ERR_CUDA;
+    attr_done = true;
+  }
+  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+  if (launch_pdl(gemm_w8a16_prefill_kernel, dim3(pl.grid), dim3(kP8Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p) != cudaSuccess)
+    return MSD_ERR_CUDA;
+  return MSD_OK;
+}
+
+}  // namespace msd

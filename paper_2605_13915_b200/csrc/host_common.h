@@ -67,6 +67,12 @@ msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int
                                    float* alpha, float* beta, float c1, float c2, cudaStream_t stream);
 inline float scaling_c1(msd_scaling_t s) { return s == MSD_SCALING_FRACTIONAL ? 127.49f : 127.0f; }
 inline float scaling_c2(msd_scaling_t s) { return s == MSD_SCALING_FRACTIONAL ? 254.98f : 254.0f; }
+// W8A16 layer for M > 128 rows (gemm_w8a16_prefill.cu); arguments checked by the caller.
+size_t w8_prefill_workspace_bytes(int64_t M, int64_t N, int64_t K);
+msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N, int64_t K,
+                               void* y, int ytype, int32_t* acc_dbg, float c1, float c2, void* workspace,
+                               size_t workspace_bytes, cudaStream_t stream);
+
 // A scale relayout that rides along with the MXFP4 decomposition kernel (extra CTAs of the same launch): row-major
 // E8M0 scales src[rows, kblocks] -> 512-byte blocks at dst, `row_blocks` = 2 x number of row tiles of `tile_rows` rows.
 struct SfRelayout {

@@ -200,3 +200,38 @@ def test_dequant_bf16_comparison_kernel(M, N, K, ctas, monkeypatch):
     msd = binding.gemm_w8a16(bf16_dev(c.x), dev(c.w), dev(c.w_scale), out_dtype=torch.float32).cpu().numpy()
     n = np.linalg.norm(truth)
     assert np.linalg.norm(msd - truth) / n <= np.linalg.norm(y.cpu().numpy() - truth) / n
+
+
+@pytest.mark.parametrize("M,N,K", [(129, 256, 128), (300, 520, 400), (1000, 264, 2048), (640, 1288, 144)])
+def test_prefill_regime_parity_fp32(M, N, K):
+    """M > 128 runs the token-major kernel (128 tokens x 256 weight rows per tile, two INT32 accumulators): ragged last
+    token tile, ragged last weight tile (also by less than a store chunk), K not a multiple of the stage, several tiles
+    per CTA; accumulators bit-exact."""
+    _check(inputs.gemm_w8_case(M, N, K, seed=5), torch.float32)
+
+
+def test_prefill_regime_parity_bf16_and_fractional_scaling():
+    c = inputs.gemm_w8_case(777, 1032, 512, seed=6)
+    _check(c, torch.bfloat16)
+    x, w, s = bf16_dev(c.x), dev(c.w), dev(c.w_scale)
+    y, acc = binding.gemm_w8a16(x, w, s, out_dtype=torch.float32, want_acc=True, fractional=True)
+    torch.cuda.synchronize()
+    binding.last_device_status()
+    ref, oacc = oracle.gemm_w8a16(c.x, c.w, c.w_scale, "f64", want_acc=True, fractional=True)
+    assert np.array_equal(acc.cpu().numpy(), oacc)
+    assert rel_row_err(y.cpu().numpy(), ref).max() <= TOL
+
+
+def test_prefill_full_size_sampled():
+    """M = 4096 on the first decode shape (N = 14336, K = 4096), BF16 out; the oracle recomputes sampled rows x columns."""
+    M, N, K = 4096, 14336, 4096
+    c = inputs.gemm_w8_case(M, N, K, seed=0)
+    y = _run(c, torch.bfloat16, want_acc=False)
+    rng = np.random.default_rng(2)
+    rows = np.unique(np.concatenate([[0, 127, 128, M - 1], rng.integers(0, M, 12)]))
+    cols = np.unique(np.concatenate([[0, 255, 256, N - 1], rng.integers(0, N, 60)]))
+    ref = oracle.gemm_w8a16(c.x[rows], c.w[cols], c.w_scale[cols], "f64")
+    got = oracle.bf16_bits_to_f64(bf16_bits(y))[np.ix_(rows, cols)]
+    slack = np.abs(ref) * 2.0 ** -8
+    n = np.linalg.norm(ref, axis=-1, keepdims=True)      # norm over the sampled columns only: smaller, so stricter
+    assert np.all(np.abs(got - ref) <= TOL * n + slack)
