@@ -6,10 +6,10 @@
 // accumulator D1 in TMEM columns [0,256), D2 in [256,512).  K stages of 128 elements (one 128-byte swizzle row per
 // operand row): 16 + 16 + 32 KB, three stages.
 //
-// Persistent CTAs, 10 warps: 0 producer (TMA), 1 MMA issuer + TMEM owner, 2..9 epilogue (warp w reads TMEM lanes
-// 32 (w % 4) .., columns 128 ((w - 2) / 4) ..: both accumulators of 32 columns at a time, combined with alpha_i,
-// beta_i and w_scale[n], through a swizzled staging buffer into a TMA store).  The 512 TMEM columns hold one
-// tile, so the epilogue of a tile does not overlap the MMAs of the next; eight warps keep it short.
+// Persistent CTAs, 18 warps: 0 producer (TMA), 1 MMA issuer + TMEM owner, 2..17 epilogue (warp w reads TMEM lanes
+// 32 (w % 4) .., columns 64 ((w - 2) / 4) .. of both accumulators, combines them with alpha_i, beta_i and w_scale[n]
+// and writes them through a swizzled staging buffer with TMA stores).  The 512 TMEM columns hold one tile, so the
+// epilogue of a tile does not overlap the MMAs of the next; sixteen warps keep it short.
 #include <cuda_bf16.h>
 
 #include <cstdlib>
@@ -22,7 +22,7 @@ namespace msd {
 constexpr int kP8TileM = 128;
 constexpr int kP8TileN = 256;
 constexpr int kP8BlockK = 128;                                  // elements (= bytes) per stage and operand row
-constexpr int kP8Threads = 320;                                 // producer, MMA, eight epilogue warps
+constexpr int kP8Threads = 576;                                 // producer, MMA, sixteen epilogue warps
 constexpr int kP8ABytes = kP8TileM * kP8BlockK;                 // 16 KB
 constexpr int kP8BBytes = kP8TileN * kP8BlockK;                 // 32 KB
 constexpr int kP8StageBytes = 2 * kP8ABytes + kP8BBytes;        // 64 KB
@@ -57,7 +57,7 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
   if (threadIdx.x == 0) {
     for (int s = 0; s < kP8Stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     mbar_init(&tfull_bar, 1);
-    mbar_init(&tempty_bar, 8);
+    mbar_init(&tempty_bar, 16);
     abort_flag = 0;
     mbar_init_fence();
     tma_prefetch_desc(&tmap_a1);
@@ -122,74 +122,82 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
         tc_commit(&tfull_bar);
       }
     }
-  } else if (warp < 10) {
-    // Epilogue (a5): a chunk is 64 bytes of every row of the warp's 32 rows (32 BF16 or 16 FP32 columns), staged in the
-    // 64-byte-swizzled layout of the output tensor map and written by a TMA store (two buffers per warp); rows past M
-    // and columns past N are clipped by the store.
-    const int quad = warp & 3, half = (warp - 2) >> 2;
-    uint8_t* stage_buf = smem + kP8Stages * kP8StageBytes + (warp - 2) * (2 * kP8StoreBytes);
+  } else {
+    // Epilogue (a5), sixteen warps: warp w reads TMEM lanes 32 (w % 4) .. and the 64 columns 64 ((w - 2) / 4) .. of both
+    // accumulators, 16 columns at a time (a TMEM load takes several hundred cycles and a thread cannot wait for one
+    // load while another is in flight, so the latency is hidden across warps: four per scheduler).  Results are staged
+    // in chunks of 64 bytes per row (32 BF16 or 16 FP32 columns) in the 64-byte-swizzled layout of the output tensor
+    // map and written by a TMA store; rows past M and columns past N are clipped by the store.
+    const int quad = warp & 3, part = (warp - 2) >> 2;
+    uint8_t* sb = smem + kP8Stages * kP8StageBytes + (warp - 2) * kP8StoreBytes;
     const int ccols = (p.ytype == MSD_OUT_BF16) ? 32 : 16;
     const uint32_t swz = static_cast<uint32_t>((lane >> 1) & 3);
-    int it = 0, buf = 0;
+    int it = 0;
     bool ok = true;
     pdl_wait_primary();             // alpha and beta come from the decomposition kernel launched just before
+    // Column scales: every lane needs the same scales of a chunk.  Lane l loads the scale of the chunk's l-th column
+    // one chunk ahead and the lanes fetch them from one another by shuffles.
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
       const int mt = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles, nt = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
       const int row0 = mt * kP8TileM + quad * 32, row = row0 + lane;
       const float a_i = row < p.M ? __ldg(p.alpha + row) : 0.0f, b_i = row < p.M ? __ldg(p.beta + row) : 0.0f;
+      const int col_base = nt * kP8TileN + part * 64;
+      const int col_w = col_base + lane;
+      float sw_next = (lane < ccols && col_w < p.N) ? __ldg(p.w_scale + col_w) : 0.0f;
       ok = wait_bounded(&tfull_bar, it & 1, abort, p.status);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + half * 128;
-      // this warp's columns of the tile that lie inside the matrix; chunks beyond them are skipped altogether, so every
-      // pass through the loop commits exactly one store group
-      const int col_base = nt * kP8TileN + half * 128;
-      const int cols_here = p.N - col_base < 128 ? p.N - col_base : 128;
+      const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + part * 64;
+      // this warp's columns of the tile that lie inside the matrix; chunks beyond them are skipped altogether
+      const int cols_here = p.N - col_base < 64 ? p.N - col_base : 64;
       const int cend = row0 < p.M ? (cols_here > 0 ? cols_here : 0) : 0;
       if (cend == 0) {
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&tempty_bar);
       }
-      for (int c0 = 0; c0 < cend; c0 += ccols, buf ^= 1) {
+      for (int c0 = 0; c0 < cend; c0 += ccols) {
         uint32_t o[16];
         const int col = col_base + c0;
-        if (p.ytype == MSD_OUT_BF16) {
-          uint32_t v1[32], v2[32];
-          tmem_ld32(trow + c0, v1);
-          tmem_ld32(trow + kP8TileN + c0, v2);
-          tmem_ld_wait();
-          if (p.acc_dbg && row < p.M) {
-            for (int j = 0; j < 32 && col + j < p.N; ++j) {
-              p.acc_dbg[static_cast<long long>(row) * p.N + col + j] = static_cast<int32_t>(v1[j]);
-              p.acc_dbg[(static_cast<long long>(p.M) + row) * p.N + col + j] = static_cast<int32_t>(v2[j]);
-            }
-          }
+        const float sw_cur = sw_next;
+        sw_next = (lane < ccols && c0 + ccols < cend && col_w + c0 + ccols < p.N) ? __ldg(p.w_scale + col_w + c0 + ccols) : 0.0f;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            // columns past N (a multiple of 8) are clipped by the store; their scale reads stay inside the array
-            const int c = col + 2 * j < p.N ? col + 2 * j : 0;
-            const float sw0 = __ldg(p.w_scale + c), sw1 = __ldg(p.w_scale + c + 1);
-            const float y0 = sw0 * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[2 * j])), b_i * static_cast<float>(static_cast<int32_t>(v2[2 * j])));
-            const float y1 = sw1 * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[2 * j + 1])), b_i * static_cast<float>(static_cast<int32_t>(v2[2 * j + 1])));
-            const __nv_bfloat162 h = __floats2bfloat162_rn(y0, y1);
-            o[j] = *reinterpret_cast<const uint32_t*>(&h);
-          }
-        } else {
+        for (int hsub = 0; hsub < 2; ++hsub) {       // 16 accumulator columns per load
+          if (hsub == 1 && p.ytype != MSD_OUT_BF16) break;
           uint32_t v1[16], v2[16];
-          tmem_ld16(trow + c0, v1);
-          tmem_ld16(trow + kP8TileN + c0, v2);
+          tmem_ld16(trow + c0 + 16 * hsub, v1);
+          tmem_ld16(trow + kP8TileN + c0 + 16 * hsub, v2);
           tmem_ld_wait();
           if (p.acc_dbg && row < p.M) {
-            for (int j = 0; j < 16 && col + j < p.N; ++j) {
-              p.acc_dbg[static_cast<long long>(row) * p.N + col + j] = static_cast<int32_t>(v1[j]);
-              p.acc_dbg[(static_cast<long long>(p.M) + row) * p.N + col + j] = static_cast<int32_t>(v2[j]);
+            for (int j = 0; j < 16 && col + 16 * hsub + j < p.N; ++j) {
+              p.acc_dbg[static_cast<long long>(row) * p.N + col + 16 * hsub + j] = static_cast<int32_t>(v1[j]);
+              p.acc_dbg[(static_cast<long long>(p.M) + row) * p.N + col + 16 * hsub + j] = static_cast<int32_t>(v2[j]);
             }
           }
+          if (p.ytype == MSD_OUT_BF16) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const float sw = __ldg(p.w_scale + (col + j < p.N ? col + j : 0));
-            o[j] = __float_as_uint(sw * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[j])), b_i * static_cast<float>(static_cast<int32_t>(v2[j]))));
+            for (int j = 0; j < 4; ++j) {
+              const int cj = 16 * hsub + 4 * j;
+              const float sx = __shfl_sync(0xffffffffu, sw_cur, cj), sy = __shfl_sync(0xffffffffu, sw_cur, cj + 1);
+              const float sz = __shfl_sync(0xffffffffu, sw_cur, cj + 2), sw_ = __shfl_sync(0xffffffffu, sw_cur, cj + 3);
+              const float y0 = sx * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[4 * j])), b_i * static_cast<float>(static_cast<int32_t>(v2[4 * j])));
+              const float y1 = sy * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[4 * j + 1])), b_i * static_cast<float>(static_cast<int32_t>(v2[4 * j + 1])));
+              const float y2 = sz * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[4 * j + 2])), b_i * static_cast<float>(static_cast<int32_t>(v2[4 * j + 2])));
+              const float y3 = sw_ * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[4 * j + 3])), b_i * static_cast<float>(static_cast<int32_t>(v2[4 * j + 3])));
+              const __nv_bfloat162 h0 = __floats2bfloat162_rn(y0, y1), h1 = __floats2bfloat162_rn(y2, y3);
+              o[8 * hsub + 2 * j] = *reinterpret_cast<const uint32_t*>(&h0);
+              o[8 * hsub + 2 * j + 1] = *reinterpret_cast<const uint32_t*>(&h1);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float sx = __shfl_sync(0xffffffffu, sw_cur, 4 * j), sy = __shfl_sync(0xffffffffu, sw_cur, 4 * j + 1);
+              const float sz = __shfl_sync(0xffffffffu, sw_cur, 4 * j + 2), sw_ = __shfl_sync(0xffffffffu, sw_cur, 4 * j + 3);
+              o[4 * j] = __float_as_uint(sx * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[4 * j])), b_i * static_cast<float>(static_cast<int32_t>(v2[4 * j]))));
+              o[4 * j + 1] = __float_as_uint(sy * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[4 * j + 1])), b_i * static_cast<float>(static_cast<int32_t>(v2[4 * j + 1]))));
+              o[4 * j + 2] = __float_as_uint(sz * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[4 * j + 2])), b_i * static_cast<float>(static_cast<int32_t>(v2[4 * j + 2]))));
+              o[4 * j + 3] = __float_as_uint(sw_ * __fmaf_rn(a_i, static_cast<float>(static_cast<int32_t>(v1[4 * j + 3])), b_i * static_cast<float>(static_cast<int32_t>(v2[4 * j + 3]))));
+            }
           }
         }
         if (c0 + ccols >= cend) {                   // all that is needed of the accumulators is in registers
@@ -197,8 +205,7 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
           __syncwarp();
           if (lane == 0) mbar_arrive(&tempty_bar);
         }
-        uint8_t* sb = stage_buf + buf * kP8StoreBytes;
-        if (lane == 0) bulk_wait_group_read<1>();    // the store that read this buffer two chunks ago is done with it
+        if (lane == 0) bulk_wait_group_read<0>();    // the store of the previous chunk is done with the staging buffer
         __syncwarp();
         uint8_t* srow = sb + lane * 64;
 #pragma unroll
