@@ -376,6 +376,20 @@ def other_configs(torch, binding, device, capture, timed):
         "frac_of_4x_measured_bf16": round(pf * 1e3 / (4 * peaks["bf16_tflops"]), 3), "frac_of_nominal_9pf": round(pf / 9.0, 3)}
     del x, w4, e4, y, wsp
 
+    # INT8 tensor-peak point: the W8A16 layer at M = 4096 on the first sweep shape (no BASELINE config exercises INT8 prefill)
+    M, N, K = 4096, 14336, 4096
+    x = torch.randn((M, K), generator=g, device=device).to(torch.bfloat16)
+    w8 = torch.randint(-127, 128, (N, K), generator=g, dtype=torch.int8, device=device)
+    s8 = torch.rand(N, generator=g, device=device) * 0.01
+    wsp = binding.workspace(binding.gemm_w8a16_workspace_bytes(M, N, K), device)
+    y = torch.empty((M, N), dtype=torch.bfloat16, device=device)
+    t = per_call_us(lambda: binding.gemm_w8a16(x, w8, s8, ws=wsp, out=y))
+    po = 4.0 * M * N * K / t / 1e9
+    res["w8a16_prefill_M4096_N14336_K4096"] = {
+        "us": round(t, 1), "executed_int8_pops": round(po, 3), "effective_pops": round(po / 2, 3),
+        "frac_of_2x_measured_bf16": round(po * 1e3 / (2 * peaks["bf16_tflops"]), 3), "frac_of_nominal_4p5": round(po / 4.5, 3)}
+    del x, w8, s8, y, wsp
+
     # grouped W8A16 GEMM (MoE experts): 32 experts of [2048, 7168], 16 routed tokens each, against one call per expert
     E, Ng, Kg, per = 32, 2048, 7168, 16
     xg = torch.randn((E * per, Kg), generator=g, device=device).to(torch.bfloat16)
