@@ -42,7 +42,9 @@ def test_argument_checks_precede_any_launch():
     assert lib.msd_decompose_int8(p, 0, 64, 64, p, p, p, p, None) == 0             # M = 0 is a no-op
     assert lib.msd_decompose_mxfp4(p, 4, 48, 48, p, p, p, p, None) == 2            # K % 32
     assert lib.msd_gemm_w8a16(p, p, p, 0, 128, 128, p, 0, None, p, 1 << 30, None) == 2       # M out of range
-    assert lib.msd_gemm_w8a16(p, p, p, 129, 128, 128, p, 0, None, p, 1 << 30, None) == 2
+    assert lib.msd_gemm_w8a16(p, p, p, (1 << 24) + 1, 128, 128, p, 0, None, p, 1 << 30, None) == 2
+    assert lib.msd_gemm_w8a16(p, p, p, 300, 130, 128, p, 1, None, p, 1 << 30, None) == 2      # FP32 rows written by TMA: N % 4
+    assert lib.msd_gemm_w8a16(p, p, p, 300, 128, 128, p, 0, None, p, 1024, None) == 5         # workspace too small
     assert lib.msd_gemm_w8a16(p, p, p, 4, 128, 128, p, 7, None, p, 1 << 30, None) == 4       # unknown output type
     assert lib.msd_gemm_w8a16(p, p, p, 4, 128, 128, p, 0, None, null, 1 << 30, None) == 1    # null workspace
     assert lib.msd_gemm_w8a16(p, p, p, 4, 128, 128, p, 0, None, C.c_void_p(4096 + 512), 1 << 30, None) == 3
