@@ -371,10 +371,25 @@ def other_configs(torch, binding, device, capture, timed):
     y = torch.empty((M, N), dtype=torch.bfloat16, device=device)
     t = per_call_us(lambda: binding.gemm_w4a16(x, w4, e4, ws=wsp, out=y))
     pf = 4.0 * M * N * K / t / 1e9
+    # comparison: the weights expanded to BF16 once per call (torch ops, several passes) and a library BF16 GEMM
+    lut = torch.tensor([0, .5, 1, 1.5, 2, 3, 4, 6, -0., -.5, -1, -1.5, -2, -3, -4, -6], dtype=torch.bfloat16, device=device)
+    wb = torch.empty((N, K), dtype=torch.bfloat16, device=device)
+
+    def w4_dequant():
+        sc = torch.exp2(e4.to(torch.float32) - 127.0).to(torch.bfloat16).repeat_interleave(32, dim=1)
+        wv = wb.view(N, K // 2, 2)
+        wv[:, :, 0] = lut[(w4 & 15).long()]
+        wv[:, :, 1] = lut[(w4 >> 4).long()]
+        wb.mul_(sc)
+    t_dq = per_call_us(w4_dequant, reps=1, steps=3)
+    t_mm = per_call_us(lambda: torch.matmul(x, wb.t(), out=y))
     res["w4a16_prefill_M4096_N8192_K8192"] = {
         "us": round(t, 1), "executed_fp4_pflops": round(pf, 3), "effective_pflops": round(pf / 2, 3),
-        "frac_of_4x_measured_bf16": round(pf * 1e3 / (4 * peaks["bf16_tflops"]), 3), "frac_of_nominal_9pf": round(pf / 9.0, 3)}
-    del x, w4, e4, y, wsp
+        "frac_of_4x_measured_bf16": round(pf * 1e3 / (4 * peaks["bf16_tflops"]), 3), "frac_of_nominal_9pf": round(pf / 9.0, 3),
+        "comparison_dequant_bf16": {"dequant_us": round(t_dq, 1), "library_bf16_gemm_us": round(t_mm, 1),
+                                    "msd_speedup_vs_gemm_alone": round(t_mm / t, 2), "msd_speedup_vs_dequant_plus_gemm": round((t_dq + t_mm) / t, 2),
+                                    "note": "dequant = torch ops (library, several passes over the weights); GEMM = torch.matmul BF16 (library)"}}
+    del x, w4, e4, y, wsp, wb, lut
 
     # INT8 tensor-peak point: the W8A16 layer at M = 4096 on the first sweep shape (no BASELINE config exercises INT8 prefill)
     M, N, K = 4096, 14336, 4096
@@ -385,10 +400,19 @@ def other_configs(torch, binding, device, capture, timed):
     y = torch.empty((M, N), dtype=torch.bfloat16, device=device)
     t = per_call_us(lambda: binding.gemm_w8a16(x, w8, s8, ws=wsp, out=y))
     po = 4.0 * M * N * K / t / 1e9
+    wb = torch.empty((N, K), dtype=torch.bfloat16, device=device)
+
+    def w8_dequant():
+        torch.mul(w8.to(torch.bfloat16), s8.to(torch.bfloat16)[:, None], out=wb)
+    t_dq = per_call_us(w8_dequant, reps=1, steps=3)
+    t_mm = per_call_us(lambda: torch.matmul(x, wb.t(), out=y))
     res["w8a16_prefill_M4096_N14336_K4096"] = {
         "us": round(t, 1), "executed_int8_pops": round(po, 3), "effective_pops": round(po / 2, 3),
-        "frac_of_2x_measured_bf16": round(po * 1e3 / (2 * peaks["bf16_tflops"]), 3), "frac_of_nominal_4p5": round(po / 4.5, 3)}
-    del x, w8, s8, y, wsp
+        "frac_of_2x_measured_bf16": round(po * 1e3 / (2 * peaks["bf16_tflops"]), 3), "frac_of_nominal_4p5": round(po / 4.5, 3),
+        "comparison_dequant_bf16": {"dequant_us": round(t_dq, 1), "library_bf16_gemm_us": round(t_mm, 1),
+                                    "msd_speedup_vs_gemm_alone": round(t_mm / t, 2), "msd_speedup_vs_dequant_plus_gemm": round((t_dq + t_mm) / t, 2),
+                                    "note": "dequant = torch ops (library); GEMM = torch.matmul BF16 (library); MSD executes twice the MACs at twice the rate"}}
+    del x, w8, s8, y, wsp, wb
 
     # grouped W8A16 GEMM (MoE experts): 32 experts of [2048, 7168], 16 routed tokens each, against one call per expert
     E, Ng, Kg, per = 32, 2048, 7168, 16
