@@ -190,6 +190,23 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
                             void* stream);
 
 /*
+ * Grouped W4A16 MSD layer for mixture-of-experts blocks (Sec. 7.2; the decomposition works per 32-element block of an
+ * activation row, so it carries over unchanged).  The rows of x are sorted by expert; expert e owns the next
+ * group_sizes[e] rows and multiplies them against its own MXFP4 weight:
+ *   y[i,:] = msd_gemm_w4a16 row result of x[i,:] with w_fp4[e], w_e8m0[e]   for the rows i of group e.
+ *   x_bf16 [M_total, K] (device), w_fp4 [E, N, K/2], w_e8m0 [E, N, K/32], y [M_total, N] (device);
+ *   group_sizes_host [E] INT32 in HOST memory, each 0..128 (decode regime per expert), M_total = their sum.
+ * Empty groups are skipped (their weights are not read).  Per 64 non-empty groups one decomposition launch (the first
+ * also brings every expert's weight scales into the blocked layout) and one GEMM launch in which group g is token tile
+ * g.  K % 128 == 0, N % 8 == 0, E * N < 2^31; x, w_fp4, y 16-byte aligned, w_e8m0 4-byte aligned.
+ * workspace: >= msd_grouped_gemm_w4a16_workspace_bytes(E, N, K), 1024-byte aligned; no initialisation needed.
+ */
+size_t msd_grouped_gemm_w4a16_workspace_bytes(int32_t E, int64_t N, int64_t K);
+msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0,
+                                    const int32_t* group_sizes_host, int32_t E, int64_t N, int64_t K, void* y,
+                                    msd_out_t ytype, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The paper-literal MXFP4 components (Sec. 3.2.1, Alg. 2; Tab. mxfp4-evolution): both passes round onto the E1M2 grid
  * {0, .25, ..., 1.75}, alpha = 2^ceil(log2(blockmax / 1.859375)) (exponent kept >= -123), beta = alpha / 16, error bound
  * alpha / 64.  Tensor cores have no E1M2 operand type; every E1M2 value is an E4M3 number, so the components are

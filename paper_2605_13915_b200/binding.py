@@ -39,6 +39,8 @@ _SIGS = {
     "msd_gemm_w8a16_ex": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_grouped_gemm_w8a16_workspace_bytes": (_sz, [_i64, _i32, _i32, _i64, _i64]),
     "msd_grouped_gemm_w8a16": (C.c_int, [_vp, _vp, _vp, _vp, _i32, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
+    "msd_grouped_gemm_w4a16_workspace_bytes": (_sz, [_i32, _i64, _i64]),
+    "msd_grouped_gemm_w4a16": (C.c_int, [_vp, _vp, _vp, _vp, _i32, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_gemm_w8a16_noalloc": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp]),
     "msd_debug_set_trace": (None, [_vp]),
     "msd_debug_set_attn_trace": (None, [_vp]),
@@ -187,6 +189,25 @@ def grouped_gemm_w8a16(x, w, w_scale, group_sizes, out_dtype=torch.bfloat16, ws=
     code = lib().msd_grouped_gemm_w8a16(_ptr(x), _ptr(w), _ptr(w_scale), C.cast(sizes, C.c_void_p), E, N, K, _ptr(y),
                                         OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream())
     _check(code, "msd_grouped_gemm_w8a16")
+    return y
+
+
+def grouped_gemm_w4a16(x, w_fp4, w_e8m0, group_sizes, out_dtype=torch.bfloat16, ws=None, out=None):
+    """MoE experts with MXFP4 weights: x [M_total,K] bf16 with rows sorted by expert, w_fp4 [E,N,K/2] u8, w_e8m0 [E,N,K/32] u8,
+    group_sizes: E host ints (rows per expert, each <= 128) -> y [M_total,N]."""
+    _need_cuda(x, w_fp4, w_e8m0)
+    E, N, K2 = w_fp4.shape
+    K = 2 * K2
+    sizes = (C.c_int32 * E)(*[int(v) for v in group_sizes])
+    M_total = int(sum(int(v) for v in group_sizes))
+    assert x.shape[0] == M_total and x.shape[1] == K
+    if ws is None:
+        ws = workspace(int(lib().msd_grouped_gemm_w4a16_workspace_bytes(E, N, K)), x.device)
+    y = out if out is not None else torch.empty((M_total, N), dtype=out_dtype, device=x.device)
+    wp, wb = _ws_ptr(ws)
+    code = lib().msd_grouped_gemm_w4a16(_ptr(x), _ptr(w_fp4), _ptr(w_e8m0), sizes, E, N, K, _ptr(y),
+                                        OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream())
+    _check(code, "msd_grouped_gemm_w4a16")
     return y
 
 

@@ -98,7 +98,7 @@ __device__ __forceinline__ float pow2f(int e) { return __uint_as_float(static_ca
 __global__ void __launch_bounds__(kMxThreads)
 decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, int K, uint8_t* __restrict__ q1,
                        uint8_t* __restrict__ q2, uint8_t* __restrict__ e1, uint8_t* __restrict__ e2, int sf_kgroups,
-                       const SfRelayout rl, unsigned* __restrict__ ready) {
+                       const SfRelayout rl, unsigned* __restrict__ ready, const RowGroups rg) {
   pdl_launch_dependents();
   const int kblocks = K >> 5;
   const int64_t nblocks = M * kblocks;
@@ -117,9 +117,15 @@ decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, i
     const int64_t b = u * kMxThreads + threadIdx.x;
     const unsigned lanes = __ballot_sync(0xffffffffu, b < nblocks);      // the lanes of this warp that have a block
     if (b < nblocks) {
-    const int64_t row = b / kblocks;
-    const int kb = static_cast<int>(b - row * kblocks);
-    const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx + kb * 32);
+    const int64_t row_in = b / kblocks;
+    const int kb = static_cast<int>(b - row_in * kblocks);
+    const uint4* src = reinterpret_cast<const uint4*>(x + row_in * ldx + kb * 32);
+    int64_t row = row_in;                   // where the row's components and scales go
+    if (rg.n > 0) {
+      int g = 0;
+      while (g + 1 < rg.n && row_in >= rg.off[g + 1]) ++g;
+      row = static_cast<int64_t>(g) * 128 + (row_in - rg.off[g]);
+    }
     uint32_t w[16];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -210,19 +216,21 @@ msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int
 
 msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
                                     uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream, SfRelayout* relayout,
-                                    unsigned* ready) {
+                                    unsigned* ready, const RowGroups* groups) {
   if (M == 0) return MSD_OK;
   // With progress flags the grid is small enough (two CTAs per SM, one more for the relayout) to be resident at
   // once and to leave room for the dependent GEMM's CTA beside it.
-  const int per_sm = ready ? 2 : 32, rl_per_sm = ready ? 1 : 4;
+  const int per_sm = ready ? 2 : 32, rl_per_sm = ready ? 1 : ((relayout && relayout->matrices > 1) ? 16 : 4);
   SfRelayout rl = {};
   if (relayout) {
     rl = *relayout;
-    const int64_t chunks = static_cast<int64_t>(rl.row_blocks) * rl.sf_kgroups * 32;
+    const int64_t chunks = static_cast<int64_t>(rl.row_blocks) * rl.sf_kgroups * 32 * (rl.matrices > 1 ? rl.matrices : 1);
     const int64_t rb = (chunks + kMxThreads - 1) / kMxThreads;
     rl.blocks = static_cast<int>(rb < rl_per_sm * sm_count() ? rb : rl_per_sm * sm_count());
     relayout->blocks = rl.blocks;
   }
+  RowGroups rg = {};
+  if (groups) rg = *groups;
   const int64_t nblocks = M * (K >> 5);
   const int64_t want = (nblocks + kMxThreads - 1) / kMxThreads;
   const int64_t cap = static_cast<int64_t>(sm_count()) * per_sm;
@@ -233,7 +241,7 @@ msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, in
     carve_done = true;
   }
   decompose_mxfp4_kernel<<<grid, kMxThreads, 0, stream>>>(static_cast<const uint16_t*>(x_bf16), ldx, M,
-                                                          static_cast<int>(K), q1, q2, e1, e2, sf_kgroups, rl, ready);
+                                                          static_cast<int>(K), q1, q2, e1, e2, sf_kgroups, rl, ready, rg);
   return launch_status();
 }
 

@@ -50,6 +50,16 @@ struct GemmW4Params {
   unsigned* status;
 };
 
+// Mixture-of-experts launch: token tile g holds the rows of group g (at most 128), which multiply the weights of expert
+// expert[g]; the rows of the result go to y rows off[g] ...
+struct GemmW4Groups {
+  int n;
+  int expert[kMaxRowGroups], off[kMaxRowGroups + 1];
+};
+struct GemmW4NoGroups {};
+template <bool kGrouped> struct W4GroupArg { using type = GemmW4NoGroups; };
+template <> struct W4GroupArg<true> { using type = GemmW4Groups; };
+
 // Bounded wait for a progress counter of the kernel this one depends on (see GemmW4Params::ready); afterwards the
 // async proxy (TMA) may read what that kernel's threads wrote.
 __device__ __forceinline__ bool wait_progress(const unsigned* counter, unsigned target, volatile int* abort, unsigned* status) {
@@ -71,11 +81,11 @@ __device__ __forceinline__ bool wait_progress(const unsigned* counter, unsigned 
 
 // kTN = weight rows per tile: 256 (one accumulator) or 224 (two accumulators of 224 columns + the two sets of scale
 // columns fill the 512 TMEM columns exactly, so the epilogue of a tile overlaps the MMAs of the next).
-template <int kTN>
+template <int kTN, bool kGrouped = false>
 __global__ void __launch_bounds__(kW4ThreadsSf, 1)
 gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
                   const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_y,
-                  const GemmW4Params p) {
+                  const GemmW4Params p, const typename W4GroupArg<kGrouped>::type grp) {
   constexpr int kBBytes = kTN * 128;
   constexpr int kStageBytes = 2 * kW4ABytes + kBBytes + kW4SfBytes;
   constexpr int kAcc = (2 * kTN + 64 <= kW4TmemCols) ? 2 : 1;       // accumulators that fit beside 2 x 32 scale columns
@@ -136,14 +146,18 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
             mbar_arrive_expect_tx(&full_bar[stage], kStageBytes);
             tma_load_2d(dst, &tmap_a1, ks * 128, mt * kW4TileM, &full_bar[stage]);
             tma_load_2d(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, &full_bar[stage]);
-            tma_load_2d(dst + 2 * kW4ABytes, &tmap_b, ks * 128, nt * kTN, &full_bar[stage]);
+            int b_row = nt * kTN;
+            if constexpr (kGrouped) b_row += grp.expert[mt] * p.N;          // the weights of the group's expert
+            tma_load_2d(dst + 2 * kW4ABytes, &tmap_b, ks * 128, b_row, &full_bar[stage]);
           } else {
             uint8_t* sf = dst + 2 * kW4ABytes + kBBytes;
             const size_t a_off = (static_cast<size_t>(mt) * p.sf_kgroups + 2 * ks) * 512;
             bulk_load(sf, p.sfa1 + a_off, 1024, &full_bar[stage]);
             bulk_load(sf + 1024, p.sfa2 + a_off, 1024, &full_bar[stage]);
-            bulk_load(sf + 2048, p.sfb + (static_cast<size_t>(2 * nt) * p.sf_kgroups + 2 * ks) * 512, 1024, &full_bar[stage]);
-            bulk_load(sf + 3072, p.sfb + (static_cast<size_t>(2 * nt + 1) * p.sf_kgroups + 2 * ks) * 512, 1024, &full_bar[stage]);
+            size_t sfb_blk = static_cast<size_t>(2 * nt);
+            if constexpr (kGrouped) sfb_blk += static_cast<size_t>(grp.expert[mt]) * 2 * p.n_tiles;
+            bulk_load(sf + 2048, p.sfb + (sfb_blk * p.sf_kgroups + 2 * ks) * 512, 1024, &full_bar[stage]);
+            bulk_load(sf + 3072, p.sfb + ((sfb_blk + 1) * p.sf_kgroups + 2 * ks) * 512, 1024, &full_bar[stage]);
           }
           if (++stage == kW4Stages) { stage = 0; phase ^= 1; }
         }
@@ -269,12 +283,17 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
       ok = wait_bounded(&tfull_bar[acc], tphase, abort, p.status);
       if (!ok) break;
       tc_fence_after();
-      const int row0 = mt * kW4TileM + quad * 32;
+      int row0 = mt * kW4TileM + quad * 32;              // first output row of this warp
+      int rows_end = p.M;                                // output rows at or past it belong to nobody (or somebody else)
+      if constexpr (kGrouped) {
+        row0 = grp.off[mt] + quad * 32;
+        rows_end = grp.off[mt + 1];
+      }
       const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * kTN;
       // columns of this tile inside the matrix (a warp whose rows are all past M has nothing to store); chunks
       // beyond them are skipped altogether, so every pass through the loop commits exactly one store group
       const int cols_here = p.N - nt * kTN < kTN ? p.N - nt * kTN : kTN;
-      const int cend = row0 < p.M ? cols_here : 0;
+      const int cend = row0 < rows_end ? cols_here : 0;
       if (cend == 0) {
         tc_fence_before();
         __syncwarp();
@@ -301,7 +320,9 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           if (lane == 0) mbar_arrive(&tempty_bar[acc]);
         }
         uint8_t* sb = stage_buf + buf * kW4StoreBytes;
-        if (lane == 0) bulk_wait_group_read<1>();    // the store that read this buffer two chunks ago is done with it
+        // the store that read this buffer two chunks ago is done with it (grouped launches may skip a commit when a
+        // group ends inside the warp's rows, so there all earlier stores are waited for)
+        if (lane == 0) { if constexpr (kGrouped) bulk_wait_group_read<0>(); else bulk_wait_group_read<1>(); }
         __syncwarp();
         uint8_t* srow = sb + lane * 64;
 #pragma unroll
@@ -309,9 +330,27 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           *reinterpret_cast<uint4*>(srow + ((static_cast<uint32_t>(j) ^ swz) << 4)) = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) {
-          tma_store_2d(&tmap_y, nt * kTN + c0, row0, sb);
-          bulk_commit_group();
+        if (!kGrouped || row0 + 32 <= rows_end) {
+          if (lane == 0) {
+            tma_store_2d(&tmap_y, nt * kTN + c0, row0, sb);
+            bulk_commit_group();
+          }
+        } else {
+          // the group ends inside this warp's 32 rows: the rows below belong to the next group, so the box store
+          // is replaced by 16-byte stores of the group's own rows (lane -> row lane / 4 + 8 i, 16-byte piece lane % 4)
+          const int esize = (p.ytype == MSD_OUT_BF16) ? 2 : 4;
+          const int col = nt * kTN + c0, piece = lane & 3;
+          if ((col + (piece + 1) * (16 / esize)) <= p.N) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int r = (lane >> 2) + 8 * i;
+              if (row0 + r < rows_end) {
+                const uint4 v = *reinterpret_cast<const uint4*>(sb + r * 64 + ((static_cast<uint32_t>(piece) ^ static_cast<uint32_t>((r >> 1) & 3)) << 4));
+                *reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.y) + (static_cast<size_t>(row0 + r) * p.N + col) * esize + piece * 16) = v;
+              }
+            }
+          }
+          __syncwarp();
         }
       }
     }
@@ -586,6 +625,30 @@ static GemmW4Plan plan_w4(int64_t M, int64_t N, int64_t K) {
   return pl;
 }
 
+// ---- grouped (mixture of experts) ----------------------------------------------------------------------------------
+// Workspace: components of up to 64 groups at a time as token tiles of 128 rows, their scale blocks, and the blocked
+// scales of all experts' weights.
+struct GroupedW4Plan {
+  int n_tiles, kstages, sf_kgroups, tile_n;
+  size_t off_q1, off_q2, off_sfa1, off_sfa2, off_sfb, bytes;
+};
+static GroupedW4Plan plan_grouped_w4(int32_t E, int64_t N, int64_t K) {
+  GroupedW4Plan pl;
+  pl.tile_n = w4_tile_n();
+  pl.n_tiles = static_cast<int>((N + pl.tile_n - 1) / pl.tile_n);
+  pl.kstages = static_cast<int>((K + kW4BlockK - 1) / kW4BlockK);
+  pl.sf_kgroups = 2 * pl.kstages;
+  const size_t rows = static_cast<size_t>(kMaxRowGroups) * kW4TileM;
+  size_t off = 0;
+  pl.off_q1 = off;   off = round_up(off + rows * (K / 2), 1024);
+  pl.off_q2 = off;   off = round_up(off + rows * (K / 2), 1024);
+  pl.off_sfa1 = off; off = round_up(off + static_cast<size_t>(kMaxRowGroups) * pl.sf_kgroups * 512, 1024);
+  pl.off_sfa2 = off; off = round_up(off + static_cast<size_t>(kMaxRowGroups) * pl.sf_kgroups * 512, 1024);
+  pl.off_sfb = off;  off = round_up(off + static_cast<size_t>(E) * 2 * pl.n_tiles * pl.sf_kgroups * 512, 1024);
+  pl.bytes = off;
+  return pl;
+}
+
 }  // namespace msd
 
 extern "C" {
@@ -688,16 +751,120 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   const size_t smem_bytes = static_cast<size_t>(kW4Stages) * (2 * kW4ABytes + pl.tile_n * 128 + kW4SfBytes) + 8 * kW4StoreBytes + 1024;
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(gemm_w4a16_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_w4a16_kernel<224>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_w4a16_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w4a16_kernel<224, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
       return MSD_ERR_CUDA;
     attr_done = true;
   }
   const cudaError_t le = pl.tile_n == 256
-      ? launch_pdl(gemm_w4a16_kernel<256>, dim3(pl.grid), dim3(kW4ThreadsSf), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p)
-      : launch_pdl(gemm_w4a16_kernel<224>, dim3(pl.grid), dim3(kW4ThreadsSf), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p);
+      ? launch_pdl(gemm_w4a16_kernel<256, false>, dim3(pl.grid), dim3(kW4ThreadsSf), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p, GemmW4NoGroups())
+      : launch_pdl(gemm_w4a16_kernel<224, false>, dim3(pl.grid), dim3(kW4ThreadsSf), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p, GemmW4NoGroups());
   if (le != cudaSuccess) return MSD_ERR_CUDA;
   return MSD_OK;
 }
+
+size_t msd_grouped_gemm_w4a16_workspace_bytes(int32_t E, int64_t N, int64_t K) {
+  if (E < 1 || N < 1 || K < 128 || K % 128 != 0) return 0;
+  return msd::plan_grouped_w4(E, N, K).bytes;
+}
+
+msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0,
+                                    const int32_t* group_sizes_host, int32_t E, int64_t N, int64_t K, void* y,
+                                    msd_out_t ytype, void* workspace, size_t workspace_bytes, void* stream) {
+  using namespace msd;
+  if (E < 1 || N < 1 || K < 128 || K % 128 != 0 || N % 8 != 0 || N > (1 << 24) || K > (1 << 24) ||
+      static_cast<int64_t>(E) * N > 0x7FFFFFFFLL)
+    return MSD_ERR_BAD_SHAPE;
+  if (ytype != MSD_OUT_BF16 && ytype != MSD_OUT_FP32) return MSD_ERR_UNSUPPORTED;
+  if (!x_bf16 || !w_fp4 || !w_e8m0 || !group_sizes_host || !y || !workspace) return MSD_ERR_NULL_POINTER;
+  if (!aligned(x_bf16, 16) || !aligned(w_fp4, 16) || !aligned(w_e8m0, 4) || !aligned(y, 16) || !aligned(workspace, 1024))
+    return MSD_ERR_BAD_ALIGNMENT;
+  int64_t M_total = 0;
+  for (int e = 0; e < E; ++e) {
+    if (group_sizes_host[e] < 0 || group_sizes_host[e] > kW4TileM) return MSD_ERR_BAD_SHAPE;     // decode regime per expert
+    M_total += group_sizes_host[e];
+  }
+  if (M_total > 0x7FFFFFFFLL) return MSD_ERR_BAD_SHAPE;
+  const GroupedW4Plan pl = plan_grouped_w4(E, N, K);
+  if (workspace_bytes < pl.bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
+  if (M_total == 0) return MSD_OK;
+  unsigned* status = device_status_ptr();
+  if (!status) return MSD_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  uint8_t* q1 = ws + pl.off_q1;
+  uint8_t* q2 = ws + pl.off_q2;
+  const bool ybf = ytype == MSD_OUT_BF16;
+  const uint64_t kb = static_cast<uint64_t>(K / 2);
+  CUtensorMap tmap_a1, tmap_a2, tmap_b, tmap_y;
+  if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, kb, static_cast<uint64_t>(kMaxRowGroups) * kW4TileM, kb, 128, kW4TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, q2, kb, static_cast<uint64_t>(kMaxRowGroups) * kW4TileM, kb, 128, kW4TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, w_fp4, kb, static_cast<uint64_t>(E) * N, kb, 128, static_cast<uint32_t>(pl.tile_n), CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, static_cast<uint64_t>(N),
+                      static_cast<uint64_t>(M_total), static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+    return MSD_ERR_CUDA;
+  const size_t smem_bytes = static_cast<size_t>(kW4Stages) * (2 * kW4ABytes + pl.tile_n * 128 + kW4SfBytes) + 8 * kW4StoreBytes + 1024;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(gemm_w4a16_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w4a16_kernel<224, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
+      return MSD_ERR_CUDA;
+    attr_done = true;
+  }
+  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+
+  // up to 64 non-empty groups per pair of launches (decomposition + GEMM); the weight scales of all experts are brought
+  // into the blocked layout by the first decomposition launch
+  bool scales_done = false;
+  int e = 0;
+  int64_t row = 0;
+  while (e < E) {
+    GemmW4Groups grp = {};
+    RowGroups rg = {};
+    const int64_t row_first = row;
+    while (e < E && grp.n < kMaxRowGroups) {
+      const int sz = group_sizes_host[e];
+      if (sz > 0) {
+        grp.expert[grp.n] = e;
+        grp.off[grp.n] = static_cast<int>(row);
+        rg.off[grp.n] = static_cast<int>(row - row_first);
+        row += sz;
+        ++grp.n;
+      }
+      ++e;
+    }
+    if (grp.n == 0) break;
+    grp.off[grp.n] = static_cast<int>(row);
+    rg.off[grp.n] = static_cast<int>(row - row_first);
+    rg.n = grp.n;
+    SfRelayout rl = {};
+    rl.src = w_e8m0; rl.dst = ws + pl.off_sfb; rl.rows = N; rl.kblocks = static_cast<int>(K / 32);
+    rl.sf_kgroups = pl.sf_kgroups; rl.tile_rows = pl.tile_n; rl.row_blocks = 2 * pl.n_tiles; rl.matrices = E;
+    msd_status_t st = launch_decompose_mxfp4(static_cast<const uint16_t*>(x_bf16) + row_first * K, row - row_first, K, K, q1, q2,
+                                             ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s, scales_done ? nullptr : &rl, nullptr, &rg);
+    if (st != MSD_OK) return st;
+    scales_done = true;
+
+    GemmW4Params p;
+    p.M = static_cast<int>(M_total); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+    p.m_tiles = grp.n; p.n_tiles = pl.n_tiles; p.kstages = pl.kstages; p.sf_kgroups = pl.sf_kgroups;
+    p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
+    p.y = y; p.ytype = ytype; p.status = status;
+    p.ready = nullptr; p.ready_sfb = 0;
+    p.n_fastest = 1;              // the CTAs of a wave share a group's components; every expert's weights are read once
+    {
+      const char* sfe = getenv("MSD_W4_SFWARPS");
+      p.sf_warps = sfe ? atoi(sfe) : 1;
+    }
+    const long long tiles = static_cast<long long>(grp.n) * pl.n_tiles;
+    const int grid = static_cast<int>(tiles < sm_count() ? tiles : sm_count());
+    const cudaError_t le = pl.tile_n == 256
+        ? launch_pdl(gemm_w4a16_kernel<256, true>, dim3(grid), dim3(kW4ThreadsSf), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p, grp)
+        : launch_pdl(gemm_w4a16_kernel<224, true>, dim3(grid), dim3(kW4ThreadsSf), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p, grp);
+    if (le != cudaSuccess) return MSD_ERR_CUDA;
+  }
+  return MSD_OK;
+}
+
 
 }  // extern "C"

@@ -80,11 +80,20 @@ struct SfRelayout {
   uint8_t* dst;
   int64_t rows;
   int kblocks, sf_kgroups, tile_rows, row_blocks;
+  int matrices;        // 0 or 1: one matrix; E > 1: E matrices of `rows` rows back to back (mixture-of-experts
+                       // weights), each cut into its own `row_blocks` blocks
   int blocks;          // filled in by the launcher (returned through the pointer when `ready` is used)
+};
+// Rows sorted by group (mixture of experts): group g owns rows [off[g], off[g+1]) and its decomposition is written as
+// token tile g (rows 128 g ...) of the component and scale buffers.
+constexpr int kMaxRowGroups = 64;
+struct RowGroups {
+  int n;                       // 0: no regrouping, output row = input row
+  int off[kMaxRowGroups + 1];
 };
 msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
                                     uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream,
-                                    SfRelayout* relayout = nullptr, unsigned* ready = nullptr);
+                                    SfRelayout* relayout = nullptr, unsigned* ready = nullptr, const RowGroups* groups = nullptr);
 
 #ifdef __CUDACC__
 // Relayout of row-major E8M0 scales [rows, kblocks] into the 512-byte blocks (128 rows x 4 scales) of the block-scaled
@@ -92,8 +101,12 @@ msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, in
 // partly used when tile_rows < 256); entries outside the matrix are written as zero.  One thread per 16 bytes of
 // the result: the four scales of rows l, l+32, l+64, l+96 of one block.
 __device__ inline void sf_relayout(const SfRelayout& j, int64_t first, int64_t step) {
-  const int64_t total = static_cast<int64_t>(j.row_blocks) * j.sf_kgroups * 32;
-  for (int64_t d = first; d < total; d += step) {
+  const int nmat = j.matrices > 1 ? j.matrices : 1;
+  const int64_t per = static_cast<int64_t>(j.row_blocks) * j.sf_kgroups * 32;
+  const int64_t total = per * nmat;
+  for (int64_t dd = first; dd < total; dd += step) {
+    const int64_t e = dd / per, d = dd - e * per;
+    const uint8_t* src = j.src + e * j.rows * j.kblocks;
     const int l = static_cast<int>(d & 31);
     const int64_t blk = d >> 5;
     const int64_t tb = blk / j.sf_kgroups;
@@ -105,9 +118,9 @@ __device__ inline void sf_relayout(const SfRelayout& j, int64_t first, int64_t s
       const int lr = static_cast<int>(tb & 1) * 128 + l + 32 * q;
       const int64_t row = t * j.tile_rows + lr;
       v[q] = (lr < j.tile_rows && row < j.rows && 4 * kg < j.kblocks)
-                 ? __ldg(reinterpret_cast<const uint32_t*>(j.src + row * j.kblocks + 4 * kg)) : 0u;
+                 ? __ldg(reinterpret_cast<const uint32_t*>(src + row * j.kblocks + 4 * kg)) : 0u;
     }
-    reinterpret_cast<uint4*>(j.dst)[d] = make_uint4(v[0], v[1], v[2], v[3]);
+    reinterpret_cast<uint4*>(j.dst)[dd] = make_uint4(v[0], v[1], v[2], v[3]);
   }
 }
 #endif
