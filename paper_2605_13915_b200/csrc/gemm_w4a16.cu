@@ -45,6 +45,9 @@ struct GemmW4Params {
   const unsigned* ready;        // progress of the decomposition kernel running beside this one (nullptr: it has finished):
                                 // [t] finished 32-element blocks of token tile t, [m_tiles] finished relayout CTAs
   unsigned ready_sfb;           // value of ready[m_tiles] when the weight scales are all in place
+  int a_rows;                   // rows of a token tile that are loaded (the box of the component tensor maps): 128, or
+                                // fewer when no group of a grouped launch is longer; the MMA reads stale rows beyond them,
+                                // whose results are never stored
   int n_fastest;                // tile index -> (token tile, weight tile): weight tile fastest (1) or token tile fastest (0)
   int sf_warps;                 // 1: warps 6..9 write the scales into TMEM (tcgen05.st); 0: the MMA thread copies them (tcgen05.cp)
   unsigned* status;
@@ -143,7 +146,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           if (!ok) break;
           uint8_t* dst = smem + stage * kStageBytes;
           if (warp == 0) {
-            mbar_arrive_expect_tx(&full_bar[stage], kStageBytes);
+            mbar_arrive_expect_tx(&full_bar[stage], kStageBytes - 2 * (kW4TileM - p.a_rows) * 128);
             tma_load_2d(dst, &tmap_a1, ks * 128, mt * kW4TileM, &full_bar[stage]);
             tma_load_2d(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, &full_bar[stage]);
             int b_row = nt * kTN;
@@ -632,9 +635,19 @@ struct GroupedW4Plan {
   int n_tiles, kstages, sf_kgroups, tile_n;
   size_t off_q1, off_q2, off_sfa1, off_sfa2, off_sfb, bytes;
 };
-static GroupedW4Plan plan_grouped_w4(int32_t E, int64_t N, int64_t K) {
+static GroupedW4Plan plan_grouped_w4(int32_t E, int64_t N, int64_t K, int groups) {
   GroupedW4Plan pl;
-  pl.tile_n = w4_tile_n();
+  // Tile width: the one whose tiles fill the SMs in fewer, or shorter, rounds (groups = non-empty groups of the first
+  // launch; the workspace is sized for the wider layout of the blocked weight scales either way)
+  const char* te = getenv("MSD_W4_TILEN");
+  if (te) {
+    pl.tile_n = atoi(te) == 256 ? 256 : 224;
+  } else {
+    const long long g = groups < 1 ? 1 : (groups > kMaxRowGroups ? kMaxRowGroups : groups);
+    const long long t224 = g * ((N + 223) / 224), t256 = g * ((N + 255) / 256);
+    const long long c224 = (t224 + sm_count() - 1) / sm_count() * 224, c256 = (t256 + sm_count() - 1) / sm_count() * 256;
+    pl.tile_n = c256 < c224 ? 256 : 224;
+  }
   pl.n_tiles = static_cast<int>((N + pl.tile_n - 1) / pl.tile_n);
   pl.kstages = static_cast<int>((K + kW4BlockK - 1) / kW4BlockK);
   pl.sf_kgroups = 2 * pl.kstages;
@@ -644,7 +657,8 @@ static GroupedW4Plan plan_grouped_w4(int32_t E, int64_t N, int64_t K) {
   pl.off_q2 = off;   off = round_up(off + rows * (K / 2), 1024);
   pl.off_sfa1 = off; off = round_up(off + static_cast<size_t>(kMaxRowGroups) * pl.sf_kgroups * 512, 1024);
   pl.off_sfa2 = off; off = round_up(off + static_cast<size_t>(kMaxRowGroups) * pl.sf_kgroups * 512, 1024);
-  pl.off_sfb = off;  off = round_up(off + static_cast<size_t>(E) * 2 * pl.n_tiles * pl.sf_kgroups * 512, 1024);
+  // (N + 223) / 224 tiles is the larger count of the two widths
+  pl.off_sfb = off;  off = round_up(off + static_cast<size_t>(E) * 2 * ((N + 223) / 224) * pl.sf_kgroups * 512, 1024);
   pl.bytes = off;
   return pl;
 }
@@ -707,6 +721,7 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
   p.y = y; p.ytype = ytype; p.status = status;
   p.ready = ready; p.ready_sfb = static_cast<unsigned>(rl.blocks);
+  p.a_rows = kW4TileM;
   {
     const char* sfe = getenv("MSD_W4_SFWARPS");
     p.sf_warps = sfe ? atoi(sfe) : 1;
@@ -765,7 +780,7 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
 
 size_t msd_grouped_gemm_w4a16_workspace_bytes(int32_t E, int64_t N, int64_t K) {
   if (E < 1 || N < 1 || K < 128 || K % 128 != 0) return 0;
-  return msd::plan_grouped_w4(E, N, K).bytes;
+  return msd::plan_grouped_w4(E, N, K, E).bytes;
 }
 
 msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0,
@@ -780,12 +795,16 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
   if (!aligned(x_bf16, 16) || !aligned(w_fp4, 16) || !aligned(w_e8m0, 4) || !aligned(y, 16) || !aligned(workspace, 1024))
     return MSD_ERR_BAD_ALIGNMENT;
   int64_t M_total = 0;
+  int nonempty = 0, largest = 0;
   for (int e = 0; e < E; ++e) {
     if (group_sizes_host[e] < 0 || group_sizes_host[e] > kW4TileM) return MSD_ERR_BAD_SHAPE;     // decode regime per expert
     M_total += group_sizes_host[e];
+    nonempty += group_sizes_host[e] > 0 ? 1 : 0;
+    if (group_sizes_host[e] > largest) largest = group_sizes_host[e];
   }
   if (M_total > 0x7FFFFFFFLL) return MSD_ERR_BAD_SHAPE;
-  const GroupedW4Plan pl = plan_grouped_w4(E, N, K);
+  const GroupedW4Plan pl = plan_grouped_w4(E, N, K, nonempty);
+  const int a_rows = (largest + 7) / 8 * 8;             // rows of a token tile worth loading (whole 8-row swizzle atoms)
   if (workspace_bytes < pl.bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
   if (M_total == 0) return MSD_OK;
   unsigned* status = device_status_ptr();
@@ -797,8 +816,8 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
   const bool ybf = ytype == MSD_OUT_BF16;
   const uint64_t kb = static_cast<uint64_t>(K / 2);
   CUtensorMap tmap_a1, tmap_a2, tmap_b, tmap_y;
-  if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, kb, static_cast<uint64_t>(kMaxRowGroups) * kW4TileM, kb, 128, kW4TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, q2, kb, static_cast<uint64_t>(kMaxRowGroups) * kW4TileM, kb, 128, kW4TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+  if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, kb, static_cast<uint64_t>(kMaxRowGroups) * kW4TileM, kb, 128, static_cast<uint32_t>(a_rows), CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, q2, kb, static_cast<uint64_t>(kMaxRowGroups) * kW4TileM, kb, 128, static_cast<uint32_t>(a_rows), CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, w_fp4, kb, static_cast<uint64_t>(E) * N, kb, 128, static_cast<uint32_t>(pl.tile_n), CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, static_cast<uint64_t>(N),
                       static_cast<uint64_t>(M_total), static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
@@ -851,6 +870,7 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
     p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
     p.y = y; p.ytype = ytype; p.status = status;
     p.ready = nullptr; p.ready_sfb = 0;
+    p.a_rows = a_rows;
     p.n_fastest = 1;              // the CTAs of a wave share a group's components; every expert's weights are read once
     {
       const char* sfe = getenv("MSD_W4_SFWARPS");
