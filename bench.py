@@ -439,7 +439,23 @@ def other_configs(torch, binding, device, capture, timed):
         "us": round(tg, 1), "weight_gbps": round(E * Ng * Kg / tg / 1e3, 1),
         "frac_of_measured_hbm": round(E * Ng * Kg / tg / 1e3 / peaks["hbm_gbs"], 3),
         "one_call_per_expert_us": round(tl, 1), "speedup": round(tl / tg, 2)}
-    del xg, wg, sg, yg, wsg
+    del wg, sg, wsg
+
+    # the same experts with MXFP4 weights (grouped W4A16): weight + scale bytes per call
+    w4g = [torch.randint(0, 256, (E, Ng, Kg // 2), generator=g, dtype=torch.uint8, device=device) for _ in range(2)]
+    e4g = torch.randint(118, 124, (E, Ng, Kg // 32), generator=g, dtype=torch.uint8, device=device)
+    ws4 = binding.workspace(int(binding.lib().msd_grouped_gemm_w4a16_workspace_bytes(E, Ng, Kg)), device)
+
+    def f_grouped4():
+        itg[0] += 1
+        binding.grouped_gemm_w4a16(xg, w4g[itg[0] % 2], e4g, [per] * E, ws=ws4, out=yg)
+    t4 = per_call_us(f_grouped4)
+    b4 = E * Ng * (Kg // 2 + Kg // 32)
+    res["moe_grouped_w4a16_E32_N2048_K7168_16_tokens_per_expert"] = {
+        "us": round(t4, 1), "weight_and_scale_gbps": round(b4 / t4 / 1e3, 1),
+        "frac_of_measured_hbm": round(b4 / t4 / 1e3 / peaks["hbm_gbs"], 3),
+        "note": "includes bringing all experts' weight scales into the blocked layout on every call"}
+    del xg, yg, w4g, e4g, ws4
 
     # configs[3] GQA and configs[4] MLA decode attention
     from paper_2605_13915_b200 import inputs as gen

@@ -45,6 +45,7 @@ struct GemmW4Params {
   const unsigned* ready;        // progress of the decomposition kernel running beside this one (nullptr: it has finished):
                                 // [t] finished 32-element blocks of token tile t, [m_tiles] finished relayout CTAs
   unsigned ready_sfb;           // value of ready[m_tiles] when the weight scales are all in place
+  int nstages;                  // grouped launches: pipeline stages that fit with a_rows rows per component tile
   int a_rows;                   // rows of a token tile that are loaded (the box of the component tensor maps): 128, or
                                 // fewer when no group of a grouped launch is longer; the MMA reads stale rows beyond them,
                                 // whose results are never stored
@@ -90,11 +91,18 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
                   const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_y,
                   const GemmW4Params p, const typename W4GroupArg<kGrouped>::type grp) {
   constexpr int kBBytes = kTN * 128;
-  constexpr int kStageBytes = 2 * kW4ABytes + kBBytes + kW4SfBytes;
+  // Shared-memory stage: the two component tiles, the weight tile, the scale blocks.  Grouped launches load only
+  // a_rows <= 128 rows per component (whole 1 KB swizzle atoms), pack the stage accordingly and use the room for more
+  // stages: their weight tiles come from HBM, not L2, and a freed stage takes twice as long to fill.  The MMA still
+  // reads 128 rows from where a component tile starts: whatever follows it there, results never stored.
+  constexpr int kMaxStages = kGrouped ? 8 : kW4Stages;
+  const int a_bytes = kGrouped ? p.a_rows * 128 : kW4ABytes;
+  const int kStageBytes = 2 * a_bytes + kBBytes + kW4SfBytes;
+  const int nstages = kGrouped ? p.nstages : kW4Stages;
   constexpr int kAcc = (2 * kTN + 64 <= kW4TmemCols) ? 2 : 1;       // accumulators that fit beside 2 x 32 scale columns
   constexpr int kSfCol = kAcc * kTN;
   extern __shared__ uint8_t smem_dyn[];
-  __shared__ __align__(8) uint64_t full_bar[kW4Stages], empty_bar[kW4Stages], tfull_bar[2], tempty_bar[2];
+  __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tfull_bar[2], tempty_bar[2];
   // the two sets of scale columns in TMEM: written by warps 6..9 (sf_ready), read by the MMAs of a stage (sf_free)
   __shared__ __align__(8) uint64_t sf_ready[2], sf_free[2];
   __shared__ uint32_t tmem_base_slot;
@@ -104,7 +112,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kW4Stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < nstages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], 4); }
     for (int a = 0; a < 2; ++a) { mbar_init(&sf_ready[a], 4); mbar_init(&sf_free[a], 1); }
     abort_flag = 0;
@@ -146,14 +154,14 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           if (!ok) break;
           uint8_t* dst = smem + stage * kStageBytes;
           if (warp == 0) {
-            mbar_arrive_expect_tx(&full_bar[stage], kStageBytes - 2 * (kW4TileM - p.a_rows) * 128);
+            mbar_arrive_expect_tx(&full_bar[stage], kStageBytes);
             tma_load_2d(dst, &tmap_a1, ks * 128, mt * kW4TileM, &full_bar[stage]);
-            tma_load_2d(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, &full_bar[stage]);
+            tma_load_2d(dst + a_bytes, &tmap_a2, ks * 128, mt * kW4TileM, &full_bar[stage]);
             int b_row = nt * kTN;
             if constexpr (kGrouped) b_row += grp.expert[mt] * p.N;          // the weights of the group's expert
-            tma_load_2d(dst + 2 * kW4ABytes, &tmap_b, ks * 128, b_row, &full_bar[stage]);
+            tma_load_2d(dst + 2 * a_bytes, &tmap_b, ks * 128, b_row, &full_bar[stage]);
           } else {
-            uint8_t* sf = dst + 2 * kW4ABytes + kBBytes;
+            uint8_t* sf = dst + 2 * a_bytes + kBBytes;
             const size_t a_off = (static_cast<size_t>(mt) * p.sf_kgroups + 2 * ks) * 512;
             bulk_load(sf, p.sfa1 + a_off, 1024, &full_bar[stage]);
             bulk_load(sf + 1024, p.sfa2 + a_off, 1024, &full_bar[stage]);
@@ -162,7 +170,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
             bulk_load(sf + 2048, p.sfb + (sfb_blk * p.sf_kgroups + 2 * ks) * 512, 1024, &full_bar[stage]);
             bulk_load(sf + 3072, p.sfb + ((sfb_blk + 1) * p.sf_kgroups + 2 * ks) * 512, 1024, &full_bar[stage]);
           }
-          if (++stage == kW4Stages) { stage = 0; phase ^= 1; }
+          if (++stage == nstages) { stage = 0; phase ^= 1; }
         }
       }
     }
@@ -192,8 +200,8 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           // memory is far below its range), so every operand costs one 64-bit add: this single thread's instruction
           // count per stage, not the tensor pipe, was what paced the kernel.
           const uint64_t enc = static_cast<uint64_t>(smem_u32(smem + stage * kStageBytes) >> 4);
-          const uint64_t a1d = op_desc + enc, a2d = a1d + (kW4ABytes >> 4), bd = a1d + (2 * kW4ABytes >> 4);
-          const uint64_t sfd = sf_desc + enc + ((2 * kW4ABytes + kBBytes) >> 4);
+          const uint64_t a1d = op_desc + enc, a2d = a1d + (a_bytes >> 4), bd = a1d + (2 * a_bytes >> 4);
+          const uint64_t sfd = sf_desc + enc + ((2 * a_bytes + kBBytes) >> 4);
           const uint32_t sfa1_t = tmem_base + kSfCol + 32 * sfpar;     // 2 k-groups x 4 columns; the two sets alternate
           const uint32_t sfa2_t = sfa1_t + 8;
           const uint32_t sfb_t = sfa1_t + 16;                            // 2 k-groups x 8 columns (256 weight rows)
@@ -223,7 +231,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           sfpar ^= 1;
           ++nstage;
           tc_commit(&empty_bar[stage]);
-          if (++stage == kW4Stages) { stage = 0; phase ^= 1; }
+          if (++stage == nstages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
         tc_commit(&tfull_bar[acc]);
@@ -249,7 +257,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
             if (!ok) break;
             tc_fence_after();
           }
-          const uint4* sf = reinterpret_cast<const uint4*>(smem + stage * kStageBytes + 2 * kW4ABytes + kBBytes) + lane;
+          const uint4* sf = reinterpret_cast<const uint4*>(smem + stage * kStageBytes + 2 * a_bytes + kBBytes) + lane;
           uint32_t v[32];
           // column order of a set: sfa1 (g0, g1), sfa2 (g0, g1), then per K group the two halves of the weight tile
           constexpr int kBlk[8] = {0, 1, 2, 3, 4, 6, 5, 7};
@@ -263,7 +271,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&sf_ready[set]);
-          if (++stage == kW4Stages) { stage = 0; phase ^= 1; }
+          if (++stage == nstages) { stage = 0; phase ^= 1; }
         }
       }
     }
@@ -274,7 +282,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
     // the store of one chunk in flight while the next is converted.  Rows past M and columns past N are clipped by
     // the store itself.
     const int quad = warp & 3;
-    uint8_t* stage_buf = smem + kW4Stages * kStageBytes + quad * (2 * kW4StoreBytes);
+    uint8_t* stage_buf = smem + nstages * kStageBytes + quad * (2 * kW4StoreBytes);
     const int ccols = (p.ytype == MSD_OUT_BF16) ? 32 : 16;
     const uint32_t swz = static_cast<uint32_t>((lane >> 1) & 3);
     int it = 0, buf = 0;
@@ -721,7 +729,7 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
   p.y = y; p.ytype = ytype; p.status = status;
   p.ready = ready; p.ready_sfb = static_cast<unsigned>(rl.blocks);
-  p.a_rows = kW4TileM;
+  p.a_rows = kW4TileM; p.nstages = kW4Stages;
   {
     const char* sfe = getenv("MSD_W4_SFWARPS");
     p.sf_warps = sfe ? atoi(sfe) : 1;
@@ -822,7 +830,10 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
       !encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, static_cast<uint64_t>(N),
                       static_cast<uint64_t>(M_total), static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
     return MSD_ERR_CUDA;
-  const size_t smem_bytes = static_cast<size_t>(kW4Stages) * (2 * kW4ABytes + pl.tile_n * 128 + kW4SfBytes) + 8 * kW4StoreBytes + 1024;
+  const size_t stage_bytes = static_cast<size_t>(2 * a_rows * 128 + pl.tile_n * 128 + kW4SfBytes);
+  int nstages = static_cast<int>((227 * 1024 - 2048 - 8 * kW4StoreBytes - 1024) / stage_bytes);
+  if (nstages > 8) nstages = 8;
+  const size_t smem_bytes = nstages * stage_bytes + 8 * kW4StoreBytes + 1024;
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(gemm_w4a16_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
@@ -870,7 +881,7 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
     p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
     p.y = y; p.ytype = ytype; p.status = status;
     p.ready = nullptr; p.ready_sfb = 0;
-    p.a_rows = a_rows;
+    p.a_rows = a_rows; p.nstages = nstages;
     p.n_fastest = 1;              // the CTAs of a wave share a group's components; every expert's weights are read once
     {
       const char* sfe = getenv("MSD_W4_SFWARPS");
