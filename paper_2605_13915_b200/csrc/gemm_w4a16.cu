@@ -45,7 +45,9 @@ struct GemmW4Params {
   const unsigned* ready;        // progress of the decomposition kernel running beside this one (nullptr: it has finished):
                                 // [t] finished 32-element blocks of token tile t, [m_tiles] finished relayout CTAs
   unsigned ready_sfb;           // value of ready[m_tiles] when the weight scales are all in place
-  int nstages;                  // grouped launches: pipeline stages that fit with a_rows rows per component tile
+  int ksplit, kper;             // K splits per output tile and K stages per split (1, kstages: no split)
+  int part_rows;                // ksplit > 1: rows per split of the partial-sum buffer the tiles are written to
+  int nstages;                  // pipeline stages that fit with a_rows rows per component tile
   int a_rows;                   // rows of a token tile that are loaded (the box of the component tensor maps): 128, or
                                 // fewer when no group of a grouped launch is longer; the MMA reads stale rows beyond them,
                                 // whose results are never stored
@@ -63,6 +65,27 @@ struct GemmW4Groups {
 struct GemmW4NoGroups {};
 template <bool kGrouped> struct W4GroupArg { using type = GemmW4NoGroups; };
 template <> struct W4GroupArg<true> { using type = GemmW4Groups; };
+
+// Sum of the K-split partial tiles, split 0 first (fixed order: the same inputs give the same bits), rounded once.
+__global__ void __launch_bounds__(256)
+w4_ksplit_reduce_kernel(const float* __restrict__ part, int ksplit, int64_t part_stride, int64_t M, int64_t N, void* __restrict__ y,
+                        int ytype) {
+  pdl_wait_primary();
+  const int64_t total = M * N / 4;                     // N is a multiple of 8
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    float4 acc = __ldg(reinterpret_cast<const float4*>(part) + i);
+    for (int s = 1; s < ksplit; ++s) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(part + s * part_stride) + i);
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    if (ytype == MSD_OUT_BF16) {
+      const __nv_bfloat162 h0 = __floats2bfloat162_rn(acc.x, acc.y), h1 = __floats2bfloat162_rn(acc.z, acc.w);
+      reinterpret_cast<uint2*>(y)[i] = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+    } else {
+      reinterpret_cast<float4*>(y)[i] = acc;
+    }
+  }
+}
 
 // Bounded wait for a progress counter of the kernel this one depends on (see GemmW4Params::ready); afterwards the
 // async proxy (TMA) may read what that kernel's threads wrote.
@@ -91,14 +114,14 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
                   const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_y,
                   const GemmW4Params p, const typename W4GroupArg<kGrouped>::type grp) {
   constexpr int kBBytes = kTN * 128;
-  // Shared-memory stage: the two component tiles, the weight tile, the scale blocks.  Grouped launches load only
-  // a_rows <= 128 rows per component (whole 1 KB swizzle atoms), pack the stage accordingly and use the room for more
+  // Shared-memory stage: the two component tiles, the weight tile, the scale blocks.  Launches with few rows (one
+  // token tile of M < 128 rows, short groups) load only a_rows <= 128 rows per component (whole 1 KB swizzle atoms), pack the stage accordingly and use the room for more
   // stages: their weight tiles come from HBM, not L2, and a freed stage takes twice as long to fill.  The MMA still
   // reads 128 rows from where a component tile starts: whatever follows it there, results never stored.
-  constexpr int kMaxStages = kGrouped ? 8 : kW4Stages;
-  const int a_bytes = kGrouped ? p.a_rows * 128 : kW4ABytes;
+  constexpr int kMaxStages = 8;
+  const int a_bytes = p.a_rows * 128;
   const int kStageBytes = 2 * a_bytes + kBBytes + kW4SfBytes;
-  const int nstages = kGrouped ? p.nstages : kW4Stages;
+  const int nstages = p.nstages;
   constexpr int kAcc = (2 * kTN + 64 <= kW4TmemCols) ? 2 : 1;       // accumulators that fit beside 2 x 32 scale columns
   constexpr int kSfCol = kAcc * kTN;
   extern __shared__ uint8_t smem_dyn[];
@@ -127,7 +150,10 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
   volatile int* abort = &abort_flag;
-  const int total_tiles = p.m_tiles * p.n_tiles;
+  // Work items: (token tile, weight tile, K split).  With ksplit > 1 (few tiles, long K: decode shapes) every item
+  // covers kper K stages and its FP32 partial tile goes to rows [split * part_rows, ...) of a partial-sum buffer that a
+  // second kernel adds up in a fixed order.
+  const int total_tiles = p.m_tiles * p.n_tiles * p.ksplit;
 
   if (warp == 0 || warp == 10) {
     // Two producer threads: issuing a bulk copy costs its thread 50-100 ns, and the time a freed stage waits for its
@@ -142,14 +168,16 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
       int stage = 0; uint32_t phase = 0;
       int mt_ready = -1;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int mt = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles, nt = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
+        const int split = tile % p.ksplit, tile_mn = tile / p.ksplit;
+        const int mt = p.n_fastest ? tile_mn / p.n_tiles : tile_mn % p.m_tiles, nt = p.n_fastest ? tile_mn % p.n_tiles : tile_mn / p.m_tiles;
+        const int ks0 = split * p.kper, ks1 = ks0 + p.kper < p.kstages ? ks0 + p.kper : p.kstages;
         if (p.ready && mt != mt_ready) {
           const int rows = p.M - mt * kW4TileM < kW4TileM ? p.M - mt * kW4TileM : kW4TileM;
           ok = wait_progress(p.ready + mt, static_cast<unsigned>(rows) * static_cast<unsigned>(p.K >> 5), abort, p.status);
           if (!ok) break;
           mt_ready = mt;
         }
-        for (int ks = 0; ks < p.kstages; ++ks) {
+        for (int ks = ks0; ks < ks1; ++ks) {
           ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
           if (!ok) break;
           uint8_t* dst = smem + stage * kStageBytes;
@@ -192,7 +220,8 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
         ok = wait_bounded(&tempty_bar[acc], tphase ^ 1, abort, p.status);      // epilogue has drained this accumulator
         if (!ok) break;
         tc_fence_after();
-        for (int ks = 0; ks < p.kstages; ++ks) {
+        const int ks0 = (tile % p.ksplit) * p.kper, ks1 = ks0 + p.kper < p.kstages ? ks0 + p.kper : p.kstages;
+        for (int ks = ks0; ks < ks1; ++ks) {
           ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
           if (!ok) break;
           tc_fence_after();
@@ -224,7 +253,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           for (int kk = 0; kk < 4; ++kk) {                    // 64 elements (32 bytes) per MMA
             const int g = kk >> 1;
             const uint32_t idesc = (kk & 1) ? idesc_hi : idesc_lo;   // which pair of scale bytes of the 4-scale column
-            mma_mxf4(d_tmem, a1d + 2 * kk, bd + 2 * kk, idesc, sfa1_t + 4 * g, sfb_t + 8 * g, (ks > 0 || kk > 0) ? 1u : 0u);
+            mma_mxf4(d_tmem, a1d + 2 * kk, bd + 2 * kk, idesc, sfa1_t + 4 * g, sfb_t + 8 * g, (ks > ks0 || kk > 0) ? 1u : 0u);
             mma_mxf4(d_tmem, a2d + 2 * kk, bd + 2 * kk, idesc, sfa2_t + 4 * g, sfb_t + 8 * g, 1u);
           }
           tc_commit(&sf_free[sfpar]);                // this set of scale columns may be rewritten once these MMAs are done
@@ -248,7 +277,8 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
       int n = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        for (int ks = 0; ks < p.kstages; ++ks, ++n) {
+        const int ks0 = (tile % p.ksplit) * p.kper, ks1 = ks0 + p.kper < p.kstages ? ks0 + p.kper : p.kstages;
+        for (int ks = ks0; ks < ks1; ++ks, ++n) {
           const int set = n & 1;
           ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
           if (!ok) break;
@@ -288,7 +318,9 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
     int it = 0, buf = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-      const int mt = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles, nt = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
+      const int split = tile % p.ksplit, tile_mn = tile / p.ksplit;
+        const int mt = p.n_fastest ? tile_mn / p.n_tiles : tile_mn % p.m_tiles, nt = p.n_fastest ? tile_mn % p.n_tiles : tile_mn / p.m_tiles;
+        const int ks0 = split * p.kper, ks1 = ks0 + p.kper < p.kstages ? ks0 + p.kper : p.kstages;
       const int acc = (kAcc == 2) ? (it & 1) : 0;
       const uint32_t tphase = (kAcc == 2) ? ((it >> 1) & 1) : (it & 1);
       ok = wait_bounded(&tfull_bar[acc], tphase, abort, p.status);
@@ -343,7 +375,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
         __syncwarp();
         if (!kGrouped || row0 + 32 <= rows_end) {
           if (lane == 0) {
-            tma_store_2d(&tmap_y, nt * kTN + c0, row0, sb);
+            tma_store_2d(&tmap_y, nt * kTN + c0, row0 + split * p.part_rows, sb);
             bulk_commit_group();
           }
         } else {
@@ -598,7 +630,8 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
 
 struct GemmW4Plan {
   int m_tiles, n_tiles, kstages, sf_kgroups, grid, tile_n;
-  size_t off_q1, off_q2, off_sfa1, off_sfa2, off_sfb, off_ready, bytes;
+  int ksplit, kper, a_rows, nstages;
+  size_t off_q1, off_q2, off_sfa1, off_sfa2, off_sfb, off_ready, off_part, bytes;
 };
 
 // Weight rows per tile: 224 (two accumulators) unless MSD_W4_TILEN=256.
@@ -622,9 +655,30 @@ static GemmW4Plan plan_w4(int64_t M, int64_t N, int64_t K) {
   pl.kstages = static_cast<int>((K + kW4BlockK - 1) / kW4BlockK);
   pl.sf_kgroups = 2 * pl.kstages;
   const int tiles = pl.m_tiles * pl.n_tiles;
+  // Few output tiles and a long K (decode shapes): split K so that there is about one work item per SM, each at
+  // least four stages long; the FP32 partial tiles are added by a second kernel.
+  pl.ksplit = 1;
+  pl.kper = pl.kstages;
+  {
+    const char* se = getenv("MSD_W4_KSPLIT");
+    int want = se ? atoi(se) : (2 * tiles <= sm_count() ? sm_count() / tiles : 1);
+    if (want > pl.kstages / 4) want = pl.kstages / 4;
+    if (want > 1) {
+      pl.kper = (pl.kstages + want - 1) / want;
+      pl.ksplit = (pl.kstages + pl.kper - 1) / pl.kper;
+    }
+  }
+  const int items = tiles * pl.ksplit;
   int grid = sm_count();
-  if (grid > tiles) grid = tiles;
+  if (grid > items) grid = items;
   pl.grid = grid;
+  // one token tile of fewer than 128 rows: only those rows are loaded and the stages are packed (more of them fit)
+  pl.a_rows = pl.m_tiles == 1 ? static_cast<int>((M + 7) / 8 * 8) : kW4TileM;
+  {
+    const size_t stage_bytes = static_cast<size_t>(2 * pl.a_rows * 128 + tile_n * 128 + kW4SfBytes);
+    int ns = static_cast<int>((227 * 1024 - 2048 - 8 * kW4StoreBytes - 1024) / stage_bytes);
+    pl.nstages = ns > 8 ? 8 : ns;
+  }
   size_t off = 0;
   pl.off_q1 = off;   off = round_up(off + static_cast<size_t>(M) * (K / 2), 1024);
   pl.off_q2 = off;   off = round_up(off + static_cast<size_t>(M) * (K / 2), 1024);
@@ -632,6 +686,8 @@ static GemmW4Plan plan_w4(int64_t M, int64_t N, int64_t K) {
   pl.off_sfa2 = off; off = round_up(off + static_cast<size_t>(pl.m_tiles) * pl.sf_kgroups * 512, 1024);
   pl.off_sfb = off;  off = round_up(off + static_cast<size_t>(2 * pl.n_tiles) * pl.sf_kgroups * 512, 1024);
   pl.off_ready = off; off = round_up(off + static_cast<size_t>(pl.m_tiles + 1) * sizeof(unsigned), 1024);
+  pl.off_part = off;
+  if (pl.ksplit > 1) off = round_up(off + static_cast<size_t>(pl.ksplit) * pl.m_tiles * kW4TileM * N * sizeof(float), 1024);
   pl.bytes = off;
   return pl;
 }
@@ -718,8 +774,8 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
 
   CUtensorMap tmap_a1, tmap_a2, tmap_b;
   const uint64_t kb = static_cast<uint64_t>(K / 2);
-  if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, kb, M, kb, 128, kW4TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, q2, kb, M, kb, 128, kW4TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+  if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, kb, M, kb, 128, static_cast<uint32_t>(use_pair ? kW4TileM : pl.a_rows), CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, q2, kb, M, kb, 128, static_cast<uint32_t>(use_pair ? kW4TileM : pl.a_rows), CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, w_fp4, kb, N, kb, 128, static_cast<uint32_t>(pl.tile_n), CU_TENSOR_MAP_SWIZZLE_128B))
     return MSD_ERR_CUDA;
 
@@ -729,7 +785,7 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
   p.y = y; p.ytype = ytype; p.status = status;
   p.ready = ready; p.ready_sfb = static_cast<unsigned>(rl.blocks);
-  p.a_rows = kW4TileM; p.nstages = kW4Stages;
+  p.a_rows = kW4TileM; p.nstages = kW4Stages; p.ksplit = 1; p.kper = pl.kstages; p.part_rows = 0;
   {
     const char* sfe = getenv("MSD_W4_SFWARPS");
     p.sf_warps = sfe ? atoi(sfe) : 1;
@@ -766,12 +822,20 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
     if (pe != cudaSuccess) return MSD_ERR_CUDA;
     return MSD_OK;
   }
+  // With a K split the kernel writes FP32 partial tiles (split s at rows s * part_rows ...) and a second kernel adds them.
   CUtensorMap tmap_y;
-  const bool ybf = ytype == MSD_OUT_BF16;
-  if (!encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, static_cast<uint64_t>(N),
-                      static_cast<uint64_t>(M), static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+  const bool split = pl.ksplit > 1;
+  const bool ybf = !split && ytype == MSD_OUT_BF16;
+  float* part = reinterpret_cast<float*>(ws + pl.off_part);
+  const uint64_t part_rows = static_cast<uint64_t>(pl.m_tiles) * kW4TileM;
+  if (!encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, split ? static_cast<void*>(part) : y,
+                      static_cast<uint64_t>(N), split ? part_rows * pl.ksplit : static_cast<uint64_t>(M),
+                      static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
     return MSD_ERR_CUDA;
-  const size_t smem_bytes = static_cast<size_t>(kW4Stages) * (2 * kW4ABytes + pl.tile_n * 128 + kW4SfBytes) + 8 * kW4StoreBytes + 1024;
+  if (split) p.ytype = MSD_OUT_FP32;
+  p.ksplit = pl.ksplit; p.kper = pl.kper; p.part_rows = static_cast<int>(part_rows);
+  p.a_rows = pl.a_rows; p.nstages = pl.nstages;
+  const size_t smem_bytes = static_cast<size_t>(pl.nstages) * (2 * pl.a_rows * 128 + pl.tile_n * 128 + kW4SfBytes) + 8 * kW4StoreBytes + 1024;
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(gemm_w4a16_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
@@ -783,6 +847,14 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
       ? launch_pdl(gemm_w4a16_kernel<256, false>, dim3(pl.grid), dim3(kW4ThreadsSf), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p, GemmW4NoGroups())
       : launch_pdl(gemm_w4a16_kernel<224, false>, dim3(pl.grid), dim3(kW4ThreadsSf), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p, GemmW4NoGroups());
   if (le != cudaSuccess) return MSD_ERR_CUDA;
+  if (split) {
+    const int64_t quads = M * N / 4;
+    int64_t blocks = (quads + 255) / 256;
+    if (blocks > 4LL * sm_count()) blocks = 4LL * sm_count();
+    if (launch_pdl(w4_ksplit_reduce_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, s, pdl, static_cast<const float*>(part), pl.ksplit,
+                   static_cast<int64_t>(part_rows) * N, M, N, y, static_cast<int>(ytype)) != cudaSuccess)
+      return MSD_ERR_CUDA;
+  }
   return MSD_OK;
 }
 
@@ -882,6 +954,7 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
     p.y = y; p.ytype = ytype; p.status = status;
     p.ready = nullptr; p.ready_sfb = 0;
     p.a_rows = a_rows; p.nstages = nstages;
+    p.ksplit = 1; p.kper = pl.kstages; p.part_rows = 0;
     p.n_fastest = 1;              // the CTAs of a wave share a group's components; every expert's weights are read once
     {
       const char* sfe = getenv("MSD_W4_SFWARPS");

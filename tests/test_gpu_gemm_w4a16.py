@@ -101,3 +101,15 @@ def test_gemm_beside_the_decomposition(monkeypatch):
         c = inputs.gemm_w4_case(M, N, K, seed=11 + M)
         y = _run(c, torch.float32).cpu().numpy().astype(np.float64)
         _close(y, oracle.gemm_w4a16(c.x, c.w_fp4, c.w_e8m0, "f64"), False)
+
+
+@pytest.mark.parametrize("M,N,K", [(16, 448, 4096), (100, 1000, 3072), (1, 232, 8192), (128, 264, 2048)])
+def test_decode_shapes_with_k_split(M, N, K):
+    """Few output tiles and a long K: the K stages are split over several CTAs, the FP32 partial tiles are added by a
+    second kernel; only the M rows present are loaded (packed stages).  Ragged last weight tile, M = 1 and M = 128."""
+    c = inputs.gemm_w4_case(M, N, K, seed=21 + M)
+    ref = oracle.gemm_w4a16(c.x, c.w_fp4, c.w_e8m0, "f64")
+    y = _run(c, torch.float32).cpu().numpy().astype(np.float64)
+    _close(y, ref, False)
+    yb = _run(c, torch.bfloat16)
+    _close(oracle.bf16_bits_to_f64(bf16_bits(yb)), ref, True)
