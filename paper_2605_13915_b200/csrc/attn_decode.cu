@@ -71,6 +71,60 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// c1 for one query row (one warp): head slot h of the group's stacked operand (rows h and HG + h of every 128-byte
+// chunk at `img`, 128-byte swizzle) and its two scales.  `img` is shared memory in the attention kernel's own set-up
+// and global memory in attn_qstack_kernel; same bit-exact rule as msd_decompose_int8.
+__device__ __forceinline__ void attn_decompose_q_row(const AttnParams& p, int b, int hk, int grp, int h, int lane, uint8_t* img,
+                                                     float* alpha_out, float* beta_out) {
+  const int r_kv = grp * p.HG + h, sq = r_kv / p.Gr;       // row of this KV head -> (query token, head of the group)
+  const uint4* qrow = reinterpret_cast<const uint4*>(
+      p.q + ((static_cast<long long>(b) * p.Sq + sq) * (p.Hkv * p.Gr) + hk * p.Gr + (r_kv - sq * p.Gr)) * p.D);
+  const int nvec = p.D >> 3;                    // 8 BF16 values per 16-byte load (D % 16 == 0, D <= 640)
+  uint4 qv[3];                                  // the whole row stays in registers between the two passes
+  float m = 0.0f;
+#pragma unroll
+  for (int j = 0; j < 3; ++j) {
+    const int i = lane + 32 * j;
+    qv[j] = (i < nvec) ? __ldg(qrow + i) : make_uint4(0, 0, 0, 0);
+  }
+#pragma unroll
+  for (int j = 0; j < 3; ++j) {
+    const uint32_t w[4] = {qv[j].x, qv[j].y, qv[j].z, qv[j].w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      m = fmaxf(m, fabsf(__uint_as_float(w[k] << 16)));
+      m = fmaxf(m, fabsf(__uint_as_float(w[k] & 0xFFFF0000u)));
+    }
+  }
+  m = warp_max(m);
+  const float alpha = __fdiv_rn(m, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
+  const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f, inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
+  if (lane == 0) { *alpha_out = alpha; *beta_out = beta; }
+#pragma unroll
+  for (int j = 0; j < 3; ++j) {
+    const int i = lane + 32 * j;
+    if (i >= nvec) continue;
+    const uint32_t w[4] = {qv[j].x, qv[j].y, qv[j].z, qv[j].w};
+    uint32_t o1[2] = {0, 0}, o2[2] = {0, 0};
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const float x = (e & 1) ? __uint_as_float(w[e >> 1] & 0xFFFF0000u) : __uint_as_float(w[e >> 1] << 16);
+      int c1 = 0, c2 = 0;
+      if (alpha > 0.0f) {
+        c1 = quant_i8(x, alpha, inv_alpha);
+        const float r = __fmaf_rn(-alpha, static_cast<float>(c1), x);
+        if (beta > 0.0f) c2 = quant_i8(r, beta, inv_beta);
+      }
+      o1[e >> 2] |= static_cast<uint32_t>(c1 & 0xFF) << (8 * (e & 3));
+      o2[e >> 2] |= static_cast<uint32_t>(c2 & 0xFF) << (8 * (e & 3));
+    }
+    const int d = i << 3;                       // eight consecutive bytes stay inside one 16-byte swizzle chunk
+    uint8_t* chunk = img + (d >> 7) * p.Rp * kChunk;
+    *reinterpret_cast<uint2*>(chunk + swz_off(h, d & 127)) = make_uint2(o1[0], o1[1]);
+    *reinterpret_cast<uint2*>(chunk + swz_off(p.HG + h, d & 127)) = make_uint2(o2[0], o2[1]);
+  }
+}
+
 // c1 (Alg. 3 lines 1-2) once per (sequence, KV head, head group) instead of once per context split: the query rows of
 // the group's heads are decomposed into two INT8 components (same bit-exact rule as msd_decompose_int8) and written
 // as the stacked operand image the attention CTAs copy into shared memory with one bulk copy per chunk.  One CTA per
@@ -91,55 +145,7 @@ attn_qstack_kernel(const AttnParams p, uint8_t* __restrict__ q_img, float* __res
   for (int i = threadIdx.x; i < img_bytes / 16; i += blockDim.x) reinterpret_cast<uint4*>(img)[i] = make_uint4(0, 0, 0, 0);
   for (int i = threadIdx.x; i < 2 * p.HG; i += blockDim.x) sc[i] = 0.0f;
   __syncthreads();
-  for (int h = warp; h < nh; h += 8) {
-    const int r_kv = grp * p.HG + h, sq = r_kv / p.Gr;       // row of this KV head -> (query token, head of the group)
-    const uint4* qrow = reinterpret_cast<const uint4*>(
-        p.q + ((static_cast<long long>(b) * p.Sq + sq) * (p.Hkv * p.Gr) + hk * p.Gr + (r_kv - sq * p.Gr)) * p.D);
-    const int nvec = p.D >> 3;                    // 8 BF16 values per 16-byte load (D % 16 == 0, D <= 640)
-    uint4 qv[3];                                  // the whole row stays in registers between the two passes
-    float m = 0.0f;
-#pragma unroll
-    for (int j = 0; j < 3; ++j) {
-      const int i = lane + 32 * j;
-      qv[j] = (i < nvec) ? __ldg(qrow + i) : make_uint4(0, 0, 0, 0);
-    }
-#pragma unroll
-    for (int j = 0; j < 3; ++j) {
-      const uint32_t w[4] = {qv[j].x, qv[j].y, qv[j].z, qv[j].w};
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        m = fmaxf(m, fabsf(__uint_as_float(w[k] << 16)));
-        m = fmaxf(m, fabsf(__uint_as_float(w[k] & 0xFFFF0000u)));
-      }
-    }
-    m = warp_max(m);
-    const float alpha = __fdiv_rn(m, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
-    const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f, inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
-    if (lane == 0) { sc[h] = alpha; sc[p.HG + h] = beta; }
-#pragma unroll
-    for (int j = 0; j < 3; ++j) {
-      const int i = lane + 32 * j;
-      if (i >= nvec) continue;
-      const uint32_t w[4] = {qv[j].x, qv[j].y, qv[j].z, qv[j].w};
-      uint32_t o1[2] = {0, 0}, o2[2] = {0, 0};
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const float x = (e & 1) ? __uint_as_float(w[e >> 1] & 0xFFFF0000u) : __uint_as_float(w[e >> 1] << 16);
-        int c1 = 0, c2 = 0;
-        if (alpha > 0.0f) {
-          c1 = quant_i8(x, alpha, inv_alpha);
-          const float r = __fmaf_rn(-alpha, static_cast<float>(c1), x);
-          if (beta > 0.0f) c2 = quant_i8(r, beta, inv_beta);
-        }
-        o1[e >> 2] |= static_cast<uint32_t>(c1 & 0xFF) << (8 * (e & 3));
-        o2[e >> 2] |= static_cast<uint32_t>(c2 & 0xFF) << (8 * (e & 3));
-      }
-      const int d = i << 3;                       // eight consecutive bytes stay inside one 16-byte swizzle chunk
-      uint8_t* chunk = img + (d >> 7) * p.Rp * kChunk;
-      *reinterpret_cast<uint2*>(chunk + swz_off(h, d & 127)) = make_uint2(o1[0], o1[1]);
-      *reinterpret_cast<uint2*>(chunk + swz_off(p.HG + h, d & 127)) = make_uint2(o2[0], o2[1]);
-    }
-  }
+  for (int h = warp; h < nh; h += 8) attn_decompose_q_row(p, b, hk, grp, h, lane, img, sc + h, sc + p.HG + h);
 }
 
 // kMaxHG: head slots one softmax thread looks after (8 or 16); kNH: heads its code is unrolled for (<= kMaxHG);
@@ -153,6 +159,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], v_full[4], v_empty[4], s_full[2], p_full[2], q_ready, o_full, o_empty;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
+  // Wide head groups (MLA) take the stacked Q operand ready-made from attn_qstack_kernel: decomposing 32 x 576 values
+  // in every context-split CTA cost a sixth of its lifetime.  Narrow ones (GQA) decompose their few rows themselves,
+  // beside the other CTAs of the SM, and save the extra kernel.
+  constexpr bool kQStack = kWG >= 2;
   constexpr int kSlots = kMaxHG * kWG;             // head slots of the stacked operands: rows [0,kSlots) first
   constexpr int kNSW = 4 * kWG;                    // component, rows [kSlots, 2*kSlots) second component
   __shared__ float s_aq[kSlots], s_bq[kSlots];
@@ -207,7 +217,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1);
     // one P barrier per P buffer: the softmax may run one tile ahead of the PV issue, and a single barrier could then
     // be two phases past the one the MMA warp is testing, which a parity test cannot tell from "not yet"
-    mbar_init(&p_full[0], kNSW); mbar_init(&p_full[1], kNSW); mbar_init(&q_ready, 1);
+    mbar_init(&p_full[0], kNSW); mbar_init(&p_full[1], kNSW); mbar_init(&q_ready, kQStack ? 1 : kNSW);
     mbar_init(&o_full, 1); mbar_init(&o_empty, kNSW);
     abort_flag = 0;
     mbar_init_fence();
@@ -215,6 +225,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     tma_prefetch_desc(&tmap_v);
   }
   if (warp == 1) tmem_alloc(&tmem_base_slot, p.tmem_cols);
+  if constexpr (!kQStack) {
+    // zero the stacked Q operand (unused head slots and the padding of the last D chunk must be zero)
+    for (int i = threadIdx.x; i < p.DC * p.Rp * kChunk / 16; i += blockDim.x) reinterpret_cast<uint4*>(sm_q)[i] = make_uint4(0, 0, 0, 0);
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -293,8 +307,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       bool ok = true;
       // the stacked Q operand of this (sequence, KV head, head group) comes ready-made from attn_qstack_kernel, the
       // kernel launched just before this one (the producer's KV loads, which do not depend on it, are already under way)
-      pdl_wait_primary();
-      {
+      if constexpr (kQStack) {
+        pdl_wait_primary();
         const int unit_q = blockIdx.y, chunk_bytes = p.Rp * kChunk;
         mbar_arrive_expect_tx(&q_ready, p.DC * chunk_bytes);
         for (int c = 0; c < p.DC; ++c)
@@ -381,12 +395,18 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const int hh = wi >> 2;                         // which group of head slots this warp looks after
     const int wq = wi & 3;
     const int hs0 = hh * kMaxHG;                    // its first head slot
-    // alpha_Q / beta_Q of this CTA's heads, computed by attn_qstack_kernel (launched just before this kernel)
-    pdl_wait_primary();
-    {
+    if constexpr (kQStack) {
+      // alpha_Q / beta_Q of this CTA's heads, computed by attn_qstack_kernel (launched just before this kernel)
+      pdl_wait_primary();
       const int i = threadIdx.x - 64;
       const float* sc = p.q_scales + static_cast<size_t>(blockIdx.y) * 2 * p.HG;
       if (i < kSlots) { s_aq[i] = __ldg(sc + i); s_bq[i] = __ldg(sc + p.HG + i); }
+    } else {
+      // c1: decompose the query rows of this CTA's heads (one warp per head, round robin) into the stacked operand
+      for (int h = wi; h < nh; h += kNSW) attn_decompose_q_row(p, b, hk, grp, h, lane, sm_q, &s_aq[h], &s_bq[h]);
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&q_ready);         // the stacked Q operand is in shared memory
     }
     named_bar_sync(8, 128 * kWG);                   // s_aq / s_bq visible to all softmax warps
     if (threadIdx.x == 64) attn_mark(p, 3);
@@ -812,11 +832,17 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
     }
   }
   dim3 grid(pl.n_splits, B * Hkv * pl.groups);
-  attn_qstack_kernel<<<B * Hkv * pl.groups, 256, 0, s>>>(p, q_img, q_scales);
-  if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
-  // programmatic dependent of the Q kernel: the CTAs start their KV loads while it runs
-  if (launch_pdl(kernel, grid, dim3(block_threads), pl.smem_bytes, s, getenv("MSD_NO_PDL") == nullptr, tmap_k, tmap_v, p) != cudaSuccess)
-    return MSD_ERR_CUDA;
+  if (block_threads > kAttnThreads) {
+    // wide head groups: the stacked Q operands come from a kernel of their own, the attention kernel is its
+    // programmatic dependent (its CTAs start their KV loads while it runs)
+    attn_qstack_kernel<<<B * Hkv * pl.groups, 256, 0, s>>>(p, q_img, q_scales);
+    if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
+    if (launch_pdl(kernel, grid, dim3(block_threads), pl.smem_bytes, s, getenv("MSD_NO_PDL") == nullptr, tmap_k, tmap_v, p) != cudaSuccess)
+      return MSD_ERR_CUDA;
+  } else {
+    kernel<<<grid, block_threads, pl.smem_bytes, s>>>(tmap_k, tmap_v, p);
+    if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
+  }
   attn_combine_kernel<<<B * Hq, 128, 0, s>>>(p.partial, pl.n_splits, Dv, static_cast<__nv_bfloat16*>(out_bf16), lse, q_len,
                                              Hq / (Hkv * q_len), Hkv);
   return launch_status();
