@@ -391,6 +391,26 @@ def other_configs(torch, binding, device, capture, timed):
                                     "note": "dequant = torch ops (library, several passes over the weights); GEMM = torch.matmul BF16 (library)"}}
     del x, w4, e4, y, wsp, wb, lut
 
+    # W4A16 at the decode sweep's shapes, M = 16 (K split over the CTAs, FP32 partial tiles + reduce kernel)
+    w4d = {}
+    for (N, K) in SHAPES:
+        x = torch.randn((16, K), generator=g, device=device).to(torch.bfloat16)
+        wq = [torch.randint(0, 256, (N, K // 2), generator=g, dtype=torch.uint8, device=device) for _ in range(8)]
+        eq = torch.randint(118, 124, (N, K // 32), generator=g, dtype=torch.uint8, device=device)
+        wsp = binding.workspace(binding.gemm_w4a16_workspace_bytes(16, N, K), device)
+        y = torch.empty((16, N), dtype=torch.bfloat16, device=device)
+        it4 = [0]
+
+        def f_w4d():
+            it4[0] += 1
+            binding.gemm_w4a16(x, wq[it4[0] % 8], eq, ws=wsp, out=y)
+        t = per_call_us(f_w4d, reps=8)
+        b = N * (K // 2 + K // 32)
+        w4d[f"M16_N{N}_K{K}"] = {"us": round(t, 2), "weight_and_scale_gbps": round(b / t / 1e3, 1),
+                                 "frac_of_measured_hbm": round(b / t / 1e3 / peaks["hbm_gbs"], 3)}
+        del x, wq, eq, wsp, y
+    res["w4a16_decode_shapes"] = w4d
+
     # INT8 tensor-peak point: the W8A16 layer at M = 4096 on the first sweep shape (no BASELINE config exercises INT8 prefill)
     M, N, K = 4096, 14336, 4096
     x = torch.randn((M, K), generator=g, device=device).to(torch.bfloat16)
