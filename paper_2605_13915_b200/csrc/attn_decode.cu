@@ -570,7 +570,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           tmem_ld_wait();
 #pragma unroll
           for (int h = 0; h < kNH; ++h)
-            o_run[j][h] = __fmaf_rn(o_run[j][h], resc_cur[h], __fmaf_rn(ap_cur, static_cast<float>(static_cast<int32_t>(v1[h])), bp_cur * static_cast<float>(static_cast<int32_t>(v2[h]))));
+            // alpha_P O1 + beta_P O2 with beta_P = alpha_P / 254: one integer multiply-add and one conversion
+            // (|254 O1 + O2| <= 255 * 128 * 127 * 127 < 2^31)
+            o_run[j][h] = __fmaf_rn(o_run[j][h], resc_cur[h], bp_cur * static_cast<float>(254 * static_cast<int32_t>(v1[h]) + static_cast<int32_t>(v2[h])));
         }
       }
       tc_fence_before();
