@@ -507,16 +507,26 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       beta_p = alpha_p * (1.0f / 254.0f);
       const float inv_a = alpha_p > 0.0f ? __frcp_rn(alpha_p) : 0.0f, inv_b = beta_p > 0.0f ? __frcp_rn(beta_p) : 0.0f;
       uint8_t* pbuf = sm_p + (t & 1) * p.Rp * kChunk;      // PV of tile t-2 (same buffer) finished before merge(t-2)
+      // Shared-memory state: the new running maximum and the rescale factor of head h are the same for every thread of
+      // the warp group; lane h of each warp computes them once and the others fetch them by shuffle (four shared
+      // loads, the maxima and an exponential per head and THREAD before).
+      float mn_lane = 0.0f, resc_lane = 0.0f;
+      if constexpr (kSmemState) {
+        if (lane < kNH) {
+          const float mt = fmaxf(fmaxf(rb[0][lane], rb[1][lane]), fmaxf(rb[2][lane], rb[3][lane]));
+          const float m_old = m_rd[hs0 + lane];
+          mn_lane = fmaxf(m_old, mt);
+          resc_lane = (m_old == -INFINITY) ? 0.0f : ex2_approx(m_old - mn_lane);
+          m_wr[hs0 + lane] = mn_lane;
+        }
+      }
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
         // branch-free: an absent head or a token past the end contributes P = 0 (s is -inf there)
         float mn, resc;
         if constexpr (kSmemState) {
-          const float mt = fmaxf(fmaxf(rb[0][h], rb[1][h]), fmaxf(rb[2][h], rb[3][h]));
-          const float m_old = m_rd[hs0 + h];
-          mn = fmaxf(m_old, mt);
-          resc = (m_old == -INFINITY) ? 0.0f : ex2_approx(m_old - mn);
-          m_wr[hs0 + h] = mn;
+          mn = __shfl_sync(0xffffffffu, mn_lane, h);
+          resc = __shfl_sync(0xffffffffu, resc_lane, h);
         } else {
           mn = mn_t[kSmemState ? 0 : h];
           resc = resc_t[kSmemState ? 0 : h];
