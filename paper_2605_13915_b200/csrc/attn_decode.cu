@@ -535,11 +535,15 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         const float pr = (hs0 + h < nh) ? ex2_approx(s[h] - fmaxf(mn, -1e30f)) : 0.0f;
         l_part[h] = __fmaf_rn(l_part[h], resc, pr);
         const float pt = pr * vs;
-        const int c1 = min(127, __float2int_rn(pt * inv_a));
-        const float r = __fmaf_rn(-alpha_p, static_cast<float>(c1), pt);
-        const int c2 = max(-128, min(127, __float2int_rn(r * inv_b)));
-        pbuf[swz_off(hs0 + h, tl)] = static_cast<uint8_t>(c1);
-        pbuf[swz_off(kSlots + hs0 + h, tl)] = static_cast<uint8_t>(c2);
+        // Two-pass INT8 by the 1.5 * 2^23 trick: adding it rounds to the nearest integer (ties to even) and leaves that
+        // integer in the low mantissa bits, so neither pass needs a float <-> int conversion.  No clamps: P <= 1 and
+        // v_scale <= its tile maximum give pt / alpha_P <= 127, and |r| <= alpha_P / 2 gives |r / beta_P| <= 127.
+        const float kMagic = 12582912.0f;
+        const float u1 = __fmaf_rn(pt, inv_a, kMagic);
+        const float r = __fmaf_rn(-alpha_p, u1 - kMagic, pt);
+        const float u2 = __fmaf_rn(r, inv_b, kMagic);
+        pbuf[swz_off(hs0 + h, tl)] = static_cast<uint8_t>(__float_as_uint(u1));
+        pbuf[swz_off(kSlots + hs0 + h, tl)] = static_cast<uint8_t>(__float_as_uint(u2));
       }
       fence_proxy_async_smem();
       tc_fence_before();
