@@ -519,6 +519,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           resc_lane = (m_old == -INFINITY) ? 0.0f : ex2_approx(m_old - mn_lane);
           m_wr[hs0 + lane] = mn_lane;
         }
+        resc_out[0] = resc_lane;          // lane h carries head h's factor to the merge of this tile
       }
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
@@ -568,8 +569,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
         if constexpr (kSmemState) {
-          const float m_b = s_m[t % 3][hs0 + h], m_a = s_m[(t + 1) % 3][hs0 + h];
-          resc_cur[h] = (m_b == -INFINITY) ? 0.0f : ex2_approx(m_b - m_a);
+          resc_cur[h] = __shfl_sync(0xffffffffu, resc_keep[0], h);       // computed by lane h in the softmax of tile t
         } else {
           resc_cur[h] = resc_keep[h];
         }
@@ -593,10 +593,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       __syncwarp();
       if (lane == 0) mbar_arrive(&o_empty);
       if (threadIdx.x == 64 && t < 6) attn_mark(p, 7 + 4 * t);
-      if constexpr (!kSmemState) {
 #pragma unroll
-        for (int h = 0; h < kNH; ++h) resc_keep[h] = resc_next[h];
-      }
+      for (int h = 0; h < kRegState; ++h) resc_keep[h] = resc_next[h];
       ap_cur = ap_nxt;
       bp_cur = bp_nxt;
     }
