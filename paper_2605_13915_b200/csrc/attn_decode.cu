@@ -425,6 +425,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       l_part[h] = 0.0f;
       if constexpr (kSmemState) {
         s_m[0][hs0 + h] = -INFINITY;
+        if (h == 0) {       // lane l keeps the query scales of head slot hs0 + l (zero for absent heads)
+          aq[0] = (lane < kNH && hs0 + lane < nh) ? s_aq[hs0 + lane] : 0.0f;
+          bq[0] = (lane < kNH && hs0 + lane < nh) ? s_bq[hs0 + lane] : 0.0f;
+        }
       } else {
         m_run[h] = -INFINITY;
         aq[h] = (hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f;
@@ -466,8 +470,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
         for (int h = 0; h < kNH; ++h)
         {
-          const float a_q = kSmemState ? ((hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f) : aq[kSmemState ? 0 : h];
-          const float b_q = kSmemState ? ((hs0 + h < nh) ? s_bq[hs0 + h] : 0.0f) : bq[kSmemState ? 0 : h];
+          // (shared-memory state: lane h holds the scales of head h, see above)
+          const float a_q = kSmemState ? __shfl_sync(0xffffffffu, aq[0], h) : aq[kSmemState ? 0 : h];
+          const float b_q = kSmemState ? __shfl_sync(0xffffffffu, bq[0], h) : bq[kSmemState ? 0 : h];
           bool vh = valid;
           if (p.Sq > 1) vh = valid && tok_rel < L - p.Sq + 1 + (grp * p.HG + hs0 + h) / p.Gr;    // causal among the new tokens
           s[h] = vh ? __fmaf_rn(a_q, static_cast<float>(static_cast<int32_t>(v1[h])), b_q * static_cast<float>(static_cast<int32_t>(v2[h]))) * ks : -INFINITY;
