@@ -445,9 +445,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     float ap_cur = 0.0f, bp_cur = 0.0f, ap_nxt = 0.0f, bp_nxt = 0.0f;
 
     // c3-c5 for tile t: scores -> running max -> P -> two INT8 components into P buffer (t & 1)
-    auto softmax_tile = [&](int t, float (&resc_out)[kRegState], float& alpha_p, float& beta_p) -> bool {
+    // Per-token scales of tile t for this thread's token lane (0 past the end of the split).  They are fetched one tile
+    // ahead: a cold 512-byte run of the scale arrays would otherwise sit on every tile's critical path.
+    auto load_scales = [&](int t, float& ks_out, float& vs_out) {
       const int tok_rel = t_begin + t * kTok + tl;
-      const bool valid = tok_rel < t_end;
+      const bool valid = t < ntiles && tok_rel < t_end;
       long long sidx;
       if constexpr (kPaged) {
         const long long prow = valid ? static_cast<long long>(__ldg(bt + (tok_rel >> p.page_shift))) * p.page + (tok_rel & (p.page - 1)) : 0;
@@ -455,8 +457,17 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       } else {
         sidx = static_cast<long long>(seq0 + tok_rel) * p.Hkv + hk;
       }
-      const float ks = valid ? __ldg(p.k_scale + sidx) * scale2 : 0.0f;
-      const float vs = valid ? __ldg(p.v_scale + sidx) : 0.0f;
+      ks_out = valid ? __ldg(p.k_scale + sidx) : 0.0f;
+      vs_out = valid ? __ldg(p.v_scale + sidx) : 0.0f;
+    };
+    float ks_pre, vs_pre;
+    load_scales(0, ks_pre, vs_pre);
+    auto softmax_tile = [&](int t, float (&resc_out)[kRegState], float& alpha_p, float& beta_p) -> bool {
+      const int tok_rel = t_begin + t * kTok + tl;
+      const bool valid = tok_rel < t_end;
+      const float ks = ks_pre * scale2;
+      const float vs = vs_pre;
+      load_scales(t + 1, ks_pre, vs_pre);
       if (!wait_bounded(&s_full[t & 1], (t >> 1) & 1, abort, p.status)) return false;
       if (threadIdx.x == 64 && t < 6) attn_mark(p, 4 + 4 * t);
       tc_fence_after();
