@@ -710,11 +710,6 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       const long long seg_end = tile_end < blk_end ? tile_end : blk_end;
       const bool complete = (blk == tile_begin) && (seg_end == tile_end);
       const int acc = seg & 1;
-      ok = wait_bounded(&tfull_bar[acc], (seg >> 1) & 1, abort, p.status);
-      if (!ok) break;
-      if (et == 0) { if (seg == 0) trace_mark(p, 8); trace_mark(p, 9); }
-      tc_fence_after();
-      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * p.NB;
       // weight row within its matrix; grouped: also which rows of x / y and which expert's scales this tile is about
       int n = band_row0 + tile * kTileN + r;
       int m_valid = p.M;
@@ -727,7 +722,13 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         sw_row0 = static_cast<long long>(grp.expert[g]) * p.N;
       }
       const bool row_ok = (r < band_h) && (n < p.N);
+      // requested before the wait for the accumulator: a cold read of the scale array would otherwise be the call's tail
       const float sw = (!kBase && row_ok) ? __ldg(p.w_scale + sw_row0 + n) : 0.0f;
+      ok = wait_bounded(&tfull_bar[acc], (seg >> 1) & 1, abort, p.status);
+      if (!ok) break;
+      if (et == 0) { if (seg == 0) trace_mark(p, 8); trace_mark(p, 9); }
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * p.NB;
       bool finish = complete;
       int32_t* acc_tile = nullptr;
       int tok0 = 0, tok1 = p.Mp;
