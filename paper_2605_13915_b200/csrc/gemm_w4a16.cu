@@ -20,18 +20,14 @@
 namespace msd {
 
 constexpr int kW4TileM = 128;
-constexpr int kW4TileN = 256;
 constexpr int kW4BlockK = 256;                                  // elements per stage (128 packed bytes)
 constexpr int kW4ThreadsSf = 352;      // producer, MMA, four epilogue warps, four warps that write the scales into TMEM, scale producer
 constexpr int kW4PairThreads = 320;    // the same without the separate scale producer
 constexpr int kW4ABytes = kW4TileM * 128;                       // 16 KB
-constexpr int kW4BBytes = kW4TileN * 128;                       // 32 KB
 constexpr int kW4SfBytes = 1024 + 1024 + 2048;                  // SFA1, SFA2 (2 k-groups each), SFB (2 row tiles x 2 k-groups)
-constexpr int kW4StageBytes = 2 * kW4ABytes + kW4BBytes + kW4SfBytes;   // 69632
 constexpr int kW4Stages = 3;
 constexpr int kW4StoreBytes = 2048;                              // one epilogue chunk: 32 rows x 64 bytes
 constexpr int kW4TmemCols = 512;
-constexpr int kW4SfCol = 256;                                   // scale columns follow the 256 accumulator columns
 
 struct GemmW4Params {
   int M, N, K;
@@ -319,8 +315,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
       const int split = tile % p.ksplit, tile_mn = tile / p.ksplit;
-        const int mt = p.n_fastest ? tile_mn / p.n_tiles : tile_mn % p.m_tiles, nt = p.n_fastest ? tile_mn % p.n_tiles : tile_mn / p.m_tiles;
-        const int ks0 = split * p.kper, ks1 = ks0 + p.kper < p.kstages ? ks0 + p.kper : p.kstages;
+      const int mt = p.n_fastest ? tile_mn / p.n_tiles : tile_mn % p.m_tiles, nt = p.n_fastest ? tile_mn % p.n_tiles : tile_mn / p.m_tiles;
       const int acc = (kAcc == 2) ? (it & 1) : 0;
       const uint32_t tphase = (kAcc == 2) ? ((it >> 1) & 1) : (it & 1);
       ok = wait_bounded(&tfull_bar[acc], tphase, abort, p.status);
