@@ -3,13 +3,15 @@
 // accumulate into the SAME FP32 tile in TMEM, so the "one add" of the two passes costs nothing and each weight tile
 // is read once for both passes.
 //
-// Tile: 128 activation rows x 224 (default) or 256 weight rows, K walked in stages of 256 elements (128 packed bytes = one 128-byte
-// swizzle row).  Per stage TMA brings the A1, A2 (128 x 128 B) and B (256 x 128 B) tiles, bulk copies bring the scale
-// blocks (512-byte blocks of 128 rows x 4 scales, the layout the shared-memory -> TMEM scale copy expects), the MMA
-// warp copies the scales into TMEM and issues 4 K-steps x 2 passes.  Persistent CTAs walk the tiles with the
-// activation-row index fastest so that concurrent CTAs share weight tiles in L2.
+// Tile: 128 activation rows x 224 (default) or 256 weight rows, K walked in stages of 256 elements (128 packed bytes =
+// one 128-byte swizzle row).  Per stage TMA brings the A1, A2 (up to 128 x 128 B) and B (224/256 x 128 B) tiles and
+// bulk copies bring the scale blocks (512-byte blocks of 128 rows x 4 scales); four warps move the scales from shared
+// memory into TMEM (tcgen05.st), one thread issues 4 K-steps x 2 passes of MMAs.  Persistent CTAs walk the work items
+// (token tile, weight tile, K split) in an order chosen by which operand stays in L2.
 //
-// Warps: 0 = producer, 1 = MMA issuer + TMEM owner, 2..5 = epilogue (FP32 -> BF16/FP32, row-major stores).
+// Warps: 0 = operand producer, 1 = MMA issuer + TMEM owner, 2..5 = epilogue (TMEM -> BF16/FP32 -> swizzled staging
+// buffer -> TMA store), 6..9 = scale warps, 10 = scale producer.  The same kernel serves the grouped
+// (mixture-of-experts) entry point: group g is token tile g.  gemm_w4a16_pair_kernel is the opt-in cta_group::2 variant.
 #include <cuda_bf16.h>
 
 #include <cstdlib>
