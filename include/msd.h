@@ -99,7 +99,8 @@ msd_status_t msd_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64
  * K % 16 == 0; N % 8 == 0 when y is BF16; x, w, y 16-byte aligned.
  * M <= 128 (decode regime): the weight rows sit on the MMA M axis and the weights are streamed once.  M > 128
  * (prefill regime): tiles of 128 tokens x 256 weight rows, both components against the same weight tile, outputs
- * written by TMA stores (N % 4 == 0 also when y is FP32).
+ * written by TMA stores (N % 4 == 0 also when y is FP32); with few output tiles K is split over the CTAs and the FP32
+ * partial results are added in a fixed order (acc_dbg != NULL keeps K unsplit: the accumulators exist only then).
  * workspace: >= msd_gemm_w8a16_workspace_bytes(M,N,K) bytes, 1024-byte aligned.
  */
 size_t msd_gemm_w8a16_workspace_bytes(int64_t M, int64_t N, int64_t K);

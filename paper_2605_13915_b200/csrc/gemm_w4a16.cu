@@ -66,7 +66,7 @@ template <> struct W4GroupArg<true> { using type = GemmW4Groups; };
 
 // Sum of the K-split partial tiles, split 0 first (fixed order: the same inputs give the same bits), rounded once.
 __global__ void __launch_bounds__(256)
-w4_ksplit_reduce_kernel(const float* __restrict__ part, int ksplit, int64_t part_stride, int64_t M, int64_t N, void* __restrict__ y,
+ksplit_reduce_kernel(const float* __restrict__ part, int ksplit, int64_t part_stride, int64_t M, int64_t N, void* __restrict__ y,
                         int ytype) {
   pdl_wait_primary();
   const int64_t total = M * N / 4;                     // N is a multiple of 8
@@ -83,6 +83,16 @@ w4_ksplit_reduce_kernel(const float* __restrict__ part, int ksplit, int64_t part
       reinterpret_cast<float4*>(y)[i] = acc;
     }
   }
+}
+
+msd_status_t launch_ksplit_reduce(const float* part, int ksplit, int64_t part_stride, int64_t M, int64_t N, void* y, int ytype,
+                                  cudaStream_t s, bool pdl) {
+  const int64_t quads = M * N / 4;
+  int64_t blocks = (quads + 255) / 256;
+  if (blocks > 4LL * sm_count()) blocks = 4LL * sm_count();
+  if (blocks < 1) blocks = 1;
+  return launch_pdl(ksplit_reduce_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, s, pdl, part, ksplit, part_stride, M, N, y, ytype) == cudaSuccess
+             ? MSD_OK : MSD_ERR_CUDA;
 }
 
 // Bounded wait for a progress counter of the kernel this one depends on (see GemmW4Params::ready); afterwards the
@@ -845,12 +855,8 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
       : launch_pdl(gemm_w4a16_kernel<224, false>, dim3(pl.grid), dim3(kW4ThreadsSf), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p, GemmW4NoGroups());
   if (le != cudaSuccess) return MSD_ERR_CUDA;
   if (split) {
-    const int64_t quads = M * N / 4;
-    int64_t blocks = (quads + 255) / 256;
-    if (blocks > 4LL * sm_count()) blocks = 4LL * sm_count();
-    if (launch_pdl(w4_ksplit_reduce_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, s, pdl, static_cast<const float*>(part), pl.ksplit,
-                   static_cast<int64_t>(part_rows) * N, M, N, y, static_cast<int>(ytype)) != cudaSuccess)
-      return MSD_ERR_CUDA;
+    const msd_status_t rs = launch_ksplit_reduce(part, pl.ksplit, static_cast<int64_t>(part_rows) * N, M, N, y, static_cast<int>(ytype), s, pdl);
+    if (rs != MSD_OK) return rs;
   }
   return MSD_OK;
 }

@@ -33,6 +33,8 @@ constexpr int kP8TmemCols = 512;
 struct GemmP8Params {
   int M, N, K;
   int m_tiles, n_tiles, kstages;
+  int ksplit, kper;             // K splits per output tile and K stages per split (1, kstages: no split)
+  int part_rows;                // ksplit > 1: rows per split of the FP32 partial-result buffer the tiles are written to
   int n_fastest;                // tile index -> (token tile, weight tile): weight tile fastest (1) or token tile fastest (0)
   const float* alpha;           // [M]
   const float* beta;            // [M]
@@ -71,7 +73,10 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
   volatile int* abort = &abort_flag;
-  const int total_tiles = p.m_tiles * p.n_tiles;
+  // Work items: (token tile, weight tile, K split).  With ksplit > 1 (few output tiles, long K) an item covers kper K
+  // stages and writes s_W (alpha D1 + beta D2) of its K range in FP32 to the partial buffer; a second kernel adds the
+  // splits in a fixed order.
+  const int total_tiles = p.m_tiles * p.n_tiles * p.ksplit;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -79,8 +84,10 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int mt = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles, nt = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
-        for (int ks = 0; ks < p.kstages; ++ks) {
+        const int split = tile % p.ksplit, tile_mn = tile / p.ksplit;
+        const int mt = p.n_fastest ? tile_mn / p.n_tiles : tile_mn % p.m_tiles, nt = p.n_fastest ? tile_mn % p.n_tiles : tile_mn / p.m_tiles;
+        const int ks0 = split * p.kper, ks1 = ks0 + p.kper < p.kstages ? ks0 + p.kper : p.kstages;
+        for (int ks = ks0; ks < ks1; ++ks) {
           ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
           if (!ok) break;
           uint8_t* dst = smem + stage * kP8StageBytes;
@@ -103,7 +110,8 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
         ok = wait_bounded(&tempty_bar, (it & 1) ^ 1, abort, p.status);        // the epilogue has drained both accumulators
         if (!ok) break;
         tc_fence_after();
-        for (int ks = 0; ks < p.kstages; ++ks) {
+        const int ks0 = (tile % p.ksplit) * p.kper, ks1 = ks0 + p.kper < p.kstages ? ks0 + p.kper : p.kstages;
+        for (int ks = ks0; ks < ks1; ++ks) {
           ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
           if (!ok) break;
           tc_fence_after();
@@ -111,7 +119,7 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
           const uint64_t a1d = op_desc + enc, a2d = a1d + (kP8ABytes >> 4), bd = a1d + (2 * kP8ABytes >> 4);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {                    // 32 elements (32 bytes) per MMA
-            const uint32_t acc = (ks > 0 || kk > 0) ? 1u : 0u;
+            const uint32_t acc = (ks > ks0 || kk > 0) ? 1u : 0u;
             mma_i8(tmem_base, a1d + 2 * kk, bd + 2 * kk, idesc, acc);
             mma_i8(tmem_base + kP8TileN, a2d + 2 * kk, bd + 2 * kk, idesc, acc);
           }
@@ -138,7 +146,8 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
     // Column scales: every lane needs the same scales of a chunk.  Lane l loads the scale of the chunk's l-th column
     // one chunk ahead and the lanes fetch them from one another by shuffles.
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-      const int mt = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles, nt = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
+      const int split = tile % p.ksplit, tile_mn = tile / p.ksplit;
+        const int mt = p.n_fastest ? tile_mn / p.n_tiles : tile_mn % p.m_tiles, nt = p.n_fastest ? tile_mn % p.n_tiles : tile_mn / p.m_tiles;
       const int row0 = mt * kP8TileM + quad * 32, row = row0 + lane;
       const float a_i = row < p.M ? __ldg(p.alpha + row) : 0.0f, b_i = row < p.M ? __ldg(p.beta + row) : 0.0f;
       const int col_base = nt * kP8TileN + part * 64;
@@ -214,7 +223,7 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          tma_store_2d(&tmap_y, col, row0, sb);
+          tma_store_2d(&tmap_y, col, row0 + split * p.part_rows, sb);
           bulk_commit_group();
         }
       }
@@ -231,8 +240,8 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
 }
 
 struct GemmP8Plan {
-  int m_tiles, n_tiles, kstages, grid;
-  size_t off_q1, off_q2, off_alpha, off_beta, bytes;
+  int m_tiles, n_tiles, kstages, grid, ksplit, kper;
+  size_t off_q1, off_q2, off_alpha, off_beta, off_part, bytes;
 };
 
 static GemmP8Plan plan_p8(int64_t M, int64_t N, int64_t K) {
@@ -241,12 +250,28 @@ static GemmP8Plan plan_p8(int64_t M, int64_t N, int64_t K) {
   pl.n_tiles = static_cast<int>((N + kP8TileN - 1) / kP8TileN);
   pl.kstages = static_cast<int>((K + kP8BlockK - 1) / kP8BlockK);
   const long long tiles = static_cast<long long>(pl.m_tiles) * pl.n_tiles;
-  pl.grid = static_cast<int>(tiles < sm_count() ? tiles : sm_count());
+  // Few output tiles and a long K (a few hundred rows on a narrow layer): split K so that there is about one work item
+  // per SM, each at least eight stages long; the FP32 partial results are added by a second kernel.
+  pl.ksplit = 1;
+  pl.kper = pl.kstages;
+  {
+    const char* se = getenv("MSD_P8_KSPLIT");
+    long long want = se ? atoi(se) : (2 * tiles <= sm_count() ? sm_count() / tiles : 1);
+    if (want > pl.kstages / 8) want = pl.kstages / 8;
+    if (want > 1) {
+      pl.kper = static_cast<int>((pl.kstages + want - 1) / want);
+      pl.ksplit = (pl.kstages + pl.kper - 1) / pl.kper;
+    }
+  }
+  const long long items = tiles * pl.ksplit;
+  pl.grid = static_cast<int>(items < sm_count() ? items : sm_count());
   size_t off = 0;
   pl.off_q1 = off;    off = round_up(off + static_cast<size_t>(M) * K, 1024);
   pl.off_q2 = off;    off = round_up(off + static_cast<size_t>(M) * K, 1024);
   pl.off_alpha = off; off = round_up(off + static_cast<size_t>(M) * sizeof(float), 1024);
   pl.off_beta = off;  off = round_up(off + static_cast<size_t>(M) * sizeof(float), 1024);
+  pl.off_part = off;
+  if (pl.ksplit > 1) off = round_up(off + static_cast<size_t>(pl.ksplit) * pl.m_tiles * kP8TileM * N * sizeof(float), 1024);
   pl.bytes = off;
   return pl;
 }
@@ -270,19 +295,27 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
   msd_status_t st = launch_decompose_int8(x_bf16, M, K, K, q1, q2, alpha, beta, c1, c2, s);
   if (st != MSD_OK) return st;
 
+  // with a K split (not when the INT32 accumulators are asked for: they exist only unsplit) the kernel writes FP32
+  // partial results, split s at rows s * part_rows ..., and the reduce kernel produces y
+  const bool split = pl.ksplit > 1 && acc_dbg == nullptr;
+  const int ksplit = split ? pl.ksplit : 1, kper = split ? pl.kper : pl.kstages;
+  float* part = reinterpret_cast<float*>(ws + pl.off_part);
+  const uint64_t part_rows = static_cast<uint64_t>(pl.m_tiles) * kP8TileM;
   CUtensorMap tmap_a1, tmap_a2, tmap_b, tmap_y;
-  const bool ybf = ytype == MSD_OUT_BF16;
+  const bool ybf = !split && ytype == MSD_OUT_BF16;
   if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, K, M, K, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, q2, K, M, K, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kP8BlockK, kP8TileN, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, static_cast<uint64_t>(N),
-                      static_cast<uint64_t>(M), static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+      !encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, split ? static_cast<void*>(part) : y,
+                      static_cast<uint64_t>(N), split ? part_rows * ksplit : static_cast<uint64_t>(M),
+                      static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
     return MSD_ERR_CUDA;
 
   GemmP8Params p;
   p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.kstages = pl.kstages;
-  p.alpha = alpha; p.beta = beta; p.w_scale = w_scale; p.acc_dbg = acc_dbg; p.ytype = ytype; p.status = status;
+  p.alpha = alpha; p.beta = beta; p.w_scale = w_scale; p.acc_dbg = acc_dbg; p.ytype = split ? MSD_OUT_FP32 : ytype; p.status = status;
+  p.ksplit = ksplit; p.kper = kper; p.part_rows = static_cast<int>(part_rows);
   {
     // A wave of CTAs either shares a few weight tiles and sweeps the token tiles (token tile fastest) or the other way
     // round; the operand that is swept should be the one that stays in L2 (40 MB assumed usable for it).
@@ -299,8 +332,11 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
     attr_done = true;
   }
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  if (launch_pdl(gemm_w8a16_prefill_kernel, dim3(pl.grid), dim3(kP8Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p) != cudaSuccess)
+  const long long items = static_cast<long long>(pl.m_tiles) * pl.n_tiles * ksplit;
+  const int grid = static_cast<int>(items < sm_count() ? items : sm_count());
+  if (launch_pdl(gemm_w8a16_prefill_kernel, dim3(grid), dim3(kP8Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p) != cudaSuccess)
     return MSD_ERR_CUDA;
+  if (split) return launch_ksplit_reduce(part, ksplit, static_cast<int64_t>(part_rows) * N, M, N, y, ytype, s, pdl);
   return MSD_OK;
 }
 

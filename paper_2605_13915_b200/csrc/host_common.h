@@ -67,6 +67,11 @@ msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int
                                    float* alpha, float* beta, float c1, float c2, cudaStream_t stream);
 inline float scaling_c1(msd_scaling_t s) { return s == MSD_SCALING_FRACTIONAL ? 127.49f : 127.0f; }
 inline float scaling_c2(msd_scaling_t s) { return s == MSD_SCALING_FRACTIONAL ? 254.98f : 254.0f; }
+// Sum of K-split FP32 partial results part[s * part_stride + i], s = 0 .. ksplit-1 in that order, rounded once to y
+// (gemm_w4a16.cu; N a multiple of 4).
+msd_status_t launch_ksplit_reduce(const float* part, int ksplit, int64_t part_stride, int64_t M, int64_t N, void* y, int ytype,
+                                  cudaStream_t s, bool pdl);
+
 // W8A16 layer for M > 128 rows (gemm_w8a16_prefill.cu); arguments checked by the caller.
 size_t w8_prefill_workspace_bytes(int64_t M, int64_t N, int64_t K);
 msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N, int64_t K,

@@ -235,3 +235,19 @@ def test_prefill_full_size_sampled():
     slack = np.abs(ref) * 2.0 ** -8
     n = np.linalg.norm(ref, axis=-1, keepdims=True)      # norm over the sampled columns only: smaller, so stricter
     assert np.all(np.abs(got - ref) <= TOL * n + slack)
+
+
+@pytest.mark.parametrize("M,N,K", [(256, 512, 4096), (400, 264, 2176), (129, 1032, 8192)])
+def test_prefill_regime_with_k_split(M, N, K):
+    """A few hundred rows on a narrow layer: few output tiles, so the K stages are split over the CTAs, every work item
+    writes s_W (alpha D1 + beta D2) of its K range in FP32 and a second kernel adds the splits (the INT32 accumulators
+    are not available in this mode, so outputs only).  Ragged token and weight tiles, a K that is not a multiple of the
+    split, FP32 and BF16 outputs."""
+    c = inputs.gemm_w8_case(M, N, K, seed=9)
+    ref = oracle.gemm_w8a16(c.x, c.w, c.w_scale, "f64")
+    y = _run(c, torch.float32, want_acc=False)
+    assert rel_row_err(y.cpu().numpy(), ref).max() <= TOL
+    yb = _run(c, torch.bfloat16, want_acc=False)
+    got = oracle.bf16_bits_to_f64(bf16_bits(yb))
+    n = np.linalg.norm(ref, axis=-1, keepdims=True)
+    assert np.all(np.abs(got - ref) <= TOL * n + np.abs(ref) * 2.0 ** -8 + 1e-30)
