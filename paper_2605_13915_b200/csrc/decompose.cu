@@ -103,7 +103,8 @@ decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, i
   const int kblocks = K >> 5;
   const int64_t nblocks = M * kblocks;
   if (static_cast<int>(blockIdx.x) < rl.blocks) {
-    sf_relayout(rl, static_cast<int64_t>(blockIdx.x) * kMxThreads + threadIdx.x, static_cast<int64_t>(rl.blocks) * kMxThreads);
+    __shared__ uint32_t sm_rl[kSfRelayoutSmemWords];
+    sf_relayout(rl, blockIdx.x, rl.blocks, sm_rl);
     if (ready) {
       __syncthreads();
       if (threadIdx.x == 0) { __threadfence(); atomicAdd(&ready[(M + 127) >> 7], 1u); }
@@ -224,8 +225,7 @@ msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, in
   SfRelayout rl = {};
   if (relayout) {
     rl = *relayout;
-    const int64_t chunks = static_cast<int64_t>(rl.row_blocks) * rl.sf_kgroups * 32 * (rl.matrices > 1 ? rl.matrices : 1);
-    const int64_t rb = (chunks + kMxThreads - 1) / kMxThreads;
+    const int64_t rb = static_cast<int64_t>(rl.row_blocks) * ((rl.sf_kgroups + 31) / 32) * (rl.matrices > 1 ? rl.matrices : 1);   // units
     rl.blocks = static_cast<int>(rb < rl_per_sm * sm_count() ? rb : rl_per_sm * sm_count());
     relayout->blocks = rl.blocks;
   }

@@ -65,7 +65,8 @@ decompose_e1m2_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, in
                       const SfRelayout rl) {
   pdl_launch_dependents();
   if (static_cast<int>(blockIdx.x) < rl.blocks) {          // the first CTAs bring the weight scales into the blocked layout
-    sf_relayout(rl, static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x, static_cast<int64_t>(rl.blocks) * 256);
+    __shared__ uint32_t sm_rl[kSfRelayoutSmemWords];
+    sf_relayout(rl, blockIdx.x, rl.blocks, sm_rl);
     return;
   }
   const int kblocks = K >> 5;
@@ -369,8 +370,7 @@ static msd_status_t launch_decompose_e1m2(const void* x_bf16, int64_t M, int64_t
   SfRelayout rl = {};
   if (relayout) {
     rl = *relayout;
-    const int64_t chunks = static_cast<int64_t>(rl.row_blocks) * rl.sf_kgroups * 32;
-    const int64_t rb = (chunks + 255) / 256;
+    const int64_t rb = static_cast<int64_t>(rl.row_blocks) * ((rl.sf_kgroups + 31) / 32);      // units of 128 rows x 32 K groups
     rl.blocks = static_cast<int>(rb < 4 * sm_count() ? rb : 4 * sm_count());
   }
   const int64_t nblocks = M * (K >> 5);
