@@ -514,14 +514,14 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
         const int acc = (kAcc == 2) ? (it & 1) : 0;
         const uint32_t tphase = (kAcc == 2) ? ((it >> 1) & 1) : (it & 1);
         const uint32_t d_tmem = tmem_base + acc * kTN;
-        ok = wait_bounded_cluster(&tempty_bar[acc], tphase ^ 1, abort, p.status);   // both epilogues have drained this accumulator
+        ok = wait_bounded(&tempty_bar[acc], tphase ^ 1, abort, p.status);   // both epilogues have drained this accumulator
         if (!ok) break;
         tc_fence_after();
         for (int ks = 0; ks < p.kstages; ++ks, ++nstage) {
           const int set = nstage & 1;
-          ok = wait_bounded_cluster(&full_bar[stage], phase, abort, p.status);
+          ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
           if (!ok) break;
-          ok = wait_bounded_cluster(&sf_ready[set], (nstage >> 1) & 1, abort, p.status);
+          ok = wait_bounded(&sf_ready[set], (nstage >> 1) & 1, abort, p.status);
           if (!ok) break;
           tc_fence_after();
           const uint64_t enc = static_cast<uint64_t>(smem_u32(smem + stage * kStageBytes) >> 4);
@@ -573,7 +573,7 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
         tmem_st_wait();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(leader_ready[set]);
+        if (lane == 0) mbar_arrive_remote(leader_ready[set]);
         if (++stage == kW4PairStages) { stage = 0; phase ^= 1; }
       }
     }
@@ -620,7 +620,7 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(leader_tempty[acc]);
+      if (lane == 0) mbar_arrive_remote(leader_tempty[acc]);
     }
   }
 

@@ -116,6 +116,12 @@ __device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.ac
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t caddr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(caddr) : "memory");
 }
+// The same arrival with the default (CTA-scope release) semantics, for hand-offs whose data are tensor-memory or
+// tensor-core operations ordered by tcgen05.fence on both sides (the CTA-pair kernel): a cluster-scope release on every
+// arrival and a cluster-scope acquire on every poll cost that kernel most of a microsecond per pipeline stage.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t caddr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(caddr) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
