@@ -24,7 +24,7 @@ namespace msd {
 constexpr int kW4TileM = 128;
 constexpr int kW4BlockK = 256;                                  // elements per stage (128 packed bytes)
 constexpr int kW4ThreadsSf = 352;      // producer, MMA, four epilogue warps, four warps that write the scales into TMEM, scale producer
-constexpr int kW4PairThreads = 320;    // the same without the separate scale producer
+constexpr int kW4PairThreads = 352;    // the CTA-pair kernel has the same warp roles
 constexpr int kW4ABytes = kW4TileM * 128;                       // 16 KB
 constexpr int kW4SfBytes = 1024 + 1024 + 2048;                  // SFA1, SFA2 (2 k-groups each), SFB (2 row tiles x 2 k-groups)
 constexpr int kW4Stages = 3;
@@ -432,7 +432,8 @@ constexpr int kW4PairStages = 4;
 template <int kTN>
 __global__ void __launch_bounds__(kW4PairThreads, 1)
 gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
-                       const __grid_constant__ CUtensorMap tmap_bh, const GemmW4Params p) {
+                       const __grid_constant__ CUtensorMap tmap_bh, const __grid_constant__ CUtensorMap tmap_y,
+                       const GemmW4Params p) {
   constexpr int kBHalfBytes = (kTN / 2) * 128;
   constexpr int kOpBytes = 2 * kW4ABytes + kBHalfBytes;             // operand bytes per CTA and stage
   constexpr int kStageBytes = kOpBytes + kW4SfBytes;
@@ -473,7 +474,8 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
   const int total_tiles = m_pairs * p.n_tiles;
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
 
-  if (warp == 0) {
+  if (warp == 0 || warp == 10) {
+    // two producer threads per CTA: warp 0 the operand tiles, warp 10 the scale blocks (see the single-CTA kernel)
     if (lane == 0) {
       pdl_wait_primary();           // components and blocked scales come from the kernels launched just before
       int stage = 0; uint32_t phase = 0;
@@ -484,20 +486,23 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
         for (int ks = 0; ks < p.kstages; ++ks) {
           ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
           if (!ok) break;
-          // the leader's barrier counts the operand bytes of both CTAs
-          if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * kOpBytes);
-          const uint32_t bar = mapa_shared(smem_u32(&full_bar[stage]), 0);
           uint8_t* dst = smem + stage * kStageBytes;
-          tma_load_2d_pair(dst, &tmap_a1, ks * 128, mt * kW4TileM, bar);
-          tma_load_2d_pair(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, bar);
-          tma_load_2d_pair(dst + 2 * kW4ABytes, &tmap_bh, ks * 128, nt * kTN + static_cast<int>(rank) * (kTN / 2), bar);
-          uint8_t* sf = dst + kOpBytes;
-          mbar_arrive_expect_tx(&sf_full[stage], kW4SfBytes);
-          const size_t a_off = (static_cast<size_t>(mt_sf) * p.sf_kgroups + 2 * ks) * 512;
-          bulk_load(sf, p.sfa1 + a_off, 1024, &sf_full[stage]);
-          bulk_load(sf + 1024, p.sfa2 + a_off, 1024, &sf_full[stage]);
-          bulk_load(sf + 2048, p.sfb + (static_cast<size_t>(2 * nt) * p.sf_kgroups + 2 * ks) * 512, 1024, &sf_full[stage]);
-          bulk_load(sf + 3072, p.sfb + (static_cast<size_t>(2 * nt + 1) * p.sf_kgroups + 2 * ks) * 512, 1024, &sf_full[stage]);
+          if (warp == 0) {
+            // the leader's barrier counts the operand bytes of both CTAs
+            if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * kOpBytes);
+            const uint32_t bar = mapa_shared(smem_u32(&full_bar[stage]), 0);
+            tma_load_2d_pair(dst, &tmap_a1, ks * 128, mt * kW4TileM, bar);
+            tma_load_2d_pair(dst + kW4ABytes, &tmap_a2, ks * 128, mt * kW4TileM, bar);
+            tma_load_2d_pair(dst + 2 * kW4ABytes, &tmap_bh, ks * 128, nt * kTN + static_cast<int>(rank) * (kTN / 2), bar);
+          } else {
+            uint8_t* sf = dst + kOpBytes;
+            mbar_arrive_expect_tx(&sf_full[stage], kW4SfBytes);
+            const size_t a_off = (static_cast<size_t>(mt_sf) * p.sf_kgroups + 2 * ks) * 512;
+            bulk_load(sf, p.sfa1 + a_off, 1024, &sf_full[stage]);
+            bulk_load(sf + 1024, p.sfa2 + a_off, 1024, &sf_full[stage]);
+            bulk_load(sf + 2048, p.sfb + (static_cast<size_t>(2 * nt) * p.sf_kgroups + 2 * ks) * 512, 1024, &sf_full[stage]);
+            bulk_load(sf + 3072, p.sfb + (static_cast<size_t>(2 * nt + 1) * p.sf_kgroups + 2 * ks) * 512, 1024, &sf_full[stage]);
+          }
           if (++stage == kW4PairStages) { stage = 0; phase ^= 1; }
         }
       }
@@ -544,7 +549,7 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
         tc_commit_pair(&tfull_bar[acc], 3);
       }
     }
-  } else if (warp >= 6) {
+  } else if (warp >= 6) {      // (warp 10 went the producers' way above)
     // Scale warps: each CTA writes its own TMEM (its activation rows' scales and all of the weight tile's).
     const int quad = warp & 3;
     const uint32_t leader_ready[2] = {mapa_shared(smem_u32(&sf_ready[0]), 0), mapa_shared(smem_u32(&sf_ready[1]), 0)};
@@ -578,9 +583,12 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
       }
     }
   } else {
+    // Epilogue as in the single-CTA kernel: TMEM -> registers -> (BF16) -> swizzled staging buffer -> TMA store.
     const int quad = warp & 3;
-    const int r = quad * 32 + lane;
-    int it = 0;
+    uint8_t* stage_buf = smem + kW4PairStages * kStageBytes + quad * (2 * kW4StoreBytes);
+    const int ccols = (p.ytype == MSD_OUT_BF16) ? 32 : 16;
+    const uint32_t swz = static_cast<uint32_t>((lane >> 1) & 3);
+    int it = 0, buf = 0;
     bool ok = true;
     const uint32_t leader_tempty[2] = {mapa_shared(smem_u32(&tempty_bar[0]), 0), mapa_shared(smem_u32(&tempty_bar[1]), 0)};
     for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++it) {
@@ -590,38 +598,51 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
       ok = wait_bounded(&tfull_bar[acc], tphase, abort, p.status);
       if (!ok) break;
       tc_fence_after();
-      const int row = mt * kW4TileM + r;
+      const int row0 = mt * kW4TileM + quad * 32;
       const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * kTN;
-      for (int c0 = 0; c0 < kTN; c0 += 16) {
-        uint32_t v[16];
-        tmem_ld16(trow + c0, v);
-        tmem_ld_wait();
-        const int col = nt * kTN + c0;
-        if (row < p.M && col < p.N) {
-          if (p.ytype == MSD_OUT_BF16) {
-            uint32_t o[8];
+      const int cols_here = p.N - nt * kTN < kTN ? p.N - nt * kTN : kTN;
+      const int cend = row0 < p.M ? cols_here : 0;
+      if (cend == 0) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_remote(leader_tempty[acc]);
+      }
+      for (int c0 = 0; c0 < cend; c0 += ccols, buf ^= 1) {
+        uint32_t o[16];
+        if (p.ytype == MSD_OUT_BF16) {
+          uint32_t v[32];
+          tmem_ld32(trow + c0, v);
+          tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-              o[j] = *reinterpret_cast<const uint32_t*>(&h);
-            }
-            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.y) + static_cast<long long>(row) * p.N + col;
-            if (col + 16 <= p.N) {
-              reinterpret_cast<uint4*>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
-              reinterpret_cast<uint4*>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
-            } else {
-              for (int j = 0; j < 16 && col + j < p.N; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
-            }
-          } else {
-            float* dst = static_cast<float*>(p.y) + static_cast<long long>(row) * p.N + col;
-            for (int j = 0; j < 16 && col + j < p.N; ++j) dst[j] = __uint_as_float(v[j]);
+          for (int j = 0; j < 16; ++j) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+            o[j] = *reinterpret_cast<const uint32_t*>(&h);
           }
+        } else {
+          tmem_ld16(trow + c0, o);
+          tmem_ld_wait();
+        }
+        if (c0 + ccols >= cend) {                   // all that is needed of this accumulator is in registers
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_remote(leader_tempty[acc]);
+        }
+        uint8_t* sb = stage_buf + buf * kW4StoreBytes;
+        if (lane == 0) bulk_wait_group_read<1>();    // the store that read this buffer two chunks ago is done with it
+        __syncwarp();
+        uint8_t* srow = sb + lane * 64;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          *reinterpret_cast<uint4*>(srow + ((static_cast<uint32_t>(j) ^ swz) << 4)) = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_2d(&tmap_y, nt * kTN + c0, row0, sb);
+          bulk_commit_group();
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_remote(leader_tempty[acc]);
     }
+    if (lane == 0) bulk_wait_group<0>();            // every store has been written before the CTA goes away
   }
 
   // Neither CTA leaves while the other may still signal its barriers or (through the pair MMAs) read its shared memory.
@@ -641,21 +662,28 @@ struct GemmW4Plan {
   size_t off_q1, off_q2, off_sfa1, off_sfa2, off_sfb, off_ready, off_part, bytes;
 };
 
-// Weight rows per tile: 224 (two accumulators) unless MSD_W4_TILEN=256.
-static int w4_tile_n() {
-  const char* e = getenv("MSD_W4_TILEN");
-  return (e && atoi(e) == 256) ? 256 : 224;
+// The CTA-pair kernel (256 tokens x 256 weight rows per pair of CTAs: half the weight tile per CTA, so less shared-memory
+// traffic per MMA, and four stages) takes the prefill shapes: at least two token tiles, more tiles than SMs, and both
+// components of x small enough to stay in L2 while the pairs sweep the token tiles (its tile order is token tile fastest).
+// MSD_W4_PAIR=0/1 forces the choice.
+static bool w4_use_pair(int64_t M, int64_t N, int64_t K) {
+  const char* pe = getenv("MSD_W4_PAIR");
+  if (pe) return atoi(pe) != 0;
+  const int64_t m_tiles = (M + kW4TileM - 1) / kW4TileM, n_tiles = (N + 255) / 256;
+  return m_tiles >= 2 && m_tiles * n_tiles > 2 * sm_count() && static_cast<double>(M) * K <= 40.0 * 1024 * 1024;
 }
 
-// The CTA-pair kernel is opt-in (MSD_W4_PAIR=1): measured slower than the single-CTA kernel.
-static bool w4_use_pair(int) {
-  const char* pe = getenv("MSD_W4_PAIR");
-  return pe && atoi(pe) != 0;
+// Weight rows per tile: MSD_W4_TILEN (224 or 256) if set; else 256 for the CTA-pair kernel (one accumulator) and 224 for
+// the single-CTA kernel (two accumulators: the epilogue of a tile overlaps the MMAs of the next).
+static int w4_tile_n(bool pair = false) {
+  const char* e = getenv("MSD_W4_TILEN");
+  if (e) return atoi(e) == 256 ? 256 : 224;
+  return pair ? 256 : 224;
 }
 
 static GemmW4Plan plan_w4(int64_t M, int64_t N, int64_t K) {
   GemmW4Plan pl;
-  const int tile_n = w4_tile_n();
+  const int tile_n = w4_tile_n(w4_use_pair(M, N, K));
   pl.tile_n = tile_n;
   pl.m_tiles = static_cast<int>((M + kW4TileM - 1) / kW4TileM);
   pl.n_tiles = static_cast<int>((N + tile_n - 1) / tile_n);
@@ -767,7 +795,7 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   // decomposed.  Measured: the GEMM's CTAs do enter 5-9 us after the decomposition starts, but the decomposition,
   // held to two CTAs per SM so that both fit, then takes 47 instead of 25 us and the GEMM beside it is slower by as
   // much as the earlier start gains.
-  const bool use_pair = w4_use_pair(pl.m_tiles);
+  const bool use_pair = w4_use_pair(M, N, K);
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
   const char* ove = getenv("MSD_W4_OVERLAP");
   const bool overlap = !use_pair && pdl && ove && atoi(ove) != 0;
@@ -806,13 +834,23 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
     p.n_fastest = oe ? (atoi(oe) != 0) : n_fast;
   }
 
+  // With a K split the kernel writes FP32 partial tiles (split s at rows s * part_rows ...) and a second kernel adds them.
+  CUtensorMap tmap_y;
+  const bool split = pl.ksplit > 1 && !use_pair;        // the CTA-pair kernel does not split K
+  const bool ybf = !split && ytype == MSD_OUT_BF16;
+  float* part = reinterpret_cast<float*>(ws + pl.off_part);
+  const uint64_t part_rows = static_cast<uint64_t>(pl.m_tiles) * kW4TileM;
+  if (!encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, split ? static_cast<void*>(part) : y,
+                      static_cast<uint64_t>(N), split ? part_rows * pl.ksplit : static_cast<uint64_t>(M),
+                      static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+    return MSD_ERR_CUDA;
   if (use_pair) {
     // CTA pairs: each CTA loads half of the weight tile's rows
     CUtensorMap tmap_bh;
     if (!encode_tmap_2d(&tmap_bh, CU_TENSOR_MAP_DATA_TYPE_UINT8, w_fp4, kb, N, kb, 128, static_cast<uint32_t>(pl.tile_n / 2),
                         CU_TENSOR_MAP_SWIZZLE_128B))
       return MSD_ERR_CUDA;
-    const size_t smem_pair = static_cast<size_t>(kW4PairStages) * (2 * kW4ABytes + (pl.tile_n / 2) * 128 + kW4SfBytes) + 1024;
+    const size_t smem_pair = static_cast<size_t>(kW4PairStages) * (2 * kW4ABytes + (pl.tile_n / 2) * 128 + kW4SfBytes) + 8 * kW4StoreBytes + 1024;
     static bool attr_pair_done = false;
     if (!attr_pair_done) {
       if (cudaFuncSetAttribute(gemm_w4a16_pair_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
@@ -824,21 +862,11 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
     int clusters = sm_count() / 2;
     if (clusters > pair_tiles) clusters = pair_tiles;
     const cudaError_t pe = pl.tile_n == 256
-        ? launch_pdl_cluster(gemm_w4a16_pair_kernel<256>, dim3(2 * clusters), dim3(kW4PairThreads), smem_pair, s, pdl, 2u, tmap_a1, tmap_a2, tmap_bh, p)
-        : launch_pdl_cluster(gemm_w4a16_pair_kernel<224>, dim3(2 * clusters), dim3(kW4PairThreads), smem_pair, s, pdl, 2u, tmap_a1, tmap_a2, tmap_bh, p);
+        ? launch_pdl_cluster(gemm_w4a16_pair_kernel<256>, dim3(2 * clusters), dim3(kW4PairThreads), smem_pair, s, pdl, 2u, tmap_a1, tmap_a2, tmap_bh, tmap_y, p)
+        : launch_pdl_cluster(gemm_w4a16_pair_kernel<224>, dim3(2 * clusters), dim3(kW4PairThreads), smem_pair, s, pdl, 2u, tmap_a1, tmap_a2, tmap_bh, tmap_y, p);
     if (pe != cudaSuccess) return MSD_ERR_CUDA;
     return MSD_OK;
   }
-  // With a K split the kernel writes FP32 partial tiles (split s at rows s * part_rows ...) and a second kernel adds them.
-  CUtensorMap tmap_y;
-  const bool split = pl.ksplit > 1;
-  const bool ybf = !split && ytype == MSD_OUT_BF16;
-  float* part = reinterpret_cast<float*>(ws + pl.off_part);
-  const uint64_t part_rows = static_cast<uint64_t>(pl.m_tiles) * kW4TileM;
-  if (!encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, split ? static_cast<void*>(part) : y,
-                      static_cast<uint64_t>(N), split ? part_rows * pl.ksplit : static_cast<uint64_t>(M),
-                      static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
-    return MSD_ERR_CUDA;
   if (split) p.ytype = MSD_OUT_FP32;
   p.ksplit = pl.ksplit; p.kper = pl.kper; p.part_rows = static_cast<int>(part_rows);
   p.a_rows = pl.a_rows; p.nstages = pl.nstages;
