@@ -481,7 +481,7 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
-        const int mt = 2 * (tile % m_pairs) + static_cast<int>(rank), nt = tile / m_pairs;
+        const int mt = 2 * (p.n_fastest ? tile / p.n_tiles : tile % m_pairs) + static_cast<int>(rank), nt = p.n_fastest ? tile % p.n_tiles : tile / m_pairs;
         const int mt_sf = mt < p.m_tiles ? mt : p.m_tiles - 1;       // the odd last pair: rows past M are zero-filled anyway
         for (int ks = 0; ks < p.kstages; ++ks) {
           ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
@@ -592,7 +592,7 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
     bool ok = true;
     const uint32_t leader_tempty[2] = {mapa_shared(smem_u32(&tempty_bar[0]), 0), mapa_shared(smem_u32(&tempty_bar[1]), 0)};
     for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++it) {
-      const int mt = 2 * (tile % m_pairs) + static_cast<int>(rank), nt = tile / m_pairs;
+      const int mt = 2 * (p.n_fastest ? tile / p.n_tiles : tile % m_pairs) + static_cast<int>(rank), nt = p.n_fastest ? tile % p.n_tiles : tile / m_pairs;
       const int acc = (kAcc == 2) ? (it & 1) : 0;
       const uint32_t tphase = (kAcc == 2) ? ((it >> 1) & 1) : (it & 1);
       ok = wait_bounded(&tfull_bar[acc], tphase, abort, p.status);
@@ -663,14 +663,13 @@ struct GemmW4Plan {
 };
 
 // The CTA-pair kernel (256 tokens x 256 weight rows per pair of CTAs: half the weight tile per CTA, so less shared-memory
-// traffic per MMA, and four stages) takes the prefill shapes: at least two token tiles, more tiles than SMs, and both
-// components of x small enough to stay in L2 while the pairs sweep the token tiles (its tile order is token tile fastest).
+// traffic per MMA, and four stages) takes the prefill shapes: at least two token tiles and more tiles than SMs.
 // MSD_W4_PAIR=0/1 forces the choice.
 static bool w4_use_pair(int64_t M, int64_t N, int64_t K) {
   const char* pe = getenv("MSD_W4_PAIR");
   if (pe) return atoi(pe) != 0;
   const int64_t m_tiles = (M + kW4TileM - 1) / kW4TileM, n_tiles = (N + 255) / 256;
-  return m_tiles >= 2 && m_tiles * n_tiles > 2 * sm_count() && static_cast<double>(M) * K <= 40.0 * 1024 * 1024;
+  return m_tiles >= 2 && m_tiles * n_tiles > 2 * sm_count();
 }
 
 // Weight rows per tile: MSD_W4_TILEN (224 or 256) if set; else 256 for the CTA-pair kernel (one accumulator) and 224 for
