@@ -663,13 +663,14 @@ struct GemmW4Plan {
 };
 
 // The CTA-pair kernel (256 tokens x 256 weight rows per pair of CTAs: half the weight tile per CTA, so less shared-memory
-// traffic per MMA, and four stages) takes the prefill shapes: at least two token tiles and more tiles than SMs.
+// traffic per MMA, and four stages) takes the prefill shapes: at least two token tiles and more than two tiles per SM.
 // MSD_W4_PAIR=0/1 forces the choice.
 static bool w4_use_pair(int64_t M, int64_t N, int64_t K) {
   const char* pe = getenv("MSD_W4_PAIR");
   if (pe) return atoi(pe) != 0;
   const int64_t m_tiles = (M + kW4TileM - 1) / kW4TileM, n_tiles = (N + 255) / 256;
-  return m_tiles >= 2 && m_tiles * n_tiles > 2 * sm_count();
+  // an odd number of token tiles leaves the last pair's second CTA without rows: only where that is a small share
+  return m_tiles >= 2 && (m_tiles % 2 == 0 || m_tiles >= 9) && m_tiles * n_tiles > 2 * sm_count();
 }
 
 // Weight rows per tile: MSD_W4_TILEN (224 or 256) if set; else 256 for the CTA-pair kernel (one accumulator) and 224 for
