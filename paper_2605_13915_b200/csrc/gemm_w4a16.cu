@@ -607,26 +607,12 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
         __syncwarp();
         if (lane == 0) mbar_arrive_remote(leader_tempty[acc]);
       }
-      for (int c0 = 0; c0 < cend; c0 += ccols, buf ^= 1) {
-        uint32_t o[16];
-        if (p.ytype == MSD_OUT_BF16) {
-          uint32_t v[32];
-          tmem_ld32(trow + c0, v);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-            o[j] = *reinterpret_cast<const uint32_t*>(&h);
-          }
-        } else {
-          tmem_ld16(trow + c0, o);
-          tmem_ld_wait();
-        }
-        if (c0 + ccols >= cend) {                   // all that is needed of this accumulator is in registers
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_remote(leader_tempty[acc]);
-        }
+      auto release_acc = [&]() {                    // all that is needed of this accumulator is in registers
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_remote(leader_tempty[acc]);
+      };
+      auto store_chunk = [&](const uint32_t (&o)[16], int c0) {
         uint8_t* sb = stage_buf + buf * kW4StoreBytes;
         if (lane == 0) bulk_wait_group_read<1>();    // the store that read this buffer two chunks ago is done with it
         __syncwarp();
@@ -639,6 +625,44 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
         if (lane == 0) {
           tma_store_2d(&tmap_y, nt * kTN + c0, row0, sb);
           bulk_commit_group();
+        }
+        buf ^= 1;
+      };
+      if (p.ytype == MSD_OUT_BF16) {
+        // The load of the next 32 columns is in flight while a chunk is converted and stored: a TMEM load takes about
+        // 450 cycles, and with one accumulator no MMA runs while the tile drains.
+        auto bf16_chunk = [&](const uint32_t (&v)[32], int c0) {
+          uint32_t o[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+            o[j] = *reinterpret_cast<const uint32_t*>(&h);
+          }
+          store_chunk(o, c0);
+        };
+        uint32_t va[32], vb[32];
+        if (cend > 0) {
+          tmem_ld32(trow, va);
+          tmem_ld_wait_for(va);
+        }
+        for (int c0 = 0; c0 < cend; c0 += 64) {
+          const bool more_b = c0 + 32 < cend;
+          if (more_b) tmem_ld32(trow + c0 + 32, vb); else release_acc();
+          bf16_chunk(va, c0);
+          if (!more_b) break;
+          tmem_ld_wait_for(vb);
+          const bool more_a = c0 + 64 < cend;
+          if (more_a) tmem_ld32(trow + c0 + 64, va); else release_acc();
+          bf16_chunk(vb, c0 + 32);
+          if (more_a) tmem_ld_wait_for(va);
+        }
+      } else {
+        for (int c0 = 0; c0 < cend; c0 += 16) {
+          uint32_t o[16];
+          tmem_ld16(trow + c0, o);
+          tmem_ld_wait();
+          if (c0 + 16 >= cend) release_acc();
+          store_chunk(o, c0);
         }
       }
     }
