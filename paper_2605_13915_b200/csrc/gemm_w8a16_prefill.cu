@@ -10,6 +10,12 @@
 // 32 (w % 4) .., columns 64 ((w - 2) / 4) .. of both accumulators, combines them with alpha_i, beta_i and w_scale[n]
 // and writes them through a swizzled staging buffer with TMA stores).  The 512 TMEM columns hold one tile, so the
 // epilogue of a tile does not overlap the MMAs of the next; sixteen warps keep it short.
+//
+// kPair: two CTAs of a cluster work on 256 tokens x 256 weight rows with tcgen05.mma.cta_group::2.  Each CTA loads its
+// own 128 token rows of both components and half of the weight tile (48 instead of 64 KB per stage, four stages),
+// all loads complete on the leader's barrier, the leader issues the MMAs and its commits reach both CTAs, each CTA's
+// epilogue drains its own 128 accumulator rows and tells the leader.  Barrier operations between the CTAs use the
+// default (CTA-scope) semantics: what is handed over is tensor memory, ordered by the tcgen05 fences.
 #include <cuda_bf16.h>
 
 #include <cstdlib>
@@ -27,6 +33,8 @@ constexpr int kP8ABytes = kP8TileM * kP8BlockK;                 // 16 KB
 constexpr int kP8BBytes = kP8TileN * kP8BlockK;                 // 32 KB
 constexpr int kP8StageBytes = 2 * kP8ABytes + kP8BBytes;        // 64 KB
 constexpr int kP8Stages = 3;
+constexpr int kP8PairStageBytes = 2 * kP8ABytes + kP8BBytes / 2;    // 48 KB per CTA of a pair
+constexpr int kP8PairStages = 4;
 constexpr int kP8StoreBytes = 2048;                             // one epilogue chunk: 32 rows x 64 bytes
 constexpr int kP8TmemCols = 512;
 
@@ -44,22 +52,26 @@ struct GemmP8Params {
   unsigned* status;
 };
 
+template <bool kPair>
 __global__ void __launch_bounds__(kP8Threads, 1)
 gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
                           const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_y,
                           const GemmP8Params p) {
+  constexpr int kStages = kPair ? kP8PairStages : kP8Stages;
+  constexpr int kStageBytes = kPair ? kP8PairStageBytes : kP8StageBytes;
   extern __shared__ uint8_t smem_dyn[];
-  __shared__ __align__(8) uint64_t full_bar[kP8Stages], empty_bar[kP8Stages], tfull_bar, tempty_bar;
+  __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages], tfull_bar, tempty_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = kPair ? cluster_ctarank() : 0u;     // 0 = leader of the pair
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kP8Stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     mbar_init(&tfull_bar, 1);
-    mbar_init(&tempty_bar, 16);
+    mbar_init(&tempty_bar, kPair ? 32 : 16);      // a pair: the epilogue warps of both CTAs arrive on the leader's
     abort_flag = 0;
     mbar_init_fence();
     tma_prefetch_desc(&tmap_a1);
@@ -67,46 +79,71 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
     tma_prefetch_desc(&tmap_b);
     tma_prefetch_desc(&tmap_y);
   }
-  if (warp == 1) tmem_alloc(&tmem_base_slot, kP8TmemCols);
+  if (warp == 1) {
+    if (kPair) tmem_alloc_pair(&tmem_base_slot, kP8TmemCols); else tmem_alloc(&tmem_base_slot, kP8TmemCols);
+  }
   tc_fence_before();
-  __syncthreads();
+  if (kPair) {               // both CTAs' barriers exist before either signals the other's
+    cluster_arrive_all();
+    cluster_wait_all();
+  } else {
+    __syncthreads();
+  }
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
   volatile int* abort = &abort_flag;
   // Work items: (token tile, weight tile, K split).  With ksplit > 1 (few output tiles, long K) an item covers kper K
   // stages and writes s_W (alpha D1 + beta D2) of its K range in FP32 to the partial buffer; a second kernel adds the
   // splits in a fixed order.
-  const int total_tiles = p.m_tiles * p.n_tiles * p.ksplit;
+  // A pair takes two token tiles at once (no K split there); its CTAs stride over the pair tiles together.
+  const int m_units = kPair ? (p.m_tiles + 1) >> 1 : p.m_tiles;
+  const int total_tiles = m_units * p.n_tiles * p.ksplit;
+  const int first = kPair ? blockIdx.x >> 1 : blockIdx.x, step = kPair ? gridDim.x >> 1 : gridDim.x;
+  auto tile_of = [&](int tile_mn, int& mt, int& nt) {
+    const int mu = p.n_fastest ? tile_mn / p.n_tiles : tile_mn % m_units;
+    nt = p.n_fastest ? tile_mn % p.n_tiles : tile_mn / m_units;
+    mt = kPair ? 2 * mu + static_cast<int>(rank) : mu;
+  };
 
   if (warp == 0) {
     if (lane == 0) {
       pdl_wait_primary();           // the components and their scales come from the kernel launched just before
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (int tile = first; tile < total_tiles && ok; tile += step) {
         const int split = tile % p.ksplit, tile_mn = tile / p.ksplit;
-        const int mt = p.n_fastest ? tile_mn / p.n_tiles : tile_mn % p.m_tiles, nt = p.n_fastest ? tile_mn % p.n_tiles : tile_mn / p.m_tiles;
+        int mt, nt;
+        tile_of(tile_mn, mt, nt);
         const int ks0 = split * p.kper, ks1 = ks0 + p.kper < p.kstages ? ks0 + p.kper : p.kstages;
         for (int ks = ks0; ks < ks1; ++ks) {
           ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
           if (!ok) break;
-          uint8_t* dst = smem + stage * kP8StageBytes;
-          mbar_arrive_expect_tx(&full_bar[stage], kP8StageBytes);
-          tma_load_2d(dst, &tmap_a1, ks * kP8BlockK, mt * kP8TileM, &full_bar[stage]);
-          tma_load_2d(dst + kP8ABytes, &tmap_a2, ks * kP8BlockK, mt * kP8TileM, &full_bar[stage]);
-          tma_load_2d(dst + 2 * kP8ABytes, &tmap_b, ks * kP8BlockK, nt * kP8TileN, &full_bar[stage]);
-          if (++stage == kP8Stages) { stage = 0; phase ^= 1; }
+          uint8_t* dst = smem + stage * kStageBytes;
+          if (kPair) {
+            // the leader's barrier counts the bytes of both CTAs; tmap_b's box is this CTA's half of the weight tile
+            if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * kStageBytes);
+            const uint32_t bar = mapa_shared(smem_u32(&full_bar[stage]), 0);
+            tma_load_2d_pair(dst, &tmap_a1, ks * kP8BlockK, mt * kP8TileM, bar);
+            tma_load_2d_pair(dst + kP8ABytes, &tmap_a2, ks * kP8BlockK, mt * kP8TileM, bar);
+            tma_load_2d_pair(dst + 2 * kP8ABytes, &tmap_b, ks * kP8BlockK, nt * kP8TileN + static_cast<int>(rank) * (kP8TileN / 2), bar);
+          } else {
+            mbar_arrive_expect_tx(&full_bar[stage], kStageBytes);
+            tma_load_2d(dst, &tmap_a1, ks * kP8BlockK, mt * kP8TileM, &full_bar[stage]);
+            tma_load_2d(dst + kP8ABytes, &tmap_a2, ks * kP8BlockK, mt * kP8TileM, &full_bar[stage]);
+            tma_load_2d(dst + 2 * kP8ABytes, &tmap_b, ks * kP8BlockK, nt * kP8TileN, &full_bar[stage]);
+          }
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       int stage = 0; uint32_t phase = 0;
       int it = 0;
       bool ok = true;
       const uint64_t op_desc = smem_desc(0, 16, 1024, kSwizzle128B);    // 128-byte-swizzled K-major operand tile
-      const uint32_t idesc = idesc_dense(/*D=S32*/ 2, /*A=S8*/ 1, /*B=S8*/ 1, 0, 0, kP8TileM, kP8TileN);
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+      const uint32_t idesc = idesc_dense(/*D=S32*/ 2, /*A=S8*/ 1, /*B=S8*/ 1, 0, 0, kPair ? 2 * kP8TileM : kP8TileM, kP8TileN);
+      for (int tile = first; tile < total_tiles && ok; tile += step, ++it) {
         ok = wait_bounded(&tempty_bar, (it & 1) ^ 1, abort, p.status);        // the epilogue has drained both accumulators
         if (!ok) break;
         tc_fence_after();
@@ -115,19 +152,24 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
           ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
           if (!ok) break;
           tc_fence_after();
-          const uint64_t enc = static_cast<uint64_t>(smem_u32(smem + stage * kP8StageBytes) >> 4);
+          const uint64_t enc = static_cast<uint64_t>(smem_u32(smem + stage * kStageBytes) >> 4);
           const uint64_t a1d = op_desc + enc, a2d = a1d + (kP8ABytes >> 4), bd = a1d + (2 * kP8ABytes >> 4);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {                    // 32 elements (32 bytes) per MMA
             const uint32_t acc = (ks > ks0 || kk > 0) ? 1u : 0u;
-            mma_i8(tmem_base, a1d + 2 * kk, bd + 2 * kk, idesc, acc);
-            mma_i8(tmem_base + kP8TileN, a2d + 2 * kk, bd + 2 * kk, idesc, acc);
+            if (kPair) {
+              mma_i8_pair(tmem_base, a1d + 2 * kk, bd + 2 * kk, idesc, acc);
+              mma_i8_pair(tmem_base + kP8TileN, a2d + 2 * kk, bd + 2 * kk, idesc, acc);
+            } else {
+              mma_i8(tmem_base, a1d + 2 * kk, bd + 2 * kk, idesc, acc);
+              mma_i8(tmem_base + kP8TileN, a2d + 2 * kk, bd + 2 * kk, idesc, acc);
+            }
           }
-          tc_commit(&empty_bar[stage]);
-          if (++stage == kP8Stages) { stage = 0; phase ^= 1; }
+          if (kPair) tc_commit_pair(&empty_bar[stage], 3); else tc_commit(&empty_bar[stage]);    // frees the stage (in both CTAs)
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
-        tc_commit(&tfull_bar);
+        if (kPair) tc_commit_pair(&tfull_bar, 3); else tc_commit(&tfull_bar);
       }
     }
   } else {
@@ -137,7 +179,15 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
     // in chunks of 64 bytes per row (32 BF16 or 16 FP32 columns) in the 64-byte-swizzled layout of the output tensor
     // map and written by a TMA store; rows past M and columns past N are clipped by the store.
     const int quad = warp & 3, part = (warp - 2) >> 2;
-    uint8_t* sb = smem + kP8Stages * kP8StageBytes + (warp - 2) * kP8StoreBytes;
+    uint8_t* sb = smem + kStages * kStageBytes + (warp - 2) * kP8StoreBytes;
+    const uint32_t leader_tempty = kPair ? mapa_shared(smem_u32(&tempty_bar), 0) : 0u;
+    auto release_acc = [&]() {                      // all that is needed of the accumulators is in registers
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if (kPair) mbar_arrive_remote(leader_tempty); else mbar_arrive(&tempty_bar);
+      }
+    };
     const int ccols = (p.ytype == MSD_OUT_BF16) ? 32 : 16;
     const uint32_t swz = static_cast<uint32_t>((lane >> 1) & 3);
     int it = 0;
@@ -145,9 +195,10 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
     pdl_wait_primary();             // alpha and beta come from the decomposition kernel launched just before
     // Column scales: every lane needs the same scales of a chunk.  Lane l loads the scale of the chunk's l-th column
     // one chunk ahead and the lanes fetch them from one another by shuffles.
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+    for (int tile = first; tile < total_tiles && ok; tile += step, ++it) {
       const int split = tile % p.ksplit, tile_mn = tile / p.ksplit;
-        const int mt = p.n_fastest ? tile_mn / p.n_tiles : tile_mn % p.m_tiles, nt = p.n_fastest ? tile_mn % p.n_tiles : tile_mn / p.m_tiles;
+      int mt, nt;
+      tile_of(tile_mn, mt, nt);
       const int row0 = mt * kP8TileM + quad * 32, row = row0 + lane;
       const float a_i = row < p.M ? __ldg(p.alpha + row) : 0.0f, b_i = row < p.M ? __ldg(p.beta + row) : 0.0f;
       const int col_base = nt * kP8TileN + part * 64;
@@ -160,11 +211,7 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
       // this warp's columns of the tile that lie inside the matrix; chunks beyond them are skipped altogether
       const int cols_here = p.N - col_base < 64 ? p.N - col_base : 64;
       const int cend = row0 < p.M ? (cols_here > 0 ? cols_here : 0) : 0;
-      if (cend == 0) {
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&tempty_bar);
-      }
+      if (cend == 0) release_acc();
       for (int c0 = 0; c0 < cend; c0 += ccols) {
         uint32_t o[16];
         const int col = col_base + c0;
@@ -209,11 +256,7 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
             }
           }
         }
-        if (c0 + ccols >= cend) {                   // all that is needed of the accumulators is in registers
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&tempty_bar);
-        }
+        if (c0 + ccols >= cend) release_acc();
         if (lane == 0) bulk_wait_group_read<0>();    // the store of the previous chunk is done with the staging buffer
         __syncwarp();
         uint8_t* srow = sb + lane * 64;
@@ -233,9 +276,13 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
 
   tc_fence_before();
   __syncthreads();
+  if (kPair) {       // neither CTA leaves while the other may still signal its barriers or read its shared memory
+    cluster_arrive_all();
+    cluster_wait_all();
+  }
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, kP8TmemCols);
+    if (kPair) tmem_dealloc_pair(tmem_base, kP8TmemCols); else tmem_dealloc(tmem_base, kP8TmemCols);
   }
 }
 
@@ -303,9 +350,18 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
   const uint64_t part_rows = static_cast<uint64_t>(pl.m_tiles) * kP8TileM;
   CUtensorMap tmap_a1, tmap_a2, tmap_b, tmap_y;
   const bool ybf = !split && ytype == MSD_OUT_BF16;
+  // CTA pairs (256 tokens x 256 weight rows per pair, half of the weight tile loaded by each CTA) where there are many
+  // tiles and no K split; MSD_P8_PAIR=0/1 forces the choice.
+  bool use_pair = false;
+  {
+    const char* pe = getenv("MSD_P8_PAIR");
+    const bool can = pl.ksplit == 1 && pl.m_tiles >= 2;
+    const bool want = (pl.m_tiles % 2 == 0 || pl.m_tiles >= 9) && static_cast<long long>(pl.m_tiles) * pl.n_tiles > 2LL * sm_count();
+    use_pair = can && (pe ? atoi(pe) != 0 : want);
+  }
   if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, K, M, K, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, q2, K, M, K, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !encode_tmap_2d(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kP8BlockK, kP8TileN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kP8BlockK, use_pair ? kP8TileN / 2 : kP8TileN, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, split ? static_cast<void*>(part) : y,
                       static_cast<uint64_t>(N), split ? part_rows * ksplit : static_cast<uint64_t>(M),
                       static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
@@ -325,16 +381,25 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
     p.n_fastest = oe ? (atoi(oe) != 0) : n_fast;
   }
   const size_t smem_bytes = static_cast<size_t>(kP8Stages) * kP8StageBytes + 16 * kP8StoreBytes + 1024;
+  const size_t smem_pair = static_cast<size_t>(kP8PairStages) * kP8PairStageBytes + 16 * kP8StoreBytes + 1024;
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(gemm_w8a16_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes)) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_w8a16_prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes)) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w8a16_prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_pair)) != cudaSuccess)
       return MSD_ERR_CUDA;
     attr_done = true;
   }
   const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+  if (use_pair) {
+    const long long pair_tiles = static_cast<long long>((pl.m_tiles + 1) / 2) * pl.n_tiles;
+    const int clusters = static_cast<int>(pair_tiles < sm_count() / 2 ? pair_tiles : sm_count() / 2);
+    if (launch_pdl_cluster(gemm_w8a16_prefill_kernel<true>, dim3(2 * clusters), dim3(kP8Threads), smem_pair, s, pdl, 2u, tmap_a1, tmap_a2, tmap_b, tmap_y, p) != cudaSuccess)
+      return MSD_ERR_CUDA;
+    return MSD_OK;
+  }
   const long long items = static_cast<long long>(pl.m_tiles) * pl.n_tiles * ksplit;
   const int grid = static_cast<int>(items < sm_count() ? items : sm_count());
-  if (launch_pdl(gemm_w8a16_prefill_kernel, dim3(grid), dim3(kP8Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p) != cudaSuccess)
+  if (launch_pdl(gemm_w8a16_prefill_kernel<false>, dim3(grid), dim3(kP8Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p) != cudaSuccess)
     return MSD_ERR_CUDA;
   if (split) return launch_ksplit_reduce(part, ksplit, static_cast<int64_t>(part_rows) * N, M, N, y, ytype, s, pdl);
   return MSD_OK;
