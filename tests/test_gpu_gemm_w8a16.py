@@ -251,3 +251,15 @@ def test_prefill_regime_with_k_split(M, N, K):
     got = oracle.bf16_bits_to_f64(bf16_bits(yb))
     n = np.linalg.norm(ref, axis=-1, keepdims=True)
     assert np.all(np.abs(got - ref) <= TOL * n + np.abs(ref) * 2.0 ** -8 + 1e-30)
+
+
+@pytest.mark.parametrize("pair", ["0", "1"])
+@pytest.mark.parametrize("M,N,K", [(129, 256, 128), (300, 520, 400), (1000, 264, 2048), (1290, 1288, 144)])
+def test_prefill_single_cta_and_cta_pair_kernels(pair, M, N, K, monkeypatch):
+    """The many-row kernel as single CTAs and as CTA pairs (256 tokens per pair of CTAs), each forced on every shape: a
+    pair whose second CTA has a single row or none, an odd number of 128-row tiles, ragged weight tiles, several tiles per
+    pair; INT32 accumulators bit-exact in both, FP32 and BF16 outputs."""
+    monkeypatch.setenv("MSD_P8_PAIR", pair)
+    c = inputs.gemm_w8_case(M, N, K, seed=11)
+    _check(c, torch.float32)
+    _check(c, torch.bfloat16)
