@@ -687,14 +687,21 @@ struct GemmW4Plan {
 };
 
 // The CTA-pair kernel (256 tokens x 256 weight rows per pair of CTAs: half the weight tile per CTA, so less shared-memory
-// traffic per MMA, and four stages) takes the prefill shapes: at least two token tiles and more than two tiles per SM.
+// traffic per MMA, and four stages) takes the shapes on which its tiles fill the GPU about as well as the single-CTA
+// kernel's: at equal rounds x tile width it is 5-15 % faster, and where the 128 x 224 tiles need an extra round
+// (M = 2048, N = 4096) by a quarter.  Not where the single-CTA kernel would split K (few tiles).
 // MSD_W4_PAIR=0/1 forces the choice.
 static bool w4_use_pair(int64_t M, int64_t N, int64_t K) {
+  (void)K;
   const char* pe = getenv("MSD_W4_PAIR");
   if (pe) return atoi(pe) != 0;
   const int64_t m_tiles = (M + kW4TileM - 1) / kW4TileM, n_tiles = (N + 255) / 256;
+  const int64_t clusters = sm_count() / 2, pair_tiles = (m_tiles + 1) / 2 * n_tiles, single_tiles = m_tiles * ((N + 223) / 224);
   // an odd number of token tiles leaves the last pair's second CTA without rows: only where that is a small share
-  return m_tiles >= 2 && (m_tiles % 2 == 0 || m_tiles >= 9) && m_tiles * n_tiles > 2 * sm_count();
+  if (!(m_tiles >= 2 && (m_tiles % 2 == 0 || m_tiles >= 9) && 2 * single_tiles > sm_count())) return false;
+  // rounds x tile width of either kernel (a pair tile takes a pair as long as a 128 x 256 tile takes a CTA)
+  const int64_t cost_pair = (pair_tiles + clusters - 1) / clusters * 256, cost_single = (single_tiles + sm_count() - 1) / sm_count() * 224;
+  return 100 * cost_pair <= 110 * cost_single;
 }
 
 // Weight rows per tile: MSD_W4_TILEN (224 or 256) if set; else 256 for the CTA-pair kernel (one accumulator) and 224 for
