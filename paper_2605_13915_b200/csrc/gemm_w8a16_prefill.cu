@@ -350,13 +350,16 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
   const uint64_t part_rows = static_cast<uint64_t>(pl.m_tiles) * kP8TileM;
   CUtensorMap tmap_a1, tmap_a2, tmap_b, tmap_y;
   const bool ybf = !split && ytype == MSD_OUT_BF16;
-  // CTA pairs (256 tokens x 256 weight rows per pair, half of the weight tile loaded by each CTA) where there are many
-  // tiles and no K split; MSD_P8_PAIR=0/1 forces the choice.
+  // CTA pairs (256 tokens x 256 weight rows per pair, half of the weight tile loaded by each CTA) where there is no K
+  // split; MSD_P8_PAIR=0/1 forces the choice.
   bool use_pair = false;
   {
     const char* pe = getenv("MSD_P8_PAIR");
     const bool can = pl.ksplit == 1 && pl.m_tiles >= 2;
-    const bool want = (pl.m_tiles % 2 == 0 || pl.m_tiles >= 9) && static_cast<long long>(pl.m_tiles) * pl.n_tiles > 2LL * sm_count();
+    // where the pair tiles need no more rounds on half as many units (an odd number of token tiles leaves a CTA idle)
+    const long long tiles = static_cast<long long>(pl.m_tiles) * pl.n_tiles, pair_tiles = static_cast<long long>((pl.m_tiles + 1) / 2) * pl.n_tiles;
+    const long long clusters = sm_count() / 2;
+    const bool want = (pair_tiles + clusters - 1) / clusters <= (tiles + sm_count() - 1) / sm_count();
     use_pair = can && (pe ? atoi(pe) != 0 : want);
   }
   if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, K, M, K, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
