@@ -238,16 +238,18 @@ def gemm_w4a16(x_bits, w_fp4, w_e8m0, ytype="f64", mode="msd", grid=GRID_E2M1, c
 
 
 # --- attention -------------------------------------------------------------------
-_ATTN_MODE = {"global": 0, "tiled": 1, "ref": 2, "dequant": 3}
+_ATTN_MODE = {"global": 0, "tiled": 1, "ref": 2, "dequant": 3, "held": 4}
 
 
 def attn_decode_int8kv(q_bits, k, v, k_scale, v_scale, cu_seqlens, softmax_scale, dv=None, mode="global", tile=0,
-                       split_starts=None, want_lse=False, want_s=False):
+                       split_starts=None, want_lse=False, want_s=False, m_margin=0.0, sv_growth=1.0):
     """Decode attention over an INT8 KV cache (Alg. 3, one scale per token per KV head).
 
     mode: 'global' (definition), 'tiled' (mirrors a tile/split schedule), 'ref' (FP64, no MSD),
-    'dequant' (KV -> BF16 comparison path).  ``v=None`` means V is the first ``dv`` entries of each K row.
-    ``split_starts`` ([B, n_splits+1] token offsets relative to each sequence) is used by 'tiled' only.
+    'dequant' (KV -> BF16 comparison path), 'held' (tiled, but the reference maximum and the probability scale
+    move only when exceeded: to the tile maximum + ``m_margin`` (natural-log units) and to ``sv_growth`` times the
+    tile's largest value scale).  ``v=None`` means V is the first ``dv`` entries of each K row.
+    ``split_starts`` ([B, n_splits+1] token offsets relative to each sequence) is used by 'tiled' and 'held'.
     """
     q_bits = _c(q_bits, np.uint16)
     B, Hq, D = q_bits.shape
@@ -265,13 +267,13 @@ def attn_decode_int8kv(q_bits, k, v, k_scale, v_scale, cu_seqlens, softmax_scale
     sdbg = np.zeros((2, Hq, T), np.int32) if want_s else None
     m = _ATTN_MODE[mode]
     ns, ss = 0, None
-    if m == 1:
+    if m in (1, 4):
         ss = _c(split_starts, np.int32)
         ns = ss.shape[1] - 1
     lib().msdo_attn_decode_int8kv(_p(q_bits), _p(k), _p(v), _p(k_scale), _p(v_scale), _p(cu), C.c_int32(B),
                                   C.c_int32(Hq), C.c_int32(Hkv), C.c_int32(D), C.c_int32(dv),
                                   C.c_float(softmax_scale), C.c_int(m), C.c_int32(tile), _p(ss), C.c_int32(ns),
-                                  _p(out), _p(lse), _p(sdbg))
+                                  _p(out), _p(lse), _p(sdbg), C.c_double(m_margin), C.c_float(sv_growth))
     res = [out]
     if want_lse:
         res.append(lse)

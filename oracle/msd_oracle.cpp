@@ -468,6 +468,11 @@ void msdo_gemm_w4a16(const uint16_t* x_bf16, const uint8_t* w_fp4, const uint8_t
 //           [B, n_splits+1]; unused trailing entries repeat the length), each split walked in tiles of
 //           `tile` tokens with a running max; each tile quantises P against the running max in force
 //           and with alpha_P = max(tile's v_scale)/127; splits merged with the usual log-sum-exp rule.
+//   mode 4  tiled with held references (reading of Sec. 4.3 for kernels that keep integer PV sums across tiles):
+//           as mode 1, but per split the reference maximum of a head moves only when a tile's maximum exceeds it,
+//           to that maximum + m_margin, and alpha_P = a_ref/127 with a_ref a running bound of the value scales
+//           that is set to sv_growth * (tile's largest value scale) when exceeded.  P <= 1 and P~ <= a_ref always
+//           hold, so nothing clips; m_margin = 0, sv_growth = 1 is the plain online softmax with a running alpha_P.
 //   mode 2  FP64 reference on the dequantized cache (no MSD).
 //   mode 3  dequantize-to-BF16 comparison path (Sec. 6.4 "Dequant"): K,V -> bf16(q*s); P -> BF16 before PV.
 // Per-token reading: s_K[j] multiplies score column j; s_V[j] is folded into P before decomposition.
@@ -477,7 +482,7 @@ void msdo_attn_decode_int8kv(const uint16_t* q_bf16, const int8_t* k, const int8
                              const float* v_scale, const int32_t* cu_seqlens, int32_t B, int32_t Hq, int32_t Hkv,
                              int32_t D, int32_t Dv, float softmax_scale, int mode, int32_t tile,
                              const int32_t* split_starts, int32_t n_splits, double* out, double* lse,
-                             int32_t* s_dbg) {
+                             int32_t* s_dbg, double m_margin, float sv_growth) {
   const int64_t T = cu_seqlens[B];
   const int G = Hq / Hkv;
   const int8_t* vv = v ? v : k;
@@ -495,7 +500,7 @@ void msdo_attn_decode_int8kv(const uint16_t* q_bf16, const int8_t* k, const int8
       if (L <= 0) continue;
       const uint16_t* qrow = q_bf16 + (static_cast<int64_t>(b) * Hq + h) * D;
       std::vector<double> S(L);
-      if (mode <= 1) {
+      if (mode <= 1 || mode == 4) {
         // lines 1-5: decompose Q, two exact integer products, merge
         std::vector<float> qf(D);
         for (int d = 0; d < D; ++d) qf[d] = bf16_to_f32(qrow[d]);
@@ -523,7 +528,7 @@ void msdo_attn_decode_int8kv(const uint16_t* q_bf16, const int8_t* k, const int8
           S[j] = s * static_cast<double>(softmax_scale);
         }
       }
-      if (mode >= 2) {
+      if (mode == 2 || mode == 3) {
         double m = -std::numeric_limits<double>::infinity();
         for (int64_t j = 0; j < L; ++j) m = std::max(m, S[j]);
         double l = 0.0;
@@ -555,15 +560,30 @@ void msdo_attn_decode_int8kv(const uint16_t* q_bf16, const int8_t* k, const int8
       for (size_t s = 0; s + 1 < bounds.size(); ++s) {
         if (bounds[s + 1] <= bounds[s]) continue;
         double m_run = -std::numeric_limits<double>::infinity(), l_run = 0.0;
+        float a_ref = 0.0f;                                  // mode 4: running bound of the value scales
         std::vector<double> o_run(Dv, 0.0);
         for (int64_t j0 = bounds[s]; j0 < bounds[s + 1]; j0 += tl) {
           int64_t j1 = std::min<int64_t>(bounds[s + 1], j0 + tl);
           double m_new = m_run;
-          for (int64_t j = j0; j < j1; ++j) m_new = std::max(m_new, S[j]);
-          double resc = std::exp(m_run - m_new);              // 0 on the first tile
           float sv_max = 0.0f;
           for (int64_t j = j0; j < j1; ++j) sv_max = std::max(sv_max, vs[(t0 + j) * Hkv + hk]);
-          float alpha_p = sv_max / 127.0f;                     // line 8 under per-token V scales
+          float alpha_p;
+          if (mode <= 1) {
+            for (int64_t j = j0; j < j1; ++j) m_new = std::max(m_new, S[j]);
+            alpha_p = sv_max / 127.0f;                         // line 8 under per-token V scales
+          } else {
+            // mode 4, held references: the reference maximum moves only when a tile's maximum exceeds it and is then
+            // set m_margin above that maximum (so P <= 1 still holds and later tiles rarely move it again); the
+            // probability scale follows a running bound of the value scales that grows by the factor sv_growth when
+            // exceeded.  Between such events both stay as they are, so integer PV sums of consecutive tiles share
+            // one scale and one reference (Alg. 3 line 12 applied once per run of tiles instead of once per tile).
+            double t_max = -std::numeric_limits<double>::infinity();
+            for (int64_t j = j0; j < j1; ++j) t_max = std::max(t_max, S[j]);
+            if (t_max > m_run) m_new = t_max + m_margin;
+            if (sv_max > a_ref) a_ref = sv_max * sv_growth;
+            alpha_p = a_ref / 127.0f;
+          }
+          double resc = std::exp(m_run - m_new);              // 0 on the first tile
           int64_t n = j1 - j0;
           std::vector<float> pt(n);
           double lsum = 0.0;

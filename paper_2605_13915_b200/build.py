@@ -1,19 +1,24 @@
-"""Builds the CUDA library in-tree: ``libmsd.so`` next to this file, for sm_100a only."""
+"""Builds the CUDA library in-tree: ``libmsd.so`` next to this file, for sm_100a only.
+
+Every ``csrc/*.cu`` is compiled to an object of its own (in parallel, and only when it or a header changed), then the
+objects are linked into one shared library.
+"""
 from __future__ import annotations
 
 import glob
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libmsd.so")
+OBJ_DIR = os.path.join(_HERE, "build")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
-    "--expt-relaxed-constexpr",
+    "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",
 ]
 
 
@@ -21,32 +26,59 @@ def sources():
     return sorted(glob.glob(os.path.join(_HERE, "csrc", "*.cu")))
 
 
+def _headers():
+    return glob.glob(os.path.join(_HERE, "csrc", "*.h")) + glob.glob(os.path.join(_HERE, "csrc", "*.cuh")) + \
+        glob.glob(os.path.join(_ROOT, "include", "*.h"))
+
+
 def needs_build() -> bool:
     if not os.path.exists(LIB_PATH):
         return True
     t = os.path.getmtime(LIB_PATH)
-    deps = sources() + glob.glob(os.path.join(_HERE, "csrc", "*.h")) + glob.glob(os.path.join(_HERE, "csrc", "*.cuh")) + \
-        glob.glob(os.path.join(_ROOT, "include", "*.h"))
-    return any(os.path.getmtime(d) > t for d in deps)
+    return any(os.path.getmtime(d) > t for d in sources() + _headers())
+
+
+def _obj(src):
+    return os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into one shared library (nvcc cross-compiles without a GPU)."""
+    """Compile every .cu under csrc/ and link them into one shared library (nvcc cross-compiles without a GPU)."""
     if not force and not needs_build():
         return LIB_PATH
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + ["-I", os.path.join(_ROOT, "include"), "-I", os.path.join(_HERE, "csrc")]
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    hdr_time = max([os.path.getmtime(h) for h in _headers()] + [os.path.getmtime(__file__)])
+    base = [nvcc] + NVCC_FLAGS + ["-I", os.path.join(_ROOT, "include"), "-I", os.path.join(_HERE, "csrc")]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += ["-o", LIB_PATH] + sources()
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose or res.returncode != 0:
-        sys.stderr.write(res.stdout + res.stderr)
-    if res.returncode != 0:
+        base += ["-Xptxas", "-v"]
+
+    def compile_one(src):
+        obj = _obj(src)
+        if not force and os.path.exists(obj) and os.path.getmtime(obj) > max(os.path.getmtime(src), hdr_time):
+            return 0, ""
+        res = subprocess.run(base + ["-c", src, "-o", obj], capture_output=True, text=True)
+        return res.returncode, res.stdout + res.stderr
+
+    srcs = sources()
+    with ThreadPoolExecutor(max_workers=min(len(srcs), os.cpu_count() or 4)) as ex:
+        results = list(ex.map(compile_one, srcs))
+    failed = False
+    for (rc, out), src in zip(results, srcs):
+        if rc != 0 or (verbose and out):
+            sys.stderr.write("== %s\n%s" % (os.path.basename(src), out))
+        failed = failed or rc != 0
+    if failed:
         raise RuntimeError("nvcc failed")
+    link = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-cudart", "static", "-o", LIB_PATH] + \
+        [_obj(s) for s in srcs]
+    res = subprocess.run(link, capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError("nvcc link failed")
     return LIB_PATH
 
 
 if __name__ == "__main__":
-    build(force=True, verbose="-v" in sys.argv)
+    build(force="-f" in sys.argv, verbose="-v" in sys.argv)
     print(LIB_PATH)

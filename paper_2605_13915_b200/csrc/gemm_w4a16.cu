@@ -810,7 +810,8 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
     return MSD_ERR_BAD_SHAPE;
   if (ytype != MSD_OUT_BF16 && ytype != MSD_OUT_FP32) return MSD_ERR_UNSUPPORTED;
   if (!x_bf16 || !w_fp4 || !w_e8m0 || !y || !workspace) return MSD_ERR_NULL_POINTER;
-  if (!aligned(x_bf16, 16) || !aligned(w_fp4, 16) || !aligned(y, 16) || !aligned(workspace, 1024)) return MSD_ERR_BAD_ALIGNMENT;
+  if (!aligned(x_bf16, 16) || !aligned(w_fp4, 16) || !aligned(w_e8m0, 4) || !aligned(y, 16) || !aligned(workspace, 1024))
+    return MSD_ERR_BAD_ALIGNMENT;     // the scale relayout reads the E8M0 rows as 32-bit words
   const GemmW4Plan pl = plan_w4(M, N, K);
   if (workspace_bytes < pl.bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
   unsigned* status = device_status_ptr();

@@ -11,9 +11,10 @@ import oracle
 from paper_2605_13915_b200 import inputs
 
 
-def _alg3_literal(q_bits, k, v, scale):
+def _alg3_literal(q_bits, k, v, scale, m_margin=0.0, a_ref=1.0):
     """Alg. 3 for one head with s_K = s_V = 1: decompose Q; S = (aS1 + bS2)/sqrt(d); P = exp(S - max);
-    alpha_P = 1/127; decompose P; O = (alpha_P O1 + beta_P O2)/l."""
+    alpha_P = 1/127; decompose P; O = (alpha_P O1 + beta_P O2)/l.  m_margin / a_ref: the reference sits that far above
+    the maximum and alpha_P = a_ref/127 (the held-reference reading; both cancel in O up to the quantisation of P)."""
     q = oracle.bf16_bits_to_f64(q_bits)
     M = np.abs(q).max()
     a = np.float32(M) / np.float32(127)
@@ -22,8 +23,8 @@ def _alg3_literal(q_bits, k, v, scale):
     b = a / np.float32(254)
     q2 = np.clip(np.rint(r.astype(np.float32) / b), -128, 127)
     S = (float(a) * (k.astype(np.int64) @ q1.astype(np.int64)) + float(b) * (k.astype(np.int64) @ q2.astype(np.int64))) * float(np.float32(scale))
-    P = np.exp(S - S.max())
-    ap = np.float32(1.0) / np.float32(127)
+    P = np.exp(S - (S.max() + m_margin))
+    ap = np.float32(a_ref) / np.float32(127)
     bp = ap / np.float32(254)
     Pf = P.astype(np.float32)
     p1 = np.clip(np.rint(Pf / ap), -128, 127)
@@ -115,6 +116,42 @@ def test_tiled_mode_tracks_definition(gqa_small):
     assert np.abs(tiled - glob).max() <= 5e-4 * rown.max()
     assert np.all(np.abs(tiled - glob) <= 1e-3 * rown)
     assert np.allclose(lse_t, lse_g, rtol=0, atol=1e-9)
+
+
+def test_held_references_mode(gqa_small):
+    """The tiled mode whose reference maximum and probability scale move only when exceeded (kernels that keep integer
+    PV sums across tiles).  Pins: (a) one tile, unit scales: Alg. 3 written out in numpy with the reference m_margin
+    above the maximum and alpha_P = sv_growth/127; (b) margin 0, growth 1 and equal value scales: bit for bit the plain
+    tiled mode; (c) the margins the CUDA path uses stay within 5e-4 of the row norm of the untiled definition, and the
+    log-sum-exp does not depend on them."""
+    rng = np.random.default_rng(4)
+    L, D = 200, 64
+    q = inputs.f32_to_bf16_bits(rng.standard_normal((1, 1, D)).astype(np.float32))
+    k = rng.integers(-127, 128, (L, 1, D), dtype=np.int8)
+    v = rng.integers(-127, 128, (L, 1, D), dtype=np.int8)
+    ones = np.ones((L, 1), np.float32)
+    ss = np.array([[0, L]], np.int32)
+    for margin, growth in ((0.0, 1.0), (1.3862943611198906, 1.25), (0.5, 2.0)):
+        got = oracle.attn_decode_int8kv(q, k, v, ones, ones, [0, L], 0.01, mode="held", tile=L, split_starts=ss,
+                                        m_margin=margin, sv_growth=growth)
+        want = _alg3_literal(q[0, 0], k[:, 0], v[:, 0], 0.01, m_margin=margin, a_ref=growth)
+        assert np.allclose(got[0, 0], want, rtol=1e-9, atol=1e-9), (margin, growth)
+    c = gqa_small
+    Ls = np.diff(c.cu_seqlens)
+    ss = np.stack([0 * Ls, Ls // 3, (2 * Ls) // 3 + 5, Ls], 1)
+    const_vs = np.full_like(c.v_scale, 0.0125)
+    args = (c.q, c.k, c.v, c.k_scale, const_vs, c.cu_seqlens, c.softmax_scale)
+    tiled = oracle.attn_decode_int8kv(*args, mode="tiled", tile=64, split_starts=ss)
+    held0 = oracle.attn_decode_int8kv(*args, mode="held", tile=64, split_starts=ss, m_margin=0.0, sv_growth=1.0)
+    assert np.array_equal(tiled, held0)
+    args = (c.q, c.k, c.v, c.k_scale, c.v_scale, c.cu_seqlens, c.softmax_scale)
+    glob, lse_g = oracle.attn_decode_int8kv(*args, mode="global", want_lse=True)
+    held, lse_h = oracle.attn_decode_int8kv(*args, mode="held", tile=128, split_starts=ss, m_margin=2 * np.log(2.0),
+                                            sv_growth=1.25, want_lse=True)
+    rown = np.linalg.norm(glob, axis=2, keepdims=True)
+    assert np.abs(held - glob).max() <= 5e-4 * rown.max()
+    assert np.all(np.abs(held - glob) <= 1e-3 * rown)
+    assert np.allclose(lse_h, lse_g, rtol=0, atol=1e-9)
 
 
 def test_mla_shape_shares_rows_and_scores_are_exact_integers():
