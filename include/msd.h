@@ -96,7 +96,8 @@ msd_status_t msd_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64
  * the two sums exact in INT32, the combine in FP32.
  *   x_bf16 [M,K]; w [N,K] INT8, K contiguous; w_scale [N] FP32; y [M,N] BF16 or FP32 (ytype);
  *   acc_dbg nullable [2,M,N] INT32 (the two accumulators, for bit-exact checks).
- * K % 16 == 0; N % 8 == 0 when y is BF16; x, w, y 16-byte aligned.
+ * K % 16 == 0; N % 8 == 0 when y is BF16; x, w, y 16-byte aligned.  K <= 131072 (beyond that the INT32 sums could
+ * overflow: MSD_ERR_UNSUPPORTED).
  * M <= 128 (decode regime): the weight rows sit on the MMA M axis and the weights are streamed once.  M > 128
  * (prefill regime): tiles of 128 tokens x 256 weight rows, both components against the same weight tile, outputs
  * written by TMA stores (N % 4 == 0 also when y is FP32); with few output tiles K is split over the CTAs and the FP32
@@ -145,7 +146,9 @@ msd_status_t msd_grouped_gemm_w8a16(const void* x_bf16, const int8_t* w, const f
  * MSD_ERR_UNSUPPORTED before any launch - use msd_gemm_w8a16 with your own workspace instead.
  * First use on a device resolves the array's device address (cudaGetSymbolAddress, with that device current); make
  * that first call outside any stream capture.  All calls on a device share the one array: it still holds the
- * previous call's contents (the parts that must start at zero are cleared on `stream` at the start of every call), and
+ * previous call's contents (the parts that must start at zero - the arrival counters, and for shapes that split K
+ * over CTAs through memory the meeting place of the partial sums, up to about 2 MB - are cleared on `stream` at the
+ * start of every call), and
  * two calls that overlap on the GPU - different streams, or a graph replayed concurrently - race on it.  Results are
  * identical to msd_gemm_w8a16.
  */
@@ -183,7 +186,7 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
  * MXFP4 weight by block-scaled FP4 MMAs accumulating in FP32,
  *   y[i,n] = sum_blocks 2^(e1+ew) <q1,w> + 2^(e2+ew) <q2,w>.
  *   x_bf16 [M,K]; w_fp4 [N,K/2] packed E2M1 (element 2i in bits 3:0); w_e8m0 [N,K/32]; y [M,N].
- * K % 128 == 0, N % 8 == 0; pointers 16-byte aligned.
+ * K % 128 == 0, N % 8 == 0; x, w_fp4, y 16-byte aligned, w_e8m0 4-byte aligned.
  */
 size_t msd_gemm_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K);
 msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0, int64_t M, int64_t N,
@@ -213,7 +216,8 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
  * alpha / 64.  Tensor cores have no E1M2 operand type; every E1M2 value is an E4M3 number, so the components are
  * emitted as E4M3 bytes and multiplied with tcgen05.mma kind::mxf8f6f4 (E4M3 x E2M1, block scales) at the FP8 rate.
  *   msd_decompose_mxfp4_e1m2: q1/q2 [M, K] E4M3 bytes, e8m0_1/e8m0_2 [M, K/32] row-major; K % 32 == 0.
- *   msd_gemm_w4a16_e1m2: same arguments and result layout as msd_gemm_w4a16; K % 128 == 0; w_fp4 32-byte aligned.
+ *   msd_gemm_w4a16_e1m2: same arguments and result layout as msd_gemm_w4a16; K % 128 == 0; w_fp4 32-byte aligned,
+ *   w_e8m0 4-byte aligned.
  */
 msd_status_t msd_decompose_mxfp4_e1m2(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1_e4m3, uint8_t* q2_e4m3,
                                       uint8_t* e8m0_1, uint8_t* e8m0_2, void* stream);
@@ -276,6 +280,22 @@ msd_status_t msd_attn_decode_int8kv_paged(const void* q_bf16, const int8_t* k_ca
  * [s*split_tokens, min(L, (s+1)*split_tokens)) and is walked in tiles of `tile` tokens (splits past L are empty). */
 msd_status_t msd_attn_decode_schedule(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen,
                                       int32_t* tile, int32_t* n_splits, int32_t* split_tokens);
+
+/* The softmax references of the kernel that msd_attn_decode_int8kv (and _spec, _paged) runs for this shape, for a
+ * checker that mirrors it (Sec. 4.3; Alg. 3 lines 6-8).  Head groups of up to 16 rows per KV head: *m_margin = 0,
+ * *sv_growth = 0 - the running maximum itself and alpha_P = (the tile's largest v_scale) / 127.  Wider groups keep the
+ * integer PV sums of consecutive tiles in one accumulator, so their references are held: per context split the
+ * reference of a row moves only when a tile's maximum exceeds it, to that maximum + *m_margin (natural-log units), and
+ * alpha_P = a_ref / 127 where a_ref is set to *sv_growth times the tile's largest v_scale whenever one exceeds it. */
+msd_status_t msd_attn_decode_softmax_rule(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen,
+                                          float* m_margin, float* sv_growth);
+
+/* Debug dumps for bit-exact checks of Alg. 3 lines 1-4.  While a pointer is non-NULL every later attention launch
+ * writes: q_dbg [2, R, D] INT8, the two components of each query row (R = B * q_len * Hq rows in the order of q_bf16);
+ * q_scale_dbg [2, R] FP32, alpha_Q then beta_Q; s_dbg [2, q_len * Hq, T] INT32, the raw sums S1, S2 of row (token s,
+ * head h) -> s * Hq + h against cache row t (T = total_tokens; paged: T = num_blocks * page_size, t the physical row),
+ * written for every token of the sequences, visible to the row or not.  NULL switches a dump off. */
+void msd_debug_set_attn_dump(int8_t* q_dbg, float* q_scale_dbg, int32_t* s_dbg);
 
 /* Comparison kernel, not part of the MSD path: the cache expansion that MSD attention removes (Sec. 2.3; the
  * "Dequant" arm of Sec. 6.4).  out[t,h,:] = bf16(scale[t,h] * cache[t,h,:]), FP32 product rounded to nearest even.

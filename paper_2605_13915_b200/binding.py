@@ -54,6 +54,8 @@ _SIGS = {
     "msd_attn_decode_int8kv": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp,
                                          _vp, _sz, _vp]),
     "msd_attn_decode_schedule": (C.c_int, [_i32] * 6 + [C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
+    "msd_attn_decode_softmax_rule": (C.c_int, [_i32] * 6 + [C.POINTER(_f32), C.POINTER(_f32)]),
+    "msd_debug_set_attn_dump": (None, [_vp, _vp, _vp]),
     "msd_decompose_mxfp4_e1m2": (C.c_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp]),
     "msd_gemm_w4a16_e1m2_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_w4a16_e1m2": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
@@ -106,9 +108,23 @@ def last_device_status():
     _check(lib().msd_last_device_status(_stream()), "msd_last_device_status")
 
 
+def _raw_empty(shape, dtype, device):
+    return torch.empty(shape, dtype=dtype, device=device)
+
+
+def _raw_workspace(nbytes, device="cuda"):
+    return torch.zeros(max(int(nbytes), 1024) + 1024, dtype=torch.uint8, device=device)
+
+
+# Every output tensor and workspace the wrappers create comes from these two hooks, so that a test harness can swap in
+# an allocator of its own (guard bands around each buffer).
+_empty = _raw_empty
+_workspace = _raw_workspace
+
+
 def workspace(nbytes, device="cuda"):
     """A zero-filled, 1024-byte aligned workspace of at least ``nbytes`` bytes."""
-    return torch.zeros(max(int(nbytes), 1024) + 1024, dtype=torch.uint8, device=device)
+    return _workspace(nbytes, device)
 
 
 def _ws_ptr(ws):
@@ -124,10 +140,10 @@ def decompose_int8(x, fractional=False):
     """x [M,K] bfloat16 -> (q1, q2 int8 [M,K], alpha, beta float32 [M]); fractional: scaling constants 127.49 / 254.98."""
     _need_cuda(x)
     M, K = x.shape
-    q1 = torch.empty((M, K), dtype=torch.int8, device=x.device)
-    q2 = torch.empty((M, K), dtype=torch.int8, device=x.device)
-    a = torch.empty(M, dtype=torch.float32, device=x.device)
-    b = torch.empty(M, dtype=torch.float32, device=x.device)
+    q1 = _empty((M, K), torch.int8, x.device)
+    q2 = _empty((M, K), torch.int8, x.device)
+    a = _empty(M, torch.float32, x.device)
+    b = _empty(M, torch.float32, x.device)
     if fractional:
         _check(lib().msd_decompose_int8_ex(_ptr(x), M, K, x.stride(0) if M else K, _ptr(q1), _ptr(q2), _ptr(a), _ptr(b),
                                            SCALING_FRACTIONAL, _stream()), "msd_decompose_int8_ex")
@@ -141,10 +157,10 @@ def decompose_mxfp4(x):
     """x [M,K] bfloat16 -> (q1, q2 uint8 [M,K/2], e8m0_1, e8m0_2 uint8 [M,K/32])."""
     _need_cuda(x)
     M, K = x.shape
-    q1 = torch.empty((M, K // 2), dtype=torch.uint8, device=x.device)
-    q2 = torch.empty((M, K // 2), dtype=torch.uint8, device=x.device)
-    e1 = torch.empty((M, K // 32), dtype=torch.uint8, device=x.device)
-    e2 = torch.empty((M, K // 32), dtype=torch.uint8, device=x.device)
+    q1 = _empty((M, K // 2), torch.uint8, x.device)
+    q2 = _empty((M, K // 2), torch.uint8, x.device)
+    e1 = _empty((M, K // 32), torch.uint8, x.device)
+    e2 = _empty((M, K // 32), torch.uint8, x.device)
     _check(lib().msd_decompose_mxfp4(_ptr(x), M, K, x.stride(0) if M else K, _ptr(q1), _ptr(q2), _ptr(e1), _ptr(e2), _stream()),
            "msd_decompose_mxfp4")
     return q1, q2, e1, e2
@@ -161,8 +177,8 @@ def gemm_w8a16(x, w, w_scale, out_dtype=torch.bfloat16, ws=None, want_acc=False,
     N = w.shape[0]
     if ws is None:
         ws = workspace(gemm_w8a16_workspace_bytes(M, N, K), x.device)
-    y = out if out is not None else torch.empty((M, N), dtype=out_dtype, device=x.device)
-    acc = torch.empty((2, M, N), dtype=torch.int32, device=x.device) if want_acc else None
+    y = out if out is not None else _empty((M, N), out_dtype, x.device)
+    acc = _empty((2, M, N), torch.int32, x.device) if want_acc else None
     wp, wb = _ws_ptr(ws)
     yt = OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32
     if fractional:
@@ -184,7 +200,7 @@ def grouped_gemm_w8a16(x, w, w_scale, group_sizes, out_dtype=torch.bfloat16, ws=
     assert x.shape[0] == M_total and x.shape[1] == K
     if ws is None:
         ws = workspace(int(lib().msd_grouped_gemm_w8a16_workspace_bytes(M_total, max(int(v) for v in group_sizes), E, N, K)), x.device)
-    y = out if out is not None else torch.empty((M_total, N), dtype=out_dtype, device=x.device)
+    y = out if out is not None else _empty((M_total, N), out_dtype, x.device)
     wp, wb = _ws_ptr(ws)
     code = lib().msd_grouped_gemm_w8a16(_ptr(x), _ptr(w), _ptr(w_scale), C.cast(sizes, C.c_void_p), E, N, K, _ptr(y),
                                         OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream())
@@ -203,7 +219,7 @@ def grouped_gemm_w4a16(x, w_fp4, w_e8m0, group_sizes, out_dtype=torch.bfloat16, 
     assert x.shape[0] == M_total and x.shape[1] == K
     if ws is None:
         ws = workspace(int(lib().msd_grouped_gemm_w4a16_workspace_bytes(E, N, K)), x.device)
-    y = out if out is not None else torch.empty((M_total, N), dtype=out_dtype, device=x.device)
+    y = out if out is not None else _empty((M_total, N), out_dtype, x.device)
     wp, wb = _ws_ptr(ws)
     code = lib().msd_grouped_gemm_w4a16(_ptr(x), _ptr(w_fp4), _ptr(w_e8m0), sizes, E, N, K, _ptr(y),
                                         OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream())
@@ -248,7 +264,7 @@ def gemm_dequant_bf16(x, w, w_scale, out_dtype=torch.bfloat16, ws=None):
     N = w.shape[0]
     if ws is None:
         ws = workspace(gemm_dequant_bf16_workspace_bytes(M, N, K), x.device)
-    y = torch.empty((M, N), dtype=out_dtype, device=x.device)
+    y = _empty((M, N), out_dtype, x.device)
     wp, wb = _ws_ptr(ws)
     _check(lib().msd_gemm_dequant_bf16(_ptr(x), _ptr(w), _ptr(w_scale), M, N, K, _ptr(y),
                                        OUT_BF16 if out_dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream()),
@@ -266,7 +282,7 @@ def gemm_w4a16(x, w_fp4, w_e8m0, out_dtype=torch.bfloat16, ws=None, out=None):
     N = w_fp4.shape[0]
     if ws is None:
         ws = workspace(gemm_w4a16_workspace_bytes(M, N, K), x.device)
-    y = out if out is not None else torch.empty((M, N), dtype=out_dtype, device=x.device)
+    y = out if out is not None else _empty((M, N), out_dtype, x.device)
     wp, wb = _ws_ptr(ws)
     _check(lib().msd_gemm_w4a16(_ptr(x), _ptr(w_fp4), _ptr(w_e8m0), M, N, K, _ptr(y),
                                 OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream()), "msd_gemm_w4a16")
@@ -280,14 +296,28 @@ def attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen):
     return tile.value, ns.value, st.value
 
 
+def attn_decode_softmax_rule(B, Hq, Hkv, D, Dv, max_seqlen):
+    """(m_margin in natural-log units, sv_growth) of the held softmax references the kernel for this shape uses;
+    (0, 0): plain running maximum and each tile's own probability scale."""
+    m, g = _f32(0), _f32(0)
+    _check(lib().msd_attn_decode_softmax_rule(B, Hq, Hkv, D, Dv, max_seqlen, C.byref(m), C.byref(g)), "msd_attn_decode_softmax_rule")
+    return m.value, g.value
+
+
+def debug_set_attn_dump(q_dbg=None, q_scale_dbg=None, s_dbg=None):
+    """Attention launches that follow write the query components [2,rows,D] int8, their scales [2,rows] f32 and the raw
+    QK^T sums [2,rows per sequence,T] int32 into these tensors; call without arguments to switch the dumps off."""
+    lib().msd_debug_set_attn_dump(_ptr(q_dbg), _ptr(q_scale_dbg), _ptr(s_dbg))
+
+
 def decompose_mxfp4_e1m2(x):
     """x [M,K] bfloat16 -> (q1, q2 uint8 [M,K] E4M3 bytes of the E1M2 components, e8m0_1, e8m0_2 uint8 [M,K/32])."""
     _need_cuda(x)
     M, K = x.shape
-    q1 = torch.empty((M, K), dtype=torch.uint8, device=x.device)
-    q2 = torch.empty((M, K), dtype=torch.uint8, device=x.device)
-    e1 = torch.empty((M, K // 32), dtype=torch.uint8, device=x.device)
-    e2 = torch.empty((M, K // 32), dtype=torch.uint8, device=x.device)
+    q1 = _empty((M, K), torch.uint8, x.device)
+    q2 = _empty((M, K), torch.uint8, x.device)
+    e1 = _empty((M, K // 32), torch.uint8, x.device)
+    e2 = _empty((M, K // 32), torch.uint8, x.device)
     _check(lib().msd_decompose_mxfp4_e1m2(_ptr(x), M, K, x.stride(0) if M else K, _ptr(q1), _ptr(q2), _ptr(e1), _ptr(e2), _stream()),
            "msd_decompose_mxfp4_e1m2")
     return q1, q2, e1, e2
@@ -300,7 +330,7 @@ def gemm_w4a16_e1m2(x, w_fp4, w_e8m0, out_dtype=torch.bfloat16, ws=None, out=Non
     N = w_fp4.shape[0]
     if ws is None:
         ws = workspace(int(lib().msd_gemm_w4a16_e1m2_workspace_bytes(M, N, K)), x.device)
-    y = out if out is not None else torch.empty((M, N), dtype=out_dtype, device=x.device)
+    y = out if out is not None else _empty((M, N), out_dtype, x.device)
     wp, wb = _ws_ptr(ws)
     code = lib().msd_gemm_w4a16_e1m2(_ptr(x), _ptr(w_fp4), _ptr(w_e8m0), M, N, K, _ptr(y),
                                      OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream())
@@ -316,8 +346,8 @@ def attn_decode_int8kv_spec(q, k, v, k_scale, v_scale, cu_seqlens, max_seqlen, s
     Dv = v.shape[2] if v is not None else int(dv)
     if ws is None:
         ws = workspace(attn_decode_int8kv_workspace_bytes(B, Hq * Sq, Hkv, D, Dv, max_seqlen), q.device)
-    o = torch.empty((B, Sq, Hq, Dv), dtype=torch.bfloat16, device=q.device)
-    lse = torch.empty((B, Sq, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    o = _empty((B, Sq, Hq, Dv), torch.bfloat16, q.device)
+    lse = _empty((B, Sq, Hq), torch.float32, q.device) if want_lse else None
     wp, wb = _ws_ptr(ws)
     code = lib().msd_attn_decode_int8kv_spec(_ptr(q), _ptr(k), _ptr(v), _ptr(k_scale), _ptr(v_scale), _ptr(cu_seqlens), int(k.shape[0]),
                                              max_seqlen, B, Sq, Hq, Hkv, D, Dv, softmax_scale, _ptr(o), _ptr(lse), wp, wb, _stream())
@@ -336,8 +366,8 @@ def attn_decode_int8kv_paged(q, k, v, k_scale, v_scale, block_table, seqlens, pa
     nblk = k.shape[0] // page_size
     if ws is None:
         ws = workspace(attn_decode_int8kv_workspace_bytes(B, Hq, Hkv, D, Dv, max_seqlen), q.device)
-    o = out if out is not None else torch.empty((B, Hq, Dv), dtype=torch.bfloat16, device=q.device)
-    lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    o = out if out is not None else _empty((B, Hq, Dv), torch.bfloat16, q.device)
+    lse = _empty((B, Hq), torch.float32, q.device) if want_lse else None
     wp, wb = _ws_ptr(ws)
     code = lib().msd_attn_decode_int8kv_paged(_ptr(q), _ptr(k), _ptr(v), _ptr(k_scale), _ptr(v_scale), _ptr(block_table), _ptr(seqlens),
                                               nblk, page_size, block_table.shape[1], max_seqlen, B, Hq, Hkv, D, Dv, softmax_scale,
@@ -351,7 +381,7 @@ def kv_dequant_bf16(cache, scale, out=None):
     _need_cuda(cache, scale)
     T, H, D = cache.shape
     if out is None:
-        out = torch.empty((T, H, D), dtype=torch.bfloat16, device=cache.device)
+        out = _empty((T, H, D), torch.bfloat16, cache.device)
     _check(lib().msd_kv_dequant_bf16(cache.data_ptr(), scale.data_ptr(), T, H, D, out.data_ptr(), _stream()),
            "msd_kv_dequant_bf16")
     return out
@@ -370,8 +400,8 @@ def attn_decode_int8kv(q, k, v, k_scale, v_scale, cu_seqlens, max_seqlen, softma
     Dv = v.shape[2] if v is not None else int(dv)
     if ws is None:
         ws = workspace(attn_decode_int8kv_workspace_bytes(B, Hq, Hkv, D, Dv, max_seqlen), q.device)
-    o = out if out is not None else torch.empty((B, Hq, Dv), dtype=torch.bfloat16, device=q.device)
-    lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    o = out if out is not None else _empty((B, Hq, Dv), torch.bfloat16, q.device)
+    lse = _empty((B, Hq), torch.float32, q.device) if want_lse else None
     wp, wb = _ws_ptr(ws)
     code = lib().msd_attn_decode_int8kv(_ptr(q), _ptr(k), _ptr(v), _ptr(k_scale), _ptr(v_scale), _ptr(cu_seqlens), int(k.shape[0]),
                                         max_seqlen, B, Hq, Hkv, D, Dv, softmax_scale, _ptr(o), _ptr(lse), wp, wb, _stream())

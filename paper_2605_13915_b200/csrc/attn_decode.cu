@@ -52,10 +52,18 @@ struct AttnParams {
   int DC, DVT;            // 128-byte chunks of D / Dv
   int n_splits, stages, chunk;   // chunk: tokens per split (a multiple of the tile)
   int v_alias;            // 1: V is the first Dv bytes of the K rows
+  int kv_chunks;          // 128-byte chunks reserved per KV stage (>= DC, and >= DVT when V aliases the K rows)
   int tmem_cols;
   float scale;
   unsigned* status;
   long long* trace;       // nullable diagnostic buffer: 32 clock samples per CTA (first 1024 CTAs)
+  // nullable debug dumps for bit-exact checks (Alg. 3 lines 1-4): the two INT8 components of every query row
+  // [2][B*Sq*Hq][D], their scales [2][B*Sq*Hq] (alpha_Q, beta_Q), and the two INT32 score planes [2][Sq*Hq][dbg_T]
+  // indexed by the token's row in the cache
+  int8_t* q_dbg;
+  float* qs_dbg;
+  int32_t* s_dbg;
+  long long dbg_T;
 };
 
 __device__ __forceinline__ void attn_mark(const AttnParams& p, int slot) {
@@ -77,8 +85,8 @@ __device__ __forceinline__ float ex2_approx(float x) {
 __device__ __forceinline__ void attn_decompose_q_row(const AttnParams& p, int b, int hk, int grp, int h, int lane, uint8_t* img,
                                                      float* alpha_out, float* beta_out) {
   const int r_kv = grp * p.HG + h, sq = r_kv / p.Gr;       // row of this KV head -> (query token, head of the group)
-  const uint4* qrow = reinterpret_cast<const uint4*>(
-      p.q + ((static_cast<long long>(b) * p.Sq + sq) * (p.Hkv * p.Gr) + hk * p.Gr + (r_kv - sq * p.Gr)) * p.D);
+  const long long q_row = (static_cast<long long>(b) * p.Sq + sq) * (p.Hkv * p.Gr) + hk * p.Gr + (r_kv - sq * p.Gr);
+  const uint4* qrow = reinterpret_cast<const uint4*>(p.q + q_row * p.D);
   const int nvec = p.D >> 3;                    // 8 BF16 values per 16-byte load (D % 16 == 0, D <= 640)
   uint4 qv[3];                                  // the whole row stays in registers between the two passes
   float m = 0.0f;
@@ -99,7 +107,13 @@ __device__ __forceinline__ void attn_decompose_q_row(const AttnParams& p, int b,
   m = warp_max(m);
   const float alpha = __fdiv_rn(m, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
   const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f, inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
-  if (lane == 0) { *alpha_out = alpha; *beta_out = beta; }
+  if (lane == 0) {
+    *alpha_out = alpha; *beta_out = beta;
+    if (p.qs_dbg) {
+      p.qs_dbg[q_row] = alpha;
+      p.qs_dbg[static_cast<long long>(p.B) * p.Hq + q_row] = beta;
+    }
+  }
 #pragma unroll
   for (int j = 0; j < 3; ++j) {
     const int i = lane + 32 * j;
@@ -122,6 +136,26 @@ __device__ __forceinline__ void attn_decompose_q_row(const AttnParams& p, int b,
     uint8_t* chunk = img + (d >> 7) * p.Rp * kChunk;
     *reinterpret_cast<uint2*>(chunk + swz_off(h, d & 127)) = make_uint2(o1[0], o1[1]);
     *reinterpret_cast<uint2*>(chunk + swz_off(p.HG + h, d & 127)) = make_uint2(o2[0], o2[1]);
+    if (p.q_dbg) {
+      *reinterpret_cast<uint2*>(p.q_dbg + q_row * p.D + d) = make_uint2(o1[0], o1[1]);
+      *reinterpret_cast<uint2*>(p.q_dbg + (static_cast<long long>(p.B) * p.Hq + q_row) * p.D + d) = make_uint2(o2[0], o2[1]);
+    }
+  }
+}
+
+// Debug dump of one thread's raw QK^T sums (Alg. 3 lines 3-4): token `tok_row` (row of the cache), head slots
+// [hs, hs + n) of head group `grp` of KV head `hk`; c1 / c2 are the two components' accumulators.
+template <int N>
+__device__ __forceinline__ void attn_dump_scores(const AttnParams& p, long long tok_row, int hk, int grp, int hs, int nh,
+                                                 const uint32_t (&c1)[N], const uint32_t (&c2)[N]) {
+#pragma unroll
+  for (int h = 0; h < N; ++h) {
+    if (hs + h < nh) {
+      const int r_kv = grp * p.HG + hs + h, sq = r_kv / p.Gr;
+      const long long row = static_cast<long long>(sq) * (p.Hkv * p.Gr) + hk * p.Gr + (r_kv - sq * p.Gr);
+      p.s_dbg[row * p.dbg_T + tok_row] = static_cast<int32_t>(c1[h]);
+      p.s_dbg[(static_cast<long long>(p.Hq) + row) * p.dbg_T + tok_row] = static_cast<int32_t>(c2[h]);
+    }
   }
 }
 
@@ -148,30 +182,22 @@ attn_qstack_kernel(const AttnParams p, uint8_t* __restrict__ q_img, float* __res
   for (int h = warp; h < nh; h += 8) attn_decompose_q_row(p, b, hk, grp, h, lane, img, sc + h, sc + p.HG + h);
 }
 
-// kMaxHG: head slots one softmax thread looks after (8 or 16); kNH: heads its code is unrolled for (<= kMaxHG);
-// kMaxDVT: 128-wide tiles of Dv; kWG: groups of four softmax warps, each owning kMaxHG of the CTA's kMaxHG*kWG
-// head slots (two groups let one CTA serve 32 heads of a KV head with one pass over its KV tiles).
+// Head groups of up to 16 query rows per KV head (GQA).  kMaxHG: head slots one softmax thread looks after (8 or 16);
+// kNH: heads its code is unrolled for (<= kMaxHG); kMaxDVT: 128-wide tiles of Dv.
 // kPaged: the cache is paged (block table); a template parameter so that the contiguous kernels carry none of it.
-template <int kMaxHG, int kNH, int kMaxDVT, int kWG, bool kPaged>
-__global__ void __launch_bounds__(64 + 128 * kWG, (kNH <= 8 && kMaxDVT == 1 && kWG == 1) ? 3 : 1)
+template <int kMaxHG, int kNH, int kMaxDVT, bool kPaged>
+__global__ void __launch_bounds__(kAttnThreads, (kNH <= 8 && kMaxDVT == 1) ? 3 : 1)
 attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], v_full[4], v_empty[4], s_full[2], p_full[2], q_ready, o_full, o_empty;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
-  // Wide head groups (MLA) take the stacked Q operand ready-made from attn_qstack_kernel: decomposing 32 x 576 values
-  // in every context-split CTA cost a sixth of its lifetime.  Narrow ones (GQA) decompose their few rows themselves,
-  // beside the other CTAs of the SM, and save the extra kernel.
-  constexpr bool kQStack = kWG >= 2;
-  constexpr int kSlots = kMaxHG * kWG;             // head slots of the stacked operands: rows [0,kSlots) first
-  constexpr int kNSW = 4 * kWG;                    // component, rows [kSlots, 2*kSlots) second component
+  // The CTA decomposes its few query rows itself (beside the other CTAs of the SM); wide head groups, where that
+  // would be repeated by every context split, take them from attn_qstack_kernel instead (attn_decode_wide_kernel).
+  constexpr int kSlots = kMaxHG;                   // head slots of the stacked operands: rows [0,kSlots) first
+  constexpr int kNSW = 4;                          // component, rows [kSlots, 2*kSlots) second component
   __shared__ float s_aq[kSlots], s_bq[kSlots];
-  // Running maxima per head slot before / after each tile, three generations (tile t reads [t % 3] and writes
-  // [(t + 1) % 3]; the merge of tile t, which runs after the softmax of tile t + 1, still finds both).  The values are
-  // the same for all 128 threads of a warp group - every thread writes them and reads back what it wrote - so they
-  // need no registers between tiles: with 32 running outputs per thread the MLA kernel has none to spare.
-  __shared__ float s_m[3][kSlots];
-  __shared__ float red[2][kWG][4][kNH + 1];        // per-warp tile maxima, double buffered by tile parity
+  __shared__ float red[2][4][kNH + 1];             // per-warp tile maxima, double buffered by tile parity
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x;
@@ -205,7 +231,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   }
 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
-  const int kv_stage_bytes = (p.DC + (p.v_alias ? 0 : p.DVT)) * kChunkBytes;
+  const int kv_stage_bytes = p.kv_chunks * kChunkBytes;
   uint8_t* sm_q = smem + p.stages * kv_stage_bytes;          // DC chunks of [Rp x 128]
   uint8_t* sm_p = sm_q + p.DC * p.Rp * kChunk;               // [Rp x 128]
 
@@ -217,7 +243,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1);
     // one P barrier per P buffer: the softmax may run one tile ahead of the PV issue, and a single barrier could then
     // be two phases past the one the MMA warp is testing, which a parity test cannot tell from "not yet"
-    mbar_init(&p_full[0], kNSW); mbar_init(&p_full[1], kNSW); mbar_init(&q_ready, kQStack ? 1 : kNSW);
+    mbar_init(&p_full[0], kNSW); mbar_init(&p_full[1], kNSW); mbar_init(&q_ready, kNSW);
     mbar_init(&o_full, 1); mbar_init(&o_empty, kNSW);
     abort_flag = 0;
     mbar_init_fence();
@@ -225,10 +251,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     tma_prefetch_desc(&tmap_v);
   }
   if (warp == 1) tmem_alloc(&tmem_base_slot, p.tmem_cols);
-  if constexpr (!kQStack) {
-    // zero the stacked Q operand (unused head slots and the padding of the last D chunk must be zero)
-    for (int i = threadIdx.x; i < p.DC * p.Rp * kChunk / 16; i += blockDim.x) reinterpret_cast<uint4*>(sm_q)[i] = make_uint4(0, 0, 0, 0);
-  }
+  // zero the stacked Q operand (unused head slots and the padding of the last D chunk must be zero)
+  for (int i = threadIdx.x; i < p.DC * p.Rp * kChunk / 16; i += blockDim.x) reinterpret_cast<uint4*>(sm_q)[i] = make_uint4(0, 0, 0, 0);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -305,16 +329,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       const uint32_t idesc_qk = idesc_dense(2, 1, 1, 0, 0, kTok, p.Rp);     // S8 x S8 -> S32, both K-major
       const uint32_t idesc_pv = idesc_dense(2, 1, 1, 1, 0, kTok, p.Rp);     // A (V^T) MN-major
       bool ok = true;
-      // the stacked Q operand of this (sequence, KV head, head group) comes ready-made from attn_qstack_kernel, the
-      // kernel launched just before this one (the producer's KV loads, which do not depend on it, are already under way)
-      if constexpr (kQStack) {
-        pdl_wait_primary();
-        const int unit_q = blockIdx.y, chunk_bytes = p.Rp * kChunk;
-        mbar_arrive_expect_tx(&q_ready, p.DC * chunk_bytes);
-        for (int c = 0; c < p.DC; ++c)
-          bulk_load(sm_q + c * chunk_bytes, p.q_img + (static_cast<size_t>(unit_q) * p.DC + c) * chunk_bytes, chunk_bytes, &q_ready);
-      }
-      ok = wait_bounded(&q_ready, 0, abort, p.status);
+      ok = wait_bounded(&q_ready, 0, abort, p.status);      // the softmax warps have decomposed the query rows
       // Operand descriptors differ from three templates only in the 16-byte-granular address field (bits 0-13), so each
       // costs one 64-bit add: with 36 MMAs per MLA tile this thread's instruction count is on the critical path.
       const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);         // K-major tiles: K, stacked Q, P
@@ -391,49 +406,30 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     // ------------------------------ softmax + merge warps ------------------------------
     const int quad = warp & 3;
     const int tl = quad * 32 + lane;                // token lane (softmax) / dv lane (merge)
-    const int wi = warp - 2;                        // 0 .. kNSW-1
-    const int hh = wi >> 2;                         // which group of head slots this warp looks after
-    const int wq = wi & 3;
-    const int hs0 = hh * kMaxHG;                    // its first head slot
-    if constexpr (kQStack) {
-      // alpha_Q / beta_Q of this CTA's heads, computed by attn_qstack_kernel (launched just before this kernel)
-      pdl_wait_primary();
-      const int i = threadIdx.x - 64;
-      const float* sc = p.q_scales + static_cast<size_t>(blockIdx.y) * 2 * p.HG;
-      if (i < kSlots) { s_aq[i] = __ldg(sc + i); s_bq[i] = __ldg(sc + p.HG + i); }
-    } else {
-      // c1: decompose the query rows of this CTA's heads (one warp per head, round robin) into the stacked operand
-      for (int h = wi; h < nh; h += kNSW) attn_decompose_q_row(p, b, hk, grp, h, lane, sm_q, &s_aq[h], &s_bq[h]);
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&q_ready);         // the stacked Q operand is in shared memory
-    }
-    named_bar_sync(8, 128 * kWG);                   // s_aq / s_bq visible to all softmax warps
+    const int wi = warp - 2;                        // 0 .. 3
+    const int wq = wi;
+    constexpr int hs0 = 0;                          // first head slot of this warp
+    // c1: decompose the query rows of this CTA's heads (one warp per head, round robin) into the stacked operand
+    for (int h = wi; h < nh; h += kNSW) attn_decompose_q_row(p, b, hk, grp, h, lane, sm_q, &s_aq[h], &s_bq[h]);
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&q_ready);           // the stacked Q operand is in shared memory
+    named_bar_sync(8, 128);                         // s_aq / s_bq visible to all softmax warps
     if (threadIdx.x == 64) attn_mark(p, 3);
-    const int bar_id = 1 + hh;                      // each group of four warps synchronises on its own
+    const int bar_id = 1;
 
     // running state per head; scores are kept in the log2 domain (log2(e) is folded into the key scale)
-    // Wide head groups (MLA) keep the warp-group-uniform state in shared memory (s_m, s_aq, s_bq above); the others
-    // have registers to spare and keep it there, off the critical path of their much shorter tiles.
-    constexpr bool kSmemState = kWG >= 2;
-    constexpr int kRegState = kSmemState ? 1 : kNH;
+    // the state that is uniform across the four warps (running maxima, query scales) lives in registers
+    constexpr int kRegState = kNH;
     float l_part[kNH];
     float m_run[kRegState], aq[kRegState], bq[kRegState], resc_keep[kRegState], resc_next[kRegState];
     float o_run[kMaxDVT][kNH];
 #pragma unroll
     for (int h = 0; h < kNH; ++h) {
       l_part[h] = 0.0f;
-      if constexpr (kSmemState) {
-        s_m[0][hs0 + h] = -INFINITY;
-        if (h == 0) {       // lane l keeps the query scales of head slot hs0 + l (zero for absent heads)
-          aq[0] = (lane < kNH && hs0 + lane < nh) ? s_aq[hs0 + lane] : 0.0f;
-          bq[0] = (lane < kNH && hs0 + lane < nh) ? s_bq[hs0 + lane] : 0.0f;
-        }
-      } else {
-        m_run[h] = -INFINITY;
-        aq[h] = (hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f;
-        bq[h] = (hs0 + h < nh) ? s_bq[hs0 + h] : 0.0f;
-      }
+      m_run[h] = -INFINITY;
+      aq[h] = (hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f;
+      bq[h] = (hs0 + h < nh) ? s_bq[hs0 + h] : 0.0f;
 #pragma unroll
       for (int j = 0; j < kMaxDVT; ++j) o_run[j][h] = 0.0f;
     }
@@ -478,19 +474,22 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         tmem_ldw<kMaxHG>(srow + hs0, v1);
         tmem_ldw<kMaxHG>(srow + kSlots + hs0, v2);
         tmem_ld_wait();
+        if (p.s_dbg && valid) {
+          long long tok_row = seq0 + tok_rel;
+          if constexpr (kPaged) tok_row = static_cast<long long>(__ldg(bt + (tok_rel >> p.page_shift))) * p.page + (tok_rel & (p.page - 1));
+          attn_dump_scores<kMaxHG>(p, tok_row, hk, grp, hs0, nh, v1, v2);
+        }
 #pragma unroll
         for (int h = 0; h < kNH; ++h)
         {
-          // (shared-memory state: lane h holds the scales of head h, see above)
-          const float a_q = kSmemState ? __shfl_sync(0xffffffffu, aq[0], h) : aq[kSmemState ? 0 : h];
-          const float b_q = kSmemState ? __shfl_sync(0xffffffffu, bq[0], h) : bq[kSmemState ? 0 : h];
+          const float a_q = aq[h], b_q = bq[h];
           bool vh = valid;
           if (p.Sq > 1) vh = valid && tok_rel < L - p.Sq + 1 + (grp * p.HG + hs0 + h) / p.Gr;    // causal among the new tokens
           s[h] = vh ? __fmaf_rn(a_q, static_cast<float>(static_cast<int32_t>(v1[h])), b_q * static_cast<float>(static_cast<int32_t>(v2[h]))) * ks : -INFINITY;
         }
       }
       // c4: tile maxima per head (and of the value scales) over the 128 token lanes
-      float (*rb)[kNH + 1] = red[t & 1][hh];
+      float (*rb)[kNH + 1] = red[t & 1];
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
         const float wm = warp_max(s[h]);
@@ -501,21 +500,16 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         if (lane == 0) rb[wq][kNH] = wv;
       }
       named_bar_sync(bar_id, 128);  // one barrier per tile: the other parity buffer is rewritten only after the next one
-      const float* m_rd = s_m[t % 3];
-      float* m_wr = s_m[(t + 1) % 3];
-      // running maximum of every head before and after the tile; rescale factor of what was accumulated so far.
-      // Register state: all heads first (as many independent exponentials in flight as there are heads); shared-memory
-      // state: inside the P loop below, head by head, so that nothing but the scores is alive across it.
+      // running maximum of every head before and after the tile; rescale factor of what was accumulated so far
+      // (all heads first: as many independent exponentials in flight as there are heads)
       float mn_t[kRegState], resc_t[kRegState];
-      if constexpr (!kSmemState) {
 #pragma unroll
-        for (int h = 0; h < kNH; ++h) {
-          const float mt = fmaxf(fmaxf(rb[0][h], rb[1][h]), fmaxf(rb[2][h], rb[3][h]));
-          mn_t[h] = fmaxf(m_run[h], mt);
-          resc_t[h] = (m_run[h] == -INFINITY) ? 0.0f : ex2_approx(m_run[h] - mn_t[h]);
-          m_run[h] = mn_t[h];
-          resc_out[h] = resc_t[h];
-        }
+      for (int h = 0; h < kNH; ++h) {
+        const float mt = fmaxf(fmaxf(rb[0][h], rb[1][h]), fmaxf(rb[2][h], rb[3][h]));
+        mn_t[h] = fmaxf(m_run[h], mt);
+        resc_t[h] = (m_run[h] == -INFINITY) ? 0.0f : ex2_approx(m_run[h] - mn_t[h]);
+        m_run[h] = mn_t[h];
+        resc_out[h] = resc_t[h];
       }
       const float vs_max = fmaxf(fmaxf(rb[0][kNH], rb[1][kNH]), fmaxf(rb[2][kNH], rb[3][kNH]));
       // c5: P = exp(S - m), fold the value scale, two-pass INT8 with the fixed scale alpha_P = max(v_scale)/127
@@ -523,31 +517,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       beta_p = alpha_p * (1.0f / 254.0f);
       const float inv_a = alpha_p > 0.0f ? __frcp_rn(alpha_p) : 0.0f, inv_b = beta_p > 0.0f ? __frcp_rn(beta_p) : 0.0f;
       uint8_t* pbuf = sm_p + (t & 1) * p.Rp * kChunk;      // PV of tile t-2 (same buffer) finished before merge(t-2)
-      // Shared-memory state: the new running maximum and the rescale factor of head h are the same for every thread of
-      // the warp group; lane h of each warp computes them once and the others fetch them by shuffle (four shared
-      // loads, the maxima and an exponential per head and THREAD before).
-      float mn_lane = 0.0f, resc_lane = 0.0f;
-      if constexpr (kSmemState) {
-        if (lane < kNH) {
-          const float mt = fmaxf(fmaxf(rb[0][lane], rb[1][lane]), fmaxf(rb[2][lane], rb[3][lane]));
-          const float m_old = m_rd[hs0 + lane];
-          mn_lane = fmaxf(m_old, mt);
-          resc_lane = (m_old == -INFINITY) ? 0.0f : ex2_approx(m_old - mn_lane);
-          m_wr[hs0 + lane] = mn_lane;
-        }
-        resc_out[0] = resc_lane;          // lane h carries head h's factor to the merge of this tile
-      }
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
         // branch-free: an absent head or a token past the end contributes P = 0 (s is -inf there)
-        float mn, resc;
-        if constexpr (kSmemState) {
-          mn = __shfl_sync(0xffffffffu, mn_lane, h);
-          resc = __shfl_sync(0xffffffffu, resc_lane, h);
-        } else {
-          mn = mn_t[kSmemState ? 0 : h];
-          resc = resc_t[kSmemState ? 0 : h];
-        }
+        const float mn = mn_t[h], resc = resc_t[h];
         // (a row that has seen no visible token yet keeps m = -inf: the clamp turns -inf - -inf into -inf, P = 0)
         const float pr = (hs0 + h < nh) ? ex2_approx(s[h] - fmaxf(mn, -1e30f)) : 0.0f;
         l_part[h] = __fmaf_rn(l_part[h], resc, pr);
@@ -581,15 +554,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       if (!ok) break;
       if (threadIdx.x == 64 && t < 6) attn_mark(p, 6 + 4 * t);
       tc_fence_after();
-      float resc_cur[kNH];                 // e^(m before tile t - m after tile t), recomputed from the stored maxima
+      float resc_cur[kNH];                 // e^(m before tile t - m after tile t), from the softmax of tile t
 #pragma unroll
-      for (int h = 0; h < kNH; ++h) {
-        if constexpr (kSmemState) {
-          resc_cur[h] = __shfl_sync(0xffffffffu, resc_keep[0], h);       // computed by lane h in the softmax of tile t
-        } else {
-          resc_cur[h] = resc_keep[h];
-        }
-      }
+      for (int h = 0; h < kNH; ++h) resc_cur[h] = resc_keep[h];
 #pragma unroll
       for (int j = 0; j < kMaxDVT; ++j) {
         if (j < p.DVT) {
@@ -617,7 +584,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     if (threadIdx.x == 64) attn_mark(p, 28);
     // partial results of this split: running max, sum of P and unnormalised output per head
     if (ok) {
-      float (*rb)[kNH + 1] = red[ntiles & 1][hh];
+      float (*rb)[kNH + 1] = red[ntiles & 1];
       named_bar_sync(bar_id, 128);
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
@@ -632,7 +599,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         if (hs0 + h < nh) {
           float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + hs0 + h) * p.n_splits + split) * (p.Dv + 2);
           // the running maximum goes out in natural-log units (it was kept in the log2 domain)
-          if (tl == 0) { dst[0] = (kSmemState ? s_m[ntiles % 3][hs0 + h] : m_run[kSmemState ? 0 : h]) * 0.6931471805599453f; dst[1] = rb[0][h] + rb[1][h] + rb[2][h] + rb[3][h]; }
+          if (tl == 0) { dst[0] = m_run[h] * 0.6931471805599453f; dst[1] = rb[0][h] + rb[1][h] + rb[2][h] + rb[3][h]; }
 #pragma unroll
           for (int j = 0; j < kMaxDVT; ++j)
             if (j < p.DVT && j * kChunk + tl < p.Dv) dst[2 + j * kChunk + tl] = o_run[j][h];
@@ -650,7 +617,519 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------------------------
+// Wide head groups (more than 16 query rows per KV head, e.g. an MLA latent cache shared by 64 heads): 32 head slots per
+// CTA, sixteen softmax warps (four groups of four; a group owns 8 head slots, a thread one token lane of them).
+//
+// The PV products of consecutive tiles accumulate in the SAME INT32 tensor-memory accumulators (Alg. 3 lines 10-12
+// applied once per run of tiles): that needs the reference maximum of every head and the probability scale alpha_P to
+// stay put between tiles, so both are HELD - the reference moves only when a score exceeds it, to that tile's maximum
+// plus kHoldMarginLog2 octaves, and alpha_P = a_ref / 127 with a_ref raised to kHoldScaleGrowth times the tile's largest
+// value scale when one exceeds it.  P <= 1 and P * v_scale <= a_ref hold at all times, so nothing clips.  A tile in
+// which nothing is exceeded (almost all of them) costs the softmax warps no reduction and no barrier among
+// themselves: scores -> exp2 -> two-pass INT8 -> shared memory.  Otherwise every warp learns it from a stamp next to
+// the P buffer, the accumulators are drained into the FP32 running output with the old scales, the references move,
+// and P of that tile is written again before the MMA warp may use it.
+//
+// L2 prefetch: a KV stage is 80 KB for a 576-byte row, so only two fit in shared memory and a tile can be requested
+// only when the PV product two tiles back is done.  The producer therefore asks for the tiles further ahead with
+// cp.async.bulk.prefetch.tensor (no shared memory needed): HBM keeps streaming and the load that follows hits L2.
+constexpr float kHoldMarginLog2 = 2.0f;
+constexpr float kHoldScaleGrowth = 1.25f;
+constexpr int kWideHS = 8;                          // head slots per softmax thread
+constexpr int kWideWG = 4;                          // groups of four softmax warps
+constexpr int kWideSlots = kWideHS * kWideWG;       // 32 head slots per CTA, Rp = 64 stacked rows
+constexpr int kWideThreads = 64 + 128 * kWideWG;
+constexpr int kWidePrefetchTiles = 4;
+
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* m, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+               ::"l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+template <bool kPaged>
+__global__ void __launch_bounds__(kWideThreads, 1)
+attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], v_full[4], v_empty[4], s_full[2], p_full[2], q_ready, o_full, o_last, p_redo;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+  __shared__ int flush_stamp[2];                    // tile number + 1 of the last tile whose references had to move, per P buffer
+  __shared__ float s_aq[kWideSlots];
+  __shared__ float red[kWideWG][4][kWideHS + 1];    // per-warp tile maxima (slow path only)
+  constexpr int kNSW = 4 * kWideWG;
+  constexpr int kDVT = 4;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x;
+  int unit = blockIdx.y;
+  const int grp = unit % p.groups; unit /= p.groups;
+  const int hk = unit % p.Hkv;
+  const int b = unit / p.Hkv;
+  const int32_t* bt = kPaged ? p.block_table + static_cast<long long>(b) * p.max_blocks : nullptr;
+  const int seq0 = kPaged ? 0 : p.cu[b];
+  const int L = kPaged ? p.seqlens[b] : p.cu[b + 1] - seq0;
+  const int t_begin = split * p.chunk;
+  const int t_end = min(L, t_begin + p.chunk);
+  const int h0 = hk * p.G + grp * p.HG;
+  const int nh = min(p.HG, p.G - grp * p.HG);
+  const int ntiles = (t_end > t_begin) ? (t_end - t_begin + kTok - 1) / kTok : 0;
+  if (threadIdx.x == 0 && p.trace) {
+    attn_mark(p, 0);
+    unsigned long long g;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g));
+    const int cta = blockIdx.y * gridDim.x + blockIdx.x;
+    if (cta < 1024) { p.trace[cta * 32 + 1] = static_cast<long long>(g); p.trace[cta * 32 + 2] = ntiles; }
+  }
+
+  if (ntiles == 0) {      // nothing in this split: neutral partials, before any barrier or TMEM use
+    for (int i = threadIdx.x; i < nh * (p.Dv + 2); i += blockDim.x) {
+      const int h = i / (p.Dv + 2), e = i % (p.Dv + 2);
+      float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + h) * p.n_splits + split) * (p.Dv + 2);
+      dst[e] = (e == 0) ? -INFINITY : 0.0f;
+    }
+    return;
+  }
+
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+  const int kv_stage_bytes = p.kv_chunks * kChunkBytes;
+  uint8_t* sm_q = smem + p.stages * kv_stage_bytes;          // DC chunks of [Rp x 128]
+  uint8_t* sm_p = sm_q + p.DC * p.Rp * kChunk;               // two buffers of [Rp x 128]
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1);
+      mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
+    }
+    mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1);
+    mbar_init(&p_full[0], kNSW); mbar_init(&p_full[1], kNSW);
+    mbar_init(&q_ready, 1);
+    mbar_init(&o_full, 1); mbar_init(&o_last, 1); mbar_init(&p_redo, kNSW);
+    abort_flag = 0;
+    flush_stamp[0] = 0; flush_stamp[1] = 0;
+    mbar_init_fence();
+    tma_prefetch_desc(&tmap_k);
+    tma_prefetch_desc(&tmap_v);
+  }
+  if (warp == 1) tmem_alloc(&tmem_base_slot, p.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  const uint32_t tmem_o = tmem_base + 2 * p.Rp;             // O^T tiles after the two S^T buffers
+  volatile int* abort = &abort_flag;
+  volatile int* stamp = flush_stamp;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer: K (and V) tiles ------------------------------
+    if (lane == 0) {
+      const int k_bytes = p.DC * kChunkBytes, v_bytes = p.DVT * kChunkBytes;
+      int kq = 0, vq = p.v_alias ? ntiles : 0;
+      if constexpr (!kPaged) {
+        // tiles that do not fit shared memory yet: ask for them in L2
+        for (int t = p.stages; t < min(ntiles, p.stages + kWidePrefetchTiles); ++t) {
+          for (int c = 0; c < p.DC; ++c) tma_prefetch_3d(&tmap_k, c * kChunk, hk, seq0 + t_begin + t * kTok);
+          if (!p.v_alias)
+            for (int j = 0; j < p.DVT; ++j) tma_prefetch_3d(&tmap_v, j * kChunk, hk, seq0 + t_begin + t * kTok);
+        }
+      }
+      long long t_idle = clock64();
+      while (kq < ntiles || vq < ntiles) {
+        bool progressed = false;
+        if (kq < ntiles && mbar_test_wait(&kv_empty[kq % p.stages], ((kq / p.stages) & 1) ^ 1)) {
+          const int st = kq % p.stages;
+          uint8_t* dst = smem + st * kv_stage_bytes;
+          const int u0 = t_begin + kq * kTok;
+          if constexpr (!kPaged) {
+            mbar_arrive_expect_tx(&kv_full[st], k_bytes);
+            for (int c = 0; c < p.DC; ++c) tma_load_3d(dst + c * kChunkBytes, &tmap_k, c * kChunk, hk, seq0 + u0, &kv_full[st]);
+            const int tp = kq + kWidePrefetchTiles;
+            if (kq >= p.stages && tp < ntiles)
+              for (int c = 0; c < p.DC; ++c) tma_prefetch_3d(&tmap_k, c * kChunk, hk, seq0 + t_begin + tp * kTok);
+          } else {
+            const int npg = min(kTok >> p.page_shift, (t_end - u0 + p.page - 1) >> p.page_shift);
+            mbar_arrive_expect_tx(&kv_full[st], p.DC * kChunk * p.page * npg);
+            for (int pg = 0; pg < npg; ++pg) {
+              const int tok = __ldg(bt + (u0 >> p.page_shift) + pg) * p.page;
+              for (int c = 0; c < p.DC; ++c)
+                tma_load_3d(dst + c * kChunkBytes + pg * p.page * kChunk, &tmap_k, c * kChunk, hk, tok, &kv_full[st]);
+            }
+          }
+          ++kq;
+          progressed = true;
+        }
+        if (vq < ntiles && mbar_test_wait(&v_empty[vq % p.stages], ((vq / p.stages) & 1) ^ 1)) {
+          const int st = vq % p.stages;
+          uint8_t* dst = smem + st * kv_stage_bytes + k_bytes;
+          const int u0 = t_begin + vq * kTok;
+          if constexpr (!kPaged) {
+            mbar_arrive_expect_tx(&v_full[st], v_bytes);
+            for (int j = 0; j < p.DVT; ++j) tma_load_3d(dst + j * kChunkBytes, &tmap_v, j * kChunk, hk, seq0 + u0, &v_full[st]);
+            const int tp = vq + kWidePrefetchTiles;
+            if (vq >= p.stages && tp < ntiles)
+              for (int j = 0; j < p.DVT; ++j) tma_prefetch_3d(&tmap_v, j * kChunk, hk, seq0 + t_begin + tp * kTok);
+          } else {
+            const int npg = min(kTok >> p.page_shift, (t_end - u0 + p.page - 1) >> p.page_shift);
+            mbar_arrive_expect_tx(&v_full[st], p.DVT * kChunk * p.page * npg);
+            for (int pg = 0; pg < npg; ++pg) {
+              const int tok = __ldg(bt + (u0 >> p.page_shift) + pg) * p.page;
+              for (int j = 0; j < p.DVT; ++j)
+                tma_load_3d(dst + j * kChunkBytes + pg * p.page * kChunk, &tmap_v, j * kChunk, hk, tok, &v_full[st]);
+            }
+          }
+          ++vq;
+          progressed = true;
+        }
+        if (progressed) {
+          t_idle = clock64();
+        } else {
+          if (*abort) break;
+          if (clock64() - t_idle > kWaitBudgetCycles) {
+            *abort = 1;
+            atomicMax(p.status, kStatusTimeout);
+            break;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      const uint32_t idesc_qk = idesc_dense(2, 1, 1, 0, 0, kTok, p.Rp);     // S8 x S8 -> S32, both K-major
+      const uint32_t idesc_pv = idesc_dense(2, 1, 1, 1, 0, kTok, p.Rp);     // A (V^T) MN-major
+      bool ok = true;
+      // the stacked Q operand of this (sequence, KV head, head group) comes ready-made from attn_qstack_kernel, the
+      // kernel launched just before this one (the producer's KV loads, which do not depend on it, are already under way)
+      pdl_wait_primary();
+      {
+        const int unit_q = blockIdx.y, chunk_bytes = p.Rp * kChunk;
+        mbar_arrive_expect_tx(&q_ready, p.DC * chunk_bytes);
+        for (int c = 0; c < p.DC; ++c)
+          bulk_load(sm_q + c * chunk_bytes, p.q_img + (static_cast<size_t>(unit_q) * p.DC + c) * chunk_bytes, chunk_bytes, &q_ready);
+      }
+      ok = wait_bounded(&q_ready, 0, abort, p.status);
+      const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);         // K-major tiles: K, stacked Q, P
+      const uint64_t dvt = smem_desc(0, 16384, 1024, kSwizzle128B);     // V^T read MN-major from the token-major tile
+      const uint64_t q_enc = dk + (smem_u32(sm_q) >> 4);
+      const uint64_t p_enc = dk + (smem_u32(sm_p) >> 4);
+      const uint32_t smem_enc = smem_u32(smem) >> 4;
+      const uint32_t q_step = static_cast<uint32_t>(p.Rp * kChunk) >> 4, p_step = q_step;
+      auto issue_qk = [&](int t) {
+        const int st = t % p.stages;
+        tc_fence_after();
+        uint64_t ka = dk + smem_enc + static_cast<uint32_t>(st * (kv_stage_bytes >> 4));
+        uint64_t qa = q_enc;
+        const uint32_t d = tmem_base + (t & 1) * p.Rp;
+        for (int c = 0; c < p.DC; ++c) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) mma_i8(d, ka + 2 * k, qa + 2 * k, idesc_qk, (c > 0 || k > 0) ? 1u : 0u);
+          ka += kChunkBytes >> 4;
+          qa += q_step;
+        }
+        tc_commit(&s_full[t & 1]);
+        if (!p.v_alias) tc_commit(&kv_empty[st]);       // separate V: the K buffer is free once QK^T has read it
+      };
+      // PV of tile t, added to what the accumulators hold unless `fresh`
+      auto issue_pv = [&](int t, bool fresh) {
+        tc_fence_after();
+        const int st = t % p.stages;
+        uint64_t va = dvt + smem_enc + static_cast<uint32_t>(st * (kv_stage_bytes >> 4)) +
+                      (p.v_alias ? 0u : static_cast<uint32_t>(p.DC * (kChunkBytes >> 4)));
+        const uint64_t pa = p_enc + (t & 1) * p_step;
+        uint32_t d = tmem_o;
+        for (int j = 0; j < p.DVT; ++j) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k)        // 32 tokens per MMA: four 8-token groups of 1024 bytes
+            mma_i8(d, va + k * (4096 >> 4), pa + 2 * k, idesc_pv, (k > 0 || !fresh) ? 1u : 0u);
+          va += kChunkBytes >> 4;
+          d += p.Rp;
+        }
+        // o_full counts every PV product (a drain in mid-split waits for the one before its tile: at that point the
+        // barrier is at most one phase behind, so a parity test is unambiguous); the last one has a barrier of its own
+        tc_commit(t == ntiles - 1 ? &o_last : &o_full);
+        tc_commit(p.v_alias ? &kv_empty[st] : &v_empty[st]);
+      };
+      // QK^T(q) needs KV tile q in shared memory and the score buffer q&1 read (P of tile q-2 final);
+      // PV(v) needs P of tile v final (written, and rewritten when the references had to move) and QK^T(v) issued.
+      int q = 0, v = 0, n_slow = 0;
+      long long t_idle = clock64();
+      while (ok && v < ntiles) {
+        bool progressed = false;
+        if (q < ntiles && q < v + 2 && mbar_test_wait(&kv_full[q % p.stages], (q / p.stages) & 1)) {
+          issue_qk(q);
+          ++q;
+          progressed = true;
+        }
+        if (v < q && mbar_test_wait(&p_full[v & 1], (v >> 1) & 1) &&
+            (p.v_alias || mbar_test_wait(&v_full[v % p.stages], (v / p.stages) & 1))) {
+          bool fresh = false;
+          if (stamp[v & 1] == v + 1) {
+            // the softmax warps drain the accumulators and write P of this tile again
+            ok = wait_bounded(&p_redo, n_slow & 1, abort, p.status);
+            if (!ok) break;
+            ++n_slow;
+            fresh = true;
+          }
+          issue_pv(v, fresh);
+          ++v;
+          progressed = true;
+        }
+        if (progressed) {
+          t_idle = clock64();
+        } else {
+          if (*abort) { ok = false; break; }
+          if (clock64() - t_idle > kWaitBudgetCycles) {
+            *abort = 1;
+            atomicMax(p.status, kStatusTimeout);
+            ok = false;
+          }
+        }
+      }
+    }
+  } else {
+    // ------------------------------ softmax warps ------------------------------
+    const int quad = warp & 3;
+    const int tl = quad * 32 + lane;                // token lane (softmax) / dv lane (drain)
+    const int wi = warp - 2;                        // 0 .. 15
+    const int hh = wi >> 2;                         // which group of head slots this warp looks after
+    const int wq = wi & 3;
+    const int hs0 = hh * kWideHS;                   // its first head slot
+    {
+      // alpha_Q of this CTA's heads, computed by attn_qstack_kernel (launched just before this kernel);
+      // beta_Q = alpha_Q / 254 is applied as a constant factor
+      pdl_wait_primary();
+      const int i = threadIdx.x - 64;
+      const float* sc = p.q_scales + static_cast<size_t>(blockIdx.y) * 2 * p.HG;
+      if (i < kWideSlots) s_aq[i] = __ldg(sc + i);
+    }
+    named_bar_sync(8, 128 * kWideWG);
+    if (threadIdx.x == 64) attn_mark(p, 3);
+    const int bar_id = 1 + hh;
+
+    // Per head slot: query scale, NEGATED reference maximum in the log2 domain (+1e30 while no score has been seen,
+    // -1e30 for a slot without a head, so that "score + nm > 0" means "exceeds the reference"), partial sum of P over
+    // this thread's tokens, running output of this thread's dv lane.
+    float aq[kWideHS], nm[kWideHS], l_part[kWideHS], o_run[kDVT][kWideHS];
+#pragma unroll
+    for (int h = 0; h < kWideHS; ++h) {
+      const bool present = hs0 + h < nh;
+      aq[h] = present ? s_aq[hs0 + h] : 0.0f;
+      nm[h] = present ? 1e30f : -1e30f;
+      l_part[h] = 0.0f;
+#pragma unroll
+      for (int j = 0; j < kDVT; ++j) o_run[j][h] = 0.0f;
+    }
+    float a_ref = 0.0f, alpha_p = 0.0f, inv_a = 0.0f, inv_b = 0.0f;
+    const float kLog2e = 1.4426950408889634f;
+    const float scale2 = p.scale * kLog2e;
+    const float kInv254 = 1.0f / 254.0f;
+    const float kMagic = 12582912.0f;
+
+    auto load_scales = [&](int t, float& ks_out, float& vs_out) {
+      const int tok_rel = t_begin + t * kTok + tl;
+      const bool valid = t < ntiles && tok_rel < t_end;
+      long long sidx;
+      if constexpr (kPaged) {
+        const long long prow = valid ? static_cast<long long>(__ldg(bt + (tok_rel >> p.page_shift))) * p.page + (tok_rel & (p.page - 1)) : 0;
+        sidx = prow * p.Hkv + hk;
+      } else {
+        sidx = static_cast<long long>(seq0 + tok_rel) * p.Hkv + hk;
+      }
+      ks_out = valid ? __ldg(p.k_scale + sidx) : 0.0f;
+      vs_out = valid ? __ldg(p.v_scale + sidx) : 0.0f;
+    };
+    // c3: scores of this thread's token against its 8 head slots in the log2 domain (-inf where the token is past the
+    // end of the split or not visible to the row)
+    auto load_scores = [&](int t, float ks, float (&s)[kWideHS]) {
+      const int tok_rel = t_begin + t * kTok + tl;
+      const bool valid = tok_rel < t_end;
+      const uint32_t srow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + (t & 1) * p.Rp;
+      uint32_t v1[kWideHS], v2[kWideHS];
+      tmem_ld8(srow + hs0, v1);
+      tmem_ld8(srow + kWideSlots + hs0, v2);
+      tmem_ld_wait();
+      if (p.s_dbg && valid) {
+        long long tok_row = seq0 + tok_rel;
+        if constexpr (kPaged) tok_row = static_cast<long long>(__ldg(bt + (tok_rel >> p.page_shift))) * p.page + (tok_rel & (p.page - 1));
+        attn_dump_scores<kWideHS>(p, tok_row, hk, grp, hs0, nh, v1, v2);
+      }
+#pragma unroll
+      for (int h = 0; h < kWideHS; ++h) {
+        bool vh = valid;
+        if (p.Sq > 1) vh = valid && tok_rel < L - p.Sq + 1 + (grp * p.HG + hs0 + h) / p.Gr;    // causal among the new tokens
+        const float tsum = __fmaf_rn(static_cast<float>(static_cast<int32_t>(v2[h])), kInv254, static_cast<float>(static_cast<int32_t>(v1[h])));
+        s[h] = vh ? (aq[h] * ks) * tsum : -INFINITY;
+      }
+    };
+    // c4-c5: P = 2^(s - reference), value scale folded in, two-pass INT8 with the scale in force, into P buffer t&1.
+    // Returns the largest s - reference of this thread (> 0: the reference must move).
+    auto write_p = [&](int t, const float (&s)[kWideHS], float vs, float (&pl)[kWideHS]) -> float {
+      uint8_t* pbuf = sm_p + (t & 1) * p.Rp * kChunk;
+      float xm = -INFINITY;
+#pragma unroll
+      for (int h = 0; h < kWideHS; ++h) {
+        const float x = s[h] + nm[h];
+        xm = fmaxf(xm, x);
+        const float pr = ex2_approx(x);
+        pl[h] = pr;
+        const float pt = pr * vs;
+        // 1.5 * 2^23 trick: the rounded integer lands in the low mantissa bits (P <= 1, v_scale <= a_ref: no clamps)
+        const float u1 = __fmaf_rn(pt, inv_a, kMagic);
+        const float r = __fmaf_rn(-alpha_p, u1 - kMagic, pt);
+        const float u2 = __fmaf_rn(r, inv_b, kMagic);
+        pbuf[swz_off(hs0 + h, tl)] = static_cast<uint8_t>(__float_as_uint(u1));
+        pbuf[swz_off(kWideSlots + hs0 + h, tl)] = static_cast<uint8_t>(__float_as_uint(u2));
+      }
+      return xm;
+    };
+    // Alg. 3 line 12 for everything accumulated since the last drain: O <- O * resc + alpha_P (O1 + O2 / 254)
+    auto drain = [&](const float (&resc)[kWideHS], float alpha_old) {
+#pragma unroll
+      for (int j = 0; j < kDVT; ++j) {
+        if (j < p.DVT) {
+          const uint32_t orow = tmem_o + (static_cast<uint32_t>(quad * 32) << 16) + j * p.Rp;
+          uint32_t v1[kWideHS], v2[kWideHS];
+          tmem_ld8(orow + hs0, v1);
+          tmem_ld8(orow + kWideSlots + hs0, v2);
+          tmem_ld_wait();
+#pragma unroll
+          for (int h = 0; h < kWideHS; ++h) {
+            const float acc = __fmaf_rn(static_cast<float>(static_cast<int32_t>(v2[h])), kInv254, static_cast<float>(static_cast<int32_t>(v1[h])));
+            o_run[j][h] = __fmaf_rn(o_run[j][h], resc[h], alpha_old * acc);
+          }
+        }
+      }
+    };
+
+    bool ok = true;
+    int n_slow = 0;
+    float ks_pre, vs_pre;
+    load_scales(0, ks_pre, vs_pre);
+    for (int t = 0; t < ntiles && ok; ++t) {
+      const float ks = ks_pre * scale2, vs = vs_pre;
+      load_scales(t + 1, ks_pre, vs_pre);
+      ok = wait_bounded(&s_full[t & 1], (t >> 1) & 1, abort, p.status);
+      if (!ok) break;
+      if (threadIdx.x == 64 && t < 6) attn_mark(p, 4 + 4 * t);
+      tc_fence_after();
+      float s[kWideHS], pl[kWideHS];
+      load_scores(t, ks, s);
+      const float xm = write_p(t, s, vs, pl);
+      const bool exceeded = __any_sync(0xffffffffu, xm > 0.0f || vs > a_ref);
+      if (exceeded && lane == 0) stamp[t & 1] = t + 1;
+      fence_proxy_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&p_full[t & 1]);
+      if (threadIdx.x == 64 && t < 6) attn_mark(p, 5 + 4 * t);
+      // every softmax warp has written its part (and its verdict): did any reference have to move?
+      ok = wait_bounded(&p_full[t & 1], (t >> 1) & 1, abort, p.status);
+      if (!ok) break;
+      if (stamp[t & 1] == t + 1) {
+        // ---- the references move: tile maxima per head over the group's 128 tokens, largest value scale ----
+#pragma unroll
+        for (int h = 0; h < kWideHS; ++h) {
+          const float wm = warp_max(s[h]);
+          if (lane == 0) red[hh][wq][h] = wm;
+        }
+        {
+          const float wv = warp_max(vs);
+          if (lane == 0) red[hh][wq][kWideHS] = wv;
+        }
+        named_bar_sync(bar_id, 128);
+        float resc[kWideHS];
+#pragma unroll
+        for (int h = 0; h < kWideHS; ++h) {
+          const float tmax = fmaxf(fmaxf(red[hh][0][h], red[hh][1][h]), fmaxf(red[hh][2][h], red[hh][3][h]));
+          resc[h] = 1.0f;
+          if (hs0 + h < nh && tmax + nm[h] > 0.0f) {
+            const float m_new = tmax + kHoldMarginLog2;
+            resc[h] = (nm[h] == 1e30f) ? 0.0f : ex2_approx(-nm[h] - m_new);
+            nm[h] = -m_new;
+          }
+        }
+        const float vmax = fmaxf(fmaxf(red[hh][0][kWideHS], red[hh][1][kWideHS]), fmaxf(red[hh][2][kWideHS], red[hh][3][kWideHS]));
+        const float alpha_old = alpha_p;
+        if (vmax > a_ref) {
+          a_ref = vmax * kHoldScaleGrowth;
+          alpha_p = a_ref * (1.0f / 127.0f);
+          inv_a = __frcp_rn(alpha_p);
+          inv_b = 254.0f * inv_a;
+        }
+        if (t > 0) {
+          // everything accumulated so far was scaled by the old references: PV(t-1) and all before it are complete
+          ok = wait_bounded(&o_full, (t - 1) & 1, abort, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          drain(resc, alpha_old);
+#pragma unroll
+          for (int h = 0; h < kWideHS; ++h) l_part[h] *= resc[h];
+        }
+        write_p(t, s, vs, pl);
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_redo);
+        ++n_slow;
+        named_bar_sync(bar_id, 128);          // `red` may be rewritten
+      }
+#pragma unroll
+      for (int h = 0; h < kWideHS; ++h) l_part[h] += pl[h];
+      if (threadIdx.x == 64 && t < 6) attn_mark(p, 6 + 4 * t);
+    }
+    if (ok) {
+      // what the accumulators still hold
+      ok = wait_bounded(&o_last, 0, abort, p.status);
+      if (ok) {
+        tc_fence_after();
+        float one[kWideHS];
+#pragma unroll
+        for (int h = 0; h < kWideHS; ++h) one[h] = 1.0f;
+        drain(one, alpha_p);
+      }
+    }
+    if (threadIdx.x == 64) attn_mark(p, 28);
+    // partial results of this split: reference maximum, sum of P and unnormalised output per head
+    if (ok) {
+#pragma unroll
+      for (int h = 0; h < kWideHS; ++h) {
+        float l = l_part[h];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+        if (lane == 0) red[hh][wq][h] = l;
+      }
+      named_bar_sync(bar_id, 128);
+#pragma unroll
+      for (int h = 0; h < kWideHS; ++h) {
+        if (hs0 + h < nh) {
+          float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + hs0 + h) * p.n_splits + split) * (p.Dv + 2);
+          if (tl == 0) {
+            // the reference goes out in natural-log units (it was kept in the log2 domain); -inf: no visible token
+            dst[0] = (nm[h] == 1e30f) ? -INFINITY : -nm[h] * 0.6931471805599453f;
+            dst[1] = red[hh][0][h] + red[hh][1][h] + red[hh][2][h] + red[hh][3][h];
+          }
+#pragma unroll
+          for (int j = 0; j < kDVT; ++j)
+            if (j < p.DVT && j * kChunk + tl < p.Dv) dst[2 + j * kChunk + tl] = o_run[j][h];
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0) attn_mark(p, 29);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, p.tmem_cols);
+  }
+}
+
 static long long* g_attn_trace = nullptr;
+static int8_t* g_attn_q_dbg = nullptr;
+static float* g_attn_qs_dbg = nullptr;
+static int32_t* g_attn_s_dbg = nullptr;
 
 // c8: merge the splits of one (sequence, query head) and normalise:  O = sum_s e^{m_s - m} O_s / sum_s e^{m_s - m} l_s
 // (a separate small kernel: letting the last-arriving split do it inside the attention kernel measured slower)
@@ -685,7 +1164,7 @@ attn_combine_kernel(const float* __restrict__ partial, int n_splits, int Dv, __n
 }
 
 struct AttnPlan {
-  int HG, Rp, groups, DC, DVT, n_splits, stages, tmem_cols, v_alias, chunk;
+  int HG, Rp, groups, DC, DVT, n_splits, stages, tmem_cols, v_alias, chunk, kv_chunks;
   size_t smem_bytes, ws_bytes, ws_partial_bytes, ws_qimg_bytes, ws_qscale_bytes;
 };
 
@@ -706,7 +1185,10 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   if (pl->DVT == 3) pl->DVT = 4;
   if (v_alias && Dv > D) return false;
   pl->v_alias = v_alias ? 1 : 0;
-  const int kv_stage = (pl->DC + (v_alias ? 0 : pl->DVT)) * kChunkBytes;
+  // V aliased to the K rows: PV reads DVT chunks of the stage, which can be one more than the DC chunks the loads fill
+  // (Dv of 257..384 bytes is computed as four 128-wide tiles) - the stage is sized for the larger of the two
+  pl->kv_chunks = v_alias ? (pl->DC > pl->DVT ? pl->DC : pl->DVT) : pl->DC + pl->DVT;
+  const int kv_stage = pl->kv_chunks * kChunkBytes;
   const size_t fixed = static_cast<size_t>(pl->DC) * pl->Rp * kChunk + 2 * pl->Rp * kChunk + 1024;   // Q stack, two P buffers
   pl->stages = (2 * static_cast<size_t>(kv_stage) + fixed <= 227 * 1024 - 2048) ? 2 : 1;
   // Splits of equal size (a fixed number of tiles) keep the CTAs' work uniform whatever the mix of sequence lengths;
@@ -741,6 +1223,23 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
 extern "C" {
 
 void msd_debug_set_attn_trace(void* device_buffer) { msd::g_attn_trace = static_cast<long long*>(device_buffer); }
+
+void msd_debug_set_attn_dump(int8_t* q_dbg, float* q_scale_dbg, int32_t* s_dbg) {
+  msd::g_attn_q_dbg = q_dbg;
+  msd::g_attn_qs_dbg = q_scale_dbg;
+  msd::g_attn_s_dbg = s_dbg;
+}
+
+msd_status_t msd_attn_decode_softmax_rule(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen,
+                                          float* m_margin, float* sv_growth) {
+  msd::AttnPlan pl;
+  if (!m_margin || !sv_growth) return MSD_ERR_NULL_POINTER;
+  if (!msd::plan_attn(B, Hq, Hkv, D, Dv, max_seqlen, false, &pl)) return MSD_ERR_BAD_SHAPE;
+  const bool held = pl.HG > 16;
+  *m_margin = held ? msd::kHoldMarginLog2 * 0.6931471805599453f : 0.0f;
+  *sv_growth = held ? msd::kHoldScaleGrowth : 0.0f;
+  return MSD_OK;
+}
 
 size_t msd_attn_decode_int8kv_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen) {
   msd::AttnPlan pl;
@@ -820,29 +1319,28 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
   p.Sq = q_len; p.Gr = Hq_real / Hkv;
   p.HG = pl.HG; p.Rp = pl.Rp; p.groups = pl.groups; p.DC = pl.DC; p.DVT = pl.DVT;
   p.chunk = pl.chunk;
-  p.n_splits = pl.n_splits; p.stages = pl.stages; p.v_alias = pl.v_alias; p.tmem_cols = pl.tmem_cols;
+  p.n_splits = pl.n_splits; p.stages = pl.stages; p.v_alias = pl.v_alias; p.kv_chunks = pl.kv_chunks; p.tmem_cols = pl.tmem_cols;
+  p.q_dbg = g_attn_q_dbg; p.qs_dbg = g_attn_qs_dbg; p.s_dbg = g_attn_s_dbg; p.dbg_T = total_tokens;
   p.scale = softmax_scale;
   p.status = status;
   p.trace = g_attn_trace;
 
   void (*kernel)(CUtensorMap, CUtensorMap, AttnParams) = nullptr;
   const int G = Hq / Hkv;
-#define MSD_ATTN_PICK_P(HG_, NH_, WG_, P_) \
-  kernel = (pl.DVT == 1) ? attn_decode_kernel<HG_, NH_, 1, WG_, P_> : (pl.DVT == 2) ? attn_decode_kernel<HG_, NH_, 2, WG_, P_> \
-                                                                                      : attn_decode_kernel<HG_, NH_, 4, WG_, P_>
-#define MSD_ATTN_PICK(HG_, NH_, WG_) \
-  do { if (paged) { MSD_ATTN_PICK_P(HG_, NH_, WG_, true); } else { MSD_ATTN_PICK_P(HG_, NH_, WG_, false); } } while (0)
+#define MSD_ATTN_PICK_P(HG_, NH_, P_) \
+  kernel = (pl.DVT == 1) ? attn_decode_kernel<HG_, NH_, 1, P_> : (pl.DVT == 2) ? attn_decode_kernel<HG_, NH_, 2, P_> \
+                                                                               : attn_decode_kernel<HG_, NH_, 4, P_>
+#define MSD_ATTN_PICK(HG_, NH_) \
+  do { if (paged) { MSD_ATTN_PICK_P(HG_, NH_, true); } else { MSD_ATTN_PICK_P(HG_, NH_, false); } } while (0)
   int block_threads = kAttnThreads;
   if (pl.HG == 8) {
-    if (G <= 4) { MSD_ATTN_PICK(8, 4, 1); } else { MSD_ATTN_PICK(8, 8, 1); }
+    if (G <= 4) { MSD_ATTN_PICK(8, 4); } else { MSD_ATTN_PICK(8, 8); }
   } else if (pl.HG == 16) {
-    MSD_ATTN_PICK(16, 16, 1);
-  } else if (attn_env_int("MSD_ATTN_WIDE", 4) == 2) {
-    MSD_ATTN_PICK(16, 16, 2);          // 32 heads per CTA as two groups of four warps, 16 heads per thread
-    block_threads = 64 + 128 * 2;
+    MSD_ATTN_PICK(16, 16);
   } else {
-    MSD_ATTN_PICK(8, 8, 4);            // 32 heads per CTA as four groups of four warps, 8 heads per thread
-    block_threads = 64 + 128 * 4;
+    // wide head groups: 32 head slots per CTA, sixteen softmax warps, held references (attn_decode_wide_kernel)
+    kernel = paged ? attn_decode_wide_kernel<true> : attn_decode_wide_kernel<false>;
+    block_threads = kWideThreads;
   }
 #undef MSD_ATTN_PICK
 #undef MSD_ATTN_PICK_P

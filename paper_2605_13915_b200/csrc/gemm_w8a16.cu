@@ -16,6 +16,7 @@
 #include <cuda_bf16.h>
 
 #include <cstdlib>
+#include <mutex>
 #include <type_traits>
 
 #include "host_common.h"
@@ -1060,9 +1061,13 @@ __global__ void dequant_w8_to_bf16_kernel(const int8_t* __restrict__ w, const fl
   }
 }
 
+constexpr int64_t kMaxExactK = 131072;
+
 static msd_status_t check_w8_args(const void* x, const void* w, const void* ws, int64_t M, int64_t N, int64_t K,
                                   const void* y, int ytype, const void* workspace, int64_t max_m = 128) {
   if (M < 1 || M > max_m || N < 1 || K < 16 || K % 16 != 0 || N > (1 << 24) || K > (1 << 24)) return MSD_ERR_BAD_SHAPE;
+  // the two sums of Alg. 1 are exact in INT32 only while 127 * 128 * K < 2^31
+  if (K > kMaxExactK) return MSD_ERR_UNSUPPORTED;
   if (ytype != MSD_OUT_BF16 && ytype != MSD_OUT_FP32) return MSD_ERR_UNSUPPORTED;
   if (ytype == MSD_OUT_BF16 && N % 8 != 0) return MSD_ERR_BAD_SHAPE;
   if (!x || !w || !ws || !y || !workspace) return MSD_ERR_NULL_POINTER;
@@ -1227,9 +1232,6 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
 }
 
 // ---------------------------------------------------------------------------------------------------------------------
-// Entry point for callers that cannot allocate device memory (see msd.h).  The scratch the GEMM needs lives in this
-// file-scope device array, which every GPU that loads the library holds until the process exits.
-// ---------------------------------------------------------------------------------------------------------------------
 // Grouped W8A16 layer (MoE experts, Sec. 7.2): x rows sorted by expert, group g = rows [off_g, off_g + m_g) against
 // expert e_g's weight.  One decomposition launch over all rows, then stream-K launches of up to kMaxGroups non-empty
 // groups each; empty groups cost nothing (their weights are never read).
@@ -1266,6 +1268,7 @@ msd_status_t msd_grouped_gemm_w8a16(const void* x_bf16, const int8_t* w, const f
                                     size_t workspace_bytes, void* stream) {
   using namespace msd;
   if (E < 1 || N < 1 || K < 16 || K % 16 != 0 || N > (1 << 24) || K > (1 << 24)) return MSD_ERR_BAD_SHAPE;
+  if (K > kMaxExactK) return MSD_ERR_UNSUPPORTED;       // INT32 sums would no longer be exact
   if (!group_sizes_host) return MSD_ERR_NULL_POINTER;
   if (ytype != MSD_OUT_BF16 && ytype != MSD_OUT_FP32) return MSD_ERR_UNSUPPORTED;
   if (ytype == MSD_OUT_BF16 && N % 8 != 0) return MSD_ERR_BAD_SHAPE;
@@ -1355,6 +1358,10 @@ msd_status_t msd_grouped_gemm_w8a16(const void* x_bf16, const int8_t* w, const f
 // ---------------------------------------------------------------------------------------------------------------------
 }  // extern "C"
 
+// ---------------------------------------------------------------------------------------------------------------------
+// Entry point for callers that cannot allocate device memory (see msd.h).  The scratch the GEMM needs lives in this
+// file-scope device array, which every GPU that loads the library holds until the process exits.
+// ---------------------------------------------------------------------------------------------------------------------
 namespace msd {
 constexpr int64_t kStaticMaxM = 16;
 constexpr int64_t kStaticMaxN = 16384;
@@ -1365,9 +1372,11 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 // Device address of the scratch array on the current device (resolved once per device); NULL on failure.
 // In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel could use.
 static unsigned char* static_scratch_ptr() {
+  static std::mutex mu;
   static unsigned char* cache[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
   if (!cache[dev]) {
     unsigned char* ptr = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess || !ptr) return nullptr;
@@ -1390,9 +1399,14 @@ msd_status_t msd_gemm_w8a16_noalloc(const void* x_bf16, const int8_t* w, const f
   const size_t avail = kStaticScratchBytes + 1024 - static_cast<size_t>(ws - raw);
   const GemmW8Plan pl = plan_w8(M, N, K);
   if (pl.bytes > avail) return MSD_ERR_UNSUPPORTED;
-  // The array keeps whatever the previous call left.  The split-K counters and meeting place must start at zero; a
-  // completed call leaves them so, but a call that gave up on a wait may not have, so they are cleared every time.
-  if (cudaMemsetAsync(ws + pl.off_counters, 0, pl.bytes - pl.off_counters, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+  // every host-detectable problem is reported before anything is enqueued (the scratch stands in for the workspace)
+  const msd_status_t st = check_w8_args(x_bf16, w, w_scale, M, N, K, y, ytype, ws);
+  if (st != MSD_OK) return st;
+  // The array keeps whatever the previous call left.  The arrival counters (and, for the stream-K split only, the
+  // meeting place of the partial sums) must start at zero; a completed call leaves them so, but a call that gave up on
+  // a wait may not have, so they are cleared every time.  The other work splits never touch the meeting place.
+  const size_t clear_bytes = (pl.mode == 0 ? pl.bytes : pl.off_slots) - pl.off_counters;
+  if (cudaMemsetAsync(ws + pl.off_counters, 0, clear_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return MSD_ERR_CUDA;
   return msd_gemm_w8a16(x_bf16, w, w_scale, M, N, K, y, ytype, nullptr, ws, avail, stream);
 }

@@ -24,3 +24,26 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _guard_bands(request):
+    """GPU tests: every tensor the binding allocates for the library (outputs, accumulator dumps, workspaces) gets
+    canary bands on both sides, checked when the test ends."""
+    if "gpu" not in request.keywords:
+        yield
+        return
+    import torch
+    if not torch.cuda.is_available():
+        yield
+        return
+    from helpers import GuardedAllocator
+    from paper_2605_13915_b200 import binding
+    g = GuardedAllocator()
+    old = (binding._empty, binding._workspace)
+    binding._empty, binding._workspace = g.empty, g.workspace
+    try:
+        yield
+        g.check()
+    finally:
+        binding._empty, binding._workspace = old

@@ -50,3 +50,12 @@ def test_argument_checks_precede_any_launch():
     assert lib.msd_gemm_w8a16(p, p, p, 4, 128, 128, p, 0, None, C.c_void_p(4096 + 512), 1 << 30, None) == 3
     assert lib.msd_gemm_w8a16(p, p, p, 4, 128, 128, p, 0, None, p, 16, None) == 5            # workspace too small
     assert lib.msd_gemm_w8a16_workspace_bytes(16, 4096, 4096) >= 2 * 16 * 4096
+    # E8M0 weight scales are read as 32-bit words: a byte-aligned pointer is refused on the host
+    odd = C.c_void_p(4096 + 1)
+    assert lib.msd_gemm_w4a16(p, p, odd, 128, 128, 128, p, 0, p, 1 << 30, None) == 3
+    assert lib.msd_gemm_w4a16_e1m2(p, p, odd, 128, 128, 128, p, 0, p, 1 << 30, None) == 3
+    # beyond K = 131072 the INT32 sums of Alg. 1 could overflow
+    assert lib.msd_gemm_w8a16(p, p, p, 4, 128, 131072 + 16, p, 0, None, p, 1 << 40, None) == 4
+    # the allocation-free entry point reports bad arguments before it clears its scratch
+    assert lib.msd_gemm_w8a16_noalloc(null, p, p, 4, 128, 128, p, 0, None) in (1, 6)
+    assert lib.msd_gemm_w8a16_noalloc(p, p, p, 17, 128, 128, p, 0, None) == 4

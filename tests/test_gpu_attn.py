@@ -35,10 +35,20 @@ def _run_gpu(c, want_lse=True):
 def _oracle_tiled(c, B_sched=None, max_seqlen=None):
     B, Hq, D = c.q.shape
     Hkv = c.k.shape[1]
-    tile, ns, st = binding.attn_decode_schedule(B_sched or B, Hq, Hkv, D, c.dv, max(max_seqlen or c.max_seqlen, 1))
+    shape = (B_sched or B, Hq, Hkv, D, c.dv, max(max_seqlen or c.max_seqlen, 1))
+    tile, ns, st = binding.attn_decode_schedule(*shape)
     ss = _split_starts(np.diff(c.cu_seqlens), ns, st)
     return oracle.attn_decode_int8kv(c.q, c.k, c.v, c.k_scale, c.v_scale, c.cu_seqlens, c.softmax_scale, dv=c.dv,
-                                     mode="tiled", tile=tile, split_starts=ss, want_lse=True)
+                                     split_starts=ss, tile=tile, want_lse=True, **_softmax_mode(*shape))
+
+
+def _softmax_mode(*shape):
+    """Which tiled mode of the oracle mirrors the kernel for this shape: the plain online softmax, or the one whose
+    references are held between tiles (wide head groups), with the margins the library reports."""
+    margin, growth = binding.attn_decode_softmax_rule(*shape)
+    if growth == 0.0:
+        return dict(mode="tiled")
+    return dict(mode="held", m_margin=margin, sv_growth=growth)
 
 
 def _assert_close(got, ref):
@@ -214,7 +224,7 @@ def _truncate(c, drop):
     return keep, cu
 
 
-@pytest.mark.parametrize("Sq,Hq,Hkv", [(4, 8, 2), (2, 16, 2), (3, 8, 8)])
+@pytest.mark.parametrize("Sq,Hq,Hkv", [(4, 8, 2), (2, 16, 2), (3, 8, 8), (3, 16, 1)])
 def test_speculative_decode_rows_are_causal_single_query_problems(Sq, Hq, Hkv):
     """Sq query tokens per sequence: query token s must equal the single-query problem on the cache without the last
     Sq - 1 - s tokens (the oracle, tiled with the kernel's tile and split boundaries)."""
@@ -232,7 +242,99 @@ def test_speculative_decode_rows_are_causal_single_query_problems(Sq, Hq, Hkv):
         keep, cu = _truncate(base, Sq - 1 - s)
         ss = _split_starts(np.diff(cu), ns, st)
         ref, lse_ref = oracle.attn_decode_int8kv(np.ascontiguousarray(q[:, s]), base.k[keep], base.v[keep], base.k_scale[keep],
-                                                 base.v_scale[keep], cu, base.softmax_scale, dv=128, mode="tiled", tile=tile,
-                                                 split_starts=ss, want_lse=True)
+                                                 base.v_scale[keep], cu, base.softmax_scale, dv=128, tile=tile,
+                                                 split_starts=ss, want_lse=True,
+                                                 **_softmax_mode(B, Hq * Sq, Hkv, 128, 128, base.max_seqlen))
         _assert_close(got[:, s], ref)
         assert np.allclose(lse.cpu().numpy()[:, s], lse_ref, rtol=0, atol=2e-3)
+
+
+# ---- Alg. 3 lines 1-4 bit for bit: query components, their scales and both INT32 score planes -------------------------
+def _dump_buffers(rows, rows_per_seq, D, T):
+    q_dbg = torch.full((2, rows, D), 99, dtype=torch.int8, device="cuda")
+    qs_dbg = torch.full((2, rows), -1.0, dtype=torch.float32, device="cuda")
+    s_dbg = torch.full((2, rows_per_seq, max(T, 1)), -(2 ** 31), dtype=torch.int32, device="cuda")
+    return q_dbg, qs_dbg, s_dbg
+
+
+def _check_q_dump(q_bits_rows, q_dbg, qs_dbg, live=None):
+    """q_bits_rows [R, D]: every query row in the order the entry point takes them; live: rows whose sequence is not
+    empty (an empty sequence has no attention to compute and its rows are not decomposed)."""
+    o1, o2, oa, ob = oracle.decompose_int8(q_bits_rows)
+    live = slice(None) if live is None else live
+    assert np.array_equal(q_dbg[0].cpu().numpy()[live], o1[live]) and np.array_equal(q_dbg[1].cpu().numpy()[live], o2[live])
+    assert np.array_equal(qs_dbg[0].cpu().numpy()[live], oa[live]) and np.array_equal(qs_dbg[1].cpu().numpy()[live], ob[live])
+
+
+def _run_with_dump(fn, rows, rows_per_seq, D, T):
+    q_dbg, qs_dbg, s_dbg = _dump_buffers(rows, rows_per_seq, D, T)
+    binding.debug_set_attn_dump(q_dbg, qs_dbg, s_dbg)
+    try:
+        fn()
+        torch.cuda.synchronize()
+        binding.last_device_status()
+    finally:
+        binding.debug_set_attn_dump()
+    return q_dbg, qs_dbg, s_dbg.cpu().numpy()
+
+
+@pytest.mark.parametrize("kind", ["gqa_narrow", "gqa_16", "mla"])
+def test_query_components_and_scores_bit_exact(kind):
+    """North-star requirement: decomposed components, scales and INT32 accumulators bit-exact.  The kernels dump what
+    they computed (msd_debug_set_attn_dump); the oracle returns the same planes (Alg. 3 lines 1-4)."""
+    if kind == "gqa_narrow":
+        c = inputs.gqa_case(3, 8, 2, 128, [700, 64, 1500], seed=41)          # rows decomposed inside the attention CTAs
+    elif kind == "gqa_16":
+        c = inputs.gqa_case(2, 32, 2, 128, [513, 2222], seed=42)            # 16 rows per KV head
+    else:
+        c = inputs.mla_case(2, 64, 576, 512, [300, 1000], seed=43)          # 64 rows: decomposed by the query-stack kernel
+    B, Hq, D = c.q.shape
+    T = c.k.shape[0]
+    q_dbg, qs_dbg, s_dbg = _run_with_dump(lambda: _run_gpu(c, want_lse=False), B * Hq, Hq, D, T)
+    _check_q_dump(c.q.reshape(B * Hq, D), q_dbg, qs_dbg)
+    _, s_ref = oracle.attn_decode_int8kv(c.q, c.k, c.v, c.k_scale, c.v_scale, c.cu_seqlens, c.softmax_scale, dv=c.dv, want_s=True)
+    # token t belongs to exactly one sequence, so the plane [row of that sequence, t] is defined for every t
+    assert np.array_equal(s_dbg, s_ref)
+
+
+def test_scores_bit_exact_paged_and_speculative():
+    # paged: the dump is indexed by the physical cache row
+    seqlens = [130, 700, 0, 257]
+    c = inputs.gqa_case(B=len(seqlens), Hq=16, Hkv=4, D=128, seqlens=seqlens, seed=44)
+    page = 32
+    k, v, ks, vs, table, sl = inputs.paginate(c, page, seed=7)
+    B, Hq, D = c.q.shape
+    q_dbg, qs_dbg, s_dbg = _run_with_dump(
+        lambda: binding.attn_decode_int8kv_paged(bf16_dev(c.q), dev(k), dev(v), dev(ks), dev(vs), dev(table), dev(sl), page,
+                                                 max(c.max_seqlen, 1), c.softmax_scale), B * Hq, Hq, D, k.shape[0])
+    _check_q_dump(c.q.reshape(B * Hq, D), q_dbg, qs_dbg, live=np.repeat(np.asarray(seqlens) > 0, Hq))
+    _, s_ref = oracle.attn_decode_int8kv(c.q, c.k, c.v, c.k_scale, c.v_scale, c.cu_seqlens, c.softmax_scale, dv=c.dv, want_s=True)
+    for b in range(B):
+        for u in range(seqlens[b]):
+            row = table[b, u // page] * page + u % page
+            assert np.array_equal(s_dbg[:, :, row], s_ref[:, :, c.cu_seqlens[b] + u])
+    # speculative decode: rows are (query token, head); every row's sums against EVERY token of its sequence are dumped
+    Sq, Hq, Hkv = 3, 8, 2
+    seqlens = [Sq, 131, 700]
+    base = inputs.gqa_case(B=len(seqlens), Hq=Hq * Sq, Hkv=Hkv, D=128, seqlens=seqlens, seed=45)
+    B = len(seqlens)
+    q = base.q.reshape(B, Sq, Hq, 128)
+    T = base.k.shape[0]
+    q_dbg, qs_dbg, s_dbg = _run_with_dump(
+        lambda: binding.attn_decode_int8kv_spec(bf16_dev(q), dev(base.k), dev(base.v), dev(base.k_scale), dev(base.v_scale),
+                                                dev(base.cu_seqlens), base.max_seqlen, base.softmax_scale),
+        B * Sq * Hq, Sq * Hq, 128, T)
+    _check_q_dump(q.reshape(B * Sq * Hq, 128), q_dbg, qs_dbg)
+    for s in range(Sq):
+        _, s_ref = oracle.attn_decode_int8kv(np.ascontiguousarray(q[:, s]), base.k, base.v, base.k_scale, base.v_scale,
+                                             base.cu_seqlens, base.softmax_scale, dv=128, want_s=True)
+        assert np.array_equal(s_dbg[:, s * Hq:(s + 1) * Hq], s_ref)
+
+
+def test_latent_head_of_384_with_aliased_values():
+    """D = Dv = 384 with V aliased to the K rows: three 128-byte chunks are loaded per tile while PV is computed as four
+    128-wide tiles, so the KV stage must be sized for four."""
+    c = inputs.mla_case(2, 8, 384, 384, [300, 129], seed=46)
+    _check(c)
+    c = inputs.mla_case(1, 32, 320, 320, [700], seed=47)
+    _check(c)

@@ -1,4 +1,4 @@
-"""The allocation-free W8A16 entry point against the regular one.
+"""The allocation-free W8A16 entry point against the regular one and against the CPU oracle.
 
 Some callers of this library may not allocate device memory at all (a plug-in inside a serving loop that forbids
 allocation on its hot path, a host whose memory pool belongs to another runtime); msd_gemm_w8a16_noalloc keeps its
@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2605_13915_b200 import binding, inputs
 from helpers import bf16_dev, dev
 
@@ -41,6 +42,10 @@ def test_noalloc_matches_regular_entry_point_twice_in_a_row(M, N, K):
         assert np.all(np.isfinite(g))
         assert np.all(np.abs(g - r) <= 1e-3 * np.linalg.norm(r, axis=1, keepdims=True))
         assert np.array_equal(g, r)
+        # and the oracle (Alg. 1 in FP64), on the smaller shapes it finishes in a moment
+        if N * K <= 4096 * 4096:
+            want = oracle.gemm_w8a16(c.x, c.w, c.w_scale, "f64")
+            assert np.all(np.abs(g - want) <= 1e-3 * np.linalg.norm(want, axis=1, keepdims=True))
     got, ref = _both(c1, torch.bfloat16)
     assert torch.equal(got, ref)
 
