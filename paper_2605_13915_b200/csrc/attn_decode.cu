@@ -983,7 +983,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       }
       return xm;
     };
-    // Alg. 3 line 12 for everything accumulated since the last drain: O <- O * resc + alpha_P (O1 + O2 / 254)
+    // Alg. 3 line 12 for everything accumulated since the last drain: O <- (O + alpha_P (O1 + O2 / 254)) * resc
     auto drain = [&](const float (&resc)[kWideHS], float alpha_old) {
 #pragma unroll
       for (int j = 0; j < kDVT; ++j) {
@@ -996,7 +996,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
 #pragma unroll
           for (int h = 0; h < kWideHS; ++h) {
             const float acc = __fmaf_rn(static_cast<float>(static_cast<int32_t>(v2[h])), kInv254, static_cast<float>(static_cast<int32_t>(v1[h])));
-            o_run[j][h] = __fmaf_rn(o_run[j][h], resc[h], alpha_old * acc);
+            o_run[j][h] = __fmaf_rn(alpha_old, acc, o_run[j][h]) * resc[h];     // the drained sums belong to the OLD reference
           }
         }
       }
