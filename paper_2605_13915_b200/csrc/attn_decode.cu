@@ -632,24 +632,24 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 // the P buffer, the accumulators are drained into the FP32 running output with the old scales, the references move,
 // and P of that tile is written again before the MMA warp may use it.
 //
-// L2 prefetch: a KV stage is 80 KB for a 576-byte row, so only two fit in shared memory and a tile can be requested
-// only when the PV product two tiles back is done.  The producer therefore asks for the tiles further ahead with
-// cp.async.bulk.prefetch.tensor (no shared memory needed): HBM keeps streaming and the load that follows hits L2.
-constexpr float kHoldMarginLog2 = 2.0f;
+// (Asking for the tiles further ahead with cp.async.bulk.prefetch.tensor was measured and dropped: the two KV stages
+// that fit shared memory for a 576-byte row bound the pipeline, not the latency of L2 misses.)
+constexpr float kHoldMarginLog2 = 3.0f;
 constexpr float kHoldScaleGrowth = 1.25f;
-constexpr int kWideHS = 8;                          // head slots per softmax thread
-constexpr int kWideWG = 4;                          // groups of four softmax warps
-constexpr int kWideSlots = kWideHS * kWideWG;       // 32 head slots per CTA, Rp = 64 stacked rows
-constexpr int kWideThreads = 64 + 128 * kWideWG;
-constexpr int kWidePrefetchTiles = 4;
-
-__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* m, int c0, int c1, int c2) {
-  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
-               ::"l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+constexpr int kWideSlots = 32;                      // head slots per CTA, Rp = 64 stacked rows
+template <int W> __device__ __forceinline__ void tmem_stw(uint32_t taddr, const uint32_t (&v)[W]) {
+  static_assert(W == 8 || W == 16, "8 or 16 columns per store");
+  if constexpr (W == 8) tmem_st8(taddr, v);
+  else tmem_st16(taddr, v);
 }
 
-template <bool kPaged>
-__global__ void __launch_bounds__(kWideThreads, 1)
+
+// kWideHS: head slots per softmax thread (8 or 16); the 32 slots of the CTA are shared out over 32 / kWideHS groups of
+// four softmax warps.  kFixDC / kFixDVT: the chunk counts of D and Dv when known at compile time (0: taken from the
+// plan) - the MMA thread shares its scheduler with four busy softmax warps, so every instruction it spends per MMA on
+// loop control and address arithmetic delays the tensor pipe; with fixed counts its loops unroll to an add per operand.
+template <int kWideHS, bool kPaged, int kFixDC, int kFixDVT>
+__global__ void __launch_bounds__(64 + 128 * (kWideSlots / kWideHS), 1)
 attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], v_full[4], v_empty[4], s_full[2], p_full[2], q_ready, o_full, o_last, p_redo;
@@ -657,7 +657,8 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
   __shared__ int abort_flag;
   __shared__ int flush_stamp[2];                    // tile number + 1 of the last tile whose references had to move, per P buffer
   __shared__ float s_aq[kWideSlots];
-  __shared__ float red[kWideWG][4][kWideHS + 1];    // per-warp tile maxima (slow path only)
+  __shared__ float red[kWideSlots / kWideHS][4][kWideHS + 1];    // per-warp tile maxima (slow path only)
+  constexpr int kWideWG = kWideSlots / kWideHS;
   constexpr int kNSW = 4 * kWideWG;
   constexpr int kDVT = 4;
 
@@ -726,14 +727,6 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
     if (lane == 0) {
       const int k_bytes = p.DC * kChunkBytes, v_bytes = p.DVT * kChunkBytes;
       int kq = 0, vq = p.v_alias ? ntiles : 0;
-      if constexpr (!kPaged) {
-        // tiles that do not fit shared memory yet: ask for them in L2
-        for (int t = p.stages; t < min(ntiles, p.stages + kWidePrefetchTiles); ++t) {
-          for (int c = 0; c < p.DC; ++c) tma_prefetch_3d(&tmap_k, c * kChunk, hk, seq0 + t_begin + t * kTok);
-          if (!p.v_alias)
-            for (int j = 0; j < p.DVT; ++j) tma_prefetch_3d(&tmap_v, j * kChunk, hk, seq0 + t_begin + t * kTok);
-        }
-      }
       long long t_idle = clock64();
       while (kq < ntiles || vq < ntiles) {
         bool progressed = false;
@@ -741,12 +734,10 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
           const int st = kq % p.stages;
           uint8_t* dst = smem + st * kv_stage_bytes;
           const int u0 = t_begin + kq * kTok;
+          if (kq >= 2 && kq < 5) attn_mark(p, 9 + 6 * (kq - 2));
           if constexpr (!kPaged) {
             mbar_arrive_expect_tx(&kv_full[st], k_bytes);
             for (int c = 0; c < p.DC; ++c) tma_load_3d(dst + c * kChunkBytes, &tmap_k, c * kChunk, hk, seq0 + u0, &kv_full[st]);
-            const int tp = kq + kWidePrefetchTiles;
-            if (kq >= p.stages && tp < ntiles)
-              for (int c = 0; c < p.DC; ++c) tma_prefetch_3d(&tmap_k, c * kChunk, hk, seq0 + t_begin + tp * kTok);
           } else {
             const int npg = min(kTok >> p.page_shift, (t_end - u0 + p.page - 1) >> p.page_shift);
             mbar_arrive_expect_tx(&kv_full[st], p.DC * kChunk * p.page * npg);
@@ -766,9 +757,6 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
           if constexpr (!kPaged) {
             mbar_arrive_expect_tx(&v_full[st], v_bytes);
             for (int j = 0; j < p.DVT; ++j) tma_load_3d(dst + j * kChunkBytes, &tmap_v, j * kChunk, hk, seq0 + u0, &v_full[st]);
-            const int tp = vq + kWidePrefetchTiles;
-            if (vq >= p.stages && tp < ntiles)
-              for (int j = 0; j < p.DVT; ++j) tma_prefetch_3d(&tmap_v, j * kChunk, hk, seq0 + t_begin + tp * kTok);
           } else {
             const int npg = min(kTok >> p.page_shift, (t_end - u0 + p.page - 1) >> p.page_shift);
             mbar_arrive_expect_tx(&v_full[st], p.DVT * kChunk * p.page * npg);
@@ -797,7 +785,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
       const uint32_t idesc_qk = idesc_dense(2, 1, 1, 0, 0, kTok, p.Rp);     // S8 x S8 -> S32, both K-major
-      const uint32_t idesc_pv = idesc_dense(2, 1, 1, 1, 0, kTok, p.Rp);     // A (V^T) MN-major
+      const uint32_t idesc_pv = idesc_dense(2, 1, 1, 1, 1, kTok, p.Rp);     // A (V^T) and B (P) MN-major
       bool ok = true;
       // the stacked Q operand of this (sequence, KV head, head group) comes ready-made from attn_qstack_kernel, the
       // kernel launched just before this one (the producer's KV loads, which do not depend on it, are already under way)
@@ -809,23 +797,39 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
           bulk_load(sm_q + c * chunk_bytes, p.q_img + (static_cast<size_t>(unit_q) * p.DC + c) * chunk_bytes, chunk_bytes, &q_ready);
       }
       ok = wait_bounded(&q_ready, 0, abort, p.status);
-      const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);         // K-major tiles: K, stacked Q, P
+      const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);         // K-major tiles: K, stacked Q
       const uint64_t dvt = smem_desc(0, 16384, 1024, kSwizzle128B);     // V^T read MN-major from the token-major tile
       const uint64_t q_enc = dk + (smem_u32(sm_q) >> 4);
-      const uint64_t p_enc = dk + (smem_u32(sm_p) >> 4);
+      // P lies token-major, [128 tokens][64 bytes = 2 x 32 head slots], 64-byte swizzle: an MN-major B operand whose
+      // groups of 8 tokens are 512 bytes apart (a softmax thread then stores its token's codes as whole words)
+      const uint64_t p_enc = smem_desc(0, 512, 512, kSwizzle64B) + (smem_u32(sm_p) >> 4);
       const uint32_t smem_enc = smem_u32(smem) >> 4;
       const uint32_t q_step = static_cast<uint32_t>(p.Rp * kChunk) >> 4, p_step = q_step;
+      const int nDC = kFixDC ? kFixDC : p.DC, nDVT = kFixDVT ? kFixDVT : p.DVT;
+      // 32-byte K steps of the last chunk of D that hold data (the stacked Q operand is zero past D)
+      const int last_steps = (p.D - (nDC - 1) * kChunk + 31) >> 5;
       auto issue_qk = [&](int t) {
         const int st = t % p.stages;
         tc_fence_after();
-        uint64_t ka = dk + smem_enc + static_cast<uint32_t>(st * (kv_stage_bytes >> 4));
-        uint64_t qa = q_enc;
+        const uint64_t ka = dk + smem_enc + static_cast<uint32_t>(st * (kv_stage_bytes >> 4));
         const uint32_t d = tmem_base + (t & 1) * p.Rp;
-        for (int c = 0; c < p.DC; ++c) {
+        if constexpr (kFixDC > 0) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) mma_i8(d, ka + 2 * k, qa + 2 * k, idesc_qk, (c > 0 || k > 0) ? 1u : 0u);
-          ka += kChunkBytes >> 4;
-          qa += q_step;
+          for (int c = 0; c < kFixDC; ++c)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              if (c + 1 < kFixDC || k < last_steps)
+                mma_i8(d, ka + (c * (kChunkBytes >> 4) + 2 * k), q_enc + (c * ((kWideSlots * 2 * kChunk) >> 4) + 2 * k), idesc_qk,
+                       (c > 0 || k > 0) ? 1u : 0u);
+        } else {
+          uint64_t kc = ka, qa = q_enc;
+          for (int c = 0; c < nDC; ++c) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              if (c + 1 < nDC || k < last_steps) mma_i8(d, kc + 2 * k, qa + 2 * k, idesc_qk, (c > 0 || k > 0) ? 1u : 0u);
+            kc += kChunkBytes >> 4;
+            qa += q_step;
+          }
         }
         tc_commit(&s_full[t & 1]);
         if (!p.v_alias) tc_commit(&kv_empty[st]);       // separate V: the K buffer is free once QK^T has read it
@@ -834,16 +838,26 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       auto issue_pv = [&](int t, bool fresh) {
         tc_fence_after();
         const int st = t % p.stages;
-        uint64_t va = dvt + smem_enc + static_cast<uint32_t>(st * (kv_stage_bytes >> 4)) +
-                      (p.v_alias ? 0u : static_cast<uint32_t>(p.DC * (kChunkBytes >> 4)));
+        const uint64_t va = dvt + smem_enc + static_cast<uint32_t>(st * (kv_stage_bytes >> 4)) +
+                            (p.v_alias ? 0u : static_cast<uint32_t>(p.DC * (kChunkBytes >> 4)));
         const uint64_t pa = p_enc + (t & 1) * p_step;
-        uint32_t d = tmem_o;
-        for (int j = 0; j < p.DVT; ++j) {
+        const uint32_t acc0 = fresh ? 0u : 1u;
+        if constexpr (kFixDVT > 0) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k)        // 32 tokens per MMA: four 8-token groups of 1024 bytes
-            mma_i8(d, va + k * (4096 >> 4), pa + 2 * k, idesc_pv, (k > 0 || !fresh) ? 1u : 0u);
-          va += kChunkBytes >> 4;
-          d += p.Rp;
+          for (int j = 0; j < kFixDVT; ++j)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)      // 32 tokens per MMA: four 8-token groups of 1024 bytes
+              mma_i8(tmem_o + j * (2 * kWideSlots), va + (j * (kChunkBytes >> 4) + k * (4096 >> 4)), pa + k * (2048 >> 4), idesc_pv,
+                     k > 0 ? 1u : acc0);
+        } else {
+          uint64_t vc = va;
+          uint32_t d = tmem_o;
+          for (int j = 0; j < nDVT; ++j) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) mma_i8(d, vc + k * (4096 >> 4), pa + k * (2048 >> 4), idesc_pv, k > 0 ? 1u : acc0);
+            vc += kChunkBytes >> 4;
+            d += p.Rp;
+          }
         }
         // o_full counts every PV product (a drain in mid-split waits for the one before its tile: at that point the
         // barrier is at most one phase behind, so a parity test is unambiguous); the last one has a barrier of its own
@@ -852,17 +866,15 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       };
       // QK^T(q) needs KV tile q in shared memory and the score buffer q&1 read (P of tile q-2 final);
       // PV(v) needs P of tile v final (written, and rewritten when the references had to move) and QK^T(v) issued.
+      // One thread issues both, so everything it has issued completes in order: when the scores of tile t are
+      // there, PV of tile t-2 is complete (the P buffer and the o_full phase the softmax warps rely on).
       int q = 0, v = 0, n_slow = 0;
       long long t_idle = clock64();
       while (ok && v < ntiles) {
         bool progressed = false;
-        if (q < ntiles && q < v + 2 && mbar_test_wait(&kv_full[q % p.stages], (q / p.stages) & 1)) {
-          issue_qk(q);
-          ++q;
-          progressed = true;
-        }
         if (v < q && mbar_test_wait(&p_full[v & 1], (v >> 1) & 1) &&
             (p.v_alias || mbar_test_wait(&v_full[v % p.stages], (v / p.stages) & 1))) {
+          // PV first when both are ready: its completion frees the KV stage the next load is waiting for
           bool fresh = false;
           if (stamp[v & 1] == v + 1) {
             // the softmax warps drain the accumulators and write P of this tile again
@@ -871,8 +883,17 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
             ++n_slow;
             fresh = true;
           }
+          if (v >= 2 && v < 5) attn_mark(p, 8 + 6 * (v - 2));
           issue_pv(v, fresh);
+          if (v >= 2 && v < 5) attn_mark(p, 20 + v);
           ++v;
+          progressed = true;
+        }
+        if (q < ntiles && q < v + 2 && mbar_test_wait(&kv_full[q % p.stages], (q / p.stages) & 1)) {
+          if (q >= 2 && q < 5) attn_mark(p, 7 + 6 * (q - 2));
+          issue_qk(q);
+          if (q >= 2 && q < 5) attn_mark(p, q == 4 ? 30 : 23 + q);
+          ++q;
           progressed = true;
         }
         if (progressed) {
@@ -909,16 +930,25 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
 
     // Per head slot: query scale, NEGATED reference maximum in the log2 domain (+1e30 while no score has been seen,
     // -1e30 for a slot without a head, so that "score + nm > 0" means "exceeds the reference"), partial sum of P over
-    // this thread's tokens, running output of this thread's dv lane.
-    float aq[kWideHS], nm[kWideHS], l_part[kWideHS], o_run[kDVT][kWideHS];
+    // this thread's tokens.  The FP32 running output of this thread's dv lane (4 x 8 values) lives in the tensor-memory
+    // columns behind the accumulators: it is touched only by the rare drains, and 32 registers fewer per thread let
+    // the compiler keep the eight heads' dependent chains of the per-tile code in flight side by side.
+    float aq[kWideHS], nm[kWideHS], l_part[kWideHS];
+    const uint32_t orun_row = tmem_o + kDVT * p.Rp + (static_cast<uint32_t>(quad * 32) << 16) + hs0;
 #pragma unroll
     for (int h = 0; h < kWideHS; ++h) {
       const bool present = hs0 + h < nh;
       aq[h] = present ? s_aq[hs0 + h] : 0.0f;
       nm[h] = present ? 1e30f : -1e30f;
       l_part[h] = 0.0f;
+    }
+    {
+      uint32_t z[kWideHS];
 #pragma unroll
-      for (int j = 0; j < kDVT; ++j) o_run[j][h] = 0.0f;
+      for (int h = 0; h < kWideHS; ++h) z[h] = 0u;
+#pragma unroll
+      for (int j = 0; j < kDVT; ++j) tmem_stw<kWideHS>(orun_row + j * kWideSlots, z);
+      tmem_st_wait();
     }
     float a_ref = 0.0f, alpha_p = 0.0f, inv_a = 0.0f, inv_b = 0.0f;
     const float kLog2e = 1.4426950408889634f;
@@ -946,8 +976,8 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       const bool valid = tok_rel < t_end;
       const uint32_t srow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + (t & 1) * p.Rp;
       uint32_t v1[kWideHS], v2[kWideHS];
-      tmem_ld8(srow + hs0, v1);
-      tmem_ld8(srow + kWideSlots + hs0, v2);
+      tmem_ldw<kWideHS>(srow + hs0, v1);
+      tmem_ldw<kWideHS>(srow + kWideSlots + hs0, v2);
       tmem_ld_wait();
       if (p.s_dbg && valid) {
         long long tok_row = seq0 + tok_rel;
@@ -965,7 +995,10 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
     // c4-c5: P = 2^(s - reference), value scale folded in, two-pass INT8 with the scale in force, into P buffer t&1.
     // Returns the largest s - reference of this thread (> 0: the reference must move).
     auto write_p = [&](int t, const float (&s)[kWideHS], float vs, float (&pl)[kWideHS]) -> float {
-      uint8_t* pbuf = sm_p + (t & 1) * p.Rp * kChunk;
+      // this token's row of the P buffer: 64 bytes, the 16-byte pieces XORed with (token / 2) % 4 (64-byte swizzle)
+      uint8_t* prow = sm_p + (t & 1) * p.Rp * kChunk + tl * 64;
+      const int sw = (tl >> 1) & 3;
+      uint32_t c1[kWideHS], c2[kWideHS];
       float xm = -INFINITY;
 #pragma unroll
       for (int h = 0; h < kWideHS; ++h) {
@@ -978,8 +1011,24 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
         const float u1 = __fmaf_rn(pt, inv_a, kMagic);
         const float r = __fmaf_rn(-alpha_p, u1 - kMagic, pt);
         const float u2 = __fmaf_rn(r, inv_b, kMagic);
-        pbuf[swz_off(hs0 + h, tl)] = static_cast<uint8_t>(__float_as_uint(u1));
-        pbuf[swz_off(kWideSlots + hs0 + h, tl)] = static_cast<uint8_t>(__float_as_uint(u2));
+        c1[h] = __float_as_uint(u1);
+        c2[h] = __float_as_uint(u2);
+      }
+      // the codes are the low bytes; kWideHS of them make one 8- or 16-byte store per component
+      uint32_t w1[kWideHS / 4], w2[kWideHS / 4];
+#pragma unroll
+      for (int g = 0; g < kWideHS / 4; ++g) {
+        w1[g] = __byte_perm(__byte_perm(c1[4 * g], c1[4 * g + 1], 0x0040), __byte_perm(c1[4 * g + 2], c1[4 * g + 3], 0x0040), 0x5410);
+        w2[g] = __byte_perm(__byte_perm(c2[4 * g], c2[4 * g + 1], 0x0040), __byte_perm(c2[4 * g + 2], c2[4 * g + 3], 0x0040), 0x5410);
+      }
+      uint8_t* d1 = prow + ((((hs0 >> 4) ^ sw) & 3) << 4) + (hs0 & 15);
+      uint8_t* d2 = prow + (((((kWideSlots + hs0) >> 4) ^ sw) & 3) << 4) + (hs0 & 15);
+      if constexpr (kWideHS == 8) {
+        *reinterpret_cast<uint2*>(d1) = make_uint2(w1[0], w1[1]);
+        *reinterpret_cast<uint2*>(d2) = make_uint2(w2[0], w2[1]);
+      } else {
+        *reinterpret_cast<uint4*>(d1) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+        *reinterpret_cast<uint4*>(d2) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
       }
       return xm;
     };
@@ -989,17 +1038,21 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       for (int j = 0; j < kDVT; ++j) {
         if (j < p.DVT) {
           const uint32_t orow = tmem_o + (static_cast<uint32_t>(quad * 32) << 16) + j * p.Rp;
-          uint32_t v1[kWideHS], v2[kWideHS];
-          tmem_ld8(orow + hs0, v1);
-          tmem_ld8(orow + kWideSlots + hs0, v2);
+          uint32_t v1[kWideHS], v2[kWideHS], o[kWideHS];
+          tmem_ldw<kWideHS>(orow + hs0, v1);
+          tmem_ldw<kWideHS>(orow + kWideSlots + hs0, v2);
+          tmem_ldw<kWideHS>(orun_row + j * kWideSlots, o);
           tmem_ld_wait();
 #pragma unroll
           for (int h = 0; h < kWideHS; ++h) {
             const float acc = __fmaf_rn(static_cast<float>(static_cast<int32_t>(v2[h])), kInv254, static_cast<float>(static_cast<int32_t>(v1[h])));
-            o_run[j][h] = __fmaf_rn(alpha_old, acc, o_run[j][h]) * resc[h];     // the drained sums belong to the OLD reference
+            // the drained sums belong to the OLD reference: add them, then rescale
+            o[h] = __float_as_uint(__fmaf_rn(alpha_old, acc, __uint_as_float(o[h])) * resc[h]);
           }
+          tmem_stw<kWideHS>(orun_row + j * kWideSlots, o);
         }
       }
+      tmem_st_wait();
     };
 
     bool ok = true;
@@ -1011,7 +1064,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       load_scales(t + 1, ks_pre, vs_pre);
       ok = wait_bounded(&s_full[t & 1], (t >> 1) & 1, abort, p.status);
       if (!ok) break;
-      if (threadIdx.x == 64 && t < 6) attn_mark(p, 4 + 4 * t);
+      if (threadIdx.x == 64 && t >= 2 && t < 5) attn_mark(p, 4 + 6 * (t - 2));
       tc_fence_after();
       float s[kWideHS], pl[kWideHS];
       load_scores(t, ks, s);
@@ -1022,10 +1075,11 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&p_full[t & 1]);
-      if (threadIdx.x == 64 && t < 6) attn_mark(p, 5 + 4 * t);
+      if (threadIdx.x == 64 && t >= 2 && t < 5) attn_mark(p, 5 + 6 * (t - 2));
       // every softmax warp has written its part (and its verdict): did any reference have to move?
       ok = wait_bounded(&p_full[t & 1], (t >> 1) & 1, abort, p.status);
       if (!ok) break;
+      if (threadIdx.x == 64 && t >= 2 && t < 5) attn_mark(p, 6 + 6 * (t - 2));
       if (stamp[t & 1] == t + 1) {
         // ---- the references move: tile maxima per head over the group's 128 tokens, largest value scale ----
 #pragma unroll
@@ -1076,7 +1130,6 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       }
 #pragma unroll
       for (int h = 0; h < kWideHS; ++h) l_part[h] += pl[h];
-      if (threadIdx.x == 64 && t < 6) attn_mark(p, 6 + 4 * t);
     }
     if (ok) {
       // what the accumulators still hold
@@ -1089,7 +1142,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
         drain(one, alpha_p);
       }
     }
-    if (threadIdx.x == 64) attn_mark(p, 28);
+    if (threadIdx.x == 64) { attn_mark(p, 28); if (p.trace && blockIdx.y * gridDim.x + blockIdx.x < 1024) p.trace[(blockIdx.y * gridDim.x + blockIdx.x) * 32 + 27] = n_slow; }
     // partial results of this split: reference maximum, sum of P and unnormalised output per head
     if (ok) {
 #pragma unroll
@@ -1109,9 +1162,19 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
             dst[0] = (nm[h] == 1e30f) ? -INFINITY : -nm[h] * 0.6931471805599453f;
             dst[1] = red[hh][0][h] + red[hh][1][h] + red[hh][2][h] + red[hh][3][h];
           }
+        }
+      }
 #pragma unroll
-          for (int j = 0; j < kDVT; ++j)
-            if (j < p.DVT && j * kChunk + tl < p.Dv) dst[2 + j * kChunk + tl] = o_run[j][h];
+      for (int j = 0; j < kDVT; ++j) {
+        if (j < p.DVT) {            // (warp-uniform: the tensor-memory load is a whole-warp instruction)
+          uint32_t o[kWideHS];
+          tmem_ldw<kWideHS>(orun_row + j * kWideSlots, o);
+          tmem_ld_wait();
+#pragma unroll
+          for (int h = 0; h < kWideHS; ++h)
+            if (hs0 + h < nh && j * kChunk + tl < p.Dv)
+              p.partial[((static_cast<long long>(b) * p.Hq + h0 + hs0 + h) * p.n_splits + split) * (p.Dv + 2) + 2 + j * kChunk + tl] =
+                  __uint_as_float(o[h]);
         }
       }
     }
@@ -1209,7 +1272,9 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   pl->chunk = chunk_tiles * kTok;
   pl->smem_bytes = static_cast<size_t>(pl->stages) * kv_stage + fixed;
   int cols = 32;
-  while (cols < 2 * pl->Rp + pl->DVT * pl->Rp) cols <<= 1;
+  // wide head groups keep the FP32 running output (4 x 32 columns) behind the two score buffers and the accumulators
+  const int cols_needed = pl->HG > 16 ? 2 * pl->Rp + 4 * pl->Rp + 4 * 32 : 2 * pl->Rp + pl->DVT * pl->Rp;
+  while (cols < cols_needed) cols <<= 1;
   pl->tmem_cols = cols;
   pl->ws_partial_bytes = round_up(static_cast<size_t>(B) * Hq * ns * (Dv + 2) * sizeof(float), 1024);
   pl->ws_qimg_bytes = round_up(static_cast<size_t>(units) * pl->DC * pl->Rp * kChunk, 1024);     // stacked Q operands
@@ -1339,8 +1404,10 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
     MSD_ATTN_PICK(16, 16);
   } else {
     // wide head groups: 32 head slots per CTA, sixteen softmax warps, held references (attn_decode_wide_kernel)
-    kernel = paged ? attn_decode_wide_kernel<true> : attn_decode_wide_kernel<false>;
-    block_threads = kWideThreads;
+    const bool mla = pl.DC == 5 && pl.DVT == 4;        // a 576-byte latent row with 512 value bytes
+    if (paged) kernel = mla ? attn_decode_wide_kernel<8, true, 5, 4> : attn_decode_wide_kernel<8, true, 0, 0>;
+    else kernel = mla ? attn_decode_wide_kernel<8, false, 5, 4> : attn_decode_wide_kernel<8, false, 0, 0>;
+    block_threads = 64 + 128 * 4;
   }
 #undef MSD_ATTN_PICK
 #undef MSD_ATTN_PICK_P

@@ -5,7 +5,9 @@
     python -m paper_2605_13915_b200.profile_cases attn_gqa B L [calls]        (32 query heads, 8 KV heads, d 128)
     python -m paper_2605_13915_b200.profile_cases attn_mla B L [calls]        (64 query heads, latent d 576 / 512)
 
-Inputs are random tensors of the right types drawn on the device; three weight / cache buffers are rotated.
+Inputs are random tensors of the right types drawn on the device (KV caches: N(0,1) values quantized per token, as in
+the benchmark); three weight / two cache buffers are rotated.  This is a driver for profilers, not part of the library's
+API.
 """
 import sys
 
@@ -40,10 +42,16 @@ def main(argv):
         T = B * L
         cu = (torch.arange(B + 1, dtype=torch.int32) * L).cuda()
         q = torch.randn(B, Hq, D, device="cuda").to(torch.bfloat16)
-        k = [torch.randint(-127, 128, (T, Hkv, D), dtype=torch.int8, device="cuda") for _ in range(2)]
-        v = None if what == "attn_mla" else [torch.randint(-127, 128, (T, Hkv, Dv), dtype=torch.int8, device="cuda") for _ in range(2)]
-        ks = torch.rand(T, Hkv, device="cuda") * 0.02 + 0.01
-        vs = None if what == "attn_mla" else torch.rand(T, Hkv, device="cuda") * 0.02 + 0.01
+        def cache(d):
+            x = torch.randn(T, Hkv, d, device="cuda")
+            s = x.abs().amax(dim=2) / 127.0
+            return torch.clamp(torch.round(x / s[:, :, None]), -127, 127).to(torch.int8), s.contiguous()
+        kk = [cache(D) for _ in range(2)]
+        k, ks = [a for a, _ in kk], kk[0][1]
+        v = vs = None
+        if what != "attn_mla":
+            vv = [cache(Dv) for _ in range(2)]
+            v, vs = [a for a, _ in vv], vv[0][1]
         ws = binding.workspace(binding.attn_decode_int8kv_workspace_bytes(B, Hq, Hkv, D, Dv, L))
         for i in range(calls):
             y = binding.attn_decode_int8kv(q, k[i % 2], None if v is None else v[i % 2], ks, vs, cu, L, D ** -0.5, dv=Dv, ws=ws)
