@@ -66,3 +66,16 @@ def test_single_rank_needs_no_process_group(monkeypatch):
     assert r.max_over_ranks(3.5) == 3.5
     thr, ms = r.job_throughput(70.0, 3.5)
     assert ms == 3.5 and abs(thr - 20000.0) < 1e-9
+
+
+def test_bench_gpus_flag_starts_the_ranks_itself():
+    """`bench.py --gpus 2` without a launcher re-executes itself under torch.distributed.run with two ranks.  The CPU
+    arm (--impl reference) exercises that path here: rank 0 prints the one JSON line, rank 1 exits 0 without work."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--steps", "1",
+                          "--warmup", "0"], env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True, timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(l) for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                       # one line for the whole job
+    assert lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2 and lines[0]["value"] > 0
