@@ -61,6 +61,16 @@ msd_status_t msd_last_device_status(void* stream);
  * and the next msd_last_device_status returns MSD_ERR_TIMEOUT; the context stays usable. */
 msd_status_t msd_debug_timeout_selftest(int64_t budget_cycles, void* stream);
 
+/* Testing and diagnostic switches.  Each is read from the environment variable of the same name once, when the first
+ * call needs one; msd_debug_set_option overrides it afterwards (value -1 = unset), msd_debug_reset_options returns to
+ * what the environment says.  Unknown names: MSD_ERR_UNSUPPORTED.  None of them changes results.
+ *   MSD_NO_PDL (1: no programmatic dependent launches), MSD_GEMM_MODE / MSD_GEMM_CTAS (work split and CTA count of the
+ *   W8A16 decode kernel: 0 stream-K, 1 row bands, 2 clusters), MSD_P8_PAIR / MSD_P8_KSPLIT (W8A16 many-row kernel: CTA
+ *   pairs, K split), MSD_W4_PAIR / MSD_W4_TILEN / MSD_W4_KSPLIT (W4A16 kernels), MSD_ATTN_SPLITS / MSD_ATTN_CHUNK_TILES
+ *   (context splits of the attention kernels; msd_attn_decode_schedule reports the schedule in force). */
+msd_status_t msd_debug_set_option(const char* name, int32_t value);
+void msd_debug_reset_options(void);
+
 /* Zero-fills a workspace (asynchronous memset on `stream`). */
 msd_status_t msd_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
@@ -115,7 +125,8 @@ msd_status_t msd_gemm_w8a16_ex(const void* x_bf16, const int8_t* w, const float*
                                void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * Grouped W8A16 MSD layer for mixture-of-experts blocks (Sec. 7.2: the decomposition works per activation row, so it
+ * Grouped W8A16 MSD layer for mixture-of-experts blocks (Discussion, "Extension to MoE and Sparse
+ * Architectures": the decomposition works per activation row, so it
  * carries over to grouped matrix multiplication unchanged).  The rows of x are sorted by expert; expert e owns the next
  * group_sizes[e] rows and multiplies them against its own weight:
  *   y[i,:] = msd_gemm_w8a16 row result of x[i,:] with w[e], w_scale[e]   for the rows i of group e.
@@ -194,7 +205,8 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
                             void* stream);
 
 /*
- * Grouped W4A16 MSD layer for mixture-of-experts blocks (Sec. 7.2; the decomposition works per 32-element block of an
+ * Grouped W4A16 MSD layer for mixture-of-experts blocks (Discussion, "Extension to MoE and Sparse
+ * Architectures"; the decomposition works per 32-element block of an
  * activation row, so it carries over unchanged).  The rows of x are sorted by expert; expert e owns the next
  * group_sizes[e] rows and multiplies them against its own MXFP4 weight:
  *   y[i,:] = msd_gemm_w4a16 row result of x[i,:] with w_fp4[e], w_e8m0[e]   for the rows i of group e.

@@ -56,6 +56,8 @@ _SIGS = {
     "msd_attn_decode_schedule": (C.c_int, [_i32] * 6 + [C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
     "msd_attn_decode_softmax_rule": (C.c_int, [_i32] * 6 + [C.POINTER(_f32), C.POINTER(_f32)]),
     "msd_debug_set_attn_dump": (None, [_vp, _vp, _vp]),
+    "msd_debug_set_option": (C.c_int, [C.c_char_p, _i32]),
+    "msd_debug_reset_options": (None, []),
     "msd_decompose_mxfp4_e1m2": (C.c_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp]),
     "msd_gemm_w4a16_e1m2_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_w4a16_e1m2": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
@@ -302,6 +304,16 @@ def attn_decode_softmax_rule(B, Hq, Hkv, D, Dv, max_seqlen):
     m, g = _f32(0), _f32(0)
     _check(lib().msd_attn_decode_softmax_rule(B, Hq, Hkv, D, Dv, max_seqlen, C.byref(m), C.byref(g)), "msd_attn_decode_softmax_rule")
     return m.value, g.value
+
+
+def debug_set_option(name, value):
+    """Sets one of the library's testing / diagnostic switches (the names of msd.h, e.g. "MSD_GEMM_MODE"); -1 unsets it."""
+    _check(lib().msd_debug_set_option(name.encode(), int(value)), "msd_debug_set_option")
+
+
+def debug_reset_options():
+    """Back to what the environment says (unset where it says nothing)."""
+    lib().msd_debug_reset_options()
 
 
 def debug_set_attn_dump(q_dbg=None, q_scale_dbg=None, s_dbg=None):

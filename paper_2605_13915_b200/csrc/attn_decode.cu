@@ -1231,11 +1231,6 @@ struct AttnPlan {
   size_t smem_bytes, ws_bytes, ws_partial_bytes, ws_qimg_bytes, ws_qscale_bytes;
 };
 
-static int attn_env_int(const char* name, int fallback) {
-  const char* e = getenv(name);
-  return (e && *e) ? atoi(e) : fallback;
-}
-
 static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, bool v_alias, AttnPlan* pl) {
   if (B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || D < 16 || D % 16 != 0 || Dv < 16 || Dv % 16 != 0) return false;
   const int G = Hq / Hkv;
@@ -1258,13 +1253,13 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   // the size is shrunk until there are enough splits to fill the machine a few times over.
   const int tiles = (max_seqlen + kTok - 1) / kTok;
   const long long units = static_cast<long long>(B) * Hkv * pl->groups;
-  int chunk_tiles = attn_env_int("MSD_ATTN_CHUNK_TILES", pl->Rp <= 16 ? 16 : 32);
-  if (chunk_tiles < 1) chunk_tiles = 1;
+  int chunk_tiles = option(OPT_ATTN_CHUNK_TILES);       // testing aid
+  if (chunk_tiles < 1) chunk_tiles = pl->Rp <= 16 ? 16 : 32;
   while (chunk_tiles > 2 && units * ((tiles + chunk_tiles - 1) / chunk_tiles) < static_cast<long long>(sm_count()) * 4) chunk_tiles >>= 1;
   int ns = (tiles + chunk_tiles - 1) / chunk_tiles;
   if (ns < 1) ns = 1;
-  if (const int forced = attn_env_int("MSD_ATTN_SPLITS", 0)) {      // testing aid: a given number of splits
-    ns = forced < 1 ? 1 : forced;
+  if (const int forced = option(OPT_ATTN_SPLITS); forced >= 1) {      // testing aid: a given number of splits
+    ns = forced;
     chunk_tiles = (tiles + ns - 1) / ns;
     if (chunk_tiles < 1) chunk_tiles = 1;
   }
@@ -1432,7 +1427,7 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
     // programmatic dependent (its CTAs start their KV loads while it runs)
     attn_qstack_kernel<<<B * Hkv * pl.groups, 256, 0, s>>>(p, q_img, q_scales);
     if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
-    if (launch_pdl(kernel, grid, dim3(block_threads), pl.smem_bytes, s, getenv("MSD_NO_PDL") == nullptr, tmap_k, tmap_v, p) != cudaSuccess)
+    if (launch_pdl(kernel, grid, dim3(block_threads), pl.smem_bytes, s, option(OPT_NO_PDL) <= 0, tmap_k, tmap_v, p) != cudaSuccess)
       return MSD_ERR_CUDA;
   } else {
     kernel<<<grid, block_threads, pl.smem_bytes, s>>>(tmap_k, tmap_v, p);

@@ -22,14 +22,10 @@ constexpr int kDecCache = 4;   // 16-element chunks a thread keeps in registers 
 template <int kDecThreads>
 __global__ void __launch_bounds__(kDecThreads)
 decompose_int8_kernel(const uint16_t* __restrict__ x, int64_t ldx, int K, int8_t* __restrict__ q1,
-                      int8_t* __restrict__ q2, float* __restrict__ alpha_out, float* __restrict__ beta_out, int early_trigger,
+                      int8_t* __restrict__ q2, float* __restrict__ alpha_out, float* __restrict__ beta_out,
                       float c1, float c2) {
-  // When launched as a programmatic dependent of whatever precedes it in the stream it may become resident early, but
-  // it reads nothing before that work has completed (the wait is a no-op for a plain launch); only then may its own
-  // dependent (the GEMM) start prefetching weights.
-  if (early_trigger) pdl_launch_dependents();
-  pdl_wait_primary();
-  if (!early_trigger) pdl_launch_dependents();
+  // the GEMM launched behind this kernel as its programmatic dependent may become resident now and prefetch weights
+  pdl_launch_dependents();
   const int row = blockIdx.x;
   const uint4* xr = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(row) * ldx);
   const int nchunks = K >> 4;
@@ -92,23 +88,17 @@ constexpr int kMxThreads = 256;
 __device__ __forceinline__ float pow2f(int e) { return __uint_as_float(static_cast<uint32_t>(e + 127) << 23); }
 
 // The first `rl.blocks` CTAs do the (independent) scale relayout `rl`, the others the decomposition, 256 consecutive
-// 32-element blocks (row-major) per CTA and round.  With `ready` != nullptr the kernel publishes its progress so that a
-// GEMM launched as its programmatic dependent can start on the first token tiles while the rest is still being
-// decomposed: ready[t] counts the finished blocks of token tile t (128 rows), ready[tiles] the finished relayout CTAs.
+// 32-element blocks (row-major) per CTA and round.
 __global__ void __launch_bounds__(kMxThreads)
 decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, int K, uint8_t* __restrict__ q1,
                        uint8_t* __restrict__ q2, uint8_t* __restrict__ e1, uint8_t* __restrict__ e2, int sf_kgroups,
-                       const SfRelayout rl, unsigned* __restrict__ ready, const RowGroups rg) {
+                       const SfRelayout rl, const RowGroups rg) {
   pdl_launch_dependents();
   const int kblocks = K >> 5;
   const int64_t nblocks = M * kblocks;
   if (static_cast<int>(blockIdx.x) < rl.blocks) {
     __shared__ uint32_t sm_rl[kSfRelayoutSmemWords];
     sf_relayout(rl, blockIdx.x, rl.blocks, sm_rl);
-    if (ready) {
-      __syncthreads();
-      if (threadIdx.x == 0) { __threadfence(); atomicAdd(&ready[(M + 127) >> 7], 1u); }
-    }
     return;
   }
   const int64_t units = (nblocks + kMxThreads - 1) / kMxThreads;
@@ -180,48 +170,34 @@ decompose_mxfp4_kernel(const uint16_t* __restrict__ x, int64_t ldx, int64_t M, i
       e2[so] = static_cast<uint8_t>(bexp + 127);
     }
     }
-    if (ready) {
-      // 128 x kblocks is a multiple of 256 (K is a multiple of 128 here), so a round never straddles two token tiles
-      __syncthreads();
-      if (threadIdx.x == 0) {
-        const int64_t first = u * kMxThreads;
-        const int64_t left = nblocks - first;
-        __threadfence();
-        atomicAdd(&ready[(first / kblocks) >> 7], static_cast<unsigned>(left < kMxThreads ? left : kMxThreads));
-      }
-    }
   }
 }
 
 msd_status_t launch_decompose_int8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q1, int8_t* q2,
                                    float* alpha, float* beta, float c1, float c2, cudaStream_t stream) {
   if (M == 0) return MSD_OK;
-  // Chained programmatic launch (this kernel resident while its predecessor still runs) is opt-in: measured slower.
-  const bool pdl = getenv("MSD_DEC_CHAIN") != nullptr && getenv("MSD_NO_PDL") == nullptr;
-  const int early = (pdl && atoi(getenv("MSD_DEC_CHAIN")) >= 2) ? 1 : 0;
-  const char* te = getenv("MSD_DEC_THREADS");
+  // A plain launch (chaining it to its predecessor as a programmatic dependent measured slower: its loads then queue
+  // behind the weight prefetch of the GEMM that follows it).
   // this kernel sits on the critical path of the GEMM behind it: more threads per row = shorter latency
-  const int threads = te ? atoi(te) : (K >= 8192 ? 1024 : (K >= 2048 ? 512 : 256));
+  const int threads = K >= 8192 ? 1024 : (K >= 2048 ? 512 : 256);
   cudaError_t err;
   if (threads >= 1024)
-    err = launch_pdl(decompose_int8_kernel<1024>, dim3(static_cast<unsigned>(M)), dim3(1024), 0, stream, pdl,
-                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, early, c1, c2);
+    err = launch_pdl(decompose_int8_kernel<1024>, dim3(static_cast<unsigned>(M)), dim3(1024), 0, stream, false,
+                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, c1, c2);
   else if (threads >= 512)
-    err = launch_pdl(decompose_int8_kernel<512>, dim3(static_cast<unsigned>(M)), dim3(512), 0, stream, pdl,
-                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, early, c1, c2);
+    err = launch_pdl(decompose_int8_kernel<512>, dim3(static_cast<unsigned>(M)), dim3(512), 0, stream, false,
+                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, c1, c2);
   else
-    err = launch_pdl(decompose_int8_kernel<256>, dim3(static_cast<unsigned>(M)), dim3(256), 0, stream, pdl,
-                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, early, c1, c2);
+    err = launch_pdl(decompose_int8_kernel<256>, dim3(static_cast<unsigned>(M)), dim3(256), 0, stream, false,
+                     static_cast<const uint16_t*>(x_bf16), static_cast<int64_t>(ldx), static_cast<int>(K), q1, q2, alpha, beta, c1, c2);
   return err == cudaSuccess ? MSD_OK : MSD_ERR_CUDA;
 }
 
 msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
                                     uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream, SfRelayout* relayout,
-                                    unsigned* ready, const RowGroups* groups) {
+                                    const RowGroups* groups) {
   if (M == 0) return MSD_OK;
-  // With progress flags the grid is small enough (two CTAs per SM, one more for the relayout) to be resident at
-  // once and to leave room for the dependent GEMM's CTA beside it.
-  const int per_sm = ready ? 2 : 32, rl_per_sm = ready ? 1 : ((relayout && relayout->matrices > 1) ? 16 : 4);
+  const int per_sm = 32, rl_per_sm = (relayout && relayout->matrices > 1) ? 16 : 4;
   SfRelayout rl = {};
   if (relayout) {
     rl = *relayout;
@@ -241,7 +217,7 @@ msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, in
     carve_done = true;
   }
   decompose_mxfp4_kernel<<<grid, kMxThreads, 0, stream>>>(static_cast<const uint16_t*>(x_bf16), ldx, M,
-                                                          static_cast<int>(K), q1, q2, e1, e2, sf_kgroups, rl, ready, rg);
+                                                          static_cast<int>(K), q1, q2, e1, e2, sf_kgroups, rl, rg);
   return launch_status();
 }
 

@@ -40,9 +40,6 @@ struct GemmW4Params {
   const uint8_t* sfb;
   void* y;
   int ytype;
-  const unsigned* ready;        // progress of the decomposition kernel running beside this one (nullptr: it has finished):
-                                // [t] finished 32-element blocks of token tile t, [m_tiles] finished relayout CTAs
-  unsigned ready_sfb;           // value of ready[m_tiles] when the weight scales are all in place
   int ksplit, kper;             // K splits per output tile and K stages per split (1, kstages: no split)
   int part_rows;                // ksplit > 1: rows per split of the partial-sum buffer the tiles are written to
   int nstages;                  // pipeline stages that fit with a_rows rows per component tile
@@ -50,7 +47,6 @@ struct GemmW4Params {
                                 // fewer when no group of a grouped launch is longer; the MMA reads stale rows beyond them,
                                 // whose results are never stored
   int n_fastest;                // tile index -> (token tile, weight tile): weight tile fastest (1) or token tile fastest (0)
-  int sf_warps;                 // 1: warps 6..9 write the scales into TMEM (tcgen05.st); 0: the MMA thread copies them (tcgen05.cp)
   unsigned* status;
 };
 
@@ -95,24 +91,6 @@ msd_status_t launch_ksplit_reduce(const float* part, int ksplit, int64_t part_st
              ? MSD_OK : MSD_ERR_CUDA;
 }
 
-// Bounded wait for a progress counter of the kernel this one depends on (see GemmW4Params::ready); afterwards the
-// async proxy (TMA) may read what that kernel's threads wrote.
-__device__ __forceinline__ bool wait_progress(const unsigned* counter, unsigned target, volatile int* abort, unsigned* status) {
-  const long long t0 = clock64();
-  while (true) {
-    unsigned v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
-    if (v >= target) break;
-    if (*abort) return false;
-    if (clock64() - t0 > kWaitBudgetCycles) {
-      *abort = 1;
-      atomicMax(status, kStatusTimeout);
-      return false;
-    }
-  }
-  fence_proxy_async_all();
-  return true;
-}
 
 // kTN = weight rows per tile: 256 (one accumulator) or 224 (two accumulators of 224 columns + the two sets of scale
 // columns fill the 512 TMEM columns exactly, so the epilogue of a tile overlaps the MMAs of the next).
@@ -168,23 +146,14 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
     // refill to be requested is part of the pipeline's round trip.  Warp 0 requests the operand tiles, warp 10 the
     // scale blocks (their bytes may be counted before warp 0's arrival announces them: the phase cannot end without it).
     if (lane == 0) {
-      // Components and blocked scales come from the kernel launched just before: either it has finished
-      // (griddepcontrol.wait), or it runs beside this one and says per token tile how far it is.
+      // components and blocked scales come from the kernel launched just before
       bool ok = true;
-      if (!p.ready) pdl_wait_primary();
-      else ok = wait_progress(p.ready + p.m_tiles, p.ready_sfb, abort, p.status);
+      pdl_wait_primary();
       int stage = 0; uint32_t phase = 0;
-      int mt_ready = -1;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const int split = tile % p.ksplit, tile_mn = tile / p.ksplit;
         const int mt = p.n_fastest ? tile_mn / p.n_tiles : tile_mn % p.m_tiles, nt = p.n_fastest ? tile_mn % p.n_tiles : tile_mn / p.m_tiles;
         const int ks0 = split * p.kper, ks1 = ks0 + p.kper < p.kstages ? ks0 + p.kper : p.kstages;
-        if (p.ready && mt != mt_ready) {
-          const int rows = p.M - mt * kW4TileM < kW4TileM ? p.M - mt * kW4TileM : kW4TileM;
-          ok = wait_progress(p.ready + mt, static_cast<unsigned>(rows) * static_cast<unsigned>(p.K >> 5), abort, p.status);
-          if (!ok) break;
-          mt_ready = mt;
-        }
         for (int ks = ks0; ks < ks1; ++ks) {
           ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
           if (!ok) break;
@@ -218,7 +187,6 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
       uint32_t sfpar = 0;
       int nstage = 0;                                                   // stages issued so far (all tiles)
       const uint64_t op_desc = smem_desc(0, 16, 1024, kSwizzle128B);    // 128-byte-swizzled K-major operand tile
-      const uint64_t sf_desc = smem_desc(0, 0, 128, 0);                 // scale block: eight-row groups 128 bytes apart, no swizzle
       const uint32_t idesc_lo = idesc_block_scaled(/*E2M1*/ 1, 1, kW4TileM, kTN, 0, 0);
       const uint32_t idesc_hi = idesc_block_scaled(/*E2M1*/ 1, 1, kW4TileM, kTN, 2, 2);
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
@@ -238,25 +206,14 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
           // count per stage, not the tensor pipe, was what paced the kernel.
           const uint64_t enc = static_cast<uint64_t>(smem_u32(smem + stage * kStageBytes) >> 4);
           const uint64_t a1d = op_desc + enc, a2d = a1d + (a_bytes >> 4), bd = a1d + (2 * a_bytes >> 4);
-          const uint64_t sfd = sf_desc + enc + ((2 * a_bytes + kBBytes) >> 4);
           const uint32_t sfa1_t = tmem_base + kSfCol + 32 * sfpar;     // 2 k-groups x 4 columns; the two sets alternate
           const uint32_t sfa2_t = sfa1_t + 8;
           const uint32_t sfb_t = sfa1_t + 16;                            // 2 k-groups x 8 columns (256 weight rows)
-          if (p.sf_warps) {
-            // the scale columns of this stage were written by warps 6..9 (the shared-memory -> TMEM copies of the tensor
-            // pipe run in order with the MMAs and cost a sixth of its time)
-            ok = wait_bounded(&sf_ready[sfpar], (nstage >> 1) & 1, abort, p.status);
-            if (!ok) break;
-            tc_fence_after();
-          } else {
-#pragma unroll
-            for (int g = 0; g < 2; ++g) {
-              tc_cp_32x128b_warpx4(sfa1_t + 4 * g, sfd + (g * 512 >> 4));
-              tc_cp_32x128b_warpx4(sfa2_t + 4 * g, sfd + ((1024 + g * 512) >> 4));
-              tc_cp_32x128b_warpx4(sfb_t + 8 * g, sfd + ((2048 + g * 512) >> 4));
-              tc_cp_32x128b_warpx4(sfb_t + 8 * g + 4, sfd + ((3072 + g * 512) >> 4));
-            }
-          }
+          // the scale columns of this stage were written by warps 6..9 (tcgen05.cp copies issued by this thread run in
+          // order with the MMAs in the tensor pipe and cost a sixth of its time)
+          ok = wait_bounded(&sf_ready[sfpar], (nstage >> 1) & 1, abort, p.status);
+          if (!ok) break;
+          tc_fence_after();
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {                    // 64 elements (32 bytes) per MMA
             const int g = kk >> 1;
@@ -279,38 +236,36 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
     // carries the four scales of rows l, l+32, l+64, l+96, and every 32-lane quadrant of TMEM wants the same four
     // 32-bit columns.  Each warp reads the stage's eight blocks (one 16-byte row per lane and block) and stores them as
     // 32 columns of its own quadrant.
-    if (p.sf_warps) {
-      const int quad = warp & 3;
-      int stage = 0; uint32_t phase = 0;
-      int n = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int ks0 = (tile % p.ksplit) * p.kper, ks1 = ks0 + p.kper < p.kstages ? ks0 + p.kper : p.kstages;
-        for (int ks = ks0; ks < ks1; ++ks, ++n) {
-          const int set = n & 1;
-          ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
+    const int quad = warp & 3;
+    int stage = 0; uint32_t phase = 0;
+    int n = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int ks0 = (tile % p.ksplit) * p.kper, ks1 = ks0 + p.kper < p.kstages ? ks0 + p.kper : p.kstages;
+      for (int ks = ks0; ks < ks1; ++ks, ++n) {
+        const int set = n & 1;
+        ok = wait_bounded(&full_bar[stage], phase, abort, p.status);
+        if (!ok) break;
+        if (n >= 2) {                        // the MMAs that read this set two stages ago are done
+          ok = wait_bounded(&sf_free[set], ((n >> 1) - 1) & 1, abort, p.status);
           if (!ok) break;
-          if (n >= 2) {                        // the MMAs that read this set two stages ago are done
-            ok = wait_bounded(&sf_free[set], ((n >> 1) - 1) & 1, abort, p.status);
-            if (!ok) break;
-            tc_fence_after();
-          }
-          const uint4* sf = reinterpret_cast<const uint4*>(smem + stage * kStageBytes + 2 * a_bytes + kBBytes) + lane;
-          uint32_t v[32];
-          // column order of a set: sfa1 (g0, g1), sfa2 (g0, g1), then per K group the two halves of the weight tile
-          constexpr int kBlk[8] = {0, 1, 2, 3, 4, 6, 5, 7};
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const uint4 q = sf[kBlk[j] * 32];
-            v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
-          }
-          tmem_st32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + kSfCol + 32 * set, v);
-          tmem_st_wait();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&sf_ready[set]);
-          if (++stage == nstages) { stage = 0; phase ^= 1; }
+          tc_fence_after();
         }
+        const uint4* sf = reinterpret_cast<const uint4*>(smem + stage * kStageBytes + 2 * a_bytes + kBBytes) + lane;
+        uint32_t v[32];
+        // column order of a set: sfa1 (g0, g1), sfa2 (g0, g1), then per K group the two halves of the weight tile
+        constexpr int kBlk[8] = {0, 1, 2, 3, 4, 6, 5, 7};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint4 q = sf[kBlk[j] * 32];
+          v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
+        }
+        tmem_st32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + kSfCol + 32 * set, v);
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sf_ready[set]);
+        if (++stage == nstages) { stage = 0; phase ^= 1; }
       }
     }
   } else {
@@ -683,7 +638,7 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
 struct GemmW4Plan {
   int m_tiles, n_tiles, kstages, sf_kgroups, grid, tile_n;
   int ksplit, kper, a_rows, nstages;
-  size_t off_q1, off_q2, off_sfa1, off_sfa2, off_sfb, off_ready, off_part, bytes;
+  size_t off_q1, off_q2, off_sfa1, off_sfa2, off_sfb, off_part, bytes;
 };
 
 // The CTA-pair kernel (256 tokens x 256 weight rows per pair of CTAs: half the weight tile per CTA, so less shared-memory
@@ -693,8 +648,7 @@ struct GemmW4Plan {
 // MSD_W4_PAIR=0/1 forces the choice.
 static bool w4_use_pair(int64_t M, int64_t N, int64_t K) {
   (void)K;
-  const char* pe = getenv("MSD_W4_PAIR");
-  if (pe) return atoi(pe) != 0;
+  if (const int forced = option(OPT_W4_PAIR); forced >= 0) return forced != 0;     // testing aid
   const int64_t m_tiles = (M + kW4TileM - 1) / kW4TileM, n_tiles = (N + 255) / 256;
   const int64_t clusters = sm_count() / 2, pair_tiles = (m_tiles + 1) / 2 * n_tiles, single_tiles = m_tiles * ((N + 223) / 224);
   // an odd number of token tiles leaves the last pair's second CTA without rows: only where that is a small share
@@ -707,8 +661,7 @@ static bool w4_use_pair(int64_t M, int64_t N, int64_t K) {
 // Weight rows per tile: MSD_W4_TILEN (224 or 256) if set; else 256 for the CTA-pair kernel (one accumulator) and 224 for
 // the single-CTA kernel (two accumulators: the epilogue of a tile overlaps the MMAs of the next).
 static int w4_tile_n(bool pair = false) {
-  const char* e = getenv("MSD_W4_TILEN");
-  if (e) return atoi(e) == 256 ? 256 : 224;
+  if (const int forced = option(OPT_W4_TILEN); forced >= 0) return forced == 256 ? 256 : 224;     // testing aid
   return pair ? 256 : 224;
 }
 
@@ -726,8 +679,8 @@ static GemmW4Plan plan_w4(int64_t M, int64_t N, int64_t K) {
   pl.ksplit = 1;
   pl.kper = pl.kstages;
   {
-    const char* se = getenv("MSD_W4_KSPLIT");
-    int want = se ? atoi(se) : (2 * tiles <= sm_count() ? sm_count() / tiles : 1);
+    const int forced = option(OPT_W4_KSPLIT);     // testing aid
+    int want = forced >= 0 ? forced : (2 * tiles <= sm_count() ? sm_count() / tiles : 1);
     if (want > pl.kstages / 4) want = pl.kstages / 4;
     if (want > 1) {
       pl.kper = (pl.kstages + want - 1) / want;
@@ -751,7 +704,6 @@ static GemmW4Plan plan_w4(int64_t M, int64_t N, int64_t K) {
   pl.off_sfa1 = off; off = round_up(off + static_cast<size_t>(pl.m_tiles) * pl.sf_kgroups * 512, 1024);
   pl.off_sfa2 = off; off = round_up(off + static_cast<size_t>(pl.m_tiles) * pl.sf_kgroups * 512, 1024);
   pl.off_sfb = off;  off = round_up(off + static_cast<size_t>(2 * pl.n_tiles) * pl.sf_kgroups * 512, 1024);
-  pl.off_ready = off; off = round_up(off + static_cast<size_t>(pl.m_tiles + 1) * sizeof(unsigned), 1024);
   pl.off_part = off;
   if (pl.ksplit > 1) off = round_up(off + static_cast<size_t>(pl.ksplit) * pl.m_tiles * kW4TileM * N * sizeof(float), 1024);
   pl.bytes = off;
@@ -769,9 +721,8 @@ static GroupedW4Plan plan_grouped_w4(int32_t E, int64_t N, int64_t K, int groups
   GroupedW4Plan pl;
   // Tile width: the one whose tiles fill the SMs in fewer, or shorter, rounds (groups = non-empty groups of the first
   // launch; the workspace is sized for the wider layout of the blocked weight scales either way)
-  const char* te = getenv("MSD_W4_TILEN");
-  if (te) {
-    pl.tile_n = atoi(te) == 256 ? 256 : 224;
+  if (const int forced = option(OPT_W4_TILEN); forced >= 0) {
+    pl.tile_n = forced == 256 ? 256 : 224;
   } else {
     const long long g = groups < 1 ? 1 : (groups > kMaxRowGroups ? kMaxRowGroups : groups);
     const long long t224 = g * ((N + 223) / 224), t256 = g * ((N + 255) / 256);
@@ -821,22 +772,16 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   uint8_t* q1 = ws + pl.off_q1;
   uint8_t* q2 = ws + pl.off_q2;
 
-  // The weight scales go into the blocked layout in the same launch as the decomposition of x.  Opt-in
-  // (MSD_W4_OVERLAP=1, single-CTA kernel): that launch also publishes its progress per token tile (counters zeroed
-  // here) and the GEMM, its programmatic dependent, starts on the first token tiles while the others are still being
-  // decomposed.  Measured: the GEMM's CTAs do enter 5-9 us after the decomposition starts, but the decomposition,
-  // held to two CTAs per SM so that both fit, then takes 47 instead of 25 us and the GEMM beside it is slower by as
-  // much as the earlier start gains.
+  // The weight scales go into the blocked layout in the same launch as the decomposition of x.  (Letting the GEMM start
+  // on the first token tiles while the others are still being decomposed, behind per-tile progress counters, was built
+  // and measured: the decomposition, held to two CTAs per SM so that both kernels fit, took twice as long and the GEMM
+  // beside it lost what the earlier start gained.)
   const bool use_pair = w4_use_pair(M, N, K);
-  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  const char* ove = getenv("MSD_W4_OVERLAP");
-  const bool overlap = !use_pair && pdl && ove && atoi(ove) != 0;
-  unsigned* ready = overlap ? reinterpret_cast<unsigned*>(ws + pl.off_ready) : nullptr;
-  if (ready && cudaMemsetAsync(ready, 0, static_cast<size_t>(pl.m_tiles + 1) * sizeof(unsigned), s) != cudaSuccess) return MSD_ERR_CUDA;
+  const bool pdl = option(OPT_NO_PDL) <= 0;
   SfRelayout rl = {};
   rl.src = w_e8m0; rl.dst = ws + pl.off_sfb; rl.rows = N; rl.kblocks = static_cast<int>(K / 32);
   rl.sf_kgroups = pl.sf_kgroups; rl.tile_rows = pl.tile_n; rl.row_blocks = 2 * pl.n_tiles;
-  msd_status_t st = launch_decompose_mxfp4(x_bf16, M, K, K, q1, q2, ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s, &rl, ready);
+  msd_status_t st = launch_decompose_mxfp4(x_bf16, M, K, K, q1, q2, ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s, &rl);
   if (st != MSD_OK) return st;
 
   CUtensorMap tmap_a1, tmap_a2, tmap_b;
@@ -851,19 +796,13 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.kstages = pl.kstages; p.sf_kgroups = pl.sf_kgroups;
   p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
   p.y = y; p.ytype = ytype; p.status = status;
-  p.ready = ready; p.ready_sfb = static_cast<unsigned>(rl.blocks);
   p.a_rows = kW4TileM; p.nstages = kW4Stages; p.ksplit = 1; p.kper = pl.kstages; p.part_rows = 0;
   {
-    const char* sfe = getenv("MSD_W4_SFWARPS");
-    p.sf_warps = sfe ? atoi(sfe) : 1;
     // Tile order.  A wave of CTAs either shares a few weight tiles and sweeps the token tiles (token tile fastest)
     // or the other way round; the operand that is swept should be the one that stays in L2 (40 MB assumed usable for
-    // it).  Both components of x weigh M x K bytes, the weights N x K / 2.  With the decomposition running beside
-    // the GEMM the first wave should need only the first token tiles: weight tile fastest.
-    const char* oe = getenv("MSD_W4_ORDER");
+    // it).  Both components of x weigh M x K bytes, the weights N x K / 2.
     const double l2 = 40.0 * 1024 * 1024, a_bytes = static_cast<double>(M) * K, w_bytes = static_cast<double>(N) * K / 2;
-    const bool n_fast = overlap ? true : (a_bytes <= l2 ? false : (w_bytes <= l2 ? true : a_bytes > w_bytes));
-    p.n_fastest = oe ? (atoi(oe) != 0) : n_fast;
+    p.n_fastest = a_bytes <= l2 ? 0 : (w_bytes <= l2 ? 1 : (a_bytes > w_bytes ? 1 : 0));
   }
 
   // With a K split the kernel writes FP32 partial tiles (split s at rows s * part_rows ...) and a second kernel adds them.
@@ -976,7 +915,7 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
       return MSD_ERR_CUDA;
     attr_done = true;
   }
-  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+  const bool pdl = option(OPT_NO_PDL) <= 0;
 
   // up to 64 non-empty groups per pair of launches (decomposition + GEMM); the weight scales of all experts are brought
   // into the blocked layout by the first decomposition launch
@@ -1006,7 +945,7 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
     rl.src = w_e8m0; rl.dst = ws + pl.off_sfb; rl.rows = N; rl.kblocks = static_cast<int>(K / 32);
     rl.sf_kgroups = pl.sf_kgroups; rl.tile_rows = pl.tile_n; rl.row_blocks = 2 * pl.n_tiles; rl.matrices = E;
     msd_status_t st = launch_decompose_mxfp4(static_cast<const uint16_t*>(x_bf16) + row_first * K, row - row_first, K, K, q1, q2,
-                                             ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s, scales_done ? nullptr : &rl, nullptr, &rg);
+                                             ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s, scales_done ? nullptr : &rl, &rg);
     if (st != MSD_OK) return st;
     scales_done = true;
 
@@ -1015,13 +954,10 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
     p.m_tiles = grp.n; p.n_tiles = pl.n_tiles; p.kstages = pl.kstages; p.sf_kgroups = pl.sf_kgroups;
     p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
     p.y = y; p.ytype = ytype; p.status = status;
-    p.ready = nullptr; p.ready_sfb = 0;
     p.a_rows = a_rows; p.nstages = nstages;
     p.ksplit = 1; p.kper = pl.kstages; p.part_rows = 0;
     p.n_fastest = 1;              // the CTAs of a wave share a group's components; every expert's weights are read once
     {
-      const char* sfe = getenv("MSD_W4_SFWARPS");
-      p.sf_warps = sfe ? atoi(sfe) : 1;
     }
     const long long tiles = static_cast<long long>(grp.n) * pl.n_tiles;
     const int grid = static_cast<int>(tiles < sm_count() ? tiles : sm_count());

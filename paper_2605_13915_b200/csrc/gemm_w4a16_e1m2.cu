@@ -448,7 +448,7 @@ msd_status_t msd_gemm_w4a16_e1m2(const void* x_bf16, const uint8_t* w_fp4, const
       return MSD_ERR_CUDA;
     attr_done = true;
   }
-  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+  const bool pdl = option(OPT_NO_PDL) <= 0;
   if (launch_pdl(gemm_w4a16_e1m2_kernel, dim3(pl.grid), dim3(kE1Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p) != cudaSuccess)
     return MSD_ERR_CUDA;
   return MSD_OK;

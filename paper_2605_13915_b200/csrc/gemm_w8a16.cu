@@ -54,13 +54,6 @@ struct GemmW8Params {
   const float* w_scale;
   float* alpha;
   float* beta;
-  const uint16_t* x;       // in-kernel decomposition: the BF16 activations [M, ldx]
-  long long ldx;
-  int inline_dec;          // 1: the first dec_ctas CTAs decompose the rows before the main loop, the others wait for a flag
-  int dec_ctas;
-  float c1, c2;            // scaling constants of the in-kernel decompositions (alpha = max/c1, beta = alpha/c2)
-  int8_t* q;               // stacked components [NB, K] (rows [0,M) = Q1, [Mp, Mp+M) = Q2) in the workspace
-  unsigned* flags;         // [2]: rows decomposed, CTAs that have seen all of them (both zero between calls)
   void* y;
   int32_t* acc_dbg;
   int32_t* accum;          // [num_tiles][NB][128] split-K meeting place, zero between calls (INT32 or FP32 bits)
@@ -69,7 +62,7 @@ struct GemmW8Params {
   long long* trace;        // nullable diagnostic buffer: 16 clock samples per CTA
 };
 
-// Grouped GEMM (MoE experts, Sec. 7.2 "Extension to MoE"): the problems of one launch.  Group g multiplies the token rows
+// Grouped GEMM (MoE experts; Discussion, "Extension to MoE and Sparse Architectures"): the problems of one launch.  Group g multiplies the token rows
 // [off[g], off[g] + m[g]) of x against expert expert[g]'s weight [N, K]; all groups share N, K and the kernel's tile shapes.
 constexpr int kMaxGroups = 64;
 struct GemmW8Groups {
@@ -226,19 +219,17 @@ __device__ __forceinline__ void epilogue_chunk(const GemmW8Params& p, uint32_t t
 }
 
 // The token chunks [tok0, tok1) of one finished tile (both multiples of 8).
-template <bool kBase, bool kFused, bool kBf16>
+template <bool kBase, bool kBf16>
 __device__ __forceinline__ void epilogue_tile(const GemmW8Params& p, uint32_t t_row, int32_t* acc_tile, int r, int n, bool row_ok,
                                               float sw, const float* s_alpha, const float* s_beta, uint8_t* stage_buf, int et,
                                               int n0, int rows_valid, int tok0, int tok1, const RecvInfo& rv, int m_valid,
                                               long long y_row0) {
   int c0 = tok0;
-  if constexpr (!kFused) {
-    if constexpr (kBase)
-      for (; c0 + 32 <= tok1; c0 += 32)
-        epilogue_chunk<kBase, kBf16, 32>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv, m_valid, y_row0);
-    for (; c0 + 16 <= tok1; c0 += 16)      // 16 tokens at a time: two sums and two scales per token stay in registers
-      epilogue_chunk<kBase, kBf16, 16>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv, m_valid, y_row0);
-  }
+  if constexpr (kBase)
+    for (; c0 + 32 <= tok1; c0 += 32)
+      epilogue_chunk<kBase, kBf16, 32>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv, m_valid, y_row0);
+  for (; c0 + 16 <= tok1; c0 += 16)      // 16 tokens at a time: two sums and two scales per token stay in registers
+    epilogue_chunk<kBase, kBf16, 16>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv, m_valid, y_row0);
   for (; c0 + 8 <= tok1; c0 += 8)
     epilogue_chunk<kBase, kBf16, 8>(p, t_row, acc_tile, c0, r, n, row_ok, sw, s_alpha, s_beta, stage_buf, et, n0, rows_valid, rv, m_valid, y_row0);
 }
@@ -256,68 +247,14 @@ __device__ __forceinline__ void partial_chunk(uint32_t t_row, int32_t* acc_tile,
   }
 }
 
-// Fused path, step a1: the scales of all M <= kFusedMaxM rows (alpha = max|x|/127, beta = alpha/254; Eq. alpha, Eq. beta)
-// computed by the 256 threads of the epilogue and quantiser warps together.  Every thread keeps one running maximum
-// per row and requests the vectors of all rows before using any, so the whole phase costs a few L2 round trips
-// instead of one per row.  x may come from the preceding kernel of the stream: nothing is read before it has finished.
-constexpr int kFusedMaxM = 8;
-__device__ __forceinline__ void fused_row_scales(const GemmW8Params& p, int t256, float (*s_qmax)[8], float* s_alpha,
-                                                 float* s_beta, float* s_inva, float* s_invb) {
-  pdl_wait_primary();
-  const int nvec_row = p.K >> 3;                // 16-byte vectors of 8 BF16 values per row
-  float m[kFusedMaxM];
-#pragma unroll
-  for (int i = 0; i < kFusedMaxM; ++i) m[i] = 0.0f;
-  for (int c = t256; c < nvec_row; c += 256) {
-    uint4 v[kFusedMaxM];
-#pragma unroll
-    for (int i = 0; i < kFusedMaxM; ++i)
-      if (i < p.M) v[i] = __ldg(reinterpret_cast<const uint4*>(p.x + static_cast<long long>(i) * p.ldx) + c);
-#pragma unroll
-    for (int i = 0; i < kFusedMaxM; ++i) {
-      if (i < p.M) {
-        const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          m[i] = fmaxf(m[i], fabsf(__uint_as_float(w[k] << 16)));
-          m[i] = fmaxf(m[i], fabsf(__uint_as_float(w[k] & 0xFFFF0000u)));
-        }
-      }
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < kFusedMaxM; ++i) {
-    if (i < p.M) {
-      const float mm = warp_max(m[i]);
-      if ((t256 & 31) == 0) s_qmax[i][t256 >> 5] = mm;
-    }
-  }
-  named_bar_sync(2, 256);
-  if (t256 < p.M) {
-    float mm = 0.0f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) mm = fmaxf(mm, s_qmax[t256][w]);
-    const float alpha = __fdiv_rn(mm, p.c1), beta = __fdiv_rn(alpha, p.c2);
-    s_alpha[t256] = alpha;
-    s_beta[t256] = beta;
-    s_inva[t256] = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f;
-    s_invb[t256] = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
-  }
-  named_bar_sync(2, 256);                       // scales visible to the quantiser and the epilogue warps
-}
-
 // kBase = false: the MSD path (INT8 x INT8 -> INT32, stacked components, scale-combine epilogue).
 // kBase = true : the comparison path the method replaces - the same pipeline on BF16 weights that a preceding kernel
 //                dequantized into the workspace, BF16 x BF16 -> FP32, no decomposition and no scales in the epilogue.
-// kFused (small M): no separate decomposition kernel - four extra warps compute the row scales and quantise the
-//                stacked operand tile of every stage straight into shared memory ("online activation decomposition",
-//                Sec. 3.9), so the activations never round-trip through HBM and nothing waits for a previous launch.
-constexpr int kFusedThreads = kGemmThreads + 128;
 // kGrouped: several (token rows, expert weight) problems in one stream-K launch; the group table travels as a kernel
 //                parameter, weight tiles are addressed in the stacked [E*N, K] weight, the two components of a
 //                group's rows come as two boxes of the component buffer.
-template <bool kBase, bool kFused, bool kGrouped = false>
-__global__ void __launch_bounds__(kFused ? kFusedThreads : kGemmThreads, 1)
+template <bool kBase, bool kGrouped = false>
+__global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_w2,
                   const __grid_constant__ CUtensorMap tmap_x, const GemmW8Params p,
                   const __grid_constant__ typename GroupArg<kGrouped>::type grp) {
@@ -327,13 +264,11 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   __shared__ __align__(8) uint64_t tfull_bar[2];
   __shared__ __align__(8) uint64_t tempty_bar[2];
   __shared__ __align__(8) uint64_t cfree_bar, crecv_bar, cdone_bar;
-  __shared__ __align__(8) uint64_t xready_bar;               // in-kernel decomposition: every row is in memory
   __shared__ float s_red[4];      // mode 2: "pipelines of the cluster drained", "partials delivered"
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ int is_last_flag;
   __shared__ __align__(16) float s_alpha[128], s_beta[128];
-  __shared__ float s_inva[kFusedMaxM], s_invb[kFusedMaxM], s_qmax[kFusedMaxM][8];   // fused path: reciprocals of the scales, row-max scratch
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -381,18 +316,17 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   // whole row instead of hitting the same 128-byte column of every row (integer sums do not depend on the order).
   const int kb_rot = (p.mode == 1) ? static_cast<int>((static_cast<long long>(blockIdx.x) * p.kb_rot_step) % p.kblocks) : 0;
   const CUtensorMap* wmap = (p.mode == 1 && band_h != p.hmax) ? &tmap_w2 : &tmap_w;
-  const int tx_bytes = p.kw * ((p.mode == 0 ? kWStageBytes : band_h * kBlockK) + (kFused ? 0 : x_chunk_bytes));
+  const int tx_bytes = p.kw * ((p.mode == 0 ? kWStageBytes : band_h * kBlockK) + x_chunk_bytes);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.num_stages; ++s) {
-      mbar_init(&full_bar[s], kFused ? 2 : 1);     // fused: the producer's arrive plus the quantiser warp of the stage
+      mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(&tfull_bar[a], 1);
       mbar_init(&tempty_bar[a], 4);      // one arrival per epilogue warp
     }
-    mbar_init(&xready_bar, 1);
     if (p.mode == 2) {
       mbar_init(&cfree_bar, p.csplit);               // one arrival per CTA of the cluster
       mbar_init(&crecv_bar, 1);                      // this CTA's own arrival; the peers' copies count in bytes
@@ -439,7 +373,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     pol_w = policy_evict_first();    // weights are streamed once
     pol_x = policy_evict_last();      // the stacked components are re-read by every CTA
     w_lane = lane < p.kw;
-    x_lane = !kFused && lane >= p.kw && lane < (kGrouped ? 3 : 2) * p.kw;     // grouped: one box per component
+    x_lane = lane >= p.kw && lane < (kGrouped ? 3 : 2) * p.kw;     // grouped: one box per component
     c = w_lane ? lane : (lane - p.kw) % p.kw;
     x_half = w_lane ? 0 : (lane - p.kw) / p.kw;
     // (tile, K block) of the next block to load, advanced by one per stage; kbr = rotated K block
@@ -476,16 +410,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   if (threadIdx.x == 0) trace_mark(p, 2);
 
   if (warp == 0) {
-    if (!kBase && !kFused && p.inline_dec) {
-      // the stacked components are written by CTAs of this very kernel: the epilogue warps tell when all rows are there
-      int okw = 1;
-      if (lane == 0) okw = wait_bounded(&xready_bar, 0, abort, p.status) ? 1 : 0;
-      okw = __shfl_sync(0xffffffffu, okw, 0);
-      fence_proxy_async_all();      // generic-proxy stores of other CTAs, acquired above, before this warp's TMA reads
-      if (!okw) pre = 0, blk_end = blk_begin;
-    } else {
-      pdl_wait_primary();
-    }
+    pdl_wait_primary();
     if (lane == 0) trace_mark(p, 4);
     {
       int kx = kbr0;
@@ -575,126 +500,14 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       }
       trace_mark(p, 7);
     }
-  } else if (kFused && warp >= 6) {
-    // ------------------------------ quantiser warps (fused path) ------------------------------
-    const int qt = threadIdx.x - kGemmThreads;    // 0..127
-    const int qw = warp - 6;
-    fused_row_scales(p, qt + 128, s_qmax, s_alpha, s_beta, s_inva, s_invb);
-    // a2-a3: per stage, quantise the M x (kw*128) slice of X into the stacked operand tile (rows i and Mp+i).
-    // Each warp owns a fixed subset of the ring's stages (stage s belongs to warp s % 4) and fills them in order, so
-    // several stages are being filled at a time (one warp's load latency does not pace the pipeline) while every
-    // barrier is still waited on phase by phase by a single warp - a warp that could run two ring cycles ahead of
-    // another would make the parity test of the wait ambiguous.
-    const int vec_per_row = p.kw * 16;            // vectors of 8 elements per row and stage
-    const int nvec = p.M * vec_per_row;
-    bool ok = true;
-    for (long long blk = blk_begin; blk < blk_end && ok; ++blk) {
-      const long long it = blk - blk_begin;
-      const int stage = static_cast<int>(it % p.num_stages);
-      if ((stage & 3) != qw) continue;
-      const uint32_t phase = static_cast<uint32_t>((it / p.num_stages) & 1);
-      const int kb = static_cast<int>((blk + kb_rot) % p.kblocks);
-      ok = wait_bounded(&empty_bar[stage], phase ^ 1, abort, p.status);
-      if (!ok) break;
-      uint8_t* xt = smem + stage * stage_bytes + w_stage_bytes;
-      for (int v = lane; v < nvec; v += 32) {
-        const int i = v / vec_per_row, r = v - i * vec_per_row;
-        const int c = r >> 4, e8 = r & 15;
-        const long long k = (static_cast<long long>(kb) * p.kw + c) * kBlockK + e8 * 8;
-        uint4 xv = make_uint4(0, 0, 0, 0);
-        if (k < p.K) xv = __ldg(reinterpret_cast<const uint4*>(p.x + static_cast<long long>(i) * p.ldx + k));
-        const float alpha = s_alpha[i], beta = s_beta[i], inva = s_inva[i], invb = s_invb[i];
-        const uint32_t w[4] = {xv.x, xv.y, xv.z, xv.w};
-        uint32_t o1[2] = {0, 0}, o2[2] = {0, 0};
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float xf = (e & 1) ? __uint_as_float(w[e >> 1] & 0xFFFF0000u) : __uint_as_float(w[e >> 1] << 16);
-          int c1 = 0, c2 = 0;
-          if (alpha > 0.0f) {
-            c1 = quant_i8(xf, alpha, inva);                                  // Eq. x1
-            const float res = __fmaf_rn(-alpha, static_cast<float>(c1), xf); // Eq. residual (exact)
-            if (beta > 0.0f) c2 = quant_i8(res, beta, invb);                 // Eq. x2
-          }
-          o1[e >> 2] |= static_cast<uint32_t>(c1 & 0xFF) << (8 * (e & 3));
-          o2[e >> 2] |= static_cast<uint32_t>(c2 & 0xFF) << (8 * (e & 3));
-        }
-        uint8_t* dst = xt + c * x_chunk_bytes;
-        *reinterpret_cast<uint2*>(dst + swz_off(i, e8 * 8)) = make_uint2(o1[0], o1[1]);
-        *reinterpret_cast<uint2*>(dst + swz_off(p.Mp + i, e8 * 8)) = make_uint2(o2[0], o2[1]);
-      }
-      fence_proxy_async_smem();                   // the MMA reads this tile through the async proxy
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&full_bar[stage]);
-    }
   } else {
     // ------------------------------ epilogue (warps 2..5) ------------------------------
     const int quad = warp & 3;                    // TMEM lane group this warp may read
     const int r = quad * 32 + lane;               // weight row within the tile == TMEM lane
     const int et = threadIdx.x - 64;              // 0..127
-    bool return_early = false;
-    if constexpr (kFused) {
-      fused_row_scales(p, et, s_qmax, s_alpha, s_beta, s_inva, s_invb);   // together with the quantiser warps
-    } else if constexpr (!kBase) {
+    if constexpr (!kBase) {
       pdl_wait_primary();
-      if (p.inline_dec) {
-        // ---- a1-a3 inside the GEMM kernel: CTA c < dec_ctas decomposes rows c, c + dec_ctas, ... with its epilogue
-        // warps (idle until the first accumulator is complete) while its producer already streams weights; a counter
-        // in the workspace tells every CTA when all rows are in memory.  No kernel boundary between a3 and a4.
-        const int ndec = static_cast<int>(gridDim.x) < p.dec_ctas ? static_cast<int>(gridDim.x) : p.dec_ctas;
-        int rows_done = 0;
-        if (static_cast<int>(blockIdx.x) < ndec) {
-          const int nchunks = p.K >> 4;
-          for (int row = blockIdx.x; row < p.M; row += ndec, ++rows_done) {
-            const uint4* xr = reinterpret_cast<const uint4*>(p.x + static_cast<long long>(row) * p.ldx);
-            float m = 0.0f;
-            for (int c = et; c < nchunks; c += 128) m = fmaxf(m, chunk_absmax(__ldg(xr + 2 * c), __ldg(xr + 2 * c + 1)));
-            m = warp_max(m);
-            if (lane == 0) s_red[warp & 3] = m;
-            named_bar_sync(1, 128);
-            m = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
-            named_bar_sync(1, 128);                              // s_red is rewritten for the next row
-            const float alpha = __fdiv_rn(m, p.c1);              // Eq. alpha
-            const float beta = __fdiv_rn(alpha, p.c2);           // Eq. beta
-            const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f;
-            const float inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
-            if (et == 0) { p.alpha[row] = alpha; p.beta[row] = beta; }
-            uint4* o1 = reinterpret_cast<uint4*>(p.q + static_cast<long long>(row) * p.K);
-            uint4* o2 = reinterpret_cast<uint4*>(p.q + static_cast<long long>(p.Mp + row) * p.K);
-            for (int c = et; c < nchunks; c += 128) {
-              uint4 r1, r2;
-              chunk_quantize(__ldg(xr + 2 * c), __ldg(xr + 2 * c + 1), alpha, beta, inv_alpha, inv_beta, r1, r2);
-              o1[c] = r1;
-              o2[c] = r2;
-            }
-          }
-        }
-        if (rows_done > 0) {
-          __threadfence();
-          fence_proxy_async_all();          // these rows are read through TMA (async proxy) by every CTA
-          named_bar_sync(1, 128);
-          if (et == 0) atomicAdd(&p.flags[0], static_cast<unsigned>(rows_done));
-        }
-        if (et == 0) {
-          // bounded poll for "all M rows decomposed"
-          const long long t0 = clock64();
-          bool seen = false;
-          while (true) {
-            unsigned v;
-            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.flags) : "memory");
-            if (v >= static_cast<unsigned>(p.M)) { seen = true; break; }
-            if (*abort) break;
-            if (clock64() - t0 > kWaitBudgetCycles) { *abort = 1; atomicMax(p.status, kStatusTimeout); break; }
-          }
-          if (seen) {
-            mbar_arrive(&xready_bar);       // lets this CTA's producer request the component tiles
-            // the CTA that is last to see the full count leaves both counters zero for the next call
-            if (atomicAdd(&p.flags[1], 1u) == gridDim.x - 1) { p.flags[0] = 0; p.flags[1] = 0; }
-          }
-        }
-        named_bar_sync(1, 128);
-        if (*abort) return_early = true;
-      }
-      if (!kGrouped && et < p.M && !return_early) {
+      if (!kGrouped && et < p.M) {
         s_alpha[et] = __ldcg(p.alpha + et);
         s_beta[et] = __ldcg(p.beta + et);
       }
@@ -702,7 +515,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     named_bar_sync(1, 128);
     int seg = 0;
     int sent_to = 0;           // mode 2: finishing CTAs whose acknowledgement is outstanding
-    bool ok = !return_early;
+    bool ok = true;
     long long blk = blk_begin;
     while (blk < blk_end && ok) {
       const int tile = static_cast<int>(blk / p.kblocks);
@@ -734,7 +547,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       int32_t* acc_tile = nullptr;
       int tok0 = 0, tok1 = p.Mp;
       RecvInfo rv = {nullptr, 0, 0, 0, 0, 0};
-      if (!kFused && p.mode == 2 && p.csplit > 1) {
+      if (p.mode == 2 && p.csplit > 1) {
         // ---- split-K inside a cluster: partial sums travel through the peers' shared memory ----
         // Finishing is shared out as well: owner f < F completes the tokens of its groups of 8 for the whole tile.
         const int S = p.csplit, rank = static_cast<int>(blockIdx.x) - tile * S;
@@ -811,8 +624,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         // add this CTA's partial sums into the tile's meeting place, then find out whether it was the last contributor
         acc_tile = p.accum + static_cast<long long>(tile) * p.NB * kTileN;
         int c0 = 0;
-        if constexpr (!kFused)
-          for (; c0 + 32 <= p.NB; c0 += 32) partial_chunk<kBase, 32>(t_row, acc_tile, c0, r);
+        for (; c0 + 32 <= p.NB; c0 += 32) partial_chunk<kBase, 32>(t_row, acc_tile, c0, r);
         if (c0 + 16 <= p.NB) partial_chunk<kBase, 16>(t_row, acc_tile, c0, r);
         named_bar_sync(1, 128);
         if (et == 0) {
@@ -839,10 +651,10 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
           named_bar_sync(1, 128);
         }
         if (p.ytype == MSD_OUT_BF16)
-          epilogue_tile<kBase, kFused, true>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h, tok0, tok1, rv,
+          epilogue_tile<kBase, true>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h, tok0, tok1, rv,
                                              m_valid, y_row0);
         else
-          epilogue_tile<kBase, kFused, false>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h, tok0, tok1, rv,
+          epilogue_tile<kBase, false>(p, t_row, acc_tile, r, n, row_ok, sw, s_alpha, s_beta, epi_buf, et, n - r, band_h, tok0, tok1, rv,
                                               m_valid, y_row0);
       }
       tc_fence_before();
@@ -886,12 +698,6 @@ struct GemmW8Plan {
   size_t smem_bytes;
 };
 
-static int env_int(const char* name, int fallback) {
-  const char* e = getenv(name);
-  if (!e || !*e) return fallback;
-  return atoi(e);
-}
-
 // `base`: plan for the dequantize-to-BF16 comparison path (K counted in bytes of BF16, one operand row per token).
 // How many clusters of S CTAs of the GEMM kernel the device can hold at once (cached per configuration); 0 on error.
 static int max_resident_clusters(bool base, int S, size_t smem_bytes);
@@ -904,21 +710,17 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   // K boxes per stage: wide stages read each weight row in runs of kw*128 bytes (good for DRAM page locality);
   // the operand tile of the stacked components grows with kw too, so wide activations get narrower stages.
   int kw = (pl.NB <= 64) ? 4 : 2;
-  kw = env_int("MSD_GEMM_KW", kw);
-  if (kw < 1) kw = 1;
-  if (kw > 8) kw = 8;
   while (kw > 1 && static_cast<int64_t>(kw) * kBlockK > kbytes) kw >>= 1;
   pl.kw = kw;
   pl.kblocks = static_cast<int>((kbytes + static_cast<int64_t>(kw) * kBlockK - 1) / (static_cast<int64_t>(kw) * kBlockK));
   pl.num_tiles = static_cast<int>((N + kTileN - 1) / kTileN);
   pl.total_blocks = static_cast<long long>(pl.kblocks) * pl.num_tiles;
   // Row bands of mode 1 come in two heights that differ by one group.  Groups of 8 rows keep every band on a 16-byte
-  // boundary of y (vector stores); balancing the bands to a single row (MSD_GEMM_GRAN=1) measured no faster.
-  pl.gran = env_int("MSD_GEMM_GRAN", 8);
-  if (pl.gran != 1 && pl.gran != 2 && pl.gran != 4) pl.gran = 8;
+  // boundary of y (vector stores); balancing the bands to a single row measured no faster.
+  pl.gran = 8;
   pl.groups8 = static_cast<int>((N + pl.gran - 1) / pl.gran);
   const int sms = sm_count();
-  int grid = env_int("MSD_GEMM_CTAS", sms);
+  int grid = option(OPT_GEMM_CTAS);       // testing aid: a given number of CTAs
   if (grid < 1) grid = sms;
   if (grid > 256) grid = 256;
   // Row partition pays when every SM gets a band of at least 64 rows (the MMA always spans 128 rows, so shorter
@@ -926,7 +728,7 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
   const int band_max = pl.gran * ((pl.groups8 + grid - 1) / grid);
   const int band_min = pl.gran * (pl.groups8 / grid);
   int mode = (band_min >= 64 && band_max <= kTileN) ? 1 : 0;
-  const int mode_env = env_int("MSD_GEMM_MODE", -1);     // 0 / 1 / 2 force a schedule where it is feasible
+  const int mode_env = option(OPT_GEMM_MODE);            // testing aid: 0 / 1 / 2 force a schedule where it is feasible
   if (mode_env == 0 || mode_env == 1) mode = mode_env;
   if (mode_env == 2) mode = 0;
   if (mode == 1 && (band_max > kTileN || band_min < 8)) mode = 0;
@@ -996,10 +798,9 @@ static GemmW8Plan plan_w8(int64_t M, int64_t N, int64_t K, bool base = false) {
 static bool ensure_smem_attr() {
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(gemm_w8a16_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_w8a16_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_w8a16_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_w8a16_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_w8a16_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w8a16_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w8a16_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
     {
       cudaGetLastError();
       return false;
@@ -1028,8 +829,8 @@ static int max_resident_clusters(bool base, int S, size_t smem_bytes) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   int n = 0;
-  const cudaError_t e = base ? cudaOccupancyMaxActiveClusters(&n, gemm_w8a16_kernel<true, false>, &cfg)
-                             : cudaOccupancyMaxActiveClusters(&n, gemm_w8a16_kernel<false, false>, &cfg);
+  const cudaError_t e = base ? cudaOccupancyMaxActiveClusters(&n, gemm_w8a16_kernel<true>, &cfg)
+                             : cudaOccupancyMaxActiveClusters(&n, gemm_w8a16_kernel<false>, &cfg);
   if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
   if (used < 32) cache[used++] = Entry{base, S, smem_bytes, n};
   return n;
@@ -1115,21 +916,12 @@ msd_status_t msd_gemm_w8a16_ex(const void* x_bf16, const int8_t* w, const float*
   float* alpha = reinterpret_cast<float*>(ws + pl.off_alpha);
   float* beta = reinterpret_cast<float*>(ws + pl.off_beta);
 
-  // Small M: the decomposition runs inside the GEMM kernel.  Otherwise a separate kernel writes the stacked operand:
-  // rows [0, M) hold Q1, rows [Mp, Mp+M) hold Q2; the padding rows are never read back.
-  // Opt-in (MSD_GEMM_FUSED_MAXM=<largest M>): with one quantiser warp per stage the in-kernel path measured no faster
-  // than the two-kernel path at M = 1 and slower from M = 2 on, so the default keeps the separate kernel.
-  const bool fused = (M <= env_int("MSD_GEMM_FUSED_MAXM", 0)) && M <= kFusedMaxM && pl.mode != 2;
-  // Opt-in (MSD_GEMM_INLINE_DEC=1): rows are decomposed inside the GEMM kernel by its first CTAs, the others wait for a
-  // counter - no kernel boundary between a3 and a4.  Measured slower (M = 1: 20.0 vs 17.0 us at K = 4096, 33 vs 20 us
-  // at K = 14336): 128 threads per row and five dependent memory round trips (load, store + fence, counter, poll,
-  // TMA) cost more than the boundary they remove, whatever the weight prefetch depth.
-  const bool inline_dec = !fused && env_int("MSD_GEMM_INLINE_DEC", 0) != 0;
-  if (!fused && !inline_dec) {
-    st = launch_decompose_int8(x_bf16, M, K, K, q, q + static_cast<size_t>(pl.Mp) * K, alpha, beta, scaling_c1(scaling),
-                               scaling_c2(scaling), s);
-    if (st != MSD_OK) return st;
-  }
+  // a1-a3: the decomposition kernel writes the stacked operand: rows [0, M) hold Q1, rows [Mp, Mp+M) hold Q2; the padding
+  // rows are never read back.  (Decomposing inside the GEMM kernel - by extra quantiser warps, or by its first CTAs
+  // behind a counter - was built and measured slower at every M: the row maximum then waits behind the weight prefetch.)
+  st = launch_decompose_int8(x_bf16, M, K, K, q, q + static_cast<size_t>(pl.Mp) * K, alpha, beta, scaling_c1(scaling),
+                             scaling_c2(scaling), s);
+  if (st != MSD_OK) return st;
 
   CUtensorMap tmap_w, tmap_w2, tmap_x;
   const uint32_t box2 = (pl.mode == 1 && pl.hmax > pl.gran) ? pl.hmax - pl.gran : pl.hmax;
@@ -1140,8 +932,8 @@ msd_status_t msd_gemm_w8a16_ex(const void* x_bf16, const int8_t* w, const float*
 
   GemmW8Params p;
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
-  p.kb_rot_step = env_int("MSD_GEMM_KROT", 5);
-  p.pre_stages = env_int("MSD_GEMM_PRE", 64);
+  p.kb_rot_step = 5;
+  p.pre_stages = 64;
   p.mode = pl.mode; p.groups8 = pl.groups8; p.gran = pl.gran; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off; p.csplit = pl.csplit;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
@@ -1151,25 +943,10 @@ msd_status_t msd_gemm_w8a16_ex(const void* x_bf16, const int8_t* w, const float*
   p.status = status;
   p.trace = g_trace;
 
-  p.x = static_cast<const uint16_t*>(x_bf16);
-  p.ldx = K;
-  p.inline_dec = inline_dec ? 1 : 0;
-  p.c1 = scaling_c1(scaling);
-  p.c2 = scaling_c2(scaling);
-  p.dec_ctas = sm_count();
-  p.q = q;
-  p.flags = p.counters + pl.num_tiles;
   if (!ensure_smem_attr()) return MSD_ERR_CUDA;
   GemmW8NoGroups no_groups;
-  if (fused) {
-    // may become resident while earlier work in the stream still runs: it prefetches weights, then waits for that
-    // work to finish before it reads x or touches the split-K workspace
-    if (launch_pdl(gemm_w8a16_kernel<false, true>, dim3(pl.grid), dim3(kFusedThreads), pl.smem_bytes, s, getenv("MSD_NO_PDL") == nullptr, tmap_w, tmap_w2, tmap_x, p, no_groups) != cudaSuccess)
-      return MSD_ERR_CUDA;
-    return MSD_OK;
-  }
-  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  if (launch_pdl_cluster(gemm_w8a16_kernel<false, false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl,
+  const bool pdl = option(OPT_NO_PDL) <= 0;
+  if (launch_pdl_cluster(gemm_w8a16_kernel<false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl,
                          static_cast<unsigned>(pl.csplit), tmap_w, tmap_w2, tmap_x, p, no_groups) != cudaSuccess)
     return MSD_ERR_CUDA;
   return MSD_OK;
@@ -1212,27 +989,25 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = 0;
   p.pre_stages = 64;
-  p.c1 = 127.0f; p.c2 = 254.0f; p.inline_dec = 0; p.dec_ctas = 0; p.q = nullptr; p.flags = nullptr; p.x = nullptr; p.ldx = 0;
   p.mode = pl.mode; p.groups8 = pl.groups8; p.gran = pl.gran; p.hmax = pl.hmax; p.w_chunk_bytes = pl.w_chunk_bytes; p.kw = pl.kw; p.epi_off = pl.epi_off; p.csplit = pl.csplit;
   p.kblocks = pl.kblocks; p.num_tiles = pl.num_tiles; p.total_blocks = pl.total_blocks;
   p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
   p.w_scale = w_scale; p.alpha = nullptr; p.beta = nullptr; p.y = y; p.acc_dbg = nullptr;
-  p.x = nullptr; p.ldx = 0;
   p.accum = reinterpret_cast<int32_t*>(ws + pl.off_slots);
   p.counters = reinterpret_cast<unsigned*>(ws + pl.off_counters);
   p.status = status;
   p.trace = nullptr;
   if (!ensure_smem_attr()) return MSD_ERR_CUDA;
   GemmW8NoGroups no_groups;
-  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
-  if (launch_pdl_cluster(gemm_w8a16_kernel<true, false>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl,
+  const bool pdl = option(OPT_NO_PDL) <= 0;
+  if (launch_pdl_cluster(gemm_w8a16_kernel<true>, dim3(pl.grid), dim3(kGemmThreads), pl.smem_bytes, s, pdl,
                          static_cast<unsigned>(pl.csplit), tmap_w, tmap_w2, tmap_x, p, no_groups) != cudaSuccess)
     return MSD_ERR_CUDA;
   return MSD_OK;
 }
 
 // ---------------------------------------------------------------------------------------------------------------------
-// Grouped W8A16 layer (MoE experts, Sec. 7.2): x rows sorted by expert, group g = rows [off_g, off_g + m_g) against
+// Grouped W8A16 layer (MoE experts; Discussion, "Extension to MoE and Sparse Architectures"): x rows sorted by expert, group g = rows [off_g, off_g + m_g) against
 // expert e_g's weight.  One decomposition launch over all rows, then stream-K launches of up to kMaxGroups non-empty
 // groups each; empty groups cost nothing (their weights are never read).
 struct GroupedPlan {
@@ -1326,9 +1101,8 @@ msd_status_t msd_grouped_gemm_w8a16(const void* x_bf16, const int8_t* w, const f
   p.accum = reinterpret_cast<int32_t*>(ws + gp.off_slots);
   p.counters = reinterpret_cast<unsigned*>(ws + gp.off_counters);
   p.status = status; p.trace = nullptr;
-  p.x = nullptr; p.ldx = 0; p.inline_dec = 0; p.dec_ctas = 0; p.c1 = 127.0f; p.c2 = 254.0f; p.q = q; p.flags = nullptr;
 
-  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+  const bool pdl = option(OPT_NO_PDL) <= 0;
   int e = 0;
   int64_t off = 0;
   while (e < E) {
@@ -1348,7 +1122,7 @@ msd_status_t msd_grouped_gemm_w8a16(const void* x_bf16, const int8_t* w, const f
     p.total_blocks = static_cast<long long>(p.num_tiles) * kblocks;
     int grid = sm_count();
     if (grid > p.total_blocks) grid = static_cast<int>(p.total_blocks);
-    if (launch_pdl(gemm_w8a16_kernel<false, false, true>, dim3(grid), dim3(kGemmThreads), smem_bytes, s, pdl, tmap_w, tmap_w, tmap_x, p, g) !=
+    if (launch_pdl(gemm_w8a16_kernel<false, true>, dim3(grid), dim3(kGemmThreads), smem_bytes, s, pdl, tmap_w, tmap_w, tmap_x, p, g) !=
         cudaSuccess)
       return MSD_ERR_CUDA;
   }

@@ -302,8 +302,8 @@ static GemmP8Plan plan_p8(int64_t M, int64_t N, int64_t K) {
   pl.ksplit = 1;
   pl.kper = pl.kstages;
   {
-    const char* se = getenv("MSD_P8_KSPLIT");
-    long long want = se ? atoi(se) : (2 * tiles <= sm_count() ? sm_count() / tiles : 1);
+    const int forced = option(OPT_P8_KSPLIT);     // testing aid
+    long long want = forced >= 0 ? forced : (2 * tiles <= sm_count() ? sm_count() / tiles : 1);
     if (want > pl.kstages / 8) want = pl.kstages / 8;
     if (want > 1) {
       pl.kper = static_cast<int>((pl.kstages + want - 1) / want);
@@ -351,16 +351,16 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
   CUtensorMap tmap_a1, tmap_a2, tmap_b, tmap_y;
   const bool ybf = !split && ytype == MSD_OUT_BF16;
   // CTA pairs (256 tokens x 256 weight rows per pair, half of the weight tile loaded by each CTA) where there is no K
-  // split; MSD_P8_PAIR=0/1 forces the choice.
+  // split (the option MSD_P8_PAIR forces the choice).
   bool use_pair = false;
   {
-    const char* pe = getenv("MSD_P8_PAIR");
+    const int forced = option(OPT_P8_PAIR);       // testing aid
     const bool can = pl.ksplit == 1 && pl.m_tiles >= 2;
     // where the pair tiles need no more rounds on half as many units (an odd number of token tiles leaves a CTA idle)
     const long long tiles = static_cast<long long>(pl.m_tiles) * pl.n_tiles, pair_tiles = static_cast<long long>((pl.m_tiles + 1) / 2) * pl.n_tiles;
     const long long clusters = sm_count() / 2;
     const bool want = (pair_tiles + clusters - 1) / clusters <= (tiles + sm_count() - 1) / sm_count();
-    use_pair = can && (pe ? atoi(pe) != 0 : want);
+    use_pair = can && (forced >= 0 ? forced != 0 : want);
   }
   if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, K, M, K, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, q2, K, M, K, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
@@ -378,10 +378,9 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
   {
     // A wave of CTAs either shares a few weight tiles and sweeps the token tiles (token tile fastest) or the other way
     // round; the operand that is swept should be the one that stays in L2 (40 MB assumed usable for it).
-    const char* oe = getenv("MSD_P8_ORDER");
     const double l2 = 40.0 * 1024 * 1024, a_bytes = 2.0 * static_cast<double>(M) * K, w_bytes = static_cast<double>(N) * K;
     const bool n_fast = a_bytes <= l2 ? false : (w_bytes <= l2 ? true : a_bytes > w_bytes);
-    p.n_fastest = oe ? (atoi(oe) != 0) : n_fast;
+    p.n_fastest = n_fast;
   }
   const size_t smem_bytes = static_cast<size_t>(kP8Stages) * kP8StageBytes + 16 * kP8StoreBytes + 1024;
   const size_t smem_pair = static_cast<size_t>(kP8PairStages) * kP8PairStageBytes + 16 * kP8StoreBytes + 1024;
@@ -392,7 +391,7 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
       return MSD_ERR_CUDA;
     attr_done = true;
   }
-  const bool pdl = getenv("MSD_NO_PDL") == nullptr;
+  const bool pdl = option(OPT_NO_PDL) <= 0;
   if (use_pair) {
     const long long pair_tiles = static_cast<long long>((pl.m_tiles + 1) / 2) * pl.n_tiles;
     const int clusters = static_cast<int>(pair_tiles < sm_count() / 2 ? pair_tiles : sm_count() / 2);

@@ -14,6 +14,23 @@ unsigned* device_status_ptr();
 
 int sm_count();
 
+// The library's few run-time switches, all testing or diagnostic aids.  Each is read from the environment variable of
+// the same name ONCE, when the first call needs one, and can be set afterwards with msd_debug_set_option(); -1 = unset.
+enum Option {
+  OPT_NO_PDL = 0,           // MSD_NO_PDL: launch dependent kernels without programmatic dependent launch
+  OPT_GEMM_MODE,            // MSD_GEMM_MODE: force a work split of the W8A16 decode kernel (0 stream-K, 1 row bands, 2 clusters)
+  OPT_GEMM_CTAS,            // MSD_GEMM_CTAS: number of CTAs of that kernel
+  OPT_P8_PAIR,              // MSD_P8_PAIR: W8A16 many-row kernel on CTA pairs (1) or single CTAs (0)
+  OPT_P8_KSPLIT,            // MSD_P8_KSPLIT: its K split
+  OPT_W4_PAIR,              // MSD_W4_PAIR: W4A16 kernel on CTA pairs (1) or single CTAs (0)
+  OPT_W4_TILEN,             // MSD_W4_TILEN: tile width of the single-CTA W4A16 kernel (224 or 256)
+  OPT_W4_KSPLIT,            // MSD_W4_KSPLIT: its K split
+  OPT_ATTN_SPLITS,          // MSD_ATTN_SPLITS: number of context splits of the attention kernels
+  OPT_ATTN_CHUNK_TILES,     // MSD_ATTN_CHUNK_TILES: tiles per context split
+  OPT_COUNT
+};
+int option(Option o);
+
 // Encodes a 2-D tiled tensor map: `inner` contiguous elements per row, `outer` rows, rows `row_stride_bytes`
 // apart; the box is box_inner x box_outer elements.  Returns false on failure.
 bool encode_tmap_2d(CUtensorMap* out, CUtensorMapDataType dtype, const void* base, uint64_t inner, uint64_t outer,
@@ -87,7 +104,7 @@ struct SfRelayout {
   int kblocks, sf_kgroups, tile_rows, row_blocks;
   int matrices;        // 0 or 1: one matrix; E > 1: E matrices of `rows` rows back to back (mixture-of-experts
                        // weights), each cut into its own `row_blocks` blocks
-  int blocks;          // filled in by the launcher (returned through the pointer when `ready` is used)
+  int blocks;          // filled in by the launcher
 };
 // Rows sorted by group (mixture of experts): group g owns rows [off[g], off[g+1]) and its decomposition is written as
 // token tile g (rows 128 g ...) of the component and scale buffers.
@@ -98,7 +115,7 @@ struct RowGroups {
 };
 msd_status_t launch_decompose_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q1, uint8_t* q2,
                                     uint8_t* e1, uint8_t* e2, int sf_kgroups, cudaStream_t stream,
-                                    SfRelayout* relayout = nullptr, unsigned* ready = nullptr, const RowGroups* groups = nullptr);
+                                    SfRelayout* relayout = nullptr, const RowGroups* groups = nullptr);
 
 #ifdef __CUDACC__
 // Relayout of row-major E8M0 scales [rows, kblocks] into the 512-byte blocks (128 rows x 4 scales) of the block-scaled

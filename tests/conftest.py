@@ -47,3 +47,4 @@ def _guard_bands(request):
         g.check()
     finally:
         binding._empty, binding._workspace = old
+        binding.debug_reset_options()        # a test may have forced a schedule (msd_debug_set_option)

@@ -92,7 +92,7 @@ def test_other_head_dims():
 
 @pytest.mark.parametrize("splits", ["1", "2", "7"])
 def test_split_counts(splits, monkeypatch):
-    monkeypatch.setenv("MSD_ATTN_SPLITS", splits)
+    binding.debug_set_option("MSD_ATTN_SPLITS", int(splits))
     _check(inputs.gqa_case(2, 8, 2, 128, [1000, 3000], seed=9))
 
 
@@ -122,7 +122,8 @@ def _subcase(c, seqs):
 
 
 def test_gqa_full_size_sampled_sequences():
-    """BASELINE config 3 in the benchmark's launch configuration; the oracle recomputes three sequences."""
+    """The GQA decode workload at full size (batch 32, 32 query / 8 KV heads, d 128, lengths in [2048, 8192]) in the
+    benchmark's launch configuration; the oracle recomputes three sequences."""
     B, Hq, Hkv, D = 32, 32, 8, 128
     c = inputs.gqa_case(B, Hq, Hkv, D, inputs.seqlens_uniform(B, 2048, 8192, seed=0), seed=0)
     o = _run_gpu(c, want_lse=False)
@@ -134,7 +135,7 @@ def test_gqa_full_size_sampled_sequences():
 
 
 def test_mla_full_size_sampled_sequence():
-    """BASELINE config 4 (B=64, 64 heads, d=576/512, 16384 tokens); the oracle recomputes one sequence."""
+    """The MLA-shaped decode workload at full size (B=64, 64 heads, d=576/512, 16384 tokens); the oracle recomputes one sequence."""
     B, Hq, D, Dv, L = 64, 64, 576, 512, 16384
     c = inputs.mla_case(B, Hq, D, Dv, [L] * B, seed=0)
     o = _run_gpu(c, want_lse=False)

@@ -64,7 +64,7 @@ def test_scale_handling_extremes():
 
 
 def test_full_size_sampled():
-    """BASELINE config 2 (M=4096, K=8192, N=8192, BF16 out); the oracle recomputes sampled rows x columns."""
+    """The prefill shape at full size (M=4096, K=8192, N=8192, BF16 out); the oracle recomputes sampled rows x columns."""
     M, N, K = 4096, 8192, 8192
     c = inputs.gemm_w4_case(M, N, K, seed=0)
     y = _run(c, torch.bfloat16)
@@ -81,26 +81,16 @@ def test_full_size_sampled():
 def test_single_cta_and_cta_pair_kernels_agree(pair, monkeypatch):
     """The single-CTA kernel and the CTA-pair kernel (one 256-token tile per pair of CTAs), each forced on every shape,
     including a pair whose second CTA has no rows at all and an odd number of 128-row tiles; both tile widths."""
-    monkeypatch.setenv("MSD_W4_PAIR", pair)
+    binding.debug_set_option("MSD_W4_PAIR", int(pair))
     for (M, N, K) in [(64, 512, 512), (384, 264, 1024), (520, 1032, 768)]:
         c = inputs.gemm_w4_case(M, N, K, seed=7 + M)
         y = _run(c, torch.float32).cpu().numpy().astype(np.float64)
         ref = oracle.gemm_w4a16(c.x, c.w_fp4, c.w_e8m0, "f64")
         _close(y, ref, False)
-        monkeypatch.setenv("MSD_W4_TILEN", "256")
+        binding.debug_set_option("MSD_W4_TILEN", int("256"))
         y = _run(c, torch.float32).cpu().numpy().astype(np.float64)
-        monkeypatch.delenv("MSD_W4_TILEN")
+        binding.debug_set_option("MSD_W4_TILEN", -1)
         _close(y, ref, False)
-
-
-def test_gemm_beside_the_decomposition(monkeypatch):
-    """Opt-in mode in which the GEMM starts while the decomposition kernel is still running and follows its per-tile
-    progress counters: same results, including a ragged last token tile and several tiles per CTA."""
-    monkeypatch.setenv("MSD_W4_OVERLAP", "1")
-    for (M, N, K) in [(1000, 4104, 1024), (130, 256, 512)]:
-        c = inputs.gemm_w4_case(M, N, K, seed=11 + M)
-        y = _run(c, torch.float32).cpu().numpy().astype(np.float64)
-        _close(y, oracle.gemm_w4a16(c.x, c.w_fp4, c.w_e8m0, "f64"), False)
 
 
 @pytest.mark.parametrize("M,N,K", [(16, 448, 4096), (100, 1000, 3072), (1, 232, 8192), (128, 264, 2048)])

@@ -60,7 +60,7 @@ def test_ragged_n_fp32_and_workspace_reuse():
 @pytest.mark.parametrize("ctas", ["1", "3", "37", "148", "200"])
 def test_split_schedules(ctas, monkeypatch):
     """Different CTA counts move the tile/segment boundaries; the integer result must not change."""
-    monkeypatch.setenv("MSD_GEMM_CTAS", ctas)
+    binding.debug_set_option("MSD_GEMM_CTAS", int(ctas))
     _check(inputs.gemm_w8_case(16, 640, 1536, seed=5), torch.float32)
     _check(inputs.gemm_w8_case(128, 256, 768, seed=6), torch.bfloat16)
 
@@ -68,8 +68,8 @@ def test_split_schedules(ctas, monkeypatch):
 @pytest.mark.parametrize("mode,ctas", [("0", "148"), ("1", "148"), ("1", "100"), ("1", "111")])
 def test_row_partition_and_stream_k_agree(mode, ctas, monkeypatch):
     """Tall weights can run either split; band heights (multiples of 8, two sizes) and a ragged last band."""
-    monkeypatch.setenv("MSD_GEMM_MODE", mode)
-    monkeypatch.setenv("MSD_GEMM_CTAS", ctas)
+    binding.debug_set_option("MSD_GEMM_MODE", int(mode))
+    binding.debug_set_option("MSD_GEMM_CTAS", int(ctas))
     _check(inputs.gemm_w8_case(16, 12000, 512, seed=8), torch.float32)
     _check(inputs.gemm_w8_case(128, 10004, 256, seed=9), torch.float32)
 
@@ -79,8 +79,8 @@ def test_cluster_split_k(ctas, monkeypatch):
     """Few weight tiles: a cluster of CTAs per tile splits K and sums the partial tiles through distributed shared
     memory.  The CTA count sets the cluster size (8, 5 / 4, 3 / 2, ...); token counts cover one finishing CTA (M <= 8),
     fewer owners than CTAs, uneven token groups and the full 128; a ragged last tile; both output types."""
-    monkeypatch.setenv("MSD_GEMM_MODE", "2")
-    monkeypatch.setenv("MSD_GEMM_CTAS", ctas)
+    binding.debug_set_option("MSD_GEMM_MODE", int("2"))
+    binding.debug_set_option("MSD_GEMM_CTAS", int(ctas))
     _check(inputs.gemm_w8_case(3, 640, 4096, seed=21), torch.float32)
     _check(inputs.gemm_w8_case(24, 1000, 4096 + 16, seed=22), torch.bfloat16)
     _check(inputs.gemm_w8_case(128, 512, 6144, seed=23), torch.float32)
@@ -88,7 +88,7 @@ def test_cluster_split_k(ctas, monkeypatch):
 
 
 def test_cluster_split_k_comparison_kernel(monkeypatch):
-    monkeypatch.setenv("MSD_GEMM_MODE", "2")
+    binding.debug_set_option("MSD_GEMM_MODE", int("2"))
     c = inputs.gemm_w8_case(40, 512, 4096, seed=25)
     y = binding.gemm_dequant_bf16(bf16_dev(c.x), dev(c.w), dev(c.w_scale), out_dtype=torch.float32)
     torch.cuda.synchronize()
@@ -97,11 +97,9 @@ def test_cluster_split_k_comparison_kernel(monkeypatch):
     assert rel_row_err(y.cpu().numpy(), ref).max() <= TOL
 
 
-@pytest.mark.parametrize("inline", ["0", "1"])
-def test_fractional_scaling_layer(inline, monkeypatch):
+def test_fractional_scaling_layer():
     """msd_gemm_w8a16_ex with the scaling constants of Sec. 3.3 (127.49 / 254.98): accumulators bit-exact against the
-    oracle run with the same constants, through the separate decomposition kernel and the in-kernel one."""
-    monkeypatch.setenv("MSD_GEMM_INLINE_DEC", inline)
+    oracle run with the same constants."""
     for (M, N, K, seed) in [(5, 384, 272, 51), (16, 4096, 4096, 52), (128, 512, 1024, 53)]:
         c = inputs.gemm_w8_case(M, N, K, seed=seed)
         y, acc = binding.gemm_w8a16(bf16_dev(c.x), dev(c.w), dev(c.w_scale), out_dtype=torch.float32, want_acc=True, fractional=True)
@@ -114,35 +112,15 @@ def test_fractional_scaling_layer(inline, monkeypatch):
         assert not np.array_equal(oacc, dacc)
 
 
-def test_rows_decomposed_by_the_gemm_kernels_first_ctas(monkeypatch):
-    """Opt-in: no separate decomposition kernel; the first CTAs of the GEMM decompose the rows and a counter in the
-    workspace releases the others.  Same bits; repeated calls on one workspace check that the counters return to zero;
-    more rows than CTAs, and more CTAs than SMs."""
-    monkeypatch.setenv("MSD_GEMM_INLINE_DEC", "1")
-    c = inputs.gemm_w8_case(16, 640, 1536, seed=41)
-    ws = binding.workspace(binding.gemm_w8a16_workspace_bytes(16, 640, 1536))
-    for _ in range(3):
-        _check(c, torch.float32, ws)
-    _check(inputs.gemm_w8_case(128, 512, 6144, seed=42), torch.bfloat16)
-    _check(inputs.gemm_w8_case(1, 14336, 4096, seed=43), torch.float32)
-    monkeypatch.setenv("MSD_GEMM_CTAS", "3")
-    _check(inputs.gemm_w8_case(40, 256, 768, seed=44), torch.float32)
-    monkeypatch.setenv("MSD_GEMM_CTAS", "200")
-    _check(inputs.gemm_w8_case(33, 1152, 2048, seed=45), torch.float32)
-
-
-@pytest.mark.parametrize("fused", ["0", "8"])
-def test_small_m_with_and_without_in_kernel_decomposition(fused, monkeypatch):
-    """M <= 8 can decompose the activations inside the GEMM kernel (opt-in); it must agree with the two-kernel path
-    and the oracle bit for bit."""
-    monkeypatch.setenv("MSD_GEMM_FUSED_MAXM", fused)
+def test_small_m_shapes():
+    """M <= 8: one weight band per CTA, a ragged last band, K not a multiple of the stage width; bit for bit."""
     _check(inputs.gemm_w8_case(1, 1152, 2048, seed=11), torch.float32)
     _check(inputs.gemm_w8_case(8, 12000, 528, seed=12), torch.float32)
     _check(inputs.gemm_w8_case(3, 640, 1536 + 16, seed=13), torch.bfloat16)
 
 
 def test_without_programmatic_dependent_launch(monkeypatch):
-    monkeypatch.setenv("MSD_NO_PDL", "1")
+    binding.debug_set_option("MSD_NO_PDL", int("1"))
     _check(inputs.gemm_w8_case(16, 1024, 1024, seed=7), torch.float32)
 
 
@@ -188,7 +166,7 @@ def test_host_buffer_entry_point():
 def test_dequant_bf16_comparison_kernel(M, N, K, ctas, monkeypatch):
     """The path MSD replaces: bf16(s_W * w) written back, then a BF16 x BF16 GEMM with FP32 accumulation."""
     if ctas:
-        monkeypatch.setenv("MSD_GEMM_CTAS", ctas)
+        binding.debug_set_option("MSD_GEMM_CTAS", int(ctas))
     c = inputs.gemm_w8_case(M, N, K, seed=4)
     y = binding.gemm_dequant_bf16(bf16_dev(c.x), dev(c.w), dev(c.w_scale), out_dtype=torch.float32)
     torch.cuda.synchronize()
@@ -259,7 +237,7 @@ def test_prefill_single_cta_and_cta_pair_kernels(pair, M, N, K, monkeypatch):
     """The many-row kernel as single CTAs and as CTA pairs (256 tokens per pair of CTAs), each forced on every shape: a
     pair whose second CTA has a single row or none, an odd number of 128-row tiles, ragged weight tiles, several tiles per
     pair; INT32 accumulators bit-exact in both, FP32 and BF16 outputs."""
-    monkeypatch.setenv("MSD_P8_PAIR", pair)
+    binding.debug_set_option("MSD_P8_PAIR", int(pair))
     c = inputs.gemm_w8_case(M, N, K, seed=11)
     _check(c, torch.float32)
     _check(c, torch.bfloat16)

@@ -35,7 +35,7 @@ def test_theorem1_bound_and_ranges(outliers):
     assert ratio.max() > 0.9                      # and the bound is nearly attained
     r1 = np.abs(x - a.astype(np.float64)[:, None] * q1).max(axis=1)
     assert np.all(r1 <= a.astype(np.float64) / 2 * (1 + 1e-4))   # slack: FP32 rounding of the quotient near a tie
-    # zero clipping: both passes stay inside [-127, 127] (Sec. 7.2)
+    # zero clipping: both passes stay inside [-127, 127] (Discussion, "Clipping vs. Zero-Clipping Trade-off")
     assert q1.min() >= -127 and q1.max() <= 127 and q2.min() >= -127 and q2.max() <= 127
     # the row maximum maps to +-127 (Sec. 3.3 "the extremal element satisfies |x/alpha| = 127 exactly")
     assert np.all(np.abs(q1).max(axis=1) == 127)
