@@ -660,6 +660,14 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
   __shared__ float red[kWideSlots / kWideHS][4][kWideHS + 1];    // per-warp tile maxima (slow path only)
   constexpr int kWideWG = kWideSlots / kWideHS;
   constexpr int kNSW = 4 * kWideWG;
+  // Latent cache of 576 bytes per token with V aliased to its first 512 (the launcher picks this instantiation only
+  // then): the two KV stages are given back chunk by chunk (five 128-byte-wide chunks of 16 KB): every chunk is
+  // requested again as soon as its last reader is done - the rotary chunk after QK^T, value chunk j after the j-th
+  // 128-wide tile of PV - instead of the whole 80 KB stage waiting for the last PV MMA.  (Starting QK^T on a tile's
+  // first chunks while the others are in flight was measured too: five short bursts of MMAs cost the issuing thread
+  // far more than one long one.)
+  constexpr bool kChunked = kFixDC == 5 && kFixDVT == 4 && !kPaged;
+  __shared__ __align__(8) uint64_t ck_empty[2][5];
   constexpr int kDVT = 4;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -707,6 +715,9 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
     mbar_init(&p_full[0], kNSW); mbar_init(&p_full[1], kNSW);
     mbar_init(&q_ready, 1);
     mbar_init(&o_full, 1); mbar_init(&o_last, 1); mbar_init(&p_redo, kNSW);
+    if constexpr (kChunked)
+      for (int s2 = 0; s2 < 2; ++s2)
+        for (int c = 0; c < 5; ++c) mbar_init(&ck_empty[s2][c], 1);
     abort_flag = 0;
     flush_stamp[0] = 0; flush_stamp[1] = 0;
     mbar_init_fence();
@@ -727,6 +738,24 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
     if (lane == 0) {
       const int k_bytes = p.DC * kChunkBytes, v_bytes = p.DVT * kChunkBytes;
       int kq = 0, vq = p.v_alias ? ntiles : 0;
+      if constexpr (kChunked) {
+        bool okp = true;
+        for (; kq < ntiles && okp; ++kq) {
+          const int st = kq & 1;
+          const uint32_t ph = (kq >> 1) & 1;
+          uint8_t* dst = smem + st * kv_stage_bytes;
+          const int tok0 = seq0 + t_begin + kq * kTok;
+          if (kq >= 2 && kq < 5) attn_mark(p, 9 + 6 * (kq - 2));
+#pragma unroll
+          for (int i = 0; i < 5; ++i) {
+            const int c = (i == 0) ? 4 : i - 1;
+            okp = wait_bounded(&ck_empty[st][c], ph ^ 1, abort, p.status);
+            if (!okp) break;
+            if (i == 0) mbar_arrive_expect_tx(&kv_full[st], 5 * kChunkBytes);
+            tma_load_3d(dst + c * kChunkBytes, &tmap_k, c * kChunk, hk, tok0, &kv_full[st]);
+          }
+        }
+      }
       long long t_idle = clock64();
       while (kq < ntiles || vq < ntiles) {
         bool progressed = false;
@@ -832,7 +861,8 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
           }
         }
         tc_commit(&s_full[t & 1]);
-        if (!p.v_alias) tc_commit(&kv_empty[st]);       // separate V: the K buffer is free once QK^T has read it
+        if constexpr (kChunked) tc_commit(&ck_empty[st][4]);       // the rotary chunk has no other reader
+        else if (!p.v_alias) tc_commit(&kv_empty[st]);       // separate V: the K buffer is free once QK^T has read it
       };
       // PV of tile t, added to what the accumulators hold unless `fresh`
       auto issue_pv = [&](int t, bool fresh) {
@@ -844,11 +874,13 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
         const uint32_t acc0 = fresh ? 0u : 1u;
         if constexpr (kFixDVT > 0) {
 #pragma unroll
-          for (int j = 0; j < kFixDVT; ++j)
+          for (int j = 0; j < kFixDVT; ++j) {
 #pragma unroll
             for (int k = 0; k < 4; ++k)      // 32 tokens per MMA: four 8-token groups of 1024 bytes
               mma_i8(tmem_o + j * (2 * kWideSlots), va + (j * (kChunkBytes >> 4) + k * (4096 >> 4)), pa + k * (2048 >> 4), idesc_pv,
                      k > 0 ? 1u : acc0);
+            if constexpr (kChunked) tc_commit(&ck_empty[st][j]);      // value chunk j may be requested again
+          }
         } else {
           uint64_t vc = va;
           uint32_t d = tmem_o;
@@ -862,7 +894,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
         // o_full counts every PV product (a drain in mid-split waits for the one before its tile: at that point the
         // barrier is at most one phase behind, so a parity test is unambiguous); the last one has a barrier of its own
         tc_commit(t == ntiles - 1 ? &o_last : &o_full);
-        tc_commit(p.v_alias ? &kv_empty[st] : &v_empty[st]);
+        if constexpr (!kChunked) tc_commit(p.v_alias ? &kv_empty[st] : &v_empty[st]);
       };
       // QK^T(q) needs KV tile q in shared memory and the score buffer q&1 read (P of tile q-2 final);
       // PV(v) needs P of tile v final (written, and rewritten when the references had to move) and QK^T(v) issued.
@@ -1399,7 +1431,7 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
     MSD_ATTN_PICK(16, 16);
   } else {
     // wide head groups: 32 head slots per CTA, sixteen softmax warps, held references (attn_decode_wide_kernel)
-    const bool mla = pl.DC == 5 && pl.DVT == 4;        // a 576-byte latent row with 512 value bytes
+    const bool mla = pl.DC == 5 && pl.DVT == 4 && pl.v_alias && pl.stages == 2;     // a 513..640-byte latent row whose first 512 bytes are V
     if (paged) kernel = mla ? attn_decode_wide_kernel<8, true, 5, 4> : attn_decode_wide_kernel<8, true, 0, 0>;
     else kernel = mla ? attn_decode_wide_kernel<8, false, 5, 4> : attn_decode_wide_kernel<8, false, 0, 0>;
     block_threads = 64 + 128 * 4;
