@@ -27,6 +27,7 @@ constexpr int kTok = 128;           // tokens per tile
 constexpr int kAttnThreads = 192;
 constexpr int kChunk = 128;         // bytes of D / Dv per TMA box and per shared-memory operand chunk
 constexpr int kChunkBytes = kTok * kChunk;
+constexpr int kPartHdr = 4;         // words in front of a split's partial output row: reference maximum, sum of P, two unused
 
 struct AttnParams {
   const uint16_t* q;      // [B,Hq,D] BF16 (read by attn_qstack_kernel only)
@@ -42,7 +43,7 @@ struct AttnParams {
   const int32_t* block_table;
   const int32_t* seqlens; // [B] (paged only)
   int page, page_shift, max_blocks;
-  float* partial;         // [B,Hq,n_splits,Dv+2]: m, l, O[Dv]
+  float* partial;         // [B,Hq,n_splits,4+Dv]: m, l, two unused words (O starts on a 16-byte boundary), O[Dv]
   int B, Hq, Hkv, D, Dv, G;   // with several query tokens per sequence Hq and G count (token, head) rows: Sq * real values
   // Speculative / multi-token decode (Sec. 4.4): Sq query tokens per sequence, the last Sq tokens of its cache.  The
   // Sq * Gr rows that share a KV head are laid out token-major: row r of a KV head = (token r / Gr, head r % Gr);
@@ -163,7 +164,7 @@ __device__ __forceinline__ void attn_dump_scores(const AttnParams& p, long long 
 // the group's heads are decomposed into two INT8 components (same bit-exact rule as msd_decompose_int8) and written
 // as the stacked operand image the attention CTAs copy into shared memory with one bulk copy per chunk.  One CTA per
 // unit, one warp per head round robin.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 attn_qstack_kernel(const AttnParams p, uint8_t* __restrict__ q_img, float* __restrict__ q_scales) {
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -179,7 +180,7 @@ attn_qstack_kernel(const AttnParams p, uint8_t* __restrict__ q_img, float* __res
   for (int i = threadIdx.x; i < img_bytes / 16; i += blockDim.x) reinterpret_cast<uint4*>(img)[i] = make_uint4(0, 0, 0, 0);
   for (int i = threadIdx.x; i < 2 * p.HG; i += blockDim.x) sc[i] = 0.0f;
   __syncthreads();
-  for (int h = warp; h < nh; h += 8) attn_decompose_q_row(p, b, hk, grp, h, lane, img, sc + h, sc + p.HG + h);
+  for (int h = warp; h < nh; h += static_cast<int>(blockDim.x >> 5)) attn_decompose_q_row(p, b, hk, grp, h, lane, img, sc + h, sc + p.HG + h);
 }
 
 // Head groups of up to 16 query rows per KV head (GQA).  kMaxHG: head slots one softmax thread looks after (8 or 16);
@@ -222,9 +223,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   }
 
   if (ntiles == 0) {      // nothing in this split: neutral partials, before any barrier or TMEM use
-    for (int i = threadIdx.x; i < nh * (p.Dv + 2); i += blockDim.x) {
-      const int h = i / (p.Dv + 2), e = i % (p.Dv + 2);
-      float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + h) * p.n_splits + split) * (p.Dv + 2);
+    for (int i = threadIdx.x; i < nh * (p.Dv + kPartHdr); i += blockDim.x) {
+      const int h = i / (p.Dv + kPartHdr), e = i % (p.Dv + kPartHdr);
+      float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + h) * p.n_splits + split) * (p.Dv + kPartHdr);
       dst[e] = (e == 0) ? -INFINITY : 0.0f;
     }
     return;
@@ -597,12 +598,12 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
       for (int h = 0; h < kNH; ++h) {
         if (hs0 + h < nh) {
-          float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + hs0 + h) * p.n_splits + split) * (p.Dv + 2);
+          float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + hs0 + h) * p.n_splits + split) * (p.Dv + kPartHdr);
           // the running maximum goes out in natural-log units (it was kept in the log2 domain)
           if (tl == 0) { dst[0] = m_run[h] * 0.6931471805599453f; dst[1] = rb[0][h] + rb[1][h] + rb[2][h] + rb[3][h]; }
 #pragma unroll
           for (int j = 0; j < kMaxDVT; ++j)
-            if (j < p.DVT && j * kChunk + tl < p.Dv) dst[2 + j * kChunk + tl] = o_run[j][h];
+            if (j < p.DVT && j * kChunk + tl < p.Dv) dst[kPartHdr + j * kChunk + tl] = o_run[j][h];
         }
       }
     }
@@ -693,9 +694,9 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
   }
 
   if (ntiles == 0) {      // nothing in this split: neutral partials, before any barrier or TMEM use
-    for (int i = threadIdx.x; i < nh * (p.Dv + 2); i += blockDim.x) {
-      const int h = i / (p.Dv + 2), e = i % (p.Dv + 2);
-      float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + h) * p.n_splits + split) * (p.Dv + 2);
+    for (int i = threadIdx.x; i < nh * (p.Dv + kPartHdr); i += blockDim.x) {
+      const int h = i / (p.Dv + kPartHdr), e = i % (p.Dv + kPartHdr);
+      float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + h) * p.n_splits + split) * (p.Dv + kPartHdr);
       dst[e] = (e == 0) ? -INFINITY : 0.0f;
     }
     return;
@@ -1188,7 +1189,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
 #pragma unroll
       for (int h = 0; h < kWideHS; ++h) {
         if (hs0 + h < nh) {
-          float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + hs0 + h) * p.n_splits + split) * (p.Dv + 2);
+          float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + hs0 + h) * p.n_splits + split) * (p.Dv + kPartHdr);
           if (tl == 0) {
             // the reference goes out in natural-log units (it was kept in the log2 domain); -inf: no visible token
             dst[0] = (nm[h] == 1e30f) ? -INFINITY : -nm[h] * 0.6931471805599453f;
@@ -1205,7 +1206,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
 #pragma unroll
           for (int h = 0; h < kWideHS; ++h)
             if (hs0 + h < nh && j * kChunk + tl < p.Dv)
-              p.partial[((static_cast<long long>(b) * p.Hq + h0 + hs0 + h) * p.n_splits + split) * (p.Dv + 2) + 2 + j * kChunk + tl] =
+              p.partial[((static_cast<long long>(b) * p.Hq + h0 + hs0 + h) * p.n_splits + split) * (p.Dv + kPartHdr) + kPartHdr + j * kChunk + tl] =
                   __uint_as_float(o[h]);
         }
       }
@@ -1227,11 +1228,17 @@ static float* g_attn_qs_dbg = nullptr;
 static int32_t* g_attn_s_dbg = nullptr;
 
 // c8: merge the splits of one (sequence, query head) and normalise:  O = sum_s e^{m_s - m} O_s / sum_s e^{m_s - m} l_s
-// (a separate small kernel: letting the last-arriving split do it inside the attention kernel measured slower)
+// (a separate small kernel: letting the last-arriving split do it inside the attention kernel measured slower).
+// One CTA per row; the weights e^{m_s - m} are computed once per split and the O_s rows are read as 16-byte vectors,
+// eight splits' loads in flight per thread.  O is summed over the splits in ascending order.
 __global__ void __launch_bounds__(128)
 attn_combine_kernel(const float* __restrict__ partial, int n_splits, int Dv, __nv_bfloat16* __restrict__ out,
                     float* __restrict__ lse, int Sq, int Gr, int Hkv) {
-  const float* base = partial + static_cast<long long>(blockIdx.x) * n_splits * (Dv + 2);
+  __shared__ float s_w[128];
+  __shared__ float s_red[2][4];
+  pdl_wait_primary();              // the partial results come from the attention kernel launched just before
+  const int PS = Dv + kPartHdr;
+  const float* base = partial + static_cast<long long>(blockIdx.x) * n_splits * PS;
   // partial rows are [B][KV head][query token][head of the group]; the output is [B][query token][head]
   long long row = blockIdx.x;
   if (Sq > 1) {
@@ -1240,22 +1247,54 @@ attn_combine_kernel(const float* __restrict__ partial, int n_splits, int Dv, __n
     const int v = static_cast<int>(row - bq * per_seq), hk = v / per_kv, r = v - hk * per_kv, sq = r / Gr;
     row = (bq * Sq + sq) * (Hkv * Gr) + hk * Gr + (r - sq * Gr);
   }
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   float m = -INFINITY;
-  for (int s = 0; s < n_splits; ++s) m = fmaxf(m, base[s * (Dv + 2)]);
-  float l = 0.0f;
-  for (int s = 0; s < n_splits; ++s) {
-    const float ms = base[s * (Dv + 2)];
-    if (ms != -INFINITY) l += expf(ms - m) * base[s * (Dv + 2) + 1];
-  }
-  for (int d = threadIdx.x; d < Dv; d += blockDim.x) {
-    float acc = 0.0f;
-    for (int s = 0; s < n_splits; ++s) {
-      const float ms = base[s * (Dv + 2)];
-      if (ms != -INFINITY) acc += expf(ms - m) * base[s * (Dv + 2) + 2 + d];
+  for (int s = tid; s < n_splits; s += 128) m = fmaxf(m, __ldg(base + static_cast<long long>(s) * PS));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if (lane == 0) s_red[0][warp] = m;
+  __syncthreads();
+  m = fmaxf(fmaxf(s_red[0][0], s_red[0][1]), fmaxf(s_red[0][2], s_red[0][3]));
+  const bool act = tid < (Dv >> 2);
+  const float4* o4 = reinterpret_cast<const float4*>(base + kPartHdr) + tid;
+  const int ps4 = PS >> 2;
+  float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+  float l = 0.0f;                  // this thread's share of the normaliser: the splits s with s % 128 == tid
+  for (int s0 = 0; s0 < n_splits; s0 += 128) {
+    float w = 0.0f;
+    if (s0 + tid < n_splits) {
+      const float2 ml = __ldg(reinterpret_cast<const float2*>(base + static_cast<long long>(s0 + tid) * PS));
+      if (ml.x != -INFINITY) { w = expf(ml.x - m); l += w * ml.y; }
     }
-    out[row * Dv + d] = __float2bfloat16_rn(l > 0.0f ? acc / l : 0.0f);
+    __syncthreads();               // the previous chunk's weights have been used
+    s_w[tid] = w;
+    __syncthreads();
+    const int n = min(128, n_splits - s0);
+    if (act) {
+      const float4* q = o4 + static_cast<long long>(s0) * ps4;
+#pragma unroll 8
+      for (int i = 0; i < n; ++i) {
+        const float4 v = __ldg(q + static_cast<long long>(i) * ps4);
+        const float wi = s_w[i];
+        acc.x += wi * v.x; acc.y += wi * v.y; acc.z += wi * v.z; acc.w += wi * v.w;
+      }
+    }
   }
-  if (lse && threadIdx.x == 0) lse[row] = (l > 0.0f) ? m + logf(l) : -INFINITY;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+  if (lane == 0) s_red[1][warp] = l;
+  __syncthreads();
+  l = (s_red[1][0] + s_red[1][1]) + (s_red[1][2] + s_red[1][3]);
+  if (act) {
+    const float o0 = l > 0.0f ? acc.x / l : 0.0f, o1 = l > 0.0f ? acc.y / l : 0.0f;
+    const float o2 = l > 0.0f ? acc.z / l : 0.0f, o3 = l > 0.0f ? acc.w / l : 0.0f;
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(o0, o1), hi = __floats2bfloat162_rn(o2, o3);
+    uint2 pk;
+    pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(out + row * Dv + 4 * tid) = pk;
+  }
+  if (lse && tid == 0) lse[row] = (l > 0.0f) ? m + logf(l) : -INFINITY;
 }
 
 struct AttnPlan {
@@ -1303,7 +1342,7 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   const int cols_needed = pl->HG > 16 ? 2 * pl->Rp + 4 * pl->Rp + 4 * 32 : 2 * pl->Rp + pl->DVT * pl->Rp;
   while (cols < cols_needed) cols <<= 1;
   pl->tmem_cols = cols;
-  pl->ws_partial_bytes = round_up(static_cast<size_t>(B) * Hq * ns * (Dv + 2) * sizeof(float), 1024);
+  pl->ws_partial_bytes = round_up(static_cast<size_t>(B) * Hq * ns * (Dv + kPartHdr) * sizeof(float), 1024);
   pl->ws_qimg_bytes = round_up(static_cast<size_t>(units) * pl->DC * pl->Rp * kChunk, 1024);     // stacked Q operands
   pl->ws_qscale_bytes = round_up(static_cast<size_t>(units) * 2 * pl->HG * sizeof(float), 1024);
   pl->ws_bytes = pl->ws_partial_bytes + round_up(static_cast<size_t>(units) * sizeof(unsigned), 1024) + pl->ws_qimg_bytes + pl->ws_qscale_bytes;
@@ -1457,7 +1496,7 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
   if (block_threads > kAttnThreads) {
     // wide head groups: the stacked Q operands come from a kernel of their own, the attention kernel is its
     // programmatic dependent (its CTAs start their KV loads while it runs)
-    attn_qstack_kernel<<<B * Hkv * pl.groups, 256, 0, s>>>(p, q_img, q_scales);
+    attn_qstack_kernel<<<B * Hkv * pl.groups, 32 * pl.HG, 0, s>>>(p, q_img, q_scales);
     if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
     if (launch_pdl(kernel, grid, dim3(block_threads), pl.smem_bytes, s, option(OPT_NO_PDL) <= 0, tmap_k, tmap_v, p) != cudaSuccess)
       return MSD_ERR_CUDA;
@@ -1465,8 +1504,9 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
     kernel<<<grid, block_threads, pl.smem_bytes, s>>>(tmap_k, tmap_v, p);
     if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
   }
-  attn_combine_kernel<<<B * Hq, 128, 0, s>>>(p.partial, pl.n_splits, Dv, static_cast<__nv_bfloat16*>(out_bf16), lse, q_len,
-                                             Hq / (Hkv * q_len), Hkv);
+  if (launch_pdl(attn_combine_kernel, dim3(B * Hq), dim3(128), 0, s, option(OPT_NO_PDL) <= 0, static_cast<const float*>(p.partial),
+                 pl.n_splits, Dv, static_cast<__nv_bfloat16*>(out_bf16), lse, q_len, Hq / (Hkv * q_len), Hkv) != cudaSuccess)
+    return MSD_ERR_CUDA;
   return launch_status();
 }
 
