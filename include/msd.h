@@ -223,6 +223,29 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
                                     msd_out_t ytype, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Weight scales prepared once.  The block-scaled MMA (Sec. 3.2.1 / Sec. 3.8.3: two FP4 GEMMs with E8M0 block scales)
+ * reads the scales of a weight tile as 512-byte blocks of 128 rows x 4 K blocks; msd_gemm_w4a16 and
+ * msd_grouped_gemm_w4a16 bring the row-major w_e8m0 into that form on every call.  Weights do not change between calls,
+ * so the relayout can be done when they are loaded:
+ *   msd_prepare_w4a16_scales: w_e8m0 [E, N, K/32] (device, 4-byte aligned; E = 1 for one matrix) -> prepared (device,
+ *     1024-byte aligned, >= msd_w4a16_prepared_scales_bytes(E, N, K) bytes, owned by the caller): the blocked scales
+ *     for both tile widths the kernels use, about twice the size of w_e8m0.  Launches on `stream`, does not synchronise.
+ *   msd_gemm_w4a16_prepared / msd_grouped_gemm_w4a16_prepared: as the entry points above with `prepared_scales` in the
+ *     place of w_e8m0 (same N, K and, for the grouped call, the same E as at preparation); results are bit-identical
+ *     to theirs.  Same status codes; a null `prepared_scales` -> MSD_ERR_NULL_POINTER, not 1024-byte aligned ->
+ *     MSD_ERR_BAD_ALIGNMENT.
+ */
+size_t msd_w4a16_prepared_scales_bytes(int32_t E, int64_t N, int64_t K);
+msd_status_t msd_prepare_w4a16_scales(const uint8_t* w_e8m0, int32_t E, int64_t N, int64_t K, uint8_t* prepared,
+                                      void* stream);
+msd_status_t msd_gemm_w4a16_prepared(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* prepared_scales, int64_t M,
+                                     int64_t N, int64_t K, void* y, msd_out_t ytype, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+msd_status_t msd_grouped_gemm_w4a16_prepared(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* prepared_scales,
+                                             const int32_t* group_sizes_host, int32_t E, int64_t N, int64_t K, void* y,
+                                             msd_out_t ytype, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The paper-literal MXFP4 components (Sec. 3.2.1, Alg. 2; Tab. mxfp4-evolution): both passes round onto the E1M2 grid
  * {0, .25, ..., 1.75}, alpha = 2^ceil(log2(blockmax / 1.859375)) (exponent kept >= -123), beta = alpha / 16, error bound
  * alpha / 64.  Tensor cores have no E1M2 operand type; every E1M2 value is an E4M3 number, so the components are

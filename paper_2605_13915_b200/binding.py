@@ -50,6 +50,10 @@ _SIGS = {
     "msd_gemm_dequant_bf16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_gemm_w4a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_w4a16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
+    "msd_w4a16_prepared_scales_bytes": (_sz, [_i32, _i64, _i64]),
+    "msd_prepare_w4a16_scales": (C.c_int, [_vp, _i32, _i64, _i64, _vp, _vp]),
+    "msd_gemm_w4a16_prepared": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
+    "msd_grouped_gemm_w4a16_prepared": (C.c_int, [_vp, _vp, _vp, _vp, _i32, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_attn_decode_int8kv_workspace_bytes": (_sz, [_i32] * 6),
     "msd_attn_decode_int8kv": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp,
                                          _vp, _sz, _vp]),
@@ -210,10 +214,11 @@ def grouped_gemm_w8a16(x, w, w_scale, group_sizes, out_dtype=torch.bfloat16, ws=
     return y
 
 
-def grouped_gemm_w4a16(x, w_fp4, w_e8m0, group_sizes, out_dtype=torch.bfloat16, ws=None, out=None):
+def grouped_gemm_w4a16(x, w_fp4, w_e8m0, group_sizes, out_dtype=torch.bfloat16, ws=None, out=None, prepared=None):
     """MoE experts with MXFP4 weights: x [M_total,K] bf16 with rows sorted by expert, w_fp4 [E,N,K/2] u8, w_e8m0 [E,N,K/32] u8,
-    group_sizes: E host ints (rows per expert, each <= 128) -> y [M_total,N]."""
-    _need_cuda(x, w_fp4, w_e8m0)
+    group_sizes: E host ints (rows per expert, each <= 128) -> y [M_total,N].
+    prepared: the result of prepare_w4a16_scales(w_e8m0); w_e8m0 may then be None."""
+    _need_cuda(x, w_fp4, prepared if prepared is not None else w_e8m0)
     E, N, K2 = w_fp4.shape
     K = 2 * K2
     sizes = (C.c_int32 * E)(*[int(v) for v in group_sizes])
@@ -223,8 +228,12 @@ def grouped_gemm_w4a16(x, w_fp4, w_e8m0, group_sizes, out_dtype=torch.bfloat16, 
         ws = workspace(int(lib().msd_grouped_gemm_w4a16_workspace_bytes(E, N, K)), x.device)
     y = out if out is not None else _empty((M_total, N), out_dtype, x.device)
     wp, wb = _ws_ptr(ws)
-    code = lib().msd_grouped_gemm_w4a16(_ptr(x), _ptr(w_fp4), _ptr(w_e8m0), sizes, E, N, K, _ptr(y),
-                                        OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream())
+    if prepared is not None:
+        code = lib().msd_grouped_gemm_w4a16_prepared(_ptr(x), _ptr(w_fp4), _ptr(prepared), sizes, E, N, K, _ptr(y),
+                                                     OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream())
+    else:
+        code = lib().msd_grouped_gemm_w4a16(_ptr(x), _ptr(w_fp4), _ptr(w_e8m0), sizes, E, N, K, _ptr(y),
+                                            OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream())
     _check(code, "msd_grouped_gemm_w4a16")
     return y
 
@@ -278,16 +287,36 @@ def gemm_w4a16_workspace_bytes(M, N, K):
     return int(lib().msd_gemm_w4a16_workspace_bytes(M, N, K))
 
 
-def gemm_w4a16(x, w_fp4, w_e8m0, out_dtype=torch.bfloat16, ws=None, out=None):
-    _need_cuda(x, w_fp4, w_e8m0)
+def prepare_w4a16_scales(w_e8m0):
+    """Blocked form of the E8M0 weight scales [N,K/32] (or [E,N,K/32]), made once per weight; pass it as `prepared`."""
+    _need_cuda(w_e8m0)
+    E = w_e8m0.shape[0] if w_e8m0.dim() == 3 else 1
+    N, KB = w_e8m0.shape[-2], w_e8m0.shape[-1]
+    nbytes = int(lib().msd_w4a16_prepared_scales_bytes(E, N, 32 * KB))
+    if nbytes == 0:
+        raise ValueError("msd_w4a16_prepared_scales_bytes: unsupported shape")
+    buf = workspace(nbytes + 1024, w_e8m0.device)
+    off = (-buf.data_ptr()) % 1024
+    prepared = buf[off:off + nbytes]          # a view that starts on a 1024-byte boundary
+    _check(lib().msd_prepare_w4a16_scales(_ptr(w_e8m0), E, N, 32 * KB, _ptr(prepared), _stream()), "msd_prepare_w4a16_scales")
+    return prepared
+
+
+def gemm_w4a16(x, w_fp4, w_e8m0, out_dtype=torch.bfloat16, ws=None, out=None, prepared=None):
+    """prepared: the result of prepare_w4a16_scales(w_e8m0); w_e8m0 may then be None."""
+    _need_cuda(x, w_fp4, prepared if prepared is not None else w_e8m0)
     M, K = x.shape
     N = w_fp4.shape[0]
     if ws is None:
         ws = workspace(gemm_w4a16_workspace_bytes(M, N, K), x.device)
     y = out if out is not None else _empty((M, N), out_dtype, x.device)
     wp, wb = _ws_ptr(ws)
-    _check(lib().msd_gemm_w4a16(_ptr(x), _ptr(w_fp4), _ptr(w_e8m0), M, N, K, _ptr(y),
-                                OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream()), "msd_gemm_w4a16")
+    yt = OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32
+    if prepared is not None:
+        _check(lib().msd_gemm_w4a16_prepared(_ptr(x), _ptr(w_fp4), _ptr(prepared), M, N, K, _ptr(y), yt, wp, wb, _stream()),
+               "msd_gemm_w4a16_prepared")
+    else:
+        _check(lib().msd_gemm_w4a16(_ptr(x), _ptr(w_fp4), _ptr(w_e8m0), M, N, K, _ptr(y), yt, wp, wb, _stream()), "msd_gemm_w4a16")
     return y
 
 

@@ -744,9 +744,61 @@ static GroupedW4Plan plan_grouped_w4(int32_t E, int64_t N, int64_t K, int groups
   return pl;
 }
 
+// Weight scales brought into the blocked layout once (msd_prepare_w4a16_scales): both tile widths' layouts back to
+// back, each E matrices of 2 * ceil(N / width) row blocks x sf_kgroups blocks of 512 bytes.
+struct PreparedScales {
+  int sf_kgroups;
+  size_t off224, off256, bytes;
+};
+static PreparedScales prepared_scales_layout(int32_t E, int64_t N, int64_t K) {
+  PreparedScales ps;
+  ps.sf_kgroups = 2 * static_cast<int>((K + kW4BlockK - 1) / kW4BlockK);
+  ps.off224 = 0;
+  ps.off256 = round_up(static_cast<size_t>(E) * 2 * ((N + 223) / 224) * ps.sf_kgroups * 512, 1024);
+  ps.bytes = ps.off256 + round_up(static_cast<size_t>(E) * 2 * ((N + 255) / 256) * ps.sf_kgroups * 512, 1024);
+  return ps;
+}
+
+__global__ void __launch_bounds__(256) sf_relayout_kernel(const SfRelayout rl) {
+  __shared__ uint32_t sm_rl[kSfRelayoutSmemWords];
+  sf_relayout(rl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x), sm_rl);
+}
+
+static msd_status_t gemm_w4a16_impl(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0, const uint8_t* prepared,
+                                    int64_t M, int64_t N, int64_t K, void* y, msd_out_t ytype, void* workspace,
+                                    size_t workspace_bytes, void* stream);
+static msd_status_t grouped_gemm_w4a16_impl(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0, const uint8_t* prepared,
+                                            const int32_t* group_sizes_host, int32_t E, int64_t N, int64_t K, void* y,
+                                            msd_out_t ytype, void* workspace, size_t workspace_bytes, void* stream);
+
 }  // namespace msd
 
 extern "C" {
+
+size_t msd_w4a16_prepared_scales_bytes(int32_t E, int64_t N, int64_t K) {
+  if (E < 1 || N < 1 || K < 128 || K % 128 != 0) return 0;
+  return msd::prepared_scales_layout(E, N, K).bytes;
+}
+
+msd_status_t msd_prepare_w4a16_scales(const uint8_t* w_e8m0, int32_t E, int64_t N, int64_t K, uint8_t* prepared, void* stream) {
+  using namespace msd;
+  if (E < 1 || N < 1 || K < 128 || K % 128 != 0 || N > (1 << 24) || K > (1 << 24) || static_cast<int64_t>(E) * N > 0x7FFFFFFFLL)
+    return MSD_ERR_BAD_SHAPE;
+  if (!w_e8m0 || !prepared) return MSD_ERR_NULL_POINTER;
+  if (!aligned(w_e8m0, 4) || !aligned(prepared, 1024)) return MSD_ERR_BAD_ALIGNMENT;
+  const PreparedScales ps = prepared_scales_layout(E, N, K);
+  for (int width = 224; width <= 256; width += 32) {
+    SfRelayout rl = {};
+    rl.src = w_e8m0; rl.dst = prepared + (width == 224 ? ps.off224 : ps.off256); rl.rows = N; rl.kblocks = static_cast<int>(K / 32);
+    rl.sf_kgroups = ps.sf_kgroups; rl.tile_rows = width; rl.row_blocks = 2 * static_cast<int>((N + width - 1) / width);
+    rl.matrices = E;
+    const long long units = static_cast<long long>(E) * rl.row_blocks * ((ps.sf_kgroups + 31) / 32);
+    const long long cap = static_cast<long long>(sm_count()) * 8;
+    sf_relayout_kernel<<<static_cast<unsigned>(units < cap ? units : cap), 256, 0, static_cast<cudaStream_t>(stream)>>>(rl);
+    if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
+  }
+  return MSD_OK;
+}
 
 size_t msd_gemm_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
   if (M < 1 || N < 1 || K < 128 || K % 128 != 0) return 0;
@@ -756,12 +808,30 @@ size_t msd_gemm_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0, int64_t M, int64_t N,
                             int64_t K, void* y, msd_out_t ytype, void* workspace, size_t workspace_bytes,
                             void* stream) {
-  using namespace msd;
+  if (!w_e8m0) return MSD_ERR_NULL_POINTER;
+  return msd::gemm_w4a16_impl(x_bf16, w_fp4, w_e8m0, nullptr, M, N, K, y, ytype, workspace, workspace_bytes, stream);
+}
+
+msd_status_t msd_gemm_w4a16_prepared(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* prepared_scales, int64_t M,
+                                     int64_t N, int64_t K, void* y, msd_out_t ytype, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+  if (!prepared_scales) return MSD_ERR_NULL_POINTER;
+  return msd::gemm_w4a16_impl(x_bf16, w_fp4, nullptr, prepared_scales, M, N, K, y, ytype, workspace, workspace_bytes, stream);
+}
+
+}  // extern "C"
+
+namespace msd {
+
+static msd_status_t gemm_w4a16_impl(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0, const uint8_t* prepared,
+                                    int64_t M, int64_t N, int64_t K, void* y, msd_out_t ytype, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
   if (M < 1 || N < 1 || K < 128 || K % 128 != 0 || N % 8 != 0 || M > (1 << 24) || N > (1 << 24) || K > (1 << 24))
     return MSD_ERR_BAD_SHAPE;
   if (ytype != MSD_OUT_BF16 && ytype != MSD_OUT_FP32) return MSD_ERR_UNSUPPORTED;
-  if (!x_bf16 || !w_fp4 || !w_e8m0 || !y || !workspace) return MSD_ERR_NULL_POINTER;
-  if (!aligned(x_bf16, 16) || !aligned(w_fp4, 16) || !aligned(w_e8m0, 4) || !aligned(y, 16) || !aligned(workspace, 1024))
+  if (!x_bf16 || !w_fp4 || !y || !workspace) return MSD_ERR_NULL_POINTER;
+  if (!aligned(x_bf16, 16) || !aligned(w_fp4, 16) || !aligned(w_e8m0, 4) || !aligned(prepared, 1024) || !aligned(y, 16) ||
+      !aligned(workspace, 1024))
     return MSD_ERR_BAD_ALIGNMENT;     // the scale relayout reads the E8M0 rows as 32-bit words
   const GemmW4Plan pl = plan_w4(M, N, K);
   if (workspace_bytes < pl.bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
@@ -781,7 +851,14 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   SfRelayout rl = {};
   rl.src = w_e8m0; rl.dst = ws + pl.off_sfb; rl.rows = N; rl.kblocks = static_cast<int>(K / 32);
   rl.sf_kgroups = pl.sf_kgroups; rl.tile_rows = pl.tile_n; rl.row_blocks = 2 * pl.n_tiles;
-  msd_status_t st = launch_decompose_mxfp4(x_bf16, M, K, K, q1, q2, ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s, &rl);
+  // (scales prepared once by msd_prepare_w4a16_scales: nothing to bring into the blocked layout here)
+  const uint8_t* sfb = ws + pl.off_sfb;
+  if (prepared) {
+    const PreparedScales ps = prepared_scales_layout(1, N, K);
+    sfb = prepared + (pl.tile_n == 224 ? ps.off224 : ps.off256);
+  }
+  msd_status_t st = launch_decompose_mxfp4(x_bf16, M, K, K, q1, q2, ws + pl.off_sfa1, ws + pl.off_sfa2, pl.sf_kgroups, s,
+                                           prepared ? nullptr : &rl);
   if (st != MSD_OK) return st;
 
   CUtensorMap tmap_a1, tmap_a2, tmap_b;
@@ -794,7 +871,7 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   GemmW4Params p;
   p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.kstages = pl.kstages; p.sf_kgroups = pl.sf_kgroups;
-  p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
+  p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = sfb;
   p.y = y; p.ytype = ytype; p.status = status;
   p.a_rows = kW4TileM; p.nstages = kW4Stages; p.ksplit = 1; p.kper = pl.kstages; p.part_rows = 0;
   {
@@ -860,6 +937,10 @@ msd_status_t msd_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint
   return MSD_OK;
 }
 
+}  // namespace msd
+
+extern "C" {
+
 size_t msd_grouped_gemm_w4a16_workspace_bytes(int32_t E, int64_t N, int64_t K) {
   if (E < 1 || N < 1 || K < 128 || K % 128 != 0) return 0;
   return msd::plan_grouped_w4(E, N, K, E).bytes;
@@ -868,13 +949,31 @@ size_t msd_grouped_gemm_w4a16_workspace_bytes(int32_t E, int64_t N, int64_t K) {
 msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0,
                                     const int32_t* group_sizes_host, int32_t E, int64_t N, int64_t K, void* y,
                                     msd_out_t ytype, void* workspace, size_t workspace_bytes, void* stream) {
-  using namespace msd;
+  if (!w_e8m0) return MSD_ERR_NULL_POINTER;
+  return msd::grouped_gemm_w4a16_impl(x_bf16, w_fp4, w_e8m0, nullptr, group_sizes_host, E, N, K, y, ytype, workspace, workspace_bytes, stream);
+}
+
+msd_status_t msd_grouped_gemm_w4a16_prepared(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* prepared_scales,
+                                             const int32_t* group_sizes_host, int32_t E, int64_t N, int64_t K, void* y,
+                                             msd_out_t ytype, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!prepared_scales) return MSD_ERR_NULL_POINTER;
+  return msd::grouped_gemm_w4a16_impl(x_bf16, w_fp4, nullptr, prepared_scales, group_sizes_host, E, N, K, y, ytype, workspace, workspace_bytes, stream);
+}
+
+}  // extern "C"
+
+namespace msd {
+
+static msd_status_t grouped_gemm_w4a16_impl(const void* x_bf16, const uint8_t* w_fp4, const uint8_t* w_e8m0, const uint8_t* prepared,
+                                            const int32_t* group_sizes_host, int32_t E, int64_t N, int64_t K, void* y,
+                                            msd_out_t ytype, void* workspace, size_t workspace_bytes, void* stream) {
   if (E < 1 || N < 1 || K < 128 || K % 128 != 0 || N % 8 != 0 || N > (1 << 24) || K > (1 << 24) ||
       static_cast<int64_t>(E) * N > 0x7FFFFFFFLL)
     return MSD_ERR_BAD_SHAPE;
   if (ytype != MSD_OUT_BF16 && ytype != MSD_OUT_FP32) return MSD_ERR_UNSUPPORTED;
-  if (!x_bf16 || !w_fp4 || !w_e8m0 || !group_sizes_host || !y || !workspace) return MSD_ERR_NULL_POINTER;
-  if (!aligned(x_bf16, 16) || !aligned(w_fp4, 16) || !aligned(w_e8m0, 4) || !aligned(y, 16) || !aligned(workspace, 1024))
+  if (!x_bf16 || !w_fp4 || !group_sizes_host || !y || !workspace) return MSD_ERR_NULL_POINTER;
+  if (!aligned(x_bf16, 16) || !aligned(w_fp4, 16) || !aligned(w_e8m0, 4) || !aligned(prepared, 1024) || !aligned(y, 16) ||
+      !aligned(workspace, 1024))
     return MSD_ERR_BAD_ALIGNMENT;
   int64_t M_total = 0;
   int nonempty = 0, largest = 0;
@@ -919,7 +1018,12 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
 
   // up to 64 non-empty groups per pair of launches (decomposition + GEMM); the weight scales of all experts are brought
   // into the blocked layout by the first decomposition launch
-  bool scales_done = false;
+  bool scales_done = prepared != nullptr;
+  const uint8_t* sfb = ws + pl.off_sfb;
+  if (prepared) {
+    const PreparedScales ps = prepared_scales_layout(E, N, K);
+    sfb = prepared + (pl.tile_n == 224 ? ps.off224 : ps.off256);
+  }
   int e = 0;
   int64_t row = 0;
   while (e < E) {
@@ -952,7 +1056,7 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
     GemmW4Params p;
     p.M = static_cast<int>(M_total); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     p.m_tiles = grp.n; p.n_tiles = pl.n_tiles; p.kstages = pl.kstages; p.sf_kgroups = pl.sf_kgroups;
-    p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = ws + pl.off_sfb;
+    p.sfa1 = ws + pl.off_sfa1; p.sfa2 = ws + pl.off_sfa2; p.sfb = sfb;
     p.y = y; p.ytype = ytype; p.status = status;
     p.a_rows = a_rows; p.nstages = nstages;
     p.ksplit = 1; p.kper = pl.kstages; p.part_rows = 0;
@@ -969,5 +1073,4 @@ msd_status_t msd_grouped_gemm_w4a16(const void* x_bf16, const uint8_t* w_fp4, co
   return MSD_OK;
 }
 
-
-}  // extern "C"
+}  // namespace msd

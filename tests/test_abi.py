@@ -59,3 +59,14 @@ def test_argument_checks_precede_any_launch():
     # the allocation-free entry point reports bad arguments before it clears its scratch
     assert lib.msd_gemm_w8a16_noalloc(null, p, p, 4, 128, 128, p, 0, None) in (1, 6)
     assert lib.msd_gemm_w8a16_noalloc(p, p, p, 17, 128, 128, p, 0, None) == 4
+    # weight scales prepared once: size query, null / misaligned buffers, shape rules as for msd_gemm_w4a16
+    assert lib.msd_w4a16_prepared_scales_bytes(1, 8192, 8192) >= 2 * 8192 * 8192 // 32
+    assert lib.msd_w4a16_prepared_scales_bytes(1, 8192, 100) == 0
+    assert lib.msd_prepare_w4a16_scales(null, 1, 128, 128, p, None) == 1
+    assert lib.msd_prepare_w4a16_scales(p, 1, 128, 128, C.c_void_p(4096 + 512), None) == 3
+    assert lib.msd_prepare_w4a16_scales(p, 0, 128, 128, p, None) == 2
+    assert lib.msd_gemm_w4a16_prepared(p, p, null, 128, 128, 128, p, 0, p, 1 << 30, None) == 1
+    assert lib.msd_gemm_w4a16_prepared(p, p, C.c_void_p(4096 + 512), 128, 128, 128, p, 0, p, 1 << 30, None) == 3
+    assert lib.msd_gemm_w4a16_prepared(p, p, p, 128, 128, 100, p, 0, p, 1 << 30, None) == 2
+    sizes = (C.c_int32 * 2)(4, 4)
+    assert lib.msd_grouped_gemm_w4a16_prepared(p, p, null, sizes, 2, 128, 128, p, 0, p, 1 << 30, None) == 1

@@ -103,3 +103,28 @@ def test_decode_shapes_with_k_split(M, N, K):
     _close(y, ref, False)
     yb = _run(c, torch.bfloat16)
     _close(oracle.bf16_bits_to_f64(bf16_bits(yb)), ref, True)
+
+
+@pytest.mark.parametrize("M,N,K,pair,tile", [(300, 264, 384, -1, -1), (520, 1032, 768, 1, 256), (520, 1032, 768, 1, 224),
+                                             (384, 776, 1024, 0, 224), (384, 776, 1024, 0, 256), (16, 448, 4096, -1, -1)])
+def test_prepared_weight_scales(M, N, K, pair, tile):
+    """Weight scales brought into the blocked layout once (msd_prepare_w4a16_scales) instead of on every call: against
+    the oracle, and bit for bit the result of the call that takes the row-major scales; single-CTA, CTA-pair and
+    K-split kernels, both tile widths, ragged last weight tile.  The prepared buffer is made once and used twice."""
+    c = inputs.gemm_w4_case(M, N, K, seed=3 + M + N)
+    ref = oracle.gemm_w4a16(c.x, c.w_fp4, c.w_e8m0, "f64")
+    xd, qd, ed = bf16_dev(c.x), dev(c.w_fp4), dev(c.w_e8m0)
+    prepared = binding.prepare_w4a16_scales(ed)
+    if pair >= 0:
+        binding.debug_set_option("MSD_W4_PAIR", pair)
+    if tile >= 0:
+        binding.debug_set_option("MSD_W4_TILEN", tile)
+    plain = binding.gemm_w4a16(xd, qd, ed, out_dtype=torch.float32)
+    for _ in range(2):
+        y = binding.gemm_w4a16(xd, qd, None, out_dtype=torch.float32, prepared=prepared)
+        torch.cuda.synchronize()
+        binding.last_device_status()
+        _close(y.cpu().numpy().astype(np.float64), ref, False)
+        assert torch.equal(y, plain)
+    yb = binding.gemm_w4a16(xd, qd, None, out_dtype=torch.bfloat16, prepared=prepared)
+    assert torch.equal(yb, binding.gemm_w4a16(xd, qd, ed, out_dtype=torch.bfloat16))

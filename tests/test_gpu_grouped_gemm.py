@@ -110,3 +110,24 @@ def test_grouped_w4a16_matches_per_expert_oracle(sizes, N, K):
     torch.cuda.synchronize()
     got = oracle.bf16_bits_to_f64(bf16_bits(yb))
     assert np.all(np.abs(got - ref) <= TOL * n + np.abs(ref) * 2.0 ** -8 + 1e-30)
+
+
+@pytest.mark.parametrize("sizes,N,K", [([128, 5, 0, 0, 64, 33, 9, 2], 1000, 1024), ([1] * 70 + [0] * 10 + [4] * 5, 232, 256)])
+def test_grouped_w4a16_with_prepared_scales(sizes, N, K):
+    """All experts' weight scales prepared once: against the per-expert oracle and bit for bit the unprepared call."""
+    x, q, e = _case_w4(sizes, N, K, seed=5 + len(sizes))
+    ref = np.zeros((x.shape[0], N), np.float64)
+    off = 0
+    for g, m in enumerate(sizes):
+        if m:
+            ref[off:off + m] = oracle.gemm_w4a16(x[off:off + m], q[g], e[g], "f64")
+        off += m
+    xd, qd, ed = bf16_dev(x), dev(q), dev(e)
+    prepared = binding.prepare_w4a16_scales(ed)
+    plain = binding.grouped_gemm_w4a16(xd, qd, ed, sizes, out_dtype=torch.float32)
+    y = binding.grouped_gemm_w4a16(xd, qd, None, sizes, out_dtype=torch.float32, prepared=prepared)
+    torch.cuda.synchronize()
+    binding.last_device_status()
+    n = np.linalg.norm(ref, axis=-1, keepdims=True)
+    assert np.all(np.abs(y.cpu().numpy() - ref) <= TOL * n + 1e-30)
+    assert torch.equal(y, plain)
