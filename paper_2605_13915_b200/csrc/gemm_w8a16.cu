@@ -41,6 +41,8 @@ struct GemmW8Params {
   int hmax;                // tallest band (box rows of tmap_w; tmap_w2 has hmax - gran)
   int w_chunk_bytes;       // shared-memory bytes reserved for one weight box (band rows x 128 B, 1 KB granules)
   int kw;                  // adjacent 128-byte K boxes per stage: each weight row is then read kw*128 B at a time
+  int tma3d;               // 1: the kw boxes of a stage travel as ONE 3-D box {128 B, rows, kw} of a tensor map whose third
+                           // dimension walks the 128-byte K blocks (needs K bytes % 128 == 0); 0: kw 2-D boxes
   int csplit;              // mode 2: CTAs per cluster = K slices per weight tile
   int pre_stages;          // stages whose weight boxes are requested before waiting for the preceding kernel
   int epi_off;             // byte offset of the epilogue's transpose buffer in dynamic shared memory
@@ -289,8 +291,6 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
   uint8_t* epi_buf = smem + p.epi_off;             // 16 KB transpose buffer of the epilogue, after the pipeline stages
   const int x_chunk_bytes = p.NB * kBlockK;
-  const int w_stage_bytes = p.kw * p.w_chunk_bytes;
-  const int stage_bytes = w_stage_bytes + p.kw * x_chunk_bytes;
 
   const long long grid = gridDim.x;
   // mode 0: this CTA's slice of the tile-major (tile, K block) sequence; mode 1: its row band and every K block
@@ -312,17 +312,23 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     blk_begin = 0;
     blk_end = p.kblocks;
   }
+  // One weight box in shared memory: a 3-D box packs its kw chunks back to back at this CTA's own band height (a
+  // multiple of 8 rows, so every chunk still starts on a 1 KB swizzle atom); 2-D boxes sit at the plan's stride.
+  const int w_chunk = (p.tma3d && p.mode == 1) ? band_h * kBlockK : p.w_chunk_bytes;
+  const int w_stage_bytes = p.kw * w_chunk;
+  const int stage_bytes = w_stage_bytes + p.kw * x_chunk_bytes;
   // Mode 1: every CTA walks K from its own starting block so that concurrent requests of the CTAs spread over the
   // whole row instead of hitting the same 128-byte column of every row (integer sums do not depend on the order).
   const int kb_rot = (p.mode == 1) ? static_cast<int>((static_cast<long long>(blockIdx.x) * p.kb_rot_step) % p.kblocks) : 0;
   const CUtensorMap* wmap = (p.mode == 1 && band_h != p.hmax) ? &tmap_w2 : &tmap_w;
   const int tx_bytes = p.kw * ((p.mode == 0 ? kWStageBytes : band_h * kBlockK) + x_chunk_bytes);
 
+  // the barriers of the pipeline stages one stage per lane of the producer warp, the others by its first lane
+  if (warp == 0 && lane < p.num_stages) {
+    mbar_init(&full_bar[lane], 1);
+    mbar_init(&empty_bar[lane], 1);
+  }
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.num_stages; ++s) {
-      mbar_init(&full_bar[s], 1);
-      mbar_init(&empty_bar[s], 1);
-    }
     for (int a = 0; a < 2; ++a) {
       mbar_init(&tfull_bar[a], 1);
       mbar_init(&tempty_bar[a], 4);      // one arrival per epilogue warp
@@ -339,7 +345,10 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       }
     }
     abort_flag = 0;
+  }
+  if (warp == 0) {
     mbar_init_fence();
+    __syncwarp();
   }
   // ------------------------------ TMA producer, first part ------------------------------
   // Runs before the CTA-wide barrier below: the thread that initialised the mbarriers is in this warp, and the sooner
@@ -365,6 +374,15 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     if (++kbi == p.kblocks) { kbi = 0; ++tile; }
     if (++kbr == p.kblocks) kbr = 0;
   };
+  // the weight box(es) / component box(es) of K block `kblk` (in units of stages) into stage memory at `dst`
+  auto load_w = [&](uint8_t* dst, int kblk, int row, uint64_t* bar) {
+    if (p.tma3d) tma_load_3d_hint(dst, wmap, 0, row, kblk * p.kw, bar, pol_w);
+    else tma_load_2d_hint(dst + c * w_chunk, wmap, (kblk * p.kw + c) * kBlockK, row, bar, pol_w);
+  };
+  auto load_x = [&](uint8_t* dst, int kblk, int row, uint64_t* bar) {
+    if (p.tma3d && !kGrouped) tma_load_3d_hint(dst + w_stage_bytes, &tmap_x, 0, row, kblk * p.kw, bar, pol_x);
+    else tma_load_2d_hint(dst + w_stage_bytes + c * x_chunk_bytes + x_half * x_half_bytes, &tmap_x, (kblk * p.kw + c) * kBlockK, row, bar, pol_x);
+  };
   if (warp == 0) {
     __syncwarp();
     // The whole warp takes part: lane 0 owns the barriers, lanes [0, kw) each issue one weight box of a stage and
@@ -372,8 +390,9 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     // of one after another by a single thread.
     pol_w = policy_evict_first();    // weights are streamed once
     pol_x = policy_evict_last();      // the stacked components are re-read by every CTA
-    w_lane = lane < p.kw;
+    w_lane = lane < (p.tma3d ? 1 : p.kw);
     x_lane = lane >= p.kw && lane < (kGrouped ? 3 : 2) * p.kw;     // grouped: one box per component
+    if (p.tma3d && !kGrouped) x_lane = lane == p.kw;              // one 3-D box of the stacked components per stage
     c = w_lane ? lane : (lane - p.kw) % p.kw;
     x_half = w_lane ? 0 : (lane - p.kw) / p.kw;
     // (tile, K block) of the next block to load, advanced by one per stage; kbr = rotated K block
@@ -393,9 +412,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     for (int i = 0; i < pre0; ++i) {
       if (lane == 0) mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
       __syncwarp();
-      if (w_lane)
-        tma_load_2d_hint(smem + i * stage_bytes + c * p.w_chunk_bytes, wmap, (kbr * p.kw + c) * kBlockK,
-                         w_row(tile), &full_bar[i], pol_w);
+      if (w_lane) load_w(smem + i * stage_bytes, kbr, w_row(tile), &full_bar[i]);
       advance();
     }
     if (lane == 0) trace_mark(p, 3);
@@ -418,14 +435,10 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         if (i >= pre0) {     // weight boxes held back so that the wait above was not queued behind them
           if (lane == 0) mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
           __syncwarp();
-          if (w_lane)
-            tma_load_2d_hint(smem + i * stage_bytes + c * p.w_chunk_bytes, wmap, (kbr * p.kw + c) * kBlockK,
-                             w_row(tile), &full_bar[i], pol_w);
+          if (w_lane) load_w(smem + i * stage_bytes, kbr, w_row(tile), &full_bar[i]);
           advance();
         }
-        if (x_lane)
-          tma_load_2d_hint(smem + i * stage_bytes + w_stage_bytes + c * x_chunk_bytes + x_half * x_half_bytes, &tmap_x,
-                           (kx * p.kw + c) * kBlockK, x_row(tile_first + (kbi_first + i) / p.kblocks), &full_bar[i], pol_x);
+        if (x_lane) load_x(smem + i * stage_bytes, kx, x_row(tile_first + (kbi_first + i) / p.kblocks), &full_bar[i]);
         if (++kx == p.kblocks) kx = 0;
       }
     }
@@ -440,11 +453,8 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
       uint8_t* dst = smem + stage * stage_bytes;
-      if (w_lane)
-        tma_load_2d_hint(dst + c * p.w_chunk_bytes, wmap, (kbr * p.kw + c) * kBlockK, w_row(tile), &full_bar[stage], pol_w);
-      else if (x_lane)
-        tma_load_2d_hint(dst + w_stage_bytes + c * x_chunk_bytes + x_half * x_half_bytes, &tmap_x, (kbr * p.kw + c) * kBlockK,
-                         x_row(tile), &full_bar[stage], pol_x);
+      if (w_lane) load_w(dst, kbr, w_row(tile), &full_bar[stage]);
+      else if (x_lane) load_x(dst, kbr, x_row(tile), &full_bar[stage]);
       advance();
       if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
     }
@@ -483,7 +493,7 @@ gemm_w8a16_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
           for (int c = 0; c < p.kw; ++c) {
 #pragma unroll
             for (int k = 0; k < kBlockK / 32; ++k) {
-              const uint64_t adesc = smem_desc(wa + c * p.w_chunk_bytes + k * 32, 16, 1024, kSwizzle128B);
+              const uint64_t adesc = smem_desc(wa + c * w_chunk + k * 32, 16, 1024, kSwizzle128B);
               const uint64_t bdesc = smem_desc(xa + c * x_chunk_bytes + k * 32, 16, 1024, kSwizzle128B);
               const uint32_t accum = (b > blk || c > 0 || k > 0) ? 1u : 0u;
               if constexpr (kBase) mma_f16(d_tmem, adesc, bdesc, idesc, accum);
@@ -862,6 +872,16 @@ __global__ void dequant_w8_to_bf16_kernel(const int8_t* __restrict__ w, const fl
   }
 }
 
+// Tensor map of a K-major byte matrix [rows, kbytes] for the GEMM's stages: with `t3` one 3-D box {128 B, box_rows, kw}
+// (third dimension = the 128-byte K blocks of a row, stride 128 B) brings the kw chunks of a stage with one copy
+// instruction; otherwise 2-D boxes of 128 B x box_rows.  t3 needs kbytes % 128 == 0 (a K block never straddles rows).
+static bool encode_stage_map(CUtensorMap* out, const void* base, uint64_t kbytes, uint64_t rows, uint32_t box_rows, int kw, bool t3) {
+  if (t3)
+    return encode_tmap_3d(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, base, kBlockK, rows, kbytes / kBlockK, kbytes, kBlockK, kBlockK, box_rows,
+                          static_cast<uint32_t>(kw), CU_TENSOR_MAP_SWIZZLE_128B);
+  return encode_tmap_2d(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, base, kbytes, rows, kbytes, kBlockK, box_rows, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
 constexpr int64_t kMaxExactK = 131072;
 
 static msd_status_t check_w8_args(const void* x, const void* w, const void* ws, int64_t M, int64_t N, int64_t K,
@@ -925,12 +945,13 @@ msd_status_t msd_gemm_w8a16_ex(const void* x_bf16, const int8_t* w, const float*
 
   CUtensorMap tmap_w, tmap_w2, tmap_x;
   const uint32_t box2 = (pl.mode == 1 && pl.hmax > pl.gran) ? pl.hmax - pl.gran : pl.hmax;
-  if (!encode_tmap_2d(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kBlockK, pl.hmax, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !encode_tmap_2d(&tmap_w2, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kBlockK, box2, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, q, K, pl.NB, K, kBlockK, pl.NB, CU_TENSOR_MAP_SWIZZLE_128B))
+  const bool t3 = K % kBlockK == 0;
+  if (!encode_stage_map(&tmap_w, w, K, N, pl.hmax, pl.kw, t3) || !encode_stage_map(&tmap_w2, w, K, N, box2, pl.kw, t3) ||
+      !encode_stage_map(&tmap_x, q, K, pl.NB, pl.NB, pl.kw, t3))
     return MSD_ERR_CUDA;
 
   GemmW8Params p;
+  p.tma3d = t3 ? 1 : 0;
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = 5;
   p.pre_stages = 64;
@@ -981,11 +1002,12 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   CUtensorMap tmap_w, tmap_w2, tmap_x;
   const uint64_t kb = static_cast<uint64_t>(2 * K);
   const uint32_t box2 = (pl.mode == 1 && pl.hmax > pl.gran) ? pl.hmax - pl.gran : pl.hmax;
-  if (!encode_tmap_2d(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, wbf, kb, N, kb, kBlockK, pl.hmax, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !encode_tmap_2d(&tmap_w2, CU_TENSOR_MAP_DATA_TYPE_UINT8, wbf, kb, N, kb, kBlockK, box2, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, x_bf16, kb, M, kb, kBlockK, pl.NB, CU_TENSOR_MAP_SWIZZLE_128B))
+  const bool t3 = kb % kBlockK == 0;
+  if (!encode_stage_map(&tmap_w, wbf, kb, N, pl.hmax, pl.kw, t3) || !encode_stage_map(&tmap_w2, wbf, kb, N, box2, pl.kw, t3) ||
+      !encode_stage_map(&tmap_x, x_bf16, kb, M, pl.NB, pl.kw, t3))
     return MSD_ERR_CUDA;
   GemmW8Params p;
+  p.tma3d = t3 ? 1 : 0;
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = 0;
   p.pre_stages = 64;
@@ -1075,8 +1097,8 @@ msd_status_t msd_grouped_gemm_w8a16(const void* x_bf16, const int8_t* w, const f
   const int kw = pl.kw;
   const int kblocks = pl.kblocks;
   CUtensorMap tmap_w, tmap_x;
-  if (!encode_tmap_2d(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, static_cast<uint64_t>(E) * N, K, kBlockK, kTileN,
-                      CU_TENSOR_MAP_SWIZZLE_128B) ||
+  const bool t3 = K % kBlockK == 0;        // the weight stages as 3-D boxes; the two component boxes of a group stay 2-D
+  if (!encode_stage_map(&tmap_w, w, K, static_cast<uint64_t>(E) * N, kTileN, kw, t3) ||
       !encode_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, q, K, 2 * static_cast<uint64_t>(gp.mt_pad), K, kBlockK, pl.Mp,
                       CU_TENSOR_MAP_SWIZZLE_128B))
     return MSD_ERR_CUDA;
@@ -1086,6 +1108,7 @@ msd_status_t msd_grouped_gemm_w8a16(const void* x_bf16, const int8_t* w, const f
   p.M = pl.Mp; p.Mp = pl.Mp; p.NB = pl.NB; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.kb_rot_step = 0; p.pre_stages = 64;
   p.mode = 0; p.groups8 = 1; p.gran = 8; p.hmax = kTileN; p.w_chunk_bytes = kWStageBytes; p.kw = kw; p.csplit = 1;
+  p.tma3d = t3 ? 1 : 0;
   p.kblocks = kblocks; p.num_stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype;
   // the planner laid the stages out for row bands when N is large; stream-K always stages full 128-row weight boxes
   {
