@@ -747,10 +747,15 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
           uint8_t* dst = smem + st * kv_stage_bytes;
           const int tok0 = seq0 + t_begin + kq * kTok;
           if (kq >= 2 && kq < 5) attn_mark(p, 9 + 6 * (kq - 2));
+          // Chunk by chunk as the tile two back lets go of the stage: the rotary chunk (read by QK^T only) when its
+          // scores are complete (s_full of that tile: same index, same phase; a commit costs its thread about 80 ns,
+          // so the rotary chunk has no barrier of its own), value chunk j when the dv tile of PV that reads it is
+          // complete.  (Parity ph ^ 1 passes at once on a barrier that has not completed a phase yet.)
 #pragma unroll
           for (int i = 0; i < 5; ++i) {
             const int c = (i == 0) ? 4 : i - 1;
-            okp = wait_bounded(&ck_empty[st][c], ph ^ 1, abort, p.status);
+            if (i == 0) okp = wait_bounded(&s_full[st], ph ^ 1, abort, p.status);
+            else okp = wait_bounded(&ck_empty[st][c], ph ^ 1, abort, p.status);
             if (!okp) break;
             if (i == 0) mbar_arrive_expect_tx(&kv_full[st], 5 * kChunkBytes);
             tma_load_3d(dst + c * kChunkBytes, &tmap_k, c * kChunk, hk, tok0, &kv_full[st]);
@@ -844,13 +849,19 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
         const uint64_t ka = dk + smem_enc + static_cast<uint32_t>(st * (kv_stage_bytes >> 4));
         const uint32_t d = tmem_base + (t & 1) * p.Rp;
         if constexpr (kFixDC > 0) {
+          // (address fields never carry out of the descriptors' lower words: shared memory is 227 KB, the field counts 16 bytes)
+          const uint32_t ka_lo = static_cast<uint32_t>(ka), k_hi = static_cast<uint32_t>(ka >> 32);
+          const uint32_t qa_lo = static_cast<uint32_t>(q_enc), q_hi = static_cast<uint32_t>(q_enc >> 32);
 #pragma unroll
           for (int c = 0; c < kFixDC; ++c)
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-              if (c + 1 < kFixDC || k < last_steps)
-                mma_i8(d, ka + (c * (kChunkBytes >> 4) + 2 * k), q_enc + (c * ((kWideSlots * 2 * kChunk) >> 4) + 2 * k), idesc_qk,
-                       (c > 0 || k > 0) ? 1u : 0u);
+              if (c + 1 < kFixDC || k < last_steps) {
+                if (c > 0 || k > 0)
+                  mma_i8_lohi<true>(d, ka_lo + (c * (kChunkBytes >> 4) + 2 * k), k_hi, qa_lo + (c * ((kWideSlots * 2 * kChunk) >> 4) + 2 * k), q_hi, idesc_qk);
+                else
+                  mma_i8_lohi<false>(d, ka_lo, k_hi, qa_lo, q_hi, idesc_qk);
+              }
         } else {
           uint64_t kc = ka, qa = q_enc;
           for (int c = 0; c < nDC; ++c) {
@@ -862,7 +873,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
           }
         }
         tc_commit(&s_full[t & 1]);
-        if constexpr (kChunked) tc_commit(&ck_empty[st][4]);       // the rotary chunk has no other reader
+        if constexpr (kChunked) { /* the producer takes s_full as "the rotary chunk has been read" */ }
         else if (!p.v_alias) tc_commit(&kv_empty[st]);       // separate V: the K buffer is free once QK^T has read it
       };
       // PV of tile t, added to what the accumulators hold unless `fresh`
@@ -874,13 +885,17 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
         const uint64_t pa = p_enc + (t & 1) * p_step;
         const uint32_t acc0 = fresh ? 0u : 1u;
         if constexpr (kFixDVT > 0) {
+          const uint32_t va_lo = static_cast<uint32_t>(va), v_hi = static_cast<uint32_t>(va >> 32);
+          const uint32_t pa_lo = static_cast<uint32_t>(pa), p_hi = static_cast<uint32_t>(pa >> 32);
 #pragma unroll
           for (int j = 0; j < kFixDVT; ++j) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k)      // 32 tokens per MMA: four 8-token groups of 1024 bytes
-              mma_i8(tmem_o + j * (2 * kWideSlots), va + (j * (kChunkBytes >> 4) + k * (4096 >> 4)), pa + k * (2048 >> 4), idesc_pv,
-                     k > 0 ? 1u : acc0);
-            if constexpr (kChunked) tc_commit(&ck_empty[st][j]);      // value chunk j may be requested again
+            for (int k = 0; k < 4; ++k) {    // 32 tokens per MMA: four 8-token groups of 1024 bytes
+              if (k > 0)
+                mma_i8_lohi<true>(tmem_o + j * (2 * kWideSlots), va_lo + (j * (kChunkBytes >> 4) + k * (4096 >> 4)), v_hi, pa_lo + k * (2048 >> 4), p_hi, idesc_pv);
+              else
+                mma_i8(tmem_o + j * (2 * kWideSlots), va + (j * (kChunkBytes >> 4)), pa, idesc_pv, acc0);
+            }
           }
         } else {
           uint64_t vc = va;
@@ -894,14 +909,32 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
         }
         // o_full counts every PV product (a drain in mid-split waits for the one before its tile: at that point the
         // barrier is at most one phase behind, so a parity test is unambiguous); the last one has a barrier of its own
-        tc_commit(t == ntiles - 1 ? &o_last : &o_full);
-        if constexpr (!kChunked) tc_commit(p.v_alias ? &kv_empty[st] : &v_empty[st]);
+        // (chunked stages: the commit after the last dv tile, ck_empty[st][3], says the same)
+        if constexpr (!kChunked) {
+          tc_commit(t == ntiles - 1 ? &o_last : &o_full);
+          tc_commit(p.v_alias ? &kv_empty[st] : &v_empty[st]);
+        }
       };
       // QK^T(q) needs KV tile q in shared memory and the score buffer q&1 read (P of tile q-2 final);
       // PV(v) needs P of tile v final (written, and rewritten when the references had to move) and QK^T(v) issued.
       // One thread issues both, so everything it has issued completes in order: when the scores of tile t are
       // there, PV of tile t-2 is complete (the P buffer and the o_full phase the softmax warps rely on).
       int q = 0, v = 0, n_slow = 0;
+      if constexpr (kChunked) {
+        // PV is issued by four softmax threads (below); this thread issues QK^T only.  QK^T(q) needs KV tile q in shared
+        // memory and the score buffer q&1 read, i.e. P of tile q-2 written by every softmax warp (the slow path works
+        // from registers).  The P buffer q&1 is free by then as well: KV tile q arrives in the stage that PV(q-2) gave
+        // back chunk by chunk, so its arrival implies that PV(q-2) is complete.
+        for (; q < ntiles && ok; ++q) {
+          if (q >= 2) ok = wait_bounded(&p_full[q & 1], ((q - 2) >> 1) & 1, abort, p.status);
+          if (ok) ok = wait_bounded(&kv_full[q & 1], (q >> 1) & 1, abort, p.status);
+          if (!ok) break;
+          if (q >= 2 && q < 5) attn_mark(p, 7 + 6 * (q - 2));
+          issue_qk(q);
+          if (q >= 2 && q < 5) attn_mark(p, q == 4 ? 30 : 23 + q);
+        }
+        v = ntiles;
+      }
       long long t_idle = clock64();
       while (ok && v < ntiles) {
         bool progressed = false;
@@ -1088,6 +1121,15 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       tmem_st_wait();
     };
 
+    // operand descriptors of PV as lower / upper words (see mma_i8_lohi): V^T read MN-major from the token-major KV tile,
+    // P an MN-major operand too (token-major, 64-byte swizzle, groups of 8 tokens 512 bytes apart)
+    const uint64_t pv_vdesc = smem_desc(0, 16384, 1024, kSwizzle128B) + (smem_u32(smem) >> 4);
+    const uint64_t pv_pdesc = smem_desc(0, 512, 512, kSwizzle64B) + (smem_u32(sm_p) >> 4);
+    const uint32_t pv_va_lo = static_cast<uint32_t>(pv_vdesc), pv_v_hi = static_cast<uint32_t>(pv_vdesc >> 32);
+    const uint32_t pv_pa_lo = static_cast<uint32_t>(pv_pdesc), pv_p_hi = static_cast<uint32_t>(pv_pdesc >> 32);
+    const uint32_t pv_p_step = static_cast<uint32_t>(p.Rp * kChunk) >> 4;
+    const uint32_t pv_idesc = idesc_dense(2, 1, 1, 1, 1, kTok, p.Rp);     // S8 x S8 -> S32, A (V^T) and B (P) MN-major
+
     bool ok = true;
     int n_slow = 0;
     float ks_pre, vs_pre;
@@ -1113,6 +1155,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       ok = wait_bounded(&p_full[t & 1], (t >> 1) & 1, abort, p.status);
       if (!ok) break;
       if (threadIdx.x == 64 && t >= 2 && t < 5) attn_mark(p, 6 + 6 * (t - 2));
+      bool slow = false;
       if (stamp[t & 1] == t + 1) {
         // ---- the references move: tile maxima per head over the group's 128 tokens, largest value scale ----
 #pragma unroll
@@ -1146,7 +1189,12 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
         }
         if (t > 0) {
           // everything accumulated so far was scaled by the old references: PV(t-1) and all before it are complete
-          ok = wait_bounded(&o_full, (t - 1) & 1, abort, p.status);
+          if constexpr (kChunked) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) ok = ok && wait_bounded(&ck_empty[(t - 1) & 1][j], ((t - 1) >> 1) & 1, abort, p.status);
+          } else {
+            ok = wait_bounded(&o_full, (t - 1) & 1, abort, p.status);
+          }
           if (!ok) break;
           tc_fence_after();
           drain(resc, alpha_old);
@@ -1160,13 +1208,45 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
         if (lane == 0) mbar_arrive(&p_redo);
         ++n_slow;
         named_bar_sync(bar_id, 128);          // `red` may be rewritten
+        slow = true;
+      }
+      if constexpr (kChunked) {
+        // PV(t), one dv tile per thread: lane 0 of the first four softmax warps, which sit on the four different warp
+        // schedulers.  The softmax warps are idle here (the next score tile is not there yet), the product starts the
+        // moment P is final instead of when the QK^T-issuing thread gets round to it, and its 16 MMAs are issued four
+        // abreast.  An accumulator is only ever written by its own thread, so its MMAs stay in program order.
+        if (hh == 0 && lane == 0) {
+          const int st = t & 1;
+          if (slow) ok = wait_bounded(&p_redo, (n_slow - 1) & 1, abort, p.status);      // every warp has drained and rewritten P
+          if (ok) ok = wait_bounded(&kv_full[st], (t >> 1) & 1, abort, p.status);      // (long complete: QK^T(t) has read the tile)
+          if (ok) {
+            tc_fence_after();
+            if (wq == 0 && t >= 2 && t < 5) attn_mark(p, 8 + 6 * (t - 2));
+            const uint32_t va_lo = pv_va_lo + static_cast<uint32_t>(st * (kv_stage_bytes >> 4)) + wq * (kChunkBytes >> 4);
+            const uint32_t pa_lo = pv_pa_lo + (t & 1) * pv_p_step;
+            const uint32_t acc = tmem_o + wq * (2 * kWideSlots);
+            if (slow) mma_i8_lohi<false>(acc, va_lo, pv_v_hi, pa_lo, pv_p_hi, pv_idesc);
+            else mma_i8_lohi<true>(acc, va_lo, pv_v_hi, pa_lo, pv_p_hi, pv_idesc);
+#pragma unroll
+            for (int k = 1; k < 4; ++k)      // 32 tokens per MMA: four 8-token groups of 1024 bytes
+              mma_i8_lohi<true>(acc, va_lo + k * (4096 >> 4), pv_v_hi, pa_lo + k * (2048 >> 4), pv_p_hi, pv_idesc);
+            tc_commit(&ck_empty[st][wq]);      // value chunk wq may be requested again; also "this dv tile of PV(t) is complete"
+            if (wq == 0 && t >= 2 && t < 5) attn_mark(p, 20 + t);
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       }
 #pragma unroll
       for (int h = 0; h < kWideHS; ++h) l_part[h] += pl[h];
     }
     if (ok) {
       // what the accumulators still hold
-      ok = wait_bounded(&o_last, 0, abort, p.status);
+      if constexpr (kChunked) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) ok = ok && wait_bounded(&ck_empty[(ntiles - 1) & 1][j], ((ntiles - 1) >> 1) & 1, abort, p.status);
+      } else {
+        ok = wait_bounded(&o_last, 0, abort, p.status);
+      }
       if (ok) {
         tc_fence_after();
         float one[kWideHS];
