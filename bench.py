@@ -614,6 +614,12 @@ def measure_configs(torch, binding, device, capture, timed_clocked, peaks, peak_
         entry = {"us": round(t, 1), "sm_mhz": clk["sm_mhz"], "executed_int8_pops": round(po, 3),
                  "roofline": roofline_block("tensor", po, NOMINAL["int8_pops"], "POP/s", "nominal dense INT8",
                                             frac_of_2x_measured_bf16=round(po * 1e3 / (2 * bf16), 3))}
+        # the comparison path as this library's own kernels: weights expanded to BF16, then the same pipeline as a BF16 GEMM
+        wsb = binding.workspace(binding.gemm_dequant_bf16_workspace_bytes(M, N, K), device)
+        tdq, _ = per_call_us(lambda: binding.gemm_dequant_bf16(x, w, s, ws=wsb), reps=2)
+        entry["comparison_dequant_bf16_kernel"] = {"us": round(tdq, 1), "msd_speedup": round(tdq / t, 2),
+                                                   "note": "msd_gemm_dequant_bf16: dequantize kernel + BF16 tcgen05 GEMM (ours)"}
+        del wsb
         if (N, K) == SHAPES[0]:
             wb = torch.empty((N, K), dtype=torch.bfloat16, device=device)
 

@@ -184,8 +184,9 @@ msd_status_t msd_gemm_w8a16_host(const void* x_bf16_host, const int8_t* w, const
 
 /*
  * Comparison path the method replaces (Sec. 3.1 first equation): weights dequantized to BF16,
- * bf16(w_scale[n]*w[n,k]), then a BF16 x BF16 GEMM with FP32 accumulation.  Same shapes as msd_gemm_w8a16.
- * workspace: >= msd_gemm_dequant_bf16_workspace_bytes(M,N,K) (holds the dequantized weights).
+ * bf16(w_scale[n]*w[n,k]), then a BF16 x BF16 GEMM with FP32 accumulation.  Same shapes as msd_gemm_w8a16, M > 128
+ * included (there K % 64 == 0, and N % 4 == 0 for FP32 output: the same many-row pipeline as msd_gemm_w8a16's, run as a
+ * BF16 GEMM).  workspace: >= msd_gemm_dequant_bf16_workspace_bytes(M,N,K) (holds the dequantized weights).
  */
 size_t msd_gemm_dequant_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K);
 msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M,

@@ -882,6 +882,15 @@ static bool encode_stage_map(CUtensorMap* out, const void* base, uint64_t kbytes
   return encode_tmap_2d(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, base, kbytes, rows, kbytes, kBlockK, box_rows, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
+msd_status_t launch_dequant_w8_to_bf16(const int8_t* w, const float* w_scale, int64_t N, int64_t K, void* out_bf16, cudaStream_t s) {
+  const int64_t total = N * (K >> 4);
+  int64_t blocks = (total + 255) / 256;
+  const int64_t cap = static_cast<int64_t>(sm_count()) * 16;
+  if (blocks > cap) blocks = cap;
+  dequant_w8_to_bf16_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(w, w_scale, N, K, static_cast<__nv_bfloat16*>(out_bf16));
+  return cudaGetLastError() == cudaSuccess ? MSD_OK : MSD_ERR_CUDA;
+}
+
 constexpr int64_t kMaxExactK = 131072;
 
 static msd_status_t check_w8_args(const void* x, const void* w, const void* ws, int64_t M, int64_t N, int64_t K,
@@ -974,7 +983,8 @@ msd_status_t msd_gemm_w8a16_ex(const void* x_bf16, const int8_t* w, const float*
 }
 
 size_t msd_gemm_dequant_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
-  if (M < 1 || M > 128 || N < 1 || K < 16) return 0;
+  if (M < 1 || M > (1 << 24) || N < 1 || K < 16) return 0;
+  if (M > 128) return msd::w8_prefill_base_workspace_bytes(M, N, K);
   return msd::plan_w8(M, N, K, true).bytes;
 }
 
@@ -982,8 +992,13 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
                                    int64_t K, void* y, msd_out_t ytype, void* workspace, size_t workspace_bytes,
                                    void* stream) {
   using namespace msd;
-  msd_status_t st = check_w8_args(x_bf16, w, w_scale, M, N, K, y, ytype, workspace);
+  msd_status_t st = check_w8_args(x_bf16, w, w_scale, M, N, K, y, ytype, workspace, 1 << 24);
   if (st != MSD_OK) return st;
+  if (M > 128) {
+    if (K % 64 != 0) return MSD_ERR_BAD_SHAPE;          // a K stage of the many-row kernel is 64 BF16 elements
+    if (ytype == MSD_OUT_FP32 && N % 4 != 0) return MSD_ERR_BAD_SHAPE;
+    return w8_prefill_base_launch(x_bf16, w, w_scale, M, N, K, y, ytype, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+  }
   const GemmW8Plan pl = plan_w8(M, N, K, true);
   if (workspace_bytes < pl.bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
   unsigned* status = device_status_ptr();
@@ -991,14 +1006,8 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   __nv_bfloat16* wbf = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_q);
-  {
-    const int64_t total = N * (K >> 4);
-    int64_t blocks = (total + 255) / 256;
-    const int64_t cap = static_cast<int64_t>(sm_count()) * 16;
-    if (blocks > cap) blocks = cap;
-    dequant_w8_to_bf16_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(w, w_scale, N, K, wbf);
-    if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
-  }
+  st = launch_dequant_w8_to_bf16(w, w_scale, N, K, wbf, s);
+  if (st != MSD_OK) return st;
   CUtensorMap tmap_w, tmap_w2, tmap_x;
   const uint64_t kb = static_cast<uint64_t>(2 * K);
   const uint32_t box2 = (pl.mode == 1 && pl.hmax > pl.gran) ? pl.hmax - pl.gran : pl.hmax;

@@ -52,7 +52,10 @@ struct GemmP8Params {
   unsigned* status;
 };
 
-template <bool kPair>
+// kBase: the comparison path the method replaces (Sec. 3.1, first equation) on the same pipeline: tmap_a1 describes
+// the BF16 activations and tmap_b the weights a preceding kernel dequantized to BF16 (both as byte matrices, a stage is
+// 64 elements), one BF16 x BF16 -> FP32 accumulator, no second component and no scales in the epilogue.
+template <bool kPair, bool kBase = false>
 __global__ void __launch_bounds__(kP8Threads, 1)
 gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
                           const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_y,
@@ -75,7 +78,7 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
     abort_flag = 0;
     mbar_init_fence();
     tma_prefetch_desc(&tmap_a1);
-    tma_prefetch_desc(&tmap_a2);
+    if (!kBase) tma_prefetch_desc(&tmap_a2);
     tma_prefetch_desc(&tmap_b);
     tma_prefetch_desc(&tmap_y);
   }
@@ -121,15 +124,15 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
           uint8_t* dst = smem + stage * kStageBytes;
           if (kPair) {
             // the leader's barrier counts the bytes of both CTAs; tmap_b's box is this CTA's half of the weight tile
-            if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * kStageBytes);
+            if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * (kStageBytes - (kBase ? kP8ABytes : 0)));
             const uint32_t bar = mapa_shared(smem_u32(&full_bar[stage]), 0);
             tma_load_2d_pair(dst, &tmap_a1, ks * kP8BlockK, mt * kP8TileM, bar);
-            tma_load_2d_pair(dst + kP8ABytes, &tmap_a2, ks * kP8BlockK, mt * kP8TileM, bar);
+            if (!kBase) tma_load_2d_pair(dst + kP8ABytes, &tmap_a2, ks * kP8BlockK, mt * kP8TileM, bar);
             tma_load_2d_pair(dst + 2 * kP8ABytes, &tmap_b, ks * kP8BlockK, nt * kP8TileN + static_cast<int>(rank) * (kP8TileN / 2), bar);
           } else {
-            mbar_arrive_expect_tx(&full_bar[stage], kStageBytes);
+            mbar_arrive_expect_tx(&full_bar[stage], kStageBytes - (kBase ? kP8ABytes : 0));
             tma_load_2d(dst, &tmap_a1, ks * kP8BlockK, mt * kP8TileM, &full_bar[stage]);
-            tma_load_2d(dst + kP8ABytes, &tmap_a2, ks * kP8BlockK, mt * kP8TileM, &full_bar[stage]);
+            if (!kBase) tma_load_2d(dst + kP8ABytes, &tmap_a2, ks * kP8BlockK, mt * kP8TileM, &full_bar[stage]);
             tma_load_2d(dst + 2 * kP8ABytes, &tmap_b, ks * kP8BlockK, nt * kP8TileN, &full_bar[stage]);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1; }
@@ -142,7 +145,8 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
       int it = 0;
       bool ok = true;
       const uint64_t op_desc = smem_desc(0, 16, 1024, kSwizzle128B);    // 128-byte-swizzled K-major operand tile
-      const uint32_t idesc = idesc_dense(/*D=S32*/ 2, /*A=S8*/ 1, /*B=S8*/ 1, 0, 0, kPair ? 2 * kP8TileM : kP8TileM, kP8TileN);
+      const uint32_t idesc = kBase ? idesc_dense(/*D=F32*/ 1, /*A=BF16*/ 1, /*B=BF16*/ 1, 0, 0, kPair ? 2 * kP8TileM : kP8TileM, kP8TileN)
+                                   : idesc_dense(/*D=S32*/ 2, /*A=S8*/ 1, /*B=S8*/ 1, 0, 0, kPair ? 2 * kP8TileM : kP8TileM, kP8TileN);
       for (int tile = first; tile < total_tiles && ok; tile += step, ++it) {
         ok = wait_bounded(&tempty_bar, (it & 1) ^ 1, abort, p.status);        // the epilogue has drained both accumulators
         if (!ok) break;
@@ -157,7 +161,10 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {                    // 32 elements (32 bytes) per MMA
             const uint32_t acc = (ks > ks0 || kk > 0) ? 1u : 0u;
-            if (kPair) {
+            if constexpr (kBase) {              // 16 BF16 elements (32 bytes) per MMA
+              if (kPair) mma_f16_pair(tmem_base, a1d + 2 * kk, bd + 2 * kk, idesc, acc);
+              else mma_f16(tmem_base, a1d + 2 * kk, bd + 2 * kk, idesc, acc);
+            } else if (kPair) {
               mma_i8_pair(tmem_base, a1d + 2 * kk, bd + 2 * kk, idesc, acc);
               mma_i8_pair(tmem_base + kP8TileN, a2d + 2 * kk, bd + 2 * kk, idesc, acc);
             } else {
@@ -200,10 +207,13 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
       int mt, nt;
       tile_of(tile_mn, mt, nt);
       const int row0 = mt * kP8TileM + quad * 32, row = row0 + lane;
-      const float a_i = row < p.M ? __ldg(p.alpha + row) : 0.0f, b_i = row < p.M ? __ldg(p.beta + row) : 0.0f;
+      float a_i = 0.0f, b_i = 0.0f;
+      if constexpr (!kBase) {
+        if (row < p.M) { a_i = __ldg(p.alpha + row); b_i = __ldg(p.beta + row); }
+      }
       const int col_base = nt * kP8TileN + part * 64;
       const int col_w = col_base + lane;
-      float sw_next = (lane < ccols && col_w < p.N) ? __ldg(p.w_scale + col_w) : 0.0f;
+      float sw_next = (!kBase && lane < ccols && col_w < p.N) ? __ldg(p.w_scale + col_w) : 0.0f;
       ok = wait_bounded(&tfull_bar, it & 1, abort, p.status);
       if (!ok) break;
       tc_fence_after();
@@ -216,14 +226,28 @@ gemm_w8a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __g
         uint32_t o[16];
         const int col = col_base + c0;
         const float sw_cur = sw_next;
-        sw_next = (lane < ccols && c0 + ccols < cend && col_w + c0 + ccols < p.N) ? __ldg(p.w_scale + col_w + c0 + ccols) : 0.0f;
+        sw_next = (!kBase && lane < ccols && c0 + ccols < cend && col_w + c0 + ccols < p.N) ? __ldg(p.w_scale + col_w + c0 + ccols) : 0.0f;
 #pragma unroll
         for (int hsub = 0; hsub < 2; ++hsub) {       // 16 accumulator columns per load
           if (hsub == 1 && p.ytype != MSD_OUT_BF16) break;
           uint32_t v1[16], v2[16];
           tmem_ld16(trow + c0 + 16 * hsub, v1);
-          tmem_ld16(trow + kP8TileN + c0 + 16 * hsub, v2);
+          if constexpr (!kBase) tmem_ld16(trow + kP8TileN + c0 + 16 * hsub, v2);
           tmem_ld_wait();
+          if constexpr (kBase) {
+            // the FP32 sums as they are, rounded once to the output type
+            if (p.ytype == MSD_OUT_BF16) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v1[2 * j]), __uint_as_float(v1[2 * j + 1]));
+                o[8 * hsub + j] = *reinterpret_cast<const uint32_t*>(&h);
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) o[j] = v1[j];
+            }
+            continue;
+          }
           if (p.acc_dbg && row < p.M) {
             for (int j = 0; j < 16 && col + 16 * hsub + j < p.N; ++j) {
               p.acc_dbg[static_cast<long long>(row) * p.N + col + 16 * hsub + j] = static_cast<int32_t>(v1[j]);
@@ -291,11 +315,12 @@ struct GemmP8Plan {
   size_t off_q1, off_q2, off_alpha, off_beta, off_part, bytes;
 };
 
-static GemmP8Plan plan_p8(int64_t M, int64_t N, int64_t K) {
+// base: the dequantize-to-BF16 comparison path (K counted in bytes of BF16; off_q1 holds the BF16 weights)
+static GemmP8Plan plan_p8(int64_t M, int64_t N, int64_t K, bool base = false) {
   GemmP8Plan pl;
   pl.m_tiles = static_cast<int>((M + kP8TileM - 1) / kP8TileM);
   pl.n_tiles = static_cast<int>((N + kP8TileN - 1) / kP8TileN);
-  pl.kstages = static_cast<int>((K + kP8BlockK - 1) / kP8BlockK);
+  pl.kstages = static_cast<int>(((base ? 2 * K : K) + kP8BlockK - 1) / kP8BlockK);
   const long long tiles = static_cast<long long>(pl.m_tiles) * pl.n_tiles;
   // Few output tiles and a long K (a few hundred rows on a narrow layer): split K so that there is about one work item
   // per SM, each at least eight stages long; the FP32 partial results are added by a second kernel.
@@ -313,8 +338,8 @@ static GemmP8Plan plan_p8(int64_t M, int64_t N, int64_t K) {
   const long long items = tiles * pl.ksplit;
   pl.grid = static_cast<int>(items < sm_count() ? items : sm_count());
   size_t off = 0;
-  pl.off_q1 = off;    off = round_up(off + static_cast<size_t>(M) * K, 1024);
-  pl.off_q2 = off;    off = round_up(off + static_cast<size_t>(M) * K, 1024);
+  pl.off_q1 = off;    off = round_up(off + (base ? static_cast<size_t>(N) * K * 2 : static_cast<size_t>(M) * K), 1024);
+  pl.off_q2 = off;    off = round_up(off + (base ? 0 : static_cast<size_t>(M) * K), 1024);
   pl.off_alpha = off; off = round_up(off + static_cast<size_t>(M) * sizeof(float), 1024);
   pl.off_beta = off;  off = round_up(off + static_cast<size_t>(M) * sizeof(float), 1024);
   pl.off_part = off;
@@ -324,13 +349,30 @@ static GemmP8Plan plan_p8(int64_t M, int64_t N, int64_t K) {
 }
 
 size_t w8_prefill_workspace_bytes(int64_t M, int64_t N, int64_t K) { return plan_p8(M, N, K).bytes; }
+size_t w8_prefill_base_workspace_bytes(int64_t M, int64_t N, int64_t K) { return plan_p8(M, N, K, true).bytes; }
+
+static msd_status_t p8_launch(bool base, const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N, int64_t K,
+                              void* y, int ytype, int32_t* acc_dbg, float c1, float c2, void* workspace, size_t workspace_bytes,
+                              cudaStream_t s);
 
 // Arguments already checked by the caller (msd_gemm_w8a16_ex); M > 128.
 msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N, int64_t K,
                                void* y, int ytype, int32_t* acc_dbg, float c1, float c2, void* workspace,
                                size_t workspace_bytes, cudaStream_t s) {
+  return p8_launch(false, x_bf16, w, w_scale, M, N, K, y, ytype, acc_dbg, c1, c2, workspace, workspace_bytes, s);
+}
+// The comparison path for M > 128 (msd_gemm_dequant_bf16): weights dequantized to BF16 in the workspace, then the same
+// pipeline as a BF16 GEMM with FP32 accumulation.
+msd_status_t w8_prefill_base_launch(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N, int64_t K,
+                                    void* y, int ytype, void* workspace, size_t workspace_bytes, cudaStream_t s) {
+  return p8_launch(true, x_bf16, w, w_scale, M, N, K, y, ytype, nullptr, 0.0f, 0.0f, workspace, workspace_bytes, s);
+}
+
+static msd_status_t p8_launch(bool base, const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N, int64_t K,
+                              void* y, int ytype, int32_t* acc_dbg, float c1, float c2, void* workspace, size_t workspace_bytes,
+                              cudaStream_t s) {
   if (static_cast<long long>((M + kP8TileM - 1) / kP8TileM) * ((N + kP8TileN - 1) / kP8TileN) > 0x7FFFFFFFLL) return MSD_ERR_BAD_SHAPE;
-  const GemmP8Plan pl = plan_p8(M, N, K);
+  const GemmP8Plan pl = plan_p8(M, N, K, base);
   if (workspace_bytes < pl.bytes) return MSD_ERR_WORKSPACE_TOO_SMALL;
   unsigned* status = device_status_ptr();
   if (!status) return MSD_ERR_CUDA;
@@ -339,8 +381,14 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
   int8_t* q2 = reinterpret_cast<int8_t*>(ws + pl.off_q2);
   float* alpha = reinterpret_cast<float*>(ws + pl.off_alpha);
   float* beta = reinterpret_cast<float*>(ws + pl.off_beta);
-  msd_status_t st = launch_decompose_int8(x_bf16, M, K, K, q1, q2, alpha, beta, c1, c2, s);
+  msd_status_t st = MSD_OK;
+  if (base) st = launch_dequant_w8_to_bf16(w, w_scale, N, K, q1, s);
+  else st = launch_decompose_int8(x_bf16, M, K, K, q1, q2, alpha, beta, c1, c2, s);
   if (st != MSD_OK) return st;
+  // operand matrices as bytes: [M, kb] activations (components, or the BF16 x itself) and [N, kb] weights
+  const uint64_t kb = static_cast<uint64_t>(base ? 2 * K : K);
+  const void* a1_ptr = base ? x_bf16 : static_cast<const void*>(q1);
+  const void* b_ptr = base ? static_cast<const void*>(q1) : static_cast<const void*>(w);
 
   // with a K split (not when the INT32 accumulators are asked for: they exist only unsplit) the kernel writes FP32
   // partial results, split s at rows s * part_rows ..., and the reduce kernel produces y
@@ -362,9 +410,9 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
     const bool want = (pair_tiles + clusters - 1) / clusters <= (tiles + sm_count() - 1) / sm_count();
     use_pair = can && (forced >= 0 ? forced != 0 : want);
   }
-  if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, q1, K, M, K, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, q2, K, M, K, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !encode_tmap_2d(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, K, N, K, kP8BlockK, use_pair ? kP8TileN / 2 : kP8TileN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+  if (!encode_tmap_2d(&tmap_a1, CU_TENSOR_MAP_DATA_TYPE_UINT8, a1_ptr, kb, M, kb, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_a2, CU_TENSOR_MAP_DATA_TYPE_UINT8, base ? a1_ptr : static_cast<const void*>(q2), kb, M, kb, kP8BlockK, kP8TileM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !encode_tmap_2d(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b_ptr, kb, N, kb, kP8BlockK, use_pair ? kP8TileN / 2 : kP8TileN, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !encode_tmap_2d(&tmap_y, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, split ? static_cast<void*>(part) : y,
                       static_cast<uint64_t>(N), split ? part_rows * ksplit : static_cast<uint64_t>(M),
                       static_cast<uint64_t>(N) * (ybf ? 2 : 4), ybf ? 32 : 16, 32, CU_TENSOR_MAP_SWIZZLE_64B))
@@ -378,7 +426,7 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
   {
     // A wave of CTAs either shares a few weight tiles and sweeps the token tiles (token tile fastest) or the other way
     // round; the operand that is swept should be the one that stays in L2 (40 MB assumed usable for it).
-    const double l2 = 40.0 * 1024 * 1024, a_bytes = 2.0 * static_cast<double>(M) * K, w_bytes = static_cast<double>(N) * K;
+    const double l2 = 40.0 * 1024 * 1024, a_bytes = 2.0 * static_cast<double>(M) * K, w_bytes = (base ? 2.0 : 1.0) * static_cast<double>(N) * K;
     const bool n_fast = a_bytes <= l2 ? false : (w_bytes <= l2 ? true : a_bytes > w_bytes);
     p.n_fastest = n_fast;
   }
@@ -387,7 +435,9 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(gemm_w8a16_prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes)) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_w8a16_prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_pair)) != cudaSuccess)
+        cudaFuncSetAttribute(gemm_w8a16_prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_pair)) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w8a16_prefill_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes)) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w8a16_prefill_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_pair)) != cudaSuccess)
       return MSD_ERR_CUDA;
     attr_done = true;
   }
@@ -395,14 +445,18 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
   if (use_pair) {
     const long long pair_tiles = static_cast<long long>((pl.m_tiles + 1) / 2) * pl.n_tiles;
     const int clusters = static_cast<int>(pair_tiles < sm_count() / 2 ? pair_tiles : sm_count() / 2);
-    if (launch_pdl_cluster(gemm_w8a16_prefill_kernel<true>, dim3(2 * clusters), dim3(kP8Threads), smem_pair, s, pdl, 2u, tmap_a1, tmap_a2, tmap_b, tmap_y, p) != cudaSuccess)
-      return MSD_ERR_CUDA;
+    const cudaError_t pe = base
+        ? launch_pdl_cluster(gemm_w8a16_prefill_kernel<true, true>, dim3(2 * clusters), dim3(kP8Threads), smem_pair, s, pdl, 2u, tmap_a1, tmap_a2, tmap_b, tmap_y, p)
+        : launch_pdl_cluster(gemm_w8a16_prefill_kernel<true>, dim3(2 * clusters), dim3(kP8Threads), smem_pair, s, pdl, 2u, tmap_a1, tmap_a2, tmap_b, tmap_y, p);
+    if (pe != cudaSuccess) return MSD_ERR_CUDA;
     return MSD_OK;
   }
   const long long items = static_cast<long long>(pl.m_tiles) * pl.n_tiles * ksplit;
   const int grid = static_cast<int>(items < sm_count() ? items : sm_count());
-  if (launch_pdl(gemm_w8a16_prefill_kernel<false>, dim3(grid), dim3(kP8Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p) != cudaSuccess)
-    return MSD_ERR_CUDA;
+  const cudaError_t le = base
+      ? launch_pdl(gemm_w8a16_prefill_kernel<false, true>, dim3(grid), dim3(kP8Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p)
+      : launch_pdl(gemm_w8a16_prefill_kernel<false>, dim3(grid), dim3(kP8Threads), smem_bytes, s, pdl, tmap_a1, tmap_a2, tmap_b, tmap_y, p);
+  if (le != cudaSuccess) return MSD_ERR_CUDA;
   if (split) return launch_ksplit_reduce(part, ksplit, static_cast<int64_t>(part_rows) * N, M, N, y, ytype, s, pdl);
   return MSD_OK;
 }

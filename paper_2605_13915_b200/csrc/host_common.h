@@ -95,6 +95,13 @@ msd_status_t w8_prefill_launch(const void* x_bf16, const int8_t* w, const float*
                                void* y, int ytype, int32_t* acc_dbg, float c1, float c2, void* workspace,
                                size_t workspace_bytes, cudaStream_t stream);
 
+// The comparison path (dequantize to BF16, then a BF16 GEMM) for M > 128 rows, and the kernel launch that expands the
+// INT8 weights to bf16(w_scale[n] * w[n,k]) (gemm_w8a16.cu).
+size_t w8_prefill_base_workspace_bytes(int64_t M, int64_t N, int64_t K);
+msd_status_t w8_prefill_base_launch(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N, int64_t K,
+                                    void* y, int ytype, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+msd_status_t launch_dequant_w8_to_bf16(const int8_t* w, const float* w_scale, int64_t N, int64_t K, void* out_bf16, cudaStream_t stream);
+
 // A scale relayout that rides along with the MXFP4 decomposition kernel (extra CTAs of the same launch): row-major
 // E8M0 scales src[rows, kblocks] -> 512-byte blocks at dst, `row_blocks` = 2 x number of row tiles of `tile_rows` rows.
 struct SfRelayout {

@@ -241,3 +241,31 @@ def test_prefill_single_cta_and_cta_pair_kernels(pair, M, N, K, monkeypatch):
     c = inputs.gemm_w8_case(M, N, K, seed=11)
     _check(c, torch.float32)
     _check(c, torch.bfloat16)
+
+
+@pytest.mark.parametrize("M,N,K,pair,ksplit", [(129, 256, 128, -1, -1), (300, 520, 448, 0, -1), (300, 520, 448, 1, -1),
+                                               (640, 1288, 192, -1, -1), (256, 264, 4096, 0, 4)])
+def test_dequant_bf16_comparison_kernel_many_rows(M, N, K, pair, ksplit):
+    """The comparison path beyond 128 rows: weights expanded to BF16, then the many-row pipeline as a BF16 x BF16 GEMM
+    with FP32 accumulation (single-CTA and CTA-pair kernels, K split): against the oracle's dequantize-to-BF16 product,
+    FP32 and BF16 outputs; and MSD is the more accurate of the two against the FP64 product."""
+    if pair >= 0:
+        binding.debug_set_option("MSD_P8_PAIR", pair)
+    if ksplit >= 0:
+        binding.debug_set_option("MSD_P8_KSPLIT", ksplit)
+    c = inputs.gemm_w8_case(M, N, K, seed=9 + M)
+    xd, wd, sd = bf16_dev(c.x), dev(c.w), dev(c.w_scale)
+    ref = oracle.gemm_dequant_bf16_w8(c.x, c.w, c.w_scale)
+    for _ in range(2):
+        y = binding.gemm_dequant_bf16(xd, wd, sd, out_dtype=torch.float32)
+        torch.cuda.synchronize()
+        binding.last_device_status()
+        assert rel_row_err(y.cpu().numpy(), ref).max() <= TOL
+    yb = binding.gemm_dequant_bf16(xd, wd, sd, out_dtype=torch.bfloat16)
+    torch.cuda.synchronize()
+    got = oracle.bf16_bits_to_f64(bf16_bits(yb))
+    n = np.linalg.norm(ref, axis=1, keepdims=True)
+    assert np.all(np.abs(got - ref) <= TOL * n + np.abs(ref) * 2.0 ** -8)
+    truth = oracle.gemm_ref_w8(c.x, c.w, c.w_scale)
+    msd = binding.gemm_w8a16(xd, wd, sd, out_dtype=torch.float32).cpu().numpy()
+    assert np.linalg.norm(msd - truth) <= np.linalg.norm(y.cpu().numpy() - truth)
