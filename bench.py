@@ -616,7 +616,7 @@ def measure_configs(torch, binding, device, capture, timed_clocked, peaks, peak_
                                             frac_of_2x_measured_bf16=round(po * 1e3 / (2 * bf16), 3))}
         # the comparison path as this library's own kernels: weights expanded to BF16, then the same pipeline as a BF16 GEMM
         wsb = binding.workspace(binding.gemm_dequant_bf16_workspace_bytes(M, N, K), device)
-        tdq, _ = per_call_us(lambda: binding.gemm_dequant_bf16(x, w, s, ws=wsb), reps=2)
+        tdq, _ = per_call_us(lambda: binding.gemm_dequant_bf16(x, w8, s8, ws=wsb), reps=2)
         entry["comparison_dequant_bf16_kernel"] = {"us": round(tdq, 1), "msd_speedup": round(tdq / t, 2),
                                                    "note": "msd_gemm_dequant_bf16: dequantize kernel + BF16 tcgen05 GEMM (ours)"}
         del wsb
