@@ -570,9 +570,19 @@ def measure_configs(torch, binding, device, capture, timed_clocked, peaks, peak_
             it[0] += 1
             wq, sc = ws[it[0] % 4]
             binding.gemm_w8a16(x, wq, sc, ws=wsp_m, out=y)
-        (tb, _), (tm, _) = per_call_us(f_base), per_call_us(f_msd)
-        base[f"M16_N{N}_K{K}"] = {"dequant_bf16_us": round(tb, 2), "msd_us": round(tm, 2), "speedup": round(tb / tm, 2)}
+        wsp_f = binding.workspace(max(1024, int(binding.lib().msd_gemm_w8a16_fused_dequant_workspace_bytes(16, N, K))), device)
+
+        def f_fused():
+            it[0] += 1
+            wq, sc = ws[it[0] % 4]
+            binding.gemm_w8a16_fused_dequant(x, wq, sc, ws=wsp_f, out=y)
+        (tb, _), (tm, _), (tf, _) = per_call_us(f_base), per_call_us(f_msd), per_call_us(f_fused)
+        base[f"M16_N{N}_K{K}"] = {"dequant_bf16_us": round(tb, 2), "fused_dequant_us": round(tf, 2), "msd_us": round(tm, 2),
+                                  "speedup": round(tb / tm, 2), "speedup_vs_fused_dequant": round(tf / tm, 2)}
         del ws
+    base["note"] = ("dequant_bf16 = msd_gemm_dequant_bf16 (weights written back as BF16, then a BF16 GEMM); fused_dequant = "
+                    "msd_gemm_w8a16_fused_dequant (INT8 weights converted inside the GEMM; bound by shared-memory traffic: "
+                    "every weight byte crosses shared memory about seven times)")
     extras["w8a16_vs_dequant_bf16_kernel"] = base
 
     # ---- extras: W4A16 at the decode sweep's shapes, M = 16 ----

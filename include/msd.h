@@ -194,6 +194,21 @@ msd_status_t msd_gemm_dequant_bf16(const void* x_bf16, const int8_t* w, const fl
                                    size_t workspace_bytes, void* stream);
 
 /*
+ * The stronger comparison path: dequantization fused into the GEMM, as weight-only-quantization kernels do it
+ * (Sec. 2.3).  The INT8 weights are read once, converted to BF16 inside the kernel (exact) and multiplied against the
+ * BF16 activations with FP32 accumulation; the weight scale is applied to the sums:
+ *   y[m,n] = w_scale[n] * sum_k x[m,k] * w[n,k].
+ * No decomposition, no rounding of the weights: it is more accurate than msd_gemm_dequant_bf16 and moves the same
+ * bytes as msd_gemm_w8a16.  Decode regime only: 1 <= M <= 128; K % 64 == 0; N % 8 == 0; pointers as for msd_gemm_w8a16.
+ * workspace: >= msd_gemm_w8a16_fused_dequant_workspace_bytes(M,N,K) (FP32 partial results when K is split), 1024-byte
+ * aligned, no initialisation needed.  Errors as msd_gemm_w8a16; shapes it cannot stage -> MSD_ERR_UNSUPPORTED.
+ */
+size_t msd_gemm_w8a16_fused_dequant_workspace_bytes(int64_t M, int64_t N, int64_t K);
+msd_status_t msd_gemm_w8a16_fused_dequant(const void* x_bf16, const int8_t* w, const float* w_scale, int64_t M, int64_t N,
+                                          int64_t K, void* y, msd_out_t ytype, void* workspace, size_t workspace_bytes,
+                                          void* stream);
+
+/*
  * W4A16 MSD linear layer (Alg. 2 + Tab. mxfp4-compute): both MXFP4 components are multiplied against the
  * MXFP4 weight by block-scaled FP4 MMAs accumulating in FP32,
  *   y[i,n] = sum_blocks 2^(e1+ew) <q1,w> + 2^(e2+ew) <q2,w>.

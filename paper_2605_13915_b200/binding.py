@@ -48,6 +48,8 @@ _SIGS = {
     "msd_gemm_w8a16_host": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_gemm_dequant_bf16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_dequant_bf16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
+    "msd_gemm_w8a16_fused_dequant_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "msd_gemm_w8a16_fused_dequant": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_gemm_w4a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "msd_gemm_w4a16": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, C.c_int, _vp, _sz, _vp]),
     "msd_w4a16_prepared_scales_bytes": (_sz, [_i32, _i64, _i64]),
@@ -280,6 +282,21 @@ def gemm_dequant_bf16(x, w, w_scale, out_dtype=torch.bfloat16, ws=None):
     _check(lib().msd_gemm_dequant_bf16(_ptr(x), _ptr(w), _ptr(w_scale), M, N, K, _ptr(y),
                                        OUT_BF16 if out_dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream()),
            "msd_gemm_dequant_bf16")
+    return y
+
+
+def gemm_w8a16_fused_dequant(x, w, w_scale, out_dtype=torch.bfloat16, ws=None, out=None):
+    """Comparison kernel: INT8 weights converted to BF16 inside the GEMM (M <= 128)."""
+    _need_cuda(x, w, w_scale)
+    M, K = x.shape
+    N = w.shape[0]
+    if ws is None:
+        ws = workspace(max(1024, int(lib().msd_gemm_w8a16_fused_dequant_workspace_bytes(M, N, K))), x.device)
+    y = out if out is not None else _empty((M, N), out_dtype, x.device)
+    wp, wb = _ws_ptr(ws)
+    _check(lib().msd_gemm_w8a16_fused_dequant(_ptr(x), _ptr(w), _ptr(w_scale), M, N, K, _ptr(y),
+                                              OUT_BF16 if y.dtype == torch.bfloat16 else OUT_FP32, wp, wb, _stream()),
+           "msd_gemm_w8a16_fused_dequant")
     return y
 
 

@@ -269,3 +269,24 @@ def test_dequant_bf16_comparison_kernel_many_rows(M, N, K, pair, ksplit):
     truth = oracle.gemm_ref_w8(c.x, c.w, c.w_scale)
     msd = binding.gemm_w8a16(xd, wd, sd, out_dtype=torch.float32).cpu().numpy()
     assert np.linalg.norm(msd - truth) <= np.linalg.norm(y.cpu().numpy() - truth)
+
+
+@pytest.mark.parametrize("M,N,K", [(16, 1024, 1024), (1, 4096, 4096), (128, 640, 1536), (5, 12000, 512), (33, 264, 2048),
+                                   (16, 14336, 4096), (64, 4096, 2048)])
+def test_fused_dequant_comparison_kernel(M, N, K):
+    """The stronger comparison arm: INT8 weights converted to BF16 inside the GEMM, scale applied to the FP32 sums.
+    Row bands and K-split tiles, ragged last band, M not a multiple of 16.  Against the FP64 product with the
+    dequantized weights (the kernel rounds nothing but the FP32 accumulation and the output)."""
+    c = inputs.gemm_w8_case(M, N, K, seed=31 + M)
+    xd, wd, sd = bf16_dev(c.x), dev(c.w), dev(c.w_scale)
+    truth = oracle.gemm_ref_w8(c.x, c.w, c.w_scale)
+    for _ in range(2):
+        y = binding.gemm_w8a16_fused_dequant(xd, wd, sd, out_dtype=torch.float32)
+        torch.cuda.synchronize()
+        binding.last_device_status()
+        assert rel_row_err(y.cpu().numpy(), truth).max() <= 1e-5
+    yb = binding.gemm_w8a16_fused_dequant(xd, wd, sd, out_dtype=torch.bfloat16)
+    torch.cuda.synchronize()
+    got = oracle.bf16_bits_to_f64(bf16_bits(yb))
+    n = np.linalg.norm(truth, axis=1, keepdims=True)
+    assert np.all(np.abs(got - truth) <= 1e-5 * n + np.abs(truth) * 2.0 ** -8)
