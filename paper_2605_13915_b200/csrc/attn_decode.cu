@@ -201,8 +201,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   __shared__ float red[2][4][kNH + 1];             // per-warp tile maxima, double buffered by tile parity
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int split = blockIdx.x;
-  int unit = blockIdx.y;
+  // units along x (launched first), splits along y: the early splits of every sequence, which are always full, start
+  // before the last, shorter ones (and the two head groups of a wide group, which read the same tiles, side by side)
+  const int split = blockIdx.y;
+  int unit = blockIdx.x;
   const int grp = unit % p.groups; unit /= p.groups;
   const int hk = unit % p.Hkv;
   const int b = unit / p.Hkv;
@@ -672,6 +674,8 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
   constexpr int kDVT = 4;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // splits along x, units along y (the two head groups of a sequence split, which read the same tiles, a few CTAs apart:
+  // launched side by side they miss L2 together, measured 4 us slower)
   const int split = blockIdx.x;
   int unit = blockIdx.y;
   const int grp = unit % p.groups; unit /= p.groups;
@@ -1407,6 +1411,7 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   int chunk_tiles = option(OPT_ATTN_CHUNK_TILES);       // testing aid
   if (chunk_tiles < 1) chunk_tiles = pl->Rp <= 16 ? 16 : 32;
   while (chunk_tiles > 2 && units * ((tiles + chunk_tiles - 1) / chunk_tiles) < static_cast<long long>(sm_count()) * 4) chunk_tiles >>= 1;
+  while ((tiles + chunk_tiles - 1) / chunk_tiles > 65535) chunk_tiles <<= 1;      // splits may run along the grid's y axis
   int ns = (tiles + chunk_tiles - 1) / chunk_tiles;
   if (ns < 1) ns = 1;
   if (const int forced = option(OPT_ATTN_SPLITS); forced >= 1) {      // testing aid: a given number of splits
@@ -1572,7 +1577,9 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
       if (free_slot >= 0) done[free_slot] = reinterpret_cast<void*>(kernel);
     }
   }
-  dim3 grid(pl.n_splits, B * Hkv * pl.groups);
+  // narrow groups: units along x; wide groups: splits along x (see the kernels)
+  dim3 grid(B * Hkv * pl.groups, pl.n_splits);
+  if (block_threads > kAttnThreads) grid = dim3(pl.n_splits, B * Hkv * pl.groups);
   if (block_threads > kAttnThreads) {
     // wide head groups: the stacked Q operands come from a kernel of their own, the attention kernel is its
     // programmatic dependent (its CTAs start their KV loads while it runs)
