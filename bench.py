@@ -586,8 +586,7 @@ def measure_configs(torch, binding, device, capture, timed_clocked, peaks, peak_
                                   "speedup": round(tb / tm, 2), "speedup_vs_fused_dequant": round(tf / tm, 2)}
         del ws
     base["note"] = ("dequant_bf16 = msd_gemm_dequant_bf16 (weights written back as BF16, then a BF16 GEMM); fused_dequant = "
-                    "msd_gemm_w8a16_fused_dequant (INT8 weights converted inside the GEMM; bound by shared-memory traffic: "
-                    "every weight byte crosses shared memory about seven times)")
+                    "msd_gemm_w8a16_fused_dequant (INT8 weights converted to BF16 inside the GEMM, into tensor memory)")
     extras["w8a16_vs_dequant_bf16_kernel"] = base
 
     # ---- extras: W4A16 at the decode sweep's shapes, M = 16 ----

@@ -1,17 +1,20 @@
 // W8A16 comparison kernel with the dequantization fused into the GEMM (the stronger of the two baselines MSD is measured
 // against; Sec. 2.3 "kernel optimization methods reduce its cost"): the INT8 weights are read from HBM once, as in MSD,
-// converted to BF16 by four warps on their way from the TMA staging buffer to the MMA operand buffer, and multiplied
-// against the BF16 activations with FP32 accumulation (tcgen05.mma kind::f16); the per-channel weight scale is applied
-// to the sums.  No decomposition kernel, no second component:
+// converted to BF16 (exactly) by twelve warps on their way from the TMA staging buffer into TENSOR MEMORY, from where they are
+// the A operand of BF16 x BF16 -> FP32 MMAs (tcgen05.mma kind::f16, A in tensor memory, the BF16 activations as B in
+// shared memory); the per-channel weight scale is applied to the sums.  No decomposition kernel, no second component:
 //   y[m,n] = w_scale[n] * sum_k x[m,k] * float(w[n,k])          (the INT8 values are exact in BF16)
 // Decode regime only (M <= 128).  The weight rows sit on the MMA M axis as in the MSD decode kernel: one band of up to
 // 128 rows per CTA when the bands are at least 64 rows high, else 128-row tiles with the K stages of a tile split over
 // several CTAs (FP32 partial results, added by ksplit_reduce_kernel in a fixed order).
 //
 // Warp roles: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 2..13 = converters; 2..5 then run the epilogue.
-// A stage holds kw K blocks of 64 elements: INT8 weights [kw][rows][64 B] (no swizzle, read linearly by the converters)
-// and BF16 activations [kw][Mp][128 B] (128-byte swizzle, read by the MMAs).  The converters write the weights as BF16
-// chunks [rows][128 B] in the 128-byte-swizzled K-major layout into one of two operand buffers.
+// A stage holds kw K blocks of 64 elements: INT8 weights [kw][rows][64 B] (64-byte swizzle: a converter thread reads
+// its own row 16 bytes at a time without bank conflicts) and BF16 activations [kw][Mp][128 B] (128-byte swizzle).
+// A converter thread owns one weight row (= tensor-memory lane) of one K block: 64 bytes in, 32 columns of
+// two BF16 values out (tcgen05.st).  Two sets of kw x 32 columns alternate.  (With the converted weights written to shared memory
+// instead, every weight byte crossed the shared-memory port seven times and the kernel ran at 27-29 us where this one
+// needs less; that version is what the TMA-to-MMA path of MSD avoids.)
 #include <cuda_bf16.h>
 
 #include "host_common.h"
@@ -19,10 +22,12 @@
 
 namespace msd {
 
-constexpr int kFzConvWarps = 12;             // three per warp scheduler: one alone cannot hide its own latencies
+constexpr int kFzConvWarps = 12;             // three per warp scheduler and tensor-memory lane quadrant
 constexpr int kFzThreads = 64 + 32 * kFzConvWarps;
 constexpr int kFzMaxStages = 8;
 constexpr int kFzBlockK = 64;               // elements per K block: 64 B of INT8 weights, 128 B of BF16 activations
+constexpr int kFzAccCols = 128;             // tensor-memory columns of the accumulator; the operand sets follow
+constexpr int kFzTmemCols = 512;
 
 struct FzParams {
   int M, Mp, N, K;
@@ -30,9 +35,8 @@ struct FzParams {
   int bands;             // work items along N
   int ksplit, kper;      // K splits per band and K stages per split
   int kstages;           // K stages in all: ceil(K / (64 kw))
-  int kw;                // K blocks per stage
+  int kw;                // K blocks per stage: 3 or 6 (a multiple of the three converter warps per lane quadrant)
   int stages;            // pipeline stages
-  int tmem_cols;
   int ytype;
   const float* w_scale;
   void* y;
@@ -40,11 +44,13 @@ struct FzParams {
   unsigned* status;
 };
 
-// 16 signed bytes -> 16 BF16 values (exact).  x ^ 0x80 is the byte of x + 128; 0x4B0000uu is the float 2^23 + uu, so
-// one byte permute and one subtraction give float(x), whose upper half is its BF16 form (|x| <= 128 has 8 significant bits).
-__device__ __forceinline__ void cvt_s8x16_bf16(const uint4& v, uint4& lo, uint4& hi) {
+// 16 signed bytes -> 16 BF16 values (exact), two per word.  x ^ 0x80 is the byte of x + 128; 0x4B0000uu is the float
+// 2^23 + uu, so one byte permute and one subtraction give float(x), whose upper half is its BF16 form (|x| <= 128 has 8
+// significant bits): 2.75 instructions per element.  (The FP16 route - 0x64uu is 1024 + uu, one packed subtraction per
+// two elements, 1.25 instructions per element - needs an FP16 A operand against the BF16 activations; an MMA of
+// kind::f16 with the two operand formats set differently raised an illegal-instruction error, so both are BF16.)
+__device__ __forceinline__ void cvt_s8x16_bf16(const uint4& v, uint32_t (&o)[8]) {
   const uint32_t w[4] = {v.x ^ 0x80808080u, v.y ^ 0x80808080u, v.z ^ 0x80808080u, v.w ^ 0x80808080u};
-  uint32_t o[8];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const float f0 = __uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7650)) - 8388736.0f;
@@ -54,8 +60,6 @@ __device__ __forceinline__ void cvt_s8x16_bf16(const uint4& v, uint4& lo, uint4&
     o[2 * i] = __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x7632);
     o[2 * i + 1] = __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x7632);
   }
-  lo = make_uint4(o[0], o[1], o[2], o[3]);
-  hi = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
 __global__ void __launch_bounds__(kFzThreads, 1)
@@ -72,8 +76,6 @@ gemm_w8a16_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   const int x_chunk_bytes = p.Mp * 128;
   const int stage_bytes = ((w_stage_bytes + 1023) & ~1023) + p.kw * x_chunk_bytes;
   const int x_off = (w_stage_bytes + 1023) & ~1023;
-  const int bf_chunk_bytes = p.band_h * 128;                             // one converted K block: [rows][128 B], whole swizzle atoms
-  uint8_t* bf_buf = smem + p.stages * stage_bytes;                       // two buffers of kw chunks
 
   const int band = blockIdx.x / p.ksplit, split = blockIdx.x - band * p.ksplit;
   const int row0 = band * p.band_h;
@@ -82,14 +84,14 @@ gemm_w8a16_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&conv_full[b], kFzConvWarps); mbar_init(&conv_free[b], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&conv_full[b], kFzConvWarps); mbar_init(&conv_free[b], 1); }     // the two operand sets
     mbar_init(&tfull_bar, 1);
     abort_flag = 0;
     mbar_init_fence();
     tma_prefetch_desc(&tmap_w);
     tma_prefetch_desc(&tmap_x);
   }
-  if (warp == 1) tmem_alloc(&tmem_base_slot, p.tmem_cols);
+  if (warp == 1) tmem_alloc(&tmem_base_slot, kFzTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -128,42 +130,53 @@ gemm_w8a16_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
         if (ok) ok = wait_bounded(&conv_full[b], (i >> 1) & 1, abort, p.status);       // its weights, converted
         if (!ok) break;
         tc_fence_after();
-        const uint64_t ad = op_desc + (smem_u32(bf_buf + b * p.kw * bf_chunk_bytes) >> 4);
+        const uint32_t at = tmem_base + kFzAccCols + b * (p.kw * 32);      // operand set b: 32 columns per K block
         const uint64_t xd = op_desc + (smem_u32(smem + s * stage_bytes + x_off) >> 4);
         for (int c = 0; c < p.kw; ++c) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k)        // 16 BF16 elements (32 bytes) per MMA
-            mma_f16(tmem_base, ad + ((c * bf_chunk_bytes) >> 4) + 2 * k, xd + ((c * x_chunk_bytes) >> 4) + 2 * k, idesc,
-                    (i > 0 || c > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < 4; ++k)        // 16 BF16 elements per MMA: 8 columns of A, 32 bytes of every B row
+            mma_f16_ts(tmem_base, at + c * 32 + k * 8, xd + ((c * x_chunk_bytes) >> 4) + 2 * k, idesc,
+                       (i > 0 || c > 0 || k > 0) ? 1u : 0u);
         }
         tc_commit(&empty_bar[s]);         // the stage (its activation chunks; the converters are long done with the weights)
-        tc_commit(&conv_free[b]);         // the operand buffer may be overwritten
+        tc_commit(&conv_free[b]);         // the operand set may be overwritten
       }
       if (ok) tc_commit(&tfull_bar);
     }
   } else {
     // ------------------------------ converters (warps 2..13), then epilogue (warps 2..5) ------------------------------
-    const int t = threadIdx.x - 64;                 // 0 .. 32 kFzConvWarps - 1
-    const int pieces = p.band_h * 4;                // 16-byte pieces of one K block of the band
+    const int quad = warp & 3;                      // tensor-memory lane quadrant this warp may touch
+    const int grp = (warp - 2) >> 2;                // 0..2: which K blocks of a stage (c = grp, grp + 3)
+    const int r = quad * 32 + lane;                 // weight row of the band = tensor-memory lane
+    const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+    const int sw = (r >> 1) & 3;                    // 64-byte swizzle: the 16-byte piece index is XORed with (row / 2) % 4
     bool ok = true;
     for (int i = 0; i < nst && ok; ++i) {
       const int s = i % p.stages, b = i & 1;
       ok = wait_bounded(&full_bar[s], (i / p.stages) & 1, abort, p.status);
       if (ok && i >= 2) ok = wait_bounded(&conv_free[b], ((i >> 1) - 1) & 1, abort, p.status);
       if (!ok) break;
-      const uint4* src = reinterpret_cast<const uint4*>(smem + s * stage_bytes);
-      uint8_t* dstb = bf_buf + b * p.kw * bf_chunk_bytes;
-      for (int c = 0; c < p.kw; ++c) {
-        for (int q = t; q < pieces; q += 32 * kFzConvWarps) {
-          const int row = q >> 2, pc = q & 3;
-          uint4 lo, hi;
-          cvt_s8x16_bf16(src[c * pieces + q], lo, hi);
-          uint8_t* drow = dstb + c * bf_chunk_bytes + row * 128;
-          *reinterpret_cast<uint4*>(drow + (((2 * pc) ^ (row & 7)) << 4)) = lo;
-          *reinterpret_cast<uint4*>(drow + (((2 * pc + 1) ^ (row & 7)) << 4)) = hi;
+      tc_fence_after();
+      const uint8_t* src = smem + s * stage_bytes;
+      for (int c = grp; c < p.kw; c += 3) {
+        uint32_t o[32];
+        if (r < p.band_h) {
+          const uint8_t* row = src + (c * p.band_h + r) * kFzBlockK;
+#pragma unroll
+          for (int pc = 0; pc < 4; ++pc) {
+            uint32_t h[8];
+            cvt_s8x16_bf16(*reinterpret_cast<const uint4*>(row + ((pc ^ sw) << 4)), h);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) o[8 * pc + j] = h[j];
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[j] = 0u;     // rows past the band: zeros (their sums are never stored)
         }
+        tmem_st32(trow + kFzAccCols + b * (p.kw * 32) + c * 32, o);
       }
-      fence_proxy_async_smem();           // the tensor core reads what these threads wrote
+      tmem_st_wait();
+      tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&conv_full[b]);
     }
@@ -171,10 +184,9 @@ gemm_w8a16_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     if (ok && warp < 6) ok = wait_bounded(&tfull_bar, 0, abort, p.status);
     if (ok && warp < 6) {
       tc_fence_after();
-      const int quad = warp & 3, r = quad * 32 + lane, n = row0 + r;
+      const int n = row0 + r;
       const bool row_ok = r < p.band_h && n < p.N;
-      const float sw = row_ok ? __ldg(p.w_scale + n) : 0.0f;
-      const uint32_t trow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+      const float wsc = row_ok ? __ldg(p.w_scale + n) : 0.0f;
       for (int c0 = 0; c0 < p.Mp; c0 += 16) {
         uint32_t v[16];
         tmem_ld16(trow + c0, v);
@@ -184,7 +196,7 @@ gemm_w8a16_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
           for (int j = 0; j < 16; ++j) {
             const int m = c0 + j;
             if (m < p.M) {
-              const float val = sw * __uint_as_float(v[j]);
+              const float val = wsc * __uint_as_float(v[j]);
               if (p.ksplit > 1) p.part[(static_cast<size_t>(split) * p.M + m) * p.N + n] = val;
               else if (p.ytype == MSD_OUT_BF16) static_cast<__nv_bfloat16*>(p.y)[static_cast<size_t>(m) * p.N + n] = __float2bfloat16_rn(val);
               else static_cast<float*>(p.y)[static_cast<size_t>(m) * p.N + n] = val;
@@ -199,12 +211,12 @@ gemm_w8a16_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, p.tmem_cols);
+    tmem_dealloc(tmem_base, kFzTmemCols);
   }
 }
 
 struct FzPlan {
-  int Mp, band_h, bands, ksplit, kper, kstages, kw, stages, tmem_cols;
+  int Mp, band_h, bands, ksplit, kper, kstages, kw, stages;
   size_t smem_bytes, bytes;
 };
 
@@ -219,28 +231,25 @@ static FzPlan plan_fz(int64_t M, int64_t N, int64_t K) {
   pl.band_h = band_h;
   pl.bands = static_cast<int>((N + band_h - 1) / band_h);
   // K blocks per stage: wide stages read each weight row in longer runs; the activation chunks grow with M
-  pl.kw = pl.Mp <= 32 ? 4 : 2;         // (the two operand buffers hold kw converted chunks each: 13-16 KB per chunk)
-  while (pl.kw > 1 && static_cast<int64_t>(pl.kw) * kFzBlockK > K) pl.kw >>= 1;
+  // six K blocks per stage (two per converter warp; 2 x 192 operand columns + 128 accumulator columns = all of tensor
+  // memory), three where the activation chunks are large
+  pl.kw = pl.Mp <= 32 ? 6 : 3;
   pl.kstages = static_cast<int>((K + static_cast<int64_t>(pl.kw) * kFzBlockK - 1) / (static_cast<int64_t>(pl.kw) * kFzBlockK));
   pl.ksplit = 1;
   if (2 * pl.bands <= sms) {
     int want = sms / pl.bands;
-    if (want > pl.kstages / 4) want = pl.kstages / 4;
+    if (want > pl.kstages / 2) want = pl.kstages / 2;
     if (want > 1) pl.ksplit = want;
   }
   pl.kper = (pl.kstages + pl.ksplit - 1) / pl.ksplit;
   pl.ksplit = (pl.kstages + pl.kper - 1) / pl.kper;
   const size_t w_stage = round_up(static_cast<size_t>(pl.kw) * band_h * kFzBlockK, 1024);
   const size_t stage = w_stage + static_cast<size_t>(pl.kw) * pl.Mp * 128;
-  const size_t bf = 2 * static_cast<size_t>(pl.kw) * band_h * 128 + (128 - band_h) * 128;     // the MMA reads 128 rows from every chunk
   const size_t budget = 227 * 1024 - 2048 - 1024;
-  int stages = bf < budget ? static_cast<int>((budget - bf) / stage) : 0;
+  int stages = static_cast<int>(budget / stage);
   if (stages > kFzMaxStages) stages = kFzMaxStages;
   pl.stages = stages;
-  pl.smem_bytes = static_cast<size_t>(stages) * stage + bf + 1024;
-  int cols = 32;
-  while (cols < pl.Mp) cols <<= 1;
-  pl.tmem_cols = cols;
+  pl.smem_bytes = static_cast<size_t>(stages) * stage + 1024;
   pl.bytes = pl.ksplit > 1 ? round_up(static_cast<size_t>(pl.ksplit) * M * N * sizeof(float), 1024) : 1024;
   return pl;
 }
@@ -272,14 +281,14 @@ msd_status_t msd_gemm_w8a16_fused_dequant(const void* x_bf16, const int8_t* w, c
   CUtensorMap tmap_w, tmap_x;
   // weights: {64 B of a K block, rows, K blocks}; activations as bytes: {128 B of a K block, rows, K blocks}
   if (!encode_tmap_3d(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w, kFzBlockK, N, K / kFzBlockK, K, kFzBlockK, kFzBlockK,
-                      static_cast<uint32_t>(pl.band_h), static_cast<uint32_t>(pl.kw), CU_TENSOR_MAP_SWIZZLE_NONE) ||
+                      static_cast<uint32_t>(pl.band_h), static_cast<uint32_t>(pl.kw), CU_TENSOR_MAP_SWIZZLE_64B) ||
       !encode_tmap_3d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, x_bf16, 128, M, K / kFzBlockK, 2 * K, 128, 128,
                       static_cast<uint32_t>(pl.Mp), static_cast<uint32_t>(pl.kw), CU_TENSOR_MAP_SWIZZLE_128B))
     return MSD_ERR_CUDA;
   FzParams p;
   p.M = static_cast<int>(M); p.Mp = pl.Mp; p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.band_h = pl.band_h; p.bands = pl.bands; p.ksplit = pl.ksplit; p.kper = pl.kper; p.kstages = pl.kstages; p.kw = pl.kw;
-  p.stages = pl.stages; p.tmem_cols = pl.tmem_cols; p.ytype = ytype; p.w_scale = w_scale; p.y = y;
+  p.stages = pl.stages; p.ytype = ytype; p.w_scale = w_scale; p.y = y;
   p.part = static_cast<float*>(workspace); p.status = status;
   static bool attr_done = false;
   if (!attr_done) {
