@@ -1155,7 +1155,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       __syncwarp();
       if (lane == 0) mbar_arrive(&p_full[t & 1]);
       if (threadIdx.x == 64 && t >= 2 && t < 5) attn_mark(p, 5 + 6 * (t - 2));
-      // every softmax warp has written its part (and its verdict): did any reference have to move?
+      // every softmax warp has written its part (and said whether it saw a reference exceeded): did any have to move?
       ok = wait_bounded(&p_full[t & 1], (t >> 1) & 1, abort, p.status);
       if (!ok) break;
       if (threadIdx.x == 64 && t >= 2 && t < 5) attn_mark(p, 6 + 6 * (t - 2));
