@@ -670,7 +670,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
   // first chunks while the others are in flight was measured too: five short bursts of MMAs cost the issuing thread
   // far more than one long one.)
   constexpr bool kChunked = kFixDC == 5 && kFixDVT == 4 && !kPaged;
-  __shared__ __align__(8) uint64_t ck_empty[2][5];
+  __shared__ __align__(8) uint64_t ck_empty[2][5], ck_full[2][5];      // per stage and chunk: free again / landed
   constexpr int kDVT = 4;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -722,7 +722,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
     mbar_init(&o_full, 1); mbar_init(&o_last, 1); mbar_init(&p_redo, kNSW);
     if constexpr (kChunked)
       for (int s2 = 0; s2 < 2; ++s2)
-        for (int c = 0; c < 5; ++c) mbar_init(&ck_empty[s2][c], 1);
+        for (int c = 0; c < 5; ++c) { mbar_init(&ck_empty[s2][c], 1); mbar_init(&ck_full[s2][c], 1); }
     abort_flag = 0;
     flush_stamp[0] = 0; flush_stamp[1] = 0;
     mbar_init_fence();
@@ -761,8 +761,8 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
             if (i == 0) okp = wait_bounded(&s_full[st], ph ^ 1, abort, p.status);
             else okp = wait_bounded(&ck_empty[st][c], ph ^ 1, abort, p.status);
             if (!okp) break;
-            if (i == 0) mbar_arrive_expect_tx(&kv_full[st], 5 * kChunkBytes);
-            tma_load_3d(dst + c * kChunkBytes, &tmap_k, c * kChunk, hk, tok0, &kv_full[st]);
+            mbar_arrive_expect_tx(&ck_full[st][c], kChunkBytes);      // every chunk lands on a barrier of its own
+            tma_load_3d(dst + c * kChunkBytes, &tmap_k, c * kChunk, hk, tok0, &ck_full[st][c]);
           }
         }
       }
@@ -929,12 +929,35 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
         // memory and the score buffer q&1 read, i.e. P of tile q-2 written by every softmax warp (the slow path works
         // from registers).  The P buffer q&1 is free by then as well: KV tile q arrives in the stage that PV(q-2) gave
         // back chunk by chunk, so its arrival implies that PV(q-2) is complete.
+        // The K steps of a chunk are issued as soon as that chunk has landed, in the order the chunks are requested
+        // (rotary chunk first: it was free long before the value chunks): by the time the last chunk arrives only its
+        // own four MMAs are left to run.
+        const uint32_t k_hi = static_cast<uint32_t>(dk >> 32), q_hi = static_cast<uint32_t>(q_enc >> 32);
+        const uint32_t k_lo0 = static_cast<uint32_t>(dk) + smem_enc, q_lo0 = static_cast<uint32_t>(q_enc);
         for (; q < ntiles && ok; ++q) {
+          const int st = q & 1;
+          const uint32_t ph = (q >> 1) & 1;
           if (q >= 2) ok = wait_bounded(&p_full[q & 1], ((q - 2) >> 1) & 1, abort, p.status);
-          if (ok) ok = wait_bounded(&kv_full[q & 1], (q >> 1) & 1, abort, p.status);
           if (!ok) break;
-          if (q >= 2 && q < 5) attn_mark(p, 7 + 6 * (q - 2));
-          issue_qk(q);
+          const uint32_t d = tmem_base + (q & 1) * p.Rp;
+          const uint32_t k_lo = k_lo0 + static_cast<uint32_t>(st * (kv_stage_bytes >> 4));
+#pragma unroll
+          for (int i = 0; i < 5; ++i) {
+            const int c = (i == 0) ? 4 : i - 1;
+            ok = wait_bounded(&ck_full[st][c], ph, abort, p.status);
+            if (!ok) break;
+            if (i == 0 && q >= 2 && q < 5) attn_mark(p, 7 + 6 * (q - 2));
+            tc_fence_after();
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              if (c < 4 || k < last_steps) {
+                const uint32_t ka = k_lo + (c * (kChunkBytes >> 4) + 2 * k), qa = q_lo0 + (c * ((kWideSlots * 2 * kChunk) >> 4) + 2 * k);
+                if (i == 0 && k == 0) mma_i8_lohi<false>(d, ka, k_hi, qa, q_hi, idesc_qk);
+                else mma_i8_lohi<true>(d, ka, k_hi, qa, q_hi, idesc_qk);
+              }
+          }
+          if (!ok) break;
+          tc_commit(&s_full[q & 1]);
           if (q >= 2 && q < 5) attn_mark(p, q == 4 ? 30 : 23 + q);
         }
         v = ntiles;
@@ -1222,7 +1245,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
         if (hh == 0 && lane == 0) {
           const int st = t & 1;
           if (slow) ok = wait_bounded(&p_redo, (n_slow - 1) & 1, abort, p.status);      // every warp has drained and rewritten P
-          if (ok) ok = wait_bounded(&kv_full[st], (t >> 1) & 1, abort, p.status);      // (long complete: QK^T(t) has read the tile)
+          if (ok) ok = wait_bounded(&ck_full[st][wq], (t >> 1) & 1, abort, p.status);      // its value chunk (long landed: QK^T(t) has read the tile)
           if (ok) {
             tc_fence_after();
             if (wq == 0 && t >= 2 && t < 5) attn_mark(p, 8 + 6 * (t - 2));
