@@ -666,9 +666,10 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
   // Latent cache of 576 bytes per token with V aliased to its first 512 (the launcher picks this instantiation only
   // then): the two KV stages are given back chunk by chunk (five 128-byte-wide chunks of 16 KB): every chunk is
   // requested again as soon as its last reader is done - the rotary chunk after QK^T, value chunk j after the j-th
-  // 128-wide tile of PV - instead of the whole 80 KB stage waiting for the last PV MMA.  (Starting QK^T on a tile's
-  // first chunks while the others are in flight was measured too: five short bursts of MMAs cost the issuing thread
-  // far more than one long one.)
+  // 128-wide tile of PV - instead of the whole 80 KB stage waiting for the last PV MMA.  Every chunk lands on a barrier of
+  // its own and QK^T starts on a tile's first chunks while the others are in flight.  (While one thread issued both
+  // products that measured slower - five short bursts cost it far more than one long one; with PV issued elsewhere
+  // the thread has nothing else to do and the scores are ready 0.2-0.5 us earlier.)
   constexpr bool kChunked = kFixDC == 5 && kFixDVT == 4 && !kPaged;
   __shared__ __align__(8) uint64_t ck_empty[2][5], ck_full[2][5];      // per stage and chunk: free again / landed
   constexpr int kDVT = 4;
