@@ -52,8 +52,9 @@ typedef enum { MSD_OUT_BF16 = 0, MSD_OUT_FP32 = 1 } msd_out_t;
 const char* msd_status_string(msd_status_t s);
 
 /* Reads and clears the device status word after synchronising `stream`.  Returns MSD_OK, MSD_ERR_TIMEOUT
- * (some kernel gave up on a bounded wait; its outputs are invalid and its workspace must be re-initialised)
- * or MSD_ERR_CUDA. */
+ * (some kernel gave up on a bounded wait; its outputs are invalid and its workspace must be re-initialised),
+ * MSD_ERR_BAD_SHAPE (a kernel found device-side input that contradicts the sizes the call was given) or
+ * MSD_ERR_CUDA. */
 msd_status_t msd_last_device_status(void* stream);
 
 /* Self-test of the give-up path every device-side wait of this library has: launches a tiny kernel that waits, with
@@ -67,7 +68,9 @@ msd_status_t msd_debug_timeout_selftest(int64_t budget_cycles, void* stream);
  *   MSD_NO_PDL (1: no programmatic dependent launches), MSD_GEMM_MODE / MSD_GEMM_CTAS (work split and CTA count of the
  *   W8A16 decode kernel: 0 stream-K, 1 row bands, 2 clusters), MSD_P8_PAIR / MSD_P8_KSPLIT (W8A16 many-row kernel: CTA
  *   pairs, K split), MSD_W4_PAIR / MSD_W4_TILEN / MSD_W4_KSPLIT (W4A16 kernels), MSD_ATTN_SPLITS / MSD_ATTN_CHUNK_TILES
- *   (context splits of the attention kernels; msd_attn_decode_schedule reports the schedule in force). */
+ *   (context splits of the attention kernels; msd_attn_decode_schedule reports the schedule in force),
+ *   MSD_ATTN_BALANCED (1: the balanced split schedule for every shape that has a kernel for it, 0: never; a forced
+ *   split count or size switches it off as well). */
 msd_status_t msd_debug_set_option(const char* name, int32_t value);
 void msd_debug_reset_options(void);
 
@@ -287,7 +290,9 @@ msd_status_t msd_gemm_w4a16_e1m2(const void* x_bf16, const uint8_t* w_fp4, const
  *   total_tokens = T, the number of token rows the caches hold (>= cu_seqlens[B]); max_seqlen >= every length;
  *   out_bf16 [B,Hq,Dv]; lse nullable [B,Hq] FP32 (natural-log sum of exp of the scaled scores).
  * Hq % Hkv == 0; D % 16 == 0, D <= 640; Dv % 16 == 0, Dv <= 512; Dv <= D when v_cache is NULL.
- * Empty sequences give zeros and lse = -inf.
+ * Empty sequences give zeros and lse = -inf.  A sequence longer than max_seqlen: tokens past max_seqlen may be left
+ * out, and msd_last_device_status may report MSD_ERR_BAD_SHAPE (the workspace has no room for that sequence's partial
+ * results; nothing is written outside it).
  */
 size_t msd_attn_decode_int8kv_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
                                               int32_t max_seqlen);
@@ -326,11 +331,27 @@ msd_status_t msd_attn_decode_int8kv_paged(const void* q_bf16, const int8_t* k_ca
                                           int32_t D, int32_t Dv, float softmax_scale, void* out_bf16, float* lse,
                                           void* workspace, size_t workspace_bytes, void* stream);
 
-/* The split schedule msd_attn_decode_int8kv uses (so a checker can mirror it): writes the tile size, the number of
- * context splits and the tokens per split; split s of a sequence of length L covers tokens
- * [s*split_tokens, min(L, (s+1)*split_tokens)) and is walked in tiles of `tile` tokens (splits past L are empty). */
+/* The split schedule msd_attn_decode_int8kv uses (so a checker can mirror it): writes the tile size, the largest
+ * number of context splits a (sequence, query row) can have and the tokens per split.  With *split_tokens > 0 split s
+ * of a sequence of length L covers tokens [s*split_tokens, min(L, (s+1)*split_tokens)) and is walked in tiles of
+ * `tile` tokens (splits past L are empty).  *split_tokens = 0: the splits depend on the lengths of all sequences of
+ * the call (Sec. 4.3 leaves the partition of the context open; head groups of up to 16 rows per KV head cut the list
+ * of all sequences' tiles into equal runs, as many as fit the machine at once, so that no SM is left with more work
+ * than another) - msd_attn_decode_split_starts lists them. */
 msd_status_t msd_attn_decode_schedule(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen,
                                       int32_t* tile, int32_t* n_splits, int32_t* split_tokens);
+
+/* The context splits of one call, for a checker (host arithmetic; needs the CUDA device only to ask how many CTAs of
+ * the kernel are resident at once).  seqlens: HOST, [B] tokens per sequence (as the call's cu_seqlens / seqlens say).
+ * q_len, Hq as for msd_attn_decode_int8kv_spec (q_len = 1 otherwise); paged / v_aliased: non-zero for a paged cache /
+ * for v_cache == NULL.  starts: HOST, written, [B][Hkv][q_len * Hq / Hkv][n_splits + 1] INT32 with n_splits as
+ * msd_attn_decode_schedule(B, q_len * Hq, ...) reports it: row r of a KV head (query token r / (Hq / Hkv), head
+ * r % (Hq / Hkv) of the group) of sequence b has its split s over tokens [starts[..][s], starts[..][s + 1]) of the
+ * sequence; every start is a multiple of the tile; trailing entries repeat the length (empty splits).  The partial
+ * results are merged in this order.  Errors: MSD_ERR_NULL_POINTER, MSD_ERR_BAD_SHAPE, MSD_ERR_CUDA. */
+msd_status_t msd_attn_decode_split_starts(int32_t B, int32_t q_len, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
+                                          int32_t max_seqlen, int32_t paged, int32_t v_aliased, const int32_t* seqlens,
+                                          int32_t* starts);
 
 /* The softmax references of the kernel that msd_attn_decode_int8kv (and _spec, _paged) runs for this shape, for a
  * checker that mirrors it (Sec. 4.3; Alg. 3 lines 6-8).  Head groups of up to 16 rows per KV head: *m_margin = 0,

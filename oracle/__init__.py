@@ -249,7 +249,8 @@ def attn_decode_int8kv(q_bits, k, v, k_scale, v_scale, cu_seqlens, softmax_scale
     'dequant' (KV -> BF16 comparison path), 'held' (tiled, but the reference maximum and the probability scale
     move only when exceeded: to the tile maximum + ``m_margin`` (natural-log units) and to ``sv_growth`` times the
     tile's largest value scale).  ``v=None`` means V is the first ``dv`` entries of each K row.
-    ``split_starts`` ([B, n_splits+1] token offsets relative to each sequence) is used by 'tiled' and 'held'.
+    ``split_starts`` ([B, n_splits+1] token offsets relative to each sequence, or [B, Hq, n_splits+1] when the splits
+    differ between the query heads) is used by 'tiled' and 'held'.
     """
     q_bits = _c(q_bits, np.uint16)
     B, Hq, D = q_bits.shape
@@ -269,11 +270,13 @@ def attn_decode_int8kv(q_bits, k, v, k_scale, v_scale, cu_seqlens, softmax_scale
     ns, ss = 0, None
     if m in (1, 4):
         ss = _c(split_starts, np.int32)
-        ns = ss.shape[1] - 1
+        assert ss.shape[:-1] in ((B,), (B, Hq)), ss.shape
+        ns = ss.shape[-1] - 1
     lib().msdo_attn_decode_int8kv(_p(q_bits), _p(k), _p(v), _p(k_scale), _p(v_scale), _p(cu), C.c_int32(B),
                                   C.c_int32(Hq), C.c_int32(Hkv), C.c_int32(D), C.c_int32(dv),
                                   C.c_float(softmax_scale), C.c_int(m), C.c_int32(tile), _p(ss), C.c_int32(ns),
-                                  _p(out), _p(lse), _p(sdbg), C.c_double(m_margin), C.c_float(sv_growth))
+                                  _p(out), _p(lse), _p(sdbg), C.c_double(m_margin), C.c_float(sv_growth),
+                                  C.c_int32(1 if m in (1, 4) and ss.ndim == 3 else 0))
     res = [out]
     if want_lse:
         res.append(lse)

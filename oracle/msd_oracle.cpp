@@ -465,7 +465,8 @@ void msdo_gemm_w4a16(const uint16_t* x_bf16, const uint8_t* w_fp4, const uint8_t
 //   k_scale [T,Hkv]; v_scale [T,Hkv] or NULL (= k_scale); cu_seqlens [B+1] token offsets.
 //   mode 0  definition: one softmax over the whole context (Alg. 3 lines 6-12 with a global row max).
 //   mode 1  tiled (Sec. 4.3): context cut at split_starts (per sequence, relative token offsets,
-//           [B, n_splits+1]; unused trailing entries repeat the length), each split walked in tiles of
+//           [B, n_splits+1], or with starts_per_head != 0 per sequence and query head, [B, Hq, n_splits+1];
+//           unused trailing entries repeat the length), each split walked in tiles of
 //           `tile` tokens with a running max; each tile quantises P against the running max in force
 //           and with alpha_P = max(tile's v_scale)/127; splits merged with the usual log-sum-exp rule.
 //   mode 4  tiled with held references (reading of Sec. 4.3 for kernels that keep integer PV sums across tiles):
@@ -482,7 +483,7 @@ void msdo_attn_decode_int8kv(const uint16_t* q_bf16, const int8_t* k, const int8
                              const float* v_scale, const int32_t* cu_seqlens, int32_t B, int32_t Hq, int32_t Hkv,
                              int32_t D, int32_t Dv, float softmax_scale, int mode, int32_t tile,
                              const int32_t* split_starts, int32_t n_splits, double* out, double* lse,
-                             int32_t* s_dbg, double m_margin, float sv_growth) {
+                             int32_t* s_dbg, double m_margin, float sv_growth, int32_t starts_per_head) {
   const int64_t T = cu_seqlens[B];
   const int G = Hq / Hkv;
   const int8_t* vv = v ? v : k;
@@ -552,7 +553,8 @@ void msdo_attn_decode_int8kv(const uint16_t* q_bf16, const int8_t* k, const int8
       int64_t tl = L;
       if (mode == 0) { bounds = {0, static_cast<int32_t>(L)}; }
       else {
-        for (int s = 0; s <= n_splits; ++s) bounds.push_back(std::min<int64_t>(L, split_starts[static_cast<int64_t>(b) * (n_splits + 1) + s]));
+        const int64_t row = starts_per_head ? static_cast<int64_t>(b) * Hq + h : b;
+        for (int s = 0; s <= n_splits; ++s) bounds.push_back(std::min<int64_t>(L, split_starts[row * (n_splits + 1) + s]));
         tl = tile;
       }
       double m_tot = -std::numeric_limits<double>::infinity(), l_tot = 0.0;

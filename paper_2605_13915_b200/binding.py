@@ -60,6 +60,7 @@ _SIGS = {
     "msd_attn_decode_int8kv": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp,
                                          _vp, _sz, _vp]),
     "msd_attn_decode_schedule": (C.c_int, [_i32] * 6 + [C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
+    "msd_attn_decode_split_starts": (C.c_int, [_i32] * 9 + [C.c_void_p, C.c_void_p]),
     "msd_attn_decode_softmax_rule": (C.c_int, [_i32] * 6 + [C.POINTER(_f32), C.POINTER(_f32)]),
     "msd_debug_set_attn_dump": (None, [_vp, _vp, _vp]),
     "msd_debug_set_option": (C.c_int, [C.c_char_p, _i32]),
@@ -342,6 +343,19 @@ def attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen):
     _check(lib().msd_attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen, C.byref(tile), C.byref(ns), C.byref(st)),
            "msd_attn_decode_schedule")
     return tile.value, ns.value, st.value
+
+
+def attn_decode_split_starts(seqlens, Hq, Hkv, D, Dv, max_seqlen, q_len=1, paged=False, v_aliased=False):
+    """Context splits of a call with these sequence lengths: int32 array [B, Hkv, q_len * Hq // Hkv, n_splits + 1] of
+    token offsets (see msd_attn_decode_split_starts), plus the tile size."""
+    import numpy as np
+    L = np.ascontiguousarray(seqlens, dtype=np.int32)
+    B = int(L.shape[0])
+    tile, ns, _ = attn_decode_schedule(B, Hq * q_len, Hkv, D, Dv, max(int(max_seqlen), 1))
+    starts = np.zeros((B, Hkv, q_len * Hq // Hkv, ns + 1), dtype=np.int32)
+    _check(lib().msd_attn_decode_split_starts(B, q_len, Hq, Hkv, D, Dv, max(int(max_seqlen), 1), int(paged), int(v_aliased),
+                                              L.ctypes.data, starts.ctypes.data), "msd_attn_decode_split_starts")
+    return starts, tile
 
 
 def attn_decode_softmax_rule(B, Hq, Hkv, D, Dv, max_seqlen):

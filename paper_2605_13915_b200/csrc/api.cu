@@ -39,7 +39,7 @@ int sm_count() {
 
 static const char* const kOptionNames[OPT_COUNT] = {
     "MSD_NO_PDL", "MSD_GEMM_MODE", "MSD_GEMM_CTAS", "MSD_P8_PAIR", "MSD_P8_KSPLIT", "MSD_W4_PAIR", "MSD_W4_TILEN", "MSD_W4_KSPLIT",
-    "MSD_ATTN_SPLITS", "MSD_ATTN_CHUNK_TILES"};
+    "MSD_ATTN_SPLITS", "MSD_ATTN_CHUNK_TILES", "MSD_ATTN_BALANCED"};
 static int g_options[OPT_COUNT];
 static std::mutex g_options_mu;
 static bool g_options_read = false;
@@ -200,7 +200,7 @@ msd_status_t msd_last_device_status(void* stream) {
     if (cudaMemsetAsync(p, 0, sizeof(unsigned), s) != cudaSuccess) return MSD_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return MSD_ERR_CUDA;
   }
-  return v == 0 ? MSD_OK : (v == MSD_ERR_TIMEOUT ? MSD_ERR_TIMEOUT : MSD_ERR_CUDA);
+  return v == 0 ? MSD_OK : (v == MSD_ERR_TIMEOUT ? MSD_ERR_TIMEOUT : (v == MSD_ERR_BAD_SHAPE ? MSD_ERR_BAD_SHAPE : MSD_ERR_CUDA));
 }
 
 msd_status_t msd_debug_timeout_selftest(int64_t budget_cycles, void* stream) {

@@ -14,6 +14,7 @@
 // buffered in TMEM).  Every wait is bounded.
 #include <cuda_bf16.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstdlib>
 
@@ -52,6 +53,12 @@ struct AttnParams {
   int HG, Rp, groups;     // heads per CTA, stacked rows, head groups per KV head
   int DC, DVT;            // 128-byte chunks of D / Dv
   int n_splits, stages, chunk;   // chunk: tokens per split (a multiple of the tile)
+  // Balanced schedule (narrow head groups): the tiles of all sequences, in order, form one list that is cut into equal
+  // runs (of at least q_min tiles), each walked by one CTA per (KV head, head group); a CTA writes one partial result
+  // per sequence its run touches, into the slot that counts the runs which began on that sequence before it, and the
+  // CTA that reaches a sequence's end records how many slots there are (n_slots, one per sequence, KV head, head group).
+  int balanced, q_min;
+  int32_t* n_slots;
   int v_alias;            // 1: V is the first Dv bytes of the K rows
   int kv_chunks;          // 128-byte chunks reserved per KV stage (>= DC, and >= DVT when V aliases the K rows)
   int tmem_cols;
@@ -72,6 +79,14 @@ __device__ __forceinline__ void attn_mark(const AttnParams& p, int slot) {
   if (p.trace && cta < 1024) p.trace[cta * 32 + slot] = clock64();
 }
 
+
+// a read-only global load that stays where it is written (volatile: the compiler neither moves it nor issues it again
+// later to save a register)
+__device__ __forceinline__ float ldg_f32_pinned(const float* ptr) {
+  float v;
+  asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(ptr));
+  return v;
+}
 
 // 2^x for x <= 0 (flushes tiny results to zero): one MUFU instruction
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -160,6 +175,95 @@ __device__ __forceinline__ void attn_dump_scores(const AttnParams& p, long long 
   }
 }
 
+// A CTA's position in its run of tiles: sequence b (seq0: its first row in a contiguous cache, L: its tokens), tile t
+// of the nb tiles of that sequence, the tiles the CTA still has to do, and the unit u (KV head * groups + head group)
+// whose rows it computes throughout.
+struct AttnWalk { int b, u, t, nb, left, seq0, L; };
+
+__device__ __forceinline__ int attn_seq_tokens(const AttnParams& p, int b) {
+  return p.block_table ? __ldg(p.seqlens + b) : __ldg(p.cu + b + 1) - __ldg(p.cu + b);
+}
+__device__ __forceinline__ int attn_seq_tiles(const AttnParams& p, int b) {
+  const int L = attn_seq_tokens(p, b);
+  return L > 0 ? (L + kTok - 1) / kTok : 0;
+}
+__device__ __forceinline__ void attn_walk_load(const AttnParams& p, AttnWalk& w) {      // L, nb, seq0 of sequence w.b
+  w.seq0 = p.block_table ? 0 : __ldg(p.cu + w.b);
+  w.L = max(attn_seq_tokens(p, w.b), 0);
+  w.nb = (w.L + kTok - 1) / kTok;
+}
+// n tiles further (n never crosses the end of the sequence): on to the next sequence that has tokens
+template <bool kBalanced>
+__device__ __forceinline__ void attn_walk_advance(const AttnParams& p, AttnWalk& w, int n) {
+  w.t += n;
+  w.left -= n;
+  if constexpr (!kBalanced) return;          // a fixed split never leaves its sequence
+  if (w.t >= w.nb && w.left > 0) {
+    w.t = 0;
+    do {
+      if (++w.b >= p.B) { w.left = 0; w.nb = 1; break; }     // cannot happen while the lengths stay what they were when the runs were cut
+      attn_walk_load(p, w);
+    } while (w.nb == 0);
+  }
+}
+
+// Balanced schedule.  The tiles of all sequences, in order, form one list; it is cut into R equal runs, and run i is
+// walked by the U = Hkv * groups consecutive CTAs [i U, (i+1) U), one per unit - so the CTAs that are dispatched
+// together read the same token rows of the cache, one KV head each (whole DRAM pages between them), and every CTA
+// has the same number of tiles.  Computes this CTA's run and the slot of its first partial result (the runs that
+// began on the same sequence before it).  Called by all threads; false: nothing to do for this CTA.
+__device__ __forceinline__ bool attn_walk_init(const AttnParams& p, int* s_scan, AttnWalk* w, int* slot0) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int U = p.Hkv * p.groups;
+  const int per = (p.B + kAttnThreads - 1) / kAttnThreads;
+  int sum = 0;
+  for (int b = tid * per; b < min(p.B, (tid + 1) * per); ++b) {
+    const int n = attn_seq_tiles(p, b);
+    sum += n;
+    if (blockIdx.x < U && n == 0) p.n_slots[static_cast<long long>(b) * U + blockIdx.x] = 0;     // no tokens, no partial result
+  }
+  s_scan[tid] = sum;
+  __syncthreads();
+  // every warp for itself: lane l sums the entries of threads [6 l, 6 l + 6), then a scan over the lanes
+  constexpr int kPerLane = kAttnThreads / 32;
+  int v = 0;
+#pragma unroll
+  for (int j = 0; j < kPerLane; ++j) v += s_scan[lane * kPerLane + j];
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  const int W = __shfl_sync(0xffffffffu, incl, 31);            // tiles in the list (< 2^24: the cache has < 2^31 rows)
+  if (W == 0) return false;
+  int R = min(W / p.q_min, static_cast<int>(gridDim.x) / U);   // runs: of at least q_min tiles, no more than fit the grid
+  R = R < 1 ? 1 : R;
+  const int ri = blockIdx.x / U;
+  if (ri >= R) return false;
+  const int lo = static_cast<int>(static_cast<long long>(ri) * W / R), hi = static_cast<int>(static_cast<long long>(ri + 1) * W / R);
+  const unsigned bal = __ballot_sync(0xffffffffu, incl > lo);  // not 0: W > lo
+  const int sel = __ffs(bal) - 1;
+  int P = __shfl_sync(0xffffffffu, incl - v, sel);             // tiles of the sequences in front
+  int idx = sel * kPerLane;
+  while (idx < sel * kPerLane + kPerLane - 1 && P + s_scan[idx] <= lo) { P += s_scan[idx]; ++idx; }
+  int b = idx * per, nb = 0;
+  for (; b < p.B; ++b) {
+    nb = attn_seq_tiles(p, b);
+    if (P + nb > lo) break;
+    P += nb;
+  }
+  if (b >= p.B || nb == 0) return false;     // (unreachable)
+  w->b = b;
+  attn_walk_load(p, *w);
+  w->u = blockIdx.x - ri * U;
+  w->t = lo - P;
+  w->left = hi - lo;
+  // the run that owns list position f is floor(((f + 1) R - 1) / W); the sequence began at position P
+  *slot0 = (w->t > 0) ? ri - static_cast<int>((static_cast<long long>(P + 1) * R - 1) / W) : 0;
+  return true;
+}
+
 // c1 (Alg. 3 lines 1-2) once per (sequence, KV head, head group) instead of once per context split: the query rows of
 // the group's heads are decomposed into two INT8 components (same bit-exact rule as msd_decompose_int8) and written
 // as the stacked operand image the attention CTAs copy into shared memory with one bulk copy per chunk.  One CTA per
@@ -186,7 +290,7 @@ attn_qstack_kernel(const AttnParams p, uint8_t* __restrict__ q_img, float* __res
 // Head groups of up to 16 query rows per KV head (GQA).  kMaxHG: head slots one softmax thread looks after (8 or 16);
 // kNH: heads its code is unrolled for (<= kMaxHG); kMaxDVT: 128-wide tiles of Dv.
 // kPaged: the cache is paged (block table); a template parameter so that the contiguous kernels carry none of it.
-template <int kMaxHG, int kNH, int kMaxDVT, bool kPaged>
+template <int kMaxHG, int kNH, int kMaxDVT, bool kPaged, bool kBalanced>
 __global__ void __launch_bounds__(kAttnThreads, (kNH <= 8 && kMaxDVT == 1) ? 3 : 1)
 attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
   extern __shared__ uint8_t smem_dyn[];
@@ -199,38 +303,63 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   constexpr int kNSW = 4;                          // component, rows [kSlots, 2*kSlots) second component
   __shared__ float s_aq[kSlots], s_bq[kSlots];
   __shared__ float red[2][4][kNH + 1];             // per-warp tile maxima, double buffered by tile parity
+  __shared__ int s_scan[kAttnThreads];
+  __shared__ AttnWalk s_walk;                      // the softmax warps' walk (kept here, not in registers, between segments)
+  __shared__ int s_slot;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // units along x (launched first), splits along y: the early splits of every sequence, which are always full, start
-  // before the last, shorter ones (and the two head groups of a wide group, which read the same tiles, side by side)
-  const int split = blockIdx.y;
-  int unit = blockIdx.x;
-  const int grp = unit % p.groups; unit /= p.groups;
-  const int hk = unit % p.Hkv;
-  const int b = unit / p.Hkv;
-  const int32_t* bt = kPaged ? p.block_table + static_cast<long long>(b) * p.max_blocks : nullptr;
-  const int seq0 = kPaged ? 0 : p.cu[b];
-  const int L = kPaged ? p.seqlens[b] : p.cu[b + 1] - seq0;
-  const int t_begin = split * p.chunk;                       // every split covers the same number of tokens
-  const int t_end = min(L, t_begin + p.chunk);
-  const int h0 = hk * p.G + grp * p.HG;                      // first query head of this CTA
-  const int nh = min(p.HG, p.G - grp * p.HG);                // heads actually present
-  const int ntiles = (t_end > t_begin) ? (t_end - t_begin + kTok - 1) / kTok : 0;
+  const int U = p.Hkv * p.groups;
+  // The CTA's tiles: a run of the list of all sequences' tiles (balanced schedule), or one context split of one
+  // sequence (fixed splits: units along x, launched first, splits along y - the early splits of every sequence, which
+  // are always full, start before the last, shorter ones); always for one unit.  Either way the run is walked sequence
+  // by sequence ("segments"): all roles below step through the same AttnWalk, and tiles, buffers and barrier phases
+  // are counted over the whole run, not per segment.
+  AttnWalk w0;
+  int slot0;
+  if constexpr (kBalanced) {
+    if (!attn_walk_init(p, s_scan, &w0, &slot0)) return;
+  } else {
+    const int split = blockIdx.y, b = blockIdx.x / U;
+    const int L = attn_seq_tokens(p, b);
+    const int t_begin = split * p.chunk;                       // every split covers the same number of tokens
+    const int t_end = min(L, t_begin + p.chunk);
+    const int ntiles = (t_end > t_begin) ? (t_end - t_begin + kTok - 1) / kTok : 0;
+    if (ntiles == 0) {      // nothing in this split: neutral partials, before any barrier or TMEM use
+      const int grp = blockIdx.x % p.groups, hk = (blockIdx.x / p.groups) % p.Hkv;
+      const int h0 = hk * p.G + grp * p.HG, nh = min(p.HG, p.G - grp * p.HG);
+      for (int i = threadIdx.x; i < nh * (p.Dv + kPartHdr); i += blockDim.x) {
+        const int h = i / (p.Dv + kPartHdr), e = i % (p.Dv + kPartHdr);
+        float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + h) * p.n_splits + split) * (p.Dv + kPartHdr);
+        dst[e] = (e == 0) ? -INFINITY : 0.0f;
+      }
+      return;
+    }
+    w0.b = b; w0.u = blockIdx.x % U; w0.t = t_begin / kTok; w0.left = ntiles;
+    attn_walk_load(p, w0);
+    slot0 = split;
+  }
+  const int total_tiles = w0.left;
+  // The scales of the CTA's first tile, asked for as early as their address is known (softmax threads: one token each):
+  // at the start everything is a cold read that queues behind the first KV tiles of every CTA of the grid.
+  float ks_first = 0.0f, vs_first = 0.0f;
+  if (threadIdx.x >= 64) {
+    const int tok_rel = w0.t * kTok + (warp & 3) * 32 + lane;      // the thread's token lane (its warp's quarter of tensor memory)
+    if (tok_rel < w0.L) {
+      long long row = w0.seq0 + tok_rel;
+      if constexpr (kPaged)
+        row = static_cast<long long>(__ldg(p.block_table + static_cast<long long>(w0.b) * p.max_blocks + (tok_rel >> p.page_shift))) * p.page +
+              (tok_rel & (p.page - 1));
+      const long long sidx = row * p.Hkv + (blockIdx.x % U) / p.groups;
+      ks_first = ldg_f32_pinned(p.k_scale + sidx);
+      vs_first = ldg_f32_pinned(p.v_scale + sidx);
+    }
+  }
   if (threadIdx.x == 0 && p.trace) {
     attn_mark(p, 0);
     unsigned long long g;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g));
     const int cta = blockIdx.y * gridDim.x + blockIdx.x;
-    if (cta < 1024) { p.trace[cta * 32 + 1] = static_cast<long long>(g); p.trace[cta * 32 + 2] = ntiles; }
-  }
-
-  if (ntiles == 0) {      // nothing in this split: neutral partials, before any barrier or TMEM use
-    for (int i = threadIdx.x; i < nh * (p.Dv + kPartHdr); i += blockDim.x) {
-      const int h = i / (p.Dv + kPartHdr), e = i % (p.Dv + kPartHdr);
-      float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + h) * p.n_splits + split) * (p.Dv + kPartHdr);
-      dst[e] = (e == 0) ? -INFINITY : 0.0f;
-    }
-    return;
+    if (cta < 1024) { p.trace[cta * 32 + 1] = static_cast<long long>(g); p.trace[cta * 32 + 2] = total_tiles; }
   }
 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -249,6 +378,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     mbar_init(&p_full[0], kNSW); mbar_init(&p_full[1], kNSW); mbar_init(&q_ready, kNSW);
     mbar_init(&o_full, 1); mbar_init(&o_empty, kNSW);
     abort_flag = 0;
+    s_walk = w0;
+    s_slot = slot0;
     mbar_init_fence();
     tma_prefetch_desc(&tmap_k);
     tma_prefetch_desc(&tmap_v);
@@ -270,47 +401,42 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       // soon as QK^T has read it, long before the PV product of the same tile releases the V buffer, so the next K
       // tile can be fetched that much earlier.  With V aliased to the K rows there is only the K ring.
       const int k_bytes = p.DC * kChunkBytes, v_bytes = p.DVT * kChunkBytes;
-      int kq = 0, vq = p.v_alias ? ntiles : 0;
-      long long t_idle = clock64();
-      while (kq < ntiles || vq < ntiles) {
-        bool progressed = false;
-        if (kq < ntiles && mbar_test_wait(&kv_empty[kq % p.stages], ((kq / p.stages) & 1) ^ 1)) {
-          const int st = kq % p.stages;
-          uint8_t* dst = smem + st * kv_stage_bytes;
-          const int u0 = t_begin + kq * kTok;
-          if constexpr (!kPaged) {
-            mbar_arrive_expect_tx(&kv_full[st], k_bytes);
-            for (int c = 0; c < p.DC; ++c) tma_load_3d(dst + c * kChunkBytes, &tmap_k, c * kChunk, hk, seq0 + u0, &kv_full[st]);
-          } else {
-            // one box per page that holds tokens of this split; rows of the tile past them keep stale (finite) codes
-            // and are masked like every token past the end
-            const int npg = min(kTok >> p.page_shift, (t_end - u0 + p.page - 1) >> p.page_shift);
-            mbar_arrive_expect_tx(&kv_full[st], p.DC * kChunk * p.page * npg);
-            for (int pg = 0; pg < npg; ++pg) {
-              const int tok = __ldg(bt + (u0 >> p.page_shift) + pg) * p.page;
-              for (int c = 0; c < p.DC; ++c)
-                tma_load_3d(dst + c * kChunkBytes + pg * p.page * kChunk, &tmap_k, c * kChunk, hk, tok, &kv_full[st]);
-            }
+      AttnWalk wk = w0, wv = w0;                 // where the next K / V tile comes from
+      int kq = 0, vq = p.v_alias ? total_tiles : 0;
+      // the tile at walk position w: chunks [0, nchunks) of the rows of KV head hk into dst
+      const int hk = w0.u / p.groups;
+      auto load_tile = [&](const AttnWalk& w, const CUtensorMap* tmap, int nchunks, uint8_t* dst, uint64_t* bar) {
+        const int u0 = w.t * kTok;
+        if constexpr (!kPaged) {
+          mbar_arrive_expect_tx(bar, nchunks * kChunkBytes);
+          for (int c = 0; c < nchunks; ++c) tma_load_3d(dst + c * kChunkBytes, tmap, c * kChunk, hk, w.seq0 + u0, bar);
+        } else {
+          // one box per page that holds tokens of the sequence; rows of the tile past them keep stale (finite) codes
+          // and are masked like every token past the end
+          const int32_t* bt = p.block_table + static_cast<long long>(w.b) * p.max_blocks;
+          const int npg = min(kTok >> p.page_shift, (w.L - u0 + p.page - 1) >> p.page_shift);
+          mbar_arrive_expect_tx(bar, nchunks * kChunk * p.page * npg);
+          for (int pg = 0; pg < npg; ++pg) {
+            const int tok = __ldg(bt + (u0 >> p.page_shift) + pg) * p.page;
+            for (int c = 0; c < nchunks; ++c)
+              tma_load_3d(dst + c * kChunkBytes + pg * p.page * kChunk, tmap, c * kChunk, hk, tok, bar);
           }
+        }
+      };
+      long long t_idle = clock64();
+      while (kq < total_tiles || vq < total_tiles) {
+        bool progressed = false;
+        if (kq < total_tiles && mbar_test_wait(&kv_empty[kq % p.stages], ((kq / p.stages) & 1) ^ 1)) {
+          const int st = kq % p.stages;
+          load_tile(wk, &tmap_k, p.DC, smem + st * kv_stage_bytes, &kv_full[st]);
+          attn_walk_advance<kBalanced>(p, wk, 1);
           ++kq;
           progressed = true;
         }
-        if (vq < ntiles && mbar_test_wait(&v_empty[vq % p.stages], ((vq / p.stages) & 1) ^ 1)) {
+        if (vq < total_tiles && mbar_test_wait(&v_empty[vq % p.stages], ((vq / p.stages) & 1) ^ 1)) {
           const int st = vq % p.stages;
-          uint8_t* dst = smem + st * kv_stage_bytes + k_bytes;
-          const int u0 = t_begin + vq * kTok;
-          if constexpr (!kPaged) {
-            mbar_arrive_expect_tx(&v_full[st], v_bytes);
-            for (int j = 0; j < p.DVT; ++j) tma_load_3d(dst + j * kChunkBytes, &tmap_v, j * kChunk, hk, seq0 + u0, &v_full[st]);
-          } else {
-            const int npg = min(kTok >> p.page_shift, (t_end - u0 + p.page - 1) >> p.page_shift);
-            mbar_arrive_expect_tx(&v_full[st], p.DVT * kChunk * p.page * npg);
-            for (int pg = 0; pg < npg; ++pg) {
-              const int tok = __ldg(bt + (u0 >> p.page_shift) + pg) * p.page;
-              for (int j = 0; j < p.DVT; ++j)
-                tma_load_3d(dst + j * kChunkBytes + pg * p.page * kChunk, &tmap_v, j * kChunk, hk, tok, &v_full[st]);
-            }
-          }
+          load_tile(wv, &tmap_v, p.DVT, smem + st * kv_stage_bytes + k_bytes, &v_full[st]);
+          attn_walk_advance<kBalanced>(p, wv, 1);
           ++vq;
           progressed = true;
         }
@@ -325,6 +451,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           }
         }
       }
+      (void)v_bytes;
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
@@ -332,7 +459,6 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       const uint32_t idesc_qk = idesc_dense(2, 1, 1, 0, 0, kTok, p.Rp);     // S8 x S8 -> S32, both K-major
       const uint32_t idesc_pv = idesc_dense(2, 1, 1, 1, 0, kTok, p.Rp);     // A (V^T) MN-major
       bool ok = true;
-      ok = wait_bounded(&q_ready, 0, abort, p.status);      // the softmax warps have decomposed the query rows
       // Operand descriptors differ from three templates only in the 16-byte-granular address field (bits 0-13), so each
       // costs one 64-bit add: with 36 MMAs per MLA tile this thread's instruction count is on the critical path.
       const uint64_t dk = smem_desc(0, 16, 1024, kSwizzle128B);         // K-major tiles: K, stacked Q, P
@@ -374,16 +500,24 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         tc_commit(p.v_alias ? &kv_empty[st] : &v_empty[st]);
       };
       // Two streams of work, each in tile order, issued as soon as their inputs are there (whichever comes first):
-      //   QK^T(q) needs the KV tile q in shared memory and the score buffer q&1 drained (P of tile q-2 written);
+      //   QK^T(q) needs the KV tile q in shared memory, the score buffer q&1 drained (P of tile q-2 written) and, for
+      //           the first tile of a segment, that segment's stacked Q operand (written once the previous segment's
+      //           last merge is done, so every earlier QK^T has read the old one);
       //   PV(v)   needs P of tile v written, O^T of tile v-1 merged, and QK^T(v) already issued.
       // A QK^T that waits for its KV tile must not hold back a PV whose operands are ready, and vice versa.
-      int q = 0, v = 0;
+      AttnWalk wq = w0;
+      int q = 0, v = 0, seg = 0;                 // seg: segments whose stacked Q operand has been waited for
+      bool q_first = true;                       // tile q is the first of its segment
       long long t_idle = clock64();
-      while (ok && v < ntiles) {
+      while (ok && v < total_tiles) {
         bool progressed = false;
-        if (q < ntiles && q < v + 2 &&
-            mbar_test_wait(&kv_full[q % p.stages], (q / p.stages) & 1)) {    // (q < v + 2 implies P of tile q-2 is written)
+        if (q < total_tiles && q < v + 2 &&
+            mbar_test_wait(&kv_full[q % p.stages], (q / p.stages) & 1) &&    // (q < v + 2 implies P of tile q-2 is written)
+            (!q_first || mbar_test_wait(&q_ready, seg & 1))) {
+          if (q_first) ++seg;
           issue_qk(q);
+          attn_walk_advance<kBalanced>(p, wq, 1);
+          q_first = kBalanced && wq.t == 0;
           ++q;
           progressed = true;
         }
@@ -412,201 +546,245 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const int wi = warp - 2;                        // 0 .. 3
     const int wq = wi;
     constexpr int hs0 = 0;                          // first head slot of this warp
-    // c1: decompose the query rows of this CTA's heads (one warp per head, round robin) into the stacked operand
-    for (int h = wi; h < nh; h += kNSW) attn_decompose_q_row(p, b, hk, grp, h, lane, sm_q, &s_aq[h], &s_bq[h]);
-    fence_proxy_async_smem();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&q_ready);           // the stacked Q operand is in shared memory
-    named_bar_sync(8, 128);                         // s_aq / s_bq visible to all softmax warps
-    if (threadIdx.x == 64) attn_mark(p, 3);
     const int bar_id = 1;
-
-    // running state per head; scores are kept in the log2 domain (log2(e) is folded into the key scale)
-    // the state that is uniform across the four warps (running maxima, query scales) lives in registers
     constexpr int kRegState = kNH;
-    float l_part[kNH];
-    float m_run[kRegState], aq[kRegState], bq[kRegState], resc_keep[kRegState], resc_next[kRegState];
-    float o_run[kMaxDVT][kNH];
-#pragma unroll
-    for (int h = 0; h < kNH; ++h) {
-      l_part[h] = 0.0f;
-      m_run[h] = -INFINITY;
-      aq[h] = (hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f;
-      bq[h] = (hs0 + h < nh) ? s_bq[hs0 + h] : 0.0f;
-#pragma unroll
-      for (int j = 0; j < kMaxDVT; ++j) o_run[j][h] = 0.0f;
-    }
     const float kLog2e = 1.4426950408889634f;
     const float scale2 = p.scale * kLog2e;
     bool ok = true;
-    // State a tile's softmax hands to its merge: rescale factors and the P scales.  The softmax of tile t+1 runs
-    // BEFORE the merge of tile t (it overlaps the PV product of tile t), so two sets are alive at a time.
-    float ap_cur = 0.0f, bp_cur = 0.0f, ap_nxt = 0.0f, bp_nxt = 0.0f;
-
-    // c3-c5 for tile t: scores -> running max -> P -> two INT8 components into P buffer (t & 1)
-    // Per-token scales of tile t for this thread's token lane (0 past the end of the split).  They are fetched one tile
-    // ahead: a cold 512-byte run of the scale arrays would otherwise sit on every tile's critical path.
-    auto load_scales = [&](int t, float& ks_out, float& vs_out) {
-      const int tok_rel = t_begin + t * kTok + tl;
-      const bool valid = t < ntiles && tok_rel < t_end;
-      long long sidx;
-      if constexpr (kPaged) {
-        const long long prow = valid ? static_cast<long long>(__ldg(bt + (tok_rel >> p.page_shift))) * p.page + (tok_rel & (p.page - 1)) : 0;
-        sidx = prow * p.Hkv + hk;
-      } else {
-        sidx = static_cast<long long>(seq0 + tok_rel) * p.Hkv + hk;
-      }
-      ks_out = valid ? __ldg(p.k_scale + sidx) : 0.0f;
-      vs_out = valid ? __ldg(p.v_scale + sidx) : 0.0f;
-    };
-    float ks_pre, vs_pre;
-    load_scales(0, ks_pre, vs_pre);
-    auto softmax_tile = [&](int t, float (&resc_out)[kRegState], float& alpha_p, float& beta_p) -> bool {
-      const int tok_rel = t_begin + t * kTok + tl;
-      const bool valid = tok_rel < t_end;
-      const float ks = ks_pre * scale2;
-      const float vs = vs_pre;
-      load_scales(t + 1, ks_pre, vs_pre);
-      if (!wait_bounded(&s_full[t & 1], (t >> 1) & 1, abort, p.status)) return false;
-      if (threadIdx.x == 64 && t < 6) attn_mark(p, 4 + 4 * t);
-      tc_fence_after();
-      float s[kNH];
-      const uint32_t srow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + (t & 1) * p.Rp;
-      {
-        uint32_t v1[kMaxHG], v2[kMaxHG];          // first / second component columns
-        tmem_ldw<kMaxHG>(srow + hs0, v1);
-        tmem_ldw<kMaxHG>(srow + kSlots + hs0, v2);
-        tmem_ld_wait();
-        if (p.s_dbg && valid) {
-          long long tok_row = seq0 + tok_rel;
-          if constexpr (kPaged) tok_row = static_cast<long long>(__ldg(bt + (tok_rel >> p.page_shift))) * p.page + (tok_rel & (p.page - 1));
-          attn_dump_scores<kMaxHG>(p, tok_row, hk, grp, hs0, nh, v1, v2);
-        }
-#pragma unroll
-        for (int h = 0; h < kNH; ++h)
-        {
-          const float a_q = aq[h], b_q = bq[h];
-          bool vh = valid;
-          if (p.Sq > 1) vh = valid && tok_rel < L - p.Sq + 1 + (grp * p.HG + hs0 + h) / p.Gr;    // causal among the new tokens
-          s[h] = vh ? __fmaf_rn(a_q, static_cast<float>(static_cast<int32_t>(v1[h])), b_q * static_cast<float>(static_cast<int32_t>(v2[h]))) * ks : -INFINITY;
-        }
-      }
-      // c4: tile maxima per head (and of the value scales) over the 128 token lanes
-      float (*rb)[kNH + 1] = red[t & 1];
-#pragma unroll
-      for (int h = 0; h < kNH; ++h) {
-        const float wm = warp_max(s[h]);
-        if (lane == 0) rb[wq][h] = wm;
-      }
-      {
-        const float wv = warp_max(vs);
-        if (lane == 0) rb[wq][kNH] = wv;
-      }
-      named_bar_sync(bar_id, 128);  // one barrier per tile: the other parity buffer is rewritten only after the next one
-      // running maximum of every head before and after the tile; rescale factor of what was accumulated so far
-      // (all heads first: as many independent exponentials in flight as there are heads)
-      float mn_t[kRegState], resc_t[kRegState];
-#pragma unroll
-      for (int h = 0; h < kNH; ++h) {
-        const float mt = fmaxf(fmaxf(rb[0][h], rb[1][h]), fmaxf(rb[2][h], rb[3][h]));
-        mn_t[h] = fmaxf(m_run[h], mt);
-        resc_t[h] = (m_run[h] == -INFINITY) ? 0.0f : ex2_approx(m_run[h] - mn_t[h]);
-        m_run[h] = mn_t[h];
-        resc_out[h] = resc_t[h];
-      }
-      const float vs_max = fmaxf(fmaxf(rb[0][kNH], rb[1][kNH]), fmaxf(rb[2][kNH], rb[3][kNH]));
-      // c5: P = exp(S - m), fold the value scale, two-pass INT8 with the fixed scale alpha_P = max(v_scale)/127
-      alpha_p = vs_max * (1.0f / 127.0f);
-      beta_p = alpha_p * (1.0f / 254.0f);
-      const float inv_a = alpha_p > 0.0f ? __frcp_rn(alpha_p) : 0.0f, inv_b = beta_p > 0.0f ? __frcp_rn(beta_p) : 0.0f;
-      uint8_t* pbuf = sm_p + (t & 1) * p.Rp * kChunk;      // PV of tile t-2 (same buffer) finished before merge(t-2)
-#pragma unroll
-      for (int h = 0; h < kNH; ++h) {
-        // branch-free: an absent head or a token past the end contributes P = 0 (s is -inf there)
-        const float mn = mn_t[h], resc = resc_t[h];
-        // (a row that has seen no visible token yet keeps m = -inf: the clamp turns -inf - -inf into -inf, P = 0)
-        const float pr = (hs0 + h < nh) ? ex2_approx(s[h] - fmaxf(mn, -1e30f)) : 0.0f;
-        l_part[h] = __fmaf_rn(l_part[h], resc, pr);
-        const float pt = pr * vs;
-        // Two-pass INT8 by the 1.5 * 2^23 trick: adding it rounds to the nearest integer (ties to even) and leaves that
-        // integer in the low mantissa bits, so neither pass needs a float <-> int conversion.  No clamps: P <= 1 and
-        // v_scale <= its tile maximum give pt / alpha_P <= 127, and |r| <= alpha_P / 2 gives |r / beta_P| <= 127.
-        const float kMagic = 12582912.0f;
-        const float u1 = __fmaf_rn(pt, inv_a, kMagic);
-        const float r = __fmaf_rn(-alpha_p, u1 - kMagic, pt);
-        const float u2 = __fmaf_rn(r, inv_b, kMagic);
-        pbuf[swz_off(hs0 + h, tl)] = static_cast<uint8_t>(__float_as_uint(u1));
-        pbuf[swz_off(kSlots + hs0 + h, tl)] = static_cast<uint8_t>(__float_as_uint(u2));
-      }
+    int g0 = 0;                                     // tiles of the segments done so far
+    // the CTA's unit: the same KV head and head group in every segment
+    const int hk = (blockIdx.x % U) / p.groups, grp = (blockIdx.x % U) - hk * p.groups;
+    const int nh = min(p.HG, p.G - grp * p.HG);                // heads actually present
+    bool more = true;
+    while (ok && more) {
+      // ---- one segment: tiles [t, t + ntiles) of sequence b, from the walk in shared memory (it is advanced by one
+      // thread between two barriers at the end of the segment; what the tile loop does not need is read again after it)
+      const int ntiles = min(s_walk.left, s_walk.nb - s_walk.t);
+      const int b = s_walk.b;
+      const int32_t* bt = kPaged ? p.block_table + static_cast<long long>(b) * p.max_blocks : nullptr;
+      const int seq0 = s_walk.seq0, L = s_walk.L;
+      const int t_begin = s_walk.t * kTok;
+      const int t_end = min(L, t_begin + ntiles * kTok);
+      // c1: decompose the query rows of this segment's heads (one warp per head, round robin) into the stacked operand
+      // (the head slots and padding columns that were zeroed at the start are never written)
+      for (int h = wi; h < nh; h += kNSW) attn_decompose_q_row(p, b, hk, grp, h, lane, sm_q, &s_aq[h], &s_bq[h]);
       fence_proxy_async_smem();
-      tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&p_full[t & 1]);
-      if (threadIdx.x == 64 && t < 6) attn_mark(p, 5 + 4 * t);
-      return true;
-    };
+      if (lane == 0) mbar_arrive(&q_ready);           // the stacked Q operand is in shared memory
+      named_bar_sync(8, 128);                         // s_aq / s_bq visible to all softmax warps
+      if (threadIdx.x == 64 && g0 == 0) attn_mark(p, 3);
 
-    ok = softmax_tile(0, resc_keep, ap_cur, bp_cur);
-    for (int t = 0; t < ntiles && ok; ++t) {
-      if (t + 1 < ntiles) {
-        ok = softmax_tile(t + 1, resc_next, ap_nxt, bp_nxt);     // overlaps the PV product of tile t
-        if (!ok) break;
+      // running state per head; scores are kept in the log2 domain (log2(e) is folded into the key scale)
+      // the state that is uniform across the four warps (running maxima, query scales) lives in registers
+      float l_part[kNH];
+      float m_run[kRegState], aq[kRegState], bq[kRegState], resc_keep[kRegState], resc_next[kRegState];
+      float o_run[kMaxDVT][kNH];
+#pragma unroll
+      for (int h = 0; h < kNH; ++h) {
+        l_part[h] = 0.0f;
+        m_run[h] = -INFINITY;
+        aq[h] = (hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f;
+        bq[h] = (hs0 + h < nh) ? s_bq[hs0 + h] : 0.0f;
+#pragma unroll
+        for (int j = 0; j < kMaxDVT; ++j) o_run[j][h] = 0.0f;
       }
-      // c6/c7: wait for O^T of tile t, merge it into the running output with that tile's rescale factors
-      ok = wait_bounded(&o_full, t & 1, abort, p.status);
-      if (!ok) break;
-      if (threadIdx.x == 64 && t < 6) attn_mark(p, 6 + 4 * t);
-      tc_fence_after();
-      float resc_cur[kNH];                 // e^(m before tile t - m after tile t), from the softmax of tile t
-#pragma unroll
-      for (int h = 0; h < kNH; ++h) resc_cur[h] = resc_keep[h];
-#pragma unroll
-      for (int j = 0; j < kMaxDVT; ++j) {
-        if (j < p.DVT) {
-          const uint32_t orow = tmem_o + (static_cast<uint32_t>(quad * 32) << 16) + j * p.Rp;
-          uint32_t v1[kMaxHG], v2[kMaxHG];
-          tmem_ldw<kMaxHG>(orow + hs0, v1);
-          tmem_ldw<kMaxHG>(orow + kSlots + hs0, v2);
+      // State a tile's softmax hands to its merge: rescale factors and the P scales.  The softmax of tile t+1 runs
+      // BEFORE the merge of tile t (it overlaps the PV product of tile t), so two sets are alive at a time.
+      float ap_cur = 0.0f, bp_cur = 0.0f, ap_nxt = 0.0f, bp_nxt = 0.0f;
+
+      // Per-token scales of tile t for this thread's token lane (0 past the end of the segment).  They are fetched one
+      // tile ahead: a cold 512-byte run of the scale arrays would otherwise sit on every tile's critical path.
+      auto load_scales = [&](int t, float& ks_out, float& vs_out) {
+        const int tok_rel = t_begin + t * kTok + tl;
+        const bool valid = t < ntiles && tok_rel < t_end;
+        long long sidx;
+        if constexpr (kPaged) {
+          const long long prow = valid ? static_cast<long long>(__ldg(bt + (tok_rel >> p.page_shift))) * p.page + (tok_rel & (p.page - 1)) : 0;
+          sidx = prow * p.Hkv + hk;
+        } else {
+          sidx = static_cast<long long>(seq0 + tok_rel) * p.Hkv + hk;
+        }
+        ks_out = valid ? __ldg(p.k_scale + sidx) : 0.0f;
+        vs_out = valid ? __ldg(p.v_scale + sidx) : 0.0f;
+      };
+      float ks_pre, vs_pre;
+      if (g0 == 0) { ks_pre = ks_first; vs_pre = vs_first; }
+      else load_scales(0, ks_pre, vs_pre);
+      // c3-c5 for tile t of the segment (tile g0 + t of the CTA): scores -> running max -> P -> two INT8 components
+      // into P buffer ((g0 + t) & 1)
+      auto softmax_tile = [&](int t, float (&resc_out)[kRegState], float& alpha_p, float& beta_p) -> bool {
+        const int gt = g0 + t;
+        const int tok_rel = t_begin + t * kTok + tl;
+        const bool valid = tok_rel < t_end;
+        const float ks = ks_pre * scale2;
+        const float vs = vs_pre;
+        load_scales(t + 1, ks_pre, vs_pre);
+        if (!wait_bounded(&s_full[gt & 1], (gt >> 1) & 1, abort, p.status)) return false;
+        if (threadIdx.x == 64 && gt < 6) attn_mark(p, 4 + 4 * gt);
+        tc_fence_after();
+        float s[kNH];
+        const uint32_t srow = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + (gt & 1) * p.Rp;
+        {
+          uint32_t v1[kMaxHG], v2[kMaxHG];          // first / second component columns
+          tmem_ldw<kMaxHG>(srow + hs0, v1);
+          tmem_ldw<kMaxHG>(srow + kSlots + hs0, v2);
           tmem_ld_wait();
+          if (p.s_dbg && valid) {
+            long long tok_row = seq0 + tok_rel;
+            if constexpr (kPaged) tok_row = static_cast<long long>(__ldg(bt + (tok_rel >> p.page_shift))) * p.page + (tok_rel & (p.page - 1));
+            attn_dump_scores<kMaxHG>(p, tok_row, hk, grp, hs0, nh, v1, v2);
+          }
 #pragma unroll
           for (int h = 0; h < kNH; ++h)
-            // alpha_P O1 + beta_P O2 with beta_P = alpha_P / 254: one integer multiply-add and one conversion
-            // (|254 O1 + O2| <= 255 * 128 * 127 * 127 < 2^31)
-            o_run[j][h] = __fmaf_rn(o_run[j][h], resc_cur[h], bp_cur * static_cast<float>(254 * static_cast<int32_t>(v1[h]) + static_cast<int32_t>(v2[h])));
+          {
+            const float a_q = aq[h], b_q = bq[h];
+            bool vh = valid;
+            if (p.Sq > 1) vh = valid && tok_rel < L - p.Sq + 1 + (grp * p.HG + hs0 + h) / p.Gr;    // causal among the new tokens
+            s[h] = vh ? __fmaf_rn(a_q, static_cast<float>(static_cast<int32_t>(v1[h])), b_q * static_cast<float>(static_cast<int32_t>(v2[h]))) * ks : -INFINITY;
+          }
         }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&o_empty);
-      if (threadIdx.x == 64 && t < 6) attn_mark(p, 7 + 4 * t);
+        // c4: tile maxima per head (and of the value scales) over the 128 token lanes
+        float (*rb)[kNH + 1] = red[gt & 1];
 #pragma unroll
-      for (int h = 0; h < kRegState; ++h) resc_keep[h] = resc_next[h];
-      ap_cur = ap_nxt;
-      bp_cur = bp_nxt;
-    }
-    if (threadIdx.x == 64) attn_mark(p, 28);
-    // partial results of this split: running max, sum of P and unnormalised output per head
-    if (ok) {
-      float (*rb)[kNH + 1] = red[ntiles & 1];
-      named_bar_sync(bar_id, 128);
-#pragma unroll
-      for (int h = 0; h < kNH; ++h) {
-        float l = l_part[h];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-        if (lane == 0) rb[wq][h] = l;
-      }
-      named_bar_sync(bar_id, 128);
-#pragma unroll
-      for (int h = 0; h < kNH; ++h) {
-        if (hs0 + h < nh) {
-          float* dst = p.partial + ((static_cast<long long>(b) * p.Hq + h0 + hs0 + h) * p.n_splits + split) * (p.Dv + kPartHdr);
-          // the running maximum goes out in natural-log units (it was kept in the log2 domain)
-          if (tl == 0) { dst[0] = m_run[h] * 0.6931471805599453f; dst[1] = rb[0][h] + rb[1][h] + rb[2][h] + rb[3][h]; }
-#pragma unroll
-          for (int j = 0; j < kMaxDVT; ++j)
-            if (j < p.DVT && j * kChunk + tl < p.Dv) dst[kPartHdr + j * kChunk + tl] = o_run[j][h];
+        for (int h = 0; h < kNH; ++h) {
+          const float wm = warp_max(s[h]);
+          if (lane == 0) rb[wq][h] = wm;
         }
+        {
+          const float wv = warp_max(vs);
+          if (lane == 0) rb[wq][kNH] = wv;
+        }
+        named_bar_sync(bar_id, 128);  // one barrier per tile: the other parity buffer is rewritten only after the next one
+        // running maximum of every head before and after the tile; rescale factor of what was accumulated so far
+        // (all heads first: as many independent exponentials in flight as there are heads)
+        float mn_t[kRegState], resc_t[kRegState];
+#pragma unroll
+        for (int h = 0; h < kNH; ++h) {
+          const float mt = fmaxf(fmaxf(rb[0][h], rb[1][h]), fmaxf(rb[2][h], rb[3][h]));
+          mn_t[h] = fmaxf(m_run[h], mt);
+          resc_t[h] = (m_run[h] == -INFINITY) ? 0.0f : ex2_approx(m_run[h] - mn_t[h]);
+          m_run[h] = mn_t[h];
+          resc_out[h] = resc_t[h];
+        }
+        const float vs_max = fmaxf(fmaxf(rb[0][kNH], rb[1][kNH]), fmaxf(rb[2][kNH], rb[3][kNH]));
+        // c5: P = exp(S - m), fold the value scale, two-pass INT8 with the fixed scale alpha_P = max(v_scale)/127
+        alpha_p = vs_max * (1.0f / 127.0f);
+        beta_p = alpha_p * (1.0f / 254.0f);
+        const float inv_a = alpha_p > 0.0f ? __frcp_rn(alpha_p) : 0.0f, inv_b = beta_p > 0.0f ? __frcp_rn(beta_p) : 0.0f;
+        uint8_t* pbuf = sm_p + (gt & 1) * p.Rp * kChunk;      // PV of tile gt-2 (same buffer) finished before merge(gt-2)
+#pragma unroll
+        for (int h = 0; h < kNH; ++h) {
+          // branch-free: an absent head or a token past the end contributes P = 0 (s is -inf there)
+          const float mn = mn_t[h], resc = resc_t[h];
+          // (a row that has seen no visible token yet keeps m = -inf: the clamp turns -inf - -inf into -inf, P = 0)
+          const float pr = (hs0 + h < nh) ? ex2_approx(s[h] - fmaxf(mn, -1e30f)) : 0.0f;
+          l_part[h] = __fmaf_rn(l_part[h], resc, pr);
+          const float pt = pr * vs;
+          // Two-pass INT8 by the 1.5 * 2^23 trick: adding it rounds to the nearest integer (ties to even) and leaves that
+          // integer in the low mantissa bits, so neither pass needs a float <-> int conversion.  No clamps: P <= 1 and
+          // v_scale <= its tile maximum give pt / alpha_P <= 127, and |r| <= alpha_P / 2 gives |r / beta_P| <= 127.
+          const float kMagic = 12582912.0f;
+          const float u1 = __fmaf_rn(pt, inv_a, kMagic);
+          const float r = __fmaf_rn(-alpha_p, u1 - kMagic, pt);
+          const float u2 = __fmaf_rn(r, inv_b, kMagic);
+          pbuf[swz_off(hs0 + h, tl)] = static_cast<uint8_t>(__float_as_uint(u1));
+          pbuf[swz_off(kSlots + hs0 + h, tl)] = static_cast<uint8_t>(__float_as_uint(u2));
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_full[gt & 1]);
+        if (threadIdx.x == 64 && gt < 6) attn_mark(p, 5 + 4 * gt);
+        return true;
+      };
+
+      ok = softmax_tile(0, resc_keep, ap_cur, bp_cur);
+      for (int t = 0; t < ntiles && ok; ++t) {
+        const int gt = g0 + t;
+        if (t + 1 < ntiles) {
+          ok = softmax_tile(t + 1, resc_next, ap_nxt, bp_nxt);     // overlaps the PV product of tile t
+          if (!ok) break;
+        }
+        // c6/c7: wait for O^T of tile t, merge it into the running output with that tile's rescale factors
+        ok = wait_bounded(&o_full, gt & 1, abort, p.status);
+        if (!ok) break;
+        if (threadIdx.x == 64 && gt < 6) attn_mark(p, 6 + 4 * gt);
+        tc_fence_after();
+        float resc_cur[kNH];                 // e^(m before tile t - m after tile t), from the softmax of tile t
+#pragma unroll
+        for (int h = 0; h < kNH; ++h) resc_cur[h] = resc_keep[h];
+#pragma unroll
+        for (int j = 0; j < kMaxDVT; ++j) {
+          if (j < p.DVT) {
+            const uint32_t orow = tmem_o + (static_cast<uint32_t>(quad * 32) << 16) + j * p.Rp;
+            uint32_t v1[kMaxHG], v2[kMaxHG];
+            tmem_ldw<kMaxHG>(orow + hs0, v1);
+            tmem_ldw<kMaxHG>(orow + kSlots + hs0, v2);
+            tmem_ld_wait();
+#pragma unroll
+            for (int h = 0; h < kNH; ++h)
+              // alpha_P O1 + beta_P O2 with beta_P = alpha_P / 254: one integer multiply-add and one conversion
+              // (|254 O1 + O2| <= 255 * 128 * 127 * 127 < 2^31)
+              o_run[j][h] = __fmaf_rn(o_run[j][h], resc_cur[h], bp_cur * static_cast<float>(254 * static_cast<int32_t>(v1[h]) + static_cast<int32_t>(v2[h])));
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&o_empty);
+        if (threadIdx.x == 64 && gt < 6) attn_mark(p, 7 + 4 * gt);
+#pragma unroll
+        for (int h = 0; h < kRegState; ++h) resc_keep[h] = resc_next[h];
+        ap_cur = ap_nxt;
+        bp_cur = bp_nxt;
+      }
+      (void)ap_cur;
+      if (threadIdx.x == 64) attn_mark(p, 28);
+      // partial results of this segment: running max, sum of P and unnormalised output per head
+      if (ok) {
+        float (*rb)[kNH + 1] = red[(g0 + ntiles) & 1];
+        named_bar_sync(bar_id, 128);
+#pragma unroll
+        for (int h = 0; h < kNH; ++h) {
+          float l = l_part[h];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+          if (lane == 0) rb[wq][h] = l;
+        }
+        named_bar_sync(bar_id, 128);
+        const int slot = s_slot, bb = s_walk.b;
+        const int h0 = hk * p.G + grp * p.HG;                      // first query head
+        if (slot < p.n_splits) {
+#pragma unroll
+          for (int h = 0; h < kNH; ++h) {
+            if (hs0 + h < nh) {
+              float* dst = p.partial + ((static_cast<long long>(bb) * p.Hq + h0 + hs0 + h) * p.n_splits + slot) * (p.Dv + kPartHdr);
+              // the running maximum goes out in natural-log units (it was kept in the log2 domain)
+              if (tl == 0) { dst[0] = m_run[h] * 0.6931471805599453f; dst[1] = rb[0][h] + rb[1][h] + rb[2][h] + rb[3][h]; }
+#pragma unroll
+              for (int j = 0; j < kMaxDVT; ++j)
+                if (j < p.DVT && j * kChunk + tl < p.Dv) dst[kPartHdr + j * kChunk + tl] = o_run[j][h];
+            }
+          }
+        } else if (tl == 0) {
+          atomicMax(p.status, kStatusBadShape);     // a sequence longer than the max_seqlen the workspace was sized for
+        }
+        // the CTA that reaches the end of a sequence records how many partial results its unit of the sequence has
+        if (kBalanced && tl == 0 && s_walk.t + ntiles == s_walk.nb)
+          p.n_slots[static_cast<long long>(bb) * U + blockIdx.x % U] = min(slot + 1, p.n_splits);
+      }
+      if constexpr (kBalanced) {
+        g0 += ntiles;
+        named_bar_sync(bar_id, 128);                 // everybody has read the walk
+        if (tl == 0) {
+          AttnWalk w = s_walk;
+          attn_walk_advance<true>(p, w, ntiles);
+          s_walk = w;
+          s_slot = 0;                                // every later segment starts its sequence
+        }
+        named_bar_sync(bar_id, 128);
+        more = s_walk.left > 0;
+      } else {
+        more = false;                                // a fixed split is one segment
       }
     }
   }
@@ -1340,13 +1518,21 @@ static int32_t* g_attn_s_dbg = nullptr;
 // One CTA per row; the weights e^{m_s - m} are computed once per split and the O_s rows are read as 16-byte vectors,
 // eight splits' loads in flight per thread.  O is summed over the splits in ascending order.
 __global__ void __launch_bounds__(128)
-attn_combine_kernel(const float* __restrict__ partial, int n_splits, int Dv, __nv_bfloat16* __restrict__ out,
-                    float* __restrict__ lse, int Sq, int Gr, int Hkv) {
+attn_combine_kernel(const float* __restrict__ partial, int n_splits_alloc, const int32_t* __restrict__ n_slots, int G, int HG,
+                    int groups, int Dv, __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int Sq, int Gr, int Hkv) {
   __shared__ float s_w[128];
   __shared__ float s_red[2][4];
   pdl_wait_primary();              // the partial results come from the attention kernel launched just before
   const int PS = Dv + kPartHdr;
-  const float* base = partial + static_cast<long long>(blockIdx.x) * n_splits * PS;
+  const float* base = partial + static_cast<long long>(blockIdx.x) * n_splits_alloc * PS;
+  // balanced schedule: only the first n_slots[unit] partial results of the row exist (unit = (sequence, KV head, head
+  // group) of the row; rows are [B][KV head][G rows], HG rows per group)
+  int n_splits = n_splits_alloc;
+  if (n_slots) {
+    const long long kvh = blockIdx.x / G;
+    const int r = static_cast<int>(blockIdx.x - kvh * G);
+    n_splits = min(n_splits_alloc, __ldg(n_slots + kvh * groups + r / HG));
+  }
   // partial rows are [B][KV head][query token][head of the group]; the output is [B][query token][head]
   long long row = blockIdx.x;
   if (Sq > 1) {
@@ -1407,6 +1593,7 @@ attn_combine_kernel(const float* __restrict__ partial, int n_splits, int Dv, __n
 
 struct AttnPlan {
   int HG, Rp, groups, DC, DVT, n_splits, stages, tmem_cols, v_alias, chunk, kv_chunks;
+  int balanced, q_min;      // balanced schedule: n_splits is the largest number of partial results a unit can have
   size_t smem_bytes, ws_bytes, ws_partial_bytes, ws_qimg_bytes, ws_qscale_bytes;
 };
 
@@ -1445,6 +1632,21 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   }
   pl->n_splits = ns;
   pl->chunk = chunk_tiles * kTok;
+  // Balanced schedule: every CTA of a grid that just fills the machine gets the same number of tiles, at least q_min
+  // (a unit of n tiles then meets at most ceil(n / q_min) + 1 CTAs).  It pays where the fixed splits would leave the
+  // SMs between one and three full-size CTAs each to share out - there the SMs that get one more finish a whole split
+  // later - and costs a few percent elsewhere (every CTA starts at once and cuts its own run first), so it is taken for
+  // that range only, and only by the kernel that keeps three CTAs per SM (up to 4 rows per KV head, D and Dv <= 128).
+  const bool can_balance = pl->HG == 8 && G <= 4 && pl->DC == 1 && pl->DVT == 1 && option(OPT_ATTN_SPLITS) < 1 &&
+                           option(OPT_ATTN_CHUNK_TILES) < 1;
+  const long long items = units * ns, resident = 3LL * sm_count();
+  const int want = option(OPT_ATTN_BALANCED);
+  pl->balanced = (can_balance && (want >= 0 ? want > 0 : (chunk_tiles >= 16 && items >= resident && items <= 3 * resident))) ? 1 : 0;
+  pl->q_min = chunk_tiles >= 4 ? chunk_tiles / 2 : 2;
+  if (pl->balanced) {
+    pl->n_splits = (tiles + pl->q_min - 1) / pl->q_min + 1;
+    ns = pl->n_splits;
+  }
   pl->smem_bytes = static_cast<size_t>(pl->stages) * kv_stage + fixed;
   int cols = 32;
   // wide head groups keep the FP32 running output (4 x 32 columns) behind the two score buffers and the accumulators
@@ -1456,6 +1658,80 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   pl->ws_qscale_bytes = round_up(static_cast<size_t>(units) * 2 * pl->HG * sizeof(float), 1024);
   pl->ws_bytes = pl->ws_partial_bytes + round_up(static_cast<size_t>(units) * sizeof(unsigned), 1024) + pl->ws_qimg_bytes + pl->ws_qscale_bytes;
   return pl->smem_bytes <= 227 * 1024 - 2048;
+}
+
+using AttnKernel = void (*)(CUtensorMap, CUtensorMap, AttnParams);
+
+// The kernel instantiation for a plan (G: query rows per KV head) and its block size.
+static AttnKernel pick_attn_kernel(const AttnPlan& pl, int G, bool paged, int* block_threads) {
+  AttnKernel kernel = nullptr;
+#define MSD_ATTN_PICK_B(HG_, NH_, P_, B_) \
+  kernel = (pl.DVT == 1) ? attn_decode_kernel<HG_, NH_, 1, P_, B_> : (pl.DVT == 2) ? attn_decode_kernel<HG_, NH_, 2, P_, B_> \
+                                                                                   : attn_decode_kernel<HG_, NH_, 4, P_, B_>
+#define MSD_ATTN_PICK(HG_, NH_) \
+  do { if (paged) { MSD_ATTN_PICK_B(HG_, NH_, true, false); } else { MSD_ATTN_PICK_B(HG_, NH_, false, false); } } while (0)
+  *block_threads = kAttnThreads;
+  if (pl.balanced) {        // (plan_attn: HG == 8, G <= 4, one chunk of D and of Dv)
+    kernel = paged ? attn_decode_kernel<8, 4, 1, true, true> : attn_decode_kernel<8, 4, 1, false, true>;
+  } else if (pl.HG == 8) {
+    if (G <= 4) { MSD_ATTN_PICK(8, 4); } else { MSD_ATTN_PICK(8, 8); }
+  } else if (pl.HG == 16) {
+    MSD_ATTN_PICK(16, 16);
+  } else {
+    // wide head groups: 32 head slots per CTA, sixteen softmax warps, held references (attn_decode_wide_kernel)
+    const bool mla = pl.DC == 5 && pl.DVT == 4 && pl.v_alias && pl.stages == 2;     // a 513..640-byte latent row whose first 512 bytes are V
+    if (paged) kernel = mla ? attn_decode_wide_kernel<8, true, 5, 4> : attn_decode_wide_kernel<8, true, 0, 0>;
+    else kernel = mla ? attn_decode_wide_kernel<8, false, 5, 4> : attn_decode_wide_kernel<8, false, 0, 0>;
+    *block_threads = 64 + 128 * 4;
+  }
+#undef MSD_ATTN_PICK
+#undef MSD_ATTN_PICK_B
+  return kernel;
+}
+
+// Raises the dynamic shared-memory limit once per kernel instantiation.
+static bool prepare_attn_kernel(AttnKernel kernel) {
+  static void* done[32] = {};
+  int free_slot = -1;
+  for (int i = 0; i < 32; ++i) {
+    if (done[i] == reinterpret_cast<void*>(kernel)) return true;
+    if (!done[i] && free_slot < 0) free_slot = i;
+  }
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess) return false;
+  if (free_slot >= 0) done[free_slot] = reinterpret_cast<void*>(kernel);
+  return true;
+}
+
+// Grid of the balanced schedule: as many CTAs as are resident at once, rounded down to whole sets of U (one CTA per
+// unit), at least one set (0: the query failed).
+static int attn_balanced_ctas(AttnKernel kernel, int block_threads, size_t smem_bytes, int tmem_cols, int U) {
+  struct Entry { void* k; size_t smem; int ctas; };
+  static Entry cache[32] = {};
+  for (const Entry& e : cache)
+    if (e.k == reinterpret_cast<void*>(kernel) && e.smem == smem_bytes) return std::max(e.ctas / U, 1) * U;
+  // Resident CTAs per SM from the kernel's own resource use (the runtime's occupancy query assumes the default
+  // shared-memory carve-out, not the one a kernel with this much dynamic shared memory gets).
+  cudaFuncAttributes fa;
+  int dev = 0, smem_sm = 0, smem_resv = 0, regs_sm = 0, threads_sm = 0;
+  if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess || cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&smem_resv, cudaDevAttrReservedSharedMemoryPerBlock, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&regs_sm, cudaDevAttrMaxRegistersPerMultiprocessor, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&threads_sm, cudaDevAttrMaxThreadsPerMultiProcessor, dev) != cudaSuccess)
+    return 0;
+  const int warps = (block_threads + 31) / 32;
+  const int regs_warp = (fa.numRegs * 32 + 255) / 256 * 256;                 // registers are handed out per warp, 256 at a time
+  int per_sm = static_cast<int>(smem_sm / (smem_bytes + fa.sharedSizeBytes + smem_resv));
+  // (the register file is four banks, one per scheduler; a CTA's warps are dealt out over them)
+  while (per_sm > 1 && (per_sm * warps + 3) / 4 * regs_warp > regs_sm / 4) --per_sm;
+  per_sm = std::min(per_sm, threads_sm / block_threads);
+  per_sm = std::min(per_sm, 512 / tmem_cols);                                // tensor memory: 512 columns per SM
+  if (per_sm < 1) per_sm = 1;
+  const int ctas = per_sm * sm_count();
+  for (Entry& e : cache)
+    if (!e.k) { e.k = reinterpret_cast<void*>(kernel); e.smem = smem_bytes; e.ctas = ctas; break; }
+  return std::max(ctas / U, 1) * U;
 }
 
 }  // namespace msd
@@ -1494,7 +1770,49 @@ msd_status_t msd_attn_decode_schedule(int32_t B, int32_t Hq, int32_t Hkv, int32_
   if (!msd::plan_attn(B, Hq, Hkv, D, Dv, max_seqlen, false, &pl)) return MSD_ERR_BAD_SHAPE;
   *tile = msd::kTok;
   *n_splits = pl.n_splits;
-  if (split_tokens) *split_tokens = pl.chunk;
+  if (split_tokens) *split_tokens = pl.balanced ? 0 : pl.chunk;
+  return MSD_OK;
+}
+
+msd_status_t msd_attn_decode_split_starts(int32_t B, int32_t q_len, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
+                                          int32_t max_seqlen, int32_t paged, int32_t v_aliased, const int32_t* seqlens,
+                                          int32_t* starts) {
+  using namespace msd;
+  if (!seqlens || !starts) return MSD_ERR_NULL_POINTER;
+  if (q_len < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || B < 1) return MSD_ERR_BAD_SHAPE;
+  AttnPlan pl;
+  if (!plan_attn(B, Hq * q_len, Hkv, D, Dv, max_seqlen > 0 ? max_seqlen : 1, v_aliased != 0, &pl)) return MSD_ERR_BAD_SHAPE;
+  const int G = Hq * q_len / Hkv, U = Hkv * pl.groups, ns = pl.n_splits;
+  long long R = 0, W = 0;
+  if (pl.balanced) {
+    int block_threads = 0;
+    AttnKernel kernel = pick_attn_kernel(pl, G, paged != 0, &block_threads);
+    if (!prepare_attn_kernel(kernel)) return MSD_ERR_CUDA;
+    const int ctas = attn_balanced_ctas(kernel, block_threads, pl.smem_bytes, pl.tmem_cols, U);
+    if (ctas < 1) return MSD_ERR_CUDA;
+    for (int b = 0; b < B; ++b) W += seqlens[b] > 0 ? (seqlens[b] + kTok - 1) / kTok : 0;
+    R = std::min<long long>(W / pl.q_min, ctas / U);
+    R = R < 1 ? 1 : R;
+  }
+  long long P = 0;                                   // tiles of the sequences in front
+  for (int b = 0; b < B; ++b) {
+    const int L = seqlens[b] > 0 ? seqlens[b] : 0;
+    const long long nb = (L + kTok - 1) / kTok;
+    int32_t* first_row = starts + static_cast<long long>(b) * Hkv * G * (ns + 1);
+    int n = 0;
+    first_row[n++] = 0;
+    if (pl.balanced) {
+      // the runs [i W / R, (i+1) W / R) that begin inside this sequence's tiles [P, P + nb)
+      if (nb > 0)
+        for (long long i = ((P + 1) * R - 1) / W + 1; i < R && i * W / R < P + nb && n < ns; ++i)
+          first_row[n++] = static_cast<int32_t>((i * W / R - P) * kTok);
+    } else {
+      for (int sidx = 1; sidx < ns; ++sidx) first_row[n++] = static_cast<int32_t>(std::min<long long>(L, static_cast<long long>(sidx) * pl.chunk));
+    }
+    while (n <= ns) first_row[n++] = L;
+    for (int r = 1; r < Hkv * G; ++r) std::copy(first_row, first_row + ns + 1, first_row + static_cast<long long>(r) * (ns + 1));
+    P += nb;
+  }
   return MSD_OK;
 }
 
@@ -1565,45 +1883,17 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
   p.status = status;
   p.trace = g_attn_trace;
 
-  void (*kernel)(CUtensorMap, CUtensorMap, AttnParams) = nullptr;
-  const int G = Hq / Hkv;
-#define MSD_ATTN_PICK_P(HG_, NH_, P_) \
-  kernel = (pl.DVT == 1) ? attn_decode_kernel<HG_, NH_, 1, P_> : (pl.DVT == 2) ? attn_decode_kernel<HG_, NH_, 2, P_> \
-                                                                               : attn_decode_kernel<HG_, NH_, 4, P_>
-#define MSD_ATTN_PICK(HG_, NH_) \
-  do { if (paged) { MSD_ATTN_PICK_P(HG_, NH_, true); } else { MSD_ATTN_PICK_P(HG_, NH_, false); } } while (0)
   int block_threads = kAttnThreads;
-  if (pl.HG == 8) {
-    if (G <= 4) { MSD_ATTN_PICK(8, 4); } else { MSD_ATTN_PICK(8, 8); }
-  } else if (pl.HG == 16) {
-    MSD_ATTN_PICK(16, 16);
-  } else {
-    // wide head groups: 32 head slots per CTA, sixteen softmax warps, held references (attn_decode_wide_kernel)
-    const bool mla = pl.DC == 5 && pl.DVT == 4 && pl.v_alias && pl.stages == 2;     // a 513..640-byte latent row whose first 512 bytes are V
-    if (paged) kernel = mla ? attn_decode_wide_kernel<8, true, 5, 4> : attn_decode_wide_kernel<8, true, 0, 0>;
-    else kernel = mla ? attn_decode_wide_kernel<8, false, 5, 4> : attn_decode_wide_kernel<8, false, 0, 0>;
-    block_threads = 64 + 128 * 4;
-  }
-#undef MSD_ATTN_PICK
-#undef MSD_ATTN_PICK_P
-  {
-    // raise the dynamic shared-memory limit once per kernel instantiation
-    static void* done[32] = {};
-    bool seen = false;
-    int free_slot = -1;
-    for (int i = 0; i < 32; ++i) {
-      if (done[i] == reinterpret_cast<void*>(kernel)) seen = true;
-      if (!done[i] && free_slot < 0) free_slot = i;
-    }
-    if (!seen) {
-      if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess)
-        return MSD_ERR_CUDA;
-      if (free_slot >= 0) done[free_slot] = reinterpret_cast<void*>(kernel);
-    }
-  }
+  AttnKernel kernel = pick_attn_kernel(pl, Hq / Hkv, paged, &block_threads);
+  if (!prepare_attn_kernel(kernel)) return MSD_ERR_CUDA;
+  p.balanced = pl.balanced; p.q_min = pl.q_min;
+  p.n_slots = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + pl.ws_partial_bytes);
+  int balanced_ctas = 0;
+  if (pl.balanced && (balanced_ctas = attn_balanced_ctas(kernel, block_threads, pl.smem_bytes, pl.tmem_cols, Hkv * pl.groups)) < 1) return MSD_ERR_CUDA;
   // narrow groups: units along x; wide groups: splits along x (see the kernels)
   dim3 grid(B * Hkv * pl.groups, pl.n_splits);
   if (block_threads > kAttnThreads) grid = dim3(pl.n_splits, B * Hkv * pl.groups);
+  if (pl.balanced) grid = dim3(balanced_ctas);
   if (block_threads > kAttnThreads) {
     // wide head groups: the stacked Q operands come from a kernel of their own, the attention kernel is its
     // programmatic dependent (its CTAs start their KV loads while it runs)
@@ -1616,7 +1906,8 @@ static msd_status_t attn_launch(const void* q_bf16, const int8_t* k_cache, const
     if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
   }
   if (launch_pdl(attn_combine_kernel, dim3(B * Hq), dim3(128), 0, s, option(OPT_NO_PDL) <= 0, static_cast<const float*>(p.partial),
-                 pl.n_splits, Dv, static_cast<__nv_bfloat16*>(out_bf16), lse, q_len, Hq / (Hkv * q_len), Hkv) != cudaSuccess)
+                 pl.n_splits, static_cast<const int32_t*>(pl.balanced ? p.n_slots : nullptr), Hq / Hkv, pl.HG, pl.groups, Dv,
+                 static_cast<__nv_bfloat16*>(out_bf16), lse, q_len, Hq / (Hkv * q_len), Hkv) != cudaSuccess)
     return MSD_ERR_CUDA;
   return launch_status();
 }

@@ -27,6 +27,7 @@ enum Option {
   OPT_W4_KSPLIT,            // MSD_W4_KSPLIT: its K split
   OPT_ATTN_SPLITS,          // MSD_ATTN_SPLITS: number of context splits of the attention kernels
   OPT_ATTN_CHUNK_TILES,     // MSD_ATTN_CHUNK_TILES: tiles per context split
+  OPT_ATTN_BALANCED,        // MSD_ATTN_BALANCED: 1 balanced schedule wherever a kernel for it exists, 0 never
   OPT_COUNT
 };
 int option(Option o);

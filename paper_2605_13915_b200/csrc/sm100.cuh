@@ -9,6 +9,7 @@
 namespace msd {
 
 constexpr unsigned kStatusTimeout = 7;                   // == MSD_ERR_TIMEOUT
+constexpr unsigned kStatusBadShape = 2;                  // == MSD_ERR_BAD_SHAPE (an input on the device contradicts the call's sizes)
 constexpr long long kWaitBudgetCycles = 2000000000LL;    // about one second of SM clocks
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

@@ -12,9 +12,13 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-3
 
 
-def _split_starts(seqlens, ns, split_tokens):
-    L = np.asarray(seqlens, dtype=np.int64)
-    return np.minimum(L[:, None], np.arange(ns + 1)[None, :] * split_tokens).astype(np.int32)
+def _split_starts(c, all_seqlens=None, max_seqlen=None, q_len=1, paged=False):
+    """The kernel's context splits for every (sequence, query head) of a call over sequences of these lengths:
+    ([B, Hkv, q_len * Hq / Hkv, n_splits + 1] token offsets, tile)."""
+    Hq, D = c.q.shape[1] // q_len, c.q.shape[2]
+    L = np.diff(c.cu_seqlens) if all_seqlens is None else np.asarray(all_seqlens)
+    return binding.attn_decode_split_starts(L, Hq, c.k.shape[1], D, c.dv, max(max_seqlen or int(L.max()), 1), q_len=q_len,
+                                            paged=paged, v_aliased=c.v is None)
 
 
 def _run_gpu(c, want_lse=True):
@@ -32,14 +36,18 @@ def _run_gpu(c, want_lse=True):
     return out
 
 
-def _oracle_tiled(c, B_sched=None, max_seqlen=None):
+def _oracle_tiled(c, all_seqlens=None, seqs=None, max_seqlen=None, paged=False):
+    """The oracle's tiled mode on case c with the splits the kernel takes.  all_seqlens / seqs: c holds only the
+    sequences `seqs` of a call over sequences of lengths all_seqlens (the splits depend on all of them)."""
     B, Hq, D = c.q.shape
     Hkv = c.k.shape[1]
-    shape = (B_sched or B, Hq, Hkv, D, c.dv, max(max_seqlen or c.max_seqlen, 1))
-    tile, ns, st = binding.attn_decode_schedule(*shape)
-    ss = _split_starts(np.diff(c.cu_seqlens), ns, st)
+    starts, tile = _split_starts(c, all_seqlens, max_seqlen, paged=paged)
+    ss = starts.reshape(starts.shape[0], Hq, -1)
+    if seqs is not None:
+        ss = ss[seqs]
+    shape = (starts.shape[0], Hq, Hkv, D, c.dv, max(max_seqlen or c.max_seqlen, 1))
     return oracle.attn_decode_int8kv(c.q, c.k, c.v, c.k_scale, c.v_scale, c.cu_seqlens, c.softmax_scale, dv=c.dv,
-                                     split_starts=ss, tile=tile, want_lse=True, **_softmax_mode(*shape))
+                                     split_starts=np.ascontiguousarray(ss), tile=tile, want_lse=True, **_softmax_mode(*shape))
 
 
 def _softmax_mode(*shape):
@@ -96,6 +104,57 @@ def test_split_counts(splits, monkeypatch):
     _check(inputs.gqa_case(2, 8, 2, 128, [1000, 3000], seed=9))
 
 
+# ---- the balanced split schedule (equal runs of the list of all sequences' tiles, one CTA per run and unit) ------------
+@pytest.mark.parametrize("B,Hq,Hkv,seqlens", [
+    (3, 8, 2, [700, 64, 1500]),                       # runs that cross sequence boundaries
+    (4, 8, 8, [1, 127, 0, 300]),                      # one row per KV head, an empty sequence in the middle
+    (2, 32, 8, [129, 4000]),                          # many runs inside one sequence
+    (6, 12, 4, [0, 0, 513, 0, 90, 0]),                # empty sequences first, between and last; 3 rows per KV head
+    (1, 4, 1, [128]),                                 # a single tile
+])
+def test_balanced_schedule_parity(B, Hq, Hkv, seqlens):
+    binding.debug_set_option("MSD_ATTN_BALANCED", 1)
+    c = inputs.gqa_case(B, Hq, Hkv, 128, seqlens, seed=3 * B + Hq)
+    assert binding.attn_decode_schedule(B, Hq, Hkv, 128, 128, max(c.max_seqlen, 1))[2] == 0      # the balanced schedule is in force
+    _check(c)
+
+
+def test_balanced_schedule_many_short_sequences():
+    """Every CTA walks several sequences (segments), some of them empty, with a different number of tiles each."""
+    binding.debug_set_option("MSD_ATTN_BALANCED", 1)
+    rng = np.random.default_rng(5)
+    seqlens = [int(x) for x in rng.integers(0, 1200, 300)]
+    seqlens[7] = seqlens[8] = seqlens[299] = 0
+    c = inputs.gqa_case(len(seqlens), 8, 2, 128, seqlens, seed=77)
+    starts, _ = _split_starts(c)
+    assert (np.diff(starts[:, 0, 0], axis=1) > 0).sum(axis=1).max() >= 2       # some sequence is cut by a run boundary
+    _check(c)
+
+
+def test_balanced_schedule_is_the_default_where_it_pays():
+    """Between one and three fixed splits per resident CTA the balanced schedule is taken; with many more it is not."""
+    assert binding.attn_decode_schedule(32, 32, 8, 128, 128, 8192)[2] == 0
+    assert binding.attn_decode_schedule(512, 32, 8, 128, 128, 8192)[2] > 0
+    assert binding.attn_decode_schedule(1, 32, 8, 128, 128, 8192)[2] > 0
+    assert binding.attn_decode_schedule(32, 64, 8, 128, 128, 8192)[2] > 0        # 8 rows per KV head: fixed splits
+    binding.debug_set_option("MSD_ATTN_BALANCED", 0)
+    assert binding.attn_decode_schedule(32, 32, 8, 128, 128, 8192)[2] > 0
+
+
+def test_balanced_schedule_sequence_longer_than_declared():
+    """A sequence longer than the max_seqlen the workspace was sized for: reported, nothing written out of bounds
+    (the guard bands of the workspace are checked when the test ends)."""
+    binding.debug_set_option("MSD_ATTN_BALANCED", 1)
+    c = inputs.gqa_case(1, 8, 2, 128, [4000], seed=4)
+    binding.attn_decode_int8kv(bf16_dev(c.q), dev(c.k), dev(c.v), dev(c.k_scale), dev(c.v_scale), dev(c.cu_seqlens), 512,
+                               c.softmax_scale, dv=c.dv)
+    torch.cuda.synchronize()
+    with pytest.raises(binding.MsdError) as e:
+        binding.last_device_status()
+    assert e.value.code == 2                          # MSD_ERR_BAD_SHAPE
+    binding.last_device_status()                      # cleared
+
+
 def test_accuracy_ordering_vs_dequant():
     c = inputs.gqa_case(4, 32, 8, 128, [2048, 3000, 4096, 777], seed=1)
     o = _run_gpu(c, want_lse=False)
@@ -130,7 +189,7 @@ def test_gqa_full_size_sampled_sequences():
     got = oracle.bf16_bits_to_f64(bf16_bits(o))
     seqs = [0, 17, 31]
     sub = _subcase(c, seqs)
-    ref, _ = _oracle_tiled(sub, B_sched=B, max_seqlen=c.max_seqlen)
+    ref, _ = _oracle_tiled(sub, all_seqlens=np.diff(c.cu_seqlens), seqs=seqs, max_seqlen=c.max_seqlen)
     _assert_close(got[seqs], ref)
 
 
@@ -141,7 +200,7 @@ def test_mla_full_size_sampled_sequence():
     o = _run_gpu(c, want_lse=False)
     got = oracle.bf16_bits_to_f64(bf16_bits(o))
     sub = _subcase(c, [37])
-    ref, _ = _oracle_tiled(sub, B_sched=B, max_seqlen=L)
+    ref, _ = _oracle_tiled(sub, all_seqlens=[L] * B, seqs=[37], max_seqlen=L)
     _assert_close(got[[37]], ref)
 
 
@@ -180,10 +239,13 @@ def test_dequant_bf16_comparison_arm_is_less_accurate():
     assert np.linalg.norm(msd - ref) <= np.linalg.norm(got - ref) * 1.05
 
 
-@pytest.mark.parametrize("page", [16, 64, 128])
+@pytest.mark.parametrize("page", [16, 64, 128, -64])
 def test_paged_cache_gqa(page):
     """The same sequences scattered over a paged cache (random block order, noise in the unused blocks and in the tails
     of the last blocks) must give what the contiguous cache gives: the oracle's tiled mode on the contiguous case."""
+    if page < 0:                                      # the same under the balanced split schedule
+        binding.debug_set_option("MSD_ATTN_BALANCED", 1)
+        page = -page
     seqlens = [1, 130, 700, 0, 257, 2049]
     c = inputs.gqa_case(B=len(seqlens), Hq=16, Hkv=4, D=128, seqlens=seqlens, seed=61)
     k, v, ks, vs, table, sl = inputs.paginate(c, page, seed=page)
@@ -191,7 +253,7 @@ def test_paged_cache_gqa(page):
                                               max(c.max_seqlen, 1), c.softmax_scale, want_lse=True)
     torch.cuda.synchronize()
     binding.last_device_status()
-    ref, lse_ref = _oracle_tiled(c)
+    ref, lse_ref = _oracle_tiled(c, paged=True)
     got = oracle.bf16_bits_to_f64(bf16_bits(o))
     live = np.isfinite(lse_ref)
     _assert_close(got[live], ref[live])
@@ -209,7 +271,7 @@ def test_paged_cache_mla_and_bad_page_size():
                                          c.softmax_scale, dv=c.dv)
     torch.cuda.synchronize()
     binding.last_device_status()
-    ref, _ = _oracle_tiled(c)
+    ref, _ = _oracle_tiled(c, paged=True)
     _assert_close(oracle.bf16_bits_to_f64(bf16_bits(o)), ref)
     with pytest.raises(binding.MsdError):
         binding.attn_decode_int8kv_paged(bf16_dev(c.q), dev(k), None, dev(ks), None, dev(table), dev(sl), 48, c.max_seqlen,
@@ -225,10 +287,13 @@ def _truncate(c, drop):
     return keep, cu
 
 
-@pytest.mark.parametrize("Sq,Hq,Hkv", [(4, 8, 2), (2, 16, 2), (3, 8, 8), (3, 16, 1)])
+@pytest.mark.parametrize("Sq,Hq,Hkv", [(4, 8, 2), (2, 16, 2), (3, 8, 8), (3, 16, 1), (-3, 8, 8), (-2, 8, 4)])
 def test_speculative_decode_rows_are_causal_single_query_problems(Sq, Hq, Hkv):
     """Sq query tokens per sequence: query token s must equal the single-query problem on the cache without the last
     Sq - 1 - s tokens (the oracle, tiled with the kernel's tile and split boundaries)."""
+    if Sq < 0:                                        # the same under the balanced split schedule
+        binding.debug_set_option("MSD_ATTN_BALANCED", 1)
+        Sq = -Sq
     seqlens = [Sq, 131, 700, 2100]
     base = inputs.gqa_case(B=len(seqlens), Hq=Hq * Sq, Hkv=Hkv, D=128, seqlens=seqlens, seed=71)
     B = len(seqlens)
@@ -238,10 +303,11 @@ def test_speculative_decode_rows_are_causal_single_query_problems(Sq, Hq, Hkv):
     torch.cuda.synchronize()
     binding.last_device_status()
     got = oracle.bf16_bits_to_f64(bf16_bits(out))
-    tile, ns, st = binding.attn_decode_schedule(B, Hq * Sq, Hkv, 128, 128, base.max_seqlen)
+    starts, tile = _split_starts(base, q_len=Sq)             # [B, Hkv, Sq * Gr, n_splits + 1], rows token-major
+    Gr = Hq // Hkv
     for s in range(Sq):
         keep, cu = _truncate(base, Sq - 1 - s)
-        ss = _split_starts(np.diff(cu), ns, st)
+        ss = np.ascontiguousarray(starts[:, :, s * Gr:(s + 1) * Gr]).reshape(B, Hq, -1)     # (clipped to the shorter cache by the oracle)
         ref, lse_ref = oracle.attn_decode_int8kv(np.ascontiguousarray(q[:, s]), base.k[keep], base.v[keep], base.k_scale[keep],
                                                  base.v_scale[keep], cu, base.softmax_scale, dv=128, tile=tile,
                                                  split_starts=ss, want_lse=True,

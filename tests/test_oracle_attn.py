@@ -116,6 +116,18 @@ def test_tiled_mode_tracks_definition(gqa_small):
     assert np.abs(tiled - glob).max() <= 5e-4 * rown.max()
     assert np.all(np.abs(tiled - glob) <= 1e-3 * rown)
     assert np.allclose(lse_t, lse_g, rtol=0, atol=1e-9)
+    # splits given per (sequence, head): the same per head as per sequence, and a head with splits of its own gets
+    # exactly what a call with those splits for everybody gives that head
+    B, Hq = c.q.shape[:2]
+    per_head = np.repeat(ss[:, None, :], Hq, axis=1)
+    assert np.array_equal(oracle.attn_decode_int8kv(*args, mode="tiled", tile=64, split_starts=per_head), tiled)
+    other = np.stack([0 * L, L // 2, L // 2, L], 1)
+    mixed = per_head.copy()
+    mixed[:, 1] = other
+    got = oracle.attn_decode_int8kv(*args, mode="tiled", tile=64, split_starts=mixed)
+    alt = oracle.attn_decode_int8kv(*args, mode="tiled", tile=64, split_starts=other)
+    assert np.array_equal(got[:, 1], alt[:, 1]) and np.array_equal(got[:, 0], tiled[:, 0]) and np.array_equal(got[:, 2:], tiled[:, 2:])
+    assert not np.array_equal(alt[:, 1], tiled[:, 1])
 
 
 def test_held_references_mode(gqa_small):
