@@ -98,10 +98,18 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // c1 for one query row (one warp): head slot h of the group's stacked operand (rows h and HG + h of every 128-byte
 // chunk at `img`, 128-byte swizzle) and its two scales.  `img` is shared memory in the attention kernel's own set-up
 // and global memory in attn_qstack_kernel; same bit-exact rule as msd_decompose_int8.
+// index of the query row behind head slot h of a group: row r of the KV head -> (query token, head of the group)
+__device__ __forceinline__ long long attn_q_row_index(const AttnParams& p, int b, int hk, int grp, int h) {
+  const int r_kv = grp * p.HG + h, sq = r_kv / p.Gr;
+  return (static_cast<long long>(b) * p.Sq + sq) * (p.Hkv * p.Gr) + hk * p.Gr + (r_kv - sq * p.Gr);
+}
+__device__ __forceinline__ void prefetch_l2(const void* ptr) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+}
+
 __device__ __forceinline__ void attn_decompose_q_row(const AttnParams& p, int b, int hk, int grp, int h, int lane, uint8_t* img,
                                                      float* alpha_out, float* beta_out) {
-  const int r_kv = grp * p.HG + h, sq = r_kv / p.Gr;       // row of this KV head -> (query token, head of the group)
-  const long long q_row = (static_cast<long long>(b) * p.Sq + sq) * (p.Hkv * p.Gr) + hk * p.Gr + (r_kv - sq * p.Gr);
+  const long long q_row = attn_q_row_index(p, b, hk, grp, h);
   const uint4* qrow = reinterpret_cast<const uint4*>(p.q + q_row * p.D);
   const int nvec = p.D >> 3;                    // 8 BF16 values per 16-byte load (D % 16 == 0, D <= 640)
   uint4 qv[3];                                  // the whole row stays in registers between the two passes
@@ -303,6 +311,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   constexpr int kNSW = 4;                          // component, rows [kSlots, 2*kSlots) second component
   __shared__ float s_aq[kSlots], s_bq[kSlots];
   __shared__ float red[2][4][kNH + 1];             // per-warp tile maxima, double buffered by tile parity
+  // More than 4 heads per thread: what is the same in all threads of a warp and only read now and then - the query
+  // scales, and the rescale factors a tile's softmax hands to its merge - stays in shared memory (per warp, by tile
+  // parity), or the kernel does not fit the 96 registers that three CTAs per SM allow.
+  constexpr bool kSmemState = kNH > 4;
+  __shared__ float s_resc[kSmemState ? 2 : 1][4][kNH];
   __shared__ int s_scan[kAttnThreads];
   __shared__ AttnWalk s_walk;                      // the softmax warps' walk (kept here, not in registers, between segments)
   __shared__ int s_slot;
@@ -378,6 +391,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     mbar_init(&p_full[0], kNSW); mbar_init(&p_full[1], kNSW); mbar_init(&q_ready, kNSW);
     mbar_init(&o_full, 1); mbar_init(&o_empty, kNSW);
     abort_flag = 0;
+    for (int h = 0; h < kSlots; ++h) { s_aq[h] = 0.0f; s_bq[h] = 0.0f; }      // head slots without a head
     s_walk = w0;
     s_slot = slot0;
     mbar_init_fence();
@@ -567,7 +581,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       const int t_end = min(L, t_begin + ntiles * kTok);
       // c1: decompose the query rows of this segment's heads (one warp per head, round robin) into the stacked operand
       // (the head slots and padding columns that were zeroed at the start are never written)
-      for (int h = wi; h < nh; h += kNSW) attn_decompose_q_row(p, b, hk, grp, h, lane, sm_q, &s_aq[h], &s_bq[h]);
+      for (int h = wi; h < nh; h += kNSW) {
+        // a warp with a second row asks for it now: two cold reads one after the other cost microseconds
+        if (h + kNSW < nh && lane * 64 < p.D) prefetch_l2(p.q + attn_q_row_index(p, b, hk, grp, h + kNSW) * p.D + lane * 64);
+        attn_decompose_q_row(p, b, hk, grp, h, lane, sm_q, &s_aq[h], &s_bq[h]);
+      }
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&q_ready);           // the stacked Q operand is in shared memory
@@ -583,8 +601,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       for (int h = 0; h < kNH; ++h) {
         l_part[h] = 0.0f;
         m_run[h] = -INFINITY;
-        aq[h] = (hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f;
-        bq[h] = (hs0 + h < nh) ? s_bq[hs0 + h] : 0.0f;
+        aq[h] = (!kSmemState && hs0 + h < nh) ? s_aq[hs0 + h] : 0.0f;
+        bq[h] = (!kSmemState && hs0 + h < nh) ? s_bq[hs0 + h] : 0.0f;
 #pragma unroll
         for (int j = 0; j < kMaxDVT; ++j) o_run[j][h] = 0.0f;
       }
@@ -637,7 +655,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
           for (int h = 0; h < kNH; ++h)
           {
-            const float a_q = aq[h], b_q = bq[h];
+            const float a_q = kSmemState ? s_aq[hs0 + h] : aq[h], b_q = kSmemState ? s_bq[hs0 + h] : bq[h];
             bool vh = valid;
             if (p.Sq > 1) vh = valid && tok_rel < L - p.Sq + 1 + (grp * p.HG + hs0 + h) / p.Gr;    // causal among the new tokens
             s[h] = vh ? __fmaf_rn(a_q, static_cast<float>(static_cast<int32_t>(v1[h])), b_q * static_cast<float>(static_cast<int32_t>(v2[h]))) * ks : -INFINITY;
@@ -664,7 +682,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           mn_t[h] = fmaxf(m_run[h], mt);
           resc_t[h] = (m_run[h] == -INFINITY) ? 0.0f : ex2_approx(m_run[h] - mn_t[h]);
           m_run[h] = mn_t[h];
-          resc_out[h] = resc_t[h];
+          if constexpr (kSmemState) { if (lane == 0) s_resc[gt & 1][wq][h] = resc_t[h]; }      // (__syncwarp below, before P is announced)
+          else resc_out[h] = resc_t[h];
         }
         const float vs_max = fmaxf(fmaxf(rb[0][kNH], rb[1][kNH]), fmaxf(rb[2][kNH], rb[3][kNH]));
         // c5: P = exp(S - m), fold the value scale, two-pass INT8 with the fixed scale alpha_P = max(v_scale)/127
@@ -712,7 +731,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         tc_fence_after();
         float resc_cur[kNH];                 // e^(m before tile t - m after tile t), from the softmax of tile t
 #pragma unroll
-        for (int h = 0; h < kNH; ++h) resc_cur[h] = resc_keep[h];
+        for (int h = 0; h < kNH; ++h) resc_cur[h] = kSmemState ? s_resc[gt & 1][wq][h] : resc_keep[h];
 #pragma unroll
         for (int j = 0; j < kMaxDVT; ++j) {
           if (j < p.DVT) {
@@ -1633,15 +1652,17 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   pl->n_splits = ns;
   pl->chunk = chunk_tiles * kTok;
   // Balanced schedule: every CTA of a grid that just fills the machine gets the same number of tiles, at least q_min
-  // (a unit of n tiles then meets at most ceil(n / q_min) + 1 CTAs).  It pays where the fixed splits would leave the
-  // SMs between one and three full-size CTAs each to share out - there the SMs that get one more finish a whole split
-  // later - and costs a few percent elsewhere (every CTA starts at once and cuts its own run first), so it is taken for
-  // that range only, and only by the kernel that keeps three CTAs per SM (up to 4 rows per KV head, D and Dv <= 128).
-  const bool can_balance = pl->HG == 8 && G <= 4 && pl->DC == 1 && pl->DVT == 1 && option(OPT_ATTN_SPLITS) < 1 &&
+  // (a unit of n tiles then meets at most ceil(n / q_min) + 1 CTAs).  It pays where full-size fixed splits (16 tiles)
+  // would leave the resident CTAs between one and three items each to share out - there the SMs that get one more
+  // finish a whole split later - and the sequences are long enough (32 tiles) for a run to stay inside one or two of
+  // them; elsewhere it costs a few percent (every CTA starts at once and cuts its own run first; every sequence a run
+  // enters is a new set-up).  Built for the kernels that keep three CTAs per SM (up to 8 rows per KV head, D and
+  // Dv <= 128).
+  const bool can_balance = pl->HG == 8 && pl->DC == 1 && pl->DVT == 1 && option(OPT_ATTN_SPLITS) < 1 &&
                            option(OPT_ATTN_CHUNK_TILES) < 1;
-  const long long items = units * ns, resident = 3LL * sm_count();
+  const long long items16 = units * ((tiles + 15) / 16), resident = 3LL * sm_count();
   const int want = option(OPT_ATTN_BALANCED);
-  pl->balanced = (can_balance && (want >= 0 ? want > 0 : (chunk_tiles >= 16 && items >= resident && items <= 3 * resident))) ? 1 : 0;
+  pl->balanced = (can_balance && (want >= 0 ? want > 0 : (tiles >= 32 && items16 >= resident && items16 <= 3 * resident))) ? 1 : 0;
   pl->q_min = chunk_tiles >= 4 ? chunk_tiles / 2 : 2;
   if (pl->balanced) {
     pl->n_splits = (tiles + pl->q_min - 1) / pl->q_min + 1;
@@ -1671,8 +1692,9 @@ static AttnKernel pick_attn_kernel(const AttnPlan& pl, int G, bool paged, int* b
 #define MSD_ATTN_PICK(HG_, NH_) \
   do { if (paged) { MSD_ATTN_PICK_B(HG_, NH_, true, false); } else { MSD_ATTN_PICK_B(HG_, NH_, false, false); } } while (0)
   *block_threads = kAttnThreads;
-  if (pl.balanced) {        // (plan_attn: HG == 8, G <= 4, one chunk of D and of Dv)
-    kernel = paged ? attn_decode_kernel<8, 4, 1, true, true> : attn_decode_kernel<8, 4, 1, false, true>;
+  if (pl.balanced) {        // (plan_attn: HG == 8, one chunk of D and of Dv)
+    if (G <= 4) kernel = paged ? attn_decode_kernel<8, 4, 1, true, true> : attn_decode_kernel<8, 4, 1, false, true>;
+    else kernel = paged ? attn_decode_kernel<8, 8, 1, true, true> : attn_decode_kernel<8, 8, 1, false, true>;
   } else if (pl.HG == 8) {
     if (G <= 4) { MSD_ATTN_PICK(8, 4); } else { MSD_ATTN_PICK(8, 8); }
   } else if (pl.HG == 16) {

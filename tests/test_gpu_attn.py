@@ -111,6 +111,8 @@ def test_split_counts(splits, monkeypatch):
     (2, 32, 8, [129, 4000]),                          # many runs inside one sequence
     (6, 12, 4, [0, 0, 513, 0, 90, 0]),                # empty sequences first, between and last; 3 rows per KV head
     (1, 4, 1, [128]),                                 # a single tile
+    (3, 16, 2, [700, 64, 1500]),                      # 8 rows per KV head
+    (2, 14, 2, [0, 2100]),                            # 7 rows per KV head
 ])
 def test_balanced_schedule_parity(B, Hq, Hkv, seqlens):
     binding.debug_set_option("MSD_ATTN_BALANCED", 1)
@@ -136,7 +138,9 @@ def test_balanced_schedule_is_the_default_where_it_pays():
     assert binding.attn_decode_schedule(32, 32, 8, 128, 128, 8192)[2] == 0
     assert binding.attn_decode_schedule(512, 32, 8, 128, 128, 8192)[2] > 0
     assert binding.attn_decode_schedule(1, 32, 8, 128, 128, 8192)[2] > 0
-    assert binding.attn_decode_schedule(32, 64, 8, 128, 128, 8192)[2] > 0        # 8 rows per KV head: fixed splits
+    assert binding.attn_decode_schedule(32, 64, 8, 128, 128, 8192)[2] == 0       # 8 rows per KV head as well
+    assert binding.attn_decode_schedule(32, 128, 8, 128, 128, 8192)[2] > 0       # 16 rows per KV head: fixed splits
+    assert binding.attn_decode_schedule(256, 32, 8, 128, 128, 1024)[2] > 0       # short sequences: fixed splits
     binding.debug_set_option("MSD_ATTN_BALANCED", 0)
     assert binding.attn_decode_schedule(32, 32, 8, 128, 128, 8192)[2] > 0
 
