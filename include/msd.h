@@ -335,7 +335,7 @@ msd_status_t msd_attn_decode_int8kv_paged(const void* q_bf16, const int8_t* k_ca
  * number of context splits a (sequence, query row) can have and the tokens per split.  With *split_tokens > 0 split s
  * of a sequence of length L covers tokens [s*split_tokens, min(L, (s+1)*split_tokens)) and is walked in tiles of
  * `tile` tokens (splits past L are empty).  *split_tokens = 0: the splits depend on the lengths of all sequences of
- * the call (Sec. 4.3 leaves the partition of the context open; head groups of up to 16 rows per KV head cut the list
+ * the call (Sec. 4.3 leaves the partition of the context open; head groups of up to 8 rows per KV head may cut the list
  * of all sequences' tiles into equal runs, as many as fit the machine at once, so that no SM is left with more work
  * than another) - msd_attn_decode_split_starts lists them. */
 msd_status_t msd_attn_decode_schedule(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen,
@@ -354,7 +354,7 @@ msd_status_t msd_attn_decode_split_starts(int32_t B, int32_t q_len, int32_t Hq, 
                                           int32_t* starts);
 
 /* The softmax references of the kernel that msd_attn_decode_int8kv (and _spec, _paged) runs for this shape, for a
- * checker that mirrors it (Sec. 4.3; Alg. 3 lines 6-8).  Head groups of up to 16 rows per KV head: *m_margin = 0,
+ * checker that mirrors it (Sec. 4.3; Alg. 3 lines 6-8).  Head groups of up to 8 rows per KV head: *m_margin = 0,
  * *sv_growth = 0 - the running maximum itself and alpha_P = (the tile's largest v_scale) / 127.  Wider groups keep the
  * integer PV sums of consecutive tiles in one accumulator, so their references are held: per context split the
  * reference of a row moves only when a tile's maximum exceeds it, to that maximum + *m_margin (natural-log units), and

@@ -295,7 +295,8 @@ attn_qstack_kernel(const AttnParams p, uint8_t* __restrict__ q_img, float* __res
   for (int h = warp; h < nh; h += static_cast<int>(blockDim.x >> 5)) attn_decompose_q_row(p, b, hk, grp, h, lane, img, sc + h, sc + p.HG + h);
 }
 
-// Head groups of up to 16 query rows per KV head (GQA).  kMaxHG: head slots one softmax thread looks after (8 or 16);
+// Head groups of up to 8 query rows per KV head (GQA).  kMaxHG: head slots one softmax thread looks after (8; the code
+// also compiles for 16, which the planner no longer picks);
 // kNH: heads its code is unrolled for (<= kMaxHG); kMaxDVT: 128-wide tiles of Dv.
 // kPaged: the cache is paged (block table); a template parameter so that the contiguous kernels carry none of it.
 template <int kMaxHG, int kNH, int kMaxDVT, bool kPaged, bool kBalanced>
@@ -1619,7 +1620,9 @@ struct AttnPlan {
 static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, bool v_alias, AttnPlan* pl) {
   if (B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || D < 16 || D % 16 != 0 || Dv < 16 || Dv % 16 != 0) return false;
   const int G = Hq / Hkv;
-  pl->HG = (G <= 8) ? 8 : (G <= 16 ? 16 : 32);
+  // up to 8 rows per KV head: the narrow kernel (three CTAs per SM); more: the wide kernel's 32 head slots (a 16-slot
+  // narrow kernel needs 166 registers, runs one or two CTAs per SM and measured 5-12 % slower than the wide one half full)
+  pl->HG = (G <= 8) ? 8 : 32;
   pl->Rp = 2 * pl->HG;
   pl->groups = (G + pl->HG - 1) / pl->HG;
   pl->DC = (D + kChunk - 1) / kChunk;
@@ -1697,8 +1700,6 @@ static AttnKernel pick_attn_kernel(const AttnPlan& pl, int G, bool paged, int* b
     else kernel = paged ? attn_decode_kernel<8, 8, 1, true, true> : attn_decode_kernel<8, 8, 1, false, true>;
   } else if (pl.HG == 8) {
     if (G <= 4) { MSD_ATTN_PICK(8, 4); } else { MSD_ATTN_PICK(8, 8); }
-  } else if (pl.HG == 16) {
-    MSD_ATTN_PICK(16, 16);
   } else {
     // wide head groups: 32 head slots per CTA, sixteen softmax warps, held references (attn_decode_wide_kernel)
     const bool mla = pl.DC == 5 && pl.DVT == 4 && pl.v_alias && pl.stages == 2;     // a 513..640-byte latent row whose first 512 bytes are V
