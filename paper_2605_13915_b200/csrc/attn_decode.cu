@@ -850,10 +850,10 @@ template <int W> __device__ __forceinline__ void tmem_stw(uint32_t taddr, const 
 // plan) - the MMA thread shares its scheduler with four busy softmax warps, so every instruction it spends per MMA on
 // loop control and address arithmetic delays the tensor pipe; with fixed counts its loops unroll to an add per operand.
 template <int kWideHS, bool kPaged, int kFixDC, int kFixDVT>
-__global__ void __launch_bounds__(64 + 128 * (kWideSlots / kWideHS), 1)
+__global__ void __launch_bounds__(96 + 128 * (kWideSlots / kWideHS), 1)
 attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
   extern __shared__ uint8_t smem_dyn[];
-  __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], v_full[4], v_empty[4], s_full[2], p_full[2], q_ready, o_full, o_last, p_redo;
+  __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], v_full[4], v_empty[4], s_full[2], p_full[2], q_ready, pv_done[2], p_redo;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ int flush_stamp[2];                    // tile number + 1 of the last tile whose references had to move, per P buffer
@@ -918,7 +918,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
     mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1);
     mbar_init(&p_full[0], kNSW); mbar_init(&p_full[1], kNSW);
     mbar_init(&q_ready, 1);
-    mbar_init(&o_full, 1); mbar_init(&o_last, 1); mbar_init(&p_redo, kNSW);
+    mbar_init(&pv_done[0], 1); mbar_init(&pv_done[1], 1); mbar_init(&p_redo, kNSW);
     if constexpr (kChunked)
       for (int s2 = 0; s2 < 2; ++s2)
         for (int c = 0; c < 5; ++c) { mbar_init(&ck_empty[s2][c], 1); mbar_init(&ck_full[s2][c], 1); }
@@ -1042,8 +1042,8 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       // groups of 8 tokens are 512 bytes apart (a softmax thread then stores its token's codes as whole words)
       const uint64_t p_enc = smem_desc(0, 512, 512, kSwizzle64B) + (smem_u32(sm_p) >> 4);
       const uint32_t smem_enc = smem_u32(smem) >> 4;
-      const uint32_t q_step = static_cast<uint32_t>(p.Rp * kChunk) >> 4, p_step = q_step;
-      const int nDC = kFixDC ? kFixDC : p.DC, nDVT = kFixDVT ? kFixDVT : p.DVT;
+      const uint32_t q_step = static_cast<uint32_t>(p.Rp * kChunk) >> 4;
+      const int nDC = kFixDC ? kFixDC : p.DC;
       // 32-byte K steps of the last chunk of D that hold data (the stacked Q operand is zero past D)
       const int last_steps = (p.D - (nDC - 1) * kChunk + 31) >> 5;
       auto issue_qk = [&](int t) {
@@ -1079,50 +1079,8 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
         if constexpr (kChunked) { /* the producer takes s_full as "the rotary chunk has been read" */ }
         else if (!p.v_alias) tc_commit(&kv_empty[st]);       // separate V: the K buffer is free once QK^T has read it
       };
-      // PV of tile t, added to what the accumulators hold unless `fresh`
-      auto issue_pv = [&](int t, bool fresh) {
-        tc_fence_after();
-        const int st = t % p.stages;
-        const uint64_t va = dvt + smem_enc + static_cast<uint32_t>(st * (kv_stage_bytes >> 4)) +
-                            (p.v_alias ? 0u : static_cast<uint32_t>(p.DC * (kChunkBytes >> 4)));
-        const uint64_t pa = p_enc + (t & 1) * p_step;
-        const uint32_t acc0 = fresh ? 0u : 1u;
-        if constexpr (kFixDVT > 0) {
-          const uint32_t va_lo = static_cast<uint32_t>(va), v_hi = static_cast<uint32_t>(va >> 32);
-          const uint32_t pa_lo = static_cast<uint32_t>(pa), p_hi = static_cast<uint32_t>(pa >> 32);
-#pragma unroll
-          for (int j = 0; j < kFixDVT; ++j) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {    // 32 tokens per MMA: four 8-token groups of 1024 bytes
-              if (k > 0)
-                mma_i8_lohi<true>(tmem_o + j * (2 * kWideSlots), va_lo + (j * (kChunkBytes >> 4) + k * (4096 >> 4)), v_hi, pa_lo + k * (2048 >> 4), p_hi, idesc_pv);
-              else
-                mma_i8(tmem_o + j * (2 * kWideSlots), va + (j * (kChunkBytes >> 4)), pa, idesc_pv, acc0);
-            }
-          }
-        } else {
-          uint64_t vc = va;
-          uint32_t d = tmem_o;
-          for (int j = 0; j < nDVT; ++j) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) mma_i8(d, vc + k * (4096 >> 4), pa + k * (2048 >> 4), idesc_pv, k > 0 ? 1u : acc0);
-            vc += kChunkBytes >> 4;
-            d += p.Rp;
-          }
-        }
-        // o_full counts every PV product (a drain in mid-split waits for the one before its tile: at that point the
-        // barrier is at most one phase behind, so a parity test is unambiguous); the last one has a barrier of its own
-        // (chunked stages: the commit after the last dv tile, ck_empty[st][3], says the same)
-        if constexpr (!kChunked) {
-          tc_commit(t == ntiles - 1 ? &o_last : &o_full);
-          tc_commit(p.v_alias ? &kv_empty[st] : &v_empty[st]);
-        }
-      };
-      // QK^T(q) needs KV tile q in shared memory and the score buffer q&1 read (P of tile q-2 final);
-      // PV(v) needs P of tile v final (written, and rewritten when the references had to move) and QK^T(v) issued.
-      // One thread issues both, so everything it has issued completes in order: when the scores of tile t are
-      // there, PV of tile t-2 is complete (the P buffer and the o_full phase the softmax warps rely on).
-      int q = 0, v = 0, n_slow = 0;
+      // PV is issued by softmax threads (below), one dv tile each; this thread issues QK^T only.
+      int q = 0;
       if constexpr (kChunked) {
         // PV is issued by four softmax threads (below); this thread issues QK^T only.  QK^T(q) needs KV tile q in shared
         // memory and the score buffer q&1 read, i.e. P of tile q-2 written by every softmax warp (the slow path works
@@ -1159,44 +1117,63 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
           tc_commit(&s_full[q & 1]);
           if (q >= 2 && q < 5) attn_mark(p, q == 4 ? 30 : 23 + q);
         }
-        v = ntiles;
-      }
-      long long t_idle = clock64();
-      while (ok && v < ntiles) {
-        bool progressed = false;
-        if (v < q && mbar_test_wait(&p_full[v & 1], (v >> 1) & 1) &&
-            (p.v_alias || mbar_test_wait(&v_full[v % p.stages], (v / p.stages) & 1))) {
-          // PV first when both are ready: its completion frees the KV stage the next load is waiting for
-          bool fresh = false;
-          if (stamp[v & 1] == v + 1) {
-            // the softmax warps drain the accumulators and write P of this tile again
-            ok = wait_bounded(&p_redo, n_slow & 1, abort, p.status);
-            if (!ok) break;
-            ++n_slow;
-            fresh = true;
-          }
-          if (v >= 2 && v < 5) attn_mark(p, 8 + 6 * (v - 2));
-          issue_pv(v, fresh);
-          if (v >= 2 && v < 5) attn_mark(p, 20 + v);
-          ++v;
-          progressed = true;
-        }
-        if (q < ntiles && q < v + 2 && mbar_test_wait(&kv_full[q % p.stages], (q / p.stages) & 1)) {
+      } else {
+        // QK^T(q) needs KV tile q in shared memory and the score buffer q&1 read (P of tile q-2 written by every softmax
+        // warp; the slow path works from registers).  PV is issued by a warp of its own (below); that PV(q-2) has read
+        // the P buffer before P of tile q is written there is the softmax warps' wait on pv_done.
+        for (; q < ntiles && ok; ++q) {
+          if (q >= 2) ok = wait_bounded(&p_full[q & 1], ((q - 2) >> 1) & 1, abort, p.status);
+          if (ok) ok = wait_bounded(&kv_full[q % p.stages], (q / p.stages) & 1, abort, p.status);
+          if (!ok) break;
           if (q >= 2 && q < 5) attn_mark(p, 7 + 6 * (q - 2));
           issue_qk(q);
           if (q >= 2 && q < 5) attn_mark(p, q == 4 ? 30 : 23 + q);
-          ++q;
-          progressed = true;
         }
-        if (progressed) {
-          t_idle = clock64();
-        } else {
-          if (*abort) { ok = false; break; }
-          if (clock64() - t_idle > kWaitBudgetCycles) {
-            *abort = 1;
-            atomicMax(p.status, kStatusTimeout);
-            ok = false;
+      }
+    }
+  } else if (warp == 2 + kNSW) {
+    // ------------------------------ PV issuer (rows whose tiles are not handled chunk by chunk) ------------------------------
+    // A warp of its own: one thread issuing QK^T and PV alike was never idle (1.7 us per tile at D = Dv = 128 for 8 MMAs,
+    // 4 commits and its polling, everything else waiting for it), and a softmax thread issuing PV puts it on the
+    // softmax warps' critical path.
+    if constexpr (!kChunked) {
+      if (lane == 0) {
+        const uint64_t vdesc = smem_desc(0, 16384, 1024, kSwizzle128B) + (smem_u32(smem) >> 4);       // V^T, MN-major from the token-major tile
+        const uint64_t pdesc = smem_desc(0, 512, 512, kSwizzle64B) + (smem_u32(sm_p) >> 4);           // P, token-major
+        const uint32_t va0 = static_cast<uint32_t>(vdesc), v_hi = static_cast<uint32_t>(vdesc >> 32);
+        const uint32_t pa0 = static_cast<uint32_t>(pdesc), p_hi = static_cast<uint32_t>(pdesc >> 32);
+        const uint32_t p_step = static_cast<uint32_t>(p.Rp * kChunk) >> 4;
+        const uint32_t idesc = idesc_dense(2, 1, 1, 1, 1, kTok, p.Rp);     // S8 x S8 -> S32, A (V^T) and B (P) MN-major
+        const int n_dvt = kFixDVT ? kFixDVT : p.DVT;
+        bool ok = true;
+        int n_slow = 0;
+        for (int t = 0; t < ntiles && ok; ++t) {
+          const int st = t % p.stages;
+          // P of tile t final: written by every softmax warp and, when the references had to move, written again
+          ok = wait_bounded(&p_full[t & 1], (t >> 1) & 1, abort, p.status);
+          bool fresh = false;
+          if (ok && stamp[t & 1] == t + 1) {
+            ok = wait_bounded(&p_redo, n_slow & 1, abort, p.status);
+            ++n_slow;
+            fresh = true;                          // the accumulators were drained: start them again
           }
+          if (ok) ok = wait_bounded(p.v_alias ? &kv_full[st] : &v_full[st], (t / p.stages) & 1, abort, p.status);     // the value tile
+          if (!ok) break;
+          tc_fence_after();
+          if (t >= 2 && t < 5) attn_mark(p, 8 + 6 * (t - 2));
+          const uint32_t va = va0 + static_cast<uint32_t>(st * (kv_stage_bytes >> 4)) + (p.v_alias ? 0u : static_cast<uint32_t>(p.DC * (kChunkBytes >> 4)));
+          const uint32_t pa = pa0 + (t & 1) * p_step;
+          for (int j = 0; j < n_dvt; ++j) {
+            const uint32_t acc = tmem_o + j * (2 * kWideSlots);
+            if (fresh) mma_i8_lohi<false>(acc, va + j * (kChunkBytes >> 4), v_hi, pa, p_hi, idesc);
+            else mma_i8_lohi<true>(acc, va + j * (kChunkBytes >> 4), v_hi, pa, p_hi, idesc);
+#pragma unroll
+            for (int k = 1; k < 4; ++k)      // 32 tokens per MMA: four 8-token groups of 1024 bytes
+              mma_i8_lohi<true>(acc, va + j * (kChunkBytes >> 4) + k * (4096 >> 4), v_hi, pa + k * (2048 >> 4), p_hi, idesc);
+          }
+          tc_commit(&pv_done[t & 1]);
+          tc_commit(p.v_alias ? &kv_empty[st] : &v_empty[st]);
+          if (t >= 2 && t < 5) attn_mark(p, 20 + t);
         }
       }
     }
@@ -1358,6 +1335,9 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
 
     bool ok = true;
     int n_slow = 0;
+    // this warp's group of head slots holds at least one head (the kernel for 576-byte rows, where every instruction
+    // in the tile loop counts and all 32 slots are normally in use, is compiled without the distinction)
+    const bool active = kChunked ? true : hs0 < nh;
     float ks_pre, vs_pre;
     load_scales(0, ks_pre, vs_pre);
     for (int t = 0; t < ntiles && ok; ++t) {
@@ -1368,10 +1348,22 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       if (threadIdx.x == 64 && t >= 2 && t < 5) attn_mark(p, 4 + 6 * (t - 2));
       tc_fence_after();
       float s[kWideHS], pl[kWideHS];
-      load_scores(t, ks, s);
-      const float xm = write_p(t, s, vs, pl);
-      const bool exceeded = __any_sync(0xffffffffu, xm > 0.0f || vs > a_ref);
-      if (exceeded && lane == 0) stamp[t & 1] = t + 1;
+      if (active) {
+        load_scores(t, ks, s);
+        if constexpr (!kChunked) {
+          // the P buffer t&1 was the operand of PV(t-2), issued by another thread than QK^T(t): its completion is not implied
+          if (t >= 2) ok = wait_bounded(&pv_done[t & 1], ((t - 2) >> 1) & 1, abort, p.status);
+          if (!ok) break;
+        }
+        const float xm = write_p(t, s, vs, pl);
+        const bool exceeded = __any_sync(0xffffffffu, xm > 0.0f || vs > a_ref);
+        if (exceeded && lane == 0) stamp[t & 1] = t + 1;
+      } else {
+        // a group of head slots without a head (9 to 24 rows per KV head): nothing to compute, but the barriers count
+        // every softmax warp; its P columns keep whatever codes they hold and its accumulator columns are never read
+#pragma unroll
+        for (int h = 0; h < kWideHS; ++h) pl[h] = 0.0f;
+      }
       fence_proxy_async_smem();
       tc_fence_before();
       __syncwarp();
@@ -1382,7 +1374,14 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
       if (!ok) break;
       if (threadIdx.x == 64 && t >= 2 && t < 5) attn_mark(p, 6 + 6 * (t - 2));
       bool slow = false;
-      if (stamp[t & 1] == t + 1) {
+      if (!active) {
+        if (stamp[t & 1] == t + 1) {      // the other groups drain and write P again: be counted among the warps that are done
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&p_redo);
+          ++n_slow;
+          slow = true;
+        }
+      } else if (stamp[t & 1] == t + 1) {
         // ---- the references move: tile maxima per head over the group's 128 tokens, largest value scale ----
 #pragma unroll
         for (int h = 0; h < kWideHS; ++h) {
@@ -1419,7 +1418,7 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
 #pragma unroll
             for (int j = 0; j < 4; ++j) ok = ok && wait_bounded(&ck_empty[(t - 1) & 1][j], ((t - 1) >> 1) & 1, abort, p.status);
           } else {
-            ok = wait_bounded(&o_full, (t - 1) & 1, abort, p.status);
+            ok = wait_bounded(&pv_done[(t - 1) & 1], ((t - 1) >> 1) & 1, abort, p.status);
           }
           if (!ok) break;
           tc_fence_after();
@@ -1471,9 +1470,9 @@ attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid
 #pragma unroll
         for (int j = 0; j < 4; ++j) ok = ok && wait_bounded(&ck_empty[(ntiles - 1) & 1][j], ((ntiles - 1) >> 1) & 1, abort, p.status);
       } else {
-        ok = wait_bounded(&o_last, 0, abort, p.status);
+        ok = wait_bounded(&pv_done[(ntiles - 1) & 1], ((ntiles - 1) >> 1) & 1, abort, p.status);
       }
-      if (ok) {
+      if (ok && active) {
         tc_fence_after();
         float one[kWideHS];
 #pragma unroll
@@ -1705,7 +1704,7 @@ static AttnKernel pick_attn_kernel(const AttnPlan& pl, int G, bool paged, int* b
     const bool mla = pl.DC == 5 && pl.DVT == 4 && pl.v_alias && pl.stages == 2;     // a 513..640-byte latent row whose first 512 bytes are V
     if (paged) kernel = mla ? attn_decode_wide_kernel<8, true, 5, 4> : attn_decode_wide_kernel<8, true, 0, 0>;
     else kernel = mla ? attn_decode_wide_kernel<8, false, 5, 4> : attn_decode_wide_kernel<8, false, 0, 0>;
-    *block_threads = 64 + 128 * 4;
+    *block_threads = 96 + 128 * 4;
   }
 #undef MSD_ATTN_PICK
 #undef MSD_ATTN_PICK_B
