@@ -850,7 +850,7 @@ template <int W> __device__ __forceinline__ void tmem_stw(uint32_t taddr, const 
 // plan) - the MMA thread shares its scheduler with four busy softmax warps, so every instruction it spends per MMA on
 // loop control and address arithmetic delays the tensor pipe; with fixed counts its loops unroll to an add per operand.
 template <int kWideHS, bool kPaged, int kFixDC, int kFixDVT>
-__global__ void __launch_bounds__(96 + 128 * (kWideSlots / kWideHS), 1)
+__global__ void __launch_bounds__(((kFixDC == 5 && kFixDVT == 4 && !kPaged) ? 64 : 96) + 128 * (kWideSlots / kWideHS), 1)
 attn_decode_wide_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ __align__(8) uint64_t kv_full[4], kv_empty[4], v_full[4], v_empty[4], s_full[2], p_full[2], q_ready, pv_done[2], p_redo;
@@ -1704,7 +1704,7 @@ static AttnKernel pick_attn_kernel(const AttnPlan& pl, int G, bool paged, int* b
     const bool mla = pl.DC == 5 && pl.DVT == 4 && pl.v_alias && pl.stages == 2;     // a 513..640-byte latent row whose first 512 bytes are V
     if (paged) kernel = mla ? attn_decode_wide_kernel<8, true, 5, 4> : attn_decode_wide_kernel<8, true, 0, 0>;
     else kernel = mla ? attn_decode_wide_kernel<8, false, 5, 4> : attn_decode_wide_kernel<8, false, 0, 0>;
-    *block_threads = 96 + 128 * 4;
+    *block_threads = ((mla && !paged) ? 64 : 96) + 128 * 4;      // producer, QK^T issuer, 16 softmax warps and, except for the chunk-wise kernel, a PV issuer
   }
 #undef MSD_ATTN_PICK
 #undef MSD_ATTN_PICK_B
