@@ -376,6 +376,21 @@ void msd_debug_set_attn_dump(int8_t* q_dbg, float* q_scale_dbg, int32_t* s_dbg);
 msd_status_t msd_kv_dequant_bf16(const int8_t* cache, const float* scale, int64_t T, int32_t H, int32_t D,
                                  void* out_bf16, void* stream);
 
+/* Comparison kernel, not part of the MSD path: decode attention over a BF16 KV cache, the second half of the "Dequant"
+ * arm of Sec. 6.4 (msd_kv_dequant_bf16 is the first).  out = softmax(softmax_scale * Q K^T) V per sequence and head
+ * with Q, K, V and the probabilities as BF16 tensor-core operands and FP32 accumulation, split over the context and
+ * merged like msd_attn_decode_int8kv; no decomposition anywhere.
+ *   q_bf16 [B,Hq,D], k_bf16 [T,Hkv,D], v_bf16 [T,Hkv,Dv] BF16, 16-byte aligned; cu_seqlens [B+1] INT32 token offsets
+ *   (device); total_tokens = T; max_seqlen >= every length; out_bf16 [B,Hq,Dv]; lse nullable [B,Hq] FP32.
+ * Shapes: D = 64 or 128, Dv = 128, Hq % Hkv == 0, Hq / Hkv <= 16; anything else: MSD_ERR_UNSUPPORTED.  Workspace:
+ * msd_attn_decode_bf16kv_workspace_bytes (0 for a shape it does not take), 1024-byte aligned, no initialisation.
+ * Errors as msd_attn_decode_int8kv; empty sequences give zeros and lse = -inf. */
+size_t msd_attn_decode_bf16kv_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen);
+msd_status_t msd_attn_decode_bf16kv(const void* q_bf16, const void* k_bf16, const void* v_bf16, const int32_t* cu_seqlens,
+                                    int64_t total_tokens, int32_t max_seqlen, int32_t B, int32_t Hq, int32_t Hkv, int32_t D,
+                                    int32_t Dv, float softmax_scale, void* out_bf16, float* lse, void* workspace,
+                                    size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

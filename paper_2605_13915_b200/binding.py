@@ -73,6 +73,8 @@ _SIGS = {
                                                 _sz, _vp]),
     "msd_debug_timeout_selftest": (C.c_int, [_i64, _vp]),
     "msd_kv_dequant_bf16": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, _i32, _i32, C.c_void_p, C.c_void_p]),
+    "msd_attn_decode_bf16kv_workspace_bytes": (_sz, [_i32] * 6),
+    "msd_attn_decode_bf16kv": (C.c_int, [_vp, _vp, _vp, _vp, _i64] + [_i32] * 6 + [_f32, _vp, _vp, _vp, _sz, _vp]),
 }
 
 
@@ -457,6 +459,23 @@ def kv_dequant_bf16(cache, scale, out=None):
     _check(lib().msd_kv_dequant_bf16(cache.data_ptr(), scale.data_ptr(), T, H, D, out.data_ptr(), _stream()),
            "msd_kv_dequant_bf16")
     return out
+
+
+def attn_decode_bf16kv(q, k, v, cu_seqlens, max_seqlen, softmax_scale, ws=None, want_lse=False, out=None):
+    """The comparison arm's attention: q [B,Hq,D], k [T,Hkv,D], v [T,Hkv,Dv] bf16 (e.g. from kv_dequant_bf16)."""
+    _need_cuda(q, k, v, cu_seqlens)
+    B, Hq, D = q.shape
+    T, Hkv, Dv = v.shape
+    if ws is None:
+        ws = workspace(int(lib().msd_attn_decode_bf16kv_workspace_bytes(B, Hq, Hkv, D, Dv, max_seqlen)))
+    if out is None:
+        out = _empty((B, Hq, Dv), torch.bfloat16, q.device)
+    lse = _empty((B, Hq), torch.float32, q.device) if want_lse else None
+    wp, wb = _ws_ptr(ws)
+    _check(lib().msd_attn_decode_bf16kv(_ptr(q), _ptr(k), _ptr(v), _ptr(cu_seqlens), T, max_seqlen, B, Hq, Hkv, D, Dv,
+                                        float(softmax_scale), _ptr(out), None if lse is None else _ptr(lse), wp, wb, _stream()),
+           "msd_attn_decode_bf16kv")
+    return (out, lse) if want_lse else out
 
 
 def attn_decode_int8kv_workspace_bytes(B, Hq, Hkv, D, Dv, max_seqlen):

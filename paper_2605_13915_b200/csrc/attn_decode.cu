@@ -1683,6 +1683,14 @@ static bool plan_attn(int B, int Hq, int Hkv, int D, int Dv, int max_seqlen, boo
   return pl->smem_bytes <= 227 * 1024 - 2048;
 }
 
+// The split merge for another attention kernel of this library (rows in output order, every row n_splits partial results).
+msd_status_t launch_attn_combine(const float* partial, int n_splits, int Dv, void* out_bf16, float* lse, int rows, cudaStream_t s) {
+  if (launch_pdl(attn_combine_kernel, dim3(rows), dim3(128), 0, s, option(OPT_NO_PDL) <= 0, partial, n_splits,
+                 static_cast<const int32_t*>(nullptr), 1, 1, 1, Dv, static_cast<__nv_bfloat16*>(out_bf16), lse, 1, 1, 1) != cudaSuccess)
+    return MSD_ERR_CUDA;
+  return launch_status();
+}
+
 using AttnKernel = void (*)(CUtensorMap, CUtensorMap, AttnParams);
 
 // The kernel instantiation for a plan (G: query rows per KV head) and its block size.

@@ -43,6 +43,9 @@ bool encode_tmap_3d(CUtensorMap* out, CUtensorMapDataType dtype, const void* bas
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// attn_decode.cu: merges the context splits' partial results [rows][n_splits][4 + Dv] into out_bf16 [rows][Dv] (and lse)
+msd_status_t launch_attn_combine(const float* partial, int n_splits, int Dv, void* out_bf16, float* lse, int rows, cudaStream_t s);
+
 inline msd_status_t launch_status() { return cudaGetLastError() == cudaSuccess ? MSD_OK : MSD_ERR_CUDA; }
 
 // Kernel launch with the programmatic-dependent-launch attribute (the kernel may start while its predecessor in

@@ -243,6 +243,40 @@ def test_dequant_bf16_comparison_arm_is_less_accurate():
     assert np.linalg.norm(msd - ref) <= np.linalg.norm(got - ref) * 1.05
 
 
+@pytest.mark.parametrize("B,Hq,Hkv,D,seqlens", [
+    (2, 8, 2, 128, [700, 333]), (3, 32, 8, 128, [129, 0, 4000]), (1, 16, 1, 128, [1]), (2, 12, 4, 64, [2049, 128]),
+])
+def test_bf16_kv_comparison_kernel(B, Hq, Hkv, D, seqlens):
+    """The whole comparison arm in our own kernels (Sec. 6.4 "Dequant"): cache expansion to BF16, then BF16 decode
+    attention with FP32 accumulation.  It follows the oracle's dequantize-to-BF16 mode (same tolerance as the library
+    attention above: summation order and the tile-wise running maximum differ from the oracle's single pass), and
+    against the FP64 reference on the dequantized cache it is no better than the MSD kernel."""
+    c = inputs.gqa_case(B=B, Hq=Hq, Hkv=Hkv, D=D, seqlens=seqlens, seed=40 + Hq)
+    if c.dv != 128:                                    # values of width 128 whatever the key width
+        rng = np.random.default_rng(3)
+        T = c.k.shape[0]
+        c = inputs.AttnCase(c.q, c.k, rng.integers(-127, 128, (T, Hkv, 128), dtype=np.int8), c.k_scale,
+                            (rng.random((T, Hkv), dtype=np.float32) * 0.02 + 0.01), c.cu_seqlens, 128, c.softmax_scale)
+    kb = binding.kv_dequant_bf16(dev(c.k), dev(c.k_scale))
+    vb = binding.kv_dequant_bf16(dev(c.v), dev(c.v_scale))
+    o, lse = binding.attn_decode_bf16kv(bf16_dev(c.q), kb, vb, dev(c.cu_seqlens), max(c.max_seqlen, 1), c.softmax_scale, want_lse=True)
+    torch.cuda.synchronize()
+    binding.last_device_status()
+    got = oracle.bf16_bits_to_f64(bf16_bits(o))
+    args = (c.q, c.k, c.v, c.k_scale, c.v_scale, c.cu_seqlens, c.softmax_scale)
+    deq, lse_ref = oracle.attn_decode_int8kv(*args, dv=c.dv, mode="dequant", want_lse=True)
+    ref = oracle.attn_decode_int8kv(*args, dv=c.dv, mode="ref")
+    n = np.linalg.norm(ref, axis=-1, keepdims=True)
+    assert np.all(np.abs(got - deq) <= 1e-2 * n + 1e-30)
+    live = np.isfinite(lse_ref)
+    assert np.allclose(lse.cpu().numpy()[live], lse_ref[live], rtol=0, atol=2e-3)
+    assert np.all(np.isneginf(lse.cpu().numpy()[~live])) and np.all(got[~live] == 0)
+    msd = oracle.bf16_bits_to_f64(bf16_bits(_run_gpu(c)[0]))
+    assert np.linalg.norm(msd - ref) <= np.linalg.norm(got - ref) * 1.05
+    with pytest.raises(binding.MsdError):             # shapes the comparison kernel does not take
+        binding.attn_decode_bf16kv(bf16_dev(c.q), kb, vb[:, :, :64].contiguous(), dev(c.cu_seqlens), max(c.max_seqlen, 1), c.softmax_scale)
+
+
 @pytest.mark.parametrize("page", [16, 64, 128, -64])
 def test_paged_cache_gqa(page):
     """The same sequences scattered over a paged cache (random block order, noise in the unused blocks and in the tails
