@@ -541,7 +541,6 @@ gemm_w4a16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid
     // Epilogue as in the single-CTA kernel: TMEM -> registers -> (BF16) -> swizzled staging buffer -> TMA store.
     const int quad = warp & 3;
     uint8_t* stage_buf = smem + kW4PairStages * kStageBytes + quad * (2 * kW4StoreBytes);
-    const int ccols = (p.ytype == MSD_OUT_BF16) ? 32 : 16;
     const uint32_t swz = static_cast<uint32_t>((lane >> 1) & 3);
     int it = 0, buf = 0;
     bool ok = true;
