@@ -167,6 +167,58 @@ __device__ __forceinline__ void attn_decompose_q_row(const AttnParams& p, int b,
   }
 }
 
+// Two rows of at most 128 values at once: lanes 0-15 take head slot h_a, lanes 16-31 head slot h_b (h_b < 0: none), 8
+// values per lane; the same arithmetic per element as attn_decompose_q_row, the row maximum reduced over 16 lanes.
+__device__ __forceinline__ void attn_decompose_q_pair(const AttnParams& p, int b, int hk, int grp, int h_a, int h_b, int lane, uint8_t* img,
+                                                      float* alpha_out, float* beta_out) {
+  const int h = (lane < 16) ? h_a : h_b;
+  const int i = lane & 15;
+  const int nvec = p.D >> 3;                    // <= 16
+  const bool row = h >= 0, live = row && i < nvec;
+  const long long q_row = row ? attn_q_row_index(p, b, hk, grp, h) : 0;
+  uint4 qv = make_uint4(0, 0, 0, 0);
+  if (live) qv = __ldg(reinterpret_cast<const uint4*>(p.q + q_row * p.D) + i);
+  const uint32_t w[4] = {qv.x, qv.y, qv.z, qv.w};
+  float m = 0.0f;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    m = fmaxf(m, fabsf(__uint_as_float(w[k] << 16)));
+    m = fmaxf(m, fabsf(__uint_as_float(w[k] & 0xFFFF0000u)));
+  }
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));      // stays inside the 16 lanes
+  const float alpha = __fdiv_rn(m, 127.0f), beta = __fdiv_rn(alpha, 254.0f);
+  const float inv_alpha = alpha > 0.0f ? __frcp_rn(alpha) : 0.0f, inv_beta = beta > 0.0f ? __frcp_rn(beta) : 0.0f;
+  if (row && i == 0) {
+    alpha_out[h] = alpha; beta_out[h] = beta;
+    if (p.qs_dbg) {
+      p.qs_dbg[q_row] = alpha;
+      p.qs_dbg[static_cast<long long>(p.B) * p.Hq + q_row] = beta;
+    }
+  }
+  if (!live) return;
+  uint32_t o1[2] = {0, 0}, o2[2] = {0, 0};
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const float x = (e & 1) ? __uint_as_float(w[e >> 1] & 0xFFFF0000u) : __uint_as_float(w[e >> 1] << 16);
+    int c1 = 0, c2 = 0;
+    if (alpha > 0.0f) {
+      c1 = quant_i8(x, alpha, inv_alpha);
+      const float r = __fmaf_rn(-alpha, static_cast<float>(c1), x);
+      if (beta > 0.0f) c2 = quant_i8(r, beta, inv_beta);
+    }
+    o1[e >> 2] |= static_cast<uint32_t>(c1 & 0xFF) << (8 * (e & 3));
+    o2[e >> 2] |= static_cast<uint32_t>(c2 & 0xFF) << (8 * (e & 3));
+  }
+  const int d = i << 3;                         // < 128: the row's single chunk
+  *reinterpret_cast<uint2*>(img + swz_off(h, d)) = make_uint2(o1[0], o1[1]);
+  *reinterpret_cast<uint2*>(img + swz_off(p.HG + h, d)) = make_uint2(o2[0], o2[1]);
+  if (p.q_dbg) {
+    *reinterpret_cast<uint2*>(p.q_dbg + q_row * p.D + d) = make_uint2(o1[0], o1[1]);
+    *reinterpret_cast<uint2*>(p.q_dbg + (static_cast<long long>(p.B) * p.Hq + q_row) * p.D + d) = make_uint2(o2[0], o2[1]);
+  }
+}
+
 // Debug dump of one thread's raw QK^T sums (Alg. 3 lines 3-4): token `tok_row` (row of the cache), head slots
 // [hs, hs + n) of head group `grp` of KV head `hk`; c1 / c2 are the two components' accumulators.
 template <int N>
@@ -582,10 +634,12 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       const int t_end = min(L, t_begin + ntiles * kTok);
       // c1: decompose the query rows of this segment's heads (one warp per head, round robin) into the stacked operand
       // (the head slots and padding columns that were zeroed at the start are never written)
-      for (int h = wi; h < nh; h += kNSW) {
-        // a warp with a second row asks for it now: two cold reads one after the other cost microseconds
-        if (h + kNSW < nh && lane * 64 < p.D) prefetch_l2(p.q + attn_q_row_index(p, b, hk, grp, h + kNSW) * p.D + lane * 64);
-        attn_decompose_q_row(p, b, hk, grp, h, lane, sm_q, &s_aq[h], &s_bq[h]);
+      if (kNH > 4 && kMaxHG == 8 && p.D <= 128) {
+        // more than four rows of at most 128 values: a warp takes its two rows side by side, 16 lanes each (one after
+        // the other the stacked operand was ready 5.4 us after the CTA's start instead of 3.0 us with one row per warp)
+        if (wi < nh) attn_decompose_q_pair(p, b, hk, grp, wi, wi + kNSW < nh ? wi + kNSW : -1, lane, sm_q, s_aq, s_bq);
+      } else {
+        for (int h = wi; h < nh; h += kNSW) attn_decompose_q_row(p, b, hk, grp, h, lane, sm_q, &s_aq[h], &s_bq[h]);
       }
       fence_proxy_async_smem();
       __syncwarp();

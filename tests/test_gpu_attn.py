@@ -383,12 +383,19 @@ def _run_with_dump(fn, rows, rows_per_seq, D, T):
     return q_dbg, qs_dbg, s_dbg.cpu().numpy()
 
 
-@pytest.mark.parametrize("kind", ["gqa_narrow", "gqa_16", "mla"])
+@pytest.mark.parametrize("kind", ["gqa_narrow", "gqa_8", "gqa_7_d64", "gqa_8_balanced", "gqa_16", "mla"])
 def test_query_components_and_scores_bit_exact(kind):
     """North-star requirement: decomposed components, scales and INT32 accumulators bit-exact.  The kernels dump what
     they computed (msd_debug_set_attn_dump); the oracle returns the same planes (Alg. 3 lines 1-4)."""
     if kind == "gqa_narrow":
         c = inputs.gqa_case(3, 8, 2, 128, [700, 64, 1500], seed=41)          # rows decomposed inside the attention CTAs
+    elif kind == "gqa_8":
+        c = inputs.gqa_case(3, 16, 2, 128, [700, 64, 1500], seed=45)         # 8 rows: a warp decomposes two, 16 lanes each
+    elif kind == "gqa_7_d64":
+        c = inputs.gqa_case(2, 14, 2, 64, [300, 129], seed=46)               # an odd row count, half a chunk of d
+    elif kind == "gqa_8_balanced":
+        binding.debug_set_option("MSD_ATTN_BALANCED", 1)                     # rows decomposed again in every segment
+        c = inputs.gqa_case(5, 16, 2, 128, [200, 0, 1100, 64, 900], seed=47)
     elif kind == "gqa_16":
         c = inputs.gqa_case(2, 32, 2, 128, [513, 2222], seed=42)            # 16 rows per KV head
     else:
@@ -396,7 +403,7 @@ def test_query_components_and_scores_bit_exact(kind):
     B, Hq, D = c.q.shape
     T = c.k.shape[0]
     q_dbg, qs_dbg, s_dbg = _run_with_dump(lambda: _run_gpu(c, want_lse=False), B * Hq, Hq, D, T)
-    _check_q_dump(c.q.reshape(B * Hq, D), q_dbg, qs_dbg)
+    _check_q_dump(c.q.reshape(B * Hq, D), q_dbg, qs_dbg, live=np.repeat(np.diff(c.cu_seqlens) > 0, Hq))
     _, s_ref = oracle.attn_decode_int8kv(c.q, c.k, c.v, c.k_scale, c.v_scale, c.cu_seqlens, c.softmax_scale, dv=c.dv, want_s=True)
     # token t belongs to exactly one sequence, so the plane [row of that sequence, t] is defined for every t
     assert np.array_equal(s_dbg, s_ref)
