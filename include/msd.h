@@ -353,6 +353,12 @@ msd_status_t msd_attn_decode_split_starts(int32_t B, int32_t q_len, int32_t Hq, 
                                           int32_t max_seqlen, int32_t paged, int32_t v_aliased, const int32_t* seqlens,
                                           int32_t* starts);
 
+/* The same arithmetic with the number of resident CTAs given instead of asked of the device (no CUDA call at all: for
+ * tests of the schedule on a host without a GPU).  resident_ctas >= 1, otherwise MSD_ERR_BAD_SHAPE. */
+msd_status_t msd_debug_attn_split_starts(int32_t B, int32_t q_len, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
+                                         int32_t max_seqlen, int32_t v_aliased, int32_t resident_ctas, const int32_t* seqlens,
+                                         int32_t* starts);
+
 /* The softmax references of the kernel that msd_attn_decode_int8kv (and _spec, _paged) runs for this shape, for a
  * checker that mirrors it (Sec. 4.3; Alg. 3 lines 6-8).  Head groups of up to 8 rows per KV head: *m_margin = 0,
  * *sv_growth = 0 - the running maximum itself and alpha_P = (the tile's largest v_scale) / 127.  Wider groups keep the

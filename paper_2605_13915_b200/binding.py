@@ -61,6 +61,7 @@ _SIGS = {
                                          _vp, _sz, _vp]),
     "msd_attn_decode_schedule": (C.c_int, [_i32] * 6 + [C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
     "msd_attn_decode_split_starts": (C.c_int, [_i32] * 9 + [C.c_void_p, C.c_void_p]),
+    "msd_debug_attn_split_starts": (C.c_int, [_i32] * 9 + [C.c_void_p, C.c_void_p]),
     "msd_attn_decode_softmax_rule": (C.c_int, [_i32] * 6 + [C.POINTER(_f32), C.POINTER(_f32)]),
     "msd_debug_set_attn_dump": (None, [_vp, _vp, _vp]),
     "msd_debug_set_option": (C.c_int, [C.c_char_p, _i32]),
@@ -347,16 +348,21 @@ def attn_decode_schedule(B, Hq, Hkv, D, Dv, max_seqlen):
     return tile.value, ns.value, st.value
 
 
-def attn_decode_split_starts(seqlens, Hq, Hkv, D, Dv, max_seqlen, q_len=1, paged=False, v_aliased=False):
+def attn_decode_split_starts(seqlens, Hq, Hkv, D, Dv, max_seqlen, q_len=1, paged=False, v_aliased=False, resident_ctas=None):
     """Context splits of a call with these sequence lengths: int32 array [B, Hkv, q_len * Hq // Hkv, n_splits + 1] of
-    token offsets (see msd_attn_decode_split_starts), plus the tile size."""
+    token offsets (see msd_attn_decode_split_starts), plus the tile size.  resident_ctas: take that many CTAs for the
+    balanced schedule's grid instead of asking the device (host arithmetic only)."""
     import numpy as np
     L = np.ascontiguousarray(seqlens, dtype=np.int32)
     B = int(L.shape[0])
     tile, ns, _ = attn_decode_schedule(B, Hq * q_len, Hkv, D, Dv, max(int(max_seqlen), 1))
     starts = np.zeros((B, Hkv, q_len * Hq // Hkv, ns + 1), dtype=np.int32)
-    _check(lib().msd_attn_decode_split_starts(B, q_len, Hq, Hkv, D, Dv, max(int(max_seqlen), 1), int(paged), int(v_aliased),
-                                              L.ctypes.data, starts.ctypes.data), "msd_attn_decode_split_starts")
+    if resident_ctas is None:
+        _check(lib().msd_attn_decode_split_starts(B, q_len, Hq, Hkv, D, Dv, max(int(max_seqlen), 1), int(paged), int(v_aliased),
+                                                  L.ctypes.data, starts.ctypes.data), "msd_attn_decode_split_starts")
+    else:
+        _check(lib().msd_debug_attn_split_starts(B, q_len, Hq, Hkv, D, Dv, max(int(max_seqlen), 1), int(v_aliased),
+                                                 int(resident_ctas), L.ctypes.data, starts.ctypes.data), "msd_debug_attn_split_starts")
     return starts, tile
 
 

@@ -1858,9 +1858,10 @@ msd_status_t msd_attn_decode_schedule(int32_t B, int32_t Hq, int32_t Hkv, int32_
   return MSD_OK;
 }
 
-msd_status_t msd_attn_decode_split_starts(int32_t B, int32_t q_len, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
-                                          int32_t max_seqlen, int32_t paged, int32_t v_aliased, const int32_t* seqlens,
-                                          int32_t* starts) {
+// resident_ctas > 0: the number of CTAs the balanced schedule's grid would have is given (host arithmetic only, no
+// CUDA call: what the CPU tests use); <= 0: asked of the device as the launch does.
+static msd_status_t attn_split_starts(int32_t B, int32_t q_len, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv, int32_t max_seqlen,
+                                      int32_t paged, int32_t v_aliased, int32_t resident_ctas, const int32_t* seqlens, int32_t* starts) {
   using namespace msd;
   if (!seqlens || !starts) return MSD_ERR_NULL_POINTER;
   if (q_len < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || B < 1) return MSD_ERR_BAD_SHAPE;
@@ -1869,10 +1870,13 @@ msd_status_t msd_attn_decode_split_starts(int32_t B, int32_t q_len, int32_t Hq, 
   const int G = Hq * q_len / Hkv, U = Hkv * pl.groups, ns = pl.n_splits;
   long long R = 0, W = 0;
   if (pl.balanced) {
-    int block_threads = 0;
-    AttnKernel kernel = pick_attn_kernel(pl, G, paged != 0, &block_threads);
-    if (!prepare_attn_kernel(kernel)) return MSD_ERR_CUDA;
-    const int ctas = attn_balanced_ctas(kernel, block_threads, pl.smem_bytes, pl.tmem_cols, U);
+    int ctas = resident_ctas > 0 ? std::max(resident_ctas / U, 1) * U : 0;
+    if (ctas == 0) {
+      int block_threads = 0;
+      AttnKernel kernel = pick_attn_kernel(pl, G, paged != 0, &block_threads);
+      if (!prepare_attn_kernel(kernel)) return MSD_ERR_CUDA;
+      ctas = attn_balanced_ctas(kernel, block_threads, pl.smem_bytes, pl.tmem_cols, U);
+    }
     if (ctas < 1) return MSD_ERR_CUDA;
     for (int b = 0; b < B; ++b) W += seqlens[b] > 0 ? (seqlens[b] + kTok - 1) / kTok : 0;
     R = std::min<long long>(W / pl.q_min, ctas / U);
@@ -1898,6 +1902,19 @@ msd_status_t msd_attn_decode_split_starts(int32_t B, int32_t q_len, int32_t Hq, 
     P += nb;
   }
   return MSD_OK;
+}
+
+msd_status_t msd_attn_decode_split_starts(int32_t B, int32_t q_len, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
+                                          int32_t max_seqlen, int32_t paged, int32_t v_aliased, const int32_t* seqlens,
+                                          int32_t* starts) {
+  return attn_split_starts(B, q_len, Hq, Hkv, D, Dv, max_seqlen, paged, v_aliased, 0, seqlens, starts);
+}
+
+msd_status_t msd_debug_attn_split_starts(int32_t B, int32_t q_len, int32_t Hq, int32_t Hkv, int32_t D, int32_t Dv,
+                                         int32_t max_seqlen, int32_t v_aliased, int32_t resident_ctas, const int32_t* seqlens,
+                                         int32_t* starts) {
+  if (resident_ctas < 1) return MSD_ERR_BAD_SHAPE;
+  return attn_split_starts(B, q_len, Hq, Hkv, D, Dv, max_seqlen, 0, v_aliased, resident_ctas, seqlens, starts);
 }
 
 }  // extern "C"
