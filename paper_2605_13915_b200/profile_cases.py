@@ -4,6 +4,8 @@
     python -m paper_2605_13915_b200.profile_cases gemm_w4a16 M N K [calls]
     python -m paper_2605_13915_b200.profile_cases attn_gqa B L [calls]        (32 query heads, 8 KV heads, d 128)
     python -m paper_2605_13915_b200.profile_cases attn_mla B L [calls]        (64 query heads, latent d 576 / 512)
+    python -m paper_2605_13915_b200.profile_cases attn_gqa16 B L [calls]      (128 query heads, 8 KV heads, d 128)
+    python -m paper_2605_13915_b200.profile_cases attn_bf16 B L [calls]       (the BF16-KV comparison kernel, 32 / 8 heads)
 
 Inputs are random tensors of the right types drawn on the device (KV caches: N(0,1) values quantized per token, as in
 the benchmark); three weight / two cache buffers are rotated.  This is a driver for profilers, not part of the library's
@@ -35,10 +37,21 @@ def main(argv):
             ws = binding.workspace(binding.gemm_w4a16_workspace_bytes(M, N, K))
             for i in range(calls):
                 y = binding.gemm_w4a16(x, w[i % 3], e, ws=ws)
-    elif what in ("attn_gqa", "attn_mla"):
+    elif what == "attn_bf16":
         B, L = int(argv[1]), int(argv[2])
         calls = int(argv[3]) if len(argv) > 3 else 3
-        Hq, Hkv, D, Dv = (32, 8, 128, 128) if what == "attn_gqa" else (64, 1, 576, 512)
+        Hq, Hkv, D = 32, 8, 128
+        T = B * L
+        cu = (torch.arange(B + 1, dtype=torch.int32) * L).cuda()
+        q = torch.randn(B, Hq, D, device="cuda").to(torch.bfloat16)
+        k = [torch.randn(T, Hkv, D, device="cuda").to(torch.bfloat16) for _ in range(2)]
+        v = [torch.randn(T, Hkv, D, device="cuda").to(torch.bfloat16) for _ in range(2)]
+        for i in range(calls):
+            y = binding.attn_decode_bf16kv(q, k[i % 2], v[i % 2], cu, L, D ** -0.5)
+    elif what in ("attn_gqa", "attn_mla", "attn_gqa16"):
+        B, L = int(argv[1]), int(argv[2])
+        calls = int(argv[3]) if len(argv) > 3 else 3
+        Hq, Hkv, D, Dv = {"attn_gqa": (32, 8, 128, 128), "attn_mla": (64, 1, 576, 512), "attn_gqa16": (128, 8, 128, 128)}[what]
         T = B * L
         cu = (torch.arange(B + 1, dtype=torch.int32) * L).cuda()
         q = torch.randn(B, Hq, D, device="cuda").to(torch.bfloat16)
