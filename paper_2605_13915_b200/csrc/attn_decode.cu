@@ -16,6 +16,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <mutex>
 #include <cstdlib>
 
 #include "host_common.h"
@@ -1775,7 +1776,9 @@ static AttnKernel pick_attn_kernel(const AttnPlan& pl, int G, bool paged, int* b
 
 // Raises the dynamic shared-memory limit once per kernel instantiation.
 static bool prepare_attn_kernel(AttnKernel kernel) {
+  static std::mutex mu;
   static void* done[32] = {};
+  std::lock_guard<std::mutex> lock(mu);
   int free_slot = -1;
   for (int i = 0; i < 32; ++i) {
     if (done[i] == reinterpret_cast<void*>(kernel)) return true;
@@ -1791,7 +1794,9 @@ static bool prepare_attn_kernel(AttnKernel kernel) {
 // unit), at least one set (0: the query failed).
 static int attn_balanced_ctas(AttnKernel kernel, int block_threads, size_t smem_bytes, int tmem_cols, int U) {
   struct Entry { void* k; size_t smem; int ctas; };
+  static std::mutex mu;
   static Entry cache[32] = {};
+  std::lock_guard<std::mutex> lock(mu);
   for (const Entry& e : cache)
     if (e.k == reinterpret_cast<void*>(kernel) && e.smem == smem_bytes) return std::max(e.ctas / U, 1) * U;
   // Resident CTAs per SM from the kernel's own resource use (the runtime's occupancy query assumes the default

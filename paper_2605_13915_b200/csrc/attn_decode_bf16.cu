@@ -10,6 +10,7 @@
 #include <cuda_bf16.h>
 
 #include <cmath>
+#include <mutex>
 
 #include "host_common.h"
 #include "sm100.cuh"
@@ -406,13 +407,17 @@ msd_status_t msd_attn_decode_bf16kv(const void* q_bf16, const void* k_bf16, cons
 
   void (*kernel)(CUtensorMap, CUtensorMap, AttnBf16Params) =
       p.G <= 4 ? attn_decode_bf16_kernel<4> : (p.G <= 8 ? attn_decode_bf16_kernel<8> : attn_decode_bf16_kernel<16>);
-  static void* prepared[4] = {};
-  bool seen = false;
-  for (void* k : prepared) seen = seen || k == reinterpret_cast<void*>(kernel);
-  if (!seen) {
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess) return MSD_ERR_CUDA;
-    for (void*& k : prepared)
-      if (!k) { k = reinterpret_cast<void*>(kernel); break; }
+  {
+    static std::mutex mu;
+    static void* prepared[4] = {};
+    std::lock_guard<std::mutex> lock(mu);
+    bool seen = false;
+    for (void* k : prepared) seen = seen || k == reinterpret_cast<void*>(kernel);
+    if (!seen) {
+      if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) != cudaSuccess) return MSD_ERR_CUDA;
+      for (void*& k : prepared)
+        if (!k) { k = reinterpret_cast<void*>(kernel); break; }
+    }
   }
   kernel<<<dim3(B * Hkv, pl.n_splits), kBThreads, pl.smem_bytes, s>>>(tmap_k, tmap_v, p);
   if (cudaGetLastError() != cudaSuccess) return MSD_ERR_CUDA;
